@@ -1,0 +1,476 @@
+"""Pins of the CPU eager oracle against facts it did not produce itself:
+hand-computed values, closed forms, invariants, published known answers and
+independent library routines (numpy / torch CPU in float64)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.eager import EagerOracle, OTensor, lib
+from workloads import configs, rng, traces
+
+F32 = np.float32
+
+
+def f32(*v):
+    return np.array(v, dtype=np.float32)
+
+
+@pytest.fixture()
+def B():
+    return EagerOracle()
+
+
+def leaf(B, a, dtype="f32"):
+    return B.leaf(np.asarray(a), dtype)
+
+
+# ------------------------------------------------------------------ bf16
+
+def test_bf16_rounding_hand_cases():
+    L = lib()
+    cases = {
+        0x3F800000: 0x3F80,  # 1.0 exact
+        0x3F808000: 0x3F80,  # tie -> even (down)
+        0x3F818000: 0x3F82,  # tie -> even (up)
+        0x3F808001: 0x3F81,  # just above tie
+        0x3F807FFF: 0x3F80,  # just below tie
+        0x7F7FFFFF: 0x7F80,  # max finite rounds to +inf
+        0xFF7FFFFF: 0xFF80,  # -max rounds to -inf
+        0x7F800000: 0x7F80,  # inf
+        0x00000001: 0x0000,  # smallest subnormal -> 0
+        0x00008000: 0x0000,  # subnormal tie -> even
+        0x00018000: 0x0002,  # subnormal tie -> even (up)
+        0x80000000: 0x8000,  # -0
+    }
+    for bits, want in cases.items():
+        x = np.array(bits, dtype=np.uint32).view(np.float32)
+        assert L.orc_f32_to_bf16(float(x)) == want, hex(bits)
+    nan = L.orc_f32_to_bf16(float("nan"))
+    assert (nan & 0x7F80) == 0x7F80 and (nan & 0x007F) != 0
+
+
+def test_bf16_matches_torch_cpu(B):
+    g = rng.generator(11)
+    x = np.concatenate([rng.normal_f32(g, (4096,), 3.0),
+                        rng.normal_f32(g, (512,), 1e-39),  # subnormals
+                        f32(0.0, -0.0, np.inf, -np.inf, 3.3895314e38, 1.00390625, 1.01171875)])
+    got = B.op("convert", leaf(B, x), dtype="bf16").array
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(got, want)
+    # the input generator's quantiser agrees as well
+    np.testing.assert_array_equal(rng.to_bf16_bits(x), want)
+    # widening is exact
+    back = B.op("convert", OTensor(want.copy(), "bf16"), dtype="f32").array
+    np.testing.assert_array_equal(back.view(np.uint32), want.astype(np.uint32) << 16)
+
+
+def test_bf16_node_rounds_after_f32_op(B):
+    # 1 + 2^-8 in bf16 arithmetic: exact sum 1.00390625 is a tie -> 1.0
+    a = OTensor(np.array([0x3F80], dtype=np.uint16), "bf16")
+    b = OTensor(np.array([0x3B80], dtype=np.uint16), "bf16")  # 2^-8
+    assert B.op("add", a, b).array[0] == 0x3F80
+    c = OTensor(np.array([0x3C00], dtype=np.uint16), "bf16")  # 2^-7
+    assert B.op("add", a, c).array[0] == 0x3F81
+
+
+# ------------------------------------------------- elementwise arithmetic
+
+def test_chain_hand_computed(B):
+    # relu(a*b + c) * 0.5 - d, all values exact in binary
+    a = f32(0.5, -1.0, 0.25, 2.0)
+    b = f32(4.0, 3.0, -8.0, 0.5)
+    c = f32(1.0, 1.0, 1.0, -1.0)
+    d = f32(0.25, 0.5, -1.0, 0.0)
+    y = traces.elementwise_chain(B, *(leaf(B, v) for v in (a, b, c, d)))
+    np.testing.assert_array_equal(y.array, f32(1.25, -0.5, 1.0, 0.0))
+
+
+def test_binary_ops_match_numpy_float32(B):
+    g = rng.generator(5)
+    x = rng.normal_f32(g, (37, 19), 2.0)
+    y = rng.normal_f32(g, (37, 19), 2.0)
+    for name, fn in (("add", np.add), ("sub", np.subtract), ("mul", np.multiply), ("div", np.divide),
+                     ("max", np.maximum), ("min", np.minimum)):
+        got = B.op(name, leaf(B, x), leaf(B, y)).array
+        np.testing.assert_array_equal(got.view(np.uint32), fn(x, y).astype(F32).view(np.uint32), err_msg=name)
+    # operand order matters for sub/div: a transposed operand fails here
+    assert B.op("sub", leaf(B, f32(3)), leaf(B, f32(1))).array[0] == 2.0
+    assert B.op("div", leaf(B, f32(3)), leaf(B, f32(2))).array[0] == 1.5
+
+
+def test_single_rounding_per_op(B):
+    # (1 + 2^-24) is not representable: a*b+c with contraction would differ from two roundings
+    a, b, c = f32(1 + 2**-12), f32(1 + 2**-12), f32(-1.0)
+    prod = B.op("mul", leaf(B, a), leaf(B, b))
+    assert prod.array[0] == F32(1 + 2**-11)  # 2^-24 term rounded away (ties to even)
+    s = B.op("add", prod, leaf(B, c))
+    assert s.array[0] == F32(2**-11)
+
+
+def test_identities(B):
+    g = rng.generator(6)
+    x = rng.normal_f32(g, (1000,), 10.0)
+    X = leaf(B, x)
+    np.testing.assert_array_equal(B.op("mul", X, B.scalar(1.0)).array, x)
+    np.testing.assert_array_equal(B.op("add", X, B.scalar(0.0)).array, x)
+    np.testing.assert_array_equal(B.op("sub", X, X).array, np.zeros_like(x))
+    np.testing.assert_array_equal(B.op("square", X).array, x * x)
+    np.testing.assert_array_equal(B.op("neg", X).array, -x)
+    np.testing.assert_array_equal(B.op("abs", X).array, np.abs(x))
+    relu = B.op("relu", X).array
+    np.testing.assert_array_equal(relu, np.maximum(x, 0))
+    np.testing.assert_array_equal(relu, B.op("max", X, B.scalar(0.0)).array)
+    half = B.op("mul", B.op("add", X, B.op("abs", X)), B.scalar(0.5)).array  # (x+|x|)/2, exact
+    np.testing.assert_array_equal(relu, half)
+
+
+def test_nan_propagation(B):
+    nan = float("nan")
+    a, b = leaf(B, f32(nan, 1.0, nan, -0.0)), leaf(B, f32(1.0, nan, nan, 0.0))
+    assert np.isnan(B.op("max", a, b).array[:3]).all()
+    assert np.isnan(B.op("min", a, b).array[:3]).all()
+    assert np.isnan(B.op("relu", leaf(B, f32(nan))).array[0])
+    assert B.op("relu", leaf(B, f32(-0.0))).array[0] == 0.0
+
+
+def test_unary_against_float64_library(B):
+    g = rng.generator(7)
+    x = rng.normal_f32(g, (5000,), 3.0)
+    pos = np.abs(x) + F32(1e-3)
+    checks = [("exp", x, np.exp), ("tanh", x, np.tanh), ("log", pos, np.log),
+              ("rsqrt", pos, lambda v: 1 / np.sqrt(v)), ("recip", pos, lambda v: 1 / v),
+              ("sigmoid", x, lambda v: 1 / (1 + np.exp(-v)))]
+    for name, arg, fn in checks:
+        got = B.op(name, leaf(B, arg)).array
+        want = fn(arg.astype(np.float64))
+        np.testing.assert_allclose(got, want, rtol=6e-8, atol=0, err_msg=name)  # half an ulp
+    np.testing.assert_array_equal(B.op("sqrt", leaf(B, pos)).array, np.sqrt(pos))
+    assert B.op("exp", leaf(B, f32(0.0))).array[0] == 1.0
+    assert B.op("tanh", leaf(B, f32(0.0))).array[0] == 0.0
+
+
+def test_integer_and_mask_ops_bruteforce(B):
+    a = np.array([0, 1, -1, 2**31 - 1, -2**31, 7], dtype=np.int32)
+    b = np.array([5, -1, -1, 1, -1, 7], dtype=np.int32)
+    A, Bv = leaf(B, a, "i32"), leaf(B, b, "i32")
+    want = {"add": a + b, "sub": a - b, "mul": a * b, "max": np.maximum(a, b), "min": np.minimum(a, b)}
+    with np.errstate(over="ignore"):
+        for name, w in want.items():
+            np.testing.assert_array_equal(B.op(name, A, Bv).array, w, err_msg=name)
+    for name, fn in (("gt", np.greater), ("ge", np.greater_equal), ("lt", np.less), ("le", np.less_equal),
+                     ("eq", np.equal), ("ne", np.not_equal)):
+        np.testing.assert_array_equal(B.op(name, A, Bv).array, fn(a, b).astype(np.uint8), err_msg=name)
+    # unsigned compare differs from signed on the top bit
+    ua, ub = a.view(np.uint32), b.view(np.uint32)
+    np.testing.assert_array_equal(B.op("gt", leaf(B, ua, "u32"), leaf(B, ub, "u32")).array, (ua > ub).astype(np.uint8))
+    m1 = leaf(B, np.array([1, 0, 1, 0], dtype=np.uint8), "u8")
+    m2 = leaf(B, np.array([1, 1, 0, 0], dtype=np.uint8), "u8")
+    np.testing.assert_array_equal(B.op("and", m1, m2).array, [1, 0, 0, 0])
+    np.testing.assert_array_equal(B.op("or", m1, m2).array, [1, 1, 1, 0])
+    np.testing.assert_array_equal(B.op("not", m1).array, [0, 1, 0, 1])
+    x, y = leaf(B, f32(1, 2, 3, 4)), leaf(B, f32(-1, -2, -3, -4))
+    np.testing.assert_array_equal(B.op("where", m1, x, y).array, f32(1, -2, 3, -4))
+    np.testing.assert_array_equal(B.op("where", m1, x, B.scalar(0.0)).array, f32(1, 0, 3, 0))
+
+
+def test_float_compare_nan(B):
+    a, b = leaf(B, f32(float("nan"), 1.0)), leaf(B, f32(1.0, 1.0))
+    assert list(B.op("eq", a, b).array) == [0, 1]
+    assert list(B.op("ne", a, b).array) == [1, 0]
+    assert list(B.op("ge", a, b).array) == [0, 1]
+
+
+def test_convert_table(B):
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, f32(1.9, -1.9, 0.5, -0.0, float("nan"), 3e9, -3e9)), dtype="i32").array,
+        np.array([1, -1, 0, 0, 0, 2**31 - 1, -2**31], dtype=np.int32))
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, np.array([0, 1, 255], np.uint8), "u8"), dtype="f32").array, f32(0, 1, 255))
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, np.array([-3, 2**24 + 1], np.int32), "i32"), dtype="f32").array,
+        f32(-3, 2**24))  # ties to even
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, np.array([2**32 - 1], np.uint32), "u32"), dtype="f32").array, f32(2**32))
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, f32(0.0, -0.0, 0.1, float("nan"))), dtype="u8").array, [0, 0, 1, 1])
+
+
+def test_iota_bruteforce(B):
+    shape = (2, 3, 4)
+    for dim in range(3):
+        got = B.op("iota", shape=shape, dim=dim).array
+        want = np.indices(shape)[dim].astype(np.int32)
+        np.testing.assert_array_equal(got, want)
+
+
+def test_broadcast_classes_match_numpy(B):
+    g = rng.generator(8)
+    full = rng.normal_f32(g, (3, 5, 7))
+    for other_shape in [(7,), (1, 7), (5, 1), (3, 5, 1), (3, 1, 7), ()]:
+        other = rng.normal_f32(g, other_shape)
+        got = B.op("sub", leaf(B, full), leaf(B, other)).array
+        np.testing.assert_array_equal(got, full - other, err_msg=str(other_shape))
+        got = B.op("sub", leaf(B, other), leaf(B, full)).array
+        np.testing.assert_array_equal(got, other - full, err_msg=str(other_shape))
+    with pytest.raises(ValueError):
+        B.op("add", leaf(B, full), leaf(B, np.zeros((4,), F32)))
+
+
+# ---------------------------------------------------------------- reductions
+
+def test_row_sum_exact_rounding(B):
+    g = rng.generator(9)
+    x = rng.normal_f32(g, (17, 301), 100.0)
+    got = B.op("row_sum", leaf(B, x)).array
+    assert got.shape == (17, 1)
+    for r in range(17):
+        exact = math.fsum(float(v) for v in x[r])  # correctly rounded double sum
+        assert abs(float(got[r, 0]) - exact) <= abs(exact) * 2**-24 + 1e-30
+    # cancellation that float32 accumulation would lose: 2^25 + 1 + ... - 2^25
+    row = np.array([[2.0**25] + [1.0] * 16 + [-(2.0**25)]], dtype=F32)
+    assert B.op("row_sum", leaf(B, row)).array[0, 0] == 16.0
+
+
+def test_row_max_min(B):
+    x = f32(1, 5, -2, 5, 0, -7).reshape(2, 3)
+    np.testing.assert_array_equal(B.op("row_max", leaf(B, x)).array, f32(5, 5).reshape(2, 1))
+    np.testing.assert_array_equal(B.op("row_min", leaf(B, x)).array, f32(-2, -7).reshape(2, 1))
+    y = f32(1, float("nan"), 3).reshape(1, 3)
+    assert np.isnan(B.op("row_max", leaf(B, y)).array[0, 0])
+    np.testing.assert_array_equal(B.op("row_max", leaf(B, f32(-np.inf, -np.inf).reshape(1, 2))).array, [[-np.inf]])
+
+
+# ---------------------------------------------------------------------- GELU
+
+def test_gelu_closed_forms(B):
+    assert B.op("gelu_tanh", leaf(B, f32(0.0))).array[0] == 0.0
+    x = f32(-12, -3, -1, -0.1, 0.1, 1, 3, 12)
+    y = B.op("gelu_tanh", leaf(B, x)).array
+    assert y[-1] == 12.0 and abs(y[0]) < 1e-20  # x >> 0 -> x ; x << 0 -> 0
+    ym = B.op("gelu_tanh", leaf(B, -x)).array
+    np.testing.assert_allclose(y - ym, x, rtol=1e-6)  # odd part: gelu(x) - gelu(-x) = x
+    want = torch.nn.functional.gelu(torch.from_numpy(x).double(), approximate="tanh").numpy()
+    np.testing.assert_allclose(y, want, rtol=1e-7, atol=1e-30)
+
+
+def test_gelu_primitive_trace_matches_definition(B):
+    g = rng.generator(10)
+    xb, hb, bb = configs.c2_inputs(10, (33, 40))
+    for prim in (True, False):
+        out = traces.mlp_epilogue(B, leaf(B, xb, "bf16"), leaf(B, hb, "bf16"), leaf(B, bb, "bf16"),
+                                  primitive_gelu=prim)
+        assert out.dtype == "bf16" and out.shape == (33, 40)
+        x, h, b = (torch.from_numpy(rng.bf16_bits_to_f32(v)).double() for v in (xb, hb, bb))
+        want = (x + torch.nn.functional.gelu(h + b, approximate="tanh")).numpy()
+        # bf16 storage: half an ulp of bf16 is 2^-9 relative
+        np.testing.assert_allclose(out.as_f32(), want, rtol=2**-8, atol=1e-6)
+
+
+# ------------------------------------------------------------------- softmax
+
+def _softmax(B, x, scale=1.0, out_dtype="f32"):
+    return traces.causal_softmax(B, leaf(B, rng.to_bf16_bits(x), "bf16"), shape=x.shape, scale=scale,
+                                 out_dtype=out_dtype)
+
+
+def test_softmax_invariants(B):
+    g = rng.generator(12)
+    x = rng.bf16_bits_to_f32(rng.normal_bf16(g, (2, 24, 24), 4.0))
+    y = _softmax(B, x, scale=0.25).array
+    np.testing.assert_allclose(y.astype(np.float64).sum(-1), 1.0, atol=2e-6)  # rows sum to 1
+    iu = np.triu_indices(24, k=1)
+    assert (y[:, iu[0], iu[1]].view(np.uint32) == 0).all()  # masked entries are exactly +0
+    np.testing.assert_array_equal(y[:, 0, :], np.tile(f32(1, *[0] * 23), (2, 1)))  # row 0 = (1,0,..,0)
+    # library routine in float64
+    t = torch.from_numpy(x).double() * 0.25
+    mask = torch.triu(torch.ones(24, 24, dtype=torch.bool), diagonal=1)
+    want = torch.softmax(t.masked_fill(mask, -math.inf), dim=-1).numpy()
+    np.testing.assert_allclose(y, want, rtol=3e-6, atol=1e-9)
+
+
+def test_softmax_shift_invariance_and_uniform_rows(B):
+    x = np.zeros((1, 8, 8), dtype=F32) + F32(3.0)
+    y = _softmax(B, x).array
+    for r in range(8):
+        np.testing.assert_allclose(y[0, r, : r + 1], 1.0 / (r + 1), rtol=1e-6)  # uniform over unmasked
+    g = rng.generator(13)
+    a = rng.bf16_bits_to_f32(rng.normal_bf16(g, (1, 16, 16), 1.0))
+    a = np.round(a * 8) / 8  # keep a + 4 exactly representable in bf16
+    np.testing.assert_array_equal(_softmax(B, a.astype(F32)).array, _softmax(B, (a + 4).astype(F32)).array)
+
+
+def test_softmax_fully_masked_row_is_nan(B):
+    s = leaf(B, f32(-np.inf, -np.inf, 0, 1).reshape(2, 2))
+    mx = B.op("row_max", s)
+    e = B.op("exp", B.op("sub", s, mx))
+    y = B.op("div", e, B.op("row_sum", e)).array
+    assert np.isnan(y[0]).all() and not np.isnan(y[1]).any()
+
+
+# ----------------------------------------------------------------- LayerNorm
+
+def _ln(B, x, h, gamma, beta, p, eps=1e-5, seed=1, offset=0, out_dtype="f32"):
+    return traces.residual_dropout_layernorm(
+        B, leaf(B, rng.to_bf16_bits(x), "bf16"), leaf(B, rng.to_bf16_bits(h), "bf16"), leaf(B, gamma),
+        leaf(B, beta), shape=x.shape, p=p, eps=eps, seed=seed, offset=offset, out_dtype=out_dtype)
+
+
+def test_layernorm_invariants(B):
+    g = rng.generator(14)
+    C = 256
+    x = rng.bf16_bits_to_f32(rng.normal_bf16(g, (12, C), 1.0))
+    h = rng.bf16_bits_to_f32(rng.normal_bf16(g, (12, C), 1.0))
+    ones, zeros = np.ones(C, F32), np.zeros(C, F32)
+    z, keep = _ln(B, x, h, ones, zeros, p=0.0)
+    assert keep.array.all()  # p = 0 keeps everything
+    z64 = z.array.astype(np.float64)
+    assert np.abs(z64.mean(-1)).max() < 1e-6
+    t = x.astype(np.float64) + h
+    var = t.var(-1)
+    np.testing.assert_allclose(z64.var(-1), var / (var + 1e-5), rtol=1e-5)
+    want = torch.nn.functional.layer_norm(torch.from_numpy(t), (C,), eps=1e-5).numpy()
+    np.testing.assert_allclose(z.array, want, rtol=1e-5, atol=1e-6)
+    # affine parameters: per-column scale and shift
+    gamma, beta = rng.normal_f32(g, (C,), 0.02, 1.0), rng.normal_f32(g, (C,), 0.02)
+    z2, _ = _ln(B, x, h, gamma, beta, p=0.0)
+    np.testing.assert_allclose(z2.array, want * gamma + beta, rtol=1e-5, atol=1e-6)
+    # a constant row normalises to beta
+    z3, _ = _ln(B, np.full((2, C), 3.0, F32), np.full((2, C), 1.0, F32), gamma, beta, p=0.0)
+    np.testing.assert_allclose(z3.array, np.tile(beta, (2, 1)), atol=1e-6)
+    # LN(a*t + b) = sign(a) LN(t) as eps -> 0
+    xq, hq = np.round(x * 8) / 8, np.round(h * 8) / 8  # keeps -2*t + 1 exact in bf16 storage
+    z4, _ = _ln(B, (-2 * xq + 0.5).astype(F32), (-2 * hq + 0.5).astype(F32), ones, zeros, p=0.0, eps=1e-12)
+    z5, _ = _ln(B, xq.astype(F32), hq.astype(F32), ones, zeros, p=0.0, eps=1e-12)
+    np.testing.assert_allclose(z4.array, -z5.array, rtol=1e-4, atol=2e-5)
+
+
+def test_dropout_semantics(B):
+    g = rng.generator(15)
+    C = 64
+    x = np.zeros((40, C), F32)
+    h = rng.bf16_bits_to_f32(rng.normal_bf16(g, (40, C), 1.0))
+    p = 0.25
+    # reconstruct the pre-LayerNorm tensor with the identity LN turned off: use the mask directly
+    _, keep = _ln(B, x, h, np.ones(C, F32), np.zeros(C, F32), p=p, seed=99, offset=3)
+    bits = B.op("philox_bits", shape=(40, C), seed=99, offset=3).array
+    np.testing.assert_array_equal(keep.array, (bits >= np.uint32(2**30)).astype(np.uint8))
+    hs = B.op("mul", leaf(B, h), B.scalar(1.0 / (1.0 - p)))
+    hd = B.op("where", keep, hs, B.scalar(0.0)).array
+    np.testing.assert_array_equal(hd[keep.array == 0], 0.0)
+    np.testing.assert_allclose(hd[keep.array == 1], (h * F32(4.0 / 3.0))[keep.array == 1], rtol=1e-7)
+    assert traces.dropout_threshold(0.1) == 429496729 and traces.dropout_threshold(0.0) == 0
+
+
+# -------------------------------------------------------------------- Philox
+
+def _philox_ref(ctr, key):
+    """Second implementation with Python integers, written from the round description."""
+    c = list(ctr)
+    k = list(key)
+    for _ in range(10):
+        p0 = 0xD2511F53 * c[0]
+        p1 = 0xCD9E8D57 * c[2]
+        c = [(p1 >> 32) ^ c[1] ^ k[0], p1 & 0xFFFFFFFF, (p0 >> 32) ^ c[3] ^ k[1], p0 & 0xFFFFFFFF]
+        k = [(k[0] + 0x9E3779B9) & 0xFFFFFFFF, (k[1] + 0xBB67AE85) & 0xFFFFFFFF]
+    return c
+
+
+def test_philox_known_answers():
+    import ctypes
+    import os
+    L = lib()
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 3
+    for row in rows:
+        w = [int(t, 16) for t in row]
+        out = (ctypes.c_uint32 * 4)()
+        L.orc_philox4x32_10((ctypes.c_uint32 * 4)(*w[:4]), (ctypes.c_uint32 * 2)(*w[4:6]), out)
+        assert list(out) == w[6:]
+        assert _philox_ref(w[:4], w[4:6]) == w[6:]
+
+
+def test_philox_bits_layout_and_determinism(B):
+    seed, offset = 0x123456789ABCDEF0, 0x1_0000_0007
+    bits = B.op("philox_bits", shape=(5, 7), seed=seed, offset=offset).array.reshape(-1)
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for i in range(35):
+        q = i // 4
+        want = _philox_ref([q & 0xFFFFFFFF, q >> 32, offset & 0xFFFFFFFF, offset >> 32], key)[i % 4]
+        assert int(bits[i]) == want
+    again = B.op("philox_bits", shape=(5, 7), seed=seed, offset=offset).array.reshape(-1)
+    np.testing.assert_array_equal(bits, again)
+    other = B.op("philox_bits", shape=(5, 7), seed=seed, offset=offset + 1).array.reshape(-1)
+    assert (bits != other).mean() > 0.9
+    other = B.op("philox_bits", shape=(5, 7), seed=seed + 1, offset=offset).array.reshape(-1)
+    assert (bits != other).mean() > 0.9
+
+
+def test_philox_keep_rate(B):
+    n = 1 << 22
+    bits = B.op("philox_bits", shape=(n,), seed=7, offset=0).array
+    p = 0.1
+    keep = (bits >= np.uint32(traces.dropout_threshold(p))).mean()
+    sigma = math.sqrt(p * (1 - p) / n)
+    assert abs(keep - (1 - p)) < 4 * sigma
+    assert abs(bits.astype(np.float64).mean() / 2**32 - 0.5) < 4 * math.sqrt(1 / 12 / n)
+
+
+# ---------------------------------------------------------------------- Adam
+
+def test_adam_first_step_closed_form(B):
+    g_ = rng.generator(16)
+    p0 = rng.normal_f32(g_, (300,), 0.05)
+    gr = rng.normal_f32(g_, (300,), 1e-3)
+    p, g, m, v = leaf(B, p0), leaf(B, gr), leaf(B, np.zeros(300, F32)), leaf(B, np.zeros(300, F32))
+    traces.adam_step(B, [p], [g], [m], [v], step=1)
+    # m0 = v0 = 0: m_hat = g, v_hat = g^2, so the step is -lr * g / (|g| + eps)
+    want = p0.astype(np.float64) - 1e-3 * gr.astype(np.float64) / (np.abs(gr.astype(np.float64)) + 1e-8)
+    np.testing.assert_allclose(p.array, want, rtol=1e-6, atol=5e-9)  # f32 rounding of p - step
+    np.testing.assert_allclose(m.array, 0.1 * gr.astype(np.float64), rtol=1e-6)
+    np.testing.assert_allclose(v.array, 0.001 * gr.astype(np.float64) ** 2, rtol=1e-6)
+
+
+def test_adam_matches_torch_float64(B):
+    g_ = rng.generator(17)
+    p0 = rng.normal_f32(g_, (4, 50), 0.05)
+    grads = [rng.normal_f32(g_, (4, 50), 1e-3) for _ in range(5)]
+    tp = torch.nn.Parameter(torch.from_numpy(p0).double())
+    opt = torch.optim.Adam([tp], lr=1e-3, betas=(0.9, 0.999), eps=1e-8)
+    p, m, v = leaf(B, p0), leaf(B, np.zeros_like(p0)), leaf(B, np.zeros_like(p0))
+    for step, gr in enumerate(grads, start=1):
+        tp.grad = torch.from_numpy(gr).double()
+        opt.step()
+        traces.adam_step(B, [p], [leaf(B, gr)], [m], [v], step=step)
+        np.testing.assert_allclose(p.array, tp.detach().numpy(), rtol=2e-6, atol=1e-9)
+
+
+# ------------------------------------------------------------ workload recipe
+
+def test_resnet50_parameter_census():
+    from workloads.resnet50 import parameter_shapes
+    shapes = parameter_shapes()
+    sizes = [math.prod(s) for s in shapes]
+    assert len(shapes) == 161 and sum(sizes) == 25_557_032
+    assert sum(1 for n in sizes if n < 4096) == 107
+    assert min(sizes) == 64 and max(sizes) == 2_359_296
+    assert configs.algorithmic_bytes("c5") == 715_596_896
+    assert configs.algorithmic_bytes("c2") == 201_334_784
+    assert configs.algorithmic_bytes("c3") == 117_448_704
+    assert configs.algorithmic_bytes("c4") == 268_435_456
+    assert configs.algorithmic_bytes("c1") == 20_971_520
+
+
+def test_input_distributions():
+    x, h, bias = configs.c2_inputs(0, (256, 512))
+    xf = rng.bf16_bits_to_f32(x).astype(np.float64)
+    assert abs(xf.mean()) < 0.02 and abs(xf.std() - 1) < 0.02
+    assert abs(rng.bf16_bits_to_f32(bias).astype(np.float64).std() - 0.02) < 0.004
+    s = rng.bf16_bits_to_f32(configs.c4_inputs(0, (2, 128, 128))).astype(np.float64)
+    assert abs(s.std() - 4) < 0.1
+    a = configs.c1_inputs(0, (128, 128))[0]
+    assert a.min() >= -1 and a.max() <= 1 and abs(a.mean()) < 0.02
+    again = configs.c1_inputs(0, (128, 128))[0]
+    np.testing.assert_array_equal(a, again)
