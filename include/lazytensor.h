@@ -1,0 +1,254 @@
+/*
+ * lazytensor.h -- C ABI of the fused-graph LazyTensor executor for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the runtime half of the LazyTensor method (Suhan et al.,
+ * "LazyTensor: combining eager execution with domain-specific compilers"):
+ * tensor operations are recorded into an IR graph instead of being dispatched
+ * (Section 3); a barrier call ends the graph, canonicalises and hashes it, looks
+ * it up in a compile cache and executes it (Section 4); in-place updates are a
+ * substitution of the destination's computation, with input buffers donated to
+ * outputs at the barrier (Section 4.3).  Where the paper hands the graph to the
+ * XLA compiler, this library cuts it into fusion groups and runs each group as
+ * one hand-written CUDA kernel that interprets a small register program.
+ *
+ * Conventions
+ *   - Every call returns an lt_status; LT_OK is 0.  A human-readable message for the
+ *     last failing call on a context is available from lt_last_error().  No call
+ *     throws, aborts or exits.  A failed lt_op records nothing; a failed lt_barrier
+ *     leaves the pending graph in place so it can be flushed again.
+ *   - "host" pointers are ordinary process memory; "device" pointers are CUDA global
+ *     memory on the context's device.
+ *   - A context and its tensors may be used by one thread at a time.
+ *   - Tensors are dense, row-major, contiguous.  Rank is at most LT_MAX_RANK.
+ *   - Handles belong to the context that made them; a handle used with another
+ *     context gives LT_ERR_DEVICE (Section 4.1: no implicit cross-device transfers).
+ */
+#ifndef LAZYTENSOR_H_
+#define LAZYTENSOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LT_MAX_RANK 6
+
+/* One context per device: the liveness arena of Section 4 ("DeviceContextArena"). */
+typedef struct lt_ctx lt_ctx;
+
+/* Unique tensor identifier (Section 4: RegisterTensor / UnregisterTensor). 0 is never valid. */
+typedef uint64_t lt_tensor;
+
+typedef enum {
+    LT_OK = 0,
+    LT_ERR_INVALID_ARG = 1,   /* null pointer, unknown handle, bad rank, ...             */
+    LT_ERR_SHAPE = 2,         /* operand shapes are not one of the supported broadcasts  */
+    LT_ERR_DTYPE = 3,         /* dtype combination not defined for the op                */
+    LT_ERR_DEVICE = 4,        /* handle of another context / device                      */
+    LT_ERR_UNSUPPORTED = 5,   /* op or shape outside what the kernels implement          */
+    LT_ERR_OOM = 6,           /* the allocator callback returned NULL                    */
+    LT_ERR_CUDA = 7,          /* a CUDA runtime call failed (message has the CUDA text)  */
+    LT_ERR_DEVICE_TIMEOUT = 8 /* a bounded device-side wait gave up                      */
+} lt_status;
+
+typedef enum { LT_F32 = 0, LT_BF16 = 1, LT_U8 = 2, LT_I32 = 3, LT_U32 = 4 } lt_dtype;
+
+/*
+ * Traced operations ("IR compatible" operations, Section 3).  Arithmetic on LT_BF16
+ * nodes is done in binary32 on widened operands and rounded to bf16 (ties to even).
+ *
+ * Broadcasting (Fig. 1 shows only scalar expansion; the classes here are the four the
+ * kernels implement): an operand either has the result's shape, or is rank 0, or
+ * has every dimension 1 except a last dimension equal to the result's ("column
+ * vector", e.g. [C] or [1,C]), or equals the result's shape except for a last
+ * dimension of 1 ("row scalar", e.g. [R,1]).  Anything else is LT_ERR_SHAPE.
+ * Operands share one dtype; a rank-0 scalar adopts the dtype of the tensor it meets.
+ */
+typedef enum {
+    /* binary: 2 inputs.  f32/bf16: ADD..MIN; i32/u32: ADD SUB MUL MAX MIN AND OR XOR; u8: AND OR XOR */
+    LT_OP_ADD = 1, LT_OP_SUB = 2, LT_OP_MUL = 3, LT_OP_DIV = 4, LT_OP_MAX = 5, LT_OP_MIN = 6,
+    LT_OP_AND = 7, LT_OP_OR = 8, LT_OP_XOR = 9,
+    /* compare: 2 inputs of one dtype -> LT_U8 holding 0 or 1 */
+    LT_OP_GT = 10, LT_OP_GE = 11, LT_OP_LT = 12, LT_OP_LE = 13, LT_OP_EQ = 14, LT_OP_NE = 15,
+    /* select: inputs (mask u8, a, b) -> mask != 0 ? a : b */
+    LT_OP_WHERE = 16,
+    /* unary, float dtypes (NEG and ABS also i32; NOT on u8: x == 0) */
+    LT_OP_NEG = 20, LT_OP_ABS = 21, LT_OP_RELU = 22, LT_OP_EXP = 23, LT_OP_LOG = 24, LT_OP_TANH = 25,
+    LT_OP_SQRT = 26, LT_OP_RSQRT = 27, LT_OP_RECIP = 28, LT_OP_SQUARE = 29, LT_OP_SIGMOID = 30,
+    LT_OP_GELU_TANH = 31, /* 0.5 t (1 + tanh(sqrt(2/pi) (t + 0.044715 t^3))) */
+    LT_OP_NOT = 32,
+    /* type conversion: 1 input, attrs = {lt_dtype}.  f32->i32 truncates and saturates (NaN -> 0);
+       anything -> u8 is (x != 0); i32 <-> u32 keeps the bits; u8 -> wider zero-extends. */
+    LT_OP_CONVERT = 40,
+    /* factory "range" (Section 3): 0 inputs, attrs = {dim, rank, d0, .., d(rank-1)} -> i32 coordinate along dim */
+    LT_OP_IOTA = 41,
+    /* factory "random" (Section 3): 0 inputs, attrs = {seed, offset, rank, d0, ..} -> u32.
+       Element i is word (i mod 4) of the Philox4x32-10 block with counter
+       (lo32(i/4), hi32(i/4), lo32(offset), hi32(offset)) and key (lo32(seed), hi32(seed)).
+       seed and offset are run-time parameters: they do not enter the graph hash. */
+    LT_OP_PHILOX_BITS = 42,
+    /* reductions over the last dimension, kept with extent 1; float dtypes */
+    LT_OP_ROW_SUM = 50, LT_OP_ROW_MAX = 51, LT_OP_ROW_MIN = 52
+} lt_opcode;
+
+/*
+ * Device memory comes from the caller (e.g. PyTorch's caching allocator).  `alloc`
+ * returns device memory of at least `nbytes`, aligned to 256 bytes, usable on `stream`
+ * in stream order, or NULL.  `free` is called with a pointer `alloc` returned, after the
+ * last kernel using it has been enqueued on `stream` (stream-ordered reuse is safe).
+ * With a NULL lt_allocator the library uses cudaMallocAsync / cudaFreeAsync on the stream.
+ */
+typedef struct {
+    void *(*alloc)(size_t nbytes, void *stream, void *user);
+    void (*free)(void *dptr, void *stream, void *user);
+    void *user;
+} lt_allocator;
+
+/* Counters since context creation or the last lt_reset_stats. Times are host nanoseconds. */
+typedef struct {
+    uint64_t nodes_recorded;     /* IR nodes appended by lt_op / factories                   */
+    uint64_t barriers;           /* lt_barrier calls that found pending work                  */
+    uint64_t compiles;           /* cache misses: graphs planned                             */
+    uint64_t cache_hits;         /* barriers served from the plan cache                      */
+    uint64_t kernels_launched;   /* all kernels                                              */
+    uint64_t launches_elementwise, launches_row, launches_multi;
+    uint64_t bytes_planned;      /* bytes the launched kernels were planned to read + write  */
+    uint64_t outputs_donated;    /* outputs written into a donated input buffer              */
+    uint64_t outputs_allocated;  /* outputs given fresh memory                               */
+    uint64_t temporaries_allocated; /* cross-kernel intermediates given scratch memory        */
+    uint64_t ns_record;          /* inside lt_op and the factory calls                       */
+    uint64_t ns_canonicalise;    /* root gathering + post-order serialisation                */
+    uint64_t ns_hash_lookup;     /* hashing + cache probe                                    */
+    uint64_t ns_plan;            /* fusion planning + program generation (misses only)       */
+    uint64_t ns_bind_launch;     /* argument binding, allocation and kernel launches         */
+    uint64_t ns_rebind;          /* turning roots into device-data leaves, freeing IR        */
+} lt_stats;
+
+/* Device time per kernel family, measured with CUDA events when kernel timing is on. */
+typedef struct {
+    uint64_t launches[3];        /* 0 elementwise, 1 row-reduction, 2 multi-tensor */
+    double ms[3];
+    uint64_t bytes[3];           /* planned bytes of those launches */
+} lt_kernel_timing;
+
+/*
+ * Context lifetime.  `device` is a CUDA device ordinal, or LT_DEVICE_NONE for a
+ * record-and-plan-only context (no CUDA call is ever made; lt_barrier plans, counts
+ * and rebinds but launches nothing; lt_fetch fails) used to test host logic.
+ * `cuda_stream` is a cudaStream_t (NULL = default stream) on which all work is enqueued.
+ * `allocator` may be NULL (see lt_allocator).  The context copies the struct.
+ */
+#define LT_DEVICE_NONE (-1)
+lt_status lt_ctx_create(int device, void *cuda_stream, const lt_allocator *allocator, lt_ctx **out);
+lt_status lt_ctx_destroy(lt_ctx *ctx);
+
+/*
+ * Options: "fusion" (1 default; 0 = one kernel per traced op, the unfused baseline),
+ * "verify" (1 default: on a cache hit compare the canonical bytes, not just the hash),
+ * "fast_math" (1 default: groups whose stored results are all bf16/u8 may use approximate
+ * exp/tanh/rsqrt/division and fused multiply-add; groups storing f32 never do),
+ * "horizontal" (1 default: bundle isomorphic independent groups into multi-tensor launches),
+ * "cache_capacity" (0 = unbounded).  Options are part of the cache key.
+ * Unknown key: LT_ERR_INVALID_ARG.  The environment variables LT_FUSION, LT_VERIFY,
+ * LT_FAST_MATH, LT_HORIZONTAL preset the same options at context creation.
+ */
+lt_status lt_ctx_set_option(lt_ctx *ctx, const char *key, int64_t value);
+
+/*
+ * Factory from existing data (Section 3; the "device_data" leaves of Fig. 1).
+ * lt_tensor_from_device BORROWS `dptr` (device): the caller keeps it alive and unchanged
+ * while any tensor or pending graph refers to it; the library never frees it and writes
+ * it only when the tensor is the destination of lt_assign (donation, Section 4.3).
+ * 16-byte alignment enables 128-bit accesses; other alignments work, slower.
+ * lt_tensor_from_host copies `hptr` (host) into memory from the allocator (owned by the
+ * library, freed when the last tensor naming it is released); the copy is enqueued on the
+ * stream and `hptr` may be reused after the call returns only if it is pageable memory
+ * (for pinned memory: after the next blocking barrier or stream synchronisation).
+ */
+lt_status lt_tensor_from_device(lt_ctx *ctx, void *dptr, lt_dtype dtype, int rank, const int64_t *shape,
+                                lt_tensor *out);
+lt_status lt_tensor_from_host(lt_ctx *ctx, const void *hptr, lt_dtype dtype, int rank, const int64_t *shape,
+                              lt_tensor *out);
+
+/*
+ * Rank-0 constant (Fig. 1: prim::Constant).  Section 4.1's heuristic: the values 0 and 1
+ * (bit-equal to +0.0 or 1.0 as the double passed here) are encoded in the graph and its
+ * hash; every other value is a run-time parameter, so graphs that differ only in such
+ * values share one cache entry.  lt_scalar_dynamic forces the run-time class even for 0/1.
+ * `dtype` is the dtype the scalar has when it meets no tensor; next to a tensor it adopts
+ * the tensor's dtype (integer dtypes need an integral value: else LT_ERR_DTYPE at lt_op).
+ */
+lt_status lt_scalar(lt_ctx *ctx, double value, lt_dtype dtype, lt_tensor *out);
+lt_status lt_scalar_dynamic(lt_ctx *ctx, double value, lt_dtype dtype, lt_tensor *out);
+
+/*
+ * Record one operation (Section 3: ops are buffered, not dispatched).  `in` holds `n_in`
+ * handles, `attrs` holds `n_attrs` integers as the opcode requires.  Result shape and dtype
+ * are inferred; nothing is launched.
+ */
+lt_status lt_op(lt_ctx *ctx, int opcode, const lt_tensor *in, int n_in, const int64_t *attrs, int n_attrs,
+                lt_tensor *out);
+
+/*
+ * In-place update (Section 4.3): `dst` from now on denotes the computation behind `src`
+ * (shape and dtype must match).  If `dst` was materialised data, its buffer becomes a
+ * donation candidate: at the next barrier the new value is written into that buffer when
+ * no other live tensor still names the old value and every read of the buffer is by the
+ * kernel that overwrites it, at the same element index, or by an earlier kernel.
+ */
+lt_status lt_assign(lt_ctx *ctx, lt_tensor dst, lt_tensor src);
+
+/* UnregisterTensor: the handle dies; a pending computation nobody names is never run. */
+lt_status lt_release(lt_ctx *ctx, lt_tensor t);
+
+/*
+ * Barrier (Section 4; mark_step / LazyTensorBarrier): materialise every live tensor that
+ * has pending computation.  With `blocking` non-zero, return after the stream has drained.
+ */
+lt_status lt_barrier(lt_ctx *ctx, int blocking);
+
+/*
+ * IR-incompatible read-out (Section 3): runs a blocking barrier if `t` is pending, then
+ * copies the tensor to `host_dst` (host).  `nbytes` must equal the tensor's byte size.
+ */
+lt_status lt_fetch(lt_ctx *ctx, lt_tensor t, void *host_dst, size_t nbytes);
+
+/* Device pointer of a materialised tensor (LT_ERR_INVALID_ARG while it is pending). */
+lt_status lt_device_ptr(lt_ctx *ctx, lt_tensor t, void **dptr);
+
+/* Shape query; `shape` has room for LT_MAX_RANK entries; any out pointer may be NULL. */
+lt_status lt_tensor_info(lt_ctx *ctx, lt_tensor t, int *dtype, int *rank, int64_t *shape, int *materialised);
+
+lt_status lt_get_stats(lt_ctx *ctx, lt_stats *out);
+lt_status lt_reset_stats(lt_ctx *ctx);
+
+/* Number of plans in the cache. */
+lt_status lt_cache_size(lt_ctx *ctx, uint64_t *out);
+
+/*
+ * Kernel timing: when enabled, every launch is bracketed by CUDA events on the stream.
+ * lt_get_kernel_timing synchronises the stream, adds up the finished brackets since the
+ * last call (or since enabling) and returns them.
+ */
+lt_status lt_set_kernel_timing(lt_ctx *ctx, int enable);
+lt_status lt_get_kernel_timing(lt_ctx *ctx, lt_kernel_timing *out);
+
+/*
+ * Text dumps.  Both write at most `cap` bytes including the terminator into `buf` (may be
+ * NULL with cap 0) and report the size needed in `*need`.
+ * lt_dump_ir: the pending graph in the textual form of Fig. 1 ("%3 = f32[2,4] mul(%2, %1)",
+ * roots marked ROOT=k).  lt_dump_plan: the plan the last barrier executed -- one block per
+ * kernel launch with its family, geometry, inputs, outputs and register program.
+ */
+lt_status lt_dump_ir(lt_ctx *ctx, char *buf, size_t cap, size_t *need);
+lt_status lt_dump_plan(lt_ctx *ctx, char *buf, size_t cap, size_t *need);
+
+const char *lt_last_error(lt_ctx *ctx);
+const char *lt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAZYTENSOR_H_ */

@@ -1,0 +1,349 @@
+"""Python binding of liblazytensor.so (argument marshalling only).
+
+`LazyContext` and `LazyTensor` mirror the C ABI in include/lazytensor.h one to one:
+every method forwards to the entry point of the same name.  All recording, hashing,
+planning and execution happens in the shared library; there is no Python or CPU
+fallback -- if the library is missing, importing this module raises.
+
+PyTorch is used for device memory (its caching allocator backs the allocator
+callbacks) and for the CUDA stream the kernels are enqueued on.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+LIB_PATH = _HERE / "liblazytensor.so"
+
+if not LIB_PATH.exists():
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+        "(there is no fallback implementation)")
+
+_lib = ctypes.CDLL(str(LIB_PATH))
+
+LT_MAX_RANK = 6
+LT_DEVICE_NONE = -1
+DTYPES = {"f32": 0, "bf16": 1, "u8": 2, "i32": 3, "u32": 4}
+DTYPE_NAMES = {v: k for k, v in DTYPES.items()}
+NP_DTYPES = {"f32": np.float32, "bf16": np.uint16, "u8": np.uint8, "i32": np.int32, "u32": np.uint32}
+OPCODES = {
+    "add": 1, "sub": 2, "mul": 3, "div": 4, "max": 5, "min": 6, "and": 7, "or": 8, "xor": 9,
+    "gt": 10, "ge": 11, "lt": 12, "le": 13, "eq": 14, "ne": 15, "where": 16,
+    "neg": 20, "abs": 21, "relu": 22, "exp": 23, "log": 24, "tanh": 25, "sqrt": 26, "rsqrt": 27,
+    "recip": 28, "square": 29, "sigmoid": 30, "gelu_tanh": 31, "not": 32,
+    "convert": 40, "iota": 41, "philox_bits": 42, "row_sum": 50, "row_max": 51, "row_min": 52,
+}
+STATUS_NAMES = ["LT_OK", "LT_ERR_INVALID_ARG", "LT_ERR_SHAPE", "LT_ERR_DTYPE", "LT_ERR_DEVICE",
+                "LT_ERR_UNSUPPORTED", "LT_ERR_OOM", "LT_ERR_CUDA", "LT_ERR_DEVICE_TIMEOUT"]
+
+ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)
+FREE_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p)
+
+
+class lt_allocator(ctypes.Structure):
+    _fields_ = [("alloc", ALLOC_FN), ("free", FREE_FN), ("user", ctypes.c_void_p)]
+
+
+class lt_stats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in (
+        "nodes_recorded", "barriers", "compiles", "cache_hits", "kernels_launched",
+        "launches_elementwise", "launches_row", "launches_multi", "bytes_planned",
+        "outputs_donated", "outputs_allocated", "temporaries_allocated",
+        "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind")]
+
+
+class lt_kernel_timing(ctypes.Structure):
+    _fields_ = [("launches", ctypes.c_uint64 * 3), ("ms", ctypes.c_double * 3), ("bytes", ctypes.c_uint64 * 3)]
+
+
+_P = ctypes.POINTER
+_vp, _i64, _u64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_uint64, ctypes.c_int
+
+_SIGNATURES = {
+    "lt_ctx_create": [_int, _vp, _P(lt_allocator), _P(_vp)],
+    "lt_ctx_destroy": [_vp],
+    "lt_ctx_set_option": [_vp, ctypes.c_char_p, _i64],
+    "lt_tensor_from_device": [_vp, _vp, _int, _int, _P(_i64), _P(_u64)],
+    "lt_tensor_from_host": [_vp, _vp, _int, _int, _P(_i64), _P(_u64)],
+    "lt_scalar": [_vp, ctypes.c_double, _int, _P(_u64)],
+    "lt_scalar_dynamic": [_vp, ctypes.c_double, _int, _P(_u64)],
+    "lt_op": [_vp, _int, _P(_u64), _int, _P(_i64), _int, _P(_u64)],
+    "lt_assign": [_vp, _u64, _u64],
+    "lt_release": [_vp, _u64],
+    "lt_barrier": [_vp, _int],
+    "lt_fetch": [_vp, _u64, _vp, ctypes.c_size_t],
+    "lt_device_ptr": [_vp, _u64, _P(_vp)],
+    "lt_tensor_info": [_vp, _u64, _P(_int), _P(_int), _P(_i64), _P(_int)],
+    "lt_get_stats": [_vp, _P(lt_stats)],
+    "lt_reset_stats": [_vp],
+    "lt_cache_size": [_vp, _P(_u64)],
+    "lt_set_kernel_timing": [_vp, _int],
+    "lt_get_kernel_timing": [_vp, _P(lt_kernel_timing)],
+    "lt_dump_ir": [_vp, ctypes.c_char_p, ctypes.c_size_t, _P(ctypes.c_size_t)],
+    "lt_dump_plan": [_vp, ctypes.c_char_p, ctypes.c_size_t, _P(ctypes.c_size_t)],
+}
+for _name, _args in _SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.argtypes = _args
+    _fn.restype = _int
+_lib.lt_last_error.argtypes = [_vp]
+_lib.lt_last_error.restype = ctypes.c_char_p
+_lib.lt_version.argtypes = []
+_lib.lt_version.restype = ctypes.c_char_p
+
+EXPORTED_SYMBOLS = sorted(list(_SIGNATURES) + ["lt_last_error", "lt_version"])
+
+
+class LazyTensorError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {message}")
+        self.status = status
+
+
+def version() -> str:
+    return _lib.lt_version().decode()
+
+
+def _torch_allocator():
+    import torch
+
+    def _alloc(nbytes, stream, user):
+        try:
+            return torch.cuda.caching_allocator_alloc(int(nbytes), stream=int(stream or 0))
+        except Exception:  # out of memory: report NULL, the library turns it into LT_ERR_OOM
+            return None
+
+    def _free(ptr, stream, user):
+        torch.cuda.caching_allocator_delete(int(ptr))
+
+    return ALLOC_FN(_alloc), FREE_FN(_free)
+
+
+class LazyTensor:
+    """A handle of the C library; its value may still be a pending IR graph (paper Section 3)."""
+
+    __slots__ = ("ctx", "handle", "dtype", "shape", "_keep", "__weakref__")
+
+    def __init__(self, ctx: "LazyContext", handle: int, dtype: str, shape, keep=None):
+        self.ctx = ctx
+        self.handle = handle
+        self.dtype = dtype
+        self.shape = tuple(shape)
+        self._keep = keep  # device storage this tensor borrows
+
+    def __del__(self):
+        ctx = self.ctx
+        if ctx is not None and ctx._ctx:
+            _lib.lt_release(ctx._ctx, self.handle)
+
+    # the eager-looking API: every operator only records
+    def _bin(self, name, other, swap=False):
+        if not isinstance(other, LazyTensor):
+            other = self.ctx.scalar(other, self.dtype)
+        return self.ctx.op(name, other, self) if swap else self.ctx.op(name, self, other)
+
+    def __add__(self, o): return self._bin("add", o)
+    def __radd__(self, o): return self._bin("add", o, True)
+    def __sub__(self, o): return self._bin("sub", o)
+    def __rsub__(self, o): return self._bin("sub", o, True)
+    def __mul__(self, o): return self._bin("mul", o)
+    def __rmul__(self, o): return self._bin("mul", o, True)
+    def __truediv__(self, o): return self._bin("div", o)
+    def __rtruediv__(self, o): return self._bin("div", o, True)
+    def __neg__(self): return self.ctx.op("neg", self)
+    def __gt__(self, o): return self._bin("gt", o)
+    def __ge__(self, o): return self._bin("ge", o)
+    def __lt__(self, o): return self._bin("lt", o)
+    def __le__(self, o): return self._bin("le", o)
+
+    def __iadd__(self, o):
+        self.ctx.assign(self, self + o)
+        return self
+
+    def __isub__(self, o):
+        self.ctx.assign(self, self - o)
+        return self
+
+    def __imul__(self, o):
+        self.ctx.assign(self, self * o)
+        return self
+
+    def numpy(self) -> np.ndarray:
+        return self.ctx.fetch(self)
+
+
+class LazyContext:
+    """One per device: the liveness arena, IR recorder, compile cache and executor."""
+
+    def __init__(self, device: int | None = 0, stream: int | None = None, allocator: str = "torch"):
+        self._ctx = None
+        self.device = LT_DEVICE_NONE if device is None else int(device)
+        self._alloc_struct = None
+        alloc_ptr = None
+        if self.device != LT_DEVICE_NONE and allocator == "torch":
+            import torch
+
+            torch.cuda.set_device(self.device)
+            if stream is None:
+                stream = torch.cuda.current_stream(self.device).cuda_stream
+            a, f = _torch_allocator()
+            self._alloc_struct = lt_allocator(a, f, None)
+            alloc_ptr = ctypes.byref(self._alloc_struct)
+        out = _vp()
+        st = _lib.lt_ctx_create(self.device, _vp(stream or 0), alloc_ptr, ctypes.byref(out))
+        if st != 0:
+            raise LazyTensorError(st, "lt_ctx_create failed (is a CUDA device present?)")
+        self._ctx = out
+        self.stream = stream or 0
+        self._h = _u64()
+
+    def close(self):
+        if self._ctx:
+            ctx, self._ctx = self._ctx, None
+            _lib.lt_ctx_destroy(ctx)
+
+    def __del__(self):
+        self.close()
+
+    def _check(self, st: int):
+        if st != 0:
+            raise LazyTensorError(st, _lib.lt_last_error(self._ctx).decode())
+
+    def set_option(self, key: str, value: int) -> None:
+        self._check(_lib.lt_ctx_set_option(self._ctx, key.encode(), int(value)))
+
+    # ---- factories
+    def from_device_ptr(self, ptr: int, dtype: str, shape, keep=None) -> LazyTensor:
+        shp = (_i64 * max(len(shape), 1))(*shape)
+        self._check(_lib.lt_tensor_from_device(self._ctx, _vp(ptr), DTYPES[dtype], len(shape), shp, ctypes.byref(self._h)))
+        return LazyTensor(self, self._h.value, dtype, shape, keep)
+
+    def from_torch(self, t, dtype: str | None = None) -> LazyTensor:
+        """Wrap a contiguous CUDA torch tensor without copying (the tensor is kept alive)."""
+        import torch
+
+        names = {torch.float32: "f32", torch.bfloat16: "bf16", torch.uint8: "u8", torch.int32: "i32",
+                 torch.uint16: "bf16", torch.int16: "bf16", torch.uint32: "u32"}
+        if dtype is None:
+            dtype = names[t.dtype]
+        if not t.is_contiguous():
+            raise ValueError("tensor must be contiguous")
+        return self.from_device_ptr(t.data_ptr(), dtype, tuple(t.shape), keep=t)
+
+    def from_host(self, array: np.ndarray, dtype: str) -> LazyTensor:
+        a = np.ascontiguousarray(array, dtype=NP_DTYPES[dtype])
+        shp = (_i64 * max(a.ndim, 1))(*a.shape)
+        self._check(_lib.lt_tensor_from_host(self._ctx, _vp(a.ctypes.data), DTYPES[dtype], a.ndim, shp, ctypes.byref(self._h)))
+        return LazyTensor(self, self._h.value, dtype, a.shape, keep=a)
+
+    def leaf(self, array: np.ndarray, dtype: str) -> LazyTensor:
+        """Materialised input from a numpy array in storage representation (bf16 as uint16 bits)."""
+        a = np.ascontiguousarray(array, dtype=NP_DTYPES[dtype])
+        if self.device == LT_DEVICE_NONE:
+            return self.from_device_ptr(a.ctypes.data or 16, dtype, a.shape, keep=a)
+        import torch
+
+        host = torch.from_numpy(a.view(np.int16) if dtype == "bf16" else a.view(np.int32) if dtype == "u32" else a)
+        dev = host.to(f"cuda:{self.device}")
+        return self.from_device_ptr(dev.data_ptr(), dtype, a.shape, keep=dev)
+
+    def scalar(self, value: float, dtype: str = "f32", dynamic: bool = False) -> LazyTensor:
+        fn = _lib.lt_scalar_dynamic if dynamic else _lib.lt_scalar
+        self._check(fn(self._ctx, float(value), DTYPES[dtype], ctypes.byref(self._h)))
+        return LazyTensor(self, self._h.value, dtype, ())
+
+    # ---- recording
+    def op(self, name: str, *inputs, **attrs) -> LazyTensor:
+        n = len(inputs)
+        ins = (_u64 * max(n, 1))(*[t.handle for t in inputs])
+        if name == "convert":
+            a = [DTYPES[attrs["dtype"]]]
+        elif name == "iota":
+            shp = tuple(attrs["shape"])
+            a = [int(attrs["dim"]), len(shp), *shp]
+        elif name == "philox_bits":
+            shp = tuple(attrs["shape"])
+            seed, off = int(attrs["seed"]), int(attrs["offset"])
+            # 64-bit patterns travel as signed int64
+            a = [seed - (1 << 64) if seed >= (1 << 63) else seed, off - (1 << 64) if off >= (1 << 63) else off,
+                 len(shp), *shp]
+        else:
+            a = []
+        at = (_i64 * max(len(a), 1))(*a)
+        self._check(_lib.lt_op(self._ctx, OPCODES[name], ins, n, at, len(a), ctypes.byref(self._h)))
+        h = self._h.value
+        dt, rk, shp, _ = self._info(h)
+        return LazyTensor(self, h, dt, shp)
+
+    def _info(self, handle: int):
+        dt, rk, mat = _int(), _int(), _int()
+        shp = (_i64 * LT_MAX_RANK)()
+        self._check(_lib.lt_tensor_info(self._ctx, handle, ctypes.byref(dt), ctypes.byref(rk), shp, ctypes.byref(mat)))
+        return DTYPE_NAMES[dt.value], rk.value, tuple(shp[: rk.value]), bool(mat.value)
+
+    def is_materialised(self, t: LazyTensor) -> bool:
+        return self._info(t.handle)[3]
+
+    def assign(self, dst: LazyTensor, src: LazyTensor) -> None:
+        self._check(_lib.lt_assign(self._ctx, dst.handle, src.handle))
+
+    def release(self, t: LazyTensor) -> None:
+        t.ctx = None
+        self._check(_lib.lt_release(self._ctx, t.handle))
+
+    def barrier(self, blocking: bool = False) -> None:
+        self._check(_lib.lt_barrier(self._ctx, 1 if blocking else 0))
+
+    def fetch(self, t: LazyTensor) -> np.ndarray:
+        out = np.empty(t.shape, dtype=NP_DTYPES[t.dtype])
+        self._check(_lib.lt_fetch(self._ctx, t.handle, _vp(out.ctypes.data), out.nbytes))
+        return out
+
+    def fetch_into(self, t: LazyTensor, host_ptr: int, nbytes: int) -> None:
+        self._check(_lib.lt_fetch(self._ctx, t.handle, _vp(host_ptr), nbytes))
+
+    def device_ptr(self, t: LazyTensor) -> int:
+        p = _vp()
+        self._check(_lib.lt_device_ptr(self._ctx, t.handle, ctypes.byref(p)))
+        return p.value or 0
+
+    # ---- introspection
+    def stats(self) -> dict:
+        s = lt_stats()
+        self._check(_lib.lt_get_stats(self._ctx, ctypes.byref(s)))
+        return {n: getattr(s, n) for n, _ in lt_stats._fields_}
+
+    def reset_stats(self) -> None:
+        self._check(_lib.lt_reset_stats(self._ctx))
+
+    def cache_size(self) -> int:
+        n = _u64()
+        self._check(_lib.lt_cache_size(self._ctx, ctypes.byref(n)))
+        return n.value
+
+    def set_kernel_timing(self, on: bool) -> None:
+        self._check(_lib.lt_set_kernel_timing(self._ctx, 1 if on else 0))
+
+    def kernel_timing(self) -> dict:
+        t = lt_kernel_timing()
+        self._check(_lib.lt_get_kernel_timing(self._ctx, ctypes.byref(t)))
+        names = ("elementwise", "row", "multi")
+        return {n: {"launches": t.launches[i], "ms": t.ms[i], "bytes": t.bytes[i]} for i, n in enumerate(names)}
+
+    def _text(self, fn) -> str:
+        need = ctypes.c_size_t()
+        self._check(fn(self._ctx, None, 0, ctypes.byref(need)))
+        buf = ctypes.create_string_buffer(need.value)
+        self._check(fn(self._ctx, buf, need.value, ctypes.byref(need)))
+        return buf.value.decode()
+
+    def dump_ir(self) -> str:
+        return self._text(_lib.lt_dump_ir)
+
+    def dump_plan(self) -> str:
+        return self._text(_lib.lt_dump_plan)

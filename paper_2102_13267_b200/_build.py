@@ -1,0 +1,61 @@
+"""Builds liblazytensor.so (host runtime + sm_100a kernels) in-tree with nvcc and g++."""
+from __future__ import annotations
+
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+from pathlib import Path
+
+HERE = Path(__file__).resolve().parent
+CSRC = HERE / "csrc"
+OBJ = HERE / "_build"
+LIB = HERE / "liblazytensor.so"
+CUDA_HOME = Path(os.environ.get("CUDA_HOME", "/usr/local/cuda"))
+
+CU_SOURCES = ["kernels.cu"]
+CPP_SOURCES = ["engine.cpp", "canon.cpp", "planner.cpp", "executor.cpp"]
+HEADERS = ["engine.h", "vm.h", "launch.h", "../../include/lazytensor.h"]
+
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+              "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
+CXX_FLAGS = ["-O2", "-std=c++17", "-fPIC", "-Wall", "-Wno-unused-function", f"-I{CUDA_HOME}/include"]
+
+
+def _stale(target: Path, deps) -> bool:
+    if not target.exists():
+        return True
+    t = target.stat().st_mtime
+    return any(Path(d).stat().st_mtime > t for d in deps)
+
+
+def _compile(src: str) -> Path:
+    path = CSRC / src
+    obj = OBJ / (src + ".o")
+    deps = [path] + [CSRC / h for h in HEADERS]
+    if _stale(obj, deps):
+        if src.endswith(".cu"):
+            cmd = [str(CUDA_HOME / "bin" / "nvcc"), *NVCC_FLAGS, "-c", str(path), "-o", str(obj)]
+        else:
+            cmd = ["g++", *CXX_FLAGS, "-c", str(path), "-o", str(obj)]
+        subprocess.check_call(cmd)
+    return obj
+
+
+def build(force: bool = False) -> Path:
+    """Compile what changed and link the shared library; returns its path."""
+    OBJ.mkdir(exist_ok=True)
+    if force:
+        for f in OBJ.glob("*.o"):
+            f.unlink()
+    with ThreadPoolExecutor(max_workers=4) as pool:
+        objs = list(pool.map(_compile, CU_SOURCES + CPP_SOURCES))
+    if force or _stale(LIB, objs):
+        tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.check_call([str(CUDA_HOME / "bin" / "nvcc"), "-shared", "-o", str(tmp), *map(str, objs),
+                               "-gencode", "arch=compute_100a,code=sm_100a", "-cudart", "static"])
+        os.replace(tmp, LIB)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build())

@@ -1,0 +1,919 @@
+// Recorder, liveness arena and the C ABI (lazytensor.h).
+#include "engine.h"
+#include "launch.h"
+
+#include <atomic>
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <algorithm>
+
+using namespace lt;
+
+namespace {
+
+std::atomic<uint32_t> g_next_tag{1};
+
+inline uint64_t now_ns() {
+    return (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(
+               std::chrono::steady_clock::now().time_since_epoch())
+        .count();
+}
+
+struct Timer {
+    uint64_t &acc;
+    uint64_t t0;
+    explicit Timer(uint64_t &a) : acc(a), t0(now_ns()) {}
+    ~Timer() { acc += now_ns() - t0; }
+};
+
+inline lt_tensor make_handle(const lt_ctx *c, uint32_t slot) {
+    return ((uint64_t)c->tag << 48) | ((uint64_t)(c->tensors[slot].gen & 0xffffu) << 32) | (uint64_t)(slot + 1);
+}
+
+lt_status lookup(lt_ctx *c, lt_tensor h, uint32_t *slot) {
+    if ((uint16_t)(h >> 48) != c->tag) return fail(c, LT_ERR_DEVICE, "tensor handle belongs to another context");
+    uint32_t s = (uint32_t)(h & 0xffffffffu);
+    if (s == 0 || s > c->tensors.size()) return fail(c, LT_ERR_INVALID_ARG, "unknown tensor handle");
+    s -= 1;
+    const TensorRec &t = c->tensors[s];
+    if (!t.live || (t.gen & 0xffffu) != (uint32_t)((h >> 32) & 0xffffu))
+        return fail(c, LT_ERR_INVALID_ARG, "tensor handle was released");
+    *slot = s;
+    return LT_OK;
+}
+
+uint32_t tensor_new(lt_ctx *c, uint32_t node) {
+    uint32_t slot;
+    if (!c->free_tensors.empty()) {
+        slot = c->free_tensors.back();
+        c->free_tensors.pop_back();
+    } else {
+        slot = (uint32_t)c->tensors.size();
+        c->tensors.emplace_back();
+    }
+    TensorRec &t = c->tensors[slot];
+    t.node = node;
+    t.gen += 1;
+    t.donor = NONE;
+    t.seq = c->next_seq++;
+    t.live = true;
+    t.queued = false;
+    node_ref(c, node);
+    c->nodes[node].tensor_refs++;
+    return slot;
+}
+
+inline bool is_leaf(const Node &n) { return n.op == N_DEVICE_DATA || n.op == N_SCALAR; }
+
+void queue_pending(lt_ctx *c, uint32_t slot) {
+    TensorRec &t = c->tensors[slot];
+    if (!t.queued) {
+        t.queued = true;
+        c->pending.push_back(slot);
+    }
+}
+
+bool float_dtype(int dt) { return dt == LT_F32 || dt == LT_BF16; }
+
+bool valid_dtype(int dt) { return dt >= LT_F32 && dt <= LT_U32; }
+
+lt_status check_shape(lt_ctx *c, int rank, const int64_t *shape) {
+    if (rank < 0 || rank > LT_MAX_RANK) return fail(c, LT_ERR_INVALID_ARG, "rank must be between 0 and LT_MAX_RANK");
+    if (rank > 0 && !shape) return fail(c, LT_ERR_INVALID_ARG, "shape is null");
+    for (int i = 0; i < rank; ++i)
+        if (shape[i] < 0) return fail(c, LT_ERR_INVALID_ARG, "negative dimension");
+    return LT_OK;
+}
+
+// Collect the tensors a barrier must materialise (Section 4: all live tensors with
+// outstanding computation), in creation order.
+void gather_roots(lt_ctx *c, std::vector<uint32_t> &roots, bool consume) {
+    roots.clear();
+    for (uint32_t slot : c->pending) {
+        TensorRec &t = c->tensors[slot];
+        if (consume) t.queued = false;
+        if (t.live && !is_leaf(c->nodes[t.node])) roots.push_back(slot);
+    }
+    std::sort(roots.begin(), roots.end(),
+              [c](uint32_t a, uint32_t b) { return c->tensors[a].seq < c->tensors[b].seq; });
+    roots.erase(std::unique(roots.begin(), roots.end()), roots.end());
+    if (consume) {
+        c->pending.clear();
+    }
+}
+
+void release_donors(lt_ctx *c, const std::vector<uint32_t> &roots) {
+    for (uint32_t slot : roots) {
+        TensorRec &t = c->tensors[slot];
+        if (t.donor != NONE) {
+            buffer_unref(c, t.donor);
+            t.donor = NONE;
+        }
+    }
+}
+
+void put_text(const std::string &s, char *buf, size_t cap, size_t *need) {
+    if (need) *need = s.size() + 1;
+    if (buf && cap) {
+        size_t n = std::min(cap - 1, s.size());
+        memcpy(buf, s.data(), n);
+        buf[n] = 0;
+    }
+}
+
+std::string shape_text(int dtype, const int64_t *dims, int rank) {
+    std::string s = dtype_name(dtype);
+    s += "[";
+    for (int i = 0; i < rank; ++i) {
+        if (i) s += ",";
+        s += std::to_string(dims[i]);
+    }
+    s += "]";
+    return s;
+}
+
+}  // namespace
+
+namespace lt {
+
+size_t dtype_size(int dt) { return dt == LT_BF16 ? 2 : dt == LT_U8 ? 1 : 4; }
+
+const char *dtype_name(int dt) {
+    static const char *n[] = {"f32", "bf16", "u8", "i32", "u32"};
+    return dt >= 0 && dt <= 4 ? n[dt] : "?";
+}
+
+const char *op_name(int op) {
+    switch (op) {
+    case LT_OP_ADD: return "add"; case LT_OP_SUB: return "sub"; case LT_OP_MUL: return "mul";
+    case LT_OP_DIV: return "div"; case LT_OP_MAX: return "max"; case LT_OP_MIN: return "min";
+    case LT_OP_AND: return "and"; case LT_OP_OR: return "or"; case LT_OP_XOR: return "xor";
+    case LT_OP_GT: return "gt"; case LT_OP_GE: return "ge"; case LT_OP_LT: return "lt";
+    case LT_OP_LE: return "le"; case LT_OP_EQ: return "eq"; case LT_OP_NE: return "ne";
+    case LT_OP_WHERE: return "where";
+    case LT_OP_NEG: return "neg"; case LT_OP_ABS: return "abs"; case LT_OP_RELU: return "relu";
+    case LT_OP_EXP: return "exp"; case LT_OP_LOG: return "log"; case LT_OP_TANH: return "tanh";
+    case LT_OP_SQRT: return "sqrt"; case LT_OP_RSQRT: return "rsqrt"; case LT_OP_RECIP: return "recip";
+    case LT_OP_SQUARE: return "square"; case LT_OP_SIGMOID: return "sigmoid";
+    case LT_OP_GELU_TANH: return "gelu_tanh"; case LT_OP_NOT: return "not";
+    case LT_OP_CONVERT: return "convert"; case LT_OP_IOTA: return "iota";
+    case LT_OP_PHILOX_BITS: return "philox_bits";
+    case LT_OP_ROW_SUM: return "row_sum"; case LT_OP_ROW_MAX: return "row_max"; case LT_OP_ROW_MIN: return "row_min";
+    case N_DEVICE_DATA: return "device_data"; case N_SCALAR: return "constant";
+    default: return "?";
+    }
+}
+
+int64_t shape_numel(const int64_t *dims, int rank) {
+    int64_t n = 1;
+    for (int i = 0; i < rank; ++i) n *= dims[i];
+    return n;
+}
+
+lt_status fail(lt_ctx *c, lt_status s, const std::string &msg) {
+    if (c) c->error = msg;
+    return s;
+}
+
+uint32_t node_new(lt_ctx *c) {
+    uint32_t id;
+    if (!c->free_nodes.empty()) {
+        id = c->free_nodes.back();
+        c->free_nodes.pop_back();
+        c->nodes[id] = Node();
+    } else {
+        id = (uint32_t)c->nodes.size();
+        c->nodes.emplace_back();
+    }
+    return id;
+}
+
+void node_ref(lt_ctx *c, uint32_t n) { c->nodes[n].refs++; }
+
+void node_unref(lt_ctx *c, uint32_t n) {
+    // iterative: long chains (an unrolled loop, Section 4.2) must not recurse deeply
+    std::vector<uint32_t> &stack = c->stack_scratch;
+    size_t base = stack.size();
+    stack.push_back(n);
+    while (stack.size() > base) {
+        uint32_t id = stack.back();
+        stack.pop_back();
+        Node &nd = c->nodes[id];
+        if (--nd.refs > 0) continue;
+        for (int i = 0; i < nd.n_in; ++i) stack.push_back(nd.in[i]);
+        if (nd.op == N_DEVICE_DATA && nd.buffer != NONE) buffer_unref(c, nd.buffer);
+        nd.op = 0;
+        nd.n_in = 0;
+        c->free_nodes.push_back(id);
+    }
+}
+
+uint32_t buffer_new(lt_ctx *c, void *ptr, size_t bytes, bool owned) {
+    uint32_t id;
+    if (!c->free_buffers.empty()) {
+        id = c->free_buffers.back();
+        c->free_buffers.pop_back();
+    } else {
+        id = (uint32_t)c->buffers.size();
+        c->buffers.emplace_back();
+    }
+    Buffer &b = c->buffers[id];
+    b.ptr = ptr;
+    b.bytes = bytes;
+    b.refs = 1;
+    b.owned = owned;
+    return id;
+}
+
+void buffer_unref(lt_ctx *c, uint32_t b) {
+    Buffer &buf = c->buffers[b];
+    if (--buf.refs > 0) return;
+    if (buf.owned && buf.ptr) ctx_free(c, buf.ptr);
+    buf.ptr = nullptr;
+    c->free_buffers.push_back(b);
+}
+
+void *ctx_alloc(lt_ctx *c, size_t bytes) {
+    if (bytes == 0) bytes = 16;
+    if (c->has_alloc) return c->alloc.alloc(bytes, (void *)c->stream, c->alloc.user);
+    if (c->device == LT_DEVICE_NONE) return malloc(bytes);
+    void *p = nullptr;
+    if (cudaMallocAsync(&p, bytes, c->stream) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return p;
+}
+
+void ctx_free(lt_ctx *c, void *p) {
+    if (!p) return;
+    if (c->has_alloc) c->alloc.free(p, (void *)c->stream, c->alloc.user);
+    else if (c->device == LT_DEVICE_NONE) free(p);
+    else cudaFreeAsync(p, c->stream);
+}
+
+}  // namespace lt
+
+// ======================================================================= C ABI
+
+extern "C" {
+
+const char *lt_version(void) { return "lazytensor-b200 0.1"; }
+
+const char *lt_last_error(lt_ctx *ctx) { return ctx ? ctx->error.c_str() : "null context"; }
+
+lt_status lt_ctx_create(int device, void *cuda_stream, const lt_allocator *allocator, lt_ctx **out) {
+    if (!out) return LT_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (device < LT_DEVICE_NONE) return LT_ERR_INVALID_ARG;
+    lt_ctx *c = new (std::nothrow) lt_ctx();
+    if (!c) return LT_ERR_OOM;
+    c->device = device;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->tag = (uint16_t)(g_next_tag.fetch_add(1) & 0xffffu);
+    if (c->tag == 0) c->tag = (uint16_t)(g_next_tag.fetch_add(1) & 0xffffu);
+    if (allocator) {
+        if (!allocator->alloc || !allocator->free) {
+            delete c;
+            return LT_ERR_INVALID_ARG;
+        }
+        c->alloc = *allocator;
+        c->has_alloc = true;
+    }
+    auto env_opt = [](const char *name, int64_t *dst) {
+        const char *v = getenv(name);
+        if (v && *v) *dst = strtoll(v, nullptr, 10);
+    };
+    env_opt("LT_FUSION", &c->opt.fusion);
+    env_opt("LT_VERIFY", &c->opt.verify);
+    env_opt("LT_FAST_MATH", &c->opt.fast_math);
+    env_opt("LT_HORIZONTAL", &c->opt.horizontal);
+    if (device != LT_DEVICE_NONE) {
+        cudaError_t e = cudaSetDevice(device);
+        int sms = 0;
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (e == cudaSuccess) e = lt_kernel_occupancy(&c->occ_ew, &c->occ_row, &c->occ_multi);
+        if (e != cudaSuccess) {
+            // no usable device: report instead of falling back to anything
+            fprintf(stderr, "lt_ctx_create: CUDA device %d unusable: %s\n", device, cudaGetErrorString(e));
+            cudaGetLastError();
+            delete c;
+            return LT_ERR_CUDA;
+        }
+        c->sm_count = sms;
+        if (c->occ_ew < 1) c->occ_ew = 1;
+        if (c->occ_row < 1) c->occ_row = 1;
+        if (c->occ_multi < 1) c->occ_multi = 1;
+    }
+    *out = c;
+    return LT_OK;
+}
+
+lt_status lt_ctx_destroy(lt_ctx *c) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    if (c->device != LT_DEVICE_NONE) cudaStreamSynchronize(c->stream);
+    for (auto &t : c->timed) {
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+    }
+    for (auto e : c->event_pool) cudaEventDestroy(e);
+    for (auto &b : c->buffers)
+        if (b.owned && b.ptr && b.refs > 0) ctx_free(c, b.ptr);
+    delete c;
+    return LT_OK;
+}
+
+lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
+    if (!c || !key) return LT_ERR_INVALID_ARG;
+    if (!strcmp(key, "fusion")) c->opt.fusion = value;
+    else if (!strcmp(key, "verify")) c->opt.verify = value;
+    else if (!strcmp(key, "fast_math")) c->opt.fast_math = value;
+    else if (!strcmp(key, "horizontal")) c->opt.horizontal = value;
+    else if (!strcmp(key, "cache_capacity")) c->opt.cache_capacity = value;
+    else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
+    return LT_OK;
+}
+
+static lt_status new_device_tensor(lt_ctx *c, void *dptr, bool owned, lt_dtype dtype, int rank, const int64_t *shape,
+                                   lt_tensor *out) {
+    size_t bytes = (size_t)shape_numel(shape, rank) * dtype_size(dtype);
+    uint32_t n = node_new(c);
+    Node &nd = c->nodes[n];
+    nd.op = N_DEVICE_DATA;
+    nd.dtype = (uint8_t)dtype;
+    nd.rank = (uint8_t)rank;
+    for (int i = 0; i < rank; ++i) nd.dims[i] = shape[i];
+    nd.buffer = buffer_new(c, dptr, bytes, owned);
+    uint32_t slot = tensor_new(c, n);
+    *out = make_handle(c, slot);
+    return LT_OK;
+}
+
+lt_status lt_tensor_from_device(lt_ctx *c, void *dptr, lt_dtype dtype, int rank, const int64_t *shape,
+                                lt_tensor *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    Timer tm(c->stats.ns_record);
+    if (!valid_dtype(dtype)) return fail(c, LT_ERR_DTYPE, "unknown dtype");
+    lt_status s = check_shape(c, rank, shape);
+    if (s) return s;
+    if (!dptr && shape_numel(shape, rank) > 0) return fail(c, LT_ERR_INVALID_ARG, "device pointer is null");
+    c->stats.nodes_recorded++;
+    return new_device_tensor(c, dptr, false, dtype, rank, shape, out);
+}
+
+lt_status lt_tensor_from_host(lt_ctx *c, const void *hptr, lt_dtype dtype, int rank, const int64_t *shape,
+                              lt_tensor *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return fail(c, LT_ERR_DTYPE, "unknown dtype");
+    lt_status s = check_shape(c, rank, shape);
+    if (s) return s;
+    if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    size_t bytes = (size_t)shape_numel(shape, rank) * dtype_size(dtype);
+    if (!hptr && bytes) return fail(c, LT_ERR_INVALID_ARG, "host pointer is null");
+    void *d = ctx_alloc(c, bytes);
+    if (!d) return fail(c, LT_ERR_OOM, "allocator returned null");
+    if (bytes) {
+        cudaError_t e = cudaMemcpyAsync(d, hptr, bytes, cudaMemcpyHostToDevice, c->stream);
+        if (e != cudaSuccess) {
+            ctx_free(c, d);
+            return fail(c, LT_ERR_CUDA, std::string("cudaMemcpyAsync: ") + cudaGetErrorString(e));
+        }
+    }
+    c->stats.nodes_recorded++;
+    return new_device_tensor(c, d, true, dtype, rank, shape, out);
+}
+
+static lt_status new_scalar(lt_ctx *c, double value, lt_dtype dtype, bool force_dynamic, lt_tensor *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    Timer tm(c->stats.ns_record);
+    if (!valid_dtype(dtype)) return fail(c, LT_ERR_DTYPE, "unknown dtype");
+    uint32_t n = node_new(c);
+    Node &nd = c->nodes[n];
+    nd.op = N_SCALAR;
+    nd.dtype = (uint8_t)dtype;
+    nd.rank = 0;
+    nd.sval = value;
+    // Section 4.1 heuristic: only 0 and 1 are baked into the graph
+    uint64_t bits;
+    memcpy(&bits, &value, 8);
+    bool special = bits == 0ull || value == 1.0;
+    if (force_dynamic || !special) nd.flags |= NF_DYNAMIC;
+    c->stats.nodes_recorded++;
+    uint32_t slot = tensor_new(c, n);
+    *out = make_handle(c, slot);
+    return LT_OK;
+}
+
+lt_status lt_scalar(lt_ctx *c, double value, lt_dtype dtype, lt_tensor *out) {
+    return new_scalar(c, value, dtype, false, out);
+}
+
+lt_status lt_scalar_dynamic(lt_ctx *c, double value, lt_dtype dtype, lt_tensor *out) {
+    return new_scalar(c, value, dtype, true, out);
+}
+
+// class of operand shape relative to the result shape: 0 same, 1 scalar, 2 column vector, 3 row scalar, -1 none
+static int operand_class(const Node &a, const int64_t *od, int orank) {
+    int64_t na = shape_numel(a.dims, a.rank);
+    bool same = a.rank == orank;
+    for (int i = 0; same && i < orank; ++i) same = a.dims[i] == od[i];
+    if (same) return 0;
+    if (na == 1) return 1;
+    if (orank >= 1 && a.rank >= 1 && a.rank <= orank && a.dims[a.rank - 1] == od[orank - 1]) {
+        bool ones = true;
+        for (int i = 0; i + 1 < a.rank; ++i) ones = ones && a.dims[i] == 1;
+        if (ones) return 2;
+    }
+    if (a.rank == orank && orank >= 1 && a.dims[orank - 1] == 1) {
+        bool lead = true;
+        for (int i = 0; i + 1 < orank; ++i) lead = lead && a.dims[i] == od[i];
+        if (lead) return 3;
+    }
+    return -1;
+}
+
+// result shape of broadcasting the operands against each other (dimensions aligned at the right)
+static bool broadcast_shape(const Node *const *ops, int n, int64_t *od, int *orank) {
+    int r = 0;
+    for (int k = 0; k < n; ++k) r = std::max(r, (int)ops[k]->rank);
+    for (int i = 0; i < r; ++i) od[i] = 1;
+    for (int k = 0; k < n; ++k) {
+        const Node &a = *ops[k];
+        for (int i = 0; i < a.rank; ++i) {
+            int o = r - a.rank + i;
+            if (a.dims[i] == 1) continue;
+            if (od[o] == 1) od[o] = a.dims[i];
+            else if (od[o] != a.dims[i]) return false;
+        }
+    }
+    *orank = r;
+    return true;
+}
+
+static bool scalar_fits(const Node &s, int dtype) {
+    if (s.op != N_SCALAR) return true;
+    if (float_dtype(dtype)) return true;
+    double v = s.sval;
+    if (v != std::floor(v)) return false;
+    if (dtype == LT_U8) return v >= 0 && v <= 255;
+    if (dtype == LT_I32) return v >= -2147483648.0 && v <= 2147483647.0;
+    return v >= 0 && v <= 4294967295.0;
+}
+
+lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int64_t *attrs, int n_attrs,
+                lt_tensor *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    Timer tm(c->stats.ns_record);
+    if (n_in < 0 || n_in > 3 || (n_in > 0 && !in) || n_attrs < 0 || (n_attrs > 0 && !attrs))
+        return fail(c, LT_ERR_INVALID_ARG, "bad operand or attribute list");
+    uint32_t ids[3] = {NONE, NONE, NONE};
+    for (int i = 0; i < n_in; ++i) {
+        uint32_t slot;
+        lt_status s = lookup(c, in[i], &slot);
+        if (s) return s;
+        ids[i] = c->tensors[slot].node;
+    }
+    const Node *ops[3] = {nullptr, nullptr, nullptr};
+    for (int i = 0; i < n_in; ++i) ops[i] = &c->nodes[ids[i]];
+
+    int64_t od[LT_MAX_RANK] = {0};
+    int orank = 0;
+    int odtype = LT_F32;
+    int64_t a0 = 0, a1 = 0;
+
+    auto common_dtype = [&](int first, int count, int *dt) -> bool {
+        int found = -1;
+        for (int i = first; i < first + count; ++i)
+            if (ops[i]->op != N_SCALAR) {
+                if (found >= 0 && ops[i]->dtype != found) return false;
+                found = ops[i]->dtype;
+            }
+        if (found < 0) found = ops[first]->dtype;
+        for (int i = first; i < first + count; ++i)
+            if (!scalar_fits(*ops[i], found)) return false;
+        *dt = found;
+        return true;
+    };
+    auto check_classes = [&](int count) -> bool {
+        for (int i = 0; i < count; ++i)
+            if (operand_class(*ops[i], od, orank) < 0) return false;
+        return true;
+    };
+
+    const bool is_binary = opcode >= LT_OP_ADD && opcode <= LT_OP_XOR;
+    const bool is_compare = opcode >= LT_OP_GT && opcode <= LT_OP_NE;
+    const bool is_unary = opcode >= LT_OP_NEG && opcode <= LT_OP_NOT;
+    const bool is_reduce = opcode >= LT_OP_ROW_SUM && opcode <= LT_OP_ROW_MIN;
+
+    if (is_binary || is_compare) {
+        if (n_in != 2) return fail(c, LT_ERR_INVALID_ARG, "binary op takes 2 inputs");
+        int dt;
+        if (!common_dtype(0, 2, &dt)) return fail(c, LT_ERR_DTYPE, "operands must share one dtype");
+        if (!broadcast_shape(ops, 2, od, &orank) || !check_classes(2))
+            return fail(c, LT_ERR_SHAPE, "operand shapes are not a supported broadcast");
+        if (is_binary) {
+            bool ok;
+            if (float_dtype(dt)) ok = opcode <= LT_OP_MIN;
+            else if (dt == LT_U8) ok = opcode >= LT_OP_AND;
+            else ok = opcode != LT_OP_DIV;
+            if (!ok) return fail(c, LT_ERR_DTYPE, std::string(op_name(opcode)) + " is not defined for " + dtype_name(dt));
+            odtype = dt;
+        } else {
+            odtype = LT_U8;
+        }
+    } else if (opcode == LT_OP_WHERE) {
+        if (n_in != 3) return fail(c, LT_ERR_INVALID_ARG, "where takes 3 inputs");
+        if (ops[0]->dtype != LT_U8 || ops[0]->op == N_SCALAR) return fail(c, LT_ERR_DTYPE, "where mask must be a u8 tensor");
+        int dt;
+        if (!common_dtype(1, 2, &dt)) return fail(c, LT_ERR_DTYPE, "where branches must share one dtype");
+        if (!broadcast_shape(ops, 3, od, &orank) || !check_classes(3))
+            return fail(c, LT_ERR_SHAPE, "operand shapes are not a supported broadcast");
+        odtype = dt;
+    } else if (is_unary) {
+        if (n_in != 1) return fail(c, LT_ERR_INVALID_ARG, "unary op takes 1 input");
+        int dt = ops[0]->dtype;
+        bool ok;
+        if (opcode == LT_OP_NOT) ok = dt == LT_U8;
+        else if (dt == LT_I32) ok = opcode == LT_OP_NEG || opcode == LT_OP_ABS;
+        else ok = float_dtype(dt);
+        if (!ok) return fail(c, LT_ERR_DTYPE, std::string(op_name(opcode)) + " is not defined for " + dtype_name(dt));
+        orank = ops[0]->rank;
+        memcpy(od, ops[0]->dims, sizeof(od));
+        odtype = dt;
+    } else if (opcode == LT_OP_CONVERT) {
+        if (n_in != 1 || n_attrs != 1) return fail(c, LT_ERR_INVALID_ARG, "convert takes 1 input and attrs {dtype}");
+        int si = ops[0]->dtype, so = (int)attrs[0];
+        if (!valid_dtype(so)) return fail(c, LT_ERR_DTYPE, "unknown target dtype");
+        bool ok = (float_dtype(si) && float_dtype(so)) || (so == LT_F32 && !float_dtype(si)) ||
+                  (si == LT_F32 && so == LT_I32) || (si == LT_U8 && (so == LT_I32 || so == LT_U32)) ||
+                  ((si == LT_I32 || si == LT_U32) && (so == LT_I32 || so == LT_U32)) ||
+                  (so == LT_U8 && si != LT_BF16);
+        if (!ok) return fail(c, LT_ERR_DTYPE, std::string("convert ") + dtype_name(si) + " -> " + dtype_name(so) + " is not defined");
+        orank = ops[0]->rank;
+        memcpy(od, ops[0]->dims, sizeof(od));
+        odtype = so;
+        a0 = so;
+    } else if (opcode == LT_OP_IOTA || opcode == LT_OP_PHILOX_BITS) {
+        const int head = opcode == LT_OP_IOTA ? 1 : 2;
+        if (n_in != 0 || n_attrs < head + 1) return fail(c, LT_ERR_INVALID_ARG, "factory op takes no inputs and attrs {.., rank, dims}");
+        int r = (int)attrs[head];
+        if (r < 1 || r > LT_MAX_RANK || n_attrs != head + 1 + r) return fail(c, LT_ERR_INVALID_ARG, "bad rank in attrs");
+        lt_status s = check_shape(c, r, attrs + head + 1);
+        if (s) return s;
+        orank = r;
+        for (int i = 0; i < r; ++i) od[i] = attrs[head + 1 + i];
+        if (opcode == LT_OP_IOTA) {
+            if (attrs[0] < 0 || attrs[0] >= r) return fail(c, LT_ERR_INVALID_ARG, "iota dim out of range");
+            if (od[attrs[0]] > 2147483647LL) return fail(c, LT_ERR_UNSUPPORTED, "iota extent exceeds int32");
+            odtype = LT_I32;
+            a0 = attrs[0];
+        } else {
+            odtype = LT_U32;
+            a0 = attrs[0];
+            a1 = attrs[1];
+        }
+    } else if (is_reduce) {
+        if (n_in != 1) return fail(c, LT_ERR_INVALID_ARG, "reduction takes 1 input");
+        if (!float_dtype(ops[0]->dtype)) return fail(c, LT_ERR_DTYPE, "row reductions need a float dtype");
+        if (ops[0]->rank < 1) return fail(c, LT_ERR_SHAPE, "row reduction needs rank >= 1");
+        if (ops[0]->dims[ops[0]->rank - 1] > (int64_t)LT_VM_V * 1024)
+            return fail(c, LT_ERR_UNSUPPORTED, "row reductions support rows of at most 8192 elements");
+        orank = ops[0]->rank;
+        memcpy(od, ops[0]->dims, sizeof(od));
+        od[orank - 1] = 1;
+        odtype = ops[0]->dtype;
+    } else {
+        return fail(c, LT_ERR_UNSUPPORTED, "unknown opcode " + std::to_string(opcode));
+    }
+
+    uint32_t n = node_new(c);  // may grow the arena: `ops` pointers are dead from here on
+    Node &nd = c->nodes[n];
+    nd.op = (uint16_t)opcode;
+    nd.dtype = (uint8_t)odtype;
+    nd.rank = (uint8_t)orank;
+    nd.n_in = (uint8_t)n_in;
+    for (int i = 0; i < orank; ++i) nd.dims[i] = od[i];
+    nd.attr[0] = a0;
+    nd.attr[1] = a1;
+    for (int i = 0; i < n_in; ++i) {
+        nd.in[i] = ids[i];
+        node_ref(c, ids[i]);
+    }
+    c->stats.nodes_recorded++;
+    uint32_t slot = tensor_new(c, n);
+    queue_pending(c, slot);
+    *out = make_handle(c, slot);
+    return LT_OK;
+}
+
+lt_status lt_assign(lt_ctx *c, lt_tensor dst, lt_tensor src) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    Timer tm(c->stats.ns_record);
+    uint32_t ds, ss;
+    lt_status s = lookup(c, dst, &ds);
+    if (s) return s;
+    s = lookup(c, src, &ss);
+    if (s) return s;
+    TensorRec &d = c->tensors[ds];
+    const TensorRec &sr = c->tensors[ss];
+    if (d.node == sr.node) return LT_OK;
+    const Node &dn = c->nodes[d.node];
+    const Node &sn = c->nodes[sr.node];
+    bool same = dn.dtype == sn.dtype && dn.rank == sn.rank;
+    for (int i = 0; same && i < dn.rank; ++i) same = dn.dims[i] == sn.dims[i];
+    if (!same) return fail(c, LT_ERR_SHAPE, "lt_assign needs equal shape and dtype");
+    // Section 4.3: the destination's computation is replaced by the source's; the buffer it
+    // named is remembered so the barrier can write the new value in place.
+    if (dn.op == N_DEVICE_DATA && dn.buffer != NONE) {
+        if (d.donor != NONE) buffer_unref(c, d.donor);
+        d.donor = dn.buffer;
+        c->buffers[d.donor].refs++;
+    }
+    uint32_t old = d.node;
+    d.node = sr.node;
+    node_ref(c, d.node);
+    c->nodes[d.node].tensor_refs++;
+    c->nodes[old].tensor_refs--;
+    node_unref(c, old);
+    queue_pending(c, ds);
+    return LT_OK;
+}
+
+lt_status lt_release(lt_ctx *c, lt_tensor t) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    Timer tm(c->stats.ns_record);
+    uint32_t slot;
+    lt_status s = lookup(c, t, &slot);
+    if (s) return s;
+    TensorRec &tr = c->tensors[slot];
+    tr.live = false;
+    tr.queued = false;
+    if (tr.donor != NONE) {
+        buffer_unref(c, tr.donor);
+        tr.donor = NONE;
+    }
+    c->nodes[tr.node].tensor_refs--;
+    node_unref(c, tr.node);
+    tr.node = NONE;
+    c->free_tensors.push_back(slot);
+    return LT_OK;
+}
+
+lt_status lt_barrier(lt_ctx *c, int blocking) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    std::vector<uint32_t> &roots = c->roots_scratch;
+    Canonical &cg = c->canon;
+    {
+        Timer tm(c->stats.ns_canonicalise);
+        gather_roots(c, roots, false);
+        if (!roots.empty()) canonicalise(c, roots, cg);
+    }
+    if (roots.empty()) {
+        gather_roots(c, roots, true);
+        if (blocking && c->device != LT_DEVICE_NONE) {
+            cudaError_t e = cudaStreamSynchronize(c->stream);
+            if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
+        }
+        return LT_OK;
+    }
+    c->stats.barriers++;
+    Plan *plan = nullptr;
+    {
+        Timer tm(c->stats.ns_hash_lookup);
+        hash_bytes(cg.bytes.data(), cg.bytes.size(), cg.hash);
+        HashKey key{{cg.hash[0], cg.hash[1]}};
+        auto it = c->cache.find(key);
+        if (it != c->cache.end()) {
+            Plan *p = it->second.get();
+            if (!c->opt.verify ||
+                (p->canon_bytes.size() == cg.bytes.size() && !memcmp(p->canon_bytes.data(), cg.bytes.data(), cg.bytes.size())))
+                plan = p;
+            else
+                c->cache.erase(it);  // a colliding entry: replace it below
+        }
+    }
+    if (plan) {
+        c->stats.cache_hits++;
+    } else {
+        Timer tm(c->stats.ns_plan);
+        std::unique_ptr<Plan> np(new Plan());
+        lt_status s = build_plan(c, cg, *np);
+        if (s) return s;  // pending graph untouched
+        np->hash[0] = cg.hash[0];
+        np->hash[1] = cg.hash[1];
+        np->canon_bytes = cg.bytes;
+        c->stats.compiles++;
+        if (c->opt.cache_capacity > 0 && (int64_t)c->cache.size() >= c->opt.cache_capacity) {
+            auto victim = c->cache.begin();
+            for (auto it = c->cache.begin(); it != c->cache.end(); ++it)
+                if (it->second->last_used < victim->second->last_used) victim = it;
+            if (c->last_plan == victim->second.get()) {
+                c->last_plan_text = describe_plan(*c->last_plan);
+                c->last_plan = nullptr;
+            }
+            c->cache.erase(victim);
+        }
+        plan = np.get();
+        c->cache[HashKey{{cg.hash[0], cg.hash[1]}}] = std::move(np);
+    }
+    plan->last_used = ++c->use_clock;
+    c->last_plan = plan;
+    {
+        Timer tm(c->stats.ns_bind_launch);
+        lt_status s = execute_plan(c, *plan, cg);
+        if (s) return s;  // nothing was rebound: the graph can be flushed again
+    }
+    {
+        Timer tm(c->stats.ns_rebind);
+        // Roots become device-data leaves over their output buffers; the IR behind them is dropped.
+        const size_t n_out = cg.outputs.size();
+        std::vector<uint32_t> new_nodes(n_out);
+        for (size_t k = 0; k < n_out; ++k) {
+            const OutputPlan &op = plan->outputs[k];
+            uint32_t n = node_new(c);
+            Node &nd = c->nodes[n];
+            nd.op = N_DEVICE_DATA;
+            nd.dtype = op.dtype;
+            nd.rank = op.rank;
+            memcpy(nd.dims, op.dims, sizeof(nd.dims));
+            if (op.donated_param >= 0) {
+                uint32_t b = c->nodes[cg.param_node[op.donated_param]].buffer;
+                c->buffers[b].refs++;
+                nd.buffer = b;
+            } else {
+                nd.buffer = buffer_new(c, c->out_ptr[k], op.bytes, true);
+            }
+            nd.refs = 1;  // held by this loop until the tensors are repointed
+            new_nodes[k] = n;
+        }
+        gather_roots(c, roots, true);
+        for (uint32_t slot : roots) {
+            TensorRec &t = c->tensors[slot];
+            const Node &old = c->nodes[t.node];
+            int32_t k = cg.nodes[old.canon].output;
+            uint32_t nn = new_nodes[k];
+            uint32_t old_id = t.node;
+            t.node = nn;
+            node_ref(c, nn);
+            c->nodes[nn].tensor_refs++;
+            c->nodes[old_id].tensor_refs--;
+            node_unref(c, old_id);
+        }
+        release_donors(c, roots);
+        for (uint32_t n : new_nodes) node_unref(c, n);
+    }
+    if (blocking && c->device != LT_DEVICE_NONE) {
+        cudaError_t e = cudaStreamSynchronize(c->stream);
+        if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
+    }
+    return LT_OK;
+}
+
+lt_status lt_fetch(lt_ctx *c, lt_tensor t, void *host_dst, size_t nbytes) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    uint32_t slot;
+    lt_status s = lookup(c, t, &slot);
+    if (s) return s;
+    if (!host_dst && nbytes) return fail(c, LT_ERR_INVALID_ARG, "host destination is null");
+    if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    if (!is_leaf(c->nodes[c->tensors[slot].node])) {
+        s = lt_barrier(c, 1);
+        if (s) return s;
+    }
+    const Node &nd = c->nodes[c->tensors[slot].node];
+    size_t bytes = (size_t)shape_numel(nd.dims, nd.rank) * dtype_size(nd.dtype);
+    if (nbytes != bytes) return fail(c, LT_ERR_INVALID_ARG, "nbytes does not match the tensor size");
+    if (nd.op == N_SCALAR) {
+        double v = nd.sval;
+        if (nd.dtype == LT_F32) { float f = (float)v; memcpy(host_dst, &f, 4); }
+        else if (nd.dtype == LT_BF16) {
+            float f = (float)v; uint32_t u; memcpy(&u, &f, 4);
+            if ((u & 0x7fffffffu) > 0x7f800000u) u = (u >> 16) | 0x40u; else u = (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+            uint16_t h = (uint16_t)u; memcpy(host_dst, &h, 2);
+        } else if (nd.dtype == LT_U8) { uint8_t b = (uint8_t)v; memcpy(host_dst, &b, 1); }
+        else if (nd.dtype == LT_I32) { int32_t i = (int32_t)v; memcpy(host_dst, &i, 4); }
+        else { uint32_t u = (uint32_t)v; memcpy(host_dst, &u, 4); }
+        return LT_OK;
+    }
+    cudaError_t e = cudaMemcpyAsync(host_dst, c->buffers[nd.buffer].ptr, bytes, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("device to host copy: ") + cudaGetErrorString(e));
+    return LT_OK;
+}
+
+lt_status lt_device_ptr(lt_ctx *c, lt_tensor t, void **dptr) {
+    if (!c || !dptr) return LT_ERR_INVALID_ARG;
+    uint32_t slot;
+    lt_status s = lookup(c, t, &slot);
+    if (s) return s;
+    const Node &nd = c->nodes[c->tensors[slot].node];
+    if (nd.op != N_DEVICE_DATA) return fail(c, LT_ERR_INVALID_ARG, "tensor is not materialised");
+    *dptr = c->buffers[nd.buffer].ptr;
+    return LT_OK;
+}
+
+lt_status lt_tensor_info(lt_ctx *c, lt_tensor t, int *dtype, int *rank, int64_t *shape, int *materialised) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    uint32_t slot;
+    lt_status s = lookup(c, t, &slot);
+    if (s) return s;
+    const Node &nd = c->nodes[c->tensors[slot].node];
+    if (dtype) *dtype = nd.dtype;
+    if (rank) *rank = nd.rank;
+    if (shape) for (int i = 0; i < nd.rank; ++i) shape[i] = nd.dims[i];
+    if (materialised) *materialised = nd.op == N_DEVICE_DATA;
+    return LT_OK;
+}
+
+lt_status lt_get_stats(lt_ctx *c, lt_stats *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    *out = c->stats;
+    return LT_OK;
+}
+
+lt_status lt_reset_stats(lt_ctx *c) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    c->stats = lt_stats{};
+    return LT_OK;
+}
+
+lt_status lt_cache_size(lt_ctx *c, uint64_t *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    *out = c->cache.size();
+    return LT_OK;
+}
+
+lt_status lt_set_kernel_timing(lt_ctx *c, int enable) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    c->timing = enable != 0;
+    return LT_OK;
+}
+
+lt_status lt_get_kernel_timing(lt_ctx *c, lt_kernel_timing *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
+    for (auto &t : c->timed) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.start, t.stop) == cudaSuccess) {
+            out->launches[t.kind]++;
+            out->ms[t.kind] += ms;
+            out->bytes[t.kind] += t.bytes;
+        }
+        c->event_pool.push_back(t.start);
+        c->event_pool.push_back(t.stop);
+    }
+    c->timed.clear();
+    return LT_OK;
+}
+
+lt_status lt_dump_ir(lt_ctx *c, char *buf, size_t cap, size_t *need) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    std::vector<uint32_t> roots;
+    gather_roots(c, roots, false);
+    std::string s = "IR {\n";
+    if (!roots.empty()) {
+        Canonical cg;
+        canonicalise(c, roots, cg);
+        for (size_t i = 0; i < cg.nodes.size(); ++i) {
+            const CNode &n = cg.nodes[i];
+            s += "    %" + std::to_string(i) + " = " + shape_text(n.dtype, n.dims, n.rank) + " lt::";
+            if (n.op == N_SCALAR && n.dyn >= 0) s += "scalar_data";
+            else s += op_name(n.op);
+            s += "(";
+            for (int k = 0; k < n.n_in; ++k) {
+                if (k) s += ", ";
+                s += "%" + std::to_string(n.in[k]);
+            }
+            s += ")";
+            if (n.op == N_DEVICE_DATA) s += ", device=" + (c->device == LT_DEVICE_NONE ? std::string("NONE") : "CUDA:" + std::to_string(c->device));
+            if (n.op == N_SCALAR && n.dyn < 0) {
+                char tmp[32];
+                snprintf(tmp, sizeof(tmp), "%g", n.sval);
+                s += std::string(", value=") + tmp;
+            }
+            if (n.op == LT_OP_CONVERT) s += std::string(", dtype=") + dtype_name((int)n.attr0);
+            if (n.op == LT_OP_IOTA) s += ", dim=" + std::to_string(n.attr0);
+            if (n.output >= 0) s += ", ROOT=" + std::to_string(n.output);
+            s += "\n";
+        }
+    }
+    s += "}\n";
+    put_text(s, buf, cap, need);
+    return LT_OK;
+}
+
+lt_status lt_dump_plan(lt_ctx *c, char *buf, size_t cap, size_t *need) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    std::string s = c->last_plan ? describe_plan(*c->last_plan) : c->last_plan_text;
+    put_text(s, buf, cap, need);
+    return LT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,236 @@
+// Host-side data structures: IR arena (recorder), canonical program, plans and the context.
+#pragma once
+#include <cuda_runtime_api.h>
+#include <stdint.h>
+
+#include <memory>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/lazytensor.h"
+#include "vm.h"
+
+namespace lt {
+
+constexpr uint16_t N_DEVICE_DATA = 200;  // leaf over a device buffer (Fig. 1: xla::device_data)
+constexpr uint16_t N_SCALAR = 201;       // rank-0 constant (Fig. 1: prim::Constant)
+constexpr uint32_t NONE = 0xffffffffu;
+
+enum : uint8_t { NF_DYNAMIC = 1 };  // scalar is a run-time parameter (not 0/1, or forced)
+
+// One IR node.  Nodes live in a flat arena and name operands by 32-bit index; shape and
+// dtype are recorded on every node (Section 4.1).
+struct Node {
+    uint16_t op = 0;
+    uint8_t dtype = 0, rank = 0;
+    uint8_t n_in = 0, flags = 0;
+    uint32_t in[3] = {NONE, NONE, NONE};
+    uint32_t refs = 0;         // tensors + consumer nodes holding this node
+    uint32_t tensor_refs = 0;  // tensors only
+    uint32_t buffer = NONE;    // N_DEVICE_DATA
+    uint32_t visit = 0;        // traversal stamp
+    uint32_t canon = 0;        // canonical index within the current traversal
+    int64_t dims[LT_MAX_RANK] = {0};
+    double sval = 0.0;         // N_SCALAR value
+    int64_t attr[2] = {0, 0};  // CONVERT: dtype; IOTA: dim; PHILOX: seed, offset
+};
+
+struct Buffer {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+    uint32_t refs = 0;
+    bool owned = false;
+};
+
+struct TensorRec {
+    uint32_t node = NONE;
+    uint32_t gen = 0;
+    uint32_t donor = NONE;  // buffer the tensor named before lt_assign, kept for donation
+    uint64_t seq = 0;       // creation order
+    bool live = false;
+    bool queued = false;    // already in the pending list
+};
+
+// ---------------------------------------------------------------- canonical form
+struct CNode {
+    uint16_t op;
+    uint8_t dtype, rank, n_in;
+    uint32_t in[3];
+    int64_t dims[LT_MAX_RANK];
+    int32_t param;   // N_DEVICE_DATA: parameter ordinal
+    int32_t dyn;     // first run-time slot (scalar: 1 slot; philox: 2 slots), else -1
+    double sval;     // static scalar value
+    int64_t attr0;   // CONVERT dtype / IOTA dim
+    int32_t output;  // index in the output list, else -1
+    uint32_t arena;  // arena node (not part of the hashed bytes)
+};
+
+union DynValue {
+    double d;
+    int64_t i;
+};
+
+struct Canonical {
+    std::vector<CNode> nodes;
+    std::vector<uint32_t> outputs;        // canonical index of each output node
+    std::vector<int32_t> donor_param;     // per output: parameter ordinal whose buffer may be donated, or -1
+    std::vector<uint32_t> param_node;     // per parameter: arena node (device-data leaf)
+    std::vector<DynValue> dyn;            // run-time values of this trace
+    std::vector<uint8_t> bytes;           // serialised form that is hashed and compared
+    uint64_t hash[2] = {0, 0};
+};
+
+// -------------------------------------------------------------------------- plan
+enum : uint8_t { ENC_F32 = 0, ENC_BF16 = 1, ENC_U8 = 2, ENC_I32 = 3, ENC_U32 = 4, ENC_LO32 = 5, ENC_HI32 = 6 };
+
+struct Imm {
+    int32_t dyn;    // run-time slot, or -1 for a static value
+    double sval;    // static value (ENC_I32/U32 static values are integral)
+    uint8_t enc;
+    bool operator==(const Imm &o) const { return dyn == o.dyn && enc == o.enc && (dyn >= 0 || sval == o.sval); }
+};
+
+enum : uint8_t { IO_PARAM = 0, IO_OUTPUT = 1, IO_TEMP = 2 };
+
+struct IoRef {
+    uint8_t kind;
+    uint8_t is_store;
+    uint8_t dtype;
+    uint8_t cls;
+    uint32_t index;   // parameter ordinal / output index / temporary index
+    uint32_t cnode;   // canonical node the slot carries
+};
+
+enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2 };
+
+struct Group {
+    uint8_t kind = K_EW;
+    bool fast = false;
+    bool rowcol = false;
+    uint64_t rows = 1, cols = 1;
+    std::vector<uint32_t> members;  // native members (canonical indices), topological order
+    std::vector<LtIns> ins;
+    std::vector<IoRef> io;
+    std::vector<Imm> imms;
+    uint64_t bytes = 0;
+};
+
+struct Launch {
+    uint8_t kind = K_EW;
+    bool fast = false;
+    std::vector<uint32_t> groups;   // one group, or the instances of a multi-tensor launch
+    uint64_t bytes = 0;
+    unsigned threads = LT_EW_THREADS;
+    std::unique_ptr<LtKParams> kp;       // K_EW / K_ROW parameter block (static parts prefilled)
+    std::unique_ptr<LtMultiParams> mp;   // K_MULTI
+};
+
+struct OutputPlan {
+    uint8_t dtype, rank;
+    int64_t dims[LT_MAX_RANK];
+    size_t bytes;
+    int32_t donated_param;  // parameter ordinal whose buffer receives this output, or -1
+};
+
+struct Plan {
+    uint64_t hash[2];
+    std::vector<uint8_t> canon_bytes;
+    uint32_t n_params = 0, n_dyn = 0;
+    std::vector<OutputPlan> outputs;
+    std::vector<size_t> temp_bytes;
+    std::vector<Group> groups;
+    std::vector<Launch> launches;
+    uint64_t last_used = 0;
+};
+
+struct Options {
+    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0;
+};
+
+struct HashKey {
+    uint64_t h[2];
+    bool operator==(const HashKey &o) const { return h[0] == o.h[0] && h[1] == o.h[1]; }
+};
+struct HashKeyHasher {
+    size_t operator()(const HashKey &k) const { return (size_t)(k.h[0] ^ (k.h[1] * 0x9E3779B97F4A7C15ull)); }
+};
+
+struct TimedLaunch {
+    cudaEvent_t start, stop;
+    uint8_t kind;
+    uint64_t bytes;
+};
+
+}  // namespace lt
+
+struct lt_ctx {
+    int device = LT_DEVICE_NONE;
+    cudaStream_t stream = nullptr;
+    lt_allocator alloc{};
+    bool has_alloc = false;
+    uint16_t tag = 0;
+    int sm_count = 148;
+    int occ_ew = 2, occ_row = 2, occ_multi = 2;
+
+    std::vector<lt::Node> nodes;
+    std::vector<uint32_t> free_nodes;
+    std::vector<lt::Buffer> buffers;
+    std::vector<uint32_t> free_buffers;
+    std::vector<lt::TensorRec> tensors;
+    std::vector<uint32_t> free_tensors;
+    std::vector<uint32_t> pending;  // tensor slots that may have pending IR
+    uint64_t next_seq = 1;
+    uint32_t stamp = 0;
+
+    lt::Options opt;
+    lt_stats stats{};
+    std::unordered_map<lt::HashKey, std::unique_ptr<lt::Plan>, lt::HashKeyHasher> cache;
+    uint64_t use_clock = 0;
+    lt::Plan *last_plan = nullptr;
+    std::string last_plan_text;  // dump of a plan that has since been evicted
+    std::string error;
+
+    bool timing = false;
+    std::vector<lt::TimedLaunch> timed;
+    std::vector<cudaEvent_t> event_pool;
+
+    // scratch reused across barriers
+    lt::Canonical canon;
+    std::vector<uint32_t> roots_scratch, stack_scratch;
+    std::vector<void *> param_ptr, out_ptr, temp_ptr;
+    std::vector<uint32_t> buf_stamp;
+    std::vector<int32_t> buf_param;
+    std::vector<uint8_t> param_taken;
+};
+
+namespace lt {
+
+// recorder (engine.cpp)
+uint32_t node_new(lt_ctx *c);
+void node_ref(lt_ctx *c, uint32_t n);
+void node_unref(lt_ctx *c, uint32_t n);
+uint32_t buffer_new(lt_ctx *c, void *ptr, size_t bytes, bool owned);
+void buffer_unref(lt_ctx *c, uint32_t b);
+size_t dtype_size(int dt);
+const char *dtype_name(int dt);
+const char *op_name(int op);
+int64_t shape_numel(const int64_t *dims, int rank);
+lt_status fail(lt_ctx *c, lt_status s, const std::string &msg);
+void *ctx_alloc(lt_ctx *c, size_t bytes);
+void ctx_free(lt_ctx *c, void *p);
+
+// canonicaliser (canon.cpp)
+void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonical &out);
+void hash_bytes(const uint8_t *data, size_t n, uint64_t out[2]);
+
+// planner (planner.cpp)
+lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan);
+std::string describe_plan(const Plan &plan);
+int broadcast_class(const int64_t *dims, int rank, uint64_t rows, uint64_t cols);
+
+// executor (executor.cpp)
+lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg);
+void fastdiv_make(uint32_t d, uint32_t *mul, uint32_t *sh1, uint32_t *sh2);
+
+}  // namespace lt

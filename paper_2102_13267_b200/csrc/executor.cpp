@@ -1,0 +1,170 @@
+// Executor: binds this trace's pointers and run-time scalars into a plan's parameter blocks
+// and launches its kernels on the context's stream.
+#include <cmath>
+#include <cstring>
+
+#include "engine.h"
+#include "launch.h"
+
+namespace lt {
+
+namespace {
+
+uint32_t f32_bits(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return u;
+}
+
+uint32_t encode_imm(const Imm &im, const std::vector<DynValue> &dyn) {
+    if (im.enc == ENC_LO32 || im.enc == ENC_HI32) {
+        uint64_t v = (uint64_t)dyn[im.dyn].i;
+        return im.enc == ENC_LO32 ? (uint32_t)v : (uint32_t)(v >> 32);
+    }
+    const double v = im.dyn >= 0 ? dyn[im.dyn].d : im.sval;
+    switch (im.enc) {
+    case ENC_F32: return f32_bits((float)v);
+    case ENC_BF16: {
+        uint32_t u = f32_bits((float)v);
+        if ((u & 0x7fffffffu) > 0x7f800000u) return u | 0x00400000u;
+        u += 0x7fffu + ((u >> 16) & 1u);
+        return u & 0xffff0000u;
+    }
+    case ENC_I32: return (uint32_t)(int32_t)(int64_t)v;
+    case ENC_U8: return (uint32_t)(int64_t)v & 0xffu;
+    default: return (uint32_t)(int64_t)v;
+    }
+}
+
+cudaEvent_t take_event(lt_ctx *c) {
+    if (!c->event_pool.empty()) {
+        cudaEvent_t e = c->event_pool.back();
+        c->event_pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+}  // namespace
+
+lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
+    const bool dry = c->device == LT_DEVICE_NONE;
+    const size_t n_out = plan.outputs.size();
+    c->param_ptr.resize(plan.n_params);
+    for (uint32_t i = 0; i < plan.n_params; ++i)
+        c->param_ptr[i] = c->buffers[c->nodes[cg.param_node[i]].buffer].ptr;
+    c->out_ptr.assign(n_out, nullptr);
+    c->temp_ptr.assign(plan.temp_bytes.size(), nullptr);
+
+    auto release_all = [&](bool outputs_too) {
+        for (void *&p : c->temp_ptr) {
+            if (p) ctx_free(c, p);
+            p = nullptr;
+        }
+        if (outputs_too)
+            for (size_t k = 0; k < n_out; ++k)
+                if (c->out_ptr[k] && plan.outputs[k].donated_param < 0) {
+                    ctx_free(c, c->out_ptr[k]);
+                    c->out_ptr[k] = nullptr;
+                }
+    };
+
+    uint64_t donated = 0, allocated = 0;
+    for (size_t k = 0; k < n_out; ++k) {
+        const OutputPlan &o = plan.outputs[k];
+        if (o.donated_param >= 0) {
+            c->out_ptr[k] = c->param_ptr[o.donated_param];
+            ++donated;
+        } else {
+            c->out_ptr[k] = ctx_alloc(c, o.bytes);
+            if (!c->out_ptr[k]) {
+                release_all(true);
+                return fail(c, LT_ERR_OOM, "allocator returned null for an output");
+            }
+            ++allocated;
+        }
+    }
+    for (size_t t = 0; t < plan.temp_bytes.size(); ++t) {
+        c->temp_ptr[t] = ctx_alloc(c, plan.temp_bytes[t]);
+        if (!c->temp_ptr[t]) {
+            release_all(true);
+            return fail(c, LT_ERR_OOM, "allocator returned null for a temporary");
+        }
+    }
+
+    auto resolve = [&](const IoRef &io) -> uint64_t {
+        void *p = io.kind == IO_PARAM ? c->param_ptr[io.index] : io.kind == IO_OUTPUT ? c->out_ptr[io.index] : c->temp_ptr[io.index];
+        return (uint64_t)(uintptr_t)p;
+    };
+
+    const unsigned waves = 4;
+    for (Launch &L : plan.launches) {
+        cudaError_t e = cudaSuccess;
+        cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+        if (c->timing && !dry) {
+            ev0 = take_event(c);
+            ev1 = take_event(c);
+        }
+        if (L.kind == K_MULTI) {
+            LtMultiParams &P = *L.mp;
+            const Group &g0 = plan.groups[L.groups[0]];
+            for (size_t q = 0; q < g0.imms.size(); ++q) P.scal[q] = encode_imm(g0.imms[q], cg.dyn);
+            const size_t slots = g0.io.size();
+            for (size_t k = 0; k < L.groups.size(); ++k) {
+                const Group &g = plan.groups[L.groups[k]];
+                for (size_t s = 0; s < slots; ++s) P.ptr[k * slots + s] = resolve(g.io[s]);
+            }
+            if (!dry) {
+                unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * c->occ_multi * waves);
+                if (grid < 1) grid = 1;
+                if (ev0) cudaEventRecord(ev0, c->stream);
+                e = lt_launch_multi(P, L.fast, grid, c->stream);
+                if (ev1) cudaEventRecord(ev1, c->stream);
+            }
+            c->stats.launches_multi++;
+        } else {
+            LtKParams &P = *L.kp;
+            const Group &g = plan.groups[L.groups[0]];
+            for (size_t q = 0; q < g.imms.size(); ++q) P.scal[q] = encode_imm(g.imms[q], cg.dyn);
+            for (size_t s = 0; s < g.io.size(); ++s) P.ptr[s] = resolve(g.io[s]);
+            if (L.kind == K_EW) {
+                if (!dry) {
+                    uint64_t need = (P.n_chunks + LT_EW_THREADS - 1) / LT_EW_THREADS;
+                    unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);
+                    if (grid < 1) grid = 1;
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    e = lt_launch_ew(P, L.fast, grid, c->stream);
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                }
+                c->stats.launches_elementwise++;
+            } else {
+                if (!dry) {
+                    uint64_t blocks = ((uint64_t)P.rows + P.rows_per_cta - 1) / P.rows_per_cta;
+                    unsigned per_sm = (unsigned)std::max(1, c->occ_row * 256 / (int)L.threads);
+                    unsigned grid = (unsigned)std::min<uint64_t>(blocks, (uint64_t)c->sm_count * per_sm * waves);
+                    if (grid < 1) grid = 1;
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    e = lt_launch_row(P, L.fast, grid, L.threads, c->stream);
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                }
+                c->stats.launches_row++;
+            }
+        }
+        if (ev0) c->timed.push_back(TimedLaunch{ev0, ev1, L.kind, L.bytes});
+        if (e != cudaSuccess) {
+            release_all(true);
+            return fail(c, LT_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e));
+        }
+        c->stats.kernels_launched++;
+        c->stats.bytes_planned += L.bytes;
+    }
+    release_all(false);  // stream-ordered: later users of this memory queue behind the kernels above
+    c->stats.outputs_donated += donated;
+    c->stats.outputs_allocated += allocated;
+    c->stats.temporaries_allocated += plan.temp_bytes.size();
+    return LT_OK;
+}
+
+}  // namespace lt

@@ -1,0 +1,566 @@
+// Fused-group kernels for sm_100a: every thread interprets the group's register program
+// (vm.h) on chunks of LT_VM_V consecutive elements.  Three shells share one interpreter:
+//   lt_ew_kernel     elementwise / broadcast groups, grid-stride over chunks
+//   lt_row_kernel    groups with row reductions: a power-of-two thread group owns a row,
+//                    reduces with warp shuffles and, across warps, through shared memory
+//   lt_multi_kernel  one program over many independent tensors (horizontal fusion)
+// The program, pointer table and immediates arrive as a __grid_constant__ parameter and
+// are read from the constant bank.  No tensor cores: nothing here is a contraction.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "launch.h"
+#include "vm.h"
+
+namespace {
+
+constexpr int V = LT_VM_V;
+
+struct Chunk {
+    uint64_t flat0;  // flat index of lane 0
+    uint32_t row;
+    uint32_t col0;   // column of lane 0
+    int nvalid;      // lanes 0..nvalid-1 exist
+    bool row_ok;
+};
+
+struct RowCtx {
+    float *smem;       // 2 x 32 floats
+    uint32_t phase;
+    uint32_t group;    // threads per row
+    uint32_t warp, lane;
+};
+
+// ---------------------------------------------------------------- environments
+struct EnvK {
+    const LtKParams &P;
+    __device__ __forceinline__ LtIns ins(uint32_t pc) const { return P.ins[pc]; }
+    __device__ __forceinline__ uint32_t n_ins() const { return P.n_ins; }
+    __device__ __forceinline__ uint32_t scal(uint32_t i) const { return P.scal[i]; }
+    __device__ __forceinline__ uint64_t ptr(uint32_t s) const { return P.ptr[s]; }
+    __device__ __forceinline__ uint32_t dtype(uint32_t s) const { return P.io_dtype[s]; }
+    __device__ __forceinline__ uint32_t cls(uint32_t s) const { return P.io_class[s]; }
+};
+
+struct EnvM {
+    const LtMultiParams &P;
+    uint32_t base;  // instance * n_slots
+    __device__ __forceinline__ LtIns ins(uint32_t pc) const { return P.ins[pc]; }
+    __device__ __forceinline__ uint32_t n_ins() const { return P.n_ins; }
+    __device__ __forceinline__ uint32_t scal(uint32_t i) const { return P.scal[i]; }
+    __device__ __forceinline__ uint64_t ptr(uint32_t s) const { return P.ptr[base + s]; }
+    __device__ __forceinline__ uint32_t dtype(uint32_t s) const { return P.io_dtype[s]; }
+    __device__ __forceinline__ uint32_t cls(uint32_t) const { return LT_CLS_FULL; }
+};
+
+// ---------------------------------------------------------------------- math
+__device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
+__device__ __forceinline__ uint32_t f2u(float f) { return __float_as_uint(f); }
+
+__device__ __forceinline__ float max_nan(float a, float b) {
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ float min_nan(float a, float b) {
+    float r;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ float tanh_approx(float x) {
+    float r;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float sqrt_approx(float x) {
+    float r;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+template <int OP, bool FAST>
+__device__ __forceinline__ float f2(float a, float b) {
+    if constexpr (OP == F2_ADD) return __fadd_rn(a, b);
+    else if constexpr (OP == F2_SUB) return __fsub_rn(a, b);
+    else if constexpr (OP == F2_RSUB) return __fsub_rn(b, a);
+    else if constexpr (OP == F2_MUL) return __fmul_rn(a, b);
+    else if constexpr (OP == F2_DIV) return FAST ? __fdividef(a, b) : __fdiv_rn(a, b);
+    else if constexpr (OP == F2_RDIV) return FAST ? __fdividef(b, a) : __fdiv_rn(b, a);
+    else if constexpr (OP == F2_MAX) return max_nan(a, b);
+    else return min_nan(a, b);
+}
+
+template <int OP>
+__device__ __forceinline__ float i2(float fa, float fb) {
+    uint32_t a = f2u(fa), b = f2u(fb), r;
+    if constexpr (OP == I2_ADD) r = a + b;
+    else if constexpr (OP == I2_SUB) r = a - b;
+    else if constexpr (OP == I2_RSUB) r = b - a;
+    else if constexpr (OP == I2_MUL) r = a * b;
+    else if constexpr (OP == I2_AND) r = a & b;
+    else if constexpr (OP == I2_OR) r = a | b;
+    else if constexpr (OP == I2_XOR) r = a ^ b;
+    else if constexpr (OP == I2_MAXS) r = (uint32_t)max((int32_t)a, (int32_t)b);
+    else if constexpr (OP == I2_MINS) r = (uint32_t)min((int32_t)a, (int32_t)b);
+    else if constexpr (OP == I2_MAXU) r = max(a, b);
+    else r = min(a, b);
+    return u2f(r);
+}
+
+template <int CC, class T>
+__device__ __forceinline__ bool cmp_t(T a, T b) {
+    if constexpr (CC == CC_GT) return a > b;
+    else if constexpr (CC == CC_GE) return a >= b;
+    else if constexpr (CC == CC_LT) return a < b;
+    else if constexpr (CC == CC_LE) return a <= b;
+    else if constexpr (CC == CC_EQ) return a == b;
+    else return a != b;
+}
+
+template <int IDX>
+__device__ __forceinline__ float cmp(float a, float b) {
+    constexpr int TY = IDX / 6, CC = IDX % 6;
+    bool r;
+    if constexpr (TY == 0) r = cmp_t<CC, float>(a, b);
+    else if constexpr (TY == 1) r = cmp_t<CC, int32_t>((int32_t)f2u(a), (int32_t)f2u(b));
+    else r = cmp_t<CC, uint32_t>(f2u(a), f2u(b));
+    return u2f(r ? 1u : 0u);
+}
+
+template <int OP, bool FAST>
+__device__ __forceinline__ float un(float x) {
+    if constexpr (OP == OP_U_NEG) return -x;
+    else if constexpr (OP == OP_U_ABS) return fabsf(x);
+    else if constexpr (OP == OP_U_RELU) return max_nan(x, 0.0f);
+    else if constexpr (OP == OP_U_EXP) return FAST ? __expf(x) : expf(x);
+    else if constexpr (OP == OP_U_LOG) return FAST ? __logf(x) : logf(x);
+    else if constexpr (OP == OP_U_TANH) return FAST ? tanh_approx(x) : tanhf(x);
+    else if constexpr (OP == OP_U_SQRT) return FAST ? sqrt_approx(x) : __fsqrt_rn(x);
+    else if constexpr (OP == OP_U_RSQRT) return rsqrtf(x);
+    else if constexpr (OP == OP_U_RECIP) return FAST ? rcp_approx(x) : __frcp_rn(x);
+    else if constexpr (OP == OP_U_SQUARE) return __fmul_rn(x, x);
+    else if constexpr (OP == OP_U_SIGMOID)
+        return FAST ? rcp_approx(1.0f + __expf(-x)) : __fdiv_rn(1.0f, 1.0f + expf(-x));
+    else if constexpr (OP == OP_U_GELU) {
+        const float k = 0.7978845608028654f;  // sqrt(2/pi)
+        float inner = k * fmaf(0.044715f * x, x * x, x);
+        float th = FAST ? tanh_approx(inner) : tanhf(inner);
+        return 0.5f * x * (1.0f + th);
+    } else if constexpr (OP == OP_U_RBF16) return __bfloat162float(__float2bfloat16_rn(x));
+    else if constexpr (OP == OP_U_INEG) return u2f(0u - f2u(x));
+    else if constexpr (OP == OP_U_IABS) return u2f((uint32_t)abs((int32_t)f2u(x)));
+    else if constexpr (OP == OP_U_NOT) return u2f(f2u(x) == 0u ? 1u : 0u);
+    else if constexpr (OP == OP_C_I2F) return __int2float_rn((int32_t)f2u(x));
+    else if constexpr (OP == OP_C_U2F) return __uint2float_rn(f2u(x));
+    else if constexpr (OP == OP_C_F2I) return u2f((uint32_t)__float2int_rz(x));
+    else if constexpr (OP == OP_C_NZF) return u2f(x != 0.0f ? 1u : 0u);
+    else return u2f(f2u(x) != 0u ? 1u : 0u);  // OP_C_NZI
+}
+
+// Philox4x32-10 (Salmon et al., SC'11): ten multiply/xor rounds, key bumped by Weyl constants.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t (&out)[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ------------------------------------------------------------------- memory
+__device__ __forceinline__ uint32_t esz_log2(uint32_t dt) { return dt == LT_ST_BF16 ? 1u : (dt == LT_ST_U8 ? 0u : 2u); }
+
+// Raw chunk load: lanes keep the storage format (bf16: 4 packed words, u8: 2 packed words,
+// 32-bit types: 8 words); CVT widens later so the load itself stays asynchronous.
+template <class Env>
+__device__ __forceinline__ void load_raw(float (&d)[V], const Env &E, uint32_t slot, const Chunk &ck) {
+    const uint32_t dt = E.dtype(slot), cls = E.cls(slot);
+    const char *base = reinterpret_cast<const char *>(E.ptr(slot));
+    if (cls >= LT_CLS_ROWVEC) {  // one element, replicated in storage format
+        const uint64_t idx = cls == LT_CLS_ROWVEC ? (ck.row_ok ? ck.row : 0) : 0;
+        if (dt == LT_ST_BF16) {
+            uint32_t h = __ldg(reinterpret_cast<const unsigned short *>(base) + idx);
+            h |= h << 16;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) d[i] = u2f(h);
+        } else if (dt == LT_ST_U8) {
+            uint32_t b = __ldg(reinterpret_cast<const unsigned char *>(base) + idx) * 0x01010101u;
+            d[0] = u2f(b);
+            d[1] = u2f(b);
+        } else {
+            float x = __ldg(reinterpret_cast<const float *>(base) + idx);
+#pragma unroll
+            for (int i = 0; i < V; ++i) d[i] = x;
+        }
+        return;
+    }
+    const bool colvec = cls == LT_CLS_COLVEC;
+    const uint64_t idx = colvec ? (uint64_t)ck.col0 : ck.flat0;
+    const char *p = base + (idx << esz_log2(dt));
+    const uintptr_t need = dt == LT_ST_U8 ? 7u : 15u;
+    if (ck.nvalid == V && (reinterpret_cast<uintptr_t>(p) & need) == 0) {
+        if (dt == LT_ST_BF16) {
+            uint4 a = colvec ? __ldg(reinterpret_cast<const uint4 *>(p)) : __ldcs(reinterpret_cast<const uint4 *>(p));
+            d[0] = u2f(a.x); d[1] = u2f(a.y); d[2] = u2f(a.z); d[3] = u2f(a.w);
+        } else if (dt == LT_ST_U8) {
+            uint2 a = colvec ? __ldg(reinterpret_cast<const uint2 *>(p)) : __ldcs(reinterpret_cast<const uint2 *>(p));
+            d[0] = u2f(a.x); d[1] = u2f(a.y);
+        } else {
+            const uint4 *q = reinterpret_cast<const uint4 *>(p);
+            uint4 a = colvec ? __ldg(q) : __ldcs(q);
+            uint4 b = colvec ? __ldg(q + 1) : __ldcs(q + 1);
+            d[0] = u2f(a.x); d[1] = u2f(a.y); d[2] = u2f(a.z); d[3] = u2f(a.w);
+            d[4] = u2f(b.x); d[5] = u2f(b.y); d[6] = u2f(b.z); d[7] = u2f(b.w);
+        }
+        return;
+    }
+    // ragged tail or unaligned pointer: element by element, packed into the same storage format
+    if (dt == LT_ST_BF16) {
+        const unsigned short *q = reinterpret_cast<const unsigned short *>(p);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t lo = 2 * j < ck.nvalid ? q[2 * j] : 0u;
+            uint32_t hi = 2 * j + 1 < ck.nvalid ? q[2 * j + 1] : 0u;
+            d[j] = u2f(lo | (hi << 16));
+        }
+    } else if (dt == LT_ST_U8) {
+        const unsigned char *q = reinterpret_cast<const unsigned char *>(p);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if (4 * j + b < ck.nvalid) w |= (uint32_t)q[4 * j + b] << (8 * b);
+            d[j] = u2f(w);
+        }
+    } else {
+        const float *q = reinterpret_cast<const float *>(p);
+#pragma unroll
+        for (int i = 0; i < V; ++i) d[i] = i < ck.nvalid ? q[i] : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void widen(float (&d)[V], uint32_t dt) {
+    if (dt == LT_ST_BF16) {
+        uint32_t w0 = f2u(d[0]), w1 = f2u(d[1]), w2 = f2u(d[2]), w3 = f2u(d[3]);
+        d[0] = u2f(w0 << 16); d[1] = u2f(w0 & 0xffff0000u);
+        d[2] = u2f(w1 << 16); d[3] = u2f(w1 & 0xffff0000u);
+        d[4] = u2f(w2 << 16); d[5] = u2f(w2 & 0xffff0000u);
+        d[6] = u2f(w3 << 16); d[7] = u2f(w3 & 0xffff0000u);
+    } else if (dt == LT_ST_U8) {
+        uint32_t w0 = f2u(d[0]), w1 = f2u(d[1]);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            d[b] = u2f((w0 >> (8 * b)) & 0xffu);
+            d[4 + b] = u2f((w1 >> (8 * b)) & 0xffu);
+        }
+    }
+}
+
+template <class Env>
+__device__ __forceinline__ void store_chunk(const float (&a)[V], const Env &E, uint32_t slot, const Chunk &ck) {
+    const uint32_t dt = E.dtype(slot), cls = E.cls(slot);
+    char *base = reinterpret_cast<char *>(E.ptr(slot));
+    if (cls == LT_CLS_ROWVEC) {  // one value per row, written by the thread that owns column 0
+        if (ck.col0 == 0 && ck.row_ok) {
+            if (dt == LT_ST_BF16) reinterpret_cast<__nv_bfloat16 *>(base)[ck.row] = __float2bfloat16_rn(a[0]);
+            else if (dt == LT_ST_U8) reinterpret_cast<unsigned char *>(base)[ck.row] = (unsigned char)f2u(a[0]);
+            else reinterpret_cast<float *>(base)[ck.row] = a[0];
+        }
+        return;
+    }
+    char *p = base + (ck.flat0 << esz_log2(dt));
+    const uintptr_t need = dt == LT_ST_U8 ? 7u : 15u;
+    if (ck.nvalid == V && (reinterpret_cast<uintptr_t>(p) & need) == 0) {
+        if (dt == LT_ST_BF16) {
+            uint4 w;
+            __nv_bfloat162 h;
+            h = __floats2bfloat162_rn(a[0], a[1]); w.x = *reinterpret_cast<uint32_t *>(&h);
+            h = __floats2bfloat162_rn(a[2], a[3]); w.y = *reinterpret_cast<uint32_t *>(&h);
+            h = __floats2bfloat162_rn(a[4], a[5]); w.z = *reinterpret_cast<uint32_t *>(&h);
+            h = __floats2bfloat162_rn(a[6], a[7]); w.w = *reinterpret_cast<uint32_t *>(&h);
+            __stcs(reinterpret_cast<uint4 *>(p), w);
+        } else if (dt == LT_ST_U8) {
+            uint2 w;
+            w.x = (f2u(a[0]) & 0xffu) | ((f2u(a[1]) & 0xffu) << 8) | ((f2u(a[2]) & 0xffu) << 16) | (f2u(a[3]) << 24);
+            w.y = (f2u(a[4]) & 0xffu) | ((f2u(a[5]) & 0xffu) << 8) | ((f2u(a[6]) & 0xffu) << 16) | (f2u(a[7]) << 24);
+            __stcs(reinterpret_cast<uint2 *>(p), w);
+        } else {
+            uint4 w0 = make_uint4(f2u(a[0]), f2u(a[1]), f2u(a[2]), f2u(a[3]));
+            uint4 w1 = make_uint4(f2u(a[4]), f2u(a[5]), f2u(a[6]), f2u(a[7]));
+            __stcs(reinterpret_cast<uint4 *>(p), w0);
+            __stcs(reinterpret_cast<uint4 *>(p) + 1, w1);
+        }
+        return;
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        if (i < ck.nvalid) {
+            if (dt == LT_ST_BF16) reinterpret_cast<__nv_bfloat16 *>(p)[i] = __float2bfloat16_rn(a[i]);
+            else if (dt == LT_ST_U8) reinterpret_cast<unsigned char *>(p)[i] = (unsigned char)f2u(a[i]);
+            else reinterpret_cast<float *>(p)[i] = a[i];
+        }
+    }
+}
+
+// ------------------------------------------------------------ row reductions
+template <int KIND>
+__device__ __forceinline__ float red_comb(float a, float b) {
+    if constexpr (KIND == 0) return __fadd_rn(a, b);
+    else if constexpr (KIND == 1) return max_nan(a, b);
+    else return min_nan(a, b);
+}
+
+template <int KIND>
+__device__ __forceinline__ void row_reduce(float (&acc)[V], const Chunk &ck, RowCtx *rc) {
+    const float ident = KIND == 0 ? 0.0f : (KIND == 1 ? -INFINITY : INFINITY);
+    float part = ident;
+#pragma unroll
+    for (int i = 0; i < V; ++i) part = red_comb<KIND>(part, i < ck.nvalid ? acc[i] : ident);
+    const uint32_t width = rc->group < 32u ? rc->group : 32u;
+    for (uint32_t off = width >> 1; off > 0; off >>= 1)
+        part = red_comb<KIND>(part, __shfl_xor_sync(0xffffffffu, part, off));
+    if (rc->group > 32u) {
+        float *buf = rc->smem + (rc->phase & 1u) * 32u;
+        rc->phase++;
+        if (rc->lane == 0) buf[rc->warp] = part;
+        __syncthreads();
+        const uint32_t wpr = rc->group >> 5;
+        const uint32_t first = (rc->warp / wpr) * wpr;
+        part = buf[first];
+        for (uint32_t w = 1; w < wpr; ++w) part = red_comb<KIND>(part, buf[first + w]);
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = part;
+}
+
+// -------------------------------------------------------------- interpreter
+#define LT_SRC_CASES(BASE, IDX, EXPR)                                                                   \
+    case (BASE) + (IDX) * LT_VM_NSRC + 0: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t0[i]; acc[i] = EXPR; } } break; \
+    case (BASE) + (IDX) * LT_VM_NSRC + 1: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t1[i]; acc[i] = EXPR; } } break; \
+    case (BASE) + (IDX) * LT_VM_NSRC + 2: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t2[i]; acc[i] = EXPR; } } break; \
+    case (BASE) + (IDX) * LT_VM_NSRC + 3: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t3[i]; acc[i] = EXPR; } } break; \
+    case (BASE) + (IDX) * LT_VM_NSRC + 4: { const float b_ = u2f(E.scal(in.imm)); _Pragma("unroll") for (int i = 0; i < V; ++i) { acc[i] = EXPR; } } break;
+
+#define LT_F2_CASE(IDX) LT_SRC_CASES(OP_F2, IDX, (f2<IDX, FAST>(acc[i], b_)))
+#define LT_I2_CASE(IDX) LT_SRC_CASES(OP_I2, IDX, (i2<IDX>(acc[i], b_)))
+#define LT_CMP_CASE(IDX) LT_SRC_CASES(OP_CMP, IDX, (cmp<IDX>(acc[i], b_)))
+#define LT_WHERE_CASES(M, TM)                                                                 \
+    LT_SRC_CASES(OP_WHERE_A, M, (f2u(TM[i]) != 0u ? acc[i] : b_))                              \
+    LT_SRC_CASES(OP_WHERE_B, M, (f2u(TM[i]) != 0u ? b_ : acc[i]))
+#define LT_UN_CASE(OPC) \
+    case OPC: { _Pragma("unroll") for (int i = 0; i < V; ++i) acc[i] = un<OPC, FAST>(acc[i]); } break;
+#define LT_T_CASES(BASE, STMT)                       \
+    case (BASE) + 0: { float(&T)[V] = t0; STMT; } break; \
+    case (BASE) + 1: { float(&T)[V] = t1; STMT; } break; \
+    case (BASE) + 2: { float(&T)[V] = t2; STMT; } break; \
+    case (BASE) + 3: { float(&T)[V] = t3; STMT; } break;
+
+template <bool FAST, bool ROW, class Env>
+__device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCtx *rc) {
+    float acc[V], t0[V], t1[V], t2[V], t3[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = t0[i] = t1[i] = t2[i] = t3[i] = 0.0f;
+    const uint32_t n_ins = E.n_ins();
+    for (uint32_t pc = 0; pc < n_ins; ++pc) {
+        const LtIns in = E.ins(pc);
+        switch (in.op) {
+            LT_T_CASES(OP_MOV_T_ACC, { _Pragma("unroll") for (int i = 0; i < V; ++i) T[i] = acc[i]; })
+            LT_T_CASES(OP_MOV_ACC_T, { _Pragma("unroll") for (int i = 0; i < V; ++i) acc[i] = T[i]; })
+            case OP_MOV_ACC_S: {
+                const float s = u2f(E.scal(in.imm));
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = s;
+            } break;
+            LT_T_CASES(OP_LD_T, load_raw(T, E, in.imm, ck))
+            case OP_LD_ACC: load_raw(acc, E, in.imm, ck); break;
+            LT_T_CASES(OP_CVT_T, widen(T, in.a))
+            case OP_CVT_ACC: widen(acc, in.a); break;
+            case OP_ST: store_chunk(acc, E, in.imm, ck); break;
+            case OP_IOTA_COL: {
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = u2f(ck.col0 + i);
+            } break;
+            case OP_IOTA_ROW: {
+                const uint32_t r = (ck.row / E.scal(in.imm)) % E.scal(in.imm + 1);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = u2f(r);
+            } break;
+            case OP_PHILOX: {
+                const uint32_t k0 = E.scal(in.imm), k1 = E.scal(in.imm + 1);
+                const uint32_t o0 = E.scal(in.imm + 2), o1 = E.scal(in.imm + 3);
+                const uint64_t q = ck.flat0 >> 2;
+                const uint32_t sh = (uint32_t)ck.flat0 & 3u;
+                uint32_t w[12];
+                philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), o0, o1, k0, k1, *reinterpret_cast<uint32_t(*)[4]>(&w[0]));
+                philox4x32_10((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), o0, o1, k0, k1,
+                              *reinterpret_cast<uint32_t(*)[4]>(&w[4]));
+                if (sh == 0) {
+#pragma unroll
+                    for (int i = 0; i < V; ++i) acc[i] = u2f(w[i]);
+                } else {  // chunk does not start on a block boundary (ragged rows)
+                    philox4x32_10((uint32_t)(q + 2), (uint32_t)((q + 2) >> 32), o0, o1, k0, k1,
+                                  *reinterpret_cast<uint32_t(*)[4]>(&w[8]));
+#pragma unroll
+                    for (int i = 0; i < V; ++i) {
+                        uint32_t x = w[i + 1];
+                        if (sh == 2) x = w[i + 2];
+                        if (sh == 3) x = w[i + 3];
+                        acc[i] = u2f(x);
+                    }
+                }
+            } break;
+            case OP_RED_SUM: if constexpr (ROW) row_reduce<0>(acc, ck, rc); break;
+            case OP_RED_MAX: if constexpr (ROW) row_reduce<1>(acc, ck, rc); break;
+            case OP_RED_MIN: if constexpr (ROW) row_reduce<2>(acc, ck, rc); break;
+            LT_UN_CASE(OP_U_NEG) LT_UN_CASE(OP_U_ABS) LT_UN_CASE(OP_U_RELU) LT_UN_CASE(OP_U_EXP)
+            LT_UN_CASE(OP_U_LOG) LT_UN_CASE(OP_U_TANH) LT_UN_CASE(OP_U_SQRT) LT_UN_CASE(OP_U_RSQRT)
+            LT_UN_CASE(OP_U_RECIP) LT_UN_CASE(OP_U_SQUARE) LT_UN_CASE(OP_U_SIGMOID) LT_UN_CASE(OP_U_GELU)
+            LT_UN_CASE(OP_U_RBF16) LT_UN_CASE(OP_U_INEG) LT_UN_CASE(OP_U_IABS) LT_UN_CASE(OP_U_NOT)
+            LT_UN_CASE(OP_C_I2F) LT_UN_CASE(OP_C_U2F) LT_UN_CASE(OP_C_F2I) LT_UN_CASE(OP_C_NZF)
+            LT_UN_CASE(OP_C_NZI)
+            LT_F2_CASE(0) LT_F2_CASE(1) LT_F2_CASE(2) LT_F2_CASE(3) LT_F2_CASE(4) LT_F2_CASE(5) LT_F2_CASE(6)
+            LT_F2_CASE(7)
+            LT_I2_CASE(0) LT_I2_CASE(1) LT_I2_CASE(2) LT_I2_CASE(3) LT_I2_CASE(4) LT_I2_CASE(5) LT_I2_CASE(6)
+            LT_I2_CASE(7) LT_I2_CASE(8) LT_I2_CASE(9) LT_I2_CASE(10)
+            LT_CMP_CASE(0) LT_CMP_CASE(1) LT_CMP_CASE(2) LT_CMP_CASE(3) LT_CMP_CASE(4) LT_CMP_CASE(5)
+            LT_CMP_CASE(6) LT_CMP_CASE(7) LT_CMP_CASE(8) LT_CMP_CASE(9) LT_CMP_CASE(10) LT_CMP_CASE(11)
+            LT_CMP_CASE(12) LT_CMP_CASE(13) LT_CMP_CASE(14) LT_CMP_CASE(15) LT_CMP_CASE(16) LT_CMP_CASE(17)
+            LT_WHERE_CASES(0, t0) LT_WHERE_CASES(1, t1) LT_WHERE_CASES(2, t2) LT_WHERE_CASES(3, t3)
+            default: break;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ kernels
+template <bool FAST>
+__global__ void __launch_bounds__(LT_EW_THREADS) lt_ew_kernel(const __grid_constant__ LtKParams P) {
+    const EnvK E{P};
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; c < P.n_chunks; c += stride) {
+        Chunk ck;
+        ck.row_ok = true;
+        if (!P.rowcol) {
+            ck.flat0 = c * V;
+            ck.row = 0;
+            ck.col0 = (uint32_t)ck.flat0;
+            const uint64_t rem = P.n - ck.flat0;
+            ck.nvalid = rem < (uint64_t)V ? (int)rem : V;
+        } else {
+            const uint32_t c32 = (uint32_t)c;
+            const uint32_t t = __umulhi(P.div_mul, c32);
+            const uint32_t row = (t + ((c32 - t) >> P.div_sh1)) >> P.div_sh2;
+            const uint32_t cc = c32 - row * P.cpr;
+            ck.row = row;
+            ck.col0 = cc * V;
+            ck.flat0 = (uint64_t)row * P.cols + ck.col0;
+            const uint32_t rem = P.cols - ck.col0;
+            ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
+        }
+        run_program<FAST, false>(E, ck, nullptr);
+    }
+}
+
+template <bool FAST, int MAXT>
+__global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ LtKParams P) {
+    __shared__ float red_smem[64];
+    const EnvK E{P};
+    RowCtx rc;
+    rc.smem = red_smem;
+    rc.phase = 0;
+    rc.group = P.group;
+    rc.warp = threadIdx.x >> 5;
+    rc.lane = threadIdx.x & 31u;
+    const uint32_t sub = threadIdx.x >> P.group_log2;           // which row of this CTA's block of rows
+    const uint32_t gl = threadIdx.x & (P.group - 1u);           // lane within the row's thread group
+    const uint32_t row_blocks = (P.rows + P.rows_per_cta - 1u) / P.rows_per_cta;
+    for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
+        Chunk ck;
+        ck.row = rb * P.rows_per_cta + sub;
+        ck.row_ok = ck.row < P.rows;
+        ck.col0 = gl * V;
+        ck.flat0 = (uint64_t)ck.row * P.cols + ck.col0;
+        int nv = 0;
+        if (ck.row_ok && ck.col0 < P.cols) {
+            const uint32_t rem = P.cols - ck.col0;
+            nv = rem < (uint32_t)V ? (int)rem : V;
+        }
+        ck.nvalid = nv;
+        run_program<FAST, true>(E, ck, &rc);
+    }
+}
+
+template <bool FAST>
+__global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
+    for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
+        // instance that owns super-chunk sc: last i with super_prefix[i] <= sc
+        uint32_t lo = 0, hi = P.n_inst;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (P.super_prefix[mid] <= sc) lo = mid; else hi = mid;
+        }
+        const EnvM E{P, lo * P.n_slots};
+        const uint32_t numel = P.numel[lo];
+        const uint32_t first = (sc - P.super_prefix[lo]) * (LT_EW_THREADS * LT_MULTI_SUB * V);
+#pragma unroll 1
+        for (int u = 0; u < LT_MULTI_SUB; ++u) {
+            const uint32_t e0 = first + (u * LT_EW_THREADS + threadIdx.x) * V;
+            if (e0 < numel) {
+                Chunk ck;
+                ck.flat0 = e0;
+                ck.row = 0;
+                ck.col0 = e0;
+                ck.row_ok = true;
+                const uint32_t rem = numel - e0;
+                ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
+                run_program<FAST, false>(E, ck, nullptr);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t lt_launch_ew(const LtKParams &p, bool fast, unsigned grid, cudaStream_t stream) {
+    if (fast) lt_ew_kernel<true><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    else lt_ew_kernel<false><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t lt_launch_row(const LtKParams &p, bool fast, unsigned grid, unsigned threads, cudaStream_t stream) {
+    if (threads <= 256) {
+        if (fast) lt_row_kernel<true, 256><<<grid, threads, 0, stream>>>(p);
+        else lt_row_kernel<false, 256><<<grid, threads, 0, stream>>>(p);
+    } else {
+        if (fast) lt_row_kernel<true, 1024><<<grid, threads, 0, stream>>>(p);
+        else lt_row_kernel<false, 1024><<<grid, threads, 0, stream>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t lt_launch_multi(const LtMultiParams &p, bool fast, unsigned grid, cudaStream_t stream) {
+    if (fast) lt_multi_kernel<true><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    else lt_multi_kernel<false><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_256, int *multi_blocks_per_sm) {
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(ew_blocks_per_sm, lt_ew_kernel<false>, LT_EW_THREADS, 0);
+    if (e != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(row_blocks_per_sm_256, lt_row_kernel<false, 256>, 256, 0);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(multi_blocks_per_sm, lt_multi_kernel<false>, LT_EW_THREADS, 0);
+}

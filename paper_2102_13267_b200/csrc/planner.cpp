@@ -1,0 +1,1164 @@
+// Planner: cuts the canonical program into fusion groups, generates each group's register
+// program (vm.h), bundles isomorphic independent groups into multi-tensor launches and
+// decides which outputs are written into donated input buffers.  This stage takes the
+// place of the domain-specific compiler in the paper's pipeline (Section 4); it runs only
+// on a compile-cache miss.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+
+#include "engine.h"
+
+namespace lt {
+
+namespace {
+
+constexpr int MAX_GROUP_NODES = 64;
+
+struct PNode {
+    uint64_t numel = 1, rows = 1, cols = 1;
+    int group = -1;      // native group, -1 for leaves and absorbed nodes
+    bool leaf = false;   // device data or scalar
+    bool absorbed = false;
+    bool reduce = false;
+    bool needs_store = false;
+    int temp = -1;       // temporary buffer index when stored but not an output
+    std::vector<uint32_t> consumers;
+};
+
+inline bool is_reduce(uint16_t op) { return op >= LT_OP_ROW_SUM && op <= LT_OP_ROW_MIN; }
+inline bool is_factory(uint16_t op) { return op == LT_OP_IOTA || op == LT_OP_PHILOX_BITS; }
+inline bool is_float(uint8_t dt) { return dt == LT_F32 || dt == LT_BF16; }
+
+void domain_of(const CNode &n, uint64_t *rows, uint64_t *cols, uint64_t *numel) {
+    uint64_t ne = 1;
+    for (int i = 0; i < n.rank; ++i) ne *= (uint64_t)n.dims[i];
+    uint64_t c = n.rank ? (uint64_t)n.dims[n.rank - 1] : 1;
+    *numel = ne;
+    *cols = c;
+    *rows = c ? ne / c : 0;
+}
+
+// class of a value with domain (r, c, ne) inside a group with domain (R, C)
+int class_in(uint64_t r, uint64_t c, uint64_t ne, uint64_t R, uint64_t C) {
+    if (r == R && c == C) return LT_CLS_FULL;
+    if (ne == 1) return LT_CLS_SCALAR;
+    if (r == 1 && c == C) return LT_CLS_COLVEC;
+    if (c == 1 && r == R) return LT_CLS_ROWVEC;
+    return -1;
+}
+
+bool approx_sensitive(uint16_t op) {
+    switch (op) {
+    case LT_OP_DIV: case LT_OP_EXP: case LT_OP_LOG: case LT_OP_TANH: case LT_OP_SQRT: case LT_OP_RSQRT:
+    case LT_OP_RECIP: case LT_OP_SIGMOID: case LT_OP_GELU_TANH:
+        return true;
+    default:
+        return false;
+    }
+}
+
+// does CONVERT from `si` to `so` leave the 32-bit register lanes unchanged?
+bool convert_is_alias(int si, int so) {
+    if (si == so) return true;
+    if (si == LT_BF16 && so == LT_F32) return true;
+    if ((si == LT_I32 || si == LT_U32) && (so == LT_I32 || so == LT_U32)) return true;
+    if (si == LT_U8 && (so == LT_I32 || so == LT_U32)) return true;
+    return false;
+}
+
+uint8_t enc_of(int dtype) { return (uint8_t)dtype; }  // ENC_* share lt_dtype numbering for 0..4
+
+// --------------------------------------------------------------------- codegen
+struct CodeGen {
+    const Canonical &cg;
+    std::vector<PNode> &pn;
+    Group &g;
+    int self;  // index of g
+    const std::vector<uint32_t> &emit;  // nodes to compute, topological order
+    const std::vector<uint8_t> &in_emit;
+
+    std::vector<int> rep, uses, temp_of, slot_of;
+    int temp_val[LT_VM_NT];
+    int temp_raw[LT_VM_NT];  // storage dtype still to widen, or -1
+    int in_acc = -1;
+    int acc_raw = -1;
+    bool ok = true;
+    bool has_reduce = false, needs_rowcol = false;
+    std::vector<uint8_t> tainted;
+
+    CodeGen(const Canonical &cg_, std::vector<PNode> &pn_, Group &g_, int self_, const std::vector<uint32_t> &emit_,
+            const std::vector<uint8_t> &in_emit_)
+        : cg(cg_), pn(pn_), g(g_), self(self_), emit(emit_), in_emit(in_emit_) {
+        size_t n = cg.nodes.size();
+        rep.assign(n, -1);
+        uses.assign(n, 0);
+        temp_of.assign(n, -1);
+        slot_of.assign(n, -1);
+        tainted.assign(n, 0);
+        for (int k = 0; k < LT_VM_NT; ++k) temp_val[k] = -1, temp_raw[k] = -1;
+    }
+
+    void emit_ins(uint16_t op, uint8_t a = 0, uint32_t imm = 0) {
+        LtIns in;
+        in.op = op;
+        in.a = a;
+        in.b = 0;
+        in.imm = imm;
+        g.ins.push_back(in);
+    }
+
+    int cls_of(uint32_t v) const {
+        const PNode &p = pn[v];
+        return class_in(p.rows, p.cols, p.numel, g.rows, g.cols);
+    }
+
+    // is v a value this group reads from memory (a device-data leaf or another group's result)?
+    bool is_input(uint32_t v) const { return !in_emit[v] && cg.nodes[v].op != N_SCALAR; }
+
+    int input_slot(uint32_t v) {
+        if (slot_of[v] >= 0) return slot_of[v];
+        const CNode &n = cg.nodes[v];
+        IoRef io;
+        io.is_store = 0;
+        io.dtype = n.dtype;
+        io.cls = (uint8_t)cls_of(v);
+        io.cnode = v;
+        if (n.op == N_DEVICE_DATA) {
+            io.kind = IO_PARAM;
+            io.index = (uint32_t)n.param;
+        } else if (n.output >= 0) {
+            io.kind = IO_OUTPUT;
+            io.index = (uint32_t)n.output;
+        } else {
+            io.kind = IO_TEMP;
+            io.index = 0;  // patched once temporaries are numbered
+        }
+        if (io.cls == LT_CLS_COLVEC || io.cls == LT_CLS_ROWVEC) needs_rowcol = true;
+        slot_of[v] = (int)g.io.size();
+        g.io.push_back(io);
+        return slot_of[v];
+    }
+
+    int imm_slot(const Imm &im, bool dedupe = true) {
+        if (dedupe)
+            for (size_t i = 0; i < g.imms.size(); ++i)
+                if (g.imms[i] == im) return (int)i;
+        g.imms.push_back(im);
+        return (int)g.imms.size() - 1;
+    }
+
+    int scalar_imm(uint32_t v, int dtype) {
+        const CNode &n = cg.nodes[v];
+        Imm im;
+        im.dyn = n.dyn;
+        im.sval = n.dyn >= 0 ? 0.0 : n.sval;
+        im.enc = enc_of(dtype);
+        return imm_slot(im);
+    }
+
+    int alloc_temp() {
+        for (int k = 0; k < LT_VM_NT; ++k)
+            if (temp_val[k] < 0) return k;
+        ok = false;
+        return 0;
+    }
+
+    void drop_if_dead(int v) {
+        if (v < 0 || uses[v] > 0) return;
+        if (temp_of[v] >= 0) {
+            temp_val[temp_of[v]] = -1;
+            temp_raw[temp_of[v]] = -1;
+            temp_of[v] = -1;
+        }
+        if (in_acc == v) in_acc = -1;
+    }
+
+    // keep the value in ACC alive in a temporary if something still needs it
+    void spill_acc(int extra_uses_consumed = 0) {
+        if (in_acc < 0) return;
+        int v = in_acc;
+        if (uses[v] - extra_uses_consumed > 0 && temp_of[v] < 0) {
+            int k = alloc_temp();
+            if (!ok) return;
+            emit_ins((uint16_t)(OP_MOV_T_ACC + k));
+            temp_val[k] = v;
+            temp_raw[k] = -1;
+            temp_of[v] = k;
+        }
+    }
+
+    static bool needs_widen(int dt) { return dt == LT_BF16 || dt == LT_U8; }
+
+    void widen_temp(int k) {
+        if (temp_raw[k] >= 0) {
+            emit_ins((uint16_t)(OP_CVT_T + k), (uint8_t)temp_raw[k]);
+            temp_raw[k] = -1;
+        }
+    }
+
+    // value v available, widened, in a temporary; returns its index
+    int ensure_temp(int v) {
+        if (temp_of[v] >= 0) {
+            widen_temp(temp_of[v]);
+            return temp_of[v];
+        }
+        int k = alloc_temp();
+        if (!ok) return 0;
+        if (in_acc == v) {
+            emit_ins((uint16_t)(OP_MOV_T_ACC + k));
+        } else if (is_input((uint32_t)v)) {
+            int s = input_slot((uint32_t)v);
+            emit_ins((uint16_t)(OP_LD_T + k), 0, (uint32_t)s);
+            int dt = cg.nodes[v].dtype;
+            if (needs_widen(dt)) emit_ins((uint16_t)(OP_CVT_T + k), (uint8_t)dt);
+        } else {
+            ok = false;  // value was never computed: planner bug
+            return 0;
+        }
+        temp_val[k] = v;
+        temp_raw[k] = -1;
+        temp_of[v] = k;
+        return k;
+    }
+
+    // value v in ACC (the value currently there is saved first if still needed)
+    void ensure_acc(int v) {
+        if (in_acc == v) return;
+        spill_acc();
+        if (!ok) return;
+        if (temp_of[v] >= 0) {
+            widen_temp(temp_of[v]);
+            emit_ins((uint16_t)(OP_MOV_ACC_T + temp_of[v]));
+        } else if (is_input((uint32_t)v)) {
+            int s = input_slot((uint32_t)v);
+            emit_ins(OP_LD_ACC, 0, (uint32_t)s);
+            int dt = cg.nodes[v].dtype;
+            if (needs_widen(dt)) emit_ins(OP_CVT_ACC, (uint8_t)dt);
+        } else {
+            ok = false;
+            return;
+        }
+        in_acc = v;
+    }
+
+    void consume(int v) {
+        uses[v]--;
+    }
+
+    void preload(int count) {
+        // issue the loads of the first `count` inputs up front so they are all in flight together
+        std::vector<uint32_t> order;
+        for (uint32_t n : emit) {
+            const CNode &cn = cg.nodes[n];
+            for (int i = 0; i < cn.n_in; ++i) {
+                uint32_t o = (uint32_t)rep_or_self(cn.in[i]);
+                if (is_input(o) && std::find(order.begin(), order.end(), o) == order.end()) order.push_back(o);
+            }
+        }
+        for (int i = 0; i < count && i < (int)order.size() && i < LT_VM_NT; ++i) {
+            uint32_t v = order[i];
+            int k = alloc_temp();
+            int s = input_slot(v);
+            emit_ins((uint16_t)(OP_LD_T + k), 0, (uint32_t)s);
+            temp_val[k] = (int)v;
+            temp_of[v] = k;
+            int dt = cg.nodes[v].dtype;
+            temp_raw[k] = needs_widen(dt) ? dt : -1;
+        }
+    }
+
+    int rep_or_self(uint32_t v) const { return rep[v] >= 0 ? rep[v] : (int)v; }
+
+    void count_uses() {
+        for (uint32_t n : emit) {
+            const CNode &cn = cg.nodes[n];
+            for (int i = 0; i < cn.n_in; ++i) uses[cn.in[i]]++;
+        }
+    }
+
+    void store_result(uint32_t n) {
+        // ACC holds node n's value
+        const CNode &cn = cg.nodes[n];
+        IoRef io;
+        io.is_store = 1;
+        io.dtype = cn.dtype;
+        io.cls = (uint8_t)cls_of(n);
+        io.cnode = n;
+        if (cn.output >= 0) {
+            io.kind = IO_OUTPUT;
+            io.index = (uint32_t)cn.output;
+        } else {
+            io.kind = IO_TEMP;
+            io.index = 0;
+        }
+        if (io.cls == LT_CLS_COLVEC || io.cls == LT_CLS_SCALAR) {
+            ok = false;  // native members are FULL or ROWVEC by construction
+            return;
+        }
+        if (io.cls == LT_CLS_ROWVEC && !has_reduce) needs_rowcol = true;
+        int s = (int)g.io.size();
+        g.io.push_back(io);
+        emit_ins(OP_ST, 0, (uint32_t)s);
+    }
+
+    // ---- one node
+    void gen_node(uint32_t n) {
+        const CNode &cn = cg.nodes[n];
+        const uint16_t op = cn.op;
+        const bool store = pn[n].group == self && pn[n].needs_store;
+        for (int i = 0; i < cn.n_in; ++i)
+            if (tainted[rep_or_self(cn.in[i])] || tainted[cn.in[i]]) tainted[n] = 1;
+        if (approx_sensitive(op)) tainted[n] = 1;
+
+        if (op == LT_OP_CONVERT && convert_is_alias(cg.nodes[cn.in[0]].dtype, cn.dtype)) {
+            int x = rep_or_self(cn.in[0]);
+            if (cg.nodes[cn.in[0]].op == N_SCALAR) { ok = false; return; }
+            rep[n] = x;
+            uses[x] += uses[n] - 1;
+            tainted[n] = tainted[x] || tainted[n];
+            if (store) {
+                ensure_acc(x);
+                if (!ok) return;
+                store_result(n);
+            }
+            drop_if_dead(x);
+            return;
+        }
+
+        int dt = cn.dtype;  // compute dtype of the node
+        if (op >= LT_OP_ADD && op <= LT_OP_NE) {
+            const bool compare = op >= LT_OP_GT;
+            uint32_t xo = cn.in[0], yo = cn.in[1];
+            bool xs = cg.nodes[xo].op == N_SCALAR, ys = cg.nodes[yo].op == N_SCALAR;
+            int odt = compare ? (xs ? cg.nodes[yo].dtype : cg.nodes[xo].dtype) : dt;  // operand dtype
+            int x = xs ? -1 : rep_or_self(xo), y = ys ? -1 : rep_or_self(yo);
+            bool swapped = false;
+            int src = -1;   // temp index or LT_VM_SRC_S
+            uint32_t imm = 0;
+            if (xs && ys) {
+                spill_acc();
+                if (!ok) return;
+                emit_ins(OP_MOV_ACC_S, 0, (uint32_t)scalar_imm(xo, odt));
+                in_acc = -1;
+                src = LT_VM_SRC_S;
+                imm = (uint32_t)scalar_imm(yo, odt);
+            } else if (ys || xs) {
+                int v = ys ? x : y;
+                swapped = xs;
+                ensure_acc(v);
+                if (!ok) return;
+                consume(v);
+                spill_acc();
+                if (!ok) return;
+                src = LT_VM_SRC_S;
+                imm = (uint32_t)scalar_imm(ys ? yo : xo, odt);
+            } else if (x == y) {
+                ensure_acc(x);
+                if (!ok) return;
+                consume(x);
+                consume(x);
+                if (!compare && is_float((uint8_t)odt) && op == LT_OP_MUL) {
+                    spill_acc();
+                    if (!ok) return;
+                    src = -2;  // square
+                } else {
+                    src = ensure_temp(x);
+                    if (!ok) return;
+                }
+            } else {
+                // put one operand in ACC (prefer the one already there), the other in a temporary
+                if (in_acc == y && in_acc != x) swapped = true;
+                else if (in_acc != x) {
+                    // neither is in ACC: move the one that is not already in a temporary, or x
+                    if (temp_of[x] >= 0 && temp_of[y] < 0) swapped = true;
+                }
+                int a = swapped ? y : x, b = swapped ? x : y;
+                ensure_acc(a);
+                if (!ok) return;
+                src = ensure_temp(b);
+                if (!ok) return;
+                consume(a);
+                consume(b);
+                spill_acc();
+                if (!ok) return;
+            }
+            // opcode
+            uint16_t code;
+            if (src == -2) {
+                code = OP_U_SQUARE;
+            } else if (compare) {
+                int cc = op - LT_OP_GT;
+                if (swapped) { static const int sw[6] = {CC_LT, CC_LE, CC_GT, CC_GE, CC_EQ, CC_NE}; cc = sw[cc]; }
+                int ty = is_float((uint8_t)odt) ? 0 : (odt == LT_I32 ? 1 : 2);
+                code = (uint16_t)(OP_CMP + (ty * 6 + cc) * LT_VM_NSRC + src);
+            } else if (is_float((uint8_t)dt)) {
+                int idx;
+                switch (op) {
+                case LT_OP_ADD: idx = F2_ADD; break;
+                case LT_OP_SUB: idx = swapped ? F2_RSUB : F2_SUB; break;
+                case LT_OP_MUL: idx = F2_MUL; break;
+                case LT_OP_DIV: idx = swapped ? F2_RDIV : F2_DIV; break;
+                case LT_OP_MAX: idx = F2_MAX; break;
+                default: idx = F2_MIN; break;
+                }
+                code = (uint16_t)(OP_F2 + idx * LT_VM_NSRC + src);
+            } else {
+                int idx;
+                const bool sgn = dt == LT_I32;
+                switch (op) {
+                case LT_OP_ADD: idx = I2_ADD; break;
+                case LT_OP_SUB: idx = swapped ? I2_RSUB : I2_SUB; break;
+                case LT_OP_MUL: idx = I2_MUL; break;
+                case LT_OP_MAX: idx = sgn ? I2_MAXS : I2_MAXU; break;
+                case LT_OP_MIN: idx = sgn ? I2_MINS : I2_MINU; break;
+                case LT_OP_AND: idx = I2_AND; break;
+                case LT_OP_OR: idx = I2_OR; break;
+                default: idx = I2_XOR; break;
+                }
+                code = (uint16_t)(OP_I2 + idx * LT_VM_NSRC + src);
+            }
+            emit_ins(code, 0, imm);
+            if (x >= 0) drop_if_dead(x);
+            if (y >= 0) drop_if_dead(y);
+        } else if (op == LT_OP_WHERE) {
+            uint32_t mo = cn.in[0], ao = cn.in[1], bo = cn.in[2];
+            int m = rep_or_self(mo);
+            bool as = cg.nodes[ao].op == N_SCALAR, bs = cg.nodes[bo].op == N_SCALAR;
+            int a = as ? -1 : rep_or_self(ao), b = bs ? -1 : rep_or_self(bo);
+            int mk = ensure_temp(m);
+            if (!ok) return;
+            bool variant_b = false;  // false: ACC = m ? ACC : src ; true: ACC = m ? src : ACC
+            int src;
+            uint32_t imm = 0;
+            if (as && bs) {
+                spill_acc();
+                if (!ok) return;
+                emit_ins(OP_MOV_ACC_S, 0, (uint32_t)scalar_imm(ao, dt));
+                in_acc = -1;
+                src = LT_VM_SRC_S;
+                imm = (uint32_t)scalar_imm(bo, dt);
+            } else if (bs) {
+                ensure_acc(a);
+                if (!ok) return;
+                consume(a);
+                spill_acc();
+                src = LT_VM_SRC_S;
+                imm = (uint32_t)scalar_imm(bo, dt);
+            } else if (as) {
+                ensure_acc(b);
+                if (!ok) return;
+                consume(b);
+                spill_acc();
+                variant_b = true;
+                src = LT_VM_SRC_S;
+                imm = (uint32_t)scalar_imm(ao, dt);
+            } else {
+                if (in_acc == b && a != b) variant_b = true;
+                int inacc = variant_b ? b : a, other = variant_b ? a : b;
+                ensure_acc(inacc);
+                if (!ok) return;
+                src = ensure_temp(other);
+                if (!ok) return;
+                consume(inacc);
+                consume(other);
+                spill_acc();
+            }
+            if (!ok) return;
+            mk = temp_of[m];  // unchanged, but re-read after possible spills
+            consume(m);
+            emit_ins((uint16_t)((variant_b ? OP_WHERE_B : OP_WHERE_A) + mk * LT_VM_NSRC + src), 0, imm);
+            drop_if_dead(m);
+            if (a >= 0) drop_if_dead(a);
+            if (b >= 0) drop_if_dead(b);
+        } else if ((op >= LT_OP_NEG && op <= LT_OP_NOT) || op == LT_OP_CONVERT || is_reduce(op)) {
+            uint32_t xo = cn.in[0];
+            if (cg.nodes[xo].op == N_SCALAR) {
+                spill_acc();
+                if (!ok) return;
+                emit_ins(OP_MOV_ACC_S, 0, (uint32_t)scalar_imm(xo, cg.nodes[xo].dtype));
+                in_acc = -1;
+            } else {
+                int x = rep_or_self(xo);
+                ensure_acc(x);
+                if (!ok) return;
+                consume(x);
+                spill_acc();
+                if (!ok) return;
+                drop_if_dead(x);
+            }
+            int si = cg.nodes[xo].dtype;
+            if (op == LT_OP_CONVERT) {
+                int so = cn.dtype;
+                int mid = si == LT_BF16 ? LT_F32 : si;  // registers hold bf16 values as f32
+                if (so == LT_F32 || so == LT_BF16) {
+                    if (mid == LT_I32) emit_ins(OP_C_I2F);
+                    else if (mid == LT_U32 || mid == LT_U8) emit_ins(OP_C_U2F);
+                } else if (so == LT_I32) {
+                    emit_ins(OP_C_F2I);
+                } else if (so == LT_U8) {
+                    emit_ins(mid == LT_F32 ? OP_C_NZF : OP_C_NZI);
+                }
+            } else if (is_reduce(op)) {
+                has_reduce = true;
+                emit_ins((uint16_t)(OP_RED_SUM + (op - LT_OP_ROW_SUM)));
+            } else {
+                uint16_t code;
+                switch (op) {
+                case LT_OP_NEG: code = dt == LT_I32 ? OP_U_INEG : OP_U_NEG; break;
+                case LT_OP_ABS: code = dt == LT_I32 ? OP_U_IABS : OP_U_ABS; break;
+                case LT_OP_RELU: code = OP_U_RELU; break;
+                case LT_OP_EXP: code = OP_U_EXP; break;
+                case LT_OP_LOG: code = OP_U_LOG; break;
+                case LT_OP_TANH: code = OP_U_TANH; break;
+                case LT_OP_SQRT: code = OP_U_SQRT; break;
+                case LT_OP_RSQRT: code = OP_U_RSQRT; break;
+                case LT_OP_RECIP: code = OP_U_RECIP; break;
+                case LT_OP_SQUARE: code = OP_U_SQUARE; break;
+                case LT_OP_SIGMOID: code = OP_U_SIGMOID; break;
+                case LT_OP_GELU_TANH: code = OP_U_GELU; break;
+                default: code = OP_U_NOT; break;
+                }
+                emit_ins(code);
+            }
+        } else if (op == LT_OP_IOTA) {
+            spill_acc();
+            if (!ok) return;
+            if ((int)cn.attr0 == cn.rank - 1) {
+                emit_ins(OP_IOTA_COL);
+                if (g.rows > 1) needs_rowcol = true;
+            } else {
+                uint64_t inner = 1;
+                for (int d = (int)cn.attr0 + 1; d + 1 < cn.rank; ++d) inner *= (uint64_t)cn.dims[d];
+                Imm a{-1, (double)inner, ENC_U32}, b{-1, (double)cn.dims[cn.attr0], ENC_U32};
+                int s = imm_slot(a, false);
+                imm_slot(b, false);
+                emit_ins(OP_IOTA_ROW, 0, (uint32_t)s);
+                needs_rowcol = true;
+            }
+        } else if (op == LT_OP_PHILOX_BITS) {
+            spill_acc();
+            if (!ok) return;
+            Imm k0{cn.dyn, 0.0, ENC_LO32}, k1{cn.dyn, 0.0, ENC_HI32}, o0{cn.dyn + 1, 0.0, ENC_LO32}, o1{cn.dyn + 1, 0.0, ENC_HI32};
+            int s = imm_slot(k0, false);
+            imm_slot(k1, false);
+            imm_slot(o0, false);
+            imm_slot(o1, false);
+            emit_ins(OP_PHILOX, 0, (uint32_t)s);
+        } else {
+            ok = false;
+            return;
+        }
+        in_acc = (int)n;
+        // bf16 nodes: arithmetic happens in f32 and the result is rounded to bf16 (ties to even);
+        // a value that is only stored is rounded by the store itself
+        if (dt == LT_BF16) {
+            bool rounds = (op >= LT_OP_ADD && op <= LT_OP_DIV) || (op >= LT_OP_EXP && op <= LT_OP_GELU_TANH) ||
+                          op == LT_OP_ROW_SUM || (op == LT_OP_CONVERT);
+            if (rounds && uses[n] > 0) emit_ins(OP_U_RBF16);
+        }
+        if (store) store_result(n);
+        if (uses[n] == 0) in_acc = -1;
+    }
+
+    bool run(int preload_count) {
+        count_uses();
+        preload(preload_count);
+        for (uint32_t n : emit) {
+            gen_node(n);
+            if (!ok) return false;
+        }
+        if (g.ins.size() > LT_VM_MAX_INS || g.io.size() > LT_VM_MAX_PTR || g.imms.size() > LT_VM_MAX_SCAL) return false;
+        return true;
+    }
+};
+
+// nodes a group must compute: its native members plus the absorbed producers they reach
+void emission_list(const Canonical &cg, const std::vector<PNode> &pn, const Group &g, std::vector<uint32_t> &emit,
+                   std::vector<uint8_t> &in_emit) {
+    emit.clear();
+    std::vector<uint32_t> stack(g.members.begin(), g.members.end());
+    for (uint32_t m : g.members) in_emit[m] = 1;
+    emit = g.members;
+    while (!stack.empty()) {
+        uint32_t n = stack.back();
+        stack.pop_back();
+        const CNode &cn = cg.nodes[n];
+        for (int i = 0; i < cn.n_in; ++i) {
+            uint32_t o = cn.in[i];
+            if (pn[o].absorbed && !in_emit[o]) {
+                in_emit[o] = 1;
+                emit.push_back(o);
+                stack.push_back(o);
+            }
+        }
+    }
+    std::sort(emit.begin(), emit.end());  // canonical order is topological
+}
+
+uint64_t io_bytes(const Group &g, const IoRef &io) {
+    uint64_t es = dtype_size(io.dtype);
+    switch (io.cls) {
+    case LT_CLS_FULL: return g.rows * g.cols * es;
+    case LT_CLS_COLVEC: return g.cols * es;
+    case LT_CLS_ROWVEC: return g.rows * es;
+    default: return es;
+    }
+}
+
+const char *src_name(int s) {
+    static const char *n[] = {"T0", "T1", "T2", "T3", "S"};
+    return n[s];
+}
+
+std::string disasm(const LtIns &in) {
+    char buf[96];
+    const int op = in.op;
+    auto src_txt = [&](int s) -> std::string {
+        if (s == LT_VM_SRC_S) return "S" + std::to_string(in.imm);
+        return src_name(s);
+    };
+    if (op >= OP_MOV_T_ACC && op < OP_MOV_ACC_T) snprintf(buf, sizeof(buf), "T%d = ACC", op - OP_MOV_T_ACC);
+    else if (op >= OP_MOV_ACC_T && op < OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = T%d", op - OP_MOV_ACC_T);
+    else if (op == OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = S%u", in.imm);
+    else if (op >= OP_LD_T && op < OP_LD_ACC) snprintf(buf, sizeof(buf), "T%d = load p%u", op - OP_LD_T, in.imm);
+    else if (op == OP_LD_ACC) snprintf(buf, sizeof(buf), "ACC = load p%u", in.imm);
+    else if (op >= OP_CVT_T && op < OP_CVT_ACC) snprintf(buf, sizeof(buf), "T%d = widen.%s T%d", op - OP_CVT_T, dtype_name(in.a), op - OP_CVT_T);
+    else if (op == OP_CVT_ACC) snprintf(buf, sizeof(buf), "ACC = widen.%s ACC", dtype_name(in.a));
+    else if (op == OP_ST) snprintf(buf, sizeof(buf), "store p%u = ACC", in.imm);
+    else if (op == OP_IOTA_COL) snprintf(buf, sizeof(buf), "ACC = iota.col");
+    else if (op == OP_IOTA_ROW) snprintf(buf, sizeof(buf), "ACC = iota.row S%u S%u", in.imm, in.imm + 1);
+    else if (op == OP_PHILOX) snprintf(buf, sizeof(buf), "ACC = philox S%u..S%u", in.imm, in.imm + 3);
+    else if (op >= OP_RED_SUM && op <= OP_RED_MIN) {
+        static const char *r[] = {"sum", "max", "min"};
+        snprintf(buf, sizeof(buf), "ACC = row_%s ACC", r[op - OP_RED_SUM]);
+    } else if (op >= OP_U_NEG && op <= OP_C_NZI) {
+        static const char *u[] = {"neg", "abs", "relu", "exp", "log", "tanh", "sqrt", "rsqrt", "recip", "square",
+                                  "sigmoid", "gelu_tanh", "round_bf16", "ineg", "iabs", "not", "i2f", "u2f", "f2i",
+                                  "nonzero.f", "nonzero.i"};
+        snprintf(buf, sizeof(buf), "ACC = %s ACC", u[op - OP_U_NEG]);
+    } else if (op >= OP_F2 && op < OP_I2) {
+        static const char *f[] = {"add", "sub", "rsub", "mul", "div", "rdiv", "max", "min"};
+        int idx = (op - OP_F2) / LT_VM_NSRC, s = (op - OP_F2) % LT_VM_NSRC;
+        snprintf(buf, sizeof(buf), "ACC = f.%s ACC, %s", f[idx], src_txt(s).c_str());
+    } else if (op >= OP_I2 && op < OP_I2 + I2_COUNT * LT_VM_NSRC) {
+        static const char *f[] = {"add", "sub", "rsub", "mul", "and", "or", "xor", "max.s", "min.s", "max.u", "min.u"};
+        int idx = (op - OP_I2) / LT_VM_NSRC, s = (op - OP_I2) % LT_VM_NSRC;
+        snprintf(buf, sizeof(buf), "ACC = i.%s ACC, %s", f[idx], src_txt(s).c_str());
+    } else if (op >= OP_CMP && op < OP_CMP + 18 * LT_VM_NSRC) {
+        static const char *cc[] = {"gt", "ge", "lt", "le", "eq", "ne"};
+        static const char *ty[] = {"f", "s", "u"};
+        int idx = (op - OP_CMP) / LT_VM_NSRC, s = (op - OP_CMP) % LT_VM_NSRC;
+        snprintf(buf, sizeof(buf), "ACC = cmp.%s.%s ACC, %s", cc[idx % 6], ty[idx / 6], src_txt(s).c_str());
+    } else if (op >= OP_WHERE_A && op < OP_WHERE_B) {
+        int m = (op - OP_WHERE_A) / LT_VM_NSRC, s = (op - OP_WHERE_A) % LT_VM_NSRC;
+        snprintf(buf, sizeof(buf), "ACC = T%d ? ACC : %s", m, src_txt(s).c_str());
+    } else if (op >= OP_WHERE_B && op < OP_LIMIT) {
+        int m = (op - OP_WHERE_B) / LT_VM_NSRC, s = (op - OP_WHERE_B) % LT_VM_NSRC;
+        snprintf(buf, sizeof(buf), "ACC = T%d ? %s : ACC", m, src_txt(s).c_str());
+    } else snprintf(buf, sizeof(buf), "op%d", op);
+    return buf;
+}
+
+}  // namespace
+
+void fastdiv_make(uint32_t d, uint32_t *mul, uint32_t *sh1, uint32_t *sh2) {
+    // Division of a 32-bit n by invariant d (Granlund & Montgomery 1994): with l = ceil(log2 d) and
+    // m' = floor(2^32 (2^l - d) / d) + 1:  t = mulhi(m', n);  q = (t + ((n - t) >> sh1)) >> sh2.
+    uint32_t l = 0;
+    while (l < 32 && (1ull << l) < d) ++l;
+    uint64_t m = ((1ull << 32) * ((1ull << l) - d)) / d + 1;
+    *mul = (uint32_t)m;
+    *sh1 = l < 1 ? l : 1;
+    *sh2 = l < 1 ? 0 : l - 1;
+}
+
+int broadcast_class(const int64_t *dims, int rank, uint64_t rows, uint64_t cols) {
+    uint64_t ne = 1;
+    for (int i = 0; i < rank; ++i) ne *= (uint64_t)dims[i];
+    uint64_t c = rank ? (uint64_t)dims[rank - 1] : 1;
+    return class_in(c ? ne / c : 0, c, ne, rows, cols);
+}
+
+lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
+    const size_t N = cg.nodes.size();
+    std::vector<PNode> pn(N);
+    const bool fuse = c->opt.fusion != 0;
+
+    for (size_t i = 0; i < N; ++i) {
+        const CNode &n = cg.nodes[i];
+        domain_of(n, &pn[i].rows, &pn[i].cols, &pn[i].numel);
+        pn[i].leaf = n.op == N_DEVICE_DATA || n.op == N_SCALAR;
+        pn[i].reduce = is_reduce(n.op);
+        for (int k = 0; k < n.n_in; ++k) pn[n.in[k]].consumers.push_back((uint32_t)i);
+        if (pn[i].numel == 0) return fail(c, LT_ERR_UNSUPPORTED, "empty tensors cannot be part of a flushed graph");
+    }
+
+    // ---- absorbed nodes: cheap producers recomputed inside every consumer group instead of
+    // being materialised (index/random factories, and computations on broadcast operands)
+    if (fuse) {
+        for (size_t i = 0; i < N; ++i) {
+            const CNode &n = cg.nodes[i];
+            PNode &p = pn[i];
+            if (p.leaf || p.reduce || n.output >= 0 || p.consumers.empty()) continue;
+            bool okc = true;
+            if (is_factory(n.op)) {
+                for (uint32_t cidx : p.consumers) {
+                    const PNode &q = pn[cidx];
+                    uint64_t qr = q.rows, qc = q.cols;
+                    if (q.reduce) { qr = p.rows; qc = p.cols; }
+                    if (qr != p.rows || qc != p.cols) okc = false;
+                }
+            } else {
+                for (uint32_t cidx : p.consumers) {
+                    const PNode &q = pn[cidx];
+                    if (q.reduce || q.numel <= p.numel) okc = false;
+                }
+                for (int k = 0; okc && k < n.n_in; ++k)
+                    if (!pn[n.in[k]].leaf && !pn[n.in[k]].absorbed) okc = false;
+            }
+            p.absorbed = okc;
+        }
+    }
+
+    // ---- native dependencies of each node (through absorbed producers)
+    auto native_deps = [&](uint32_t i, std::vector<uint32_t> &out) {
+        out.clear();
+        std::vector<uint32_t> stack{(uint32_t)i};
+        while (!stack.empty()) {
+            uint32_t n = stack.back();
+            stack.pop_back();
+            const CNode &cn = cg.nodes[n];
+            for (int k = 0; k < cn.n_in; ++k) {
+                uint32_t o = cn.in[k];
+                if (pn[o].leaf) continue;
+                if (pn[o].absorbed) stack.push_back(o);
+                else out.push_back(o);
+            }
+        }
+    };
+
+    // ---- group assignment
+    std::vector<Group> &groups = plan.groups;
+    std::vector<uint32_t> deps;
+    for (size_t i = 0; i < N; ++i) {
+        PNode &p = pn[i];
+        if (p.leaf || p.absorbed) continue;
+        const CNode &n = cg.nodes[i];
+        // the domain the node computes over: a reduction works on its input's rows
+        uint64_t dr = p.rows, dc = p.cols;
+        if (p.reduce) {
+            dr = pn[n.in[0]].rows;
+            dc = pn[n.in[0]].cols;
+        }
+        native_deps((uint32_t)i, deps);
+        int gmin = -1;
+        for (uint32_t d : deps) gmin = std::max(gmin, pn[d].group);
+        int target = -1;
+        if (fuse) {
+            auto joinable = [&](int gi) -> bool {
+                const Group &g = groups[gi];
+                if ((int)g.members.size() >= MAX_GROUP_NODES) return false;
+                if (g.rows == dr && g.cols == dc) return true;
+                // an [R,1] computation on row scalars of a wider group stays with that group
+                if (!p.reduce && p.cols == 1 && p.rows == g.rows && g.cols > 1) {
+                    for (uint32_t d : deps)
+                        if (pn[d].group == gi && pn[d].cols == 1) return true;
+                }
+                return false;
+            };
+            if (gmin >= 0 && joinable(gmin)) {
+                target = gmin;
+                // operands computed in other, older groups of the same domain: pull those groups in,
+                // unless a group in between reads them (it would end up before its producer)
+                for (uint32_t d : deps) {
+                    const int a = pn[d].group;
+                    if (a == target || a < 0) continue;
+                    Group &ga = groups[a];
+                    Group &gb = groups[target];
+                    if (ga.rows != gb.rows || ga.cols != gb.cols) continue;
+                    if (ga.members.size() + gb.members.size() >= (size_t)MAX_GROUP_NODES) continue;
+                    bool legal = true;
+                    for (uint32_t m : ga.members) {
+                        std::vector<uint32_t> stack{m};
+                        while (!stack.empty() && legal) {
+                            uint32_t x = stack.back();
+                            stack.pop_back();
+                            for (uint32_t q : pn[x].consumers) {
+                                if (q >= i) continue;  // not placed yet
+                                if (pn[q].absorbed) stack.push_back(q);
+                                else if (pn[q].group > a && pn[q].group < target) legal = false;
+                            }
+                        }
+                        if (!legal) break;
+                    }
+                    if (!legal) continue;
+                    for (uint32_t m : ga.members) pn[m].group = target;
+                    gb.members.insert(gb.members.end(), ga.members.begin(), ga.members.end());
+                    std::sort(gb.members.begin(), gb.members.end());
+                    ga.members.clear();
+                }
+            } else if (!p.reduce) {
+                // no producer group to join: share a recent group that reads one of the same buffers
+                const int lo = std::max(gmin + 1, (int)groups.size() - 8);
+                for (int gi = (int)groups.size() - 1; gi >= lo && target < 0; --gi) {
+                    const Group &g = groups[gi];
+                    if (g.rows != dr || g.cols != dc || (int)g.members.size() >= MAX_GROUP_NODES) continue;
+                    for (int k = 0; k < n.n_in && target < 0; ++k) {
+                        const uint32_t o = n.in[k];
+                        if (cg.nodes[o].op != N_DEVICE_DATA) continue;
+                        for (uint32_t q : pn[o].consumers)
+                            if (q < i && pn[q].group == gi) {
+                                target = gi;
+                                break;
+                            }
+                    }
+                }
+            }
+        }
+        if (target < 0) {
+            groups.emplace_back();
+            target = (int)groups.size() - 1;
+            groups[target].rows = dr;
+            groups[target].cols = dc;
+        }
+        groups[target].members.push_back((uint32_t)i);
+        p.group = target;
+    }
+
+    // ---- drop groups emptied by merging
+    {
+        size_t w = 0;
+        for (size_t gi = 0; gi < groups.size(); ++gi) {
+            if (groups[gi].members.empty()) continue;
+            if (w != gi) groups[w] = std::move(groups[gi]);
+            for (uint32_t m : groups[w].members) pn[m].group = (int)w;
+            ++w;
+        }
+        groups.resize(w);
+    }
+
+    // ---- code generation (splitting a group that does not fit the machine)
+    std::vector<uint8_t> in_emit(N, 0);
+    std::vector<uint32_t> emit;
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+        for (;;) {
+            Group &g = groups[gi];
+            // which members must reach memory: outputs, and values read by other groups
+            // (recomputed after every split, see below)
+            bool done = false;
+            emission_list(cg, pn, g, emit, in_emit);
+            for (uint32_t m : g.members) {
+                PNode &p = pn[m];
+                p.needs_store = cg.nodes[m].output >= 0;
+            }
+            // consumers in other groups (through absorbed chains)
+            for (uint32_t m : g.members) {
+                std::vector<uint32_t> stack{m};
+                while (!stack.empty() && !pn[m].needs_store) {
+                    uint32_t n = stack.back();
+                    stack.pop_back();
+                    for (uint32_t q : pn[n].consumers) {
+                        if (pn[q].absorbed) stack.push_back(q);
+                        else if (pn[q].group != (int)gi) pn[m].needs_store = true;
+                    }
+                }
+            }
+            int n_inputs = 0;
+            {
+                std::vector<uint32_t> seen;
+                for (uint32_t n : emit) {
+                    const CNode &cn = cg.nodes[n];
+                    for (int k = 0; k < cn.n_in; ++k) {
+                        uint32_t o = cn.in[k];
+                        if (!in_emit[o] && cg.nodes[o].op != N_SCALAR && std::find(seen.begin(), seen.end(), o) == seen.end())
+                            seen.push_back(o);
+                    }
+                }
+                n_inputs = (int)seen.size();
+            }
+            for (int pre = std::min(n_inputs, LT_VM_NT); pre >= 0 && !done; --pre) {
+                g.ins.clear();
+                g.io.clear();
+                g.imms.clear();
+                CodeGen cgen(cg, pn, g, (int)gi, emit, in_emit);
+                if (cgen.run(pre)) {
+                    done = true;
+                    g.kind = cgen.has_reduce ? K_ROW : K_EW;
+                    g.rowcol = cgen.needs_rowcol;
+                    bool fast = c->opt.fast_math != 0;
+                    bool any_store = false;
+                    for (const IoRef &io : g.io) {
+                        if (!io.is_store) continue;
+                        any_store = true;
+                        if (io.dtype == LT_F32) fast = false;
+                        else if (io.dtype != LT_BF16 && cgen.tainted[io.cnode]) fast = false;
+                    }
+                    g.fast = fast && any_store;
+                }
+            }
+            for (uint32_t n : emit) in_emit[n] = 0;
+            if (done) break;
+            if (g.members.size() <= 1) return fail(c, LT_ERR_UNSUPPORTED, "an operation does not fit the register program limits");
+            // split: the later half of the members moves to a new group right after this one
+            size_t half = g.members.size() / 2;
+            Group tail;
+            tail.rows = g.rows;
+            tail.cols = g.cols;
+            tail.members.assign(g.members.begin() + half, g.members.end());
+            g.members.resize(half);
+            groups.insert(groups.begin() + gi + 1, std::move(tail));
+            for (size_t k = gi + 1; k < groups.size(); ++k)
+                for (uint32_t m : groups[k].members) pn[m].group = (int)k;
+            // a row-scalar member that lost its reduction partner keeps the group's domain; fine
+        }
+    }
+
+    // ---- number temporaries and patch the slots that refer to them
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+        Group &g = groups[gi];
+        for (IoRef &io : g.io) {
+            if (io.kind != IO_TEMP) continue;
+            PNode &p = pn[io.cnode];
+            if (p.temp < 0) {
+                p.temp = (int)plan.temp_bytes.size();
+                plan.temp_bytes.push_back((size_t)p.numel * dtype_size(cg.nodes[io.cnode].dtype));
+            }
+            io.index = (uint32_t)p.temp;
+        }
+        g.bytes = 0;
+        for (const IoRef &io : g.io) g.bytes += io_bytes(g, io);
+        if (g.kind == K_ROW && g.cols > (uint64_t)LT_VM_V * 1024)
+            return fail(c, LT_ERR_UNSUPPORTED, "row-reduction groups support rows of at most 8192 elements");
+        if (g.kind == K_EW && g.rowcol) {
+            uint64_t cpr = (g.cols + LT_VM_V - 1) / LT_VM_V;
+            if (g.rows * cpr >= (1ull << 32) || g.rows >= (1ull << 32) || g.cols >= (1ull << 32))
+                return fail(c, LT_ERR_UNSUPPORTED, "broadcast group too large for 32-bit chunk indexing");
+        }
+        if (g.kind == K_ROW && g.rows >= (1ull << 32)) return fail(c, LT_ERR_UNSUPPORTED, "too many rows");
+    }
+
+    // ---- outputs
+    plan.n_params = (uint32_t)cg.param_node.size();
+    plan.n_dyn = (uint32_t)cg.dyn.size();
+    plan.outputs.resize(cg.outputs.size());
+    for (size_t k = 0; k < cg.outputs.size(); ++k) {
+        const CNode &n = cg.nodes[cg.outputs[k]];
+        OutputPlan &o = plan.outputs[k];
+        o.dtype = n.dtype;
+        o.rank = n.rank;
+        memcpy(o.dims, n.dims, sizeof(o.dims));
+        o.bytes = (size_t)pn[cg.outputs[k]].numel * dtype_size(n.dtype);
+        o.donated_param = -1;
+    }
+
+    // ---- launches: bundle isomorphic independent flat groups (horizontal fusion)
+    std::vector<int> launch_of(groups.size(), -1);
+    {
+        // outputs that some group loads: their producers cannot move
+        std::vector<uint8_t> output_loaded(cg.outputs.size(), 0);
+        for (const Group &g : groups)
+            for (const IoRef &io : g.io)
+                if (!io.is_store && io.kind == IO_OUTPUT) output_loaded[io.index] = 1;
+        std::map<std::string, std::vector<uint32_t>> buckets;
+        std::vector<std::string> sig(groups.size());
+        if (fuse && c->opt.horizontal) {
+            for (size_t gi = 0; gi < groups.size(); ++gi) {
+                const Group &g = groups[gi];
+                bool el = g.kind == K_EW && !g.rowcol && g.ins.size() <= LT_MULTI_MAX_INS && g.io.size() <= LT_MULTI_MAX_SLOTS &&
+                          g.rows * g.cols < (1ull << 32);
+                for (const IoRef &io : g.io) {
+                    if (io.cls != LT_CLS_FULL) el = false;
+                    if (io.is_store ? (io.kind != IO_OUTPUT || output_loaded[io.index]) : io.kind != IO_PARAM) el = false;
+                }
+                if (!el) continue;
+                std::string s;
+                s.push_back(g.fast ? 'f' : 'p');
+                s.append((const char *)g.ins.data(), g.ins.size() * sizeof(LtIns));
+                for (const Imm &im : g.imms) {
+                    s.append((const char *)&im.dyn, sizeof(im.dyn));
+                    s.append((const char *)&im.sval, sizeof(im.sval));
+                    s.push_back((char)im.enc);
+                }
+                for (const IoRef &io : g.io) {
+                    s.push_back((char)io.dtype);
+                    s.push_back((char)io.is_store);
+                }
+                sig[gi] = s;
+                buckets[s].push_back((uint32_t)gi);
+            }
+        }
+        for (size_t gi = 0; gi < groups.size(); ++gi) {
+            if (launch_of[gi] >= 0) continue;
+            const Group &g = groups[gi];
+            auto it = sig[gi].empty() ? buckets.end() : buckets.find(sig[gi]);
+            if (it != buckets.end() && it->second.size() >= 2) {
+                const std::vector<uint32_t> &all = it->second;
+                size_t pos = 0;
+                const size_t slots = g.io.size();
+                const size_t per = std::min<size_t>(LT_MULTI_MAX_INST, LT_MULTI_MAX_PTRS / std::max<size_t>(slots, 1));
+                while (pos < all.size()) {
+                    Launch L;
+                    L.kind = K_MULTI;
+                    L.fast = g.fast;
+                    size_t cnt = std::min(per, all.size() - pos);
+                    for (size_t k = 0; k < cnt; ++k) {
+                        L.groups.push_back(all[pos + k]);
+                        launch_of[all[pos + k]] = (int)plan.launches.size();
+                        L.bytes += groups[all[pos + k]].bytes;
+                    }
+                    pos += cnt;
+                    plan.launches.push_back(std::move(L));
+                }
+            } else {
+                Launch L;
+                L.kind = g.kind;
+                L.fast = g.fast;
+                L.groups.push_back((uint32_t)gi);
+                L.bytes = g.bytes;
+                launch_of[gi] = (int)plan.launches.size();
+                plan.launches.push_back(std::move(L));
+            }
+        }
+    }
+
+    // ---- donation (Section 4.3): write an output into the parameter buffer its tensor used to
+    // name when every read of that buffer is by the writing program itself, at the same element
+    // and before the store, or by an earlier launch
+    {
+        std::vector<std::vector<std::pair<uint32_t, uint32_t>>> readers(plan.n_params);  // (group, slot)
+        for (size_t gi = 0; gi < groups.size(); ++gi)
+            for (size_t s = 0; s < groups[gi].io.size(); ++s) {
+                const IoRef &io = groups[gi].io[s];
+                if (!io.is_store && io.kind == IO_PARAM) readers[io.index].push_back({(uint32_t)gi, (uint32_t)s});
+            }
+        for (size_t gi = 0; gi < groups.size(); ++gi) {
+            Group &g = groups[gi];
+            for (size_t s = 0; s < g.io.size(); ++s) {
+                const IoRef &st = g.io[s];
+                if (!st.is_store || st.kind != IO_OUTPUT) continue;
+                int32_t p = cg.donor_param[st.index];
+                if (p < 0 || st.cls != LT_CLS_FULL) continue;
+                bool safe = true;
+                for (auto &rd : readers[p]) {
+                    const uint32_t rg = rd.first;
+                    if (rg == gi) {
+                        const IoRef &ld = groups[rg].io[rd.second];
+                        if (ld.cls != LT_CLS_FULL) { safe = false; break; }
+                        // the load must come before the store in program order
+                        int ld_pos = -1, st_pos = -1;
+                        for (size_t q = 0; q < g.ins.size(); ++q) {
+                            const LtIns &in = g.ins[q];
+                            if (in.op >= OP_LD_T && in.op <= OP_LD_ACC && in.imm == rd.second && ld_pos < 0) ld_pos = (int)q;
+                            if (in.op == OP_ST && in.imm == s) st_pos = (int)q;
+                        }
+                        if (ld_pos < 0 || st_pos < 0 || ld_pos > st_pos) { safe = false; break; }
+                    } else if (launch_of[rg] >= launch_of[gi]) {
+                        safe = false;
+                        break;
+                    }
+                }
+                if (safe) plan.outputs[st.index].donated_param = p;
+            }
+        }
+    }
+
+    // ---- parameter blocks: everything that does not change between hits is filled in now
+    for (Launch &L : plan.launches) {
+        if (L.kind == K_MULTI) {
+            L.mp.reset(new LtMultiParams());
+            LtMultiParams &P = *L.mp;
+            memset(&P, 0, sizeof(P));
+            const Group &g0 = groups[L.groups[0]];
+            P.n_ins = (uint32_t)g0.ins.size();
+            memcpy(P.ins, g0.ins.data(), g0.ins.size() * sizeof(LtIns));
+            P.n_slots = (uint32_t)g0.io.size();
+            for (size_t s = 0; s < g0.io.size(); ++s) P.io_dtype[s] = g0.io[s].dtype;
+            P.n_inst = (uint32_t)L.groups.size();
+            const uint32_t per_super = LT_EW_THREADS * LT_MULTI_SUB * LT_VM_V;
+            uint32_t acc = 0;
+            for (size_t k = 0; k < L.groups.size(); ++k) {
+                const Group &g = groups[L.groups[k]];
+                uint32_t ne = (uint32_t)(g.rows * g.cols);
+                P.super_prefix[k] = acc;
+                P.numel[k] = ne;
+                acc += (ne + per_super - 1) / per_super;
+            }
+            P.super_prefix[L.groups.size()] = acc;
+            P.total_super = acc;
+        } else {
+            L.kp.reset(new LtKParams());
+            LtKParams &P = *L.kp;
+            memset(&P, 0, sizeof(P));
+            const Group &g = groups[L.groups[0]];
+            P.n_ins = (uint32_t)g.ins.size();
+            memcpy(P.ins, g.ins.data(), g.ins.size() * sizeof(LtIns));
+            for (size_t s = 0; s < g.io.size(); ++s) {
+                P.io_dtype[s] = g.io[s].dtype;
+                P.io_class[s] = g.io[s].cls;
+            }
+            P.n = g.rows * g.cols;
+            P.rowcol = g.rowcol ? 1u : 0u;
+            P.rows = (uint32_t)g.rows;
+            P.cols = (uint32_t)g.cols;
+            P.cpr = (uint32_t)((g.cols + LT_VM_V - 1) / LT_VM_V);
+            fastdiv_make(P.cpr ? P.cpr : 1, &P.div_mul, &P.div_sh1, &P.div_sh2);
+            P.n_chunks = g.rowcol ? (uint64_t)g.rows * P.cpr : (P.n + LT_VM_V - 1) / LT_VM_V;
+            if (g.kind == K_ROW) {
+                uint32_t grp = 1, lg = 0;
+                while (grp < P.cpr) grp <<= 1, ++lg;
+                P.group = grp;
+                P.group_log2 = lg;
+                L.threads = grp > 256 ? grp : 256;
+                P.rows_per_cta = L.threads / grp;
+            }
+        }
+    }
+    return LT_OK;
+}
+
+std::string describe_plan(const Plan &plan) {
+    std::string s;
+    char buf[256];
+    snprintf(buf, sizeof(buf), "plan: %zu launches, %zu groups, %u params, %u runtime slots, %zu outputs, %zu temporaries\n",
+             plan.launches.size(), plan.groups.size(), plan.n_params, plan.n_dyn, plan.outputs.size(), plan.temp_bytes.size());
+    s += buf;
+    for (size_t k = 0; k < plan.outputs.size(); ++k)
+        if (plan.outputs[k].donated_param >= 0) {
+            snprintf(buf, sizeof(buf), "  output %zu donated param %d\n", k, plan.outputs[k].donated_param);
+            s += buf;
+        }
+    static const char *kind[] = {"elementwise", "row", "multi"};
+    static const char *cls[] = {"full", "colvec", "rowvec", "scalar"};
+    static const char *iok[] = {"param", "output", "temp"};
+    for (size_t li = 0; li < plan.launches.size(); ++li) {
+        const Launch &L = plan.launches[li];
+        const Group &g = plan.groups[L.groups[0]];
+        snprintf(buf, sizeof(buf), "launch %zu: %s %s instances=%zu rows=%llu cols=%llu %s bytes=%llu\n", li, kind[L.kind],
+                 L.fast ? "fast" : "precise", L.groups.size(), (unsigned long long)g.rows, (unsigned long long)g.cols,
+                 g.rowcol ? "rowcol" : "flat", (unsigned long long)L.bytes);
+        s += buf;
+        for (size_t q = 0; q < g.io.size(); ++q) {
+            const IoRef &io = g.io[q];
+            snprintf(buf, sizeof(buf), "  p%zu: %s %s %s %s%u\n", q, io.is_store ? "store" : "load", dtype_name(io.dtype),
+                     cls[io.cls], iok[io.kind], io.index);
+            s += buf;
+        }
+        for (size_t q = 0; q < g.imms.size(); ++q) {
+            const Imm &im = g.imms[q];
+            if (im.dyn >= 0) snprintf(buf, sizeof(buf), "  S%zu: runtime slot %d enc %d\n", q, im.dyn, im.enc);
+            else snprintf(buf, sizeof(buf), "  S%zu: const %g enc %d\n", q, im.sval, im.enc);
+            s += buf;
+        }
+        for (size_t q = 0; q < g.ins.size(); ++q) {
+            snprintf(buf, sizeof(buf), "  %3zu  ", q);
+            s += buf;
+            s += disasm(g.ins[q]);
+            s += "\n";
+        }
+    }
+    return s;
+}
+
+}  // namespace lt

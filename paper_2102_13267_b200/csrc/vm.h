@@ -1,0 +1,113 @@
+// Register-program virtual machine shared by the planner (host) and the kernels (device).
+//
+// A fusion group runs as one kernel in which every thread owns a chunk of LT_VM_V
+// consecutive elements of a row and interprets the group's program on them.  The
+// machine is an accumulator machine: ACC plus LT_VM_NT temporaries, each LT_VM_V
+// 32-bit lanes wide (f32 values, or i32/u32/u8 values held as integers).  Every
+// (operation, operand source) pair has its own opcode so that one warp-uniform jump
+// reaches straight-line code that names its registers statically -- a register file
+// indexed at run time would live in local memory.
+#pragma once
+#include <stdint.h>
+
+#define LT_VM_V 8          // lanes per chunk
+#define LT_EW_THREADS 256  // CTA size of the elementwise and multi-tensor kernels
+#define LT_VM_NT 4         // temporaries T0..T3
+#define LT_VM_NSRC 5       // operand sources of two-operand opcodes: T0..T3, S (broadcast immediate)
+#define LT_VM_SRC_S 4
+#define LT_VM_MAX_INS 120
+#define LT_VM_MAX_PTR 12
+#define LT_VM_MAX_SCAL 32
+
+#define LT_MULTI_MAX_INS 64
+#define LT_MULTI_MAX_INST 384   // instances (tensors) per multi-tensor launch
+#define LT_MULTI_MAX_PTRS 2816  // pointer-table entries per launch (instances x slots)
+#define LT_MULTI_MAX_SLOTS 8
+#define LT_MULTI_SUB 4          // chunks each thread runs per super-chunk
+
+struct LtIns {
+    uint16_t op;
+    uint8_t a;     // small operand: dtype for CVT
+    uint8_t b;
+    uint32_t imm;  // pointer slot, immediate slot
+};
+
+// element classes of a pointer slot relative to the group's [rows, cols] domain
+enum { LT_CLS_FULL = 0, LT_CLS_COLVEC = 1, LT_CLS_ROWVEC = 2, LT_CLS_SCALAR = 3 };
+// storage dtypes (same numbering as lt_dtype)
+enum { LT_ST_F32 = 0, LT_ST_BF16 = 1, LT_ST_U8 = 2, LT_ST_I32 = 3, LT_ST_U32 = 4 };
+
+enum {
+    OP_END = 0,
+    OP_MOV_T_ACC = 1,    // +k : T[k] = ACC
+    OP_MOV_ACC_T = 5,    // +k : ACC = T[k]
+    OP_MOV_ACC_S = 9,    // ACC = broadcast(imm slot)
+    OP_LD_T = 10,        // +k : T[k] = raw chunk of pointer slot imm (storage format, see CVT)
+    OP_LD_ACC = 14,
+    OP_CVT_T = 15,       // +k : widen the raw chunk in T[k] from storage dtype `a` to 32-bit lanes
+    OP_CVT_ACC = 19,
+    OP_ST = 20,          // store ACC to pointer slot imm, narrowing to the slot's dtype
+    OP_IOTA_COL = 21,    // ACC = column index of each lane (i32)
+    OP_IOTA_ROW = 22,    // ACC = (row / scal[imm]) % scal[imm+1] (i32), same in every lane
+    OP_PHILOX = 23,      // ACC = random bits of each lane's flat index; scal[imm..imm+3] = seed lo,hi, offset lo,hi
+    OP_RED_SUM = 24,     // ACC = sum over the row, broadcast to every lane   (row kernel only)
+    OP_RED_MAX = 25,
+    OP_RED_MIN = 26,
+    // one-operand float ops on ACC
+    OP_U_NEG = 30, OP_U_ABS, OP_U_RELU, OP_U_EXP, OP_U_LOG, OP_U_TANH, OP_U_SQRT, OP_U_RSQRT, OP_U_RECIP,
+    OP_U_SQUARE, OP_U_SIGMOID, OP_U_GELU, OP_U_RBF16 /* round to bf16, keep as f32 */,
+    OP_U_INEG = 43, OP_U_IABS = 44, OP_U_NOT = 45,
+    OP_C_I2F = 46, OP_C_U2F = 47, OP_C_F2I = 48, OP_C_NZF = 49 /* f32 != 0 -> 0/1 */, OP_C_NZI = 50,
+    // two-operand families: opcode = base + index * LT_VM_NSRC + source
+    OP_F2 = 64,          // ACC = ACC (op) src, f32: see F2_*
+    OP_I2 = 104,         // integer: see I2_*
+    OP_CMP = 160,        // ACC = (ACC cmp src) ? 1 : 0 : see CMP_*
+    OP_WHERE_A = 256,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? ACC : src
+    OP_WHERE_B = 276,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? src : ACC
+    OP_LIMIT = 296
+};
+
+enum { F2_ADD = 0, F2_SUB, F2_RSUB, F2_MUL, F2_DIV, F2_RDIV, F2_MAX, F2_MIN, F2_COUNT };
+enum { I2_ADD = 0, I2_SUB, I2_RSUB, I2_MUL, I2_AND, I2_OR, I2_XOR, I2_MAXS, I2_MINS, I2_MAXU, I2_MINU, I2_COUNT };
+// compare index = type * 6 + cc ; type 0 f32, 1 signed, 2 unsigned ; cc: GT GE LT LE EQ NE
+enum { CC_GT = 0, CC_GE, CC_LT, CC_LE, CC_EQ, CC_NE };
+
+static_assert(OP_F2 + F2_COUNT * LT_VM_NSRC == OP_I2, "opcode map");
+static_assert(OP_I2 + I2_COUNT * LT_VM_NSRC <= OP_CMP, "opcode map");
+static_assert(OP_CMP + 18 * LT_VM_NSRC <= OP_WHERE_A, "opcode map");
+
+// Kernel parameter block of the elementwise and row-reduction kernels.  It is passed by
+// value as a __grid_constant__ kernel parameter, so program, pointers and immediates are
+// read from the constant bank with no separate upload.
+struct LtKParams {
+    uint64_t ptr[LT_VM_MAX_PTR];
+    uint32_t scal[LT_VM_MAX_SCAL];
+    LtIns ins[LT_VM_MAX_INS];
+    uint8_t io_dtype[LT_VM_MAX_PTR];
+    uint8_t io_class[LT_VM_MAX_PTR];
+    uint32_t n_ins;
+    uint32_t rowcol;        // 0: flat chunks over n elements; 1: chunks stay inside rows
+    uint64_t n;             // rows * cols
+    uint32_t rows, cols;    // rowcol only
+    uint32_t cpr;           // chunks per row = ceil(cols / V)
+    uint32_t div_mul, div_sh1, div_sh2;  // row = chunk / cpr without a divide
+    uint64_t n_chunks;
+    // row kernel geometry
+    uint32_t group;         // threads per row (power of two)
+    uint32_t group_log2;
+    uint32_t rows_per_cta;
+};
+
+// Parameter block of the multi-tensor kernel: one program, many instances.
+struct LtMultiParams {
+    LtIns ins[LT_MULTI_MAX_INS];
+    uint32_t scal[LT_VM_MAX_SCAL];
+    uint8_t io_dtype[LT_MULTI_MAX_SLOTS];
+    uint32_t n_ins;
+    uint32_t n_inst;
+    uint32_t n_slots;
+    uint32_t total_super;                          // total super-chunks
+    uint32_t super_prefix[LT_MULTI_MAX_INST + 1];  // super-chunks before instance i
+    uint32_t numel[LT_MULTI_MAX_INST];
+    uint64_t ptr[LT_MULTI_MAX_PTRS];               // [instance * n_slots + slot]
+};

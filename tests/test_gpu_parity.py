@@ -1,0 +1,167 @@
+"""GPU parity: the CUDA library against the CPU eager oracle, element by element, on the same
+seeded inputs, through the C ABI (ctypes binding)."""
+import math
+
+import numpy as np
+import pytest
+
+from helpers import assert_matches
+from oracle.eager import EagerOracle, set_threads, max_threads
+from workloads import configs, rng, traces
+from workloads.resnet50 import parameter_shapes
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lt():
+    import paper_2102_13267_b200 as lt
+    set_threads(max_threads())
+    return lt
+
+
+@pytest.fixture()
+def ctx(lt):
+    c = lt.LazyContext(device=0)
+    yield c
+    c.close()
+
+
+def both(ctx, arrays_dtypes):
+    """Leaves for the oracle and for the library from the same arrays."""
+    O = EagerOracle()
+    return O, [O.leaf(a, d) for a, d in arrays_dtypes], [ctx.leaf(a, d) for a, d in arrays_dtypes]
+
+
+# ------------------------------------------------------------------ C1
+@pytest.mark.parametrize("shape", [(1, 1), (3, 5), (37, 19), (64, 64), (1000,), (2051,), (256, 257), (1024, 1024)])
+def test_c1_chain(ctx, shape):
+    ins = [(a, "f32") for a in configs.c1_inputs(1, shape)]
+    O, ol, gl = both(ctx, ins)
+    ref = traces.elementwise_chain(O, *ol)
+    for it in range(10):
+        y = traces.elementwise_chain(ctx, *gl)
+        ctx.barrier()
+        if it in (0, 9):
+            assert_matches(ctx.fetch(y), ref.array, "f32", f"c1 {shape}", exact=True)
+        del y
+    s = ctx.stats()
+    assert (s["compiles"], s["cache_hits"]) == (1, 9)
+    assert s["kernels_launched"] == 10
+
+
+# ------------------------------------------------------------------ C2
+@pytest.mark.parametrize("shape", [(33, 40), (17, 36), (1, 8), (5, 7), (128, 4096), (8192, 4096)])
+@pytest.mark.parametrize("primitive", [True, False])
+def test_c2_mlp_epilogue(ctx, shape, primitive):
+    if shape == (8192, 4096) and not primitive:
+        pytest.skip("full size runs the primitive trace")
+    x, h, b = configs.c2_inputs(2, shape)
+    O, ol, gl = both(ctx, [(x, "bf16"), (h, "bf16"), (b, "bf16")])
+    ref = traces.mlp_epilogue(O, *ol, primitive_gelu=primitive)
+    out = traces.mlp_epilogue(ctx, *gl, primitive_gelu=primitive)
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1
+    assert_matches(ctx.fetch(out), ref.array, "bf16", f"c2 {shape}")
+
+
+# ------------------------------------------------------------------ C3
+@pytest.mark.parametrize("shape", [(32, 256), (5, 1024), (7, 48), (3, 1000), (2, 2048), (2, 4096), (3, 8192), (9, 8),
+                                   (4, 3, 64), (16384, 1024)])
+@pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
+def test_c3_residual_dropout_layernorm(ctx, shape, out_dtype):
+    if shape == (16384, 1024) and out_dtype == "f32":
+        pytest.skip("full size runs the bf16 variant")
+    x, h, g, b = configs.c3_inputs(3, shape)
+    O, ol, gl = both(ctx, [(x, "bf16"), (h, "bf16"), (g, "f32"), (b, "f32")])
+    kw = dict(shape=shape, p=0.1, eps=1e-5, seed=0xDEADBEEF12345, offset=7, out_dtype=out_dtype)
+    zr, kr = traces.residual_dropout_layernorm(O, *ol, **kw)
+    z, k = traces.residual_dropout_layernorm(ctx, *gl, **kw)
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1
+    assert_matches(ctx.fetch(k), kr.array, "u8", f"c3 mask {shape}")
+    assert_matches(ctx.fetch(z), zr.array, out_dtype, f"c3 z {shape}")
+    # a new offset gives a new mask without a recompile
+    kw["offset"] = 8
+    z2, k2 = traces.residual_dropout_layernorm(ctx, *gl, **kw)
+    _, kr2 = traces.residual_dropout_layernorm(O, *ol, **kw)
+    assert_matches(ctx.fetch(k2), kr2.array, "u8", "c3 mask, second offset")
+    s = ctx.stats()
+    assert (s["compiles"], s["cache_hits"]) == (1, 1)
+
+
+# ------------------------------------------------------------------ C4
+@pytest.mark.parametrize("shape", [(2, 64, 64), (1, 130, 130), (3, 24, 24), (1, 8, 8), (2, 1000, 1000), (1, 4, 2048),
+                                   (16, 2048, 2048)])
+@pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
+def test_c4_causal_softmax(ctx, shape, out_dtype):
+    if shape == (16, 2048, 2048) and out_dtype == "f32":
+        pytest.skip("full size runs the bf16 variant")
+    s = configs.c4_inputs(4, shape)
+    O, ol, gl = both(ctx, [(s, "bf16")])
+    kw = dict(shape=shape, scale=1.0 / math.sqrt(128.0), out_dtype=out_dtype)
+    ref = traces.causal_softmax(O, *ol, **kw)
+    y = traces.causal_softmax(ctx, *gl, **kw)
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1
+    got = ctx.fetch(y)
+    assert_matches(got, ref.array, out_dtype, f"c4 {shape}")
+    # masked entries are exactly +0
+    q, k = shape[-2], shape[-1]
+    iu = np.triu_indices(q, 1, k)
+    assert (got[..., iu[0], iu[1]] == 0).all()
+
+
+# ------------------------------------------------------------------ C5
+def _adam_case(ctx, shapes, steps, check_every=1):
+    params, grads, ms, vs = configs.c5_inputs(5, shapes)
+    O = EagerOracle()
+    op, og, om, ov = ([O.leaf(a, "f32") for a in arrs] for arrs in (params, grads, ms, vs))
+    gp, gg, gm, gv = ([ctx.leaf(a, "f32") for a in arrs] for arrs in (params, grads, ms, vs))
+    ptrs = [ctx.device_ptr(t) for t in gp + gm + gv]
+    for step in range(1, steps + 1):
+        traces.adam_step(O, op, og, om, ov, step=step)
+        traces.adam_step(ctx, gp, gg, gm, gv, step=step)
+        ctx.barrier()
+        if step % check_every == 0 or step == steps:
+            for i in range(len(shapes)):
+                for name, a, b in (("p", gp[i], op[i]), ("m", gm[i], om[i]), ("v", gv[i], ov[i])):
+                    assert_matches(ctx.fetch(a), b.array, "f32", f"c5 step {step} {name}[{i}] {shapes[i]}")
+    # in-place: every parameter, m and v still lives in its original buffer (donation)
+    assert [ctx.device_ptr(t) for t in gp + gm + gv] == ptrs
+    s = ctx.stats()
+    assert (s["compiles"], s["cache_hits"]) == (1, steps - 1)
+    assert s["outputs_allocated"] == 0 and s["outputs_donated"] == 3 * len(shapes) * steps
+    return s
+
+
+def test_c5_adam_small(ctx):
+    shapes = parameter_shapes()[:14] + [(1000,), (7,), (3, 5, 1, 1)]
+    s = _adam_case(ctx, shapes, steps=4)
+    assert s["kernels_launched"] == 4  # one multi-tensor launch per step
+
+
+def test_c5_adam_full_shapes(ctx):
+    s = _adam_case(ctx, parameter_shapes(), steps=3, check_every=3)
+    assert s["kernels_launched"] == 3 and s["launches_multi"] == 3
+    assert s["bytes_planned"] == 3 * 715_596_896
+
+
+# ------------------------------------------------------------------ unfused baseline
+def test_unfused_matches_oracle(ctx):
+    ctx.set_option("fusion", 0)
+    shape = (6, 136)
+    x, h, g, b = configs.c3_inputs(6, shape)
+    O, ol, gl = both(ctx, [(x, "bf16"), (h, "bf16"), (g, "f32"), (b, "f32")])
+    kw = dict(shape=shape, p=0.1, eps=1e-5, seed=3, offset=1)
+    zr, kr = traces.residual_dropout_layernorm(O, *ol, **kw)
+    z, k = traces.residual_dropout_layernorm(ctx, *gl, **kw)
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] >= 15  # one kernel per traced op
+    assert_matches(ctx.fetch(k), kr.array, "u8", "unfused mask")
+    assert_matches(ctx.fetch(z), zr.array, "bf16", "unfused z")
+    s = configs.c4_inputs(6, (2, 40, 40))
+    O, ol, gl = both(ctx, [(s, "bf16")])
+    ref = traces.causal_softmax(O, *ol, shape=(2, 40, 40), scale=0.1)
+    y = traces.causal_softmax(ctx, *gl, shape=(2, 40, 40), scale=0.1)
+    assert_matches(ctx.fetch(y), ref.array, "bf16", "unfused softmax")
