@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-graph executor.
+
+A step is one pass of the whole path over one batch: trace the MLP-epilogue graph
+(out = x + GELU_tanh(h + bias), bf16 [8192 x 4096], fp32 arithmetic), barrier (canonicalise,
+hash, cache lookup, bind, launch), with the inputs already resident in HBM.  The metric is
+HBM GB/s = algorithmic bytes (each input read once, the output written once) / time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs the same
+per-GPU workload on its own buffers -- the path has no exchange step -- and the value is the
+sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "fused-graph HBM GB/s"
+UNIT = "GB/s"
+WORKLOAD = "c2_mlp_epilogue_bf16_8192x4096"
+SHAPE = (8192, 4096)
+N_SETS = 6  # rotating input/output sets: 6 x 201 MB > L2 (126 MB), so every step streams from HBM
+FALLBACK_HBM_GBS = 6650.0
+
+_SAMPLER = r"""
+import sys, time
+import pynvml as nv
+nv.nvmlInit()
+h = nv.nvmlDeviceGetHandleByIndex(int(sys.argv[1]))
+mx = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+print("max", mx, flush=True)
+while True:
+    try:
+        r = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+    except Exception:
+        r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+    print(time.time(), nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM), int(r), flush=True)
+    time.sleep(0.004)
+"""
+
+_REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+            0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost",
+            0x100: "display_clock_setting"}
+
+
+class ClockSampler:
+    """Reads SM clock and throttle reasons (read-only NVML queries) from a child process."""
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen([sys.executable, "-c", _SAMPLER, str(device_index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.02)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        mx, inside, all_ = None, [], []
+        for ln in out.splitlines():
+            p = ln.split()
+            if len(p) == 2 and p[0] == "max":
+                mx = float(p[1])
+            elif len(p) == 3:
+                rec = (float(p[0]), float(p[1]), int(p[2]))
+                all_.append(rec)
+                if t0 <= rec[0] <= t1:
+                    inside.append(rec)
+        use = inside or all_[-3:]
+        reasons = set()
+        for _, _, r in use:
+            for bit, name in _REASONS.items():
+                if r & bit:
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median([c for _, c, _ in use]) if use else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(inside)}
+
+
+def measured_peak() -> tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, STREAM-style copy)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+def ncu_traffic() -> float | None:
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if it is current."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+        return float(rec[WORKLOAD]["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
+# --------------------------------------------------------------------------- oracle arm
+class OracleRun:
+    """The CPU eager oracle (one op at a time, as it stands) on the first `rows` rows of the workload."""
+
+    def __init__(self, rows: int, threads: int):
+        from oracle import eager
+        from workloads import configs
+
+        eager.set_threads(threads)
+        x, h, b = configs.c2_inputs(0, (rows, SHAPE[1]))
+        self.O = eager.EagerOracle()
+        self.leaves = (self.O.leaf(x, "bf16"), self.O.leaf(h, "bf16"), self.O.leaf(b, "bf16"))
+        self.rows = rows
+        self.nbytes = configs.algorithmic_bytes("c2", (rows, SHAPE[1]))
+
+    def step(self) -> float:
+        from workloads import traces
+
+        t0 = time.perf_counter()
+        traces.mlp_epilogue(self.O, *self.leaves, primitive_gelu=False)
+        return time.perf_counter() - t0
+
+
+def cpu_baseline(budget_s: float = 12.0) -> dict:
+    from oracle import eager
+
+    threads = eager.max_threads()
+    probe = OracleRun(256, threads)
+    probe.step()
+    t_row = probe.step() / 256
+    rows = int(min(SHAPE[0], max(256, budget_s / max(t_row, 1e-9))))
+    run = OracleRun(rows, threads)
+    run.step()
+    passes = int(max(1, min(50, budget_s / max(t_row * rows, 1e-6))))
+    sec = sum(run.step() for _ in range(passes))
+    return {"value": run.nbytes * passes / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{rows} of {SHAPE[0]} rows of the workload, {passes} passes, {sec:.2f} s, OpenMP over elements"}
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import eager
+
+    threads = eager.max_threads()
+    probe = OracleRun(256, threads)
+    probe.step()
+    t_row = probe.step() / 256
+    total = max(1, args.steps + args.warmup)
+    rows = int(max(1, min(SHAPE[0], 90.0 / total / max(t_row, 1e-9))))
+    run = OracleRun(rows, threads)
+    for _ in range(args.warmup):
+        run.step()
+    sec = sum(run.step() for _ in range(args.steps))
+    value = run.nbytes * args.steps / sec / 1e9
+    sample = f"each step: {rows} of {SHAPE[0]} rows of the workload through the CPU eager oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sec / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "trace": "convert x3, add, gelu_tanh, add, convert", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args) -> None:
+    import torch
+    import torch.distributed as dist
+
+    import paper_2102_13267_b200 as lt
+    from workloads import configs, traces
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    ctx = lt.LazyContext(device=local)
+    nbytes = configs.algorithmic_bytes("c2", SHAPE)
+
+    # seeded synthetic inputs: one host draw per rank, shifted copies for the other sets
+    x, h, b = configs.c2_inputs(1000 + rank, SHAPE)
+    tx = torch.from_numpy(x.view(np.int16)).to(dev).view(torch.bfloat16)
+    th = torch.from_numpy(h.view(np.int16)).to(dev).view(torch.bfloat16)
+    tb = torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
+    sets = []
+    for s in range(N_SETS):
+        xs = torch.roll(tx, shifts=s, dims=0).contiguous() if s else tx
+        hs = torch.roll(th, shifts=-s, dims=0).contiguous() if s else th
+        sets.append((ctx.from_torch(xs), ctx.from_torch(hs), ctx.from_torch(tb.clone())))
+    outs = [None] * N_SETS
+
+    def step(i: int, primitive: bool = False) -> None:
+        X, H, Bv = sets[i % N_SETS]
+        outs[i % N_SETS] = traces.mlp_epilogue(ctx, X, H, Bv, primitive_gelu=primitive)
+        ctx.barrier()
+
+    def sync_all() -> None:
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(n_steps: int, fn) -> float:
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n_steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    sampler = ClockSampler(local) if rank == 0 else None
+    sync_all()
+    ctx.reset_stats()
+    ctx.set_kernel_timing(True)
+    ctx.kernel_timing()
+    w0 = time.time()
+    ms = timed(args.steps, step)
+    w1 = time.time()
+    kt = ctx.kernel_timing()
+    ctx.set_kernel_timing(False)
+    st = ctx.stats()
+    clocks = sampler.stop(w0, w1) if sampler else None
+    value = world * nbytes * args.steps / (ms / 1e3) / 1e9
+
+    # ---- end to end through the C ABI with host buffers: H2D of the inputs and D2H of the result every step
+    e2e_steps = max(3, min(args.steps, 30))
+    pin = [torch.from_numpy(a.view(np.int16)).pin_memory() for a in (x, h, b)]
+    host_out = torch.empty(SHAPE, dtype=torch.int16).pin_memory()
+
+    def e2e_step(i: int) -> None:
+        X = ctx.from_host(pin[0].numpy().view(np.uint16), "bf16")
+        H = ctx.from_host(pin[1].numpy().view(np.uint16), "bf16")
+        Bv = ctx.from_host(pin[2].numpy().view(np.uint16), "bf16")
+        out = traces.mlp_epilogue(ctx, X, H, Bv, primitive_gelu=False)
+        ctx.fetch_into(out, host_out.data_ptr(), host_out.numel() * 2)
+
+    for i in range(3):
+        e2e_step(i)
+    e2e_ms = timed(e2e_steps, e2e_step)
+    e2e_value = world * nbytes * e2e_steps / (e2e_ms / 1e3) / 1e9
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel: algorithmic bytes per launch / average launch duration
+    peak, peak_src = measured_peak()
+    kern = kt["elementwise"]
+    avg_ms = kern["ms"] / max(kern["launches"], 1)
+    achieved = nbytes / (avg_ms / 1e3) / 1e9 if avg_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": ncu_traffic(), "peak_source": peak_src, "kernel": "lt_ew_kernel<fast>",
+                "launch_us": 1e3 * avg_ms, "bytes_per_launch": nbytes, "frac_of_8TBs_nominal": achieved / 8000.0}
+
+    extra = {}
+    if not args.no_extra:
+        extra = extra_measurements(ctx, lt, torch, timed, step, sets, nbytes)
+        extra["host_ns_per_barrier"] = {k: st[k] / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
+        extra["cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "barriers": st["barriers"]}
+    cpu = cpu_baseline() if world == 1 and not args.no_cpu else None
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / max(args.steps, 1), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "trace": "convert x3, add, gelu_tanh, add, convert (7 ops, 1 fused kernel)",
+                   "l2": f"{N_SETS} rotating buffer sets ({N_SETS * nbytes / 1e6:.0f} MB) larger than L2",
+                   "per_gpu_batch": list(SHAPE), "parallelism": f"replicas x{world}, no collective"},
+        "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": world * (2 * 2 * SHAPE[0] * SHAPE[1] + 2 * SHAPE[1]),
+                "d2h_bytes_per_step": world * 2 * SHAPE[0] * SHAPE[1], "steps": e2e_steps,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(st["kernels_launched"]) * world,
+        "clocks": clocks,
+    }
+    if cpu:
+        line["cpu_baseline"] = cpu
+    if extra:
+        line["extra"] = extra
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
+    """Context numbers: unfused baseline, primitive-op trace, and the other configurations."""
+    from workloads import configs, traces
+
+    out = {}
+    n = 200
+    # the same graph traced from primitive ops (16 ops) instead of the gelu_tanh op
+    for i in range(5):
+        step(i, True)
+    ms = timed(n, lambda i: step(i, True))
+    out["c2_primitive_trace_gbs"] = nbytes * n / (ms / 1e3) / 1e9
+    # unfused: one kernel per traced op (same library, fusion off)
+    un = lt.LazyContext(device=ctx.device)
+    un.set_option("fusion", 0)
+    usets = [tuple(un.from_device_ptr(ctx.device_ptr(t), "bf16", t.shape) for t in s) for s in sets]
+    keep = [None] * len(usets)
+
+    def ustep(i, primitive=False):
+        X, H, Bv = usets[i % len(usets)]
+        keep[i % len(usets)] = traces.mlp_epilogue(un, X, H, Bv, primitive_gelu=primitive)
+        un.barrier()
+
+    for prim, key in ((False, "c2_unfused_gbs"), (True, "c2_primitive_unfused_gbs")):
+        for i in range(3):
+            ustep(i, prim)
+        ms = timed(50, lambda i: ustep(i, prim))
+        out[key] = nbytes * 50 / (ms / 1e3) / 1e9
+    un.set_kernel_timing(False)
+    ms_f = timed(n, step)
+    out["c2_fused_gbs"] = nbytes * n / (ms_f / 1e3) / 1e9
+    out["c2_speedup_vs_unfused"] = out["c2_fused_gbs"] / out["c2_unfused_gbs"]
+    out["c2_primitive_speedup_vs_unfused"] = out["c2_primitive_trace_gbs"] / out["c2_primitive_unfused_gbs"]
+    keep.clear()
+    del usets
+    un.close()
+    return out
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the context measurements (unfused baseline etc.)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

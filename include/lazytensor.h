@@ -200,8 +200,11 @@ lt_status lt_op(lt_ctx *ctx, int opcode, const lt_tensor *in, int n_in, const in
  */
 lt_status lt_assign(lt_ctx *ctx, lt_tensor dst, lt_tensor src);
 
-/* UnregisterTensor: the handle dies; a pending computation nobody names is never run. */
+/* UnregisterTensor: the handle dies; a pending computation nobody names is never run.
+   lt_release_many releases `n` handles in one call (language bindings batch the handles their
+   garbage collector retires); it stops at the first invalid handle and reports it. */
 lt_status lt_release(lt_ctx *ctx, lt_tensor t);
+lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
 
 /*
  * Barrier (Section 4; mark_step / LazyTensorBarrier): materialise every live tensor that

@@ -75,6 +75,7 @@ _SIGNATURES = {
     "lt_op": [_vp, _int, _P(_u64), _int, _P(_i64), _int, _P(_u64)],
     "lt_assign": [_vp, _u64, _u64],
     "lt_release": [_vp, _u64],
+    "lt_release_many": [_vp, _P(_u64), ctypes.c_size_t],
     "lt_barrier": [_vp, _int],
     "lt_fetch": [_vp, _u64, _vp, ctypes.c_size_t],
     "lt_device_ptr": [_vp, _u64, _P(_vp)],
@@ -125,21 +126,40 @@ def _torch_allocator():
 
 
 class LazyTensor:
-    """A handle of the C library; its value may still be a pending IR graph (paper Section 3)."""
+    """A handle of the C library; its value may still be a pending IR graph (paper Section 3).
 
-    __slots__ = ("ctx", "handle", "dtype", "shape", "_keep", "__weakref__")
+    Dropping the last Python reference unregisters the tensor: the handle is queued on the context
+    and released in one batch before the next barrier, fetch or dump.
+    """
 
-    def __init__(self, ctx: "LazyContext", handle: int, dtype: str, shape, keep=None):
+    __slots__ = ("ctx", "handle", "_keep", "_dtype", "_shape", "__weakref__")
+
+    def __init__(self, ctx: "LazyContext", handle: int, dtype: str | None = None, shape=None, keep=None):
         self.ctx = ctx
         self.handle = handle
-        self.dtype = dtype
-        self.shape = tuple(shape)
+        self._dtype = dtype
+        self._shape = None if shape is None else tuple(shape)
         self._keep = keep  # device storage this tensor borrows
 
     def __del__(self):
         ctx = self.ctx
-        if ctx is not None and ctx._ctx:
-            _lib.lt_release(ctx._ctx, self.handle)
+        if ctx is not None:
+            ctx._dead.append(self.handle)
+            if self._keep is not None:
+                # a pending graph may still read the borrowed storage: keep it until the next barrier
+                ctx._keeps.append(self._keep)
+
+    @property
+    def dtype(self) -> str:
+        if self._dtype is None:
+            self._dtype, _, self._shape, _ = self.ctx._info(self.handle)
+        return self._dtype
+
+    @property
+    def shape(self) -> tuple:
+        if self._shape is None:
+            self._dtype, _, self._shape, _ = self.ctx._info(self.handle)
+        return self._shape
 
     # the eager-looking API: every operator only records
     def _bin(self, name, other, swap=False):
@@ -201,11 +221,24 @@ class LazyContext:
         self._ctx = out
         self.stream = stream or 0
         self._h = _u64()
+        self._hp = ctypes.byref(self._h)
+        self._ins = (_u64 * 3)()
+        self._attrs = (_i64 * (3 + LT_MAX_RANK))()
+        self._dead: list[int] = []
+        self._keeps: list = []
 
     def close(self):
         if self._ctx:
             ctx, self._ctx = self._ctx, None
             _lib.lt_ctx_destroy(ctx)
+
+    def _flush_dead(self):
+        """Unregister the tensors Python has dropped since the last flush."""
+        dead = self._dead
+        if dead and self._ctx:
+            self._dead = []
+            n = len(dead)
+            self._check(_lib.lt_release_many(self._ctx, (_u64 * n)(*dead), n))
 
     def __del__(self):
         self.close()
@@ -259,26 +292,32 @@ class LazyContext:
 
     # ---- recording
     def op(self, name: str, *inputs, **attrs) -> LazyTensor:
-        n = len(inputs)
-        ins = (_u64 * max(n, 1))(*[t.handle for t in inputs])
-        if name == "convert":
-            a = [DTYPES[attrs["dtype"]]]
-        elif name == "iota":
-            shp = tuple(attrs["shape"])
-            a = [int(attrs["dim"]), len(shp), *shp]
-        elif name == "philox_bits":
-            shp = tuple(attrs["shape"])
-            seed, off = int(attrs["seed"]), int(attrs["offset"])
-            # 64-bit patterns travel as signed int64
-            a = [seed - (1 << 64) if seed >= (1 << 63) else seed, off - (1 << 64) if off >= (1 << 63) else off,
-                 len(shp), *shp]
-        else:
-            a = []
-        at = (_i64 * max(len(a), 1))(*a)
-        self._check(_lib.lt_op(self._ctx, OPCODES[name], ins, n, at, len(a), ctypes.byref(self._h)))
-        h = self._h.value
-        dt, rk, shp, _ = self._info(h)
-        return LazyTensor(self, h, dt, shp)
+        ins = self._ins
+        n = 0
+        for t in inputs:
+            ins[n] = t.handle
+            n += 1
+        at = self._attrs
+        na = 0
+        if attrs:
+            if name == "convert":
+                a = [DTYPES[attrs["dtype"]]]
+            elif name == "iota":
+                shp = tuple(attrs["shape"])
+                a = [int(attrs["dim"]), len(shp), *shp]
+            else:  # philox_bits
+                shp = tuple(attrs["shape"])
+                seed, off = int(attrs["seed"]), int(attrs["offset"])
+                # 64-bit patterns travel as signed int64
+                a = [seed - (1 << 64) if seed >= (1 << 63) else seed, off - (1 << 64) if off >= (1 << 63) else off,
+                     len(shp), *shp]
+            na = len(a)
+            for i in range(na):
+                at[i] = a[i]
+        st = _lib.lt_op(self._ctx, OPCODES[name], ins, n, at, na, self._hp)
+        if st:
+            self._check(st)
+        return LazyTensor(self, self._h.value)
 
     def _info(self, handle: int):
         dt, rk, mat = _int(), _int(), _int()
@@ -297,15 +336,31 @@ class LazyContext:
         self._check(_lib.lt_release(self._ctx, t.handle))
 
     def barrier(self, blocking: bool = False) -> None:
-        self._check(_lib.lt_barrier(self._ctx, 1 if blocking else 0))
+        if self._dead:
+            self._flush_dead()
+        keeps, self._keeps = self._keeps, []
+        st = _lib.lt_barrier(self._ctx, 1 if blocking else 0)
+        if st:
+            self._keeps.extend(keeps)
+            self._check(st)
 
     def fetch(self, t: LazyTensor) -> np.ndarray:
+        self._flush_dead()
         out = np.empty(t.shape, dtype=NP_DTYPES[t.dtype])
-        self._check(_lib.lt_fetch(self._ctx, t.handle, _vp(out.ctypes.data), out.nbytes))
+        keeps, self._keeps = self._keeps, []
+        st = _lib.lt_fetch(self._ctx, t.handle, _vp(out.ctypes.data), out.nbytes)
+        if st:
+            self._keeps.extend(keeps)
+            self._check(st)
         return out
 
     def fetch_into(self, t: LazyTensor, host_ptr: int, nbytes: int) -> None:
-        self._check(_lib.lt_fetch(self._ctx, t.handle, _vp(host_ptr), nbytes))
+        self._flush_dead()
+        keeps, self._keeps = self._keeps, []
+        st = _lib.lt_fetch(self._ctx, t.handle, _vp(host_ptr), nbytes)
+        if st:
+            self._keeps.extend(keeps)
+            self._check(st)
 
     def device_ptr(self, t: LazyTensor) -> int:
         p = _vp()
@@ -343,6 +398,7 @@ class LazyContext:
         return buf.value.decode()
 
     def dump_ir(self) -> str:
+        self._flush_dead()
         return self._text(_lib.lt_dump_ir)
 
     def dump_plan(self) -> str:

@@ -662,6 +662,15 @@ lt_status lt_release(lt_ctx *c, lt_tensor t) {
     return LT_OK;
 }
 
+lt_status lt_release_many(lt_ctx *c, const lt_tensor *handles, size_t n) {
+    if (!c || (n && !handles)) return LT_ERR_INVALID_ARG;
+    for (size_t i = 0; i < n; ++i) {
+        lt_status s = lt_release(c, handles[i]);
+        if (s) return s;
+    }
+    return LT_OK;
+}
+
 lt_status lt_barrier(lt_ctx *c, int blocking) {
     if (!c) return LT_ERR_INVALID_ARG;
     std::vector<uint32_t> &roots = c->roots_scratch;

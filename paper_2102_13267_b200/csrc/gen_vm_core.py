@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Generates vm_core.inc: the interpreter core of the fused-group kernels, as inline PTX.
+
+nvcc lowers a C++ `switch` over the opcode space to a tree of compares and branches (a dozen
+branches per interpreted instruction).  Written in PTX instead, the dispatch is one indexed
+branch (`brx.idx`) through a table with one entry per opcode, and the twenty 64-bit operands of
+the asm statement are the machine state: ACC and T0..T3, eight f32 lanes each, held as four
+register pairs so that add/sub/mul/fma run as packed `.f32x2` instructions.
+
+The core executes register-to-register opcodes and the aligned full-chunk loads and stores
+itself.  Everything else (ragged or unaligned chunks, broadcast loads, reductions, random
+bits, correctly rounded transcendentals) leaves the asm statement with the opcode in an output
+operand ("escape") and is handled by the surrounding C++.
+
+Run `python gen_vm_core.py` after changing vm.h's opcode map; the output is committed.
+"""
+from __future__ import annotations
+
+import re
+import struct
+from pathlib import Path
+
+HERE = Path(__file__).resolve().parent
+
+
+def opcodes() -> dict[str, int]:
+    """Opcode bases and indices, read from vm.h so the two cannot drift apart."""
+    text = (HERE / "vm.h").read_text()
+    vals: dict[str, int] = {}
+    for block in re.findall(r"enum\s*\{(.*?)\};", text, flags=re.S):
+        block = re.sub(r"/\*.*?\*/", "", block, flags=re.S)
+        block = re.sub(r"//[^\n]*", "", block)
+        nxt = 0
+        for item in block.split(","):
+            item = item.strip()
+            if not item:
+                continue
+            if "=" in item:
+                name, expr = (s.strip() for s in item.split("=", 1))
+                nxt = int(eval(expr, {}, vals))
+            else:
+                name = item
+            vals[name] = nxt
+            nxt += 1
+    for m in re.finditer(r"#define\s+(LT_VM_\w+)\s+(\d+)", text):
+        vals[m.group(1)] = int(m.group(2))
+    return vals
+
+
+OPS = opcodes()
+NSRC = OPS["LT_VM_NSRC"]
+
+A = [f"%{i}" for i in range(4)]
+T = [[f"%{4 + 4 * k + j}" for j in range(4)] for k in range(4)]
+REG = T + [A]  # destination index 0..3 = temporaries, 4 = ACC
+PC, EOP, EIMM, SB, PB, OFF4, COFF4, TAIL = "%20", "%21", "%22", "%23", "%24", "%25", "%26", "%27"
+
+
+def f32_hex(x: float) -> int:
+    return struct.unpack("<I", struct.pack("<f", x))[0]
+
+
+def pair_imm(x: float) -> str:
+    h = f32_hex(x)
+    return f"0x{h:08X}{h:08X}"
+
+
+def const_pair(reg: str, x: float) -> str:
+    return f"mov.b64 {reg}, {pair_imm(x)};"
+
+
+def unpack(pairs, names):
+    return [f"mov.b64 {{{names[2 * j]}, {names[2 * j + 1]}}}, {pairs[j]};" for j in range(4)]
+
+
+def pack(pairs, names):
+    return [f"mov.b64 {pairs[j]}, {{{names[2 * j]}, {names[2 * j + 1]}}};" for j in range(4)]
+
+
+X = [f"x{i}" for i in range(8)]
+Y = [f"y{i}" for i in range(8)]
+M = [f"m{i}" for i in range(8)]
+
+
+class Src:
+    """Second operand of a two-operand opcode: a temporary or a broadcast immediate."""
+
+    def __init__(self, kind: int):
+        self.kind = kind
+        if kind < 4:
+            self.pre = []
+            self.pairs = T[kind]
+            self._lanes = None
+        else:
+            self.pre = ["shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SB};", "ld.shared.b32 sv, [sa];", "mov.b64 ss, {sv, sv};"]
+            self.pairs = ["ss"] * 4
+
+    def lanes(self, out):
+        """PTX that makes the operand available lane by lane; returns (lines, lane names)."""
+        if self.kind < 4:
+            return unpack(self.pairs, Y), Y
+        return [], ["sv"] * 8
+
+
+def f2_body(idx: int, src: Src, fast: bool):
+    names = ["add", "sub", "rsub", "mul", "div", "rdiv", "max", "min"]
+    op = names[idx]
+    lines = list(src.pre)
+    if op in ("add", "sub", "mul"):
+        lines += [f"{op}.rn.f32x2 {A[j]}, {A[j]}, {src.pairs[j]};" for j in range(4)]
+    elif op == "rsub":
+        lines += [f"sub.rn.f32x2 {A[j]}, {src.pairs[j]}, {A[j]};" for j in range(4)]
+    else:
+        ul, y = src.lanes(Y)
+        lines += unpack(A, X) + ul
+        for i in range(8):
+            if op == "div":
+                lines.append(f"div.{'approx' if fast else 'rn'}.f32 {X[i]}, {X[i]}, {y[i]};")
+            elif op == "rdiv":
+                lines.append(f"div.{'approx' if fast else 'rn'}.f32 {X[i]}, {y[i]}, {X[i]};")
+            else:
+                lines.append(f"{op}.NaN.f32 {X[i]}, {X[i]}, {y[i]};")
+        lines += pack(A, X)
+    return lines
+
+
+def i2_body(idx: int, src: Src):
+    ops = ["add.s32", "sub.s32", "rsub", "mul.lo.s32", "and.b32", "or.b32", "xor.b32", "max.s32", "min.s32", "max.u32", "min.u32"]
+    op = ops[idx]
+    ul, y = src.lanes(Y)
+    lines = list(src.pre) + unpack(A, X) + ul
+    for i in range(8):
+        if op == "rsub":
+            lines.append(f"sub.s32 {X[i]}, {y[i]}, {X[i]};")
+        else:
+            lines.append(f"{op} {X[i]}, {X[i]}, {y[i]};")
+    return lines + pack(A, X)
+
+
+def cmp_body(idx: int, src: Src):
+    ty, cc = divmod(idx, 6)
+    ccn = ["gt", "ge", "lt", "le", "eq", "ne"][cc]
+    if ty == 0:
+        ins = f"setp.{'neu' if ccn == 'ne' else ccn}.f32"
+    elif ty == 1:
+        ins = f"setp.{ccn}.s32"
+    else:
+        ins = f"setp.{ {'gt': 'hi', 'ge': 'hs', 'lt': 'lo', 'le': 'ls', 'eq': 'eq', 'ne': 'ne'}[ccn] }.u32"
+    ul, y = src.lanes(Y)
+    lines = list(src.pre) + unpack(A, X) + ul
+    for i in range(8):
+        lines += [f"{ins} p, {X[i]}, {y[i]};", f"selp.b32 {X[i]}, 1, 0, p;"]
+    return lines + pack(A, X)
+
+
+def where_body(m: int, src: Src, variant_b: bool):
+    ul, y = src.lanes(Y)
+    lines = list(src.pre) + unpack(A, X) + unpack(T[m], M) + ul
+    for i in range(8):
+        lines.append(f"setp.ne.u32 p, {M[i]}, 0;")
+        lines.append(f"selp.b32 {X[i]}, {y[i]}, {X[i]}, p;" if variant_b else f"selp.b32 {X[i]}, {X[i]}, {y[i]}, p;")
+    return lines + pack(A, X)
+
+
+LOG2E, LN2 = 1.4426950408889634, 0.6931471805599453
+GELU_K = 0.7978845608028654
+GELU_KC = GELU_K * 0.044715
+
+
+def lanes_op(fmt: str):
+    return unpack(A, X) + [fmt.format(x=X[i]) for i in range(8)] + pack(A, X)
+
+
+def unary_body(name: str, fast: bool):
+    """Returns PTX lines, or None when the opcode escapes to C++ in this flavour."""
+    if name == "OP_U_NEG":
+        return [f"xor.b64 {a}, {a}, 0x8000000080000000;" for a in A]
+    if name == "OP_U_ABS":
+        return [f"and.b64 {a}, {a}, 0x7FFFFFFF7FFFFFFF;" for a in A]
+    if name == "OP_U_RELU":
+        return lanes_op("max.NaN.f32 {x}, {x}, 0f00000000;")
+    if name == "OP_U_SQUARE":
+        return [f"mul.rn.f32x2 {a}, {a}, {a};" for a in A]
+    if name == "OP_U_SQRT":
+        return lanes_op("sqrt.approx.f32 {x}, {x};" if fast else "sqrt.rn.f32 {x}, {x};")
+    if name == "OP_U_RSQRT":
+        return lanes_op("rsqrt.approx.f32 {x}, {x};")
+    if name == "OP_U_RECIP":
+        return lanes_op("rcp.approx.ftz.f32 {x}, {x};" if fast else "rcp.rn.f32 {x}, {x};")
+    if name == "OP_U_RBF16":
+        lines = unpack(A, X)
+        for j in range(4):
+            lines += [f"cvt.rn.bf16x2.f32 w0, {X[2 * j + 1]}, {X[2 * j]};", f"shl.b32 {X[2 * j]}, w0, 16;",
+                      f"and.b32 {X[2 * j + 1]}, w0, 0xFFFF0000;"]
+        return lines + pack(A, X)
+    if name == "OP_U_INEG":
+        return lanes_op("neg.s32 {x}, {x};")
+    if name == "OP_U_IABS":
+        return lanes_op("abs.s32 {x}, {x};")
+    if name == "OP_U_NOT":
+        return unpack(A, X) + sum(([f"setp.eq.u32 p, {x}, 0;", f"selp.b32 {x}, 1, 0, p;"] for x in X), []) + pack(A, X)
+    if name == "OP_C_I2F":
+        return lanes_op("cvt.rn.f32.s32 {x}, {x};")
+    if name == "OP_C_U2F":
+        return lanes_op("cvt.rn.f32.u32 {x}, {x};")
+    if name == "OP_C_F2I":
+        return lanes_op("cvt.rzi.s32.f32 {x}, {x};")
+    if name == "OP_C_NZF":
+        return unpack(A, X) + sum(([f"setp.neu.f32 p, {x}, 0f00000000;", f"selp.b32 {x}, 1, 0, p;"] for x in X), []) + pack(A, X)
+    if name == "OP_C_NZI":
+        return unpack(A, X) + sum(([f"setp.ne.u32 p, {x}, 0;", f"selp.b32 {x}, 1, 0, p;"] for x in X), []) + pack(A, X)
+    if not fast:
+        return None  # exp, log, tanh, sigmoid, gelu: correctly rounded versions live in C++
+    if name == "OP_U_EXP":
+        return ([const_pair("c0", LOG2E)] + [f"mul.rn.f32x2 {a}, {a}, c0;" for a in A] + lanes_op("ex2.approx.ftz.f32 {x}, {x};"))
+    if name == "OP_U_LOG":
+        return lanes_op("lg2.approx.f32 {x}, {x};") + [const_pair("c0", LN2)] + [f"mul.rn.f32x2 {a}, {a}, c0;" for a in A]
+    if name == "OP_U_TANH":
+        return lanes_op("tanh.approx.f32 {x}, {x};")
+    if name == "OP_U_SIGMOID":
+        lines = [const_pair("c0", -LOG2E), const_pair("c1", 1.0)] + [f"mul.rn.f32x2 {a}, {a}, c0;" for a in A]
+        lines += lanes_op("ex2.approx.ftz.f32 {x}, {x};")
+        lines += [f"add.rn.f32x2 {a}, {a}, c1;" for a in A]
+        return lines + lanes_op("rcp.approx.ftz.f32 {x}, {x};")
+    if name == "OP_U_GELU":
+        lines = [const_pair("c0", GELU_KC), const_pair("c1", GELU_K), const_pair("c2", 0.5)]
+        for j, a in enumerate(A):
+            g = f"g{j}"
+            lines += [f"mul.rn.f32x2 {g}, {a}, {a};",
+                      f"fma.rn.f32x2 {g}, {g}, c0, c1;",
+                      f"mul.rn.f32x2 {g}, {g}, {a};",
+                      f"mov.b64 {{{X[2 * j]}, {X[2 * j + 1]}}}, {g};",
+                      f"tanh.approx.f32 {X[2 * j]}, {X[2 * j]};", f"tanh.approx.f32 {X[2 * j + 1]}, {X[2 * j + 1]};",
+                      f"mov.b64 {g}, {{{X[2 * j]}, {X[2 * j + 1]}}};",
+                      f"mul.rn.f32x2 {a}, {a}, c2;",
+                      f"fma.rn.f32x2 {a}, {a}, {g}, {a};"]
+        return lines
+    raise KeyError(name)
+
+
+def cvt_bf16(d: int):
+    P = REG[d]
+    lines = [f"mov.b64 {{w0, w1}}, {P[0]};", f"mov.b64 {{w2, w3}}, {P[1]};"]
+    for j in (3, 2, 1, 0):
+        lines += [f"shl.b32 x0, w{j}, 16;", f"and.b32 x1, w{j}, 0xFFFF0000;", f"mov.b64 {P[j]}, {{x0, x1}};"]
+    return lines
+
+
+def cvt_u8(d: int):
+    P = REG[d]
+    lines = [f"mov.b64 {{w0, w1}}, {P[0]};"]
+    for i in range(8):
+        lines.append(f"bfe.u32 {X[i]}, w{i // 4}, {8 * (i % 4)}, 8;")
+    return lines + pack(P, X)
+
+
+def slot_pointer():
+    """ptr = pointer-table entry of slot `imm`; leaves for the slow path when the entry is flagged
+    (bit 63: not vector-aligned) or the chunk is ragged."""
+    return ["shl.b32 sa, imm, 3;", f"add.u32 sa, sa, {PB};", "ld.shared.b64 ptr, [sa];", "setp.lt.s64 p, ptr, 0;",
+            "@p bra L_ESC;", "@ptail bra L_ESC;"]
+
+
+def ldv_body(sz: int, cls: int, d: int):
+    P = REG[d]
+    lines = slot_pointer()
+    if cls == 0:
+        lines.append(f"shr.u64 offs, {OFF4}, {sz};" if sz else f"mov.b64 offs, {OFF4};")
+    else:
+        lines += [f"cvt.u64.u32 offs, {COFF4};"] + ([f"shr.u64 offs, offs, {sz};"] if sz else [])
+    lines.append("add.u64 ptr, ptr, offs;")
+    ld = "ld.global.cs" if cls == 0 else "ld.global.nc"
+    if sz == 0:
+        lines += [f"{ld}.v4.b32 {{x0, x1, x2, x3}}, [ptr];", f"{ld}.v4.b32 {{x4, x5, x6, x7}}, [ptr+16];"] + pack(P, X)
+    elif sz == 1:
+        lines += [f"{ld}.v4.b32 {{x0, x1, x2, x3}}, [ptr];", f"mov.b64 {P[0]}, {{x0, x1}};", f"mov.b64 {P[1]}, {{x2, x3}};"]
+    else:
+        lines += [f"{ld}.v2.b32 {{x0, x1}}, [ptr];", f"mov.b64 {P[0]}, {{x0, x1}};"]
+    return lines
+
+
+def stv_body(sz: int):
+    lines = slot_pointer()
+    lines.append(f"shr.u64 offs, {OFF4}, {sz};" if sz else f"mov.b64 offs, {OFF4};")
+    lines.append("add.u64 ptr, ptr, offs;")
+    lines += unpack(A, X)
+    if sz == 0:
+        lines += ["st.global.cs.v4.b32 [ptr], {x0, x1, x2, x3};", "st.global.cs.v4.b32 [ptr+16], {x4, x5, x6, x7};"]
+    elif sz == 1:
+        for j in range(4):
+            lines.append(f"cvt.rn.bf16x2.f32 w{j}, {X[2 * j + 1]}, {X[2 * j]};")
+        lines.append("st.global.cs.v4.b32 [ptr], {w0, w1, w2, w3};")
+    else:
+        for h in range(2):
+            b = 4 * h
+            lines += [f"prmt.b32 y0, {X[b]}, {X[b + 1]}, 0x0040;", f"prmt.b32 y1, {X[b + 2]}, {X[b + 3]}, 0x0040;",
+                      f"prmt.b32 w{h}, y0, y1, 0x5410;"]
+        lines.append("st.global.cs.v2.b32 [ptr], {w0, w1};")
+    return lines
+
+
+def build(fast: bool) -> list[str]:
+    limit = OPS["OP_LIMIT"]
+    bodies: dict[int, list[str]] = {}
+
+    for k in range(4):
+        bodies[OPS["OP_MOV_T_ACC"] + k] = [f"mov.b64 {T[k][j]}, {A[j]};" for j in range(4)]
+        bodies[OPS["OP_MOV_ACC_T"] + k] = [f"mov.b64 {A[j]}, {T[k][j]};" for j in range(4)]
+    s = Src(4)
+    bodies[OPS["OP_MOV_ACC_S"]] = s.pre + [f"mov.b64 {a}, ss;" for a in A]
+    for d in range(5):
+        bodies[OPS["OP_CVT_BF16"] + d] = cvt_bf16(d)
+        bodies[OPS["OP_CVT_U8"] + d] = cvt_u8(d)
+    bodies[OPS["OP_IOTA_COL"]] = ([f"shr.u32 w0, {COFF4}, 2;"] + [f"add.u32 {X[i]}, w0, {i};" for i in range(8)] + pack(A, X))
+    for name in ("OP_U_NEG", "OP_U_ABS", "OP_U_RELU", "OP_U_EXP", "OP_U_LOG", "OP_U_TANH", "OP_U_SQRT", "OP_U_RSQRT",
+                 "OP_U_RECIP", "OP_U_SQUARE", "OP_U_SIGMOID", "OP_U_GELU", "OP_U_RBF16", "OP_U_INEG", "OP_U_IABS",
+                 "OP_U_NOT", "OP_C_I2F", "OP_C_U2F", "OP_C_F2I", "OP_C_NZF", "OP_C_NZI"):
+        b = unary_body(name, fast)
+        if b is not None:
+            bodies[OPS[name]] = b
+    for sz in range(3):
+        for cls in range(2):
+            for d in range(5):
+                bodies[OPS["OP_LDV"] + (sz * 2 + cls) * 5 + d] = ldv_body(sz, cls, d)
+        bodies[OPS["OP_STV"] + sz] = stv_body(sz)
+    for idx in range(OPS["F2_COUNT"]):
+        for k in range(NSRC):
+            bodies[OPS["OP_F2"] + idx * NSRC + k] = f2_body(idx, Src(k), fast)
+    for idx in range(OPS["I2_COUNT"]):
+        for k in range(NSRC):
+            bodies[OPS["OP_I2"] + idx * NSRC + k] = i2_body(idx, Src(k))
+    for idx in range(18):
+        for k in range(NSRC):
+            bodies[OPS["OP_CMP"] + idx * NSRC + k] = cmp_body(idx, Src(k))
+    for m in range(4):
+        for k in range(NSRC):
+            bodies[OPS["OP_WHERE_A"] + m * NSRC + k] = where_body(m, Src(k), False)
+            bodies[OPS["OP_WHERE_B"] + m * NSRC + k] = where_body(m, Src(k), True)
+
+    out = ["{"]
+    out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3;")
+    out.append(".reg .b32 " + ", ".join(X + Y + M) + ";")
+    out.append(".reg .b64 ss, ptr, offs, g0, g1, g2, g3, c0, c1, c2;")
+    out.append(".reg .pred p, ptail;")
+    table = ", ".join(f"L_{i}" if i in bodies else "L_ESC" for i in range(limit))
+    out.append(f"TBL: .branchtargets {table};")
+    out.append(f"setp.ne.u32 ptail, {TAIL}, 0;")
+    out.append(f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];")
+    out.append("L_DISPATCH:")
+    out.append("mov.b32 op, nop;")
+    out.append("mov.b32 imm, nimm;")
+    out.append(f"add.u32 {PC}, {PC}, 8;")
+    out.append(f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];")  # the slot after the last instruction is padding
+    out.append("brx.idx op, TBL;")
+    for code in sorted(bodies):
+        out.append(f"L_{code}:")
+        out += bodies[code]
+        out.append("bra.uni L_DISPATCH;")
+    out.append("L_ESC:")
+    out.append(f"mov.b32 {EOP}, op;")
+    out.append(f"mov.b32 {EIMM}, imm;")
+    out.append("}")
+    return out
+
+
+def as_macro(name: str, lines: list[str]) -> str:
+    body = " \\\n".join('    "' + ln + '\\n"' for ln in lines)
+    return f"#define {name} \\\n{body}\n"
+
+
+def main() -> None:
+    text = ("// Generated by gen_vm_core.py from vm.h -- do not edit.\n"
+            "// Operands: %0-%3 ACC, %4-%19 T0..T3 (f32x2 pairs); %20 pc (shared address); %21 escape opcode;\n"
+            "// %22 escape immediate; %23 immediates base; %24 pointer table base (shared addresses);\n"
+            "// %25 chunk byte offset for 4-byte elements; %26 column byte offset; %27 ragged-chunk flag.\n"
+            "#pragma once\n\n")
+    text += as_macro("LT_VM_CORE_FAST", build(True)) + "\n" + as_macro("LT_VM_CORE_PRECISE", build(False))
+    (HERE / "vm_core.inc").write_text(text)
+    print(f"wrote vm_core.inc ({len(text)} bytes)")
+
+
+if __name__ == "__main__":
+    main()

@@ -12,6 +12,7 @@
 
 #include "launch.h"
 #include "vm.h"
+#include "vm_core.inc"
 
 namespace {
 
@@ -180,8 +181,57 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// Random bits of the V lanes whose flat indices start at flat0 (element i uses word i mod 4 of
+// block i / 4).  Kept out of line: its ten rounds would otherwise inflate the register budget of
+// the whole interpreter.
+__device__ __noinline__ void philox_chunk(uint32_t *out, uint64_t flat0, uint32_t k0, uint32_t k1, uint32_t o0,
+                                          uint32_t o1) {
+    const uint64_t q = flat0 >> 2;
+    const uint32_t sh = (uint32_t)flat0 & 3u;
+    uint32_t a[4], b[4];
+    philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), o0, o1, k0, k1, a);
+    philox4x32_10((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), o0, o1, k0, k1, b);
+    if (sh == 0) {
+        out[0] = a[0]; out[1] = a[1]; out[2] = a[2]; out[3] = a[3];
+        out[4] = b[0]; out[5] = b[1]; out[6] = b[2]; out[7] = b[3];
+        return;
+    }
+    // chunk does not start on a block boundary (ragged rows): a third block covers the tail
+    uint32_t c[4];
+    philox4x32_10((uint32_t)(q + 2), (uint32_t)((q + 2) >> 32), o0, o1, k0, k1, c);
+    const uint32_t w[12] = {a[0], a[1], a[2], a[3], b[0], b[1], b[2], b[3], c[0], c[1], c[2], c[3]};
+    for (int i = 0; i < V; ++i) out[i] = w[i + sh];
+}
+
 // ------------------------------------------------------------------- memory
 __device__ __forceinline__ uint32_t esz_log2(uint32_t dt) { return dt == LT_ST_BF16 ? 1u : (dt == LT_ST_U8 ? 0u : 2u); }
+
+// ragged tail or unaligned pointer: element by element, packed into the same storage format
+__device__ __noinline__ void load_raw_slow(float *d, const char *p, uint32_t dt, int nvalid) {
+    if (dt == LT_ST_BF16) {
+        const unsigned short *q = reinterpret_cast<const unsigned short *>(p);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t lo = 2 * j < nvalid ? q[2 * j] : 0u;
+            uint32_t hi = 2 * j + 1 < nvalid ? q[2 * j + 1] : 0u;
+            d[j] = u2f(lo | (hi << 16));
+        }
+    } else if (dt == LT_ST_U8) {
+        const unsigned char *q = reinterpret_cast<const unsigned char *>(p);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if (4 * j + b < nvalid) w |= (uint32_t)q[4 * j + b] << (8 * b);
+            d[j] = u2f(w);
+        }
+    } else {
+        const float *q = reinterpret_cast<const float *>(p);
+#pragma unroll
+        for (int i = 0; i < V; ++i) d[i] = i < nvalid ? q[i] : 0.0f;
+    }
+}
 
 // Raw chunk load: lanes keep the storage format (bf16: 4 packed words, u8: 2 packed words,
 // 32-bit types: 8 words); CVT widens later so the load itself stays asynchronous.
@@ -227,29 +277,12 @@ __device__ __forceinline__ void load_raw(float (&d)[V], const Env &E, uint32_t s
         }
         return;
     }
-    // ragged tail or unaligned pointer: element by element, packed into the same storage format
-    if (dt == LT_ST_BF16) {
-        const unsigned short *q = reinterpret_cast<const unsigned short *>(p);
+    {
+        // staged through a scratch array so the register-resident lanes never have their address taken
+        float tmp[V];
+        load_raw_slow(tmp, p, dt, ck.nvalid);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t lo = 2 * j < ck.nvalid ? q[2 * j] : 0u;
-            uint32_t hi = 2 * j + 1 < ck.nvalid ? q[2 * j + 1] : 0u;
-            d[j] = u2f(lo | (hi << 16));
-        }
-    } else if (dt == LT_ST_U8) {
-        const unsigned char *q = reinterpret_cast<const unsigned char *>(p);
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            uint32_t w = 0;
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-                if (4 * j + b < ck.nvalid) w |= (uint32_t)q[4 * j + b] << (8 * b);
-            d[j] = u2f(w);
-        }
-    } else {
-        const float *q = reinterpret_cast<const float *>(p);
-#pragma unroll
-        for (int i = 0; i < V; ++i) d[i] = i < ck.nvalid ? q[i] : 0.0f;
+        for (int i = 0; i < V; ++i) d[i] = tmp[i];
     }
 }
 
@@ -266,6 +299,16 @@ __device__ __forceinline__ void widen(float (&d)[V], uint32_t dt) {
         for (int b = 0; b < 4; ++b) {
             d[b] = u2f((w0 >> (8 * b)) & 0xffu);
             d[4 + b] = u2f((w1 >> (8 * b)) & 0xffu);
+        }
+    }
+}
+
+__device__ __noinline__ void store_chunk_slow(const float *a, char *p, uint32_t dt, int nvalid) {
+    for (int i = 0; i < V; ++i) {
+        if (i < nvalid) {
+            if (dt == LT_ST_BF16) reinterpret_cast<__nv_bfloat16 *>(p)[i] = __float2bfloat16_rn(a[i]);
+            else if (dt == LT_ST_U8) reinterpret_cast<unsigned char *>(p)[i] = (unsigned char)f2u(a[i]);
+            else reinterpret_cast<float *>(p)[i] = a[i];
         }
     }
 }
@@ -306,13 +349,11 @@ __device__ __forceinline__ void store_chunk(const float (&a)[V], const Env &E, u
         }
         return;
     }
+    {
+        float tmp[V];
 #pragma unroll
-    for (int i = 0; i < V; ++i) {
-        if (i < ck.nvalid) {
-            if (dt == LT_ST_BF16) reinterpret_cast<__nv_bfloat16 *>(p)[i] = __float2bfloat16_rn(a[i]);
-            else if (dt == LT_ST_U8) reinterpret_cast<unsigned char *>(p)[i] = (unsigned char)f2u(a[i]);
-            else reinterpret_cast<float *>(p)[i] = a[i];
-        }
+        for (int i = 0; i < V; ++i) tmp[i] = a[i];
+        store_chunk_slow(tmp, p, dt, ck.nvalid);
     }
 }
 
@@ -348,107 +389,131 @@ __device__ __forceinline__ void row_reduce(float (&acc)[V], const Chunk &ck, Row
 }
 
 // -------------------------------------------------------------- interpreter
-#define LT_SRC_CASES(BASE, IDX, EXPR)                                                                   \
-    case (BASE) + (IDX) * LT_VM_NSRC + 0: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t0[i]; acc[i] = EXPR; } } break; \
-    case (BASE) + (IDX) * LT_VM_NSRC + 1: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t1[i]; acc[i] = EXPR; } } break; \
-    case (BASE) + (IDX) * LT_VM_NSRC + 2: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t2[i]; acc[i] = EXPR; } } break; \
-    case (BASE) + (IDX) * LT_VM_NSRC + 3: { _Pragma("unroll") for (int i = 0; i < V; ++i) { const float b_ = t3[i]; acc[i] = EXPR; } } break; \
-    case (BASE) + (IDX) * LT_VM_NSRC + 4: { const float b_ = u2f(E.scal(in.imm)); _Pragma("unroll") for (int i = 0; i < V; ++i) { acc[i] = EXPR; } } break;
+// Program, immediates and pointer table staged in shared memory, where the PTX core reads them
+// with uniform (broadcast) loads.
+struct Staged {
+    LtIns ins[LT_VM_MAX_INS + 2];
+    uint32_t scal[LT_VM_MAX_SCAL];
+    uint64_t ptr[LT_VM_MAX_PTR];
+    float red[64];
+};
 
-#define LT_F2_CASE(IDX) LT_SRC_CASES(OP_F2, IDX, (f2<IDX, FAST>(acc[i], b_)))
-#define LT_I2_CASE(IDX) LT_SRC_CASES(OP_I2, IDX, (i2<IDX>(acc[i], b_)))
-#define LT_CMP_CASE(IDX) LT_SRC_CASES(OP_CMP, IDX, (cmp<IDX>(acc[i], b_)))
-#define LT_WHERE_CASES(M, TM)                                                                 \
-    LT_SRC_CASES(OP_WHERE_A, M, (f2u(TM[i]) != 0u ? acc[i] : b_))                              \
-    LT_SRC_CASES(OP_WHERE_B, M, (f2u(TM[i]) != 0u ? b_ : acc[i]))
-#define LT_UN_CASE(OPC) \
-    case OPC: { _Pragma("unroll") for (int i = 0; i < V; ++i) acc[i] = un<OPC, FAST>(acc[i]); } break;
-#define LT_T_CASES(BASE, STMT)                       \
-    case (BASE) + 0: { float(&T)[V] = t0; STMT; } break; \
-    case (BASE) + 1: { float(&T)[V] = t1; STMT; } break; \
-    case (BASE) + 2: { float(&T)[V] = t2; STMT; } break; \
-    case (BASE) + 3: { float(&T)[V] = t3; STMT; } break;
+// Pointer-table entry for the PTX core: bit 63 marks a slot whose chunks cannot use 128-bit accesses.
+__device__ __forceinline__ uint64_t flag_pointer(uint64_t p, uint32_t dt, bool rows_aligned) {
+    const uint64_t need = dt == LT_ST_U8 ? 7u : 15u;
+    return ((p & need) == 0 && rows_aligned) ? p : (p | (1ull << 63));
+}
 
-template <bool FAST, bool ROW, class Env>
-__device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCtx *rc) {
-    float acc[V], t0[V], t1[V], t2[V], t3[V];
+__device__ __forceinline__ void lanes_of(const uint64_t (&p)[4], float (&f)[V]) {
 #pragma unroll
-    for (int i = 0; i < V; ++i) acc[i] = t0[i] = t1[i] = t2[i] = t3[i] = 0.0f;
-    const uint32_t n_ins = E.n_ins();
-    for (uint32_t pc = 0; pc < n_ins; ++pc) {
-        const LtIns in = E.ins(pc);
-        switch (in.op) {
-            LT_T_CASES(OP_MOV_T_ACC, { _Pragma("unroll") for (int i = 0; i < V; ++i) T[i] = acc[i]; })
-            LT_T_CASES(OP_MOV_ACC_T, { _Pragma("unroll") for (int i = 0; i < V; ++i) acc[i] = T[i]; })
-            case OP_MOV_ACC_S: {
-                const float s = u2f(E.scal(in.imm));
-#pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = s;
-            } break;
-            LT_T_CASES(OP_LD_T, load_raw(T, E, in.imm, ck))
-            case OP_LD_ACC: load_raw(acc, E, in.imm, ck); break;
-            LT_T_CASES(OP_CVT_T, widen(T, in.a))
-            case OP_CVT_ACC: widen(acc, in.a); break;
-            case OP_ST: store_chunk(acc, E, in.imm, ck); break;
-            case OP_IOTA_COL: {
-#pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = u2f(ck.col0 + i);
-            } break;
-            case OP_IOTA_ROW: {
-                const uint32_t r = (ck.row / E.scal(in.imm)) % E.scal(in.imm + 1);
-#pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = u2f(r);
-            } break;
-            case OP_PHILOX: {
-                const uint32_t k0 = E.scal(in.imm), k1 = E.scal(in.imm + 1);
-                const uint32_t o0 = E.scal(in.imm + 2), o1 = E.scal(in.imm + 3);
-                const uint64_t q = ck.flat0 >> 2;
-                const uint32_t sh = (uint32_t)ck.flat0 & 3u;
-                uint32_t w[12];
-                philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), o0, o1, k0, k1, *reinterpret_cast<uint32_t(*)[4]>(&w[0]));
-                philox4x32_10((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), o0, o1, k0, k1,
-                              *reinterpret_cast<uint32_t(*)[4]>(&w[4]));
-                if (sh == 0) {
-#pragma unroll
-                    for (int i = 0; i < V; ++i) acc[i] = u2f(w[i]);
-                } else {  // chunk does not start on a block boundary (ragged rows)
-                    philox4x32_10((uint32_t)(q + 2), (uint32_t)((q + 2) >> 32), o0, o1, k0, k1,
-                                  *reinterpret_cast<uint32_t(*)[4]>(&w[8]));
-#pragma unroll
-                    for (int i = 0; i < V; ++i) {
-                        uint32_t x = w[i + 1];
-                        if (sh == 2) x = w[i + 2];
-                        if (sh == 3) x = w[i + 3];
-                        acc[i] = u2f(x);
-                    }
-                }
-            } break;
-            case OP_RED_SUM: if constexpr (ROW) row_reduce<0>(acc, ck, rc); break;
-            case OP_RED_MAX: if constexpr (ROW) row_reduce<1>(acc, ck, rc); break;
-            case OP_RED_MIN: if constexpr (ROW) row_reduce<2>(acc, ck, rc); break;
-            LT_UN_CASE(OP_U_NEG) LT_UN_CASE(OP_U_ABS) LT_UN_CASE(OP_U_RELU) LT_UN_CASE(OP_U_EXP)
-            LT_UN_CASE(OP_U_LOG) LT_UN_CASE(OP_U_TANH) LT_UN_CASE(OP_U_SQRT) LT_UN_CASE(OP_U_RSQRT)
-            LT_UN_CASE(OP_U_RECIP) LT_UN_CASE(OP_U_SQUARE) LT_UN_CASE(OP_U_SIGMOID) LT_UN_CASE(OP_U_GELU)
-            LT_UN_CASE(OP_U_RBF16) LT_UN_CASE(OP_U_INEG) LT_UN_CASE(OP_U_IABS) LT_UN_CASE(OP_U_NOT)
-            LT_UN_CASE(OP_C_I2F) LT_UN_CASE(OP_C_U2F) LT_UN_CASE(OP_C_F2I) LT_UN_CASE(OP_C_NZF)
-            LT_UN_CASE(OP_C_NZI)
-            LT_F2_CASE(0) LT_F2_CASE(1) LT_F2_CASE(2) LT_F2_CASE(3) LT_F2_CASE(4) LT_F2_CASE(5) LT_F2_CASE(6)
-            LT_F2_CASE(7)
-            LT_I2_CASE(0) LT_I2_CASE(1) LT_I2_CASE(2) LT_I2_CASE(3) LT_I2_CASE(4) LT_I2_CASE(5) LT_I2_CASE(6)
-            LT_I2_CASE(7) LT_I2_CASE(8) LT_I2_CASE(9) LT_I2_CASE(10)
-            LT_CMP_CASE(0) LT_CMP_CASE(1) LT_CMP_CASE(2) LT_CMP_CASE(3) LT_CMP_CASE(4) LT_CMP_CASE(5)
-            LT_CMP_CASE(6) LT_CMP_CASE(7) LT_CMP_CASE(8) LT_CMP_CASE(9) LT_CMP_CASE(10) LT_CMP_CASE(11)
-            LT_CMP_CASE(12) LT_CMP_CASE(13) LT_CMP_CASE(14) LT_CMP_CASE(15) LT_CMP_CASE(16) LT_CMP_CASE(17)
-            LT_WHERE_CASES(0, t0) LT_WHERE_CASES(1, t1) LT_WHERE_CASES(2, t2) LT_WHERE_CASES(3, t3)
-            default: break;
-        }
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = u2f((uint32_t)p[j]);
+        f[2 * j + 1] = u2f((uint32_t)(p[j] >> 32));
     }
+}
+
+__device__ __forceinline__ void pairs_of(const float (&f)[V], uint64_t (&p)[4]) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) p[j] = (uint64_t)f2u(f[2 * j]) | ((uint64_t)f2u(f[2 * j + 1]) << 32);
+}
+
+#define LT_VM_OPERANDS                                                                                              \
+    : "+l"(R[4][0]), "+l"(R[4][1]), "+l"(R[4][2]), "+l"(R[4][3]), "+l"(R[0][0]), "+l"(R[0][1]), "+l"(R[0][2]),      \
+      "+l"(R[0][3]), "+l"(R[1][0]), "+l"(R[1][1]), "+l"(R[1][2]), "+l"(R[1][3]), "+l"(R[2][0]), "+l"(R[2][1]),      \
+      "+l"(R[2][2]), "+l"(R[2][3]), "+l"(R[3][0]), "+l"(R[3][1]), "+l"(R[3][2]), "+l"(R[3][3]), "+r"(pc),           \
+      "=r"(eop), "=r"(eimm)                                                                                         \
+    : "r"(scal_s), "r"(ptr_s), "l"(off4), "r"(coff4), "r"(tail)                                                     \
+    : "memory"
+
+// Runs the group's program on one chunk.  R[0..3] are T0..T3, R[4] is ACC.  The PTX core runs until an
+// opcode it does not implement (see gen_vm_core.py); that opcode is executed here and the core re-entered.
+template <bool FAST, bool ROW, class Env>
+__device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCtx *rc, uint32_t prog_s, uint32_t scal_s,
+                                            uint32_t ptr_s) {
+    uint64_t R[5][4];
+#pragma unroll
+    for (int k = 0; k < 5; ++k)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) R[k][j] = 0;
+    uint32_t pc = prog_s;
+    const uint64_t off4 = ck.flat0 << 2;
+    const uint32_t coff4 = ck.col0 << 2;
+    const uint32_t tail = ck.nvalid != V ? 1u : 0u;
+#pragma unroll 1
+    for (;;) {
+        uint32_t eop, eimm;
+        if constexpr (FAST) asm volatile(LT_VM_CORE_FAST LT_VM_OPERANDS);
+        else asm volatile(LT_VM_CORE_PRECISE LT_VM_OPERANDS);
+        if (eop == OP_END) break;
+        float f[V];
+        if (eop >= OP_LD && eop < OP_STV) {  // generic load, or a vector load that met a ragged chunk / unaligned pointer
+            const uint32_t d = eop < OP_LDV ? eop - OP_LD : (eop - OP_LDV) % 5u;
+            load_raw(f, E, eimm, ck);
+            if (d == 0) pairs_of(f, R[0]);
+            else if (d == 1) pairs_of(f, R[1]);
+            else if (d == 2) pairs_of(f, R[2]);
+            else if (d == 3) pairs_of(f, R[3]);
+            else pairs_of(f, R[4]);
+            continue;
+        }
+        lanes_of(R[4], f);
+        if (eop == OP_ST || (eop >= OP_STV && eop < OP_STV + 3)) {
+            store_chunk(f, E, eimm, ck);
+            continue;
+        }
+        if (eop == OP_IOTA_ROW) {
+            const uint32_t r = (ck.row / E.scal(eimm)) % E.scal(eimm + 1);
+#pragma unroll
+            for (int i = 0; i < V; ++i) f[i] = u2f(r);
+        } else if (eop == OP_PHILOX) {
+            uint32_t w[V];
+            philox_chunk(w, ck.flat0, E.scal(eimm), E.scal(eimm + 1), E.scal(eimm + 2), E.scal(eimm + 3));
+#pragma unroll
+            for (int i = 0; i < V; ++i) f[i] = u2f(w[i]);
+        } else if (eop >= OP_RED_SUM && eop <= OP_RED_MIN) {
+            if constexpr (ROW) {
+                if (eop == OP_RED_SUM) row_reduce<0>(f, ck, rc);
+                else if (eop == OP_RED_MAX) row_reduce<1>(f, ck, rc);
+                else row_reduce<2>(f, ck, rc);
+            }
+        } else {  // correctly rounded transcendentals of the precise flavour
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                if (eop == OP_U_EXP) f[i] = un<OP_U_EXP, false>(f[i]);
+                else if (eop == OP_U_LOG) f[i] = un<OP_U_LOG, false>(f[i]);
+                else if (eop == OP_U_TANH) f[i] = un<OP_U_TANH, false>(f[i]);
+                else if (eop == OP_U_SIGMOID) f[i] = un<OP_U_SIGMOID, false>(f[i]);
+                else if (eop == OP_U_GELU) f[i] = un<OP_U_GELU, false>(f[i]);
+            }
+        }
+        pairs_of(f, R[4]);
+    }
+}
+
+template <class P>
+__device__ __forceinline__ void stage_program(Staged &S, const P &prm) {
+    for (uint32_t i = threadIdx.x; i < prm.n_ins + 2; i += blockDim.x) {
+        LtIns in;
+        in.op = OP_END;
+        in.imm = 0;
+        if (i < prm.n_ins) in = prm.ins[i];
+        S.ins[i] = in;
+    }
+    for (uint32_t i = threadIdx.x; i < LT_VM_MAX_SCAL; i += blockDim.x) S.scal[i] = prm.scal[i];
 }
 
 // ------------------------------------------------------------------ kernels
 template <bool FAST>
 __global__ void __launch_bounds__(LT_EW_THREADS) lt_ew_kernel(const __grid_constant__ LtKParams P) {
+    __shared__ Staged S;
     const EnvK E{P};
+    stage_program(S, P);
+    if (threadIdx.x < LT_VM_MAX_PTR)
+        S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], !P.rowcol || (P.cols % V) == 0);
+    __syncthreads();
+    const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
+    const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
+    const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; c < P.n_chunks; c += stride) {
         Chunk ck;
@@ -470,16 +535,23 @@ __global__ void __launch_bounds__(LT_EW_THREADS) lt_ew_kernel(const __grid_const
             const uint32_t rem = P.cols - ck.col0;
             ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
         }
-        run_program<FAST, false>(E, ck, nullptr);
+        run_program<FAST, false>(E, ck, nullptr, prog_s, scal_s, ptr_s);
     }
 }
 
 template <bool FAST, int MAXT>
 __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ LtKParams P) {
-    __shared__ float red_smem[64];
+    __shared__ Staged S;
     const EnvK E{P};
+    stage_program(S, P);
+    if (threadIdx.x < LT_VM_MAX_PTR)
+        S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], (P.cols % V) == 0);
+    __syncthreads();
+    const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
+    const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
+    const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
     RowCtx rc;
-    rc.smem = red_smem;
+    rc.smem = S.red;
     rc.phase = 0;
     rc.group = P.group;
     rc.warp = threadIdx.x >> 5;
@@ -499,12 +571,17 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
             nv = rem < (uint32_t)V ? (int)rem : V;
         }
         ck.nvalid = nv;
-        run_program<FAST, true>(E, ck, &rc);
+        run_program<FAST, true>(E, ck, &rc, prog_s, scal_s, ptr_s);
     }
 }
 
 template <bool FAST>
 __global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
+    __shared__ Staged S;
+    stage_program(S, P);
+    const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
+    const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
+    const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
     for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
         // instance that owns super-chunk sc: last i with super_prefix[i] <= sc
         uint32_t lo = 0, hi = P.n_inst;
@@ -513,6 +590,9 @@ __global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_co
             if (P.super_prefix[mid] <= sc) lo = mid; else hi = mid;
         }
         const EnvM E{P, lo * P.n_slots};
+        __syncthreads();  // the previous super-chunk's pointers are no longer in use
+        if (threadIdx.x < P.n_slots) S.ptr[threadIdx.x] = flag_pointer(E.ptr(threadIdx.x), P.io_dtype[threadIdx.x], true);
+        __syncthreads();
         const uint32_t numel = P.numel[lo];
         const uint32_t first = (sc - P.super_prefix[lo]) * (LT_EW_THREADS * LT_MULTI_SUB * V);
 #pragma unroll 1
@@ -526,7 +606,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_co
                 ck.row_ok = true;
                 const uint32_t rem = numel - e0;
                 ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
-                run_program<FAST, false>(E, ck, nullptr);
+                run_program<FAST, false>(E, ck, nullptr, prog_s, scal_s, ptr_s);
             }
         }
     }

@@ -100,14 +100,26 @@ struct CodeGen {
         for (int k = 0; k < LT_VM_NT; ++k) temp_val[k] = -1, temp_raw[k] = -1;
     }
 
-    void emit_ins(uint16_t op, uint8_t a = 0, uint32_t imm = 0) {
+    void emit_ins(uint32_t op, uint32_t imm = 0) {
         LtIns in;
         in.op = op;
-        in.a = a;
-        in.b = 0;
         in.imm = imm;
         g.ins.push_back(in);
     }
+
+    static uint32_t size_class(int dt) { return dt == LT_BF16 ? 1u : dt == LT_U8 ? 2u : 0u; }
+
+    // raw chunk load of input v into register d (0..3 = T0..T3, 4 = ACC)
+    void emit_load(int d, uint32_t v) {
+        const int s = input_slot(v);
+        const IoRef &io = g.io[s];
+        if (io.cls == LT_CLS_FULL || io.cls == LT_CLS_COLVEC)
+            emit_ins(OP_LDV + (size_class(io.dtype) * 2 + (io.cls == LT_CLS_COLVEC ? 1u : 0u)) * 5 + (uint32_t)d, (uint32_t)s);
+        else
+            emit_ins(OP_LD + (uint32_t)d, (uint32_t)s);
+    }
+
+    void emit_widen(int d, int dt) { emit_ins((dt == LT_BF16 ? OP_CVT_BF16 : OP_CVT_U8) + (uint32_t)d); }
 
     int cls_of(uint32_t v) const {
         const PNode &p = pn[v];
@@ -193,7 +205,7 @@ struct CodeGen {
 
     void widen_temp(int k) {
         if (temp_raw[k] >= 0) {
-            emit_ins((uint16_t)(OP_CVT_T + k), (uint8_t)temp_raw[k]);
+            emit_widen(k, temp_raw[k]);
             temp_raw[k] = -1;
         }
     }
@@ -209,10 +221,9 @@ struct CodeGen {
         if (in_acc == v) {
             emit_ins((uint16_t)(OP_MOV_T_ACC + k));
         } else if (is_input((uint32_t)v)) {
-            int s = input_slot((uint32_t)v);
-            emit_ins((uint16_t)(OP_LD_T + k), 0, (uint32_t)s);
+            emit_load(k, (uint32_t)v);
             int dt = cg.nodes[v].dtype;
-            if (needs_widen(dt)) emit_ins((uint16_t)(OP_CVT_T + k), (uint8_t)dt);
+            if (needs_widen(dt)) emit_widen(k, dt);
         } else {
             ok = false;  // value was never computed: planner bug
             return 0;
@@ -232,10 +243,9 @@ struct CodeGen {
             widen_temp(temp_of[v]);
             emit_ins((uint16_t)(OP_MOV_ACC_T + temp_of[v]));
         } else if (is_input((uint32_t)v)) {
-            int s = input_slot((uint32_t)v);
-            emit_ins(OP_LD_ACC, 0, (uint32_t)s);
+            emit_load(4, (uint32_t)v);
             int dt = cg.nodes[v].dtype;
-            if (needs_widen(dt)) emit_ins(OP_CVT_ACC, (uint8_t)dt);
+            if (needs_widen(dt)) emit_widen(4, dt);
         } else {
             ok = false;
             return;
@@ -260,8 +270,7 @@ struct CodeGen {
         for (int i = 0; i < count && i < (int)order.size() && i < LT_VM_NT; ++i) {
             uint32_t v = order[i];
             int k = alloc_temp();
-            int s = input_slot(v);
-            emit_ins((uint16_t)(OP_LD_T + k), 0, (uint32_t)s);
+            emit_load(k, v);
             temp_val[k] = (int)v;
             temp_of[v] = k;
             int dt = cg.nodes[v].dtype;
@@ -300,7 +309,7 @@ struct CodeGen {
         if (io.cls == LT_CLS_ROWVEC && !has_reduce) needs_rowcol = true;
         int s = (int)g.io.size();
         g.io.push_back(io);
-        emit_ins(OP_ST, 0, (uint32_t)s);
+        emit_ins(io.cls == LT_CLS_FULL ? OP_STV + size_class(io.dtype) : (uint32_t)OP_ST, (uint32_t)s);
     }
 
     // ---- one node
@@ -340,7 +349,7 @@ struct CodeGen {
             if (xs && ys) {
                 spill_acc();
                 if (!ok) return;
-                emit_ins(OP_MOV_ACC_S, 0, (uint32_t)scalar_imm(xo, odt));
+                emit_ins(OP_MOV_ACC_S, (uint32_t)scalar_imm(xo, odt));
                 in_acc = -1;
                 src = LT_VM_SRC_S;
                 imm = (uint32_t)scalar_imm(yo, odt);
@@ -419,7 +428,7 @@ struct CodeGen {
                 }
                 code = (uint16_t)(OP_I2 + idx * LT_VM_NSRC + src);
             }
-            emit_ins(code, 0, imm);
+            emit_ins(code, imm);
             if (x >= 0) drop_if_dead(x);
             if (y >= 0) drop_if_dead(y);
         } else if (op == LT_OP_WHERE) {
@@ -435,7 +444,7 @@ struct CodeGen {
             if (as && bs) {
                 spill_acc();
                 if (!ok) return;
-                emit_ins(OP_MOV_ACC_S, 0, (uint32_t)scalar_imm(ao, dt));
+                emit_ins(OP_MOV_ACC_S, (uint32_t)scalar_imm(ao, dt));
                 in_acc = -1;
                 src = LT_VM_SRC_S;
                 imm = (uint32_t)scalar_imm(bo, dt);
@@ -468,7 +477,7 @@ struct CodeGen {
             if (!ok) return;
             mk = temp_of[m];  // unchanged, but re-read after possible spills
             consume(m);
-            emit_ins((uint16_t)((variant_b ? OP_WHERE_B : OP_WHERE_A) + mk * LT_VM_NSRC + src), 0, imm);
+            emit_ins((uint32_t)((variant_b ? OP_WHERE_B : OP_WHERE_A) + mk * LT_VM_NSRC + src), imm);
             drop_if_dead(m);
             if (a >= 0) drop_if_dead(a);
             if (b >= 0) drop_if_dead(b);
@@ -477,7 +486,7 @@ struct CodeGen {
             if (cg.nodes[xo].op == N_SCALAR) {
                 spill_acc();
                 if (!ok) return;
-                emit_ins(OP_MOV_ACC_S, 0, (uint32_t)scalar_imm(xo, cg.nodes[xo].dtype));
+                emit_ins(OP_MOV_ACC_S, (uint32_t)scalar_imm(xo, cg.nodes[xo].dtype));
                 in_acc = -1;
             } else {
                 int x = rep_or_self(xo);
@@ -534,7 +543,7 @@ struct CodeGen {
                 Imm a{-1, (double)inner, ENC_U32}, b{-1, (double)cn.dims[cn.attr0], ENC_U32};
                 int s = imm_slot(a, false);
                 imm_slot(b, false);
-                emit_ins(OP_IOTA_ROW, 0, (uint32_t)s);
+                emit_ins(OP_IOTA_ROW, (uint32_t)s);
                 needs_rowcol = true;
             }
         } else if (op == LT_OP_PHILOX_BITS) {
@@ -545,7 +554,7 @@ struct CodeGen {
             imm_slot(k1, false);
             imm_slot(o0, false);
             imm_slot(o1, false);
-            emit_ins(OP_PHILOX, 0, (uint32_t)s);
+            emit_ins(OP_PHILOX, (uint32_t)s);
         } else {
             ok = false;
             return;
@@ -622,11 +631,18 @@ std::string disasm(const LtIns &in) {
     if (op >= OP_MOV_T_ACC && op < OP_MOV_ACC_T) snprintf(buf, sizeof(buf), "T%d = ACC", op - OP_MOV_T_ACC);
     else if (op >= OP_MOV_ACC_T && op < OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = T%d", op - OP_MOV_ACC_T);
     else if (op == OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = S%u", in.imm);
-    else if (op >= OP_LD_T && op < OP_LD_ACC) snprintf(buf, sizeof(buf), "T%d = load p%u", op - OP_LD_T, in.imm);
-    else if (op == OP_LD_ACC) snprintf(buf, sizeof(buf), "ACC = load p%u", in.imm);
-    else if (op >= OP_CVT_T && op < OP_CVT_ACC) snprintf(buf, sizeof(buf), "T%d = widen.%s T%d", op - OP_CVT_T, dtype_name(in.a), op - OP_CVT_T);
-    else if (op == OP_CVT_ACC) snprintf(buf, sizeof(buf), "ACC = widen.%s ACC", dtype_name(in.a));
-    else if (op == OP_ST) snprintf(buf, sizeof(buf), "store p%u = ACC", in.imm);
+    else if (op >= OP_LD && op < OP_STV) {
+        const int d = op < OP_LDV ? op - OP_LD : (op - OP_LDV) % 5;
+        const char *how = op < OP_LDV ? "load" : "vload";
+        if (d < 4) snprintf(buf, sizeof(buf), "T%d = %s p%u", d, how, in.imm);
+        else snprintf(buf, sizeof(buf), "ACC = %s p%u", how, in.imm);
+    } else if (op >= OP_CVT_BF16 && op < OP_ST) {
+        const int d = (op - OP_CVT_BF16) % 5;
+        const char *ty = op < OP_CVT_U8 ? "bf16" : "u8";
+        if (d < 4) snprintf(buf, sizeof(buf), "T%d = widen.%s T%d", d, ty, d);
+        else snprintf(buf, sizeof(buf), "ACC = widen.%s ACC", ty);
+    } else if (op == OP_ST) snprintf(buf, sizeof(buf), "store p%u = ACC", in.imm);
+    else if (op >= OP_STV && op < OP_STV + 3) snprintf(buf, sizeof(buf), "vstore p%u = ACC", in.imm);
     else if (op == OP_IOTA_COL) snprintf(buf, sizeof(buf), "ACC = iota.col");
     else if (op == OP_IOTA_ROW) snprintf(buf, sizeof(buf), "ACC = iota.row S%u S%u", in.imm, in.imm + 1);
     else if (op == OP_PHILOX) snprintf(buf, sizeof(buf), "ACC = philox S%u..S%u", in.imm, in.imm + 3);
@@ -1050,8 +1066,8 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                         int ld_pos = -1, st_pos = -1;
                         for (size_t q = 0; q < g.ins.size(); ++q) {
                             const LtIns &in = g.ins[q];
-                            if (in.op >= OP_LD_T && in.op <= OP_LD_ACC && in.imm == rd.second && ld_pos < 0) ld_pos = (int)q;
-                            if (in.op == OP_ST && in.imm == s) st_pos = (int)q;
+                            if (in.op >= OP_LD && in.op < OP_STV && in.imm == rd.second && ld_pos < 0) ld_pos = (int)q;
+                            if ((in.op == OP_ST || (in.op >= OP_STV && in.op < OP_STV + 3)) && in.imm == s) st_pos = (int)q;
                         }
                         if (ld_pos < 0 || st_pos < 0 || ld_pos > st_pos) { safe = false; break; }
                     } else if (launch_of[rg] >= launch_of[gi]) {

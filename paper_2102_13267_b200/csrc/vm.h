@@ -15,7 +15,7 @@
 #define LT_VM_NT 4         // temporaries T0..T3
 #define LT_VM_NSRC 5       // operand sources of two-operand opcodes: T0..T3, S (broadcast immediate)
 #define LT_VM_SRC_S 4
-#define LT_VM_MAX_INS 120
+#define LT_VM_MAX_INS 118     // the program is followed by an END and one padding slot
 #define LT_VM_MAX_PTR 12
 #define LT_VM_MAX_SCAL 32
 
@@ -26,10 +26,8 @@
 #define LT_MULTI_SUB 4          // chunks each thread runs per super-chunk
 
 struct LtIns {
-    uint16_t op;
-    uint8_t a;     // small operand: dtype for CVT
-    uint8_t b;
-    uint32_t imm;  // pointer slot, immediate slot
+    uint32_t op;
+    uint32_t imm;  // pointer slot or immediate slot
 };
 
 // element classes of a pointer slot relative to the group's [rows, cols] domain
@@ -42,29 +40,32 @@ enum {
     OP_MOV_T_ACC = 1,    // +k : T[k] = ACC
     OP_MOV_ACC_T = 5,    // +k : ACC = T[k]
     OP_MOV_ACC_S = 9,    // ACC = broadcast(imm slot)
-    OP_LD_T = 10,        // +k : T[k] = raw chunk of pointer slot imm (storage format, see CVT)
-    OP_LD_ACC = 14,
-    OP_CVT_T = 15,       // +k : widen the raw chunk in T[k] from storage dtype `a` to 32-bit lanes
-    OP_CVT_ACC = 19,
-    OP_ST = 20,          // store ACC to pointer slot imm, narrowing to the slot's dtype
+    OP_CVT_BF16 = 10,    // +d : widen the raw bf16 chunk held in register d (0..3 = T0..T3, 4 = ACC) to f32 lanes
+    OP_CVT_U8 = 15,      // +d : widen a raw u8 chunk to 32-bit lanes
+    OP_ST = 20,          // store ACC to pointer slot imm, any class and dtype (handled outside the PTX core)
     OP_IOTA_COL = 21,    // ACC = column index of each lane (i32)
     OP_IOTA_ROW = 22,    // ACC = (row / scal[imm]) % scal[imm+1] (i32), same in every lane
     OP_PHILOX = 23,      // ACC = random bits of each lane's flat index; scal[imm..imm+3] = seed lo,hi, offset lo,hi
     OP_RED_SUM = 24,     // ACC = sum over the row, broadcast to every lane   (row kernel only)
     OP_RED_MAX = 25,
     OP_RED_MIN = 26,
-    // one-operand float ops on ACC
+    // one-operand ops on ACC
     OP_U_NEG = 30, OP_U_ABS, OP_U_RELU, OP_U_EXP, OP_U_LOG, OP_U_TANH, OP_U_SQRT, OP_U_RSQRT, OP_U_RECIP,
     OP_U_SQUARE, OP_U_SIGMOID, OP_U_GELU, OP_U_RBF16 /* round to bf16, keep as f32 */,
     OP_U_INEG = 43, OP_U_IABS = 44, OP_U_NOT = 45,
     OP_C_I2F = 46, OP_C_U2F = 47, OP_C_F2I = 48, OP_C_NZF = 49 /* f32 != 0 -> 0/1 */, OP_C_NZI = 50,
+    OP_LD = 51,          // +d : raw chunk load of pointer slot imm, any class and dtype (outside the PTX core)
+    // +(size * 2 + class) * 5 + d : raw chunk load on the vector path; size 0/1/2 = 4/2/1-byte elements,
+    // class 0 = full, 1 = column vector.  Ragged chunks and unaligned pointers fall back to OP_LD's code.
+    OP_LDV = 56,
+    OP_STV = 86,         // +size : vector-path store of ACC to a full-class slot (falls back to OP_ST's code)
     // two-operand families: opcode = base + index * LT_VM_NSRC + source
-    OP_F2 = 64,          // ACC = ACC (op) src, f32: see F2_*
-    OP_I2 = 104,         // integer: see I2_*
-    OP_CMP = 160,        // ACC = (ACC cmp src) ? 1 : 0 : see CMP_*
-    OP_WHERE_A = 256,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? ACC : src
-    OP_WHERE_B = 276,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? src : ACC
-    OP_LIMIT = 296
+    OP_F2 = 96,          // ACC = ACC (op) src, f32: see F2_*
+    OP_I2 = 136,         // integer: see I2_*
+    OP_CMP = 192,        // ACC = (ACC cmp src) ? 1 : 0 : see CC_*
+    OP_WHERE_A = 288,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? ACC : src
+    OP_WHERE_B = 308,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? src : ACC
+    OP_LIMIT = 328
 };
 
 enum { F2_ADD = 0, F2_SUB, F2_RSUB, F2_MUL, F2_DIV, F2_RDIV, F2_MAX, F2_MIN, F2_COUNT };
@@ -72,9 +73,11 @@ enum { I2_ADD = 0, I2_SUB, I2_RSUB, I2_MUL, I2_AND, I2_OR, I2_XOR, I2_MAXS, I2_M
 // compare index = type * 6 + cc ; type 0 f32, 1 signed, 2 unsigned ; cc: GT GE LT LE EQ NE
 enum { CC_GT = 0, CC_GE, CC_LT, CC_LE, CC_EQ, CC_NE };
 
+static_assert(OP_LDV + 30 == OP_STV && OP_STV + 3 <= OP_F2, "opcode map");
 static_assert(OP_F2 + F2_COUNT * LT_VM_NSRC == OP_I2, "opcode map");
 static_assert(OP_I2 + I2_COUNT * LT_VM_NSRC <= OP_CMP, "opcode map");
 static_assert(OP_CMP + 18 * LT_VM_NSRC <= OP_WHERE_A, "opcode map");
+static_assert(OP_WHERE_B + 4 * LT_VM_NSRC == OP_LIMIT, "opcode map");
 
 // Kernel parameter block of the elementwise and row-reduction kernels.  It is passed by
 // value as a __grid_constant__ kernel parameter, so program, pointers and immediates are
@@ -102,7 +105,7 @@ struct LtKParams {
 struct LtMultiParams {
     LtIns ins[LT_MULTI_MAX_INS];
     uint32_t scal[LT_VM_MAX_SCAL];
-    uint8_t io_dtype[LT_MULTI_MAX_SLOTS];
+    uint8_t io_dtype[LT_VM_MAX_PTR];
     uint32_t n_ins;
     uint32_t n_inst;
     uint32_t n_slots;
