@@ -149,6 +149,10 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * "verify" (1 default: on a cache hit compare the canonical bytes, not just the hash),
  * "fast_math" (1 default: groups whose stored results are all bf16/u8 may use approximate
  * exp/tanh/rsqrt/division and fused multiply-add; groups storing f32 never do),
+ * "ieee" (0 default: in groups storing f32, division, square root and reciprocal are accurate to
+ * 2 ulp; 1 = correctly rounded, so that a graph of + - * / sqrt matches an op-by-op binary32
+ * evaluation bit for bit, at about ten more instructions per element and op),
+ * "waves" (4 default: grid size of the persistent kernels in waves of resident thread blocks),
  * "horizontal" (1 default: bundle isomorphic independent groups into multi-tensor launches),
  * "cache_capacity" (0 = unbounded).  Options are part of the cache key.
  * Unknown key: LT_ERR_INVALID_ARG.  The environment variables LT_FUSION, LT_VERIFY,

@@ -230,7 +230,8 @@ class LazyContext:
     def close(self):
         if self._ctx:
             ctx, self._ctx = self._ctx, None
-            _lib.lt_ctx_destroy(ctx)
+            if _lib is not None:  # module globals may already be gone at interpreter shutdown
+                _lib.lt_ctx_destroy(ctx)
 
     def _flush_dead(self):
         """Unregister the tensors Python has dropped since the last flush."""

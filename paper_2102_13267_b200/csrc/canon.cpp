@@ -182,6 +182,7 @@ void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonica
     put<int64_t>(b, c->opt.fusion);
     put<int64_t>(b, c->opt.fast_math);
     put<int64_t>(b, c->opt.horizontal);
+    put<int64_t>(b, c->opt.ieee);
     put<uint32_t>(b, (uint32_t)cg.nodes.size());
     for (const CNode &n : cg.nodes) {
         put<uint16_t>(b, n.op);

@@ -333,6 +333,8 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "fast_math")) c->opt.fast_math = value;
     else if (!strcmp(key, "horizontal")) c->opt.horizontal = value;
     else if (!strcmp(key, "cache_capacity")) c->opt.cache_capacity = value;
+    else if (!strcmp(key, "ieee")) c->opt.ieee = value;
+    else if (!strcmp(key, "waves")) c->opt.waves = value;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
 }

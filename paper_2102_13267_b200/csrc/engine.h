@@ -106,7 +106,7 @@ enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2 };
 
 struct Group {
     uint8_t kind = K_EW;
-    bool fast = false;
+    uint8_t flavour = 1;  // 0 fast, 1 precise, 2 ieee (see launch.h)
     bool rowcol = false;
     uint64_t rows = 1, cols = 1;
     std::vector<uint32_t> members;  // native members (canonical indices), topological order
@@ -118,7 +118,7 @@ struct Group {
 
 struct Launch {
     uint8_t kind = K_EW;
-    bool fast = false;
+    uint8_t flavour = 1;
     std::vector<uint32_t> groups;   // one group, or the instances of a multi-tensor launch
     uint64_t bytes = 0;
     unsigned threads = LT_EW_THREADS;
@@ -145,7 +145,7 @@ struct Plan {
 };
 
 struct Options {
-    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0;
+    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 4;
 };
 
 struct HashKey {

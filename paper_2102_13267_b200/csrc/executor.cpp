@@ -99,7 +99,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
         return (uint64_t)(uintptr_t)p;
     };
 
-    const unsigned waves = 4;
+    const unsigned waves = (unsigned)std::max<int64_t>(1, c->opt.waves);
     for (Launch &L : plan.launches) {
         cudaError_t e = cudaSuccess;
         cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -120,7 +120,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * c->occ_multi * waves);
                 if (grid < 1) grid = 1;
                 if (ev0) cudaEventRecord(ev0, c->stream);
-                e = lt_launch_multi(P, L.fast, grid, c->stream);
+                e = lt_launch_multi(P, L.flavour, grid, c->stream);
                 if (ev1) cudaEventRecord(ev1, c->stream);
             }
             c->stats.launches_multi++;
@@ -135,7 +135,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_launch_ew(P, L.fast, grid, c->stream);
+                    e = lt_launch_ew(P, L.flavour, grid, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                 }
                 c->stats.launches_elementwise++;
@@ -146,7 +146,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     unsigned grid = (unsigned)std::min<uint64_t>(blocks, (uint64_t)c->sm_count * per_sm * waves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_launch_row(P, L.fast, grid, L.threads, c->stream);
+                    e = lt_launch_row(P, L.flavour, grid, L.threads, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                 }
                 c->stats.launches_row++;

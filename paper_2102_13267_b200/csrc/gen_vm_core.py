@@ -53,7 +53,7 @@ NSRC = OPS["LT_VM_NSRC"]
 A = [f"%{i}" for i in range(4)]
 T = [[f"%{4 + 4 * k + j}" for j in range(4)] for k in range(4)]
 REG = T + [A]  # destination index 0..3 = temporaries, 4 = ACC
-PC, EOP, EIMM, SB, PB, OFF4, COFF4, TAIL = "%20", "%21", "%22", "%23", "%24", "%25", "%26", "%27"
+PC, EOP, EIMM, SB, PB, OFF4, COFF4, TAIL, PF4 = "%20", "%21", "%22", "%23", "%24", "%25", "%26", "%27", "%28"
 
 
 def f32_hex(x: float) -> int:
@@ -102,7 +102,30 @@ class Src:
         return [], ["sv"] * 8
 
 
-def f2_body(idx: int, src: Src, fast: bool):
+def div_ins(flavour: str) -> str:
+    # fast: rcp-and-multiply; precise: full-range division within 2 ulp; ieee: correctly rounded
+    return {"fast": "div.approx.f32", "precise": "div.full.f32", "ieee": "div.rn.f32"}[flavour]
+
+
+def pairwise(a_pairs, src, fmt_lines):
+    """Lane-by-lane op on ACC done one register pair at a time (keeps few registers live).
+    fmt_lines(x, y) -> PTX lines computing x = op(x, y) for one lane."""
+    lines = []
+    for j in range(4):
+        lines.append(f"mov.b64 {{x0, x1}}, {a_pairs[j]};")
+        if src is None:
+            ys = (None, None)
+        elif src.kind < 4:
+            lines.append(f"mov.b64 {{y0, y1}}, {src.pairs[j]};")
+            ys = ("y0", "y1")
+        else:
+            ys = ("sv", "sv")
+        lines += fmt_lines("x0", ys[0]) + fmt_lines("x1", ys[1])
+        lines.append(f"mov.b64 {a_pairs[j]}, {{x0, x1}};")
+    return lines
+
+
+def f2_body(idx: int, src: Src, flavour: str):
     names = ["add", "sub", "rsub", "mul", "div", "rdiv", "max", "min"]
     op = names[idx]
     lines = list(src.pre)
@@ -110,31 +133,21 @@ def f2_body(idx: int, src: Src, fast: bool):
         lines += [f"{op}.rn.f32x2 {A[j]}, {A[j]}, {src.pairs[j]};" for j in range(4)]
     elif op == "rsub":
         lines += [f"sub.rn.f32x2 {A[j]}, {src.pairs[j]}, {A[j]};" for j in range(4)]
+    elif op == "div":
+        lines += pairwise(A, src, lambda x, y: [f"{div_ins(flavour)} {x}, {x}, {y};"])
+    elif op == "rdiv":
+        lines += pairwise(A, src, lambda x, y: [f"{div_ins(flavour)} {x}, {y}, {x};"])
     else:
-        ul, y = src.lanes(Y)
-        lines += unpack(A, X) + ul
-        for i in range(8):
-            if op == "div":
-                lines.append(f"div.{'approx' if fast else 'rn'}.f32 {X[i]}, {X[i]}, {y[i]};")
-            elif op == "rdiv":
-                lines.append(f"div.{'approx' if fast else 'rn'}.f32 {X[i]}, {y[i]}, {X[i]};")
-            else:
-                lines.append(f"{op}.NaN.f32 {X[i]}, {X[i]}, {y[i]};")
-        lines += pack(A, X)
+        lines += pairwise(A, src, lambda x, y: [f"{op}.NaN.f32 {x}, {x}, {y};"])
     return lines
 
 
 def i2_body(idx: int, src: Src):
     ops = ["add.s32", "sub.s32", "rsub", "mul.lo.s32", "and.b32", "or.b32", "xor.b32", "max.s32", "min.s32", "max.u32", "min.u32"]
     op = ops[idx]
-    ul, y = src.lanes(Y)
-    lines = list(src.pre) + unpack(A, X) + ul
-    for i in range(8):
-        if op == "rsub":
-            lines.append(f"sub.s32 {X[i]}, {y[i]}, {X[i]};")
-        else:
-            lines.append(f"{op} {X[i]}, {X[i]}, {y[i]};")
-    return lines + pack(A, X)
+    if op == "rsub":
+        return list(src.pre) + pairwise(A, src, lambda x, y: [f"sub.s32 {x}, {y}, {x};"])
+    return list(src.pre) + pairwise(A, src, lambda x, y: [f"{op} {x}, {x}, {y};"])
 
 
 def cmp_body(idx: int, src: Src):
@@ -146,20 +159,23 @@ def cmp_body(idx: int, src: Src):
         ins = f"setp.{ccn}.s32"
     else:
         ins = f"setp.{ {'gt': 'hi', 'ge': 'hs', 'lt': 'lo', 'le': 'ls', 'eq': 'eq', 'ne': 'ne'}[ccn] }.u32"
-    ul, y = src.lanes(Y)
-    lines = list(src.pre) + unpack(A, X) + ul
-    for i in range(8):
-        lines += [f"{ins} p, {X[i]}, {y[i]};", f"selp.b32 {X[i]}, 1, 0, p;"]
-    return lines + pack(A, X)
+    return list(src.pre) + pairwise(A, src, lambda x, y: [f"{ins} p, {x}, {y};", f"selp.b32 {x}, 1, 0, p;"])
 
 
 def where_body(m: int, src: Src, variant_b: bool):
-    ul, y = src.lanes(Y)
-    lines = list(src.pre) + unpack(A, X) + unpack(T[m], M) + ul
-    for i in range(8):
-        lines.append(f"setp.ne.u32 p, {M[i]}, 0;")
-        lines.append(f"selp.b32 {X[i]}, {y[i]}, {X[i]}, p;" if variant_b else f"selp.b32 {X[i]}, {X[i]}, {y[i]}, p;")
-    return lines + pack(A, X)
+    lines = list(src.pre)
+    for j in range(4):
+        lines += [f"mov.b64 {{x0, x1}}, {A[j]};", f"mov.b64 {{m0, m1}}, {T[m][j]};"]
+        if src.kind < 4:
+            lines.append(f"mov.b64 {{y0, y1}}, {src.pairs[j]};")
+            ys = ("y0", "y1")
+        else:
+            ys = ("sv", "sv")
+        for x, mm, y in (("x0", "m0", ys[0]), ("x1", "m1", ys[1])):
+            lines.append(f"setp.ne.u32 p, {mm}, 0;")
+            lines.append(f"selp.b32 {x}, {y}, {x}, p;" if variant_b else f"selp.b32 {x}, {x}, {y}, p;")
+        lines.append(f"mov.b64 {A[j]}, {{x0, x1}};")
+    return lines
 
 
 LOG2E, LN2 = 1.4426950408889634, 0.6931471805599453
@@ -168,10 +184,12 @@ GELU_KC = GELU_K * 0.044715
 
 
 def lanes_op(fmt: str):
-    return unpack(A, X) + [fmt.format(x=X[i]) for i in range(8)] + pack(A, X)
+    return pairwise(A, None, lambda x, y: [fmt.format(x=x)])
 
 
-def unary_body(name: str, fast: bool):
+def unary_body(name: str, flavour: str):
+    fast = flavour == "fast"
+    ieee = flavour == "ieee"
     """Returns PTX lines, or None when the opcode escapes to C++ in this flavour."""
     if name == "OP_U_NEG":
         return [f"xor.b64 {a}, {a}, 0x8000000080000000;" for a in A]
@@ -182,23 +200,23 @@ def unary_body(name: str, fast: bool):
     if name == "OP_U_SQUARE":
         return [f"mul.rn.f32x2 {a}, {a}, {a};" for a in A]
     if name == "OP_U_SQRT":
-        return lanes_op("sqrt.approx.f32 {x}, {x};" if fast else "sqrt.rn.f32 {x}, {x};")
+        return lanes_op("sqrt.rn.f32 {x}, {x};" if ieee else "sqrt.approx.f32 {x}, {x};")
     if name == "OP_U_RSQRT":
         return lanes_op("rsqrt.approx.f32 {x}, {x};")
     if name == "OP_U_RECIP":
-        return lanes_op("rcp.approx.ftz.f32 {x}, {x};" if fast else "rcp.rn.f32 {x}, {x};")
+        return lanes_op("rcp.rn.f32 {x}, {x};" if ieee else ("rcp.approx.ftz.f32 {x}, {x};" if fast else "rcp.approx.f32 {x}, {x};"))
     if name == "OP_U_RBF16":
-        lines = unpack(A, X)
+        lines = []
         for j in range(4):
-            lines += [f"cvt.rn.bf16x2.f32 w0, {X[2 * j + 1]}, {X[2 * j]};", f"shl.b32 {X[2 * j]}, w0, 16;",
-                      f"and.b32 {X[2 * j + 1]}, w0, 0xFFFF0000;"]
-        return lines + pack(A, X)
+            lines += [f"mov.b64 {{x0, x1}}, {A[j]};", "cvt.rn.bf16x2.f32 w0, x1, x0;", "shl.b32 x0, w0, 16;",
+                      "and.b32 x1, w0, 0xFFFF0000;", f"mov.b64 {A[j]}, {{x0, x1}};"]
+        return lines
     if name == "OP_U_INEG":
         return lanes_op("neg.s32 {x}, {x};")
     if name == "OP_U_IABS":
         return lanes_op("abs.s32 {x}, {x};")
     if name == "OP_U_NOT":
-        return unpack(A, X) + sum(([f"setp.eq.u32 p, {x}, 0;", f"selp.b32 {x}, 1, 0, p;"] for x in X), []) + pack(A, X)
+        return pairwise(A, None, lambda x, y: [f"setp.eq.u32 p, {x}, 0;", f"selp.b32 {x}, 1, 0, p;"])
     if name == "OP_C_I2F":
         return lanes_op("cvt.rn.f32.s32 {x}, {x};")
     if name == "OP_C_U2F":
@@ -206,9 +224,9 @@ def unary_body(name: str, fast: bool):
     if name == "OP_C_F2I":
         return lanes_op("cvt.rzi.s32.f32 {x}, {x};")
     if name == "OP_C_NZF":
-        return unpack(A, X) + sum(([f"setp.neu.f32 p, {x}, 0f00000000;", f"selp.b32 {x}, 1, 0, p;"] for x in X), []) + pack(A, X)
+        return pairwise(A, None, lambda x, y: [f"setp.neu.f32 p, {x}, 0f00000000;", f"selp.b32 {x}, 1, 0, p;"])
     if name == "OP_C_NZI":
-        return unpack(A, X) + sum(([f"setp.ne.u32 p, {x}, 0;", f"selp.b32 {x}, 1, 0, p;"] for x in X), []) + pack(A, X)
+        return pairwise(A, None, lambda x, y: [f"setp.ne.u32 p, {x}, 0;", f"selp.b32 {x}, 1, 0, p;"])
     if not fast:
         return None  # exp, log, tanh, sigmoid, gelu: correctly rounded versions live in C++
     if name == "OP_U_EXP":
@@ -225,13 +243,12 @@ def unary_body(name: str, fast: bool):
     if name == "OP_U_GELU":
         lines = [const_pair("c0", GELU_KC), const_pair("c1", GELU_K), const_pair("c2", 0.5)]
         for j, a in enumerate(A):
-            g = f"g{j}"
+            g = "g0"
             lines += [f"mul.rn.f32x2 {g}, {a}, {a};",
                       f"fma.rn.f32x2 {g}, {g}, c0, c1;",
                       f"mul.rn.f32x2 {g}, {g}, {a};",
-                      f"mov.b64 {{{X[2 * j]}, {X[2 * j + 1]}}}, {g};",
-                      f"tanh.approx.f32 {X[2 * j]}, {X[2 * j]};", f"tanh.approx.f32 {X[2 * j + 1]}, {X[2 * j + 1]};",
-                      f"mov.b64 {g}, {{{X[2 * j]}, {X[2 * j + 1]}}};",
+                      f"mov.b64 {{x0, x1}}, {g};", "tanh.approx.f32 x0, x0;", "tanh.approx.f32 x1, x1;",
+                      f"mov.b64 {g}, {{x0, x1}};",
                       f"mul.rn.f32x2 {a}, {a}, c2;",
                       f"fma.rn.f32x2 {a}, {a}, {g}, {a};"]
         return lines
@@ -269,6 +286,10 @@ def ldv_body(sz: int, cls: int, d: int):
     else:
         lines += [f"cvt.u64.u32 offs, {COFF4};"] + ([f"shr.u64 offs, offs, {sz};"] if sz else [])
     lines.append("add.u64 ptr, ptr, offs;")
+    if cls == 0:
+        # pull this thread's next chunk of the same input into L2 while the current one is processed
+        lines += [f"shr.u64 offs, {PF4}, {sz};" if sz else f"mov.b64 offs, {PF4};", "add.u64 offs, ptr, offs;",
+                  "@pnext prefetch.global.L2 [offs];"]
     ld = "ld.global.cs" if cls == 0 else "ld.global.nc"
     if sz == 0:
         lines += [f"{ld}.v4.b32 {{x0, x1, x2, x3}}, [ptr];", f"{ld}.v4.b32 {{x4, x5, x6, x7}}, [ptr+16];"] + pack(P, X)
@@ -299,7 +320,7 @@ def stv_body(sz: int):
     return lines
 
 
-def build(fast: bool) -> list[str]:
+def build(flavour: str) -> list[str]:
     limit = OPS["OP_LIMIT"]
     bodies: dict[int, list[str]] = {}
 
@@ -315,7 +336,7 @@ def build(fast: bool) -> list[str]:
     for name in ("OP_U_NEG", "OP_U_ABS", "OP_U_RELU", "OP_U_EXP", "OP_U_LOG", "OP_U_TANH", "OP_U_SQRT", "OP_U_RSQRT",
                  "OP_U_RECIP", "OP_U_SQUARE", "OP_U_SIGMOID", "OP_U_GELU", "OP_U_RBF16", "OP_U_INEG", "OP_U_IABS",
                  "OP_U_NOT", "OP_C_I2F", "OP_C_U2F", "OP_C_F2I", "OP_C_NZF", "OP_C_NZI"):
-        b = unary_body(name, fast)
+        b = unary_body(name, flavour)
         if b is not None:
             bodies[OPS[name]] = b
     for sz in range(3):
@@ -325,7 +346,7 @@ def build(fast: bool) -> list[str]:
         bodies[OPS["OP_STV"] + sz] = stv_body(sz)
     for idx in range(OPS["F2_COUNT"]):
         for k in range(NSRC):
-            bodies[OPS["OP_F2"] + idx * NSRC + k] = f2_body(idx, Src(k), fast)
+            bodies[OPS["OP_F2"] + idx * NSRC + k] = f2_body(idx, Src(k), flavour)
     for idx in range(OPS["I2_COUNT"]):
         for k in range(NSRC):
             bodies[OPS["OP_I2"] + idx * NSRC + k] = i2_body(idx, Src(k))
@@ -339,23 +360,23 @@ def build(fast: bool) -> list[str]:
 
     out = ["{"]
     out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3;")
-    out.append(".reg .b32 " + ", ".join(X + Y + M) + ";")
-    out.append(".reg .b64 ss, ptr, offs, g0, g1, g2, g3, c0, c1, c2;")
-    out.append(".reg .pred p, ptail;")
+    out.append(".reg .b32 " + ", ".join(X + ["y0", "y1", "m0", "m1"]) + ";")
+    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2;")
+    out.append(".reg .pred p, ptail, pnext;")
     table = ", ".join(f"L_{i}" if i in bodies else "L_ESC" for i in range(limit))
     out.append(f"TBL: .branchtargets {table};")
     out.append(f"setp.ne.u32 ptail, {TAIL}, 0;")
+    out.append(f"setp.ne.u64 pnext, {PF4}, 0;")
     out.append(f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];")
-    out.append("L_DISPATCH:")
-    out.append("mov.b32 op, nop;")
-    out.append("mov.b32 imm, nimm;")
-    out.append(f"add.u32 {PC}, {PC}, 8;")
-    out.append(f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];")  # the slot after the last instruction is padding
-    out.append("brx.idx op, TBL;")
+    # fetch/decode/jump; repeated at the end of every body so a body falls straight into the next jump.
+    # The next instruction word is fetched one step ahead (the slot after the last instruction is padding).
+    dispatch = ["mov.b32 op, nop;", "mov.b32 imm, nimm;", f"add.u32 {PC}, {PC}, 8;",
+                f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];", "brx.idx op, TBL;"]
+    out += dispatch
     for code in sorted(bodies):
         out.append(f"L_{code}:")
         out += bodies[code]
-        out.append("bra.uni L_DISPATCH;")
+        out += dispatch
     out.append("L_ESC:")
     out.append(f"mov.b32 {EOP}, op;")
     out.append(f"mov.b32 {EIMM}, imm;")
@@ -372,9 +393,10 @@ def main() -> None:
     text = ("// Generated by gen_vm_core.py from vm.h -- do not edit.\n"
             "// Operands: %0-%3 ACC, %4-%19 T0..T3 (f32x2 pairs); %20 pc (shared address); %21 escape opcode;\n"
             "// %22 escape immediate; %23 immediates base; %24 pointer table base (shared addresses);\n"
-            "// %25 chunk byte offset for 4-byte elements; %26 column byte offset; %27 ragged-chunk flag.\n"
+            "// %25 chunk byte offset for 4-byte elements; %26 column byte offset; %27 ragged-chunk flag;\n"
+            "// %28 byte distance (4-byte elements) to the thread's next chunk, 0 if there is none.\n"
             "#pragma once\n\n")
-    text += as_macro("LT_VM_CORE_FAST", build(True)) + "\n" + as_macro("LT_VM_CORE_PRECISE", build(False))
+    text += "\n".join(as_macro(f"LT_VM_CORE_{fl.upper()}", build(fl)) for fl in ("fast", "precise", "ieee"))
     (HERE / "vm_core.inc").write_text(text)
     print(f"wrote vm_core.inc ({len(text)} bytes)")
 

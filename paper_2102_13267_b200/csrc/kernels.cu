@@ -18,6 +18,10 @@ namespace {
 
 constexpr int V = LT_VM_V;
 
+#ifndef LT_EW_MIN_BLOCKS
+#define LT_EW_MIN_BLOCKS 3
+#endif
+
 struct Chunk {
     uint64_t flat0;  // flat index of lane 0
     uint32_t row;
@@ -36,8 +40,6 @@ struct RowCtx {
 // ---------------------------------------------------------------- environments
 struct EnvK {
     const LtKParams &P;
-    __device__ __forceinline__ LtIns ins(uint32_t pc) const { return P.ins[pc]; }
-    __device__ __forceinline__ uint32_t n_ins() const { return P.n_ins; }
     __device__ __forceinline__ uint32_t scal(uint32_t i) const { return P.scal[i]; }
     __device__ __forceinline__ uint64_t ptr(uint32_t s) const { return P.ptr[s]; }
     __device__ __forceinline__ uint32_t dtype(uint32_t s) const { return P.io_dtype[s]; }
@@ -47,8 +49,6 @@ struct EnvK {
 struct EnvM {
     const LtMultiParams &P;
     uint32_t base;  // instance * n_slots
-    __device__ __forceinline__ LtIns ins(uint32_t pc) const { return P.ins[pc]; }
-    __device__ __forceinline__ uint32_t n_ins() const { return P.n_ins; }
     __device__ __forceinline__ uint32_t scal(uint32_t i) const { return P.scal[i]; }
     __device__ __forceinline__ uint64_t ptr(uint32_t s) const { return P.ptr[base + s]; }
     __device__ __forceinline__ uint32_t dtype(uint32_t s) const { return P.io_dtype[s]; }
@@ -286,23 +286,6 @@ __device__ __forceinline__ void load_raw(float (&d)[V], const Env &E, uint32_t s
     }
 }
 
-__device__ __forceinline__ void widen(float (&d)[V], uint32_t dt) {
-    if (dt == LT_ST_BF16) {
-        uint32_t w0 = f2u(d[0]), w1 = f2u(d[1]), w2 = f2u(d[2]), w3 = f2u(d[3]);
-        d[0] = u2f(w0 << 16); d[1] = u2f(w0 & 0xffff0000u);
-        d[2] = u2f(w1 << 16); d[3] = u2f(w1 & 0xffff0000u);
-        d[4] = u2f(w2 << 16); d[5] = u2f(w2 & 0xffff0000u);
-        d[6] = u2f(w3 << 16); d[7] = u2f(w3 & 0xffff0000u);
-    } else if (dt == LT_ST_U8) {
-        uint32_t w0 = f2u(d[0]), w1 = f2u(d[1]);
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            d[b] = u2f((w0 >> (8 * b)) & 0xffu);
-            d[4 + b] = u2f((w1 >> (8 * b)) & 0xffu);
-        }
-    }
-}
-
 __device__ __noinline__ void store_chunk_slow(const float *a, char *p, uint32_t dt, int nvalid) {
     for (int i = 0; i < V; ++i) {
         if (i < nvalid) {
@@ -422,19 +405,15 @@ __device__ __forceinline__ void pairs_of(const float (&f)[V], uint64_t (&p)[4]) 
       "+l"(R[0][3]), "+l"(R[1][0]), "+l"(R[1][1]), "+l"(R[1][2]), "+l"(R[1][3]), "+l"(R[2][0]), "+l"(R[2][1]),      \
       "+l"(R[2][2]), "+l"(R[2][3]), "+l"(R[3][0]), "+l"(R[3][1]), "+l"(R[3][2]), "+l"(R[3][3]), "+r"(pc),           \
       "=r"(eop), "=r"(eimm)                                                                                         \
-    : "r"(scal_s), "r"(ptr_s), "l"(off4), "r"(coff4), "r"(tail)                                                     \
+    : "r"(scal_s), "r"(ptr_s), "l"(off4), "r"(coff4), "r"(tail), "l"(pf4)                                           \
     : "memory"
 
 // Runs the group's program on one chunk.  R[0..3] are T0..T3, R[4] is ACC.  The PTX core runs until an
 // opcode it does not implement (see gen_vm_core.py); that opcode is executed here and the core re-entered.
-template <bool FAST, bool ROW, class Env>
+template <int FLAV, bool ROW, class Env>
 __device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCtx *rc, uint32_t prog_s, uint32_t scal_s,
-                                            uint32_t ptr_s) {
-    uint64_t R[5][4];
-#pragma unroll
-    for (int k = 0; k < 5; ++k)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) R[k][j] = 0;
+                                            uint32_t ptr_s, uint64_t pf4) {
+    uint64_t R[5][4];  // not initialised: a program writes every register before it reads it
     uint32_t pc = prog_s;
     const uint64_t off4 = ck.flat0 << 2;
     const uint32_t coff4 = ck.col0 << 2;
@@ -442,8 +421,9 @@ __device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCt
 #pragma unroll 1
     for (;;) {
         uint32_t eop, eimm;
-        if constexpr (FAST) asm volatile(LT_VM_CORE_FAST LT_VM_OPERANDS);
-        else asm volatile(LT_VM_CORE_PRECISE LT_VM_OPERANDS);
+        if constexpr (FLAV == 0) asm volatile(LT_VM_CORE_FAST LT_VM_OPERANDS);
+        else if constexpr (FLAV == 1) asm volatile(LT_VM_CORE_PRECISE LT_VM_OPERANDS);
+        else asm volatile(LT_VM_CORE_IEEE LT_VM_OPERANDS);
         if (eop == OP_END) break;
         float f[V];
         if (eop >= OP_LD && eop < OP_STV) {  // generic load, or a vector load that met a ragged chunk / unaligned pointer
@@ -503,8 +483,8 @@ __device__ __forceinline__ void stage_program(Staged &S, const P &prm) {
 }
 
 // ------------------------------------------------------------------ kernels
-template <bool FAST>
-__global__ void __launch_bounds__(LT_EW_THREADS) lt_ew_kernel(const __grid_constant__ LtKParams P) {
+template <int FLAV>
+__global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(const __grid_constant__ LtKParams P) {
     __shared__ Staged S;
     const EnvK E{P};
     stage_program(S, P);
@@ -514,32 +494,37 @@ __global__ void __launch_bounds__(LT_EW_THREADS) lt_ew_kernel(const __grid_const
     const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
     const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
     const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; c < P.n_chunks; c += stride) {
+    const uint32_t stride = gridDim.x * blockDim.x;
+    const uint32_t n_chunks = (uint32_t)P.n_chunks;  // the planner keeps chunk counts below 2^32
+    // full-class slots of the next chunk a thread will run are prefetched into L2; sound when chunk c
+    // starts at element 8c: flat mode, or rows that are a multiple of the chunk
+    const bool linear = !P.rowcol || (P.cols % V) == 0;
+    const uint64_t pf_step = linear ? (uint64_t)stride * (V * 4) : 0;
+    for (uint32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < n_chunks; c += stride) {
         Chunk ck;
         ck.row_ok = true;
         if (!P.rowcol) {
-            ck.flat0 = c * V;
+            ck.flat0 = (uint64_t)c * V;
             ck.row = 0;
-            ck.col0 = (uint32_t)ck.flat0;
+            ck.col0 = c * V;
             const uint64_t rem = P.n - ck.flat0;
             ck.nvalid = rem < (uint64_t)V ? (int)rem : V;
         } else {
-            const uint32_t c32 = (uint32_t)c;
-            const uint32_t t = __umulhi(P.div_mul, c32);
-            const uint32_t row = (t + ((c32 - t) >> P.div_sh1)) >> P.div_sh2;
-            const uint32_t cc = c32 - row * P.cpr;
+            const uint32_t t = __umulhi(P.div_mul, c);
+            const uint32_t row = (t + ((c - t) >> P.div_sh1)) >> P.div_sh2;
+            const uint32_t cc = c - row * P.cpr;
             ck.row = row;
             ck.col0 = cc * V;
             ck.flat0 = (uint64_t)row * P.cols + ck.col0;
             const uint32_t rem = P.cols - ck.col0;
             ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
         }
-        run_program<FAST, false>(E, ck, nullptr, prog_s, scal_s, ptr_s);
+        const uint64_t pf4 = (n_chunks - c > stride && ck.nvalid == V) ? pf_step : 0;
+        run_program<FLAV, false>(E, ck, nullptr, prog_s, scal_s, ptr_s, pf4);
     }
 }
 
-template <bool FAST, int MAXT>
+template <int FLAV, int MAXT>
 __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ LtKParams P) {
     __shared__ Staged S;
     const EnvK E{P};
@@ -571,12 +556,14 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
             nv = rem < (uint32_t)V ? (int)rem : V;
         }
         ck.nvalid = nv;
-        run_program<FAST, true>(E, ck, &rc, prog_s, scal_s, ptr_s);
+        const uint64_t next_row = (uint64_t)ck.row + (uint64_t)gridDim.x * P.rows_per_cta;
+        const uint64_t pf4 = (next_row < P.rows && ck.nvalid == V) ? (uint64_t)gridDim.x * P.rows_per_cta * P.cols * 4 : 0;
+        run_program<FLAV, true>(E, ck, &rc, prog_s, scal_s, ptr_s, pf4);
     }
 }
 
-template <bool FAST>
-__global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
+template <int FLAV>
+__global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
     __shared__ Staged S;
     stage_program(S, P);
     const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
@@ -606,7 +593,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_co
                 ck.row_ok = true;
                 const uint32_t rem = numel - e0;
                 ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
-                run_program<FAST, false>(E, ck, nullptr, prog_s, scal_s, ptr_s);
+                run_program<FLAV, false>(E, ck, nullptr, prog_s, scal_s, ptr_s, 0);
             }
         }
     }
@@ -614,33 +601,37 @@ __global__ void __launch_bounds__(LT_EW_THREADS) lt_multi_kernel(const __grid_co
 
 }  // namespace
 
-cudaError_t lt_launch_ew(const LtKParams &p, bool fast, unsigned grid, cudaStream_t stream) {
-    if (fast) lt_ew_kernel<true><<<grid, LT_EW_THREADS, 0, stream>>>(p);
-    else lt_ew_kernel<false><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+cudaError_t lt_launch_ew(const LtKParams &p, int flavour, unsigned grid, cudaStream_t stream) {
+    if (flavour == 0) lt_ew_kernel<0><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    else if (flavour == 1) lt_ew_kernel<1><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    else lt_ew_kernel<2><<<grid, LT_EW_THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t lt_launch_row(const LtKParams &p, bool fast, unsigned grid, unsigned threads, cudaStream_t stream) {
+cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream) {
     if (threads <= 256) {
-        if (fast) lt_row_kernel<true, 256><<<grid, threads, 0, stream>>>(p);
-        else lt_row_kernel<false, 256><<<grid, threads, 0, stream>>>(p);
+        if (flavour == 0) lt_row_kernel<0, 256><<<grid, threads, 0, stream>>>(p);
+        else if (flavour == 1) lt_row_kernel<1, 256><<<grid, threads, 0, stream>>>(p);
+        else lt_row_kernel<2, 256><<<grid, threads, 0, stream>>>(p);
     } else {
-        if (fast) lt_row_kernel<true, 1024><<<grid, threads, 0, stream>>>(p);
-        else lt_row_kernel<false, 1024><<<grid, threads, 0, stream>>>(p);
+        if (flavour == 0) lt_row_kernel<0, 1024><<<grid, threads, 0, stream>>>(p);
+        else if (flavour == 1) lt_row_kernel<1, 1024><<<grid, threads, 0, stream>>>(p);
+        else lt_row_kernel<2, 1024><<<grid, threads, 0, stream>>>(p);
     }
     return cudaGetLastError();
 }
 
-cudaError_t lt_launch_multi(const LtMultiParams &p, bool fast, unsigned grid, cudaStream_t stream) {
-    if (fast) lt_multi_kernel<true><<<grid, LT_EW_THREADS, 0, stream>>>(p);
-    else lt_multi_kernel<false><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, cudaStream_t stream) {
+    if (flavour == 0) lt_multi_kernel<0><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    else if (flavour == 1) lt_multi_kernel<1><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    else lt_multi_kernel<2><<<grid, LT_EW_THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }
 
 cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_256, int *multi_blocks_per_sm) {
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(ew_blocks_per_sm, lt_ew_kernel<false>, LT_EW_THREADS, 0);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(ew_blocks_per_sm, lt_ew_kernel<1>, LT_EW_THREADS, 0);
     if (e != cudaSuccess) return e;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(row_blocks_per_sm_256, lt_row_kernel<false, 256>, 256, 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(row_blocks_per_sm_256, lt_row_kernel<1, 256>, 256, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(multi_blocks_per_sm, lt_multi_kernel<false>, LT_EW_THREADS, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(multi_blocks_per_sm, lt_multi_kernel<1>, LT_EW_THREADS, 0);
 }

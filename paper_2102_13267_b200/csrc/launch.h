@@ -1,4 +1,6 @@
 // Host-callable launch wrappers of the three kernels (defined in kernels.cu).
+// flavour: 0 fast (approximate transcendentals, for bf16 results), 1 precise (every op within 2 ulp),
+// 2 ieee (division, square root and reciprocal correctly rounded as well).
 #pragma once
 #include <cuda_runtime_api.h>
 
@@ -6,7 +8,7 @@
 
 
 
-cudaError_t lt_launch_ew(const LtKParams &p, bool fast, unsigned grid, cudaStream_t stream);
-cudaError_t lt_launch_row(const LtKParams &p, bool fast, unsigned grid, unsigned threads, cudaStream_t stream);
-cudaError_t lt_launch_multi(const LtMultiParams &p, bool fast, unsigned grid, cudaStream_t stream);
+cudaError_t lt_launch_ew(const LtKParams &p, int flavour, unsigned grid, cudaStream_t stream);
+cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream);
+cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, cudaStream_t stream);
 cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_256, int *multi_blocks_per_sm);

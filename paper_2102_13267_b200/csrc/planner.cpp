@@ -911,7 +911,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                         if (io.dtype == LT_F32) fast = false;
                         else if (io.dtype != LT_BF16 && cgen.tainted[io.cnode]) fast = false;
                     }
-                    g.fast = fast && any_store;
+                    g.flavour = (fast && any_store) ? 0 : (c->opt.ieee ? 2 : 1);
                 }
             }
             for (uint32_t n : emit) in_emit[n] = 0;
@@ -953,6 +953,8 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                 return fail(c, LT_ERR_UNSUPPORTED, "broadcast group too large for 32-bit chunk indexing");
         }
         if (g.kind == K_ROW && g.rows >= (1ull << 32)) return fail(c, LT_ERR_UNSUPPORTED, "too many rows");
+        if (g.kind == K_EW && !g.rowcol && (g.rows * g.cols + LT_VM_V - 1) / LT_VM_V >= (1ull << 32))
+            return fail(c, LT_ERR_UNSUPPORTED, "tensor too large for 32-bit chunk indexing");
     }
 
     // ---- outputs
@@ -990,7 +992,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                 }
                 if (!el) continue;
                 std::string s;
-                s.push_back(g.fast ? 'f' : 'p');
+                s.push_back((char)('0' + g.flavour));
                 s.append((const char *)g.ins.data(), g.ins.size() * sizeof(LtIns));
                 for (const Imm &im : g.imms) {
                     s.append((const char *)&im.dyn, sizeof(im.dyn));
@@ -1017,7 +1019,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                 while (pos < all.size()) {
                     Launch L;
                     L.kind = K_MULTI;
-                    L.fast = g.fast;
+                    L.flavour = g.flavour;
                     size_t cnt = std::min(per, all.size() - pos);
                     for (size_t k = 0; k < cnt; ++k) {
                         L.groups.push_back(all[pos + k]);
@@ -1030,7 +1032,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             } else {
                 Launch L;
                 L.kind = g.kind;
-                L.fast = g.fast;
+                L.flavour = g.flavour;
                 L.groups.push_back((uint32_t)gi);
                 L.bytes = g.bytes;
                 launch_of[gi] = (int)plan.launches.size();
@@ -1152,7 +1154,7 @@ std::string describe_plan(const Plan &plan) {
         const Launch &L = plan.launches[li];
         const Group &g = plan.groups[L.groups[0]];
         snprintf(buf, sizeof(buf), "launch %zu: %s %s instances=%zu rows=%llu cols=%llu %s bytes=%llu\n", li, kind[L.kind],
-                 L.fast ? "fast" : "precise", L.groups.size(), (unsigned long long)g.rows, (unsigned long long)g.cols,
+                 L.flavour == 0 ? "fast" : (L.flavour == 1 ? "precise" : "ieee"), L.groups.size(), (unsigned long long)g.rows, (unsigned long long)g.cols,
                  g.rowcol ? "rowcol" : "flat", (unsigned long long)L.bytes);
         s += buf;
         for (size_t q = 0; q < g.io.size(); ++q) {
