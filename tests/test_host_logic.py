@@ -1,0 +1,362 @@
+"""Host-side logic on a record-and-plan-only context (no GPU, no CUDA call): the C ABI's symbols,
+the IR recorder, canonical form and hash, compile cache, fusion planner and donation rules."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2102_13267_b200 as lt
+from workloads import configs, traces
+from workloads.resnet50 import parameter_shapes
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture()
+def ctx():
+    c = lt.LazyContext(device=None)
+    yield c
+    c.close()
+
+
+def fake(ctx, shape, dtype="f32", base=[1 << 30]):
+    """A device-data leaf over an address that is never dereferenced (nothing is launched)."""
+    base[0] += 1 << 28
+    return ctx.from_device_ptr(base[0], dtype, shape)
+
+
+# ------------------------------------------------------------------ C ABI surface
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "lazytensor.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(lt_[a-z_]+)\s*\(", header))
+    assert {"lt_tensor_from_device", "lt_op", "lt_barrier", "lt_fetch", "lt_assign"} <= declared
+    lib = ctypes.CDLL(str(lt.LIB_PATH))
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared in lazytensor.h but not exported"
+    assert set(lt.EXPORTED_SYMBOLS) == declared
+    assert lt.version().startswith("lazytensor")
+
+
+# ------------------------------------------------------------------ IR text (paper Fig. 1, 2)
+def test_ir_text_of_x_times_y_plus_z(ctx):
+    x, y, z = (fake(ctx, (2, 4)) for _ in range(3))
+    out = ctx.op("add", ctx.op("mul", x, y), z)
+    text = ctx.dump_ir()
+    lines = [ln.strip() for ln in text.splitlines()[1:-1]]
+    assert text.startswith("IR {") and text.rstrip().endswith("}")
+    assert len(lines) == 5
+    assert sum("lt::device_data()" in ln for ln in lines) == 3
+    assert all(ln.split(" = ")[1].startswith("f32[2,4]") for ln in lines)
+    assert lines[-1] == "%4 = f32[2,4] lt::add(%2, %3), ROOT=0"
+    assert lines[2] == "%2 = f32[2,4] lt::mul(%0, %1)"
+    assert sum("ROOT=" in ln for ln in lines) == 1
+    # the scaling constant 1 of Fig. 1 is a rank-0 constant whose value is part of the graph
+    scaled = ctx.op("add", ctx.op("mul", x, y), ctx.op("mul", z, ctx.scalar(1.0)))
+    del out
+    text = ctx.dump_ir()
+    assert "f32[] lt::constant(), value=1" in text
+
+
+def test_host_loop_unrolls_into_one_graph(ctx):
+    x, s = fake(ctx, (2, 4)), fake(ctx, (2, 4))
+    for _ in range(2):
+        s = ctx.op("add", s, x)
+    text = ctx.dump_ir()
+    assert text.count("lt::add(") == 2 and text.count("ROOT=") == 1
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1
+    assert ctx.dump_ir().count("lt::") == 0  # nothing pending after the barrier
+
+
+# ------------------------------------------------------------------ hash and cache (paper Section 4.1)
+def _flush(ctx, build):
+    before = ctx.stats()
+    keep = build()
+    ctx.barrier()
+    after = ctx.stats()
+    del keep
+    return after["compiles"] - before["compiles"], after["cache_hits"] - before["cache_hits"]
+
+
+def test_scalar_classes(ctx):
+    x = fake(ctx, (64, 64))
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(42.0))) == (1, 0)
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(43.0))) == (0, 1)   # another value: same entry
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(0.0))) == (1, 0)    # 0 is part of the graph
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(1.0))) == (1, 0)    # so is 1
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(2.0))) == (0, 1)
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(-0.0))) == (0, 1)   # -0.0 is not the special 0
+    assert _flush(ctx, lambda: ctx.op("add", x, ctx.scalar(1.0, dynamic=True))) == (0, 1)
+    assert ctx.cache_size() == 3
+
+
+def test_operand_identity_and_shape_enter_the_hash(ctx):
+    a, b = fake(ctx, (32, 32)), fake(ctx, (32, 32))
+    assert _flush(ctx, lambda: ctx.op("mul", a, b)) == (1, 0)
+    assert _flush(ctx, lambda: ctx.op("mul", a, a)) == (1, 0)      # a*a is not a*b
+    assert _flush(ctx, lambda: ctx.op("mul", b, a)) == (0, 1)      # other buffers, same program
+    c, d = fake(ctx, (32, 64)), fake(ctx, (32, 64))
+    assert _flush(ctx, lambda: ctx.op("mul", c, d)) == (1, 0)      # shape change recompiles
+    e, f = fake(ctx, (32, 32), "bf16"), fake(ctx, (32, 32), "bf16")
+    assert _flush(ctx, lambda: ctx.op("mul", e, f)) == (1, 0)      # dtype change recompiles
+    ctx.set_option("fusion", 0)
+    assert _flush(ctx, lambda: ctx.op("mul", a, b)) == (1, 0)      # options are part of the key
+
+
+def test_c1_traced_ten_times_compiles_once(ctx):
+    leaves = [fake(ctx, (1024, 1024)) for _ in range(4)]
+    for _ in range(10):
+        y = traces.elementwise_chain(ctx, *leaves)
+        ctx.barrier()
+    s = ctx.stats()
+    assert (s["compiles"], s["cache_hits"], s["kernels_launched"]) == (1, 9, 10)
+    assert s["bytes_planned"] == 10 * configs.algorithmic_bytes("c1")
+
+
+def test_c5_hundred_steps_one_compile(ctx):
+    shapes = parameter_shapes()
+    P, G, M, V = ([fake(ctx, s) for s in shapes] for _ in range(4))
+    for step in range(1, 101):
+        traces.adam_step(ctx, P, G, M, V, step=step)
+        ctx.barrier()
+    s = ctx.stats()
+    assert (s["compiles"], s["cache_hits"]) == (1, 99)
+    assert s["kernels_launched"] == 100 and s["launches_multi"] == 100
+    assert s["outputs_donated"] == 100 * 3 * 161 and s["outputs_allocated"] == 0
+    assert s["temporaries_allocated"] == 0
+    assert s["bytes_planned"] == 100 * configs.algorithmic_bytes("c5")
+    plan = ctx.dump_plan()
+    assert "launch 0: multi precise instances=161" in plan and "launch 1" not in plan
+
+
+def test_cache_capacity_evicts_least_recently_used(ctx):
+    ctx.set_option("cache_capacity", 2)
+    x = fake(ctx, (16, 16))
+    prog = {k: (lambda k=k: ctx.op(k, x, x)) for k in ("add", "sub", "max")}
+    assert _flush(ctx, prog["add"]) == (1, 0)
+    assert _flush(ctx, prog["sub"]) == (1, 0)
+    assert _flush(ctx, prog["add"]) == (0, 1)
+    assert _flush(ctx, prog["max"]) == (1, 0)   # evicts sub
+    assert _flush(ctx, prog["add"]) == (0, 1)
+    assert _flush(ctx, prog["sub"]) == (1, 0)
+    assert ctx.cache_size() == 2
+
+
+# ------------------------------------------------------------------ planner
+def test_each_config_is_one_fused_kernel(ctx):
+    x, h, b = fake(ctx, (8192, 4096), "bf16"), fake(ctx, (8192, 4096), "bf16"), fake(ctx, (4096,), "bf16")
+    out = traces.mlp_epilogue(ctx, x, h, b)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.startswith("plan: 1 launches, 1 groups") and "elementwise fast" in plan and "colvec" in plan
+    assert ctx.stats()["bytes_planned"] == configs.algorithmic_bytes("c2")
+    ctx.reset_stats()
+    shape = (16384, 1024)
+    z, keep = traces.residual_dropout_layernorm(ctx, fake(ctx, shape, "bf16"), fake(ctx, shape, "bf16"),
+                                                fake(ctx, (1024,)), fake(ctx, (1024,)), shape=shape, p=0.1,
+                                                eps=1e-5, seed=1, offset=2)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.startswith("plan: 1 launches, 1 groups") and "row fast" in plan
+    assert plan.count("row_sum") == 2 and "philox" in plan
+    assert ctx.stats()["bytes_planned"] == configs.algorithmic_bytes("c3")
+    ctx.reset_stats()
+    shape = (16, 2048, 2048)
+    y = traces.causal_softmax(ctx, fake(ctx, shape, "bf16"), shape=shape, scale=0.088)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.startswith("plan: 1 launches, 1 groups") and "row_max" in plan and "iota" in plan
+    assert ctx.stats()["bytes_planned"] == configs.algorithmic_bytes("c4")
+
+
+def test_f32_results_never_use_the_fast_flavour(ctx):
+    shape = (64, 256)
+    z, keep = traces.residual_dropout_layernorm(ctx, fake(ctx, shape, "bf16"), fake(ctx, shape, "bf16"),
+                                                fake(ctx, (256,)), fake(ctx, (256,)), shape=shape, p=0.1,
+                                                eps=1e-5, seed=1, offset=2, out_dtype="f32")
+    ctx.barrier()
+    assert "row precise" in ctx.dump_plan()
+    ctx.set_option("ieee", 1)
+    x = fake(ctx, (64, 64))
+    q = ctx.op("div", x, x)
+    ctx.barrier()
+    assert "elementwise ieee" in ctx.dump_plan()
+
+
+def test_unfused_mode_launches_one_kernel_per_op(ctx):
+    ctx.set_option("fusion", 0)
+    leaves = [fake(ctx, (256, 256)) for _ in range(4)]
+    y = traces.elementwise_chain(ctx, *leaves)
+    ctx.barrier()
+    s = ctx.stats()
+    assert s["kernels_launched"] == 5 and s["temporaries_allocated"] == 4
+
+
+def test_live_intermediate_becomes_an_output(ctx):
+    a, b = fake(ctx, (128, 128)), fake(ctx, (128, 128))
+    t = ctx.op("mul", a, b)
+    y = ctx.op("relu", t)
+    ctx.barrier()                       # t is still named: the barrier must materialise it too
+    assert ctx.stats()["outputs_allocated"] == 2 and ctx.is_materialised(t)
+    ctx.reset_stats()
+    t2 = ctx.op("mul", a, b)
+    y2 = ctx.op("relu", t2)
+    del t2
+    ctx.barrier()
+    assert ctx.stats()["outputs_allocated"] == 1
+
+
+def test_program_too_large_for_one_group_is_split(ctx):
+    xs = [fake(ctx, (64, 64)) for _ in range(9)]
+    acc = ctx.op("mul", xs[0], xs[1])
+    prods = [ctx.op("mul", xs[i], xs[i + 1]) for i in range(1, 8)]
+    # a wide tree: more simultaneously live values than the machine has registers
+    lvl = [acc] + prods
+    while len(lvl) > 1:
+        lvl = [ctx.op("add", lvl[i], lvl[i + 1]) for i in range(0, len(lvl) - 1, 2)] + (lvl[-1:] if len(lvl) % 2 else [])
+    out = lvl[0]
+    del acc, prods, lvl
+    ctx.barrier()
+    s = ctx.stats()
+    assert s["outputs_allocated"] == 1 and s["kernels_launched"] >= 1
+
+
+# ------------------------------------------------------------------ in-place updates (paper Section 4.3)
+def test_in_place_update_is_donated_once(ctx):
+    a = fake(ctx, (64, 64))
+    ptr = ctx.device_ptr(a)
+    a += 1.0
+    ctx.barrier()
+    s = ctx.stats()
+    assert (s["outputs_donated"], s["outputs_allocated"], s["kernels_launched"]) == (1, 0, 1)
+    assert ctx.device_ptr(a) == ptr
+    ctx.barrier()                        # observing a twice must not increment twice: nothing is pending
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1
+
+
+def test_second_reader_in_the_same_kernel_keeps_donation(ctx):
+    a = fake(ctx, (64, 64))
+    b = a + 2.0                          # must see the old a
+    a += 1.0
+    ctx.barrier()
+    s = ctx.stats()
+    assert s["kernels_launched"] == 1 and s["outputs_donated"] == 1 and s["outputs_allocated"] == 1
+    plan = ctx.dump_plan()
+    assert plan.index("vload p0") < plan.index("vstore")  # the old value is read before any store
+
+
+def test_no_donation_while_another_tensor_names_the_old_value(ctx):
+    a = fake(ctx, (64, 64))
+    alias = fake(ctx, (64, 64))
+    ctx.assign(alias, a)                 # alias now names a's buffer as well
+    a += 1.0
+    ctx.barrier()
+    s = ctx.stats()
+    assert s["outputs_donated"] == 0 and s["outputs_allocated"] == 1
+
+
+def test_no_donation_when_a_later_kernel_reads_the_old_value(ctx):
+    ctx.set_option("fusion", 0)          # one kernel per op: b's kernel runs after a's
+    a = fake(ctx, (64, 64))
+    new_a = a + 1.0
+    b = a * 3.0
+    ctx.assign(a, new_a)
+    del new_a
+    ctx.barrier()
+    s = ctx.stats()
+    assert s["kernels_launched"] == 2
+    # a's update is traced first, so its kernel precedes the one that still reads the old buffer
+    assert s["outputs_donated"] == 0 and s["outputs_allocated"] == 2
+
+
+def test_broadcast_reader_blocks_donation(ctx):
+    col = fake(ctx, (256,))
+    full = fake(ctx, (8, 256))
+    # the column vector is read by every row of the wide kernel: it cannot be overwritten in place there
+    wide = ctx.op("add", full, col)
+    newcol = ctx.op("mul", col, ctx.scalar(2.0))
+    ctx.assign(col, newcol)
+    del newcol
+    ctx.barrier()
+    assert ctx.stats()["outputs_donated"] in (0, 1)
+    plan = ctx.dump_plan()
+    if "donated" in plan:                # only legal when the in-place kernel runs after the wide one
+        assert plan.index("colvec") < plan.rindex("launch")
+
+
+# ------------------------------------------------------------------ errors
+def test_error_paths(ctx):
+    a, b = fake(ctx, (4, 8)), fake(ctx, (4, 7))
+    with pytest.raises(lt.LazyTensorError) as e:
+        ctx.op("add", a, b)
+    assert e.value.status == 2  # LT_ERR_SHAPE
+    with pytest.raises(lt.LazyTensorError) as e:
+        ctx.op("add", a, fake(ctx, (4, 8), "bf16"))
+    assert e.value.status == 3  # LT_ERR_DTYPE
+    with pytest.raises(lt.LazyTensorError) as e:
+        ctx.op("add", fake(ctx, (4, 8), "i32"), ctx.scalar(0.5))
+    assert e.value.status == 3
+    with pytest.raises(lt.LazyTensorError) as e:
+        ctx.op("row_sum", fake(ctx, (2, 8200)))
+    assert e.value.status == 5  # LT_ERR_UNSUPPORTED
+    with pytest.raises(lt.LazyTensorError) as e:
+        ctx.op("exp", fake(ctx, (4,), "i32"))
+    assert e.value.status == 3
+    other = lt.LazyContext(device=None)
+    foreign = other.from_device_ptr(1 << 40, "f32", (4, 8))
+    with pytest.raises(lt.LazyTensorError) as e:
+        ctx.op("add", a, foreign)
+    assert e.value.status == 4  # LT_ERR_DEVICE: no implicit cross-device operands
+    assert ctx.stats()["nodes_recorded"] == 7  # six leaves and one scalar: the failed ops recorded nothing
+    with pytest.raises(lt.LazyTensorError):
+        ctx.fetch(a)  # no device behind this context
+    with pytest.raises(lt.LazyTensorError):
+        ctx.set_option("no_such_option", 1)
+    other.close()
+
+
+def test_failed_allocation_leaves_the_graph_flushable():
+    lib = ctypes.CDLL(str(lt.LIB_PATH))
+    fail_next = {"on": True}
+    live = {}
+
+    def alloc(nbytes, stream, user):
+        if fail_next["on"]:
+            return None
+        buf = ctypes.create_string_buffer(max(int(nbytes), 16))
+        live[ctypes.addressof(buf)] = buf
+        return ctypes.addressof(buf)
+
+    def free(ptr, stream, user):
+        live.pop(ptr, None)
+
+    a_fn, f_fn = lt.ALLOC_FN(alloc), lt.FREE_FN(free)
+    st = lt.lt_allocator(a_fn, f_fn, None)
+    c = ctypes.c_void_p()
+    assert lib.lt_ctx_create(-1, None, ctypes.byref(st), ctypes.byref(c)) == 0
+    h = [ctypes.c_uint64() for _ in range(3)]
+    shape = (ctypes.c_int64 * 2)(4, 4)
+    lib.lt_tensor_from_device.argtypes = lt._SIGNATURES["lt_tensor_from_device"]
+    lib.lt_op.argtypes = lt._SIGNATURES["lt_op"]
+    lib.lt_barrier.argtypes = lt._SIGNATURES["lt_barrier"]
+    lib.lt_get_stats.argtypes = lt._SIGNATURES["lt_get_stats"]
+    lib.lt_last_error.restype = ctypes.c_char_p
+    lib.lt_last_error.argtypes = [ctypes.c_void_p]
+    for i in range(2):
+        assert lib.lt_tensor_from_device(c, ctypes.c_void_p(4096 * (i + 1)), 0, 2, shape, ctypes.byref(h[i])) == 0
+    ins = (ctypes.c_uint64 * 2)(h[0].value, h[1].value)
+    assert lib.lt_op(c, 1, ins, 2, None, 0, ctypes.byref(h[2])) == 0
+    assert lib.lt_barrier(c, 0) == 6  # LT_ERR_OOM
+    assert b"allocator" in lib.lt_last_error(c)
+    fail_next["on"] = False
+    assert lib.lt_barrier(c, 0) == 0  # the pending graph was left intact and flushes now
+    s = lt.lt_stats()
+    assert lib.lt_get_stats(c, ctypes.byref(s)) == 0
+    assert s.kernels_launched == 1 and s.outputs_allocated == 1
+    lib.lt_ctx_destroy.argtypes = [ctypes.c_void_p]
+    assert lib.lt_ctx_destroy(c) == 0
+    assert not live  # the output buffer went back through the free callback
