@@ -153,6 +153,8 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * 2 ulp; 1 = correctly rounded, so that a graph of + - * / sqrt matches an op-by-op binary32
  * evaluation bit for bit, at about ten more instructions per element and op),
  * "waves" (4 default: grid size of the persistent kernels in waves of resident thread blocks),
+ * "stage" (1 default: inputs are copied asynchronously into shared-memory staging buffers a few chunks
+ * ahead of their use; 0 = loads go straight to registers),
  * "horizontal" (1 default: bundle isomorphic independent groups into multi-tensor launches),
  * "cache_capacity" (0 = unbounded).  Options are part of the cache key.
  * Unknown key: LT_ERR_INVALID_ARG.  The environment variables LT_FUSION, LT_VERIFY,

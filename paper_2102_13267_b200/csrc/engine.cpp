@@ -295,6 +295,7 @@ lt_status lt_ctx_create(int device, void *cuda_stream, const lt_allocator *alloc
         cudaError_t e = cudaSetDevice(device);
         int sms = 0;
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (e == cudaSuccess) e = lt_kernel_setup(LT_MAX_STAGE_BYTES);
         if (e == cudaSuccess) e = lt_kernel_occupancy(&c->occ_ew, &c->occ_row, &c->occ_multi);
         if (e != cudaSuccess) {
             // no usable device: report instead of falling back to anything
@@ -335,6 +336,7 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "cache_capacity")) c->opt.cache_capacity = value;
     else if (!strcmp(key, "ieee")) c->opt.ieee = value;
     else if (!strcmp(key, "waves")) c->opt.waves = value;
+    else if (!strcmp(key, "stage")) c->opt.stage = value;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
 }

@@ -130,6 +130,31 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             for (size_t q = 0; q < g.imms.size(); ++q) P.scal[q] = encode_imm(g.imms[q], cg.dyn);
             for (size_t s = 0; s < g.io.size(); ++s) P.ptr[s] = resolve(g.io[s]);
             if (L.kind == K_EW) {
+                // Staging plan: aligned full-class inputs are copied asynchronously into per-thread
+                // shared-memory buffers a few chunks ahead (needs chunk c to start at element 8c).
+                const bool linear = !P.rowcol || (P.cols % LT_VM_V) == 0;
+                uint32_t pieces = 0;
+                for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                if (c->opt.stage && linear) {
+                    for (size_t s = 0; s < g.io.size(); ++s) {
+                        const IoRef &io = g.io[s];
+                        if (io.is_store || io.cls != LT_CLS_FULL) continue;
+                        const uint64_t need = io.dtype == LT_U8 ? 7u : 15u;
+                        if (P.ptr[s] & need) continue;
+                        P.io_stage[s] = (uint8_t)pieces;
+                        pieces += (io.dtype == LT_BF16 || io.dtype == LT_U8) ? 1u : 2u;
+                    }
+                }
+                P.stage_pieces = pieces;
+                P.stage_depth = 0;
+                if (pieces) {
+                    const uint32_t buf = pieces * LT_VM_STAGE_PIECE;
+                    uint32_t depth = (96u * 1024u + (uint32_t)c->occ_ew * buf - 1) / ((uint32_t)c->occ_ew * buf);
+                    depth = std::min(4u, std::max(2u, depth));
+                    while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
+                    if (depth >= 2) P.stage_depth = depth;
+                    else for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                }
                 if (!dry) {
                     uint64_t need = (P.n_chunks + LT_EW_THREADS - 1) / LT_EW_THREADS;
                     unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);

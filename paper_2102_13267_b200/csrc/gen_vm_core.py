@@ -53,7 +53,10 @@ NSRC = OPS["LT_VM_NSRC"]
 A = [f"%{i}" for i in range(4)]
 T = [[f"%{4 + 4 * k + j}" for j in range(4)] for k in range(4)]
 REG = T + [A]  # destination index 0..3 = temporaries, 4 = ACC
-PC, EOP, EIMM, SB, PB, OFF4, COFF4, TAIL, PF4 = "%20", "%21", "%22", "%23", "%24", "%25", "%26", "%27", "%28"
+PC, EOP, EIMM, CHUNK, OFF4, COFF4, TAIL, STG, SMB = "%20", "%21", "%22", "%23", "%24", "%25", "%26", "%27", "%28"
+PF4 = "pf4"
+SM_SCAL, SM_PTR, SM_SOFF, STAGE_PIECE, SM_LOOP, SM_STG = (OPS[k] for k in ("LT_VM_SM_SCAL", "LT_VM_SM_PTR", "LT_VM_SM_SOFF", "LT_VM_STAGE_PIECE", "LT_VM_SM_LOOP", "LT_VM_SM_STG"))
+SM_PF = SM_STG + 16 * OPS["LT_VM_MAX_PTR"]
 
 
 def f32_hex(x: float) -> int:
@@ -92,7 +95,7 @@ class Src:
             self.pairs = T[kind]
             self._lanes = None
         else:
-            self.pre = ["shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SB};", "ld.shared.b32 sv, [sa];", "mov.b64 ss, {sv, sv};"]
+            self.pre = ["shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b32 sv, [sa+{SM_SCAL}];", "mov.b64 ss, {sv, sv};"]
             self.pairs = ["ss"] * 4
 
     def lanes(self, out):
@@ -274,14 +277,24 @@ def cvt_u8(d: int):
 def slot_pointer():
     """ptr = pointer-table entry of slot `imm`; leaves for the slow path when the entry is flagged
     (bit 63: not vector-aligned) or the chunk is ragged."""
-    return ["shl.b32 sa, imm, 3;", f"add.u32 sa, sa, {PB};", "ld.shared.b64 ptr, [sa];", "setp.lt.s64 p, ptr, 0;",
+    return ["shl.b32 sa, imm, 3;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b64 ptr, [sa+{SM_PTR}];", "setp.lt.s64 p, ptr, 0;",
             "@p bra L_ESC;", "@ptail bra L_ESC;"]
 
 
-def ldv_body(sz: int, cls: int, d: int):
+def ldv_body(sz: int, cls: int, d: int, code: int):
     P = REG[d]
     lines = slot_pointer()
     if cls == 0:
+        # a slot staged by asynchronous copies is read from this thread's staging buffer instead
+        lines += ["shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b32 w0, [sa+{SM_SOFF}];",
+                  "setp.eq.s32 p, w0, -1;", f"@p bra L_G{code};", f"add.u32 w0, w0, {STG};"]
+        if sz == 0:
+            lines += ["ld.shared.v4.b32 {x0, x1, x2, x3}, [w0];", f"ld.shared.v4.b32 {{x4, x5, x6, x7}}, [w0+{STAGE_PIECE}];"] + pack(P, X)
+        elif sz == 1:
+            lines += ["ld.shared.v4.b32 {x0, x1, x2, x3}, [w0];", f"mov.b64 {P[0]}, {{x0, x1}};", f"mov.b64 {P[1]}, {{x2, x3}};"]
+        else:
+            lines += ["ld.shared.v2.b32 {x0, x1}, [w0];", f"mov.b64 {P[0]}, {{x0, x1}};"]
+        lines += ["@DISPATCH@", f"L_G{code}:"]
         lines.append(f"shr.u64 offs, {OFF4}, {sz};" if sz else f"mov.b64 offs, {OFF4};")
     else:
         lines += [f"cvt.u64.u32 offs, {COFF4};"] + ([f"shr.u64 offs, offs, {sz};"] if sz else [])
@@ -320,10 +333,71 @@ def stv_body(sz: int):
     return lines
 
 
+def entry_code():
+    """Predicates that depend on the current chunk; recomputed whenever the asm statement is (re-)entered."""
+    L = SM_LOOP
+    return [f"setp.ne.u32 ptail, {TAIL}, 0;",
+            f"ld.shared.v2.b32 {{r0, r1}}, [{SMB}+{L}];",            # stride, n_chunks
+            f"ld.shared.b32 r2, [{SMB}+{L + 56}];",                   # prefetch enabled
+            f"ld.shared.b64 pf4, [{SMB}+{SM_PF}];",
+            f"sub.u32 r1, r1, {CHUNK};", "setp.gt.u32 pnext, r1, r0;", "setp.ne.u32 p, r2, 0;",
+            "and.pred pnext, pnext, p;", "not.pred p, ptail;", "and.pred pnext, pnext, p;"]
+
+
+def end_body():
+    """OP_END.  When the core runs the chunk loop itself: refill the staging buffer just consumed, move to
+    the thread's next chunk, wait for its staged inputs and restart the program; else leave."""
+    L = SM_LOOP
+    return [
+        f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 16}];",     # buf_bytes, buf_total, stage_base, inloop
+        "setp.eq.u32 p, r7, 0;", "@p bra L_ESC;",
+        f"ld.shared.v4.b32 {{r0, r1, r2, r3}}, [{SMB}+{L}];",          # stride, n_chunks, n_full, depth
+        "setp.eq.u32 pq, r3, 0;", "@pq bra L_ADV;",
+        # chunk `depth` iterations ahead; staged only if it is complete
+        "mul.wide.u32 d0, r0, r3;", f"cvt.u64.u32 d1, {CHUNK};", "add.u64 d0, d0, d1;", "cvt.u64.u32 d1, r2;",
+        "setp.ge.u64 p, d0, d1;", "@p bra L_COMMIT;",
+        "shl.b64 d0, d0, 3;",                                            # first element of that chunk
+        f"ld.shared.b32 r7, [{SMB}+{L + 60}];",                         # number of staged inputs
+        f"add.u32 sa, {SMB}, {SM_STG};",
+        "L_STG_LOOP:",
+        "ld.shared.v4.b32 {x0, x1, x2, x3}, [sa];",                      # ptr lo, hi, dst offset, log2(bytes)
+        "mov.b64 ptr, {x0, x1};", "shl.b64 d1, d0, x3;", "add.u64 ptr, ptr, d1;", f"add.u32 x2, x2, {STG};",
+        "setp.eq.u32 p, x3, 0;", "@p cp.async.ca.shared.global [x2], [ptr], 8;",
+        "@!p cp.async.cg.shared.global [x2], [ptr], 16;",
+        "setp.eq.u32 p, x3, 2;", f"@p cp.async.cg.shared.global [x2+{STAGE_PIECE}], [ptr+16], 16;",
+        "add.u32 sa, sa, 16;", "sub.u32 r7, r7, 1;", "setp.ne.u32 p, r7, 0;", "@p bra L_STG_LOOP;",
+        "L_COMMIT:",
+        "cp.async.commit_group;",
+        # next staging buffer of this thread (a ring of `depth` buffers)
+        f"add.u32 {STG}, {STG}, r4;", "mov.u32 x0, %tid.x;", "shl.b32 x0, x0, 4;", "add.u32 x0, x0, r6;",
+        "add.u32 x0, x0, r5;", f"setp.ge.u32 p, {STG}, x0;", f"@p sub.u32 {STG}, {STG}, r5;",
+        # the copies of the next chunk are the oldest group still in flight
+        "setp.eq.u32 p, r3, 2;", "@p cp.async.wait_group 1;", "setp.eq.u32 p, r3, 3;", "@p cp.async.wait_group 2;",
+        "setp.eq.u32 p, r3, 4;", "@p cp.async.wait_group 3;",
+        "L_ADV:",
+        f"add.u32 {CHUNK}, {CHUNK}, r0;", f"setp.ge.u32 p, {CHUNK}, r1;", "@p bra L_ESC;",
+        f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 32}];",      # rowcol, cpr, div_mul, div_sh1
+        "setp.ne.u32 p, r4, 0;", "@p bra L_ROWCOL;",
+        f"mul.wide.u32 {OFF4}, {CHUNK}, 32;", f"cvt.u32.u64 {COFF4}, {OFF4};",
+        f"setp.ge.u32 ptail, {CHUNK}, r2;", "bra L_COORD_DONE;",
+        "L_ROWCOL:",
+        f"ld.shared.v2.b32 {{x2, x3}}, [{SMB}+{L + 48}];",               # div_sh2, cols
+        f"mul.hi.u32 x0, r6, {CHUNK};", f"sub.u32 x1, {CHUNK}, x0;", "shr.u32 x1, x1, r7;", "add.u32 x0, x0, x1;",
+        "shr.u32 x0, x0, x2;",                                           # row
+        f"mul.lo.u32 x1, x0, r5;", f"sub.u32 x1, {CHUNK}, x1;", "shl.b32 x1, x1, 3;",   # col0
+        "mul.wide.u32 d0, x0, x3;", "cvt.u64.u32 d1, x1;", "add.u64 d0, d0, d1;", f"shl.b64 {OFF4}, d0, 2;",
+        f"shl.b32 {COFF4}, x1, 2;", "sub.u32 x1, x3, x1;", "setp.lt.u32 ptail, x1, 8;",
+        "L_COORD_DONE:",
+        f"selp.b32 {TAIL}, 1, 0, ptail;",
+        f"mov.b32 {PC}, {SMB};",
+    ] + entry_code()[1:] + [f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];"]
+
+
 def build(flavour: str) -> list[str]:
     limit = OPS["OP_LIMIT"]
     bodies: dict[int, list[str]] = {}
 
+    bodies[OPS["OP_END"]] = end_body()
     for k in range(4):
         bodies[OPS["OP_MOV_T_ACC"] + k] = [f"mov.b64 {T[k][j]}, {A[j]};" for j in range(4)]
         bodies[OPS["OP_MOV_ACC_T"] + k] = [f"mov.b64 {A[j]}, {T[k][j]};" for j in range(4)]
@@ -342,7 +416,8 @@ def build(flavour: str) -> list[str]:
     for sz in range(3):
         for cls in range(2):
             for d in range(5):
-                bodies[OPS["OP_LDV"] + (sz * 2 + cls) * 5 + d] = ldv_body(sz, cls, d)
+                code = OPS["OP_LDV"] + (sz * 2 + cls) * 5 + d
+                bodies[code] = ldv_body(sz, cls, d, code)
         bodies[OPS["OP_STV"] + sz] = stv_body(sz)
     for idx in range(OPS["F2_COUNT"]):
         for k in range(NSRC):
@@ -359,24 +434,28 @@ def build(flavour: str) -> list[str]:
             bodies[OPS["OP_WHERE_B"] + m * NSRC + k] = where_body(m, Src(k), True)
 
     out = ["{"]
-    out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3;")
+    out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3, r0, r1, r2, r3, r4, r5, r6, r7;")
     out.append(".reg .b32 " + ", ".join(X + ["y0", "y1", "m0", "m1"]) + ";")
-    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2;")
-    out.append(".reg .pred p, ptail, pnext;")
+    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2, d0, d1, pf4;")
+    out.append(".reg .pred p, pq, ptail, pnext;")
     table = ", ".join(f"L_{i}" if i in bodies else "L_ESC" for i in range(limit))
     out.append(f"TBL: .branchtargets {table};")
-    out.append(f"setp.ne.u32 ptail, {TAIL}, 0;")
-    out.append(f"setp.ne.u64 pnext, {PF4}, 0;")
+    out += entry_code()
     out.append(f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];")
-    # fetch/decode/jump; repeated at the end of every body so a body falls straight into the next jump.
-    # The next instruction word is fetched one step ahead (the slot after the last instruction is padding).
+    # fetch/decode/jump.  The next instruction word is fetched one step ahead (the slot after the last
+    # instruction is padding).
     dispatch = ["mov.b32 op, nop;", "mov.b32 imm, nimm;", f"add.u32 {PC}, {PC}, 8;",
                 f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];", "brx.idx op, TBL;"]
+    # One shared copy: replicating the indexed branch after every body saves a jump per instruction but
+    # gives ptxas ~300 indirect branches x 328 targets to analyse, and compile time goes from seconds
+    # to tens of minutes.
+    out.append("L_DISPATCH:")
     out += dispatch
     for code in sorted(bodies):
         out.append(f"L_{code}:")
-        out += bodies[code]
-        out += dispatch
+        for ln in bodies[code]:
+            out.append("bra.uni L_DISPATCH;" if ln == "@DISPATCH@" else ln)
+        out.append("bra.uni L_DISPATCH;")
     out.append("L_ESC:")
     out.append(f"mov.b32 {EOP}, op;")
     out.append(f"mov.b32 {EIMM}, imm;")
@@ -392,9 +471,10 @@ def as_macro(name: str, lines: list[str]) -> str:
 def main() -> None:
     text = ("// Generated by gen_vm_core.py from vm.h -- do not edit.\n"
             "// Operands: %0-%3 ACC, %4-%19 T0..T3 (f32x2 pairs); %20 pc (shared address); %21 escape opcode;\n"
-            "// %22 escape immediate; %23 immediates base; %24 pointer table base (shared addresses);\n"
-            "// %25 chunk byte offset for 4-byte elements; %26 column byte offset; %27 ragged-chunk flag;\n"
-            "// %28 byte distance (4-byte elements) to the thread's next chunk, 0 if there is none.\n"
+            "// %22 escape immediate; %23 chunk index; %24 chunk byte offset for 4-byte elements; %25 column byte\n"
+            "// offset; %26 ragged-chunk flag; %27 shared address of this thread's current staging buffer;\n"
+            "// %28 shared address of the staged block (program, immediates, pointers, loop constants).\n"
+            "// %23-%27 are updated by the core when it moves to the next chunk by itself (OP_END).\n"
             "#pragma once\n\n")
     text += "\n".join(as_macro(f"LT_VM_CORE_{fl.upper()}", build(fl)) for fl in ("fast", "precise", "ieee"))
     (HERE / "vm_core.inc").write_text(text)

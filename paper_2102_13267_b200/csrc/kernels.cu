@@ -10,6 +10,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstddef>
+
 #include "launch.h"
 #include "vm.h"
 #include "vm_core.inc"
@@ -378,8 +380,15 @@ struct Staged {
     LtIns ins[LT_VM_MAX_INS + 2];
     uint32_t scal[LT_VM_MAX_SCAL];
     uint64_t ptr[LT_VM_MAX_PTR];
+    uint32_t soff[LT_VM_MAX_PTR];  // byte offset of the slot inside a staging buffer, 0xFFFFFFFF = not staged
+    LtLoop loop;
     float red[64];
 };
+static_assert(offsetof(Staged, scal) == LT_VM_SM_SCAL && offsetof(Staged, ptr) == LT_VM_SM_PTR &&
+                  offsetof(Staged, soff) == LT_VM_SM_SOFF && offsetof(Staged, loop) == LT_VM_SM_LOOP &&
+                  offsetof(Staged, loop.stg) == LT_VM_SM_STG &&
+                  offsetof(Staged, loop.pf_lo) == LT_VM_SM_STG + 16 * LT_VM_MAX_PTR,
+              "the PTX core addresses these fields by constant offset");
 
 // Pointer-table entry for the PTX core: bit 63 marks a slot whose chunks cannot use 128-bit accesses.
 __device__ __forceinline__ uint64_t flag_pointer(uint64_t p, uint32_t dt, bool rows_aligned) {
@@ -405,19 +414,22 @@ __device__ __forceinline__ void pairs_of(const float (&f)[V], uint64_t (&p)[4]) 
       "+l"(R[0][3]), "+l"(R[1][0]), "+l"(R[1][1]), "+l"(R[1][2]), "+l"(R[1][3]), "+l"(R[2][0]), "+l"(R[2][1]),      \
       "+l"(R[2][2]), "+l"(R[2][3]), "+l"(R[3][0]), "+l"(R[3][1]), "+l"(R[3][2]), "+l"(R[3][3]), "+r"(pc),           \
       "=r"(eop), "=r"(eimm)                                                                                         \
-    : "r"(scal_s), "r"(ptr_s), "l"(off4), "r"(coff4), "r"(tail), "l"(pf4)                                           \
+      , "+r"(c), "+l"(off4), "+r"(coff4), "+r"(tail), "+r"(stg)                                                     \
+    : "r"(smem_s)                                                                                                   \
     : "memory"
 
-// Runs the group's program on one chunk.  R[0..3] are T0..T3, R[4] is ACC.  The PTX core runs until an
-// opcode it does not implement (see gen_vm_core.py); that opcode is executed here and the core re-entered.
-template <int FLAV, bool ROW, class Env>
-__device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCtx *rc, uint32_t prog_s, uint32_t scal_s,
-                                            uint32_t ptr_s, uint64_t pf4) {
+// Runs the group's program.  R[0..3] are T0..T3, R[4] is ACC.  The PTX core runs until an opcode it does
+// not implement (see gen_vm_core.py); that opcode is executed here and the core re-entered.  With
+// LtLoop::inloop set the core also walks the thread's chunks by itself and `chunk_of(c)` rebuilds the
+// coordinates of chunk c for the code here; otherwise the call covers the one chunk given.
+template <int FLAV, bool ROW, class Env, class ChunkOf>
+__device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint32_t c, const Chunk &first, RowCtx *rc,
+                                            uint32_t smem_s, uint32_t stg) {
     uint64_t R[5][4];  // not initialised: a program writes every register before it reads it
-    uint32_t pc = prog_s;
-    const uint64_t off4 = ck.flat0 << 2;
-    const uint32_t coff4 = ck.col0 << 2;
-    const uint32_t tail = ck.nvalid != V ? 1u : 0u;
+    uint32_t pc = smem_s;
+    uint64_t off4 = first.flat0 << 2;
+    uint32_t coff4 = first.col0 << 2;
+    uint32_t tail = first.nvalid != V ? 1u : 0u;
 #pragma unroll 1
     for (;;) {
         uint32_t eop, eimm;
@@ -425,6 +437,7 @@ __device__ __forceinline__ void run_program(const Env &E, const Chunk &ck, RowCt
         else if constexpr (FLAV == 1) asm volatile(LT_VM_CORE_PRECISE LT_VM_OPERANDS);
         else asm volatile(LT_VM_CORE_IEEE LT_VM_OPERANDS);
         if (eop == OP_END) break;
+        const Chunk ck = chunk_of(c);
         float f[V];
         if (eop >= OP_LD && eop < OP_STV) {  // generic load, or a vector load that met a ragged chunk / unaligned pointer
             const uint32_t d = eop < OP_LDV ? eop - OP_LD : (eop - OP_LDV) % 5u;
@@ -480,61 +493,151 @@ __device__ __forceinline__ void stage_program(Staged &S, const P &prm) {
         S.ins[i] = in;
     }
     for (uint32_t i = threadIdx.x; i < LT_VM_MAX_SCAL; i += blockDim.x) S.scal[i] = prm.scal[i];
+    if (threadIdx.x < LT_VM_MAX_PTR) S.soff[threadIdx.x] = 0xffffffffu;
+    if (threadIdx.x < sizeof(LtLoop) / 4) reinterpret_cast<uint32_t *>(&S.loop)[threadIdx.x] = 0;
+}
+
+// Asynchronous 16-byte (or 8-byte) copy global -> shared; completion is tracked per thread in groups.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait(uint32_t pending) {  // at most `pending` newest groups still in flight
+    if (pending == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");
+    else if (pending == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else if (pending == 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+    else asm volatile("cp.async.wait_group 3;" ::: "memory");
+}
+
+// Starts the copies of one future chunk (first element e0) of every staged input into staging buffer `buf`.
+__device__ __forceinline__ void stage_chunk(const LtLoop &lp, uint64_t e0, uint32_t buf) {
+#pragma unroll 1
+    for (uint32_t k = 0; k < lp.stg_n; ++k) {
+        const uint32_t sh = lp.stg[k].shift;
+        const char *src = reinterpret_cast<const char *>(((uint64_t)lp.stg[k].ptr_hi << 32) | lp.stg[k].ptr_lo) + (e0 << sh);
+        const uint32_t dst = buf + lp.stg[k].dst;
+        if (sh == 0) cp_async8(dst, src);
+        else {
+            cp_async16(dst, src);
+            if (sh == 2) cp_async16(dst + LT_VM_STAGE_PIECE, src + 16);
+        }
+    }
+}
+
+__device__ __forceinline__ Chunk ew_chunk(const LtKParams &P, uint32_t c) {
+    Chunk ck;
+    ck.row_ok = true;
+    if (!P.rowcol) {
+        ck.flat0 = (uint64_t)c * V;
+        ck.row = 0;
+        ck.col0 = c * V;
+        const uint64_t rem = P.n - ck.flat0;
+        ck.nvalid = rem < (uint64_t)V ? (int)rem : V;
+    } else {
+        const uint32_t t = __umulhi(P.div_mul, c);
+        const uint32_t row = (t + ((c - t) >> P.div_sh1)) >> P.div_sh2;
+        const uint32_t cc = c - row * P.cpr;
+        ck.row = row;
+        ck.col0 = cc * V;
+        ck.flat0 = (uint64_t)row * P.cols + ck.col0;
+        const uint32_t rem = P.cols - ck.col0;
+        ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
+    }
+    return ck;
 }
 
 // ------------------------------------------------------------------ kernels
 template <int FLAV>
 __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(const __grid_constant__ LtKParams P) {
-    __shared__ Staged S;
+    __shared__ __align__(16) Staged S;
+    extern __shared__ __align__(16) unsigned char stage_mem[];
     const EnvK E{P};
     stage_program(S, P);
-    if (threadIdx.x < LT_VM_MAX_PTR)
-        S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], !P.rowcol || (P.cols % V) == 0);
     __syncthreads();
-    const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
-    const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
-    const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
+    const bool linear = !P.rowcol || (P.cols % V) == 0;  // chunk c starts at element 8c
     const uint32_t stride = gridDim.x * blockDim.x;
-    const uint32_t n_chunks = (uint32_t)P.n_chunks;  // the planner keeps chunk counts below 2^32
-    // full-class slots of the next chunk a thread will run are prefetched into L2; sound when chunk c
-    // starts at element 8c: flat mode, or rows that are a multiple of the chunk
-    const bool linear = !P.rowcol || (P.cols % V) == 0;
-    const uint64_t pf_step = linear ? (uint64_t)stride * (V * 4) : 0;
-    for (uint32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < n_chunks; c += stride) {
-        Chunk ck;
-        ck.row_ok = true;
-        if (!P.rowcol) {
-            ck.flat0 = (uint64_t)c * V;
-            ck.row = 0;
-            ck.col0 = c * V;
-            const uint64_t rem = P.n - ck.flat0;
-            ck.nvalid = rem < (uint64_t)V ? (int)rem : V;
-        } else {
-            const uint32_t t = __umulhi(P.div_mul, c);
-            const uint32_t row = (t + ((c - t) >> P.div_sh1)) >> P.div_sh2;
-            const uint32_t cc = c - row * P.cpr;
-            ck.row = row;
-            ck.col0 = cc * V;
-            ck.flat0 = (uint64_t)row * P.cols + ck.col0;
-            const uint32_t rem = P.cols - ck.col0;
-            ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
-        }
-        const uint64_t pf4 = (n_chunks - c > stride && ck.nvalid == V) ? pf_step : 0;
-        run_program<FLAV, false>(E, ck, nullptr, prog_s, scal_s, ptr_s, pf4);
+    const uint32_t n_chunks = (uint32_t)P.n_chunks;      // the planner keeps chunk counts below 2^32 - stride
+    const uint32_t depth = P.stage_depth;
+    const uint32_t buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
+    const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage_mem);
+    if (threadIdx.x < LT_VM_MAX_PTR) {
+        S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], linear);
+        if (depth && P.io_stage[threadIdx.x] != 0xffu) S.soff[threadIdx.x] = P.io_stage[threadIdx.x] * LT_VM_STAGE_PIECE;
     }
+    if (threadIdx.x == 0) {
+        LtLoop &lp = S.loop;
+        lp.stride = stride;
+        lp.n_chunks = n_chunks;
+        lp.n_full = linear ? (uint32_t)(P.n / V) : 0;  // chunks below this index are complete
+        lp.depth = depth;
+        lp.buf_bytes = buf_bytes;
+        lp.buf_total = depth * buf_bytes;
+        lp.stage_base = stage_base;
+        lp.inloop = 1;
+        lp.rowcol = P.rowcol;
+        lp.cpr = P.cpr;
+        lp.div_mul = P.div_mul;
+        lp.div_sh1 = P.div_sh1;
+        lp.div_sh2 = P.div_sh2;
+        lp.cols = P.cols;
+        lp.prefetch = (linear && !depth) ? 1u : 0u;  // without staging, pull the next chunk into L2 instead
+        const uint64_t pf = (uint64_t)stride * (V * 4);
+        lp.pf_lo = (uint32_t)pf;
+        lp.pf_hi = (uint32_t)(pf >> 32);
+        uint32_t k = 0;
+        if (depth)
+            for (uint32_t s = 0; s < LT_VM_MAX_PTR; ++s)
+                if (P.io_stage[s] != 0xffu) {
+                    lp.stg[k].ptr_lo = (uint32_t)P.ptr[s];
+                    lp.stg[k].ptr_hi = (uint32_t)(P.ptr[s] >> 32);
+                    lp.stg[k].dst = P.io_stage[s] * LT_VM_STAGE_PIECE;
+                    lp.stg[k].shift = 2u - (P.io_dtype[s] == LT_ST_BF16 ? 1u : P.io_dtype[s] == LT_ST_U8 ? 2u : 0u);
+                    ++k;
+                }
+        lp.stg_n = k;
+    }
+    __syncthreads();
+    const uint32_t c0 = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c0 >= n_chunks) return;
+    // Software pipeline: the full-class inputs of the thread's next `depth` chunks are in flight as
+    // asynchronous copies into per-thread staging buffers while the current chunk is interpreted.
+    const uint32_t buf0 = stage_base + threadIdx.x * 16u;
+    if (depth) {
+        uint64_t c = c0;
+        for (uint32_t d = 0; d < depth; ++d) {
+            if (c < S.loop.n_full) stage_chunk(S.loop, c * V, buf0 + d * buf_bytes);
+            cp_async_commit();
+            c += stride;
+        }
+        cp_async_wait(depth - 1);
+    }
+    run_program<FLAV, false>(E, [&P](uint32_t c) { return ew_chunk(P, c); }, c0, ew_chunk(P, c0), nullptr,
+                             (uint32_t)__cvta_generic_to_shared(&S), buf0);
+    if (depth) cp_async_wait(0);
 }
 
 template <int FLAV, int MAXT>
 __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ LtKParams P) {
-    __shared__ Staged S;
+    __shared__ __align__(16) Staged S;
     const EnvK E{P};
     stage_program(S, P);
+    __syncthreads();
+    const uint32_t row_blocks = (P.rows + P.rows_per_cta - 1u) / P.rows_per_cta;
     if (threadIdx.x < LT_VM_MAX_PTR)
         S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], (P.cols % V) == 0);
+    if (threadIdx.x == 0) {  // the core only needs these to prefetch the next block of rows into L2
+        S.loop.stride = gridDim.x;
+        S.loop.n_chunks = row_blocks;
+        S.loop.prefetch = 1;
+        const uint64_t pf = (uint64_t)gridDim.x * P.rows_per_cta * P.cols * 4;
+        S.loop.pf_lo = (uint32_t)pf;
+        S.loop.pf_hi = (uint32_t)(pf >> 32);
+    }
     __syncthreads();
-    const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
-    const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
-    const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
     RowCtx rc;
     rc.smem = S.red;
     rc.phase = 0;
@@ -543,7 +646,6 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
     rc.lane = threadIdx.x & 31u;
     const uint32_t sub = threadIdx.x >> P.group_log2;           // which row of this CTA's block of rows
     const uint32_t gl = threadIdx.x & (P.group - 1u);           // lane within the row's thread group
-    const uint32_t row_blocks = (P.rows + P.rows_per_cta - 1u) / P.rows_per_cta;
     for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
         Chunk ck;
         ck.row = rb * P.rows_per_cta + sub;
@@ -556,19 +658,15 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
             nv = rem < (uint32_t)V ? (int)rem : V;
         }
         ck.nvalid = nv;
-        const uint64_t next_row = (uint64_t)ck.row + (uint64_t)gridDim.x * P.rows_per_cta;
-        const uint64_t pf4 = (next_row < P.rows && ck.nvalid == V) ? (uint64_t)gridDim.x * P.rows_per_cta * P.cols * 4 : 0;
-        run_program<FLAV, true>(E, ck, &rc, prog_s, scal_s, ptr_s, pf4);
+        run_program<FLAV, true>(E, [&ck](uint32_t) { return ck; }, rb, ck, &rc, smem_s, 0);
     }
 }
 
 template <int FLAV>
 __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
-    __shared__ Staged S;
+    __shared__ __align__(16) Staged S;
     stage_program(S, P);
-    const uint32_t prog_s = (uint32_t)__cvta_generic_to_shared(S.ins);
-    const uint32_t scal_s = (uint32_t)__cvta_generic_to_shared(S.scal);
-    const uint32_t ptr_s = (uint32_t)__cvta_generic_to_shared(S.ptr);
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
     for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
         // instance that owns super-chunk sc: last i with super_prefix[i] <= sc
         uint32_t lo = 0, hi = P.n_inst;
@@ -593,7 +691,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
                 ck.row_ok = true;
                 const uint32_t rem = numel - e0;
                 ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
-                run_program<FLAV, false>(E, ck, nullptr, prog_s, scal_s, ptr_s, 0);
+                run_program<FLAV, false>(E, [&ck](uint32_t) { return ck; }, 0, ck, nullptr, smem_s, 0);
             }
         }
     }
@@ -602,10 +700,18 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
 }  // namespace
 
 cudaError_t lt_launch_ew(const LtKParams &p, int flavour, unsigned grid, cudaStream_t stream) {
-    if (flavour == 0) lt_ew_kernel<0><<<grid, LT_EW_THREADS, 0, stream>>>(p);
-    else if (flavour == 1) lt_ew_kernel<1><<<grid, LT_EW_THREADS, 0, stream>>>(p);
-    else lt_ew_kernel<2><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    const size_t dyn = (size_t)p.stage_depth * p.stage_pieces * LT_VM_STAGE_PIECE;
+    if (flavour == 0) lt_ew_kernel<0><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
+    else if (flavour == 1) lt_ew_kernel<1><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
+    else lt_ew_kernel<2><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
     return cudaGetLastError();
+}
+
+cudaError_t lt_kernel_setup(size_t max_stage_bytes) {
+    cudaError_t e = cudaFuncSetAttribute(lt_ew_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_ew_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_ew_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    return e;
 }
 
 cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream) {

@@ -3,6 +3,7 @@
 // 2 ieee (division, square root and reciprocal correctly rounded as well).
 #pragma once
 #include <cuda_runtime_api.h>
+#include <stddef.h>
 
 #include "vm.h"
 
@@ -11,4 +12,8 @@
 cudaError_t lt_launch_ew(const LtKParams &p, int flavour, unsigned grid, cudaStream_t stream);
 cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream);
 cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, cudaStream_t stream);
+#define LT_MAX_STAGE_BYTES (64u * 1024u)  // staging buffers per thread block
+
+// once per device: allow up to `max_stage_bytes` of dynamic shared memory for the staging buffers
+cudaError_t lt_kernel_setup(size_t max_stage_bytes);
 cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_256, int *multi_blocks_per_sm);

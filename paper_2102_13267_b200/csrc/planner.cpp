@@ -949,11 +949,11 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             return fail(c, LT_ERR_UNSUPPORTED, "row-reduction groups support rows of at most 8192 elements");
         if (g.kind == K_EW && g.rowcol) {
             uint64_t cpr = (g.cols + LT_VM_V - 1) / LT_VM_V;
-            if (g.rows * cpr >= (1ull << 32) || g.rows >= (1ull << 32) || g.cols >= (1ull << 32))
+            if (g.rows * cpr >= (1ull << 31) || g.rows >= (1ull << 31) || g.cols >= (1ull << 31))
                 return fail(c, LT_ERR_UNSUPPORTED, "broadcast group too large for 32-bit chunk indexing");
         }
         if (g.kind == K_ROW && g.rows >= (1ull << 32)) return fail(c, LT_ERR_UNSUPPORTED, "too many rows");
-        if (g.kind == K_EW && !g.rowcol && (g.rows * g.cols + LT_VM_V - 1) / LT_VM_V >= (1ull << 32))
+        if (g.kind == K_EW && !g.rowcol && (g.rows * g.cols + LT_VM_V - 1) / LT_VM_V >= (1ull << 31))
             return fail(c, LT_ERR_UNSUPPORTED, "tensor too large for 32-bit chunk indexing");
     }
 

@@ -18,6 +18,13 @@
 #define LT_VM_MAX_INS 118     // the program is followed by an END and one padding slot
 #define LT_VM_MAX_PTR 12
 #define LT_VM_MAX_SCAL 32
+// byte offsets inside the per-CTA shared-memory block the PTX core reads (struct Staged in kernels.cu)
+#define LT_VM_SM_SCAL 960   // immediates, after (LT_VM_MAX_INS + 2) instruction words
+#define LT_VM_SM_PTR 1088   // pointer table
+#define LT_VM_SM_SOFF 1184  // per-slot offset inside a staging buffer, or 0xFFFFFFFF
+#define LT_VM_SM_LOOP 1232  // struct LtLoop: constants of the chunk loop the PTX core runs by itself
+#define LT_VM_SM_STG 1296   // LtLoop::stg, the list of inputs staged by asynchronous copies
+#define LT_VM_STAGE_PIECE 4096  // bytes one 16-byte piece of a staged input takes per stage (256 threads x 16)
 
 #define LT_MULTI_MAX_INS 64
 #define LT_MULTI_MAX_INST 384   // instances (tensors) per multi-tensor launch
@@ -79,6 +86,18 @@ static_assert(OP_I2 + I2_COUNT * LT_VM_NSRC <= OP_CMP, "opcode map");
 static_assert(OP_CMP + 18 * LT_VM_NSRC <= OP_WHERE_A, "opcode map");
 static_assert(OP_WHERE_B + 4 * LT_VM_NSRC == OP_LIMIT, "opcode map");
 
+// Per-CTA constants of the chunk loop, in shared memory (read by the PTX core with broadcast loads).
+struct LtLoop {
+    uint32_t stride, n_chunks, n_full, depth;            // chunks between a thread's iterations; total; complete ones; staging depth
+    uint32_t buf_bytes, buf_total, stage_base, inloop;   // one staging buffer; all of them; shared address of the first; 1 = core loops by itself
+    uint32_t rowcol, cpr, div_mul, div_sh1;
+    uint32_t div_sh2, cols, prefetch, stg_n;             // prefetch: 1 = L2-prefetch the next chunk of full-class loads
+    struct {
+        uint32_t ptr_lo, ptr_hi, dst, shift;             // source pointer, offset inside a staging buffer, log2(element bytes)
+    } stg[LT_VM_MAX_PTR];
+    uint32_t pf_lo, pf_hi;                               // byte distance (4-byte elements) between a thread's iterations
+};
+
 // Kernel parameter block of the elementwise and row-reduction kernels.  It is passed by
 // value as a __grid_constant__ kernel parameter, so program, pointers and immediates are
 // read from the constant bank with no separate upload.
@@ -88,6 +107,9 @@ struct LtKParams {
     LtIns ins[LT_VM_MAX_INS];
     uint8_t io_dtype[LT_VM_MAX_PTR];
     uint8_t io_class[LT_VM_MAX_PTR];
+    uint8_t io_stage[LT_VM_MAX_PTR];  // first 16-byte piece of the slot in a staging buffer, 0xFF = not staged
+    uint32_t stage_depth;   // staging buffers per thread (0 = loads go straight to registers)
+    uint32_t stage_pieces;  // 16-byte pieces per staging buffer
     uint32_t n_ins;
     uint32_t rowcol;        // 0: flat chunks over n elements; 1: chunks stay inside rows
     uint64_t n;             // rows * cols
