@@ -7,10 +7,12 @@ branch (`brx.idx`) through a table with one entry per opcode, and the twenty 64-
 the asm statement are the machine state: ACC and T0..T3, eight f32 lanes each, held as four
 register pairs so that add/sub/mul/fma run as packed `.f32x2` instructions.
 
-The core executes register-to-register opcodes and the aligned full-chunk loads and stores
-itself.  Everything else (ragged or unaligned chunks, broadcast loads, reductions, random
-bits, correctly rounded transcendentals) leaves the asm statement with the opcode in an output
-operand ("escape") and is handled by the surrounding C++.
+The core executes register-to-register opcodes, the aligned full-chunk loads and stores (from
+global memory or from the thread's staging buffer) and, for the elementwise kernel, the loop over
+the thread's chunks with its asynchronous staging copies.  Everything else (ragged or unaligned
+chunks, broadcast loads, reductions, random bits, correctly rounded transcendentals) leaves the
+asm statement with the opcode in an output operand ("escape") and is handled by the surrounding
+C++.
 
 Run `python gen_vm_core.py` after changing vm.h's opcode map; the output is committed.
 """
@@ -274,50 +276,76 @@ def cvt_u8(d: int):
     return lines + pack(P, X)
 
 
-def slot_pointer():
-    """ptr = pointer-table entry of slot `imm`; leaves for the slow path when the entry is flagged
-    (bit 63: not vector-aligned) or the chunk is ragged."""
-    return ["shl.b32 sa, imm, 3;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b64 ptr, [sa+{SM_PTR}];", "setp.lt.s64 p, ptr, 0;",
-            "@p bra L_ESC;", "@ptail bra L_ESC;"]
-
-
-def ldv_body(sz: int, cls: int, d: int, code: int):
-    P = REG[d]
-    lines = slot_pointer()
+def slot_address(cls: int, sz: int, prefetch: bool):
+    """ptr = address of this thread's chunk in pointer slot `imm` (the slot was linked as vector-capable)."""
+    lines = ["@ptail bra L_ESC;", "shl.b32 sa, imm, 3;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b64 ptr, [sa+{SM_PTR}];",
+             "setp.lt.s64 p, ptr, 0;", "@p bra L_ESC;"]  # bit 63: this pointer cannot take vector accesses after all
     if cls == 0:
-        # a slot staged by asynchronous copies is read from this thread's staging buffer instead
-        lines += ["shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b32 w0, [sa+{SM_SOFF}];",
-                  "setp.eq.s32 p, w0, -1;", f"@p bra L_G{code};", f"add.u32 w0, w0, {STG};"]
-        if sz == 0:
-            lines += ["ld.shared.v4.b32 {x0, x1, x2, x3}, [w0];", f"ld.shared.v4.b32 {{x4, x5, x6, x7}}, [w0+{STAGE_PIECE}];"] + pack(P, X)
-        elif sz == 1:
-            lines += ["ld.shared.v4.b32 {x0, x1, x2, x3}, [w0];", f"mov.b64 {P[0]}, {{x0, x1}};", f"mov.b64 {P[1]}, {{x2, x3}};"]
-        else:
-            lines += ["ld.shared.v2.b32 {x0, x1}, [w0];", f"mov.b64 {P[0]}, {{x0, x1}};"]
-        lines += ["@DISPATCH@", f"L_G{code}:"]
         lines.append(f"shr.u64 offs, {OFF4}, {sz};" if sz else f"mov.b64 offs, {OFF4};")
     else:
         lines += [f"cvt.u64.u32 offs, {COFF4};"] + ([f"shr.u64 offs, offs, {sz};"] if sz else [])
     lines.append("add.u64 ptr, ptr, offs;")
-    if cls == 0:
+    if prefetch and cls == 0:
         # pull this thread's next chunk of the same input into L2 while the current one is processed
         lines += [f"shr.u64 offs, {PF4}, {sz};" if sz else f"mov.b64 offs, {PF4};", "add.u64 offs, ptr, offs;",
                   "@pnext prefetch.global.L2 [offs];"]
-    ld = "ld.global.cs" if cls == 0 else "ld.global.nc"
-    if sz == 0:
-        lines += [f"{ld}.v4.b32 {{x0, x1, x2, x3}}, [ptr];", f"{ld}.v4.b32 {{x4, x5, x6, x7}}, [ptr+16];"] + pack(P, X)
-    elif sz == 1:
-        lines += [f"{ld}.v4.b32 {{x0, x1, x2, x3}}, [ptr];", f"mov.b64 {P[0]}, {{x0, x1}};", f"mov.b64 {P[1]}, {{x2, x3}};"]
-    else:
-        lines += [f"{ld}.v2.b32 {{x0, x1}}, [ptr];", f"mov.b64 {P[0]}, {{x0, x1}};"]
     return lines
 
 
-def stv_body(sz: int):
-    lines = slot_pointer()
-    lines.append(f"shr.u64 offs, {OFF4}, {sz};" if sz else f"mov.b64 offs, {OFF4};")
-    lines.append("add.u64 ptr, ptr, offs;")
-    lines += unpack(A, X)
+def raw_load(sz: int, space: str, addr: str):
+    """Raw chunk into x0.. : 8 words (4-byte elements), 4 words (2-byte) or 2 words (1-byte)."""
+    if sz == 0:
+        return [f"{space}.v4.b32 {{x0, x1, x2, x3}}, [{addr}];", f"{space}.v4.b32 {{x4, x5, x6, x7}}, [{addr}+{16 if 'global' in space else STAGE_PIECE}];"]
+    if sz == 1:
+        return [f"{space}.v4.b32 {{x0, x1, x2, x3}}, [{addr}];"]
+    return [f"{space}.v2.b32 {{x0, x1}}, [{addr}];"]
+
+
+def widened_pair(sz: int, j: int, dst: str):
+    """PTX putting lanes 2j, 2j+1 of the raw chunk in x0.. into the 64-bit register `dst` as 32-bit lanes."""
+    if sz == 0:
+        return [f"mov.b64 {dst}, {{x{2 * j}, x{2 * j + 1}}};"]
+    if sz == 1:
+        return [f"shl.b32 y0, x{j}, 16;", f"and.b32 y1, x{j}, 0xFFFF0000;", f"mov.b64 {dst}, {{y0, y1}};"]
+    w, k = divmod(2 * j, 4)
+    return [f"bfe.u32 y0, x{w}, {8 * k}, 8;", f"bfe.u32 y1, x{w}, {8 * k + 8}, 8;", f"mov.b64 {dst}, {{y0, y1}};"]
+
+
+def ldg_body(sz: int, cls: int, d: int):
+    space = "ld.global.cs" if cls == 0 else "ld.global.nc"
+    lines = slot_address(cls, sz, True) + raw_load(sz, space, "ptr")
+    for j in (3, 2, 1, 0):
+        lines += widened_pair(sz, j, REG[d][j])
+    return lines
+
+
+def lds_body(sz: int, d: int):
+    lines = ["@ptail bra L_ESC;", f"add.u32 w0, imm, {STG};"] + raw_load(sz, "ld.shared", "w0")
+    for j in (3, 2, 1, 0):
+        lines += widened_pair(sz, j, REG[d][j])
+    return lines
+
+
+def f2m_tail(k: int, sz: int):
+    op = ["add", "sub", "rsub", "mul"][k]
+    lines = []
+    for j in range(4):
+        lines += widened_pair(sz, j, "g0")
+        lines.append(f"sub.rn.f32x2 {A[j]}, g0, {A[j]};" if op == "rsub" else f"{op}.rn.f32x2 {A[j]}, {A[j]}, g0;")
+    return lines
+
+
+def f2mg_body(k: int, sz: int, cls: int):
+    space = "ld.global.cs" if cls == 0 else "ld.global.nc"
+    return slot_address(cls, sz, True) + raw_load(sz, space, "ptr") + f2m_tail(k, sz)
+
+
+def f2ms_body(k: int, sz: int):
+    return ["@ptail bra L_ESC;", f"add.u32 w0, imm, {STG};"] + raw_load(sz, "ld.shared", "w0") + f2m_tail(k, sz)
+
+
+def stg_body(sz: int):
+    lines = slot_address(0, sz, False) + unpack(A, X)
     if sz == 0:
         lines += ["st.global.cs.v4.b32 [ptr], {x0, x1, x2, x3};", "st.global.cs.v4.b32 [ptr+16], {x4, x5, x6, x7};"]
     elif sz == 1:
@@ -414,11 +442,15 @@ def build(flavour: str) -> list[str]:
         if b is not None:
             bodies[OPS[name]] = b
     for sz in range(3):
-        for cls in range(2):
-            for d in range(5):
-                code = OPS["OP_LDV"] + (sz * 2 + cls) * 5 + d
-                bodies[code] = ldv_body(sz, cls, d, code)
-        bodies[OPS["OP_STV"] + sz] = stv_body(sz)
+        for d in range(5):
+            for cls in range(2):
+                bodies[OPS["OP_LDG"] + (sz * 2 + cls) * 5 + d] = ldg_body(sz, cls, d)
+            bodies[OPS["OP_LDS"] + sz * 5 + d] = lds_body(sz, d)
+        bodies[OPS["OP_STG"] + sz] = stg_body(sz)
+        for k in range(OPS["F2M_COUNT"]):
+            for cls in range(2):
+                bodies[OPS["OP_F2MG"] + (k * 3 + sz) * 2 + cls] = f2mg_body(k, sz, cls)
+            bodies[OPS["OP_F2MS"] + k * 3 + sz] = f2ms_body(k, sz)
     for idx in range(OPS["F2_COUNT"]):
         for k in range(NSRC):
             bodies[OPS["OP_F2"] + idx * NSRC + k] = f2_body(idx, Src(k), flavour)

@@ -288,6 +288,24 @@ __device__ __forceinline__ void load_raw(float (&d)[V], const Env &E, uint32_t s
     }
 }
 
+// raw chunk (storage format) -> 32-bit lanes
+__device__ __forceinline__ void widen(float (&d)[V], uint32_t dt) {
+    if (dt == LT_ST_BF16) {
+        uint32_t w0 = f2u(d[0]), w1 = f2u(d[1]), w2 = f2u(d[2]), w3 = f2u(d[3]);
+        d[0] = u2f(w0 << 16); d[1] = u2f(w0 & 0xffff0000u);
+        d[2] = u2f(w1 << 16); d[3] = u2f(w1 & 0xffff0000u);
+        d[4] = u2f(w2 << 16); d[5] = u2f(w2 & 0xffff0000u);
+        d[6] = u2f(w3 << 16); d[7] = u2f(w3 & 0xffff0000u);
+    } else if (dt == LT_ST_U8) {
+        uint32_t w0 = f2u(d[0]), w1 = f2u(d[1]);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            d[b] = u2f((w0 >> (8 * b)) & 0xffu);
+            d[4 + b] = u2f((w1 >> (8 * b)) & 0xffu);
+        }
+    }
+}
+
 __device__ __noinline__ void store_chunk_slow(const float *a, char *p, uint32_t dt, int nvalid) {
     for (int i = 0; i < V; ++i) {
         if (i < nvalid) {
@@ -422,9 +440,19 @@ __device__ __forceinline__ void pairs_of(const float (&f)[V], uint64_t (&p)[4]) 
 // not implement (see gen_vm_core.py); that opcode is executed here and the core re-entered.  With
 // LtLoop::inloop set the core also walks the thread's chunks by itself and `chunk_of(c)` rebuilds the
 // coordinates of chunk c for the code here; otherwise the call covers the one chunk given.
+// Pointer slot an escaped load/store refers to: the immediate is the slot, except for staged forms,
+// whose immediate is the slot's offset inside the staging buffer.
+__device__ __forceinline__ uint32_t slot_of(const Staged &S, bool staged, uint32_t imm) {
+    if (!staged) return imm;
+    uint32_t s = 0;
+    while (s + 1 < LT_VM_MAX_PTR && S.soff[s] != imm) ++s;
+    return s;
+}
+
 template <int FLAV, bool ROW, class Env, class ChunkOf>
 __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint32_t c, const Chunk &first, RowCtx *rc,
-                                            uint32_t smem_s, uint32_t stg) {
+                                            const Staged &S, uint32_t stg) {
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
     uint64_t R[5][4];  // not initialised: a program writes every register before it reads it
     uint32_t pc = smem_s;
     uint64_t off4 = first.flat0 << 2;
@@ -439,18 +467,36 @@ __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint
         if (eop == OP_END) break;
         const Chunk ck = chunk_of(c);
         float f[V];
-        if (eop >= OP_LD && eop < OP_STV) {  // generic load, or a vector load that met a ragged chunk / unaligned pointer
-            const uint32_t d = eop < OP_LDV ? eop - OP_LD : (eop - OP_LDV) % 5u;
-            load_raw(f, E, eimm, ck);
-            if (d == 0) pairs_of(f, R[0]);
-            else if (d == 1) pairs_of(f, R[1]);
-            else if (d == 2) pairs_of(f, R[2]);
-            else if (d == 3) pairs_of(f, R[3]);
-            else pairs_of(f, R[4]);
+        const bool is_ld = (eop >= OP_LD && eop < OP_STG) || (eop >= OP_LDS && eop < OP_F2M);
+        const bool is_f2m = eop >= OP_F2M && eop < OP_LIMIT;
+        if (is_ld || is_f2m) {
+            // a load that was not linked to a vector path (unaligned pointer, broadcast class), or one
+            // that met a ragged chunk: element-wise load, then widen
+            const bool staged = (eop >= OP_LDS && eop < OP_F2M) || eop >= OP_F2MS;
+            const uint32_t slot = slot_of(S, staged, eimm);
+            load_raw(f, E, slot, ck);
+            widen(f, E.dtype(slot));
+            if (is_ld) {
+                const uint32_t d = eop < OP_LDG ? eop - OP_LD : eop < OP_STG ? (eop - OP_LDG) % 5u : (eop - OP_LDS) % 5u;
+                if (d == 0) pairs_of(f, R[0]);
+                else if (d == 1) pairs_of(f, R[1]);
+                else if (d == 2) pairs_of(f, R[2]);
+                else if (d == 3) pairs_of(f, R[3]);
+                else pairs_of(f, R[4]);
+            } else {
+                const uint32_t k = eop < OP_F2MG ? eop - OP_F2M : eop < OP_F2MS ? (eop - OP_F2MG) / 6u : (eop - OP_F2MS) / 3u;
+                float a[V];
+                lanes_of(R[4], a);
+#pragma unroll
+                for (int i = 0; i < V; ++i)
+                    a[i] = k == F2M_ADD ? __fadd_rn(a[i], f[i]) : k == F2M_SUB ? __fsub_rn(a[i], f[i])
+                         : k == F2M_RSUB ? __fsub_rn(f[i], a[i]) : __fmul_rn(a[i], f[i]);
+                pairs_of(a, R[4]);
+            }
             continue;
         }
         lanes_of(R[4], f);
-        if (eop == OP_ST || (eop >= OP_STV && eop < OP_STV + 3)) {
+        if (eop == OP_ST || (eop >= OP_STG && eop < OP_STG + 3)) {
             store_chunk(f, E, eimm, ck);
             continue;
         }
@@ -495,6 +541,35 @@ __device__ __forceinline__ void stage_program(Staged &S, const P &prm) {
     for (uint32_t i = threadIdx.x; i < LT_VM_MAX_SCAL; i += blockDim.x) S.scal[i] = prm.scal[i];
     if (threadIdx.x < LT_VM_MAX_PTR) S.soff[threadIdx.x] = 0xffffffffu;
     if (threadIdx.x < sizeof(LtLoop) / 4) reinterpret_cast<uint32_t *>(&S.loop)[threadIdx.x] = 0;
+}
+
+// Link step: rewrites the generic load / store / memory-operand opcodes of the staged program into the
+// vector-path forms this launch's pointers allow (see vm.h).  S.ptr (bit 63 = no vector path) and S.soff
+// must be final.  `all_slots_ok` false keeps everything generic.
+__device__ __forceinline__ void link_program(Staged &S, uint32_t n_ins, const uint8_t *io_dtype, const uint8_t *io_class,
+                                             bool multi) {
+    for (uint32_t i = threadIdx.x; i < n_ins; i += blockDim.x) {
+        LtIns in = S.ins[i];
+        const uint32_t op = in.op, slot = in.imm;
+        const bool ld = op >= OP_LD && op < OP_LD + 5, st = op == OP_ST, f2m = op >= OP_F2M && op < OP_F2M + F2M_COUNT;
+        if (!(ld || st || f2m)) continue;
+        const uint32_t dt = io_dtype[slot], cls = multi ? (uint32_t)LT_CLS_FULL : (uint32_t)io_class[slot];
+        if ((S.ptr[slot] >> 63) || cls > LT_CLS_COLVEC) continue;
+        const uint32_t sz = dt == LT_ST_BF16 ? 1u : dt == LT_ST_U8 ? 2u : 0u;
+        const bool staged = S.soff[slot] != 0xffffffffu;
+        if (ld) {
+            const uint32_t d = op - OP_LD;
+            if (staged) { in.op = OP_LDS + sz * 5 + d; in.imm = S.soff[slot]; }
+            else in.op = OP_LDG + (sz * 2 + cls) * 5 + d;
+        } else if (f2m) {
+            const uint32_t k = op - OP_F2M;
+            if (staged) { in.op = OP_F2MS + k * 3 + sz; in.imm = S.soff[slot]; }
+            else in.op = OP_F2MG + (k * 3 + sz) * 2 + cls;
+        } else if (cls == LT_CLS_FULL) {
+            in.op = OP_STG + sz;
+        }
+        S.ins[i] = in;
+    }
 }
 
 // Asynchronous 16-byte (or 8-byte) copy global -> shared; completion is tracked per thread in groups.
@@ -600,6 +675,8 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
         lp.stg_n = k;
     }
     __syncthreads();
+    link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
+    __syncthreads();
     const uint32_t c0 = blockIdx.x * blockDim.x + threadIdx.x;
     if (c0 >= n_chunks) return;
     // Software pipeline: the full-class inputs of the thread's next `depth` chunks are in flight as
@@ -614,8 +691,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
         }
         cp_async_wait(depth - 1);
     }
-    run_program<FLAV, false>(E, [&P](uint32_t c) { return ew_chunk(P, c); }, c0, ew_chunk(P, c0), nullptr,
-                             (uint32_t)__cvta_generic_to_shared(&S), buf0);
+    run_program<FLAV, false>(E, [&P](uint32_t c) { return ew_chunk(P, c); }, c0, ew_chunk(P, c0), nullptr, S, buf0);
     if (depth) cp_async_wait(0);
 }
 
@@ -637,7 +713,8 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
         S.loop.pf_hi = (uint32_t)(pf >> 32);
     }
     __syncthreads();
-    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
+    link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
+    __syncthreads();
     RowCtx rc;
     rc.smem = S.red;
     rc.phase = 0;
@@ -658,7 +735,7 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
             nv = rem < (uint32_t)V ? (int)rem : V;
         }
         ck.nvalid = nv;
-        run_program<FLAV, true>(E, [&ck](uint32_t) { return ck; }, rb, ck, &rc, smem_s, 0);
+        run_program<FLAV, true>(E, [&ck](uint32_t) { return ck; }, rb, ck, &rc, S, 0);
     }
 }
 
@@ -666,7 +743,11 @@ template <int FLAV>
 __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
     __shared__ __align__(16) Staged S;
     stage_program(S, P);
-    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
+    if (threadIdx.x < LT_VM_MAX_PTR) S.ptr[threadIdx.x] = 0;
+    __syncthreads();
+    // linked once for all instances; an instance with an unaligned pointer has that slot flagged below and
+    // its accesses leave the vector path at run time
+    link_program(S, P.n_ins, P.io_dtype, nullptr, true);
     for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
         // instance that owns super-chunk sc: last i with super_prefix[i] <= sc
         uint32_t lo = 0, hi = P.n_inst;
@@ -691,7 +772,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
                 ck.row_ok = true;
                 const uint32_t rem = numel - e0;
                 ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
-                run_program<FLAV, false>(E, [&ck](uint32_t) { return ck; }, 0, ck, nullptr, smem_s, 0);
+                run_program<FLAV, false>(E, [&ck](uint32_t) { return ck; }, 0, ck, nullptr, S, 0);
             }
         }
     }

@@ -107,19 +107,9 @@ struct CodeGen {
         g.ins.push_back(in);
     }
 
-    static uint32_t size_class(int dt) { return dt == LT_BF16 ? 1u : dt == LT_U8 ? 2u : 0u; }
-
-    // raw chunk load of input v into register d (0..3 = T0..T3, 4 = ACC)
-    void emit_load(int d, uint32_t v) {
-        const int s = input_slot(v);
-        const IoRef &io = g.io[s];
-        if (io.cls == LT_CLS_FULL || io.cls == LT_CLS_COLVEC)
-            emit_ins(OP_LDV + (size_class(io.dtype) * 2 + (io.cls == LT_CLS_COLVEC ? 1u : 0u)) * 5 + (uint32_t)d, (uint32_t)s);
-        else
-            emit_ins(OP_LD + (uint32_t)d, (uint32_t)s);
-    }
-
-    void emit_widen(int d, int dt) { emit_ins((dt == LT_BF16 ? OP_CVT_BF16 : OP_CVT_U8) + (uint32_t)d); }
+    // chunk of input v, widened to 32-bit lanes, into register d (0..3 = T0..T3, 4 = ACC); the kernel
+    // rewrites the generic opcode into a vector-path one when the pointer allows (see vm.h)
+    void emit_load(int d, uint32_t v) { emit_ins(OP_LD + (uint32_t)d, (uint32_t)input_slot(v)); }
 
     int cls_of(uint32_t v) const {
         const PNode &p = pn[v];
@@ -203,12 +193,7 @@ struct CodeGen {
 
     static bool needs_widen(int dt) { return dt == LT_BF16 || dt == LT_U8; }
 
-    void widen_temp(int k) {
-        if (temp_raw[k] >= 0) {
-            emit_widen(k, temp_raw[k]);
-            temp_raw[k] = -1;
-        }
-    }
+    void widen_temp(int) {}  // loads deliver widened lanes
 
     // value v available, widened, in a temporary; returns its index
     int ensure_temp(int v) {
@@ -222,8 +207,6 @@ struct CodeGen {
             emit_ins((uint16_t)(OP_MOV_T_ACC + k));
         } else if (is_input((uint32_t)v)) {
             emit_load(k, (uint32_t)v);
-            int dt = cg.nodes[v].dtype;
-            if (needs_widen(dt)) emit_widen(k, dt);
         } else {
             ok = false;  // value was never computed: planner bug
             return 0;
@@ -244,8 +227,6 @@ struct CodeGen {
             emit_ins((uint16_t)(OP_MOV_ACC_T + temp_of[v]));
         } else if (is_input((uint32_t)v)) {
             emit_load(4, (uint32_t)v);
-            int dt = cg.nodes[v].dtype;
-            if (needs_widen(dt)) emit_widen(4, dt);
         } else {
             ok = false;
             return;
@@ -256,6 +237,9 @@ struct CodeGen {
     void consume(int v) {
         uses[v]--;
     }
+
+    // can v be read straight from memory by the one instruction that uses it?
+    bool mem_operand_ok(int v) const { return is_input((uint32_t)v) && uses[v] == 1 && temp_of[v] < 0 && in_acc != v; }
 
     void preload(int count) {
         // issue the loads of the first `count` inputs up front so they are all in flight together
@@ -273,8 +257,7 @@ struct CodeGen {
             emit_load(k, v);
             temp_val[k] = (int)v;
             temp_of[v] = k;
-            int dt = cg.nodes[v].dtype;
-            temp_raw[k] = needs_widen(dt) ? dt : -1;
+            temp_raw[k] = -1;
         }
     }
 
@@ -309,7 +292,7 @@ struct CodeGen {
         if (io.cls == LT_CLS_ROWVEC && !has_reduce) needs_rowcol = true;
         int s = (int)g.io.size();
         g.io.push_back(io);
-        emit_ins(io.cls == LT_CLS_FULL ? OP_STV + size_class(io.dtype) : (uint32_t)OP_ST, (uint32_t)s);
+        emit_ins(OP_ST, (uint32_t)s);
     }
 
     // ---- one node
@@ -376,6 +359,22 @@ struct CodeGen {
                     src = ensure_temp(x);
                     if (!ok) return;
                 }
+            } else if (!compare && is_float((uint8_t)dt) && (op == LT_OP_ADD || op == LT_OP_SUB || op == LT_OP_MUL) &&
+                       (mem_operand_ok(x) || mem_operand_ok(y))) {
+                // an input read exactly once: fold its load into the arithmetic (memory operand)
+                const bool pick_y = mem_operand_ok(y);
+                const int mem = pick_y ? y : x, reg = pick_y ? x : y;
+                swapped = !pick_y;  // ACC holds the other operand: "ACC (op) mem" must compute x (op) y
+                ensure_acc(reg);
+                if (!ok) return;
+                consume(reg);
+                consume(mem);
+                spill_acc();
+                if (!ok) return;
+                const int slot = input_slot((uint32_t)mem);
+                const uint32_t k = op == LT_OP_ADD ? F2M_ADD : op == LT_OP_MUL ? F2M_MUL : (swapped ? F2M_RSUB : F2M_SUB);
+                emit_ins(OP_F2M + k, (uint32_t)slot);
+                src = -3;  // already emitted
             } else {
                 // put one operand in ACC (prefer the one already there), the other in a temporary
                 if (in_acc == y && in_acc != x) swapped = true;
@@ -394,8 +393,9 @@ struct CodeGen {
                 if (!ok) return;
             }
             // opcode
-            uint16_t code;
-            if (src == -2) {
+            uint16_t code = 0;
+            if (src == -3) {
+            } else if (src == -2) {
                 code = OP_U_SQUARE;
             } else if (compare) {
                 int cc = op - LT_OP_GT;
@@ -428,7 +428,7 @@ struct CodeGen {
                 }
                 code = (uint16_t)(OP_I2 + idx * LT_VM_NSRC + src);
             }
-            emit_ins(code, imm);
+            if (src != -3) emit_ins(code, imm);
             if (x >= 0) drop_if_dead(x);
             if (y >= 0) drop_if_dead(y);
         } else if (op == LT_OP_WHERE) {
@@ -631,18 +631,13 @@ std::string disasm(const LtIns &in) {
     if (op >= OP_MOV_T_ACC && op < OP_MOV_ACC_T) snprintf(buf, sizeof(buf), "T%d = ACC", op - OP_MOV_T_ACC);
     else if (op >= OP_MOV_ACC_T && op < OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = T%d", op - OP_MOV_ACC_T);
     else if (op == OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = S%u", in.imm);
-    else if (op >= OP_LD && op < OP_STV) {
-        const int d = op < OP_LDV ? op - OP_LD : (op - OP_LDV) % 5;
-        const char *how = op < OP_LDV ? "load" : "vload";
-        if (d < 4) snprintf(buf, sizeof(buf), "T%d = %s p%u", d, how, in.imm);
-        else snprintf(buf, sizeof(buf), "ACC = %s p%u", how, in.imm);
-    } else if (op >= OP_CVT_BF16 && op < OP_ST) {
-        const int d = (op - OP_CVT_BF16) % 5;
-        const char *ty = op < OP_CVT_U8 ? "bf16" : "u8";
-        if (d < 4) snprintf(buf, sizeof(buf), "T%d = widen.%s T%d", d, ty, d);
-        else snprintf(buf, sizeof(buf), "ACC = widen.%s ACC", ty);
+    else if (op >= OP_LD && op < OP_LD + 5) {
+        if (op - OP_LD < 4) snprintf(buf, sizeof(buf), "T%d = load p%u", op - OP_LD, in.imm);
+        else snprintf(buf, sizeof(buf), "ACC = load p%u", in.imm);
+    } else if (op >= OP_F2M && op < OP_F2M + F2M_COUNT) {
+        static const char *f[] = {"add", "sub", "rsub", "mul"};
+        snprintf(buf, sizeof(buf), "ACC = f.%s ACC, load p%u", f[op - OP_F2M], in.imm);
     } else if (op == OP_ST) snprintf(buf, sizeof(buf), "store p%u = ACC", in.imm);
-    else if (op >= OP_STV && op < OP_STV + 3) snprintf(buf, sizeof(buf), "vstore p%u = ACC", in.imm);
     else if (op == OP_IOTA_COL) snprintf(buf, sizeof(buf), "ACC = iota.col");
     else if (op == OP_IOTA_ROW) snprintf(buf, sizeof(buf), "ACC = iota.row S%u S%u", in.imm, in.imm + 1);
     else if (op == OP_PHILOX) snprintf(buf, sizeof(buf), "ACC = philox S%u..S%u", in.imm, in.imm + 3);
@@ -894,7 +889,8 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                 }
                 n_inputs = (int)seen.size();
             }
-            for (int pre = std::min(n_inputs, LT_VM_NT); pre >= 0 && !done; --pre) {
+            (void)n_inputs;  // loads are issued where first needed: staged inputs are already on chip
+            for (int pre = 0; pre >= 0 && !done; --pre) {
                 g.ins.clear();
                 g.io.clear();
                 g.imms.clear();
@@ -1068,8 +1064,9 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                         int ld_pos = -1, st_pos = -1;
                         for (size_t q = 0; q < g.ins.size(); ++q) {
                             const LtIns &in = g.ins[q];
-                            if (in.op >= OP_LD && in.op < OP_STV && in.imm == rd.second && ld_pos < 0) ld_pos = (int)q;
-                            if ((in.op == OP_ST || (in.op >= OP_STV && in.op < OP_STV + 3)) && in.imm == s) st_pos = (int)q;
+                            const bool loads = (in.op >= OP_LD && in.op < OP_LD + 5) || (in.op >= OP_F2M && in.op < OP_F2M + F2M_COUNT);
+                            if (loads && in.imm == rd.second && ld_pos < 0) ld_pos = (int)q;
+                            if (in.op == OP_ST && in.imm == s) st_pos = (int)q;
                         }
                         if (ld_pos < 0 || st_pos < 0 || ld_pos > st_pos) { safe = false; break; }
                     } else if (launch_of[rg] >= launch_of[gi]) {

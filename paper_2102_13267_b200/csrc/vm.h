@@ -61,30 +61,42 @@ enum {
     OP_U_SQUARE, OP_U_SIGMOID, OP_U_GELU, OP_U_RBF16 /* round to bf16, keep as f32 */,
     OP_U_INEG = 43, OP_U_IABS = 44, OP_U_NOT = 45,
     OP_C_I2F = 46, OP_C_U2F = 47, OP_C_F2I = 48, OP_C_NZF = 49 /* f32 != 0 -> 0/1 */, OP_C_NZI = 50,
-    OP_LD = 51,          // +d : raw chunk load of pointer slot imm, any class and dtype (outside the PTX core)
-    // +(size * 2 + class) * 5 + d : raw chunk load on the vector path; size 0/1/2 = 4/2/1-byte elements,
-    // class 0 = full, 1 = column vector.  Ragged chunks and unaligned pointers fall back to OP_LD's code.
-    OP_LDV = 56,
-    OP_STV = 86,         // +size : vector-path store of ACC to a full-class slot (falls back to OP_ST's code)
+    // Loads deliver widened 32-bit lanes.  The planner emits the generic forms OP_LD / OP_F2M / OP_ST with
+    // the pointer slot as immediate; when a kernel starts, each is rewritten ("linked") for this launch's
+    // pointers into a vector-path opcode the PTX core executes itself -- ...G: 128-bit global access,
+    // ...S: read from the thread's staging buffer (immediate = byte offset in the buffer).  Slots that
+    // cannot use vector accesses keep the generic opcode, which the C++ around the core handles.
+    // size 0/1/2 = 4/2/1-byte elements; class 0 = full, 1 = column vector; d 0..3 = T0..T3, 4 = ACC.
+    OP_LD = 51,          // +d
+    OP_LDG = 56,         // +(size * 2 + class) * 5 + d
+    OP_STG = 86,         // +size : vector store of ACC to a full-class slot
     // two-operand families: opcode = base + index * LT_VM_NSRC + source
     OP_F2 = 96,          // ACC = ACC (op) src, f32: see F2_*
     OP_I2 = 136,         // integer: see I2_*
     OP_CMP = 192,        // ACC = (ACC cmp src) ? 1 : 0 : see CC_*
     OP_WHERE_A = 288,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? ACC : src
     OP_WHERE_B = 308,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? src : ACC
-    OP_LIMIT = 328
+    OP_LDS = 328,        // +size * 5 + d : staged load
+    OP_F2M = 343,        // +k : ACC = ACC (op) widened chunk of slot imm; k: see F2M_*
+    OP_F2MG = 347,       // +(k * 3 + size) * 2 + class
+    OP_F2MS = 371,       // +k * 3 + size
+    OP_LIMIT = 383
 };
+enum { F2M_ADD = 0, F2M_SUB, F2M_RSUB, F2M_MUL, F2M_COUNT };
 
 enum { F2_ADD = 0, F2_SUB, F2_RSUB, F2_MUL, F2_DIV, F2_RDIV, F2_MAX, F2_MIN, F2_COUNT };
 enum { I2_ADD = 0, I2_SUB, I2_RSUB, I2_MUL, I2_AND, I2_OR, I2_XOR, I2_MAXS, I2_MINS, I2_MAXU, I2_MINU, I2_COUNT };
 // compare index = type * 6 + cc ; type 0 f32, 1 signed, 2 unsigned ; cc: GT GE LT LE EQ NE
 enum { CC_GT = 0, CC_GE, CC_LT, CC_LE, CC_EQ, CC_NE };
 
-static_assert(OP_LDV + 30 == OP_STV && OP_STV + 3 <= OP_F2, "opcode map");
+static_assert(OP_LDG + 30 == OP_STG && OP_STG + 3 <= OP_F2, "opcode map");
+static_assert(OP_LDS + 15 == OP_F2M && OP_F2M + F2M_COUNT == OP_F2MG && OP_F2MG + F2M_COUNT * 6 == OP_F2MS &&
+                  OP_F2MS + F2M_COUNT * 3 == OP_LIMIT,
+              "opcode map");
 static_assert(OP_F2 + F2_COUNT * LT_VM_NSRC == OP_I2, "opcode map");
 static_assert(OP_I2 + I2_COUNT * LT_VM_NSRC <= OP_CMP, "opcode map");
 static_assert(OP_CMP + 18 * LT_VM_NSRC <= OP_WHERE_A, "opcode map");
-static_assert(OP_WHERE_B + 4 * LT_VM_NSRC == OP_LIMIT, "opcode map");
+static_assert(OP_WHERE_B + 4 * LT_VM_NSRC == OP_LDS, "opcode map");
 
 // Per-CTA constants of the chunk loop, in shared memory (read by the PTX core with broadcast loads).
 struct LtLoop {

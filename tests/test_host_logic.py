@@ -246,7 +246,7 @@ def test_second_reader_in_the_same_kernel_keeps_donation(ctx):
     s = ctx.stats()
     assert s["kernels_launched"] == 1 and s["outputs_donated"] == 1 and s["outputs_allocated"] == 1
     plan = ctx.dump_plan()
-    assert plan.index("vload p0") < plan.index("vstore")  # the old value is read before any store
+    assert plan.index("= load p0") < plan.index("  store p")  # the old value is read before any store
 
 
 def test_no_donation_while_another_tensor_names_the_old_value(ctx):
