@@ -1,0 +1,111 @@
+"""Kernel-only timing of the five benchmark configurations (also the driver for ncu captures).
+
+    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5] [--iters N] [--sets K] [key=value ...]
+
+For each configuration: traces the graph, flushes it `iters` times over rotating buffer sets
+(larger than L2 together) with per-launch CUDA events, and prints microseconds per flush and
+algorithmic GB/s.  `key=value` pairs are context options (e.g. fusion=0, stage=0, ieee=1).
+With `--iters 4 --sets 1` it is the small workload used for `ncu --set full` captures.
+"""
+from __future__ import annotations
+
+import argparse
+import math
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+import torch
+
+import paper_2102_13267_b200 as lt
+from workloads import configs, traces
+from workloads.resnet50 import parameter_shapes
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("configs", nargs="?", default="c1,c2,c2p,c3,c4,c5")
+    ap.add_argument("--iters", type=int, default=40)
+    ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate through (0 = enough for 1 GB)")
+    ap.add_argument("options", nargs="*")
+    args = ap.parse_args()
+    which = args.configs.split(",")
+    opts = dict(kv.split("=") for kv in args.options)
+    dev = torch.device("cuda", 0)
+
+    def context():
+        ctx = lt.LazyContext(device=0)
+        for k, v in opts.items():
+            ctx.set_option(k, int(v))
+        return ctx
+
+    def bf16(shape, std=1.0):
+        return (torch.randn(shape, device=dev) * std).to(torch.bfloat16)
+
+    def report(name, nbytes, ctx):
+        kt = ctx.kernel_timing()
+        ms = sum(v["ms"] for v in kt.values()) / args.iters
+        n = sum(v["launches"] for v in kt.values()) / args.iters
+        print(f"{name:4s} {1e3 * ms:9.1f} us/flush {nbytes / ms / 1e6:8.1f} GB/s  {n:.0f} launches/flush", flush=True)
+
+    def run(name, cfg, make, trace):
+        nbytes = configs.algorithmic_bytes(cfg)
+        nsets = args.sets or max(2, math.ceil(1.2e9 / nbytes))
+        ctx = context()
+        sets = [make(ctx) for _ in range(nsets)]
+        keep = [None] * nsets
+        for i in range(min(5, args.iters)):
+            keep[i % nsets] = trace(ctx, sets[i % nsets])
+            ctx.barrier()
+        torch.cuda.synchronize()
+        ctx.set_kernel_timing(True)
+        ctx.kernel_timing()
+        for i in range(args.iters):
+            keep[i % nsets] = trace(ctx, sets[i % nsets])
+            ctx.barrier()
+        report(name, nbytes, ctx)
+        del keep, sets
+        ctx.close()
+
+    if "c1" in which:
+        shape = configs.FULL["c1"]
+        run("c1", "c1", lambda c: [c.from_torch(torch.rand(shape, device=dev) * 2 - 1) for _ in range(4)],
+            lambda c, s: traces.elementwise_chain(c, *s))
+    for name, prim in (("c2", False), ("c2p", True)):
+        if name in which:
+            shape = configs.FULL["c2"]
+            run(name, "c2", lambda c: (c.from_torch(bf16(shape)), c.from_torch(bf16(shape)), c.from_torch(bf16((shape[1],), 0.02))),
+                lambda c, s, prim=prim: traces.mlp_epilogue(c, *s, primitive_gelu=prim))
+    if "c3" in which:
+        shape = configs.FULL["c3"]
+        run("c3", "c3", lambda c: (c.from_torch(bf16(shape)), c.from_torch(bf16(shape)),
+                                   c.from_torch(1 + 0.02 * torch.randn(shape[1], device=dev)),
+                                   c.from_torch(0.02 * torch.randn(shape[1], device=dev))),
+            lambda c, s: traces.residual_dropout_layernorm(c, *s, shape=shape, p=0.1, eps=1e-5, seed=1, offset=0))
+    if "c4" in which:
+        shape = configs.FULL["c4"]
+        run("c4", "c4", lambda c: (c.from_torch(bf16(shape, 4.0)),),
+            lambda c, s: traces.causal_softmax(c, *s, shape=shape, scale=1 / math.sqrt(128)))
+    if "c5" in which:
+        shapes = parameter_shapes()
+        ctx = context()
+        P, G, M, V = ([ctx.from_torch(torch.randn(s, device=dev) * 0.05) for s in shapes] for _ in range(4))
+        step = 0
+        for _ in range(min(3, args.iters)):
+            step += 1
+            traces.adam_step(ctx, P, G, M, V, step=step)
+            ctx.barrier()
+        torch.cuda.synchronize()
+        ctx.set_kernel_timing(True)
+        ctx.kernel_timing()
+        for _ in range(args.iters):
+            step += 1
+            traces.adam_step(ctx, P, G, M, V, step=step)
+            ctx.barrier()
+        report("c5", configs.algorithmic_bytes("c5"), ctx)
+        ctx.close()
+
+
+if __name__ == "__main__":
+    main()
