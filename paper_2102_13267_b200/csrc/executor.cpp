@@ -116,6 +116,32 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 const Group &g = plan.groups[L.groups[k]];
                 for (size_t s = 0; s < slots; ++s) P.ptr[k * slots + s] = resolve(g.io[s]);
             }
+            // staging plan: a slot is staged when its pointer is aligned in every instance
+            {
+                uint32_t pieces = 0;
+                for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                if (c->opt.stage) {
+                    for (size_t s = 0; s < slots; ++s) {
+                        if (g0.io[s].is_store) continue;
+                        const uint64_t need = g0.io[s].dtype == LT_U8 ? 7u : 15u;
+                        bool ok = true;
+                        for (size_t k = 0; k < L.groups.size() && ok; ++k) ok = (P.ptr[k * slots + s] & need) == 0;
+                        if (!ok) continue;
+                        P.io_stage[s] = (uint8_t)pieces;
+                        pieces += (g0.io[s].dtype == LT_BF16 || g0.io[s].dtype == LT_U8) ? 1u : 2u;
+                    }
+                }
+                P.stage_pieces = pieces;
+                P.stage_depth = 0;
+                if (pieces) {
+                    const uint32_t buf = pieces * LT_VM_STAGE_PIECE;
+                    uint32_t depth = (96u * 1024u + (uint32_t)c->occ_multi * buf - 1) / ((uint32_t)c->occ_multi * buf);
+                    depth = std::min(4u, std::max(2u, depth));
+                    while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
+                    if (depth >= 2) P.stage_depth = depth;
+                    else for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                }
+            }
             if (!dry) {
                 unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * c->occ_multi * waves);
                 if (grid < 1) grid = 1;
@@ -129,10 +155,13 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             const Group &g = plan.groups[L.groups[0]];
             for (size_t q = 0; q < g.imms.size(); ++q) P.scal[q] = encode_imm(g.imms[q], cg.dyn);
             for (size_t s = 0; s < g.io.size(); ++s) P.ptr[s] = resolve(g.io[s]);
-            if (L.kind == K_EW) {
+            {
                 // Staging plan: aligned full-class inputs are copied asynchronously into per-thread
-                // shared-memory buffers a few chunks ahead (needs chunk c to start at element 8c).
-                const bool linear = !P.rowcol || (P.cols % LT_VM_V) == 0;
+                // shared-memory buffers a few chunks ahead.  Needs rows that are a multiple of the chunk
+                // (chunk c starts at element 8c) and 256-thread blocks (the buffer layout).
+                const bool linear = L.kind == K_EW ? (!P.rowcol || (P.cols % LT_VM_V) == 0)
+                                                   : ((P.cols % LT_VM_V) == 0 && L.threads == LT_EW_THREADS);
+                const uint32_t occ = (uint32_t)(L.kind == K_EW ? c->occ_ew : c->occ_row);
                 uint32_t pieces = 0;
                 for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
                 if (c->opt.stage && linear) {
@@ -149,12 +178,14 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 P.stage_depth = 0;
                 if (pieces) {
                     const uint32_t buf = pieces * LT_VM_STAGE_PIECE;
-                    uint32_t depth = (96u * 1024u + (uint32_t)c->occ_ew * buf - 1) / ((uint32_t)c->occ_ew * buf);
+                    uint32_t depth = (96u * 1024u + occ * buf - 1) / (occ * buf);
                     depth = std::min(4u, std::max(2u, depth));
                     while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
                     if (depth >= 2) P.stage_depth = depth;
                     else for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
                 }
+            }
+            if (L.kind == K_EW) {
                 if (!dry) {
                     uint64_t need = (P.n_chunks + LT_EW_THREADS - 1) / LT_EW_THREADS;
                     unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);

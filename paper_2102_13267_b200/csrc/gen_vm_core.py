@@ -361,10 +361,17 @@ def stg_body(sz: int):
     return lines
 
 
+SM_N4 = SM_PF + 8
+SM_GROUP = SM_PF + 16
+SM_RED = OPS["LT_VM_SM_RED"]
+
+
 def entry_code():
-    """Predicates that depend on the current chunk; recomputed whenever the asm statement is (re-)entered."""
+    """Registers that depend on the current chunk or thread; recomputed whenever the asm statement is
+    (re-)entered.  TAIL bits: 1 = this chunk is ragged or absent, 2 = the thread's column range is never a
+    full chunk (row kernel), 4 = which half of the reduction exchange buffer is next."""
     L = SM_LOOP
-    return [f"setp.ne.u32 ptail, {TAIL}, 0;",
+    return [f"and.b32 r0, {TAIL}, 1;", "setp.ne.u32 ptail, r0, 0;",
             f"ld.shared.v2.b32 {{r0, r1}}, [{SMB}+{L}];",            # stride, n_chunks
             f"ld.shared.b32 r2, [{SMB}+{L + 56}];",                   # prefetch enabled
             f"ld.shared.b64 pf4, [{SMB}+{SM_PF}];",
@@ -373,19 +380,21 @@ def entry_code():
 
 
 def end_body():
-    """OP_END.  When the core runs the chunk loop itself: refill the staging buffer just consumed, move to
-    the thread's next chunk, wait for its staged inputs and restart the program; else leave."""
+    """OP_END.  When the core runs the loop itself: refill the staging buffer just consumed, move to the
+    thread's next chunk (or block of rows), wait for its staged inputs and restart the program."""
     L = SM_LOOP
     return [
         f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 16}];",     # buf_bytes, buf_total, stage_base, inloop
         "setp.eq.u32 p, r7, 0;", "@p bra L_ESC;",
         f"ld.shared.v4.b32 {{r0, r1, r2, r3}}, [{SMB}+{L}];",          # stride, n_chunks, n_full, depth
+        f"ld.shared.b64 d2, [{SMB}+{SM_N4}];",                          # 4 * elements
         "setp.eq.u32 pq, r3, 0;", "@pq bra L_ADV;",
-        # chunk `depth` iterations ahead; staged only if it is complete
-        "mul.wide.u32 d0, r0, r3;", f"cvt.u64.u32 d1, {CHUNK};", "add.u64 d0, d0, d1;", "cvt.u64.u32 d1, r2;",
-        "setp.ge.u64 p, d0, d1;", "@p bra L_COMMIT;",
-        "shl.b64 d0, d0, 3;",                                            # first element of that chunk
-        f"ld.shared.b32 r7, [{SMB}+{L + 60}];",                         # number of staged inputs
+        # the chunk `depth` iterations ahead starts depth * pf4 bytes (4-byte view) further; staged if complete
+        "cvt.u64.u32 d1, r3;", "mul.lo.u64 d1, d1, pf4;", f"add.u64 d0, {OFF4}, d1;", "add.u64 d1, d0, 32;",
+        "setp.gt.u64 p, d1, d2;", f"and.b32 x0, {TAIL}, 2;", "setp.ne.u32 pq, x0, 0;", "or.pred p, p, pq;",
+        "@p bra L_COMMIT;",
+        "shr.u64 d0, d0, 2;",                                            # first element of that chunk
+        f"ld.shared.b32 r8, [{SMB}+{L + 60}];",                         # number of staged inputs
         f"add.u32 sa, {SMB}, {SM_STG};",
         "L_STG_LOOP:",
         "ld.shared.v4.b32 {x0, x1, x2, x3}, [sa];",                      # ptr lo, hi, dst offset, log2(bytes)
@@ -393,7 +402,7 @@ def end_body():
         "setp.eq.u32 p, x3, 0;", "@p cp.async.ca.shared.global [x2], [ptr], 8;",
         "@!p cp.async.cg.shared.global [x2], [ptr], 16;",
         "setp.eq.u32 p, x3, 2;", f"@p cp.async.cg.shared.global [x2+{STAGE_PIECE}], [ptr+16], 16;",
-        "add.u32 sa, sa, 16;", "sub.u32 r7, r7, 1;", "setp.ne.u32 p, r7, 0;", "@p bra L_STG_LOOP;",
+        "add.u32 sa, sa, 16;", "sub.u32 r8, r8, 1;", "setp.ne.u32 p, r8, 0;", "@p bra L_STG_LOOP;",
         "L_COMMIT:",
         "cp.async.commit_group;",
         # next staging buffer of this thread (a ring of `depth` buffers)
@@ -404,21 +413,89 @@ def end_body():
         "setp.eq.u32 p, r3, 4;", "@p cp.async.wait_group 3;",
         "L_ADV:",
         f"add.u32 {CHUNK}, {CHUNK}, r0;", f"setp.ge.u32 p, {CHUNK}, r1;", "@p bra L_ESC;",
-        f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 32}];",      # rowcol, cpr, div_mul, div_sh1
+        "setp.eq.u32 p, r7, 2;", "@p bra L_ROWS;",
+        f"ld.shared.v4.b32 {{r4, r5, r6, r9}}, [{SMB}+{L + 32}];",      # rowcol, cpr, div_mul, div_sh1
         "setp.ne.u32 p, r4, 0;", "@p bra L_ROWCOL;",
-        f"mul.wide.u32 {OFF4}, {CHUNK}, 32;", f"cvt.u32.u64 {COFF4}, {OFF4};",
-        f"setp.ge.u32 ptail, {CHUNK}, r2;", "bra L_COORD_DONE;",
+        # flat chunks: the next chunk of this thread is pf4 bytes further
+        f"add.u64 {OFF4}, {OFF4}, pf4;", f"cvt.u32.u64 {COFF4}, {OFF4};", f"add.u64 d1, {OFF4}, 32;",
+        "setp.gt.u64 ptail, d1, d2;", "bra L_COORD_DONE;",
+        "L_ROWS:",
+        # row kernel: same columns, a block of rows further; absent once past the last row
+        f"add.u64 {OFF4}, {OFF4}, pf4;", f"setp.ge.u64 ptail, {OFF4}, d2;", f"and.b32 x0, {TAIL}, 2;",
+        "setp.ne.u32 pq, x0, 0;", "or.pred ptail, ptail, pq;", "bra L_COORD_DONE;",
         "L_ROWCOL:",
         f"ld.shared.v2.b32 {{x2, x3}}, [{SMB}+{L + 48}];",               # div_sh2, cols
-        f"mul.hi.u32 x0, r6, {CHUNK};", f"sub.u32 x1, {CHUNK}, x0;", "shr.u32 x1, x1, r7;", "add.u32 x0, x0, x1;",
+        f"mul.hi.u32 x0, r6, {CHUNK};", f"sub.u32 x1, {CHUNK}, x0;", "shr.u32 x1, x1, r9;", "add.u32 x0, x0, x1;",
         "shr.u32 x0, x0, x2;",                                           # row
         f"mul.lo.u32 x1, x0, r5;", f"sub.u32 x1, {CHUNK}, x1;", "shl.b32 x1, x1, 3;",   # col0
         "mul.wide.u32 d0, x0, x3;", "cvt.u64.u32 d1, x1;", "add.u64 d0, d0, d1;", f"shl.b64 {OFF4}, d0, 2;",
         f"shl.b32 {COFF4}, x1, 2;", "sub.u32 x1, x3, x1;", "setp.lt.u32 ptail, x1, 8;",
         "L_COORD_DONE:",
-        f"selp.b32 {TAIL}, 1, 0, ptail;",
+        f"and.b32 {TAIL}, {TAIL}, 0xFFFFFFFE;", "selp.b32 x0, 1, 0, ptail;", f"or.b32 {TAIL}, {TAIL}, x0;",
         f"mov.b32 {PC}, {SMB};",
-    ] + entry_code()[1:] + [f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];"]
+    ] + entry_code()[2:] + [f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];"]
+
+
+def inline_rows_guard():
+    """Row-wise opcodes run in the core only when rows are regular (see LtLoop::inline_rows) and the chunk
+    is complete where that matters."""
+    return [f"ld.shared.v2.b32 {{r0, r1}}, [{SMB}+{SM_GROUP}];", "setp.eq.u32 p, r1, 0;", "@p bra L_ESC;"]
+
+
+def red_body(kind: int):
+    """ACC = reduction of the row, broadcast: lanes of the thread, then shuffles within the warp, then (rows
+    wider than a warp's 256 elements) one exchange through shared memory."""
+    op = ["add.rn.f32", "max.NaN.f32", "min.NaN.f32"][kind]
+    lines = inline_rows_guard()          # r0 = threads per row
+    lines += unpack(A, X)
+    lines += [f"{op} x0, x0, x1;", f"{op} x2, x2, x3;", f"{op} x4, x4, x5;", f"{op} x6, x6, x7;",
+              f"{op} x0, x0, x2;", f"{op} x4, x4, x6;", f"{op} x0, x0, x4;"]
+    for off in (16, 8, 4, 2, 1):
+        lines += [f"setp.gt.u32 p, r0, {off};", f"@p shfl.sync.bfly.b32 y0, x0, {off}, 0x1f, 0xffffffff;",
+                  f"@p {op} x0, x0, y0;"]
+    lines += [
+        "setp.le.u32 p, r0, 32;", f"@p bra L_RED_DONE{kind};",
+        "mov.u32 r2, %tid.x;", "shr.u32 r3, r2, 5;", "and.b32 r2, r2, 31;",          # r3 warp, r2 lane
+        f"and.b32 r4, {TAIL}, 4;", "shl.b32 r4, r4, 5;", f"add.u32 r4, r4, {SMB};",   # half of the exchange buffer
+        "shl.b32 r5, r3, 2;", "add.u32 r5, r5, r4;", "setp.eq.u32 p, r2, 0;", f"@p st.shared.b32 [r5+{SM_RED}], x0;",
+        "bar.sync 0;",
+        "shr.u32 r6, r0, 5;", "sub.u32 r7, r6, 1;", "not.b32 r7, r7;", "and.b32 r7, r3, r7;",   # r6 warps per row, r7 first warp of this row
+        "shl.b32 r7, r7, 2;", "add.u32 r7, r7, r4;", f"ld.shared.b32 x0, [r7+{SM_RED}];", "sub.u32 r6, r6, 1;",
+        f"L_RED_LOOP{kind}:", "add.u32 r7, r7, 4;", f"ld.shared.b32 y0, [r7+{SM_RED}];", f"{op} x0, x0, y0;",
+        "sub.u32 r6, r6, 1;", "setp.ne.u32 p, r6, 0;", f"@p bra L_RED_LOOP{kind};",
+        f"xor.b32 {TAIL}, {TAIL}, 4;",
+        f"L_RED_DONE{kind}:",
+    ]
+    lines += [f"mov.b64 {a}, {{x0, x0}};" for a in A]
+    return lines
+
+
+def iota_row_body():
+    """ACC = (row / scal[imm]) % scal[imm+1]; the row is recovered from the chunk's byte offsets."""
+    return inline_rows_guard() + [
+        f"cvt.u64.u32 d0, {COFF4};", f"sub.u64 d0, {OFF4}, d0;", "shr.u64 d0, d0, 2;", "cvt.u32.u64 x0, d0;",   # row * cols (< 2^32)
+        f"ld.shared.b32 x1, [{SMB}+{SM_LOOP + 52}];", "div.u32 x0, x0, x1;",                                   # row
+        "shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b32 x1, [sa+{SM_SCAL}];",
+        f"ld.shared.b32 x2, [sa+{SM_SCAL + 4}];", "div.u32 x0, x0, x1;", "rem.u32 x0, x0, x2;",
+    ] + [f"mov.b64 {a}, {{x0, x0}};" for a in A]
+
+
+def philox_body():
+    """ACC = Philox4x32-10 bits of the chunk's eight elements (two counter blocks; Salmon et al., SC'11)."""
+    lines = inline_rows_guard()[:0] + ["@ptail bra L_ESC;", "shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};",
+             f"ld.shared.v2.b32 {{r0, r1}}, [sa+{SM_SCAL}];", f"ld.shared.v2.b32 {{r2, r3}}, [sa+{SM_SCAL + 8}];",
+             f"shr.u64 d0, {OFF4}, 4;"]                                   # block index q = element / 4 (a complete chunk starts a block)
+    for blk in range(2):
+        lines += ["mov.b64 {x0, x1}, d0;", "mov.b32 x2, r2;", "mov.b32 x3, r3;", "mov.b32 y0, r0;", "mov.b32 y1, r1;"]
+        for rnd in range(10):
+            lines += ["mul.hi.u32 x4, x0, 0xD2511F53;", "mul.lo.u32 x5, x0, 0xD2511F53;",
+                      "mul.hi.u32 x6, x2, 0xCD9E8D57;", "mul.lo.u32 x7, x2, 0xCD9E8D57;",
+                      "xor.b32 x0, x6, x1;", "xor.b32 x0, x0, y0;", "mov.b32 x1, x7;",
+                      "xor.b32 x2, x4, x3;", "xor.b32 x2, x2, y1;", "mov.b32 x3, x5;"]
+            if rnd < 9:
+                lines += ["add.u32 y0, y0, 0x9E3779B9;", "add.u32 y1, y1, 0xBB67AE85;"]
+        lines += [f"mov.b64 {A[2 * blk]}, {{x0, x1}};", f"mov.b64 {A[2 * blk + 1]}, {{x2, x3}};", "add.u64 d0, d0, 1;"]
+    return lines
 
 
 def build(flavour: str) -> list[str]:
@@ -426,6 +503,10 @@ def build(flavour: str) -> list[str]:
     bodies: dict[int, list[str]] = {}
 
     bodies[OPS["OP_END"]] = end_body()
+    for kind in range(3):
+        bodies[OPS["OP_RED_SUM"] + kind] = red_body(kind)
+    bodies[OPS["OP_IOTA_ROW"]] = iota_row_body()
+    bodies[OPS["OP_PHILOX"]] = philox_body()
     for k in range(4):
         bodies[OPS["OP_MOV_T_ACC"] + k] = [f"mov.b64 {T[k][j]}, {A[j]};" for j in range(4)]
         bodies[OPS["OP_MOV_ACC_T"] + k] = [f"mov.b64 {A[j]}, {T[k][j]};" for j in range(4)]
@@ -466,9 +547,9 @@ def build(flavour: str) -> list[str]:
             bodies[OPS["OP_WHERE_B"] + m * NSRC + k] = where_body(m, Src(k), True)
 
     out = ["{"]
-    out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3, r0, r1, r2, r3, r4, r5, r6, r7;")
+    out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3, r0, r1, r2, r3, r4, r5, r6, r7, r8, r9;")
     out.append(".reg .b32 " + ", ".join(X + ["y0", "y1", "m0", "m1"]) + ";")
-    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2, d0, d1, pf4;")
+    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2, d0, d1, d2, pf4;")
     out.append(".reg .pred p, pq, ptail, pnext;")
     table = ", ".join(f"L_{i}" if i in bodies else "L_ESC" for i in range(limit))
     out.append(f"TBL: .branchtargets {table};")

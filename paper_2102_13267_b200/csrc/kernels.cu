@@ -405,7 +405,8 @@ struct Staged {
 static_assert(offsetof(Staged, scal) == LT_VM_SM_SCAL && offsetof(Staged, ptr) == LT_VM_SM_PTR &&
                   offsetof(Staged, soff) == LT_VM_SM_SOFF && offsetof(Staged, loop) == LT_VM_SM_LOOP &&
                   offsetof(Staged, loop.stg) == LT_VM_SM_STG &&
-                  offsetof(Staged, loop.pf_lo) == LT_VM_SM_STG + 16 * LT_VM_MAX_PTR,
+                  offsetof(Staged, loop.pf_lo) == LT_VM_SM_STG + 16 * LT_VM_MAX_PTR &&
+                  offsetof(Staged, red) == LT_VM_SM_RED,
               "the PTX core addresses these fields by constant offset");
 
 // Pointer-table entry for the PTX core: bit 63 marks a slot whose chunks cannot use 128-bit accesses.
@@ -451,13 +452,13 @@ __device__ __forceinline__ uint32_t slot_of(const Staged &S, bool staged, uint32
 
 template <int FLAV, bool ROW, class Env, class ChunkOf>
 __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint32_t c, const Chunk &first, RowCtx *rc,
-                                            const Staged &S, uint32_t stg) {
+                                            const Staged &S, uint32_t stg, uint32_t flags = 0) {
     const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
     uint64_t R[5][4];  // not initialised: a program writes every register before it reads it
     uint32_t pc = smem_s;
     uint64_t off4 = first.flat0 << 2;
     uint32_t coff4 = first.col0 << 2;
-    uint32_t tail = first.nvalid != V ? 1u : 0u;
+    uint32_t tail = (first.nvalid != V ? 1u : 0u) | flags;  // see entry_code() in gen_vm_core.py for the bits
 #pragma unroll 1
     for (;;) {
         uint32_t eop, eimm;
@@ -602,6 +603,46 @@ __device__ __forceinline__ void stage_chunk(const LtLoop &lp, uint64_t e0, uint3
     }
 }
 
+// Fills the loop constants shared by the elementwise and row kernels (thread 0, before the link step).
+__device__ __forceinline__ void fill_loop(LtLoop &lp, const LtKParams &P, uint32_t mode, uint32_t stride, uint32_t n_iter,
+                                          uint64_t step4, uint32_t stage_base, bool prefetch) {
+    const uint32_t depth = P.stage_depth;
+    lp.stride = stride;
+    lp.n_chunks = n_iter;
+    lp.n_full = (uint32_t)(P.n / V);
+    lp.depth = depth;
+    lp.buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
+    lp.buf_total = depth * lp.buf_bytes;
+    lp.stage_base = stage_base;
+    lp.inloop = mode;
+    lp.rowcol = P.rowcol;
+    lp.cpr = P.cpr;
+    lp.div_mul = P.div_mul;
+    lp.div_sh1 = P.div_sh1;
+    lp.div_sh2 = P.div_sh2;
+    lp.cols = P.cols;
+    lp.prefetch = (prefetch && !depth) ? 1u : 0u;  // without staging, pull the next chunk into L2 instead
+    lp.pf_lo = (uint32_t)step4;
+    lp.pf_hi = (uint32_t)(step4 >> 32);
+    lp.n4_lo = (uint32_t)(P.n * 4);
+    lp.n4_hi = (uint32_t)((P.n * 4) >> 32);
+    lp.group = P.group;
+    // row-wise opcodes run inside the core when every thread of a row group owns a complete chunk
+    const bool regular = (P.cols % V) == 0 && (mode != 2 || P.group * V == P.cols);
+    lp.inline_rows = (regular && P.n < (1ull << 32)) ? 1u : 0u;
+    uint32_t k = 0;
+    if (depth)
+        for (uint32_t s = 0; s < LT_VM_MAX_PTR; ++s)
+            if (P.io_stage[s] != 0xffu) {
+                lp.stg[k].ptr_lo = (uint32_t)P.ptr[s];
+                lp.stg[k].ptr_hi = (uint32_t)(P.ptr[s] >> 32);
+                lp.stg[k].dst = P.io_stage[s] * LT_VM_STAGE_PIECE;
+                lp.stg[k].shift = 2u - (P.io_dtype[s] == LT_ST_BF16 ? 1u : P.io_dtype[s] == LT_ST_U8 ? 2u : 0u);
+                ++k;
+            }
+    lp.stg_n = k;
+}
+
 __device__ __forceinline__ Chunk ew_chunk(const LtKParams &P, uint32_t c) {
     Chunk ck;
     ck.row_ok = true;
@@ -642,38 +683,8 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
         S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], linear);
         if (depth && P.io_stage[threadIdx.x] != 0xffu) S.soff[threadIdx.x] = P.io_stage[threadIdx.x] * LT_VM_STAGE_PIECE;
     }
-    if (threadIdx.x == 0) {
-        LtLoop &lp = S.loop;
-        lp.stride = stride;
-        lp.n_chunks = n_chunks;
-        lp.n_full = linear ? (uint32_t)(P.n / V) : 0;  // chunks below this index are complete
-        lp.depth = depth;
-        lp.buf_bytes = buf_bytes;
-        lp.buf_total = depth * buf_bytes;
-        lp.stage_base = stage_base;
-        lp.inloop = 1;
-        lp.rowcol = P.rowcol;
-        lp.cpr = P.cpr;
-        lp.div_mul = P.div_mul;
-        lp.div_sh1 = P.div_sh1;
-        lp.div_sh2 = P.div_sh2;
-        lp.cols = P.cols;
-        lp.prefetch = (linear && !depth) ? 1u : 0u;  // without staging, pull the next chunk into L2 instead
-        const uint64_t pf = (uint64_t)stride * (V * 4);
-        lp.pf_lo = (uint32_t)pf;
-        lp.pf_hi = (uint32_t)(pf >> 32);
-        uint32_t k = 0;
-        if (depth)
-            for (uint32_t s = 0; s < LT_VM_MAX_PTR; ++s)
-                if (P.io_stage[s] != 0xffu) {
-                    lp.stg[k].ptr_lo = (uint32_t)P.ptr[s];
-                    lp.stg[k].ptr_hi = (uint32_t)(P.ptr[s] >> 32);
-                    lp.stg[k].dst = P.io_stage[s] * LT_VM_STAGE_PIECE;
-                    lp.stg[k].shift = 2u - (P.io_dtype[s] == LT_ST_BF16 ? 1u : P.io_dtype[s] == LT_ST_U8 ? 2u : 0u);
-                    ++k;
-                }
-        lp.stg_n = k;
-    }
+    if (threadIdx.x == 0)
+        fill_loop(S.loop, P, 1, stride, n_chunks, (uint64_t)stride * (V * 4), stage_base, linear);
     __syncthreads();
     link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
     __syncthreads();
@@ -685,7 +696,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
     if (depth) {
         uint64_t c = c0;
         for (uint32_t d = 0; d < depth; ++d) {
-            if (c < S.loop.n_full) stage_chunk(S.loop, c * V, buf0 + d * buf_bytes);
+            if (c < P.n / V) stage_chunk(S.loop, c * V, buf0 + d * buf_bytes);
             cp_async_commit();
             c += stride;
         }
@@ -698,20 +709,21 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
 template <int FLAV, int MAXT>
 __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ LtKParams P) {
     __shared__ __align__(16) Staged S;
+    extern __shared__ __align__(16) unsigned char stage_mem[];
     const EnvK E{P};
     stage_program(S, P);
     __syncthreads();
     const uint32_t row_blocks = (P.rows + P.rows_per_cta - 1u) / P.rows_per_cta;
-    if (threadIdx.x < LT_VM_MAX_PTR)
-        S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], (P.cols % V) == 0);
-    if (threadIdx.x == 0) {  // the core only needs these to prefetch the next block of rows into L2
-        S.loop.stride = gridDim.x;
-        S.loop.n_chunks = row_blocks;
-        S.loop.prefetch = 1;
-        const uint64_t pf = (uint64_t)gridDim.x * P.rows_per_cta * P.cols * 4;
-        S.loop.pf_lo = (uint32_t)pf;
-        S.loop.pf_hi = (uint32_t)(pf >> 32);
+    const bool aligned_rows = (P.cols % V) == 0;
+    const uint32_t depth = P.stage_depth;
+    const uint32_t buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
+    const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage_mem);
+    const uint64_t step = (uint64_t)gridDim.x * P.rows_per_cta * P.cols;  // elements between a thread's iterations
+    if (threadIdx.x < LT_VM_MAX_PTR) {
+        S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], aligned_rows);
+        if (depth && P.io_stage[threadIdx.x] != 0xffu) S.soff[threadIdx.x] = P.io_stage[threadIdx.x] * LT_VM_STAGE_PIECE;
     }
+    if (threadIdx.x == 0) fill_loop(S.loop, P, 2, gridDim.x, row_blocks, step * 4, stage_base, aligned_rows);
     __syncthreads();
     link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
     __syncthreads();
@@ -723,7 +735,8 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
     rc.lane = threadIdx.x & 31u;
     const uint32_t sub = threadIdx.x >> P.group_log2;           // which row of this CTA's block of rows
     const uint32_t gl = threadIdx.x & (P.group - 1u);           // lane within the row's thread group
-    for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
+    // every thread of the CTA runs the same number of iterations (row reductions synchronise the CTA)
+    auto chunk_of = [&P, sub, gl](uint32_t rb) {
         Chunk ck;
         ck.row = rb * P.rows_per_cta + sub;
         ck.row_ok = ck.row < P.rows;
@@ -735,19 +748,42 @@ __global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ Lt
             nv = rem < (uint32_t)V ? (int)rem : V;
         }
         ck.nvalid = nv;
-        run_program<FLAV, true>(E, [&ck](uint32_t) { return ck; }, rb, ck, &rc, S, 0);
+        return ck;
+    };
+    if (blockIdx.x >= row_blocks) return;
+    const Chunk first = chunk_of(blockIdx.x);
+    const bool col_full = gl * V + V <= P.cols;
+    const uint32_t buf0 = stage_base + threadIdx.x * 16u;
+    if (depth) {
+        uint64_t e = first.flat0;
+        for (uint32_t d = 0; d < depth; ++d) {
+            if (col_full && e + V <= P.n) stage_chunk(S.loop, e, buf0 + d * buf_bytes);
+            cp_async_commit();
+            e += step;
+        }
+        cp_async_wait(depth - 1);
     }
+    run_program<FLAV, true>(E, chunk_of, blockIdx.x, first, &rc, S, buf0, col_full ? 0u : 2u);
+    if (depth) cp_async_wait(0);
 }
 
 template <int FLAV>
 __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
     __shared__ __align__(16) Staged S;
+    extern __shared__ __align__(16) unsigned char stage_mem[];
     stage_program(S, P);
-    if (threadIdx.x < LT_VM_MAX_PTR) S.ptr[threadIdx.x] = 0;
+    if (threadIdx.x < LT_VM_MAX_PTR) {
+        S.ptr[threadIdx.x] = 0;
+        if (P.stage_depth && P.io_stage[threadIdx.x] != 0xffu) S.soff[threadIdx.x] = P.io_stage[threadIdx.x] * LT_VM_STAGE_PIECE;
+    }
     __syncthreads();
     // linked once for all instances; an instance with an unaligned pointer has that slot flagged below and
-    // its accesses leave the vector path at run time
+    // its accesses leave the vector path at run time (staged slots are aligned in every instance)
     link_program(S, P.n_ins, P.io_dtype, nullptr, true);
+    const uint32_t depth = P.stage_depth;
+    const uint32_t buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
+    const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage_mem);
+    const uint32_t buf0 = stage_base + threadIdx.x * 16u;
     for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
         // instance that owns super-chunk sc: last i with super_prefix[i] <= sc
         uint32_t lo = 0, hi = P.n_inst;
@@ -756,24 +792,65 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
             if (P.super_prefix[mid] <= sc) lo = mid; else hi = mid;
         }
         const EnvM E{P, lo * P.n_slots};
-        __syncthreads();  // the previous super-chunk's pointers are no longer in use
-        if (threadIdx.x < P.n_slots) S.ptr[threadIdx.x] = flag_pointer(E.ptr(threadIdx.x), P.io_dtype[threadIdx.x], true);
-        __syncthreads();
         const uint32_t numel = P.numel[lo];
-        const uint32_t first = (sc - P.super_prefix[lo]) * (LT_EW_THREADS * LT_MULTI_SUB * V);
-#pragma unroll 1
-        for (int u = 0; u < LT_MULTI_SUB; ++u) {
-            const uint32_t e0 = first + (u * LT_EW_THREADS + threadIdx.x) * V;
-            if (e0 < numel) {
-                Chunk ck;
-                ck.flat0 = e0;
-                ck.row = 0;
-                ck.col0 = e0;
-                ck.row_ok = true;
-                const uint32_t rem = numel - e0;
-                ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
-                run_program<FLAV, false>(E, [&ck](uint32_t) { return ck; }, 0, ck, nullptr, S, 0);
+        // within the instance the super-chunk is a flat range of chunks, walked by the core with stride 256
+        const uint32_t chunk_first = (sc - P.super_prefix[lo]) * (LT_EW_THREADS * LT_MULTI_SUB);
+        const uint32_t chunks_all = (numel + V - 1) / V;
+        const uint32_t chunk_end = min(chunk_first + LT_EW_THREADS * LT_MULTI_SUB, chunks_all);
+        __syncthreads();  // the previous super-chunk's tables are no longer in use
+        if (threadIdx.x < P.n_slots) S.ptr[threadIdx.x] = flag_pointer(E.ptr(threadIdx.x), P.io_dtype[threadIdx.x], true);
+        if (threadIdx.x == 32) {
+            LtLoop &lp = S.loop;
+            lp.stride = LT_EW_THREADS;
+            lp.n_chunks = chunk_end;
+            lp.depth = depth;
+            lp.buf_bytes = buf_bytes;
+            lp.buf_total = depth * buf_bytes;
+            lp.stage_base = stage_base;
+            lp.inloop = 1;
+            lp.rowcol = 0;
+            lp.prefetch = depth ? 0u : 1u;
+            lp.pf_lo = LT_EW_THREADS * V * 4;
+            lp.pf_hi = 0;
+            lp.n4_lo = numel * 4u;
+            lp.n4_hi = numel >> 30;
+            uint32_t k = 0;
+            if (depth)
+                for (uint32_t s = 0; s < P.n_slots; ++s)
+                    if (P.io_stage[s] != 0xffu) {
+                        const uint64_t ptr = E.ptr(s);
+                        lp.stg[k].ptr_lo = (uint32_t)ptr;
+                        lp.stg[k].ptr_hi = (uint32_t)(ptr >> 32);
+                        lp.stg[k].dst = P.io_stage[s] * LT_VM_STAGE_PIECE;
+                        lp.stg[k].shift = 2u - (P.io_dtype[s] == LT_ST_BF16 ? 1u : P.io_dtype[s] == LT_ST_U8 ? 2u : 0u);
+                        ++k;
+                    }
+            lp.stg_n = k;
+        }
+        __syncthreads();
+        const uint32_t c0 = chunk_first + threadIdx.x;
+        if (c0 < chunk_end) {
+            if (depth) {
+                uint32_t c = c0;
+                for (uint32_t d = 0; d < depth; ++d) {
+                    if ((uint64_t)c * V + V <= numel) stage_chunk(S.loop, (uint64_t)c * V, buf0 + d * buf_bytes);
+                    cp_async_commit();
+                    c += LT_EW_THREADS;
+                }
+                cp_async_wait(depth - 1);
             }
+            auto chunk_of = [numel](uint32_t c) {
+                Chunk ck;
+                ck.flat0 = (uint64_t)c * V;
+                ck.row = 0;
+                ck.col0 = c * V;
+                ck.row_ok = true;
+                const uint32_t rem = numel - c * V;
+                ck.nvalid = rem < (uint32_t)V ? (int)rem : V;
+                return ck;
+            };
+            run_program<FLAV, false>(E, chunk_of, c0, chunk_of(c0), nullptr, S, buf0);
+            if (depth) cp_async_wait(0);
         }
     }
 }
@@ -792,14 +869,21 @@ cudaError_t lt_kernel_setup(size_t max_stage_bytes) {
     cudaError_t e = cudaFuncSetAttribute(lt_ew_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_ew_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_ew_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_multi_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_multi_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_row_kernel<0, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_row_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(lt_row_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_stage_bytes);
     return e;
 }
 
 cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream) {
+    const size_t dyn = (size_t)p.stage_depth * p.stage_pieces * LT_VM_STAGE_PIECE;
     if (threads <= 256) {
-        if (flavour == 0) lt_row_kernel<0, 256><<<grid, threads, 0, stream>>>(p);
-        else if (flavour == 1) lt_row_kernel<1, 256><<<grid, threads, 0, stream>>>(p);
-        else lt_row_kernel<2, 256><<<grid, threads, 0, stream>>>(p);
+        if (flavour == 0) lt_row_kernel<0, 256><<<grid, threads, dyn, stream>>>(p);
+        else if (flavour == 1) lt_row_kernel<1, 256><<<grid, threads, dyn, stream>>>(p);
+        else lt_row_kernel<2, 256><<<grid, threads, dyn, stream>>>(p);
     } else {
         if (flavour == 0) lt_row_kernel<0, 1024><<<grid, threads, 0, stream>>>(p);
         else if (flavour == 1) lt_row_kernel<1, 1024><<<grid, threads, 0, stream>>>(p);
@@ -809,9 +893,10 @@ cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsign
 }
 
 cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, cudaStream_t stream) {
-    if (flavour == 0) lt_multi_kernel<0><<<grid, LT_EW_THREADS, 0, stream>>>(p);
-    else if (flavour == 1) lt_multi_kernel<1><<<grid, LT_EW_THREADS, 0, stream>>>(p);
-    else lt_multi_kernel<2><<<grid, LT_EW_THREADS, 0, stream>>>(p);
+    const size_t dyn = (size_t)p.stage_depth * p.stage_pieces * LT_VM_STAGE_PIECE;
+    if (flavour == 0) lt_multi_kernel<0><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
+    else if (flavour == 1) lt_multi_kernel<1><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
+    else lt_multi_kernel<2><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
     return cudaGetLastError();
 }
 

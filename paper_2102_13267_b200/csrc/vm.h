@@ -24,13 +24,14 @@
 #define LT_VM_SM_SOFF 1184  // per-slot offset inside a staging buffer, or 0xFFFFFFFF
 #define LT_VM_SM_LOOP 1232  // struct LtLoop: constants of the chunk loop the PTX core runs by itself
 #define LT_VM_SM_STG 1296   // LtLoop::stg, the list of inputs staged by asynchronous copies
+#define LT_VM_SM_RED 1512   // 64 floats: cross-warp exchange of the row reductions (two alternating halves)
 #define LT_VM_STAGE_PIECE 4096  // bytes one 16-byte piece of a staged input takes per stage (256 threads x 16)
 
 #define LT_MULTI_MAX_INS 64
 #define LT_MULTI_MAX_INST 384   // instances (tensors) per multi-tensor launch
 #define LT_MULTI_MAX_PTRS 2816  // pointer-table entries per launch (instances x slots)
 #define LT_MULTI_MAX_SLOTS 8
-#define LT_MULTI_SUB 4          // chunks each thread runs per super-chunk
+#define LT_MULTI_SUB 8          // chunks each thread runs per super-chunk
 
 struct LtIns {
     uint32_t op;
@@ -101,13 +102,15 @@ static_assert(OP_WHERE_B + 4 * LT_VM_NSRC == OP_LDS, "opcode map");
 // Per-CTA constants of the chunk loop, in shared memory (read by the PTX core with broadcast loads).
 struct LtLoop {
     uint32_t stride, n_chunks, n_full, depth;            // chunks between a thread's iterations; total; complete ones; staging depth
-    uint32_t buf_bytes, buf_total, stage_base, inloop;   // one staging buffer; all of them; shared address of the first; 1 = core loops by itself
+    uint32_t buf_bytes, buf_total, stage_base, inloop;   // one staging buffer; all of them; shared address of the first; core loops by itself: 1 = over chunks (elementwise), 2 = over blocks of rows
     uint32_t rowcol, cpr, div_mul, div_sh1;
     uint32_t div_sh2, cols, prefetch, stg_n;             // prefetch: 1 = L2-prefetch the next chunk of full-class loads
     struct {
         uint32_t ptr_lo, ptr_hi, dst, shift;             // source pointer, offset inside a staging buffer, log2(element bytes)
     } stg[LT_VM_MAX_PTR];
     uint32_t pf_lo, pf_hi;                               // byte distance (4-byte elements) between a thread's iterations
+    uint32_t n4_lo, n4_hi;                               // 4 * number of elements
+    uint32_t group, inline_rows;                         // row kernel: threads per row; 1 = reductions / row index / random bits run in the core
 };
 
 // Kernel parameter block of the elementwise and row-reduction kernels.  It is passed by
@@ -140,6 +143,8 @@ struct LtMultiParams {
     LtIns ins[LT_MULTI_MAX_INS];
     uint32_t scal[LT_VM_MAX_SCAL];
     uint8_t io_dtype[LT_VM_MAX_PTR];
+    uint8_t io_stage[LT_VM_MAX_PTR];               // first staging piece of the slot, 0xFF = not staged (same for all instances)
+    uint32_t stage_depth, stage_pieces;
     uint32_t n_ins;
     uint32_t n_inst;
     uint32_t n_slots;
