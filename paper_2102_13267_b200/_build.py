@@ -28,13 +28,16 @@ def _stale(target: Path, deps) -> bool:
     return any(Path(d).stat().st_mtime > t for d in deps)
 
 
+EXTRA_NVCC = os.environ.get("LT_NVCC_FLAGS", "").split()  # e.g. -DLT_EW_MIN_BLOCKS=2 for tuning experiments
+
+
 def _compile(src: str) -> Path:
     path = CSRC / src
     obj = OBJ / (src + ".o")
     deps = [path] + [CSRC / h for h in HEADERS]
     if _stale(obj, deps):
         if src.endswith(".cu"):
-            cmd = [str(CUDA_HOME / "bin" / "nvcc"), *NVCC_FLAGS, "-c", str(path), "-o", str(obj)]
+            cmd = [str(CUDA_HOME / "bin" / "nvcc"), *NVCC_FLAGS, *EXTRA_NVCC, "-c", str(path), "-o", str(obj)]
         else:
             cmd = ["g++", *CXX_FLAGS, "-c", str(path), "-o", str(obj)]
         subprocess.check_call(cmd)

@@ -138,8 +138,12 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     uint32_t depth = (96u * 1024u + (uint32_t)c->occ_multi * buf - 1) / ((uint32_t)c->occ_multi * buf);
                     depth = std::min(4u, std::max(2u, depth));
                     while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
-                    if (depth >= 2) P.stage_depth = depth;
-                    else for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                    // two buffers (one chunk of look-ahead) measured slower than L2 prefetch: need three
+                    if (depth >= 3) P.stage_depth = depth;
+                    else {
+                        P.stage_pieces = 0;
+                        for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                    }
                 }
             }
             if (!dry) {
@@ -181,8 +185,12 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     uint32_t depth = (96u * 1024u + occ * buf - 1) / (occ * buf);
                     depth = std::min(4u, std::max(2u, depth));
                     while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
-                    if (depth >= 2) P.stage_depth = depth;
-                    else for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                    // two buffers (one chunk of look-ahead) measured slower than L2 prefetch: need three
+                    if (depth >= 3) P.stage_depth = depth;
+                    else {
+                        P.stage_pieces = 0;
+                        for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
+                    }
                 }
             }
             if (L.kind == K_EW) {
