@@ -287,8 +287,8 @@ def slot_address(cls: int, sz: int, prefetch: bool):
     lines.append("add.u64 ptr, ptr, offs;")
     if prefetch and cls == 0:
         # pull this thread's next chunk of the same input into L2 while the current one is processed
-        lines += [f"shr.u64 offs, {PF4}, {sz};" if sz else f"mov.b64 offs, {PF4};", "add.u64 offs, ptr, offs;",
-                  "@pnext prefetch.global.L2 [offs];"]
+        lines += [f"@pnext ld.shared.b64 offs, [{SMB}+{SM_PF}];"] + ([f"@pnext shr.u64 offs, offs, {sz};"] if sz else []) + [
+                  "@pnext add.u64 offs, ptr, offs;", "@pnext prefetch.global.L2 [offs];"]
     return lines
 
 
@@ -374,7 +374,6 @@ def entry_code():
     return [f"and.b32 r0, {TAIL}, 1;", "setp.ne.u32 ptail, r0, 0;",
             f"ld.shared.v2.b32 {{r0, r1}}, [{SMB}+{L}];",            # stride, n_chunks
             f"ld.shared.b32 r2, [{SMB}+{L + 56}];",                   # prefetch enabled
-            f"ld.shared.b64 pf4, [{SMB}+{SM_PF}];",
             f"sub.u32 r1, r1, {CHUNK};", "setp.gt.u32 pnext, r1, r0;", "setp.ne.u32 p, r2, 0;",
             "and.pred pnext, pnext, p;", "not.pred p, ptail;", "and.pred pnext, pnext, p;"]
 
@@ -388,6 +387,7 @@ def end_body():
         "setp.eq.u32 p, r7, 0;", "@p bra L_ESC;",
         f"ld.shared.v4.b32 {{r0, r1, r2, r3}}, [{SMB}+{L}];",          # stride, n_chunks, n_full, depth
         f"ld.shared.b64 d2, [{SMB}+{SM_N4}];",                          # 4 * elements
+        f"ld.shared.b64 pf4, [{SMB}+{SM_PF}];",                         # bytes (4-byte view) between a thread's iterations
         "setp.eq.u32 pq, r3, 0;", "@pq bra L_ADV;",
         # the chunk `depth` iterations ahead starts depth * pf4 bytes (4-byte view) further; staged if complete
         "cvt.u64.u32 d1, r3;", "mul.lo.u64 d1, d1, pf4;", f"add.u64 d0, {OFF4}, d1;", "add.u64 d1, d0, 32;",

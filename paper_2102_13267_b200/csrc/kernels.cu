@@ -707,7 +707,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
 }
 
 template <int FLAV, int MAXT>
-__global__ void __launch_bounds__(MAXT) lt_row_kernel(const __grid_constant__ LtKParams P) {
+__global__ void __launch_bounds__(MAXT, MAXT == 256 ? LT_EW_MIN_BLOCKS : 1) lt_row_kernel(const __grid_constant__ LtKParams P) {
     __shared__ __align__(16) Staged S;
     extern __shared__ __align__(16) unsigned char stage_mem[];
     const EnvK E{P};
