@@ -15,6 +15,7 @@ sum over ranks divided by the slowest rank's time.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import math
 import os
@@ -107,13 +108,25 @@ def measured_peak() -> tuple[float, str]:
         return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
 
 
+# DRAM bytes of one launch of the dominant kernel on this workload, from the ncu capture summarised in
+# profiles/lt_ew_kernel_c2_mlp_epilogue.md, with the hash of the kernel sources it was taken on.
+NCU_TRAFFIC = {"bytes": 167266304, "sources_sha256": "5d4737b8f6cde80a9b96105bd21bd32435764e451fafee8e4bc6dab403cdc2ab"}
+KERNEL_SOURCES = ("paper_2102_13267_b200/csrc/kernels.cu", "paper_2102_13267_b200/csrc/vm_core.inc",
+                  "paper_2102_13267_b200/csrc/vm.h")
+
+
+def kernel_sources_sha256() -> str:
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def ncu_traffic() -> float | None:
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if it is current."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+    """Measured DRAM bytes per launch, or None once the kernel sources differ from the profiled ones."""
     try:
-        with open(path) as f:
-            rec = json.load(f)
-        return float(rec[WORKLOAD]["dram_bytes_per_launch"])
+        return float(NCU_TRAFFIC["bytes"]) if kernel_sources_sha256() == NCU_TRAFFIC["sources_sha256"] else None
     except Exception:
         return None
 
