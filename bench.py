@@ -199,6 +199,23 @@ def run_reference(args) -> None:
 
 
 # ------------------------------------------------------------------------------ our arm
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time: the replicas share no data, so the job's time is the maximum."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gbs(bytes_per_rank_step: int, steps: int, world: int, ms: float) -> float:
+    """Whole-job GB/s: every rank moved bytes_per_rank_step per step, in the slowest rank's time."""
+    return world * bytes_per_rank_step * steps / (ms / 1e3) / 1e9
+
+
 def run_ours(args) -> None:
     import torch
     import torch.distributed as dist
@@ -248,12 +265,7 @@ def run_ours(args) -> None:
             fn(i)
         e1.record()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -269,7 +281,7 @@ def run_ours(args) -> None:
     ctx.set_kernel_timing(False)
     st = ctx.stats()
     clocks = sampler.stop(w0, w1) if sampler else None
-    value = world * nbytes * args.steps / (ms / 1e3) / 1e9
+    value = aggregate_gbs(nbytes, args.steps, world, ms)
 
     # ---- end to end through the C ABI with host buffers: H2D of the inputs and D2H of the result every step
     e2e_steps = max(3, min(args.steps, 30))
@@ -286,7 +298,7 @@ def run_ours(args) -> None:
     for i in range(3):
         e2e_step(i)
     e2e_ms = timed(e2e_steps, e2e_step)
-    e2e_value = world * nbytes * e2e_steps / (e2e_ms / 1e3) / 1e9
+    e2e_value = aggregate_gbs(nbytes, e2e_steps, world, e2e_ms)
 
     if rank != 0:
         if world > 1:
