@@ -29,6 +29,8 @@ def opcodes() -> dict[str, int]:
     """Opcode bases and indices, read from vm.h so the two cannot drift apart."""
     text = (HERE / "vm.h").read_text()
     vals: dict[str, int] = {}
+    for m in re.finditer(r"#define\s+(LT_VM_\w+)\s+(\d+)", text):
+        vals[m.group(1)] = int(m.group(2))
     for block in re.findall(r"enum\s*\{(.*?)\};", text, flags=re.S):
         block = re.sub(r"/\*.*?\*/", "", block, flags=re.S)
         block = re.sub(r"//[^\n]*", "", block)
@@ -50,12 +52,13 @@ def opcodes() -> dict[str, int]:
 
 
 OPS = opcodes()
-NSRC = OPS["LT_VM_NSRC"]
+NSRC, NT, ND = OPS["LT_VM_NSRC"], OPS["LT_VM_NT"], OPS["LT_VM_ND"]
 
 A = [f"%{i}" for i in range(4)]
-T = [[f"%{4 + 4 * k + j}" for j in range(4)] for k in range(4)]
-REG = T + [A]  # destination index 0..3 = temporaries, 4 = ACC
-PC, EOP, EIMM, CHUNK, OFF4, COFF4, TAIL, STG, SMB = "%20", "%21", "%22", "%23", "%24", "%25", "%26", "%27", "%28"
+T = [[f"%{4 + 4 * k + j}" for j in range(4)] for k in range(NT)]
+REG = T + [A]  # destination index < NT = temporaries, NT = ACC
+_o = 4 + 4 * NT
+PC, EOP, EIMM, CHUNK, OFF4, COFF4, TAIL, STG, SMB = (f"%{_o + i}" for i in range(9))
 PF4 = "pf4"
 SM_SCAL, SM_PTR, SM_SOFF, STAGE_PIECE, SM_LOOP, SM_STG = (OPS[k] for k in ("LT_VM_SM_SCAL", "LT_VM_SM_PTR", "LT_VM_SM_SOFF", "LT_VM_STAGE_PIECE", "LT_VM_SM_LOOP", "LT_VM_SM_STG"))
 SM_PF = SM_STG + 16 * OPS["LT_VM_MAX_PTR"]
@@ -92,19 +95,12 @@ class Src:
 
     def __init__(self, kind: int):
         self.kind = kind
-        if kind < 4:
+        if kind < NT:
             self.pre = []
             self.pairs = T[kind]
-            self._lanes = None
         else:
             self.pre = ["shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b32 sv, [sa+{SM_SCAL}];", "mov.b64 ss, {sv, sv};"]
             self.pairs = ["ss"] * 4
-
-    def lanes(self, out):
-        """PTX that makes the operand available lane by lane; returns (lines, lane names)."""
-        if self.kind < 4:
-            return unpack(self.pairs, Y), Y
-        return [], ["sv"] * 8
 
 
 def div_ins(flavour: str) -> str:
@@ -120,7 +116,7 @@ def pairwise(a_pairs, src, fmt_lines):
         lines.append(f"mov.b64 {{x0, x1}}, {a_pairs[j]};")
         if src is None:
             ys = (None, None)
-        elif src.kind < 4:
+        elif src.kind < NT:
             lines.append(f"mov.b64 {{y0, y1}}, {src.pairs[j]};")
             ys = ("y0", "y1")
         else:
@@ -171,7 +167,7 @@ def where_body(m: int, src: Src, variant_b: bool):
     lines = list(src.pre)
     for j in range(4):
         lines += [f"mov.b64 {{x0, x1}}, {A[j]};", f"mov.b64 {{m0, m1}}, {T[m][j]};"]
-        if src.kind < 4:
+        if src.kind < NT:
             lines.append(f"mov.b64 {{y0, y1}}, {src.pairs[j]};")
             ys = ("y0", "y1")
         else:
@@ -258,22 +254,6 @@ def unary_body(name: str, flavour: str):
                       f"fma.rn.f32x2 {a}, {a}, {g}, {a};"]
         return lines
     raise KeyError(name)
-
-
-def cvt_bf16(d: int):
-    P = REG[d]
-    lines = [f"mov.b64 {{w0, w1}}, {P[0]};", f"mov.b64 {{w2, w3}}, {P[1]};"]
-    for j in (3, 2, 1, 0):
-        lines += [f"shl.b32 x0, w{j}, 16;", f"and.b32 x1, w{j}, 0xFFFF0000;", f"mov.b64 {P[j]}, {{x0, x1}};"]
-    return lines
-
-
-def cvt_u8(d: int):
-    P = REG[d]
-    lines = [f"mov.b64 {{w0, w1}}, {P[0]};"]
-    for i in range(8):
-        lines.append(f"bfe.u32 {X[i]}, w{i // 4}, {8 * (i % 4)}, 8;")
-    return lines + pack(P, X)
 
 
 def slot_address(cls: int, sz: int, prefetch: bool):
@@ -507,14 +487,11 @@ def build(flavour: str) -> list[str]:
         bodies[OPS["OP_RED_SUM"] + kind] = red_body(kind)
     bodies[OPS["OP_IOTA_ROW"]] = iota_row_body()
     bodies[OPS["OP_PHILOX"]] = philox_body()
-    for k in range(4):
+    for k in range(NT):
         bodies[OPS["OP_MOV_T_ACC"] + k] = [f"mov.b64 {T[k][j]}, {A[j]};" for j in range(4)]
         bodies[OPS["OP_MOV_ACC_T"] + k] = [f"mov.b64 {A[j]}, {T[k][j]};" for j in range(4)]
-    s = Src(4)
+    s = Src(NT)
     bodies[OPS["OP_MOV_ACC_S"]] = s.pre + [f"mov.b64 {a}, ss;" for a in A]
-    for d in range(5):
-        bodies[OPS["OP_CVT_BF16"] + d] = cvt_bf16(d)
-        bodies[OPS["OP_CVT_U8"] + d] = cvt_u8(d)
     bodies[OPS["OP_IOTA_COL"]] = ([f"shr.u32 w0, {COFF4}, 2;"] + [f"add.u32 {X[i]}, w0, {i};" for i in range(8)] + pack(A, X))
     for name in ("OP_U_NEG", "OP_U_ABS", "OP_U_RELU", "OP_U_EXP", "OP_U_LOG", "OP_U_TANH", "OP_U_SQRT", "OP_U_RSQRT",
                  "OP_U_RECIP", "OP_U_SQUARE", "OP_U_SIGMOID", "OP_U_GELU", "OP_U_RBF16", "OP_U_INEG", "OP_U_IABS",
@@ -523,10 +500,10 @@ def build(flavour: str) -> list[str]:
         if b is not None:
             bodies[OPS[name]] = b
     for sz in range(3):
-        for d in range(5):
+        for d in range(ND):
             for cls in range(2):
-                bodies[OPS["OP_LDG"] + (sz * 2 + cls) * 5 + d] = ldg_body(sz, cls, d)
-            bodies[OPS["OP_LDS"] + sz * 5 + d] = lds_body(sz, d)
+                bodies[OPS["OP_LDG"] + (sz * 2 + cls) * ND + d] = ldg_body(sz, cls, d)
+            bodies[OPS["OP_LDS"] + sz * ND + d] = lds_body(sz, d)
         bodies[OPS["OP_STG"] + sz] = stg_body(sz)
         for k in range(OPS["F2M_COUNT"]):
             for cls in range(2):
@@ -538,10 +515,10 @@ def build(flavour: str) -> list[str]:
     for idx in range(OPS["I2_COUNT"]):
         for k in range(NSRC):
             bodies[OPS["OP_I2"] + idx * NSRC + k] = i2_body(idx, Src(k))
-    for idx in range(18):
+    for idx in range(OPS["CMP_COUNT"]):
         for k in range(NSRC):
             bodies[OPS["OP_CMP"] + idx * NSRC + k] = cmp_body(idx, Src(k))
-    for m in range(4):
+    for m in range(NT):
         for k in range(NSRC):
             bodies[OPS["OP_WHERE_A"] + m * NSRC + k] = where_body(m, Src(k), False)
             bodies[OPS["OP_WHERE_B"] + m * NSRC + k] = where_body(m, Src(k), True)
@@ -583,11 +560,11 @@ def as_macro(name: str, lines: list[str]) -> str:
 
 def main() -> None:
     text = ("// Generated by gen_vm_core.py from vm.h -- do not edit.\n"
-            "// Operands: %0-%3 ACC, %4-%19 T0..T3 (f32x2 pairs); %20 pc (shared address); %21 escape opcode;\n"
-            "// %22 escape immediate; %23 chunk index; %24 chunk byte offset for 4-byte elements; %25 column byte\n"
-            "// offset; %26 ragged-chunk flag; %27 shared address of this thread's current staging buffer;\n"
-            "// %28 shared address of the staged block (program, immediates, pointers, loop constants).\n"
-            "// %23-%27 are updated by the core when it moves to the next chunk by itself (OP_END).\n"
+            f"// Operands: %0-%3 ACC, then the temporaries (f32x2 pairs); {PC} pc (shared address); {EOP} escape opcode;\n"
+            f"// {EIMM} escape immediate; {CHUNK} chunk index; {OFF4} chunk byte offset for 4-byte elements; {COFF4} column\n"
+            f"// byte offset; {TAIL} chunk flags; {STG} shared address of this thread's current staging buffer;\n"
+            f"// {SMB} shared address of the staged block (program, immediates, pointers, loop constants).\n"
+            f"// {CHUNK}-{STG} are updated by the core when it moves to the next chunk by itself (OP_END).\n"
             "#pragma once\n\n")
     text += "\n".join(as_macro(f"LT_VM_CORE_{fl.upper()}", build(fl)) for fl in ("fast", "precise", "ieee"))
     (HERE / "vm_core.inc").write_text(text)

@@ -19,6 +19,8 @@
 namespace {
 
 constexpr int V = LT_VM_V;
+constexpr int NT = LT_VM_NT;  // R[0..NT-1] are the temporaries, R[NT] is ACC
+static_assert(LT_VM_NT == 3 && LT_VM_ND == LT_VM_NT + 1, "the asm operand list below names three temporaries");
 
 #ifndef LT_EW_MIN_BLOCKS
 #define LT_EW_MIN_BLOCKS 3
@@ -429,10 +431,9 @@ __device__ __forceinline__ void pairs_of(const float (&f)[V], uint64_t (&p)[4]) 
 }
 
 #define LT_VM_OPERANDS                                                                                              \
-    : "+l"(R[4][0]), "+l"(R[4][1]), "+l"(R[4][2]), "+l"(R[4][3]), "+l"(R[0][0]), "+l"(R[0][1]), "+l"(R[0][2]),      \
+    : "+l"(R[NT][0]), "+l"(R[NT][1]), "+l"(R[NT][2]), "+l"(R[NT][3]), "+l"(R[0][0]), "+l"(R[0][1]), "+l"(R[0][2]),  \
       "+l"(R[0][3]), "+l"(R[1][0]), "+l"(R[1][1]), "+l"(R[1][2]), "+l"(R[1][3]), "+l"(R[2][0]), "+l"(R[2][1]),      \
-      "+l"(R[2][2]), "+l"(R[2][3]), "+l"(R[3][0]), "+l"(R[3][1]), "+l"(R[3][2]), "+l"(R[3][3]), "+r"(pc),           \
-      "=r"(eop), "=r"(eimm)                                                                                         \
+      "+l"(R[2][2]), "+l"(R[2][3]), "+r"(pc), "=r"(eop), "=r"(eimm)                                                 \
       , "+r"(c), "+l"(off4), "+r"(coff4), "+r"(tail), "+r"(stg)                                                     \
     : "r"(smem_s)                                                                                                   \
     : "memory"
@@ -454,7 +455,7 @@ template <int FLAV, bool ROW, class Env, class ChunkOf>
 __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint32_t c, const Chunk &first, RowCtx *rc,
                                             const Staged &S, uint32_t stg, uint32_t flags = 0) {
     const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(&S);
-    uint64_t R[5][4];  // not initialised: a program writes every register before it reads it
+    uint64_t R[NT + 1][4];  // not initialised: a program writes every register before it reads it
     uint32_t pc = smem_s;
     uint64_t off4 = first.flat0 << 2;
     uint32_t coff4 = first.col0 << 2;
@@ -468,35 +469,34 @@ __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint
         if (eop == OP_END) break;
         const Chunk ck = chunk_of(c);
         float f[V];
-        const bool is_ld = (eop >= OP_LD && eop < OP_STG) || (eop >= OP_LDS && eop < OP_F2M);
-        const bool is_f2m = eop >= OP_F2M && eop < OP_LIMIT;
+        const bool is_ld = eop >= OP_LD && eop < OP_STG;
+        const bool is_f2m = eop >= OP_F2M && eop < OP_F2;
         if (is_ld || is_f2m) {
             // a load that was not linked to a vector path (unaligned pointer, broadcast class), or one
             // that met a ragged chunk: element-wise load, then widen
-            const bool staged = (eop >= OP_LDS && eop < OP_F2M) || eop >= OP_F2MS;
+            const bool staged = (eop >= OP_LDS && eop < OP_STG) || eop >= OP_F2MS;
             const uint32_t slot = slot_of(S, staged, eimm);
             load_raw(f, E, slot, ck);
             widen(f, E.dtype(slot));
             if (is_ld) {
-                const uint32_t d = eop < OP_LDG ? eop - OP_LD : eop < OP_STG ? (eop - OP_LDG) % 5u : (eop - OP_LDS) % 5u;
+                const uint32_t d = eop < OP_LDG ? eop - OP_LD : eop < OP_LDS ? (eop - OP_LDG) % LT_VM_ND : (eop - OP_LDS) % LT_VM_ND;
                 if (d == 0) pairs_of(f, R[0]);
                 else if (d == 1) pairs_of(f, R[1]);
                 else if (d == 2) pairs_of(f, R[2]);
-                else if (d == 3) pairs_of(f, R[3]);
-                else pairs_of(f, R[4]);
+                else pairs_of(f, R[NT]);
             } else {
                 const uint32_t k = eop < OP_F2MG ? eop - OP_F2M : eop < OP_F2MS ? (eop - OP_F2MG) / 6u : (eop - OP_F2MS) / 3u;
                 float a[V];
-                lanes_of(R[4], a);
+                lanes_of(R[NT], a);
 #pragma unroll
                 for (int i = 0; i < V; ++i)
                     a[i] = k == F2M_ADD ? __fadd_rn(a[i], f[i]) : k == F2M_SUB ? __fsub_rn(a[i], f[i])
                          : k == F2M_RSUB ? __fsub_rn(f[i], a[i]) : __fmul_rn(a[i], f[i]);
-                pairs_of(a, R[4]);
+                pairs_of(a, R[NT]);
             }
             continue;
         }
-        lanes_of(R[4], f);
+        lanes_of(R[NT], f);
         if (eop == OP_ST || (eop >= OP_STG && eop < OP_STG + 3)) {
             store_chunk(f, E, eimm, ck);
             continue;
@@ -526,7 +526,7 @@ __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint
                 else if (eop == OP_U_GELU) f[i] = un<OP_U_GELU, false>(f[i]);
             }
         }
-        pairs_of(f, R[4]);
+        pairs_of(f, R[NT]);
     }
 }
 
@@ -552,7 +552,7 @@ __device__ __forceinline__ void link_program(Staged &S, uint32_t n_ins, const ui
     for (uint32_t i = threadIdx.x; i < n_ins; i += blockDim.x) {
         LtIns in = S.ins[i];
         const uint32_t op = in.op, slot = in.imm;
-        const bool ld = op >= OP_LD && op < OP_LD + 5, st = op == OP_ST, f2m = op >= OP_F2M && op < OP_F2M + F2M_COUNT;
+        const bool ld = op >= OP_LD && op < OP_LD + LT_VM_ND, st = op == OP_ST, f2m = op >= OP_F2M && op < OP_F2M + F2M_COUNT;
         if (!(ld || st || f2m)) continue;
         const uint32_t dt = io_dtype[slot], cls = multi ? (uint32_t)LT_CLS_FULL : (uint32_t)io_class[slot];
         if ((S.ptr[slot] >> 63) || cls > LT_CLS_COLVEC) continue;
@@ -560,8 +560,8 @@ __device__ __forceinline__ void link_program(Staged &S, uint32_t n_ins, const ui
         const bool staged = S.soff[slot] != 0xffffffffu;
         if (ld) {
             const uint32_t d = op - OP_LD;
-            if (staged) { in.op = OP_LDS + sz * 5 + d; in.imm = S.soff[slot]; }
-            else in.op = OP_LDG + (sz * 2 + cls) * 5 + d;
+            if (staged) { in.op = OP_LDS + sz * LT_VM_ND + d; in.imm = S.soff[slot]; }
+            else in.op = OP_LDG + (sz * 2 + cls) * LT_VM_ND + d;
         } else if (f2m) {
             const uint32_t k = op - OP_F2M;
             if (staged) { in.op = OP_F2MS + k * 3 + sz; in.imm = S.soff[slot]; }

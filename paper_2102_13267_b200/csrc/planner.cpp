@@ -226,7 +226,7 @@ struct CodeGen {
             widen_temp(temp_of[v]);
             emit_ins((uint16_t)(OP_MOV_ACC_T + temp_of[v]));
         } else if (is_input((uint32_t)v)) {
-            emit_load(4, (uint32_t)v);
+            emit_load(LT_VM_NT, (uint32_t)v);
         } else {
             ok = false;
             return;
@@ -617,7 +617,7 @@ uint64_t io_bytes(const Group &g, const IoRef &io) {
 }
 
 const char *src_name(int s) {
-    static const char *n[] = {"T0", "T1", "T2", "T3", "S"};
+    static const char *n[] = {"T0", "T1", "T2", "T3", "T4"};
     return n[s];
 }
 
@@ -631,8 +631,8 @@ std::string disasm(const LtIns &in) {
     if (op >= OP_MOV_T_ACC && op < OP_MOV_ACC_T) snprintf(buf, sizeof(buf), "T%d = ACC", op - OP_MOV_T_ACC);
     else if (op >= OP_MOV_ACC_T && op < OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = T%d", op - OP_MOV_ACC_T);
     else if (op == OP_MOV_ACC_S) snprintf(buf, sizeof(buf), "ACC = S%u", in.imm);
-    else if (op >= OP_LD && op < OP_LD + 5) {
-        if (op - OP_LD < 4) snprintf(buf, sizeof(buf), "T%d = load p%u", op - OP_LD, in.imm);
+    else if (op >= OP_LD && op < OP_LD + LT_VM_ND) {
+        if (op - OP_LD < LT_VM_NT) snprintf(buf, sizeof(buf), "T%d = load p%u", op - OP_LD, in.imm);
         else snprintf(buf, sizeof(buf), "ACC = load p%u", in.imm);
     } else if (op >= OP_F2M && op < OP_F2M + F2M_COUNT) {
         static const char *f[] = {"add", "sub", "rsub", "mul"};
@@ -657,7 +657,7 @@ std::string disasm(const LtIns &in) {
         static const char *f[] = {"add", "sub", "rsub", "mul", "and", "or", "xor", "max.s", "min.s", "max.u", "min.u"};
         int idx = (op - OP_I2) / LT_VM_NSRC, s = (op - OP_I2) % LT_VM_NSRC;
         snprintf(buf, sizeof(buf), "ACC = i.%s ACC, %s", f[idx], src_txt(s).c_str());
-    } else if (op >= OP_CMP && op < OP_CMP + 18 * LT_VM_NSRC) {
+    } else if (op >= OP_CMP && op < OP_CMP + CMP_COUNT * LT_VM_NSRC) {
         static const char *cc[] = {"gt", "ge", "lt", "le", "eq", "ne"};
         static const char *ty[] = {"f", "s", "u"};
         int idx = (op - OP_CMP) / LT_VM_NSRC, s = (op - OP_CMP) % LT_VM_NSRC;
@@ -1064,7 +1064,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                         int ld_pos = -1, st_pos = -1;
                         for (size_t q = 0; q < g.ins.size(); ++q) {
                             const LtIns &in = g.ins[q];
-                            const bool loads = (in.op >= OP_LD && in.op < OP_LD + 5) || (in.op >= OP_F2M && in.op < OP_F2M + F2M_COUNT);
+                            const bool loads = (in.op >= OP_LD && in.op < OP_LD + LT_VM_ND) || (in.op >= OP_F2M && in.op < OP_F2M + F2M_COUNT);
                             if (loads && in.imm == rd.second && ld_pos < 0) ld_pos = (int)q;
                             if (in.op == OP_ST && in.imm == s) st_pos = (int)q;
                         }

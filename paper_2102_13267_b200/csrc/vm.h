@@ -12,9 +12,10 @@
 
 #define LT_VM_V 8          // lanes per chunk
 #define LT_EW_THREADS 256  // CTA size of the elementwise and multi-tensor kernels
-#define LT_VM_NT 4         // temporaries T0..T3
-#define LT_VM_NSRC 5       // operand sources of two-operand opcodes: T0..T3, S (broadcast immediate)
-#define LT_VM_SRC_S 4
+#define LT_VM_NT 3         // temporaries T0..T2 (a fourth one costs 8 registers per thread, i.e. a resident block per SM)
+#define LT_VM_ND 4         // load destinations: the temporaries, then ACC
+#define LT_VM_NSRC 4       // operand sources of two-operand opcodes: the temporaries, then S (broadcast immediate)
+#define LT_VM_SRC_S 3
 #define LT_VM_MAX_INS 118     // the program is followed by an END and one padding slot
 #define LT_VM_MAX_PTR 12
 #define LT_VM_MAX_SCAL 32
@@ -43,13 +44,18 @@ enum { LT_CLS_FULL = 0, LT_CLS_COLVEC = 1, LT_CLS_ROWVEC = 2, LT_CLS_SCALAR = 3 
 // storage dtypes (same numbering as lt_dtype)
 enum { LT_ST_F32 = 0, LT_ST_BF16 = 1, LT_ST_U8 = 2, LT_ST_I32 = 3, LT_ST_U32 = 4 };
 
+enum { F2_ADD = 0, F2_SUB, F2_RSUB, F2_MUL, F2_DIV, F2_RDIV, F2_MAX, F2_MIN, F2_COUNT };
+enum { I2_ADD = 0, I2_SUB, I2_RSUB, I2_MUL, I2_AND, I2_OR, I2_XOR, I2_MAXS, I2_MINS, I2_MAXU, I2_MINU, I2_COUNT };
+// compare index = type * 6 + cc ; type 0 f32, 1 signed, 2 unsigned ; cc: GT GE LT LE EQ NE
+enum { CC_GT = 0, CC_GE, CC_LT, CC_LE, CC_EQ, CC_NE };
+enum { CMP_COUNT = 18 };
+enum { F2M_ADD = 0, F2M_SUB, F2M_RSUB, F2M_MUL, F2M_COUNT };
+
 enum {
     OP_END = 0,
-    OP_MOV_T_ACC = 1,    // +k : T[k] = ACC
-    OP_MOV_ACC_T = 5,    // +k : ACC = T[k]
-    OP_MOV_ACC_S = 9,    // ACC = broadcast(imm slot)
-    OP_CVT_BF16 = 10,    // +d : widen the raw bf16 chunk held in register d (0..3 = T0..T3, 4 = ACC) to f32 lanes
-    OP_CVT_U8 = 15,      // +d : widen a raw u8 chunk to 32-bit lanes
+    OP_MOV_T_ACC = 1,                        // +k : T[k] = ACC
+    OP_MOV_ACC_T = OP_MOV_T_ACC + LT_VM_NT,  // +k : ACC = T[k]
+    OP_MOV_ACC_S = OP_MOV_ACC_T + LT_VM_NT,  // ACC = broadcast(imm slot)
     OP_ST = 20,          // store ACC to pointer slot imm, any class and dtype (handled outside the PTX core)
     OP_IOTA_COL = 21,    // ACC = column index of each lane (i32)
     OP_IOTA_ROW = 22,    // ACC = (row / scal[imm]) % scal[imm+1] (i32), same in every lane
@@ -67,37 +73,23 @@ enum {
     // pointers into a vector-path opcode the PTX core executes itself -- ...G: 128-bit global access,
     // ...S: read from the thread's staging buffer (immediate = byte offset in the buffer).  Slots that
     // cannot use vector accesses keep the generic opcode, which the C++ around the core handles.
-    // size 0/1/2 = 4/2/1-byte elements; class 0 = full, 1 = column vector; d 0..3 = T0..T3, 4 = ACC.
-    OP_LD = 51,          // +d
-    OP_LDG = 56,         // +(size * 2 + class) * 5 + d
-    OP_STG = 86,         // +size : vector store of ACC to a full-class slot
+    // size 0/1/2 = 4/2/1-byte elements; class 0 = full, 1 = column vector; d < LT_VM_NT = T[d], else ACC.
+    OP_LD = 51,                              // +d
+    OP_LDG = OP_LD + LT_VM_ND,               // +(size * 2 + class) * LT_VM_ND + d
+    OP_LDS = OP_LDG + 6 * LT_VM_ND,          // +size * LT_VM_ND + d : staged load
+    OP_STG = OP_LDS + 3 * LT_VM_ND,          // +size : vector store of ACC to a full-class slot
+    OP_F2M = OP_STG + 3,                     // +k : ACC = ACC (op) widened chunk of slot imm; k: see F2M_*
+    OP_F2MG = OP_F2M + F2M_COUNT,            // +(k * 3 + size) * 2 + class
+    OP_F2MS = OP_F2MG + F2M_COUNT * 6,       // +k * 3 + size
     // two-operand families: opcode = base + index * LT_VM_NSRC + source
-    OP_F2 = 96,          // ACC = ACC (op) src, f32: see F2_*
-    OP_I2 = 136,         // integer: see I2_*
-    OP_CMP = 192,        // ACC = (ACC cmp src) ? 1 : 0 : see CC_*
-    OP_WHERE_A = 288,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? ACC : src
-    OP_WHERE_B = 308,    // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? src : ACC
-    OP_LDS = 328,        // +size * 5 + d : staged load
-    OP_F2M = 343,        // +k : ACC = ACC (op) widened chunk of slot imm; k: see F2M_*
-    OP_F2MG = 347,       // +(k * 3 + size) * 2 + class
-    OP_F2MS = 371,       // +k * 3 + size
-    OP_LIMIT = 383
+    OP_F2 = OP_F2MS + F2M_COUNT * 3,         // ACC = ACC (op) src, f32: see F2_*
+    OP_I2 = OP_F2 + F2_COUNT * LT_VM_NSRC,   // integer: see I2_*
+    OP_CMP = OP_I2 + I2_COUNT * LT_VM_NSRC,  // ACC = (ACC cmp src) ? 1 : 0 : see CC_*
+    OP_WHERE_A = OP_CMP + CMP_COUNT * LT_VM_NSRC,     // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? ACC : src
+    OP_WHERE_B = OP_WHERE_A + LT_VM_NT * LT_VM_NSRC,  // + m * LT_VM_NSRC + src : ACC = T[m] != 0 ? src : ACC
+    OP_LIMIT = OP_WHERE_B + LT_VM_NT * LT_VM_NSRC
 };
-enum { F2M_ADD = 0, F2M_SUB, F2M_RSUB, F2M_MUL, F2M_COUNT };
-
-enum { F2_ADD = 0, F2_SUB, F2_RSUB, F2_MUL, F2_DIV, F2_RDIV, F2_MAX, F2_MIN, F2_COUNT };
-enum { I2_ADD = 0, I2_SUB, I2_RSUB, I2_MUL, I2_AND, I2_OR, I2_XOR, I2_MAXS, I2_MINS, I2_MAXU, I2_MINU, I2_COUNT };
-// compare index = type * 6 + cc ; type 0 f32, 1 signed, 2 unsigned ; cc: GT GE LT LE EQ NE
-enum { CC_GT = 0, CC_GE, CC_LT, CC_LE, CC_EQ, CC_NE };
-
-static_assert(OP_LDG + 30 == OP_STG && OP_STG + 3 <= OP_F2, "opcode map");
-static_assert(OP_LDS + 15 == OP_F2M && OP_F2M + F2M_COUNT == OP_F2MG && OP_F2MG + F2M_COUNT * 6 == OP_F2MS &&
-                  OP_F2MS + F2M_COUNT * 3 == OP_LIMIT,
-              "opcode map");
-static_assert(OP_F2 + F2_COUNT * LT_VM_NSRC == OP_I2, "opcode map");
-static_assert(OP_I2 + I2_COUNT * LT_VM_NSRC <= OP_CMP, "opcode map");
-static_assert(OP_CMP + 18 * LT_VM_NSRC <= OP_WHERE_A, "opcode map");
-static_assert(OP_WHERE_B + 4 * LT_VM_NSRC == OP_LDS, "opcode map");
+static_assert(OP_MOV_ACC_S < OP_ST && OP_C_NZI < OP_LD, "opcode map");
 
 // Per-CTA constants of the chunk loop, in shared memory (read by the PTX core with broadcast loads).
 struct LtLoop {
