@@ -451,6 +451,76 @@ __device__ __forceinline__ uint32_t slot_of(const Staged &S, bool staged, uint32
     return s;
 }
 
+// Executes one opcode the PTX core left to C++ (see gen_vm_core.py).  Out of line, with the machine state
+// handed over in memory: these paths are cold (ragged or unaligned chunks, irregular rows, math-library
+// transcendentals), and inlined they would raise the register count of the whole kernel by a third.
+// r[4 * k .. 4 * k + 3] is T[k] for k < NT and ACC for k = NT.
+template <bool ROW, class Env>
+__device__ __noinline__ void handle_escape(uint64_t *r, uint32_t eop, uint32_t eimm, const Env &E, const Chunk &ck, RowCtx *rc,
+                                           const Staged &S) {
+    float f[V];
+    uint64_t(&acc)[4] = *reinterpret_cast<uint64_t(*)[4]>(r + 4 * NT);
+    const bool is_ld = eop >= OP_LD && eop < OP_STG;
+    const bool is_f2m = eop >= OP_F2M && eop < OP_F2;
+    if (is_ld || is_f2m) {
+        // a load that was not linked to a vector path (unaligned pointer, broadcast class), or one
+        // that met a ragged chunk: element-wise load, then widen
+        const bool staged = (eop >= OP_LDS && eop < OP_STG) || eop >= OP_F2MS;
+        const uint32_t slot = slot_of(S, staged, eimm);
+        load_raw(f, E, slot, ck);
+        widen(f, E.dtype(slot));
+        if (is_ld) {
+            const uint32_t d = eop < OP_LDG ? eop - OP_LD : eop < OP_LDS ? (eop - OP_LDG) % LT_VM_ND : (eop - OP_LDS) % LT_VM_ND;
+            pairs_of(f, *reinterpret_cast<uint64_t(*)[4]>(r + 4 * d));
+        } else {
+            const uint32_t k = eop < OP_F2MG ? eop - OP_F2M : eop < OP_F2MS ? (eop - OP_F2MG) / 6u : (eop - OP_F2MS) / 3u;
+            float a[V];
+            lanes_of(acc, a);
+#pragma unroll
+            for (int i = 0; i < V; ++i)
+                a[i] = k == F2M_ADD ? __fadd_rn(a[i], f[i]) : k == F2M_SUB ? __fsub_rn(a[i], f[i])
+                     : k == F2M_RSUB ? __fsub_rn(f[i], a[i]) : __fmul_rn(a[i], f[i]);
+            pairs_of(a, acc);
+        }
+        return;
+    }
+    lanes_of(acc, f);
+    if (eop == OP_ST || (eop >= OP_STG && eop < OP_STG + 3)) {
+        store_chunk(f, E, eimm, ck);
+        return;
+    }
+    if (eop == OP_IOTA_ROW) {
+        const uint32_t row = (ck.row / E.scal(eimm)) % E.scal(eimm + 1);
+#pragma unroll
+        for (int i = 0; i < V; ++i) f[i] = u2f(row);
+    } else if (eop == OP_PHILOX) {
+        uint32_t w[V];
+        philox_chunk(w, ck.flat0, E.scal(eimm), E.scal(eimm + 1), E.scal(eimm + 2), E.scal(eimm + 3));
+#pragma unroll
+        for (int i = 0; i < V; ++i) f[i] = u2f(w[i]);
+    } else if (eop >= OP_RED_SUM && eop <= OP_RED_MIN) {
+        if constexpr (ROW) {
+            if (eop == OP_RED_SUM) row_reduce<0>(f, ck, rc);
+            else if (eop == OP_RED_MAX) row_reduce<1>(f, ck, rc);
+            else row_reduce<2>(f, ck, rc);
+        }
+    } else {  // correctly rounded transcendentals of the precise flavour
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            if (eop == OP_U_EXP) f[i] = un<OP_U_EXP, false>(f[i]);
+            else if (eop == OP_U_LOG) f[i] = un<OP_U_LOG, false>(f[i]);
+            else if (eop == OP_U_TANH) f[i] = un<OP_U_TANH, false>(f[i]);
+            else if (eop == OP_U_SIGMOID) f[i] = un<OP_U_SIGMOID, false>(f[i]);
+            else if (eop == OP_U_GELU) f[i] = un<OP_U_GELU, false>(f[i]);
+        }
+    }
+    pairs_of(f, acc);
+}
+
+// Runs the group's program.  R[0..NT-1] are the temporaries, R[NT] is ACC.  The PTX core runs until an opcode
+// it does not implement; that opcode is executed by handle_escape and the core re-entered.  With
+// LtLoop::inloop set the core also walks the thread's chunks by itself and `chunk_of(c)` rebuilds the
+// coordinates of chunk c for the escape code; otherwise the call covers the one chunk given.
 template <int FLAV, bool ROW, class Env, class ChunkOf>
 __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint32_t c, const Chunk &first, RowCtx *rc,
                                             const Staged &S, uint32_t stg, uint32_t flags = 0) {
@@ -467,66 +537,17 @@ __device__ __forceinline__ void run_program(const Env &E, ChunkOf chunk_of, uint
         else if constexpr (FLAV == 1) asm volatile(LT_VM_CORE_PRECISE LT_VM_OPERANDS);
         else asm volatile(LT_VM_CORE_IEEE LT_VM_OPERANDS);
         if (eop == OP_END) break;
+        uint64_t spill[4 * (NT + 1)];  // the state travels through memory so that it never has its address taken
+#pragma unroll
+        for (int k = 0; k <= NT; ++k)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) spill[4 * k + j] = R[k][j];
         const Chunk ck = chunk_of(c);
-        float f[V];
-        const bool is_ld = eop >= OP_LD && eop < OP_STG;
-        const bool is_f2m = eop >= OP_F2M && eop < OP_F2;
-        if (is_ld || is_f2m) {
-            // a load that was not linked to a vector path (unaligned pointer, broadcast class), or one
-            // that met a ragged chunk: element-wise load, then widen
-            const bool staged = (eop >= OP_LDS && eop < OP_STG) || eop >= OP_F2MS;
-            const uint32_t slot = slot_of(S, staged, eimm);
-            load_raw(f, E, slot, ck);
-            widen(f, E.dtype(slot));
-            if (is_ld) {
-                const uint32_t d = eop < OP_LDG ? eop - OP_LD : eop < OP_LDS ? (eop - OP_LDG) % LT_VM_ND : (eop - OP_LDS) % LT_VM_ND;
-                if (d == 0) pairs_of(f, R[0]);
-                else if (d == 1) pairs_of(f, R[1]);
-                else if (d == 2) pairs_of(f, R[2]);
-                else pairs_of(f, R[NT]);
-            } else {
-                const uint32_t k = eop < OP_F2MG ? eop - OP_F2M : eop < OP_F2MS ? (eop - OP_F2MG) / 6u : (eop - OP_F2MS) / 3u;
-                float a[V];
-                lanes_of(R[NT], a);
+        handle_escape<ROW>(spill, eop, eimm, E, ck, rc, S);
 #pragma unroll
-                for (int i = 0; i < V; ++i)
-                    a[i] = k == F2M_ADD ? __fadd_rn(a[i], f[i]) : k == F2M_SUB ? __fsub_rn(a[i], f[i])
-                         : k == F2M_RSUB ? __fsub_rn(f[i], a[i]) : __fmul_rn(a[i], f[i]);
-                pairs_of(a, R[NT]);
-            }
-            continue;
-        }
-        lanes_of(R[NT], f);
-        if (eop == OP_ST || (eop >= OP_STG && eop < OP_STG + 3)) {
-            store_chunk(f, E, eimm, ck);
-            continue;
-        }
-        if (eop == OP_IOTA_ROW) {
-            const uint32_t r = (ck.row / E.scal(eimm)) % E.scal(eimm + 1);
+        for (int k = 0; k <= NT; ++k)
 #pragma unroll
-            for (int i = 0; i < V; ++i) f[i] = u2f(r);
-        } else if (eop == OP_PHILOX) {
-            uint32_t w[V];
-            philox_chunk(w, ck.flat0, E.scal(eimm), E.scal(eimm + 1), E.scal(eimm + 2), E.scal(eimm + 3));
-#pragma unroll
-            for (int i = 0; i < V; ++i) f[i] = u2f(w[i]);
-        } else if (eop >= OP_RED_SUM && eop <= OP_RED_MIN) {
-            if constexpr (ROW) {
-                if (eop == OP_RED_SUM) row_reduce<0>(f, ck, rc);
-                else if (eop == OP_RED_MAX) row_reduce<1>(f, ck, rc);
-                else row_reduce<2>(f, ck, rc);
-            }
-        } else {  // correctly rounded transcendentals of the precise flavour
-#pragma unroll
-            for (int i = 0; i < V; ++i) {
-                if (eop == OP_U_EXP) f[i] = un<OP_U_EXP, false>(f[i]);
-                else if (eop == OP_U_LOG) f[i] = un<OP_U_LOG, false>(f[i]);
-                else if (eop == OP_U_TANH) f[i] = un<OP_U_TANH, false>(f[i]);
-                else if (eop == OP_U_SIGMOID) f[i] = un<OP_U_SIGMOID, false>(f[i]);
-                else if (eop == OP_U_GELU) f[i] = un<OP_U_GELU, false>(f[i]);
-            }
-        }
-        pairs_of(f, R[NT]);
+            for (int j = 0; j < 4; ++j) R[k][j] = spill[4 * k + j];
     }
 }
 
