@@ -184,9 +184,16 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     const uint32_t buf = pieces * LT_VM_STAGE_PIECE;
                     uint32_t depth = (96u * 1024u + occ * buf - 1) / (occ * buf);
                     depth = std::min(4u, std::max(2u, depth));
-                    while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
+                    while (depth >= 1 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
+                    // iterations each thread runs: a launch that gives a thread one or two chunks gains nothing
+                    // from look-ahead, but staging still fetches all its inputs in parallel
+                    const uint64_t units = L.kind == K_EW ? (P.n_chunks + LT_EW_THREADS - 1) / LT_EW_THREADS
+                                                          : ((uint64_t)P.rows + P.rows_per_cta - 1) / P.rows_per_cta;
+                    const uint64_t resident = (uint64_t)c->sm_count * occ * waves;
+                    const uint64_t iters = (units + resident - 1) / resident;
+                    if (iters <= 2 && depth >= 1) depth = (uint32_t)std::min<uint64_t>(depth, iters);
                     // two buffers (one chunk of look-ahead) measured slower than L2 prefetch: need three
-                    if (depth >= 3) P.stage_depth = depth;
+                    if (depth >= 3 || (depth >= 1 && iters <= 2)) P.stage_depth = depth;
                     else {
                         P.stage_pieces = 0;
                         for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;

@@ -389,8 +389,8 @@ def end_body():
         f"add.u32 {STG}, {STG}, r4;", "mov.u32 x0, %tid.x;", "shl.b32 x0, x0, 4;", "add.u32 x0, x0, r6;",
         "add.u32 x0, x0, r5;", f"setp.ge.u32 p, {STG}, x0;", f"@p sub.u32 {STG}, {STG}, r5;",
         # the copies of the next chunk are the oldest group still in flight
-        "setp.eq.u32 p, r3, 2;", "@p cp.async.wait_group 1;", "setp.eq.u32 p, r3, 3;", "@p cp.async.wait_group 2;",
-        "setp.eq.u32 p, r3, 4;", "@p cp.async.wait_group 3;",
+        "setp.eq.u32 p, r3, 3;", "@p cp.async.wait_group 2;", "setp.eq.u32 p, r3, 4;", "@p cp.async.wait_group 3;",
+        "setp.eq.u32 p, r3, 2;", "@p cp.async.wait_group 1;", "setp.eq.u32 p, r3, 1;", "@p cp.async.wait_group 0;",
         "L_ADV:",
         f"add.u32 {CHUNK}, {CHUNK}, r0;", f"setp.ge.u32 p, {CHUNK}, r1;", "@p bra L_ESC;",
         "setp.eq.u32 p, r7, 2;", "@p bra L_ROWS;",
@@ -426,6 +426,7 @@ def red_body(kind: int):
     """ACC = reduction of the row, broadcast: lanes of the thread, then shuffles within the warp, then (rows
     wider than a warp's 256 elements) one exchange through shared memory."""
     op = ["add.rn.f32", "max.NaN.f32", "min.NaN.f32"][kind]
+    ident = ["0f00000000", "0fFF800000", "0f7F800000"][kind]   # 0, -inf, +inf
     lines = inline_rows_guard()          # r0 = threads per row
     lines += unpack(A, X)
     lines += [f"{op} x0, x0, x1;", f"{op} x2, x2, x3;", f"{op} x4, x4, x5;", f"{op} x6, x6, x7;",
@@ -439,10 +440,17 @@ def red_body(kind: int):
         f"and.b32 r4, {TAIL}, 4;", "shl.b32 r4, r4, 5;", f"add.u32 r4, r4, {SMB};",   # half of the exchange buffer
         "shl.b32 r5, r3, 2;", "add.u32 r5, r5, r4;", "setp.eq.u32 p, r2, 0;", f"@p st.shared.b32 [r5+{SM_RED}], x0;",
         "bar.sync 0;",
-        "shr.u32 r6, r0, 5;", "sub.u32 r7, r6, 1;", "not.b32 r7, r7;", "and.b32 r7, r3, r7;",   # r6 warps per row, r7 first warp of this row
-        "shl.b32 r7, r7, 2;", "add.u32 r7, r7, r4;", f"ld.shared.b32 x0, [r7+{SM_RED}];", "sub.u32 r6, r6, 1;",
-        f"L_RED_LOOP{kind}:", "add.u32 r7, r7, 4;", f"ld.shared.b32 y0, [r7+{SM_RED}];", f"{op} x0, x0, y0;",
-        "sub.u32 r6, r6, 1;", "setp.ne.u32 p, r6, 0;", f"@p bra L_RED_LOOP{kind};",
+        # r6 = warps per row (a power of two <= 32), r7 = first warp of this row: lane l < r6 takes that
+        # warp's partial, the others the identity, and a shuffle tree combines them
+        "shr.u32 r6, r0, 5;", "sub.u32 r7, r6, 1;", "not.b32 r7, r7;", "and.b32 r7, r3, r7;",
+        "add.u32 r7, r7, r2;", "shl.b32 r7, r7, 2;", "add.u32 r7, r7, r4;",
+        f"mov.b32 x0, {ident};", "setp.lt.u32 p, r2, r6;", f"@p ld.shared.b32 x0, [r7+{SM_RED}];",
+        "setp.gt.u32 p, r6, 16;", "@p shfl.sync.bfly.b32 y0, x0, 16, 0x1f, 0xffffffff;", f"@p {op} x0, x0, y0;",
+        "setp.gt.u32 p, r6, 8;", "@p shfl.sync.bfly.b32 y0, x0, 8, 0x1f, 0xffffffff;", f"@p {op} x0, x0, y0;",
+        "setp.gt.u32 p, r6, 4;", "@p shfl.sync.bfly.b32 y0, x0, 4, 0x1f, 0xffffffff;", f"@p {op} x0, x0, y0;",
+        "setp.gt.u32 p, r6, 2;", "@p shfl.sync.bfly.b32 y0, x0, 2, 0x1f, 0xffffffff;", f"@p {op} x0, x0, y0;",
+        "setp.gt.u32 p, r6, 1;", "@p shfl.sync.bfly.b32 y0, x0, 1, 0x1f, 0xffffffff;", f"@p {op} x0, x0, y0;",
+        "shfl.sync.idx.b32 x0, x0, 0, 0x1f, 0xffffffff;",   # lanes past the row's warp count hold the identity only
         f"xor.b32 {TAIL}, {TAIL}, 4;",
         f"L_RED_DONE{kind}:",
     ]
