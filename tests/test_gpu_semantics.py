@@ -219,3 +219,68 @@ def test_random_graphs(lt, seed, fusion):
         assert a.shape == b.shape
         np.testing.assert_allclose(a, b, rtol=2e-4, atol=2e-4, equal_nan=True, err_msg=f"seed {seed} output {k}")
     c.close()
+
+
+# ------------------------------------------------------------------ pointers that cannot take 128-bit accesses
+@pytest.mark.parametrize("dtype,offset", [("f32", 1), ("f32", 2), ("bf16", 1), ("bf16", 3), ("u8", 5)])
+def test_unaligned_device_pointers(ctx, dtype, offset):
+    import torch
+    from workloads import rng as R
+    g = R.generator(31)
+    shape = (37, 64)
+    n = shape[0] * shape[1]
+    tdt = {"f32": torch.float32, "bf16": torch.int16, "u8": torch.uint8}[dtype]
+
+    def make(values_f32):
+        if dtype == "f32":
+            host = values_f32
+        elif dtype == "bf16":
+            host = R.to_bf16_bits(values_f32)
+        else:
+            host = (values_f32 > 0).astype(np.uint8)
+        store = torch.zeros(n + 16, dtype=tdt, device="cuda:0")
+        view = store[offset:offset + n]
+        src = torch.from_numpy(host.view(np.int16) if dtype == "bf16" else host).reshape(-1).to("cuda:0")
+        view.copy_(src)
+        return host, ctx.from_device_ptr(view.data_ptr(), dtype, shape, keep=store)
+
+    a_host, a = make(R.normal_f32(g, shape))
+    b_host, b = make(R.normal_f32(g, shape))
+    O = EagerOracle()
+    oa, ob = O.leaf(a_host, dtype), O.leaf(b_host, dtype)
+    if dtype == "u8":
+        ref = O.op("xor", O.op("and", oa, ob), O.op("not", oa))
+        got = ctx.op("xor", ctx.op("and", a, b), ctx.op("not", a))
+    else:
+        ref = O.op("sub", O.op("mul", oa, ob), O.op("relu", oa))
+        got = ctx.op("sub", ctx.op("mul", a, b), ctx.op("relu", a))
+    assert_matches(ctx.fetch(got), ref.array, dtype, f"unaligned {dtype}+{offset}")
+
+
+def test_unaligned_instance_in_a_multi_tensor_launch(lt):
+    import torch
+    from workloads import configs, traces
+    c = lt.LazyContext(device=0)
+    shapes = [(96,), (40, 8), (1000,), (64,)]
+    params, grads, ms, vs = configs.c5_inputs(13, shapes)
+    O = EagerOracle()
+    op, og, om, ov = ([O.leaf(a, "f32") for a in arrs] for arrs in (params, grads, ms, vs))
+
+    def dev(arr, shift):
+        store = torch.zeros(arr.size + 8, dtype=torch.float32, device="cuda:0")
+        view = store[shift:shift + arr.size]
+        view.copy_(torch.from_numpy(arr.reshape(-1)).to("cuda:0"))
+        return c.from_device_ptr(view.data_ptr(), "f32", arr.shape, keep=store)
+
+    gp = [dev(a, 1 if i == 1 else 0) for i, a in enumerate(params)]   # one parameter is 4-byte aligned only
+    gg = [dev(a, 0) for a in grads]
+    gm = [dev(a, 2 if i == 2 else 0) for i, a in enumerate(ms)]
+    gv = [dev(a, 0) for a in vs]
+    for step in (1, 2):
+        traces.adam_step(O, op, og, om, ov, step=step)
+        traces.adam_step(c, gp, gg, gm, gv, step=step)
+        c.barrier()
+    assert c.stats()["launches_multi"] == 2
+    for a, r in zip(gp + gm + gv, op + om + ov):
+        assert_matches(c.fetch(a), r.array, "f32", "adam with unaligned instances")
+    c.close()
