@@ -111,6 +111,7 @@ struct Group {
     uint64_t rows = 1, cols = 1;
     std::vector<uint32_t> members;  // native members (canonical indices), topological order
     std::vector<LtIns> ins;
+    uint32_t n_pro = 0;             // leading instructions that run once per thread (loop-invariant loads)
     std::vector<IoRef> io;
     std::vector<Imm> imms;
     uint64_t bytes = 0;

@@ -203,7 +203,17 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             if (L.kind == K_EW) {
                 if (!dry) {
                     uint64_t need = (P.n_chunks + LT_EW_THREADS - 1) / LT_EW_THREADS;
-                    unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);
+                    uint64_t want = std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);
+                    if (g.n_pro && P.rowcol && want < need) {
+                        // loop-invariant column loads: a thread must stay on one column range, i.e. the chunk
+                        // stride (grid x 256) must be a multiple of the chunks per row
+                        uint64_t a = P.cpr, b = LT_EW_THREADS;
+                        while (b) { uint64_t t = a % b; a = b; b = t; }
+                        const uint64_t m = P.cpr / a;
+                        want = (want + m - 1) / m * m;
+                        if (want > need) want = need;  // one chunk per thread: nothing to keep invariant
+                    }
+                    unsigned grid = (unsigned)want;
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
                     e = lt_launch_ew(P, L.flavour, grid, c->stream);

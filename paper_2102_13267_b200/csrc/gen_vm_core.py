@@ -365,7 +365,7 @@ def end_body():
     return [
         f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 16}];",     # buf_bytes, buf_total, stage_base, inloop
         "setp.eq.u32 p, r7, 0;", "@p bra L_ESC;",
-        f"ld.shared.v4.b32 {{r0, r1, r2, r3}}, [{SMB}+{L}];",          # stride, n_chunks, n_full, depth
+        f"ld.shared.v4.b32 {{r0, r1, r2, r3}}, [{SMB}+{L}];",          # stride, n_chunks, body offset, depth
         f"ld.shared.b64 d2, [{SMB}+{SM_N4}];",                          # 4 * elements
         f"ld.shared.b64 pf4, [{SMB}+{SM_PF}];",                         # bytes (4-byte view) between a thread's iterations
         "setp.eq.u32 pq, r3, 0;", "@pq bra L_ADV;",
@@ -412,7 +412,7 @@ def end_body():
         f"shl.b32 {COFF4}, x1, 2;", "sub.u32 x1, x3, x1;", "setp.lt.u32 ptail, x1, 8;",
         "L_COORD_DONE:",
         f"and.b32 {TAIL}, {TAIL}, 0xFFFFFFFE;", "selp.b32 x0, 1, 0, ptail;", f"or.b32 {TAIL}, {TAIL}, x0;",
-        f"mov.b32 {PC}, {SMB};",
+        f"add.u32 {PC}, {SMB}, r2;",                                    # restart after the once-per-thread part
     ] + entry_code()[2:] + [f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];"]
 
 

@@ -630,7 +630,7 @@ __device__ __forceinline__ void fill_loop(LtLoop &lp, const LtKParams &P, uint32
     const uint32_t depth = P.stage_depth;
     lp.stride = stride;
     lp.n_chunks = n_iter;
-    lp.n_full = (uint32_t)(P.n / V);
+    lp.body_off = P.n_pro * (uint32_t)sizeof(LtIns);
     lp.depth = depth;
     lp.buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
     lp.buf_total = depth * lp.buf_bytes;

@@ -241,24 +241,26 @@ struct CodeGen {
     // can v be read straight from memory by the one instruction that uses it?
     bool mem_operand_ok(int v) const { return is_input((uint32_t)v) && uses[v] == 1 && temp_of[v] < 0 && in_acc != v; }
 
-    void preload(int count) {
-        // issue the loads of the first `count` inputs up front so they are all in flight together
-        std::vector<uint32_t> order;
+    // Loop-invariant loads: a column vector is the same for every chunk a thread runs (the kernels keep a
+    // thread on one column range), so up to `count` of them are loaded once, before the per-chunk body,
+    // into temporaries that stay reserved.
+    void hoist(int count) {
+        int done = 0;
         for (uint32_t n : emit) {
             const CNode &cn = cg.nodes[n];
-            for (int i = 0; i < cn.n_in; ++i) {
-                uint32_t o = (uint32_t)rep_or_self(cn.in[i]);
-                if (is_input(o) && std::find(order.begin(), order.end(), o) == order.end()) order.push_back(o);
+            for (int i = 0; i < cn.n_in && done < count; ++i) {
+                const uint32_t o = (uint32_t)rep_or_self(cn.in[i]);
+                if (!is_input(o) || temp_of[o] >= 0 || cls_of(o) != LT_CLS_COLVEC) continue;
+                const int k = alloc_temp();
+                emit_load(k, o);
+                temp_val[k] = (int)o;
+                temp_of[o] = k;
+                temp_raw[k] = -1;
+                uses[o] += 1 << 20;  // never released
+                ++done;
             }
         }
-        for (int i = 0; i < count && i < (int)order.size() && i < LT_VM_NT; ++i) {
-            uint32_t v = order[i];
-            int k = alloc_temp();
-            emit_load(k, v);
-            temp_val[k] = (int)v;
-            temp_of[v] = k;
-            temp_raw[k] = -1;
-        }
+        g.n_pro = (uint32_t)g.ins.size();
     }
 
     int rep_or_self(uint32_t v) const { return rep[v] >= 0 ? rep[v] : (int)v; }
@@ -360,7 +362,8 @@ struct CodeGen {
                     if (!ok) return;
                 }
             } else if (!compare && is_float((uint8_t)dt) && (op == LT_OP_ADD || op == LT_OP_SUB || op == LT_OP_MUL) &&
-                       (mem_operand_ok(x) || mem_operand_ok(y))) {
+                       ((mem_operand_ok(y) && (in_acc == x || temp_of[x] < 0)) ||
+                        (mem_operand_ok(x) && !mem_operand_ok(y) && (in_acc == y || temp_of[y] < 0)))) {
                 // an input read exactly once: fold its load into the arithmetic (memory operand)
                 const bool pick_y = mem_operand_ok(y);
                 const int mem = pick_y ? y : x, reg = pick_y ? x : y;
@@ -571,9 +574,9 @@ struct CodeGen {
         if (uses[n] == 0) in_acc = -1;
     }
 
-    bool run(int preload_count) {
+    bool run(int hoist_count) {
         count_uses();
-        preload(preload_count);
+        hoist(hoist_count);
         for (uint32_t n : emit) {
             gen_node(n);
             if (!ok) return false;
@@ -890,7 +893,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                 n_inputs = (int)seen.size();
             }
             (void)n_inputs;  // loads are issued where first needed: staged inputs are already on chip
-            for (int pre = 0; pre >= 0 && !done; --pre) {
+            for (int pre = (g.rows > 1 ? LT_VM_NT - 1 : 0); pre >= 0 && !done; --pre) {
                 g.ins.clear();
                 g.io.clear();
                 g.imms.clear();
@@ -1108,6 +1111,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             memset(&P, 0, sizeof(P));
             const Group &g = groups[L.groups[0]];
             P.n_ins = (uint32_t)g.ins.size();
+            P.n_pro = g.n_pro;
             memcpy(P.ins, g.ins.data(), g.ins.size() * sizeof(LtIns));
             for (size_t s = 0; s < g.io.size(); ++s) {
                 P.io_dtype[s] = g.io[s].dtype;
@@ -1167,6 +1171,7 @@ std::string describe_plan(const Plan &plan) {
             s += buf;
         }
         for (size_t q = 0; q < g.ins.size(); ++q) {
+            if (q == g.n_pro && g.n_pro) s += "       -- per chunk:\n";
             snprintf(buf, sizeof(buf), "  %3zu  ", q);
             s += buf;
             s += disasm(g.ins[q]);

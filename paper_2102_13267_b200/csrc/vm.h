@@ -93,7 +93,7 @@ static_assert(OP_MOV_ACC_S < OP_ST && OP_C_NZI < OP_LD, "opcode map");
 
 // Per-CTA constants of the chunk loop, in shared memory (read by the PTX core with broadcast loads).
 struct LtLoop {
-    uint32_t stride, n_chunks, n_full, depth;            // chunks between a thread's iterations; total; complete ones; staging depth
+    uint32_t stride, n_chunks, body_off, depth;          // chunks between a thread's iterations; total; byte offset of the per-chunk part of the program; staging depth
     uint32_t buf_bytes, buf_total, stage_base, inloop;   // one staging buffer; all of them; shared address of the first; core loops by itself: 1 = over chunks (elementwise), 2 = over blocks of rows
     uint32_t rowcol, cpr, div_mul, div_sh1;
     uint32_t div_sh2, cols, prefetch, stg_n;             // prefetch: 1 = L2-prefetch the next chunk of full-class loads
@@ -118,6 +118,7 @@ struct LtKParams {
     uint32_t stage_depth;   // staging buffers per thread (0 = loads go straight to registers)
     uint32_t stage_pieces;  // 16-byte pieces per staging buffer
     uint32_t n_ins;
+    uint32_t n_pro;         // leading instructions run once per thread; the chunk loop restarts after them
     uint32_t rowcol;        // 0: flat chunks over n elements; 1: chunks stay inside rows
     uint64_t n;             // rows * cols
     uint32_t rows, cols;    // rowcol only
