@@ -152,7 +152,8 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * "ieee" (0 default: in groups storing f32, division, square root and reciprocal are accurate to
  * 2 ulp; 1 = correctly rounded, so that a graph of + - * / sqrt matches an op-by-op binary32
  * evaluation bit for bit, at about ten more instructions per element and op),
- * "waves" (4 default: grid size of the persistent kernels in waves of resident thread blocks),
+ * "waves" (1 default: grid size of the persistent kernels in waves of resident thread blocks; every
+ * block pays a fixed set-up -- program staging and linking -- so one wave measured fastest),
  * "stage" (1 default: inputs are copied asynchronously into shared-memory staging buffers a few chunks
  * ahead of their use; 0 = loads go straight to registers),
  * "horizontal" (1 default: bundle isomorphic independent groups into multi-tensor launches),
