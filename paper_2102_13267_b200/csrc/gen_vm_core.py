@@ -344,6 +344,7 @@ def stg_body(sz: int):
 SM_N4 = SM_PF + 8
 SM_GROUP = SM_PF + 16
 SM_RED = OPS["LT_VM_SM_RED"]
+SM_DPF = SM_PF + 24
 
 
 def entry_code():
@@ -352,55 +353,79 @@ def entry_code():
     full chunk (row kernel), 4 = which half of the reduction exchange buffer is next."""
     L = SM_LOOP
     return [f"and.b32 r0, {TAIL}, 1;", "setp.ne.u32 ptail, r0, 0;",
-            f"ld.shared.v2.b32 {{r0, r1}}, [{SMB}+{L}];",            # stride, n_chunks
+            f"ld.shared.b32 r3, [{SMB}+{L + 12}];",                   # staging depth: which wait_group the loop uses
+            "setp.eq.u32 pd1, r3, 1;", "setp.eq.u32 pd2, r3, 2;", "setp.eq.u32 pd3, r3, 3;", "setp.eq.u32 pd4, r3, 4;",
+            ] + next_chunk_predicate()
+
+
+def next_chunk_predicate():
+    """pnext: the thread has a further chunk and L2 prefetch is on (full-class vector loads then prefetch it)."""
+    L = SM_LOOP
+    return [f"ld.shared.v2.b32 {{r0, r1}}, [{SMB}+{L}];",            # stride, n_chunks
             f"ld.shared.b32 r2, [{SMB}+{L + 56}];",                   # prefetch enabled
             f"sub.u32 r1, r1, {CHUNK};", "setp.gt.u32 pnext, r1, r0;", "setp.ne.u32 p, r2, 0;",
             "and.pred pnext, pnext, p;", "not.pred p, ptail;", "and.pred pnext, pnext, p;"]
+
+
+def stage_loop(label: str, count_shift: int, shift: int):
+    """Copies of the staged inputs of one element size (list entries: pointer lo, hi, offset in the buffer)."""
+    lines = [f"bfe.u32 r8, r9, {count_shift}, 8;", "setp.eq.u32 p, r8, 0;", f"@p bra L_STG_END{label};"]
+    if shift == 2:
+        lines.append("mov.b64 d1, d0;")
+    else:
+        lines.append(f"shr.u64 d1, d0, {2 - shift};")       # byte offset for this element size
+    lines += [f"L_STG_LOOP{label}:", "ld.shared.v4.b32 {x0, x1, x2, x3}, [sa];", "mov.b64 ptr, {x0, x1};",
+              "add.u64 ptr, ptr, d1;", f"add.u32 x2, x2, {STG};"]
+    if shift == 0:
+        lines.append("cp.async.ca.shared.global [x2], [ptr], 8;")
+    else:
+        lines.append("cp.async.cg.shared.global [x2], [ptr], 16;")
+        if shift == 2:
+            lines.append(f"cp.async.cg.shared.global [x2+{STAGE_PIECE}], [ptr+16], 16;")
+    lines += ["add.u32 sa, sa, 16;", "sub.u32 r8, r8, 1;", "setp.ne.u32 p, r8, 0;", f"@p bra L_STG_LOOP{label};",
+              f"L_STG_END{label}:"]
+    return lines
 
 
 def end_body():
     """OP_END.  When the core runs the loop itself: refill the staging buffer just consumed, move to the
     thread's next chunk (or block of rows), wait for its staged inputs and restart the program."""
     L = SM_LOOP
-    return [
-        f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 16}];",     # buf_bytes, buf_total, stage_base, inloop
-        "setp.eq.u32 p, r7, 0;", "@p bra L_ESC;",
+    lines = [
+        f"ld.shared.v4.b32 {{r4, r5, r6, r7}}, [{SMB}+{L + 16}];",     # buf_bytes, buf_total, stage_base, inloop | flags
+        "and.b32 x0, r7, 3;", "setp.eq.u32 p, x0, 0;", "@p bra L_ESC;",
         f"ld.shared.v4.b32 {{r0, r1, r2, r3}}, [{SMB}+{L}];",          # stride, n_chunks, body offset, depth
         f"ld.shared.b64 d2, [{SMB}+{SM_N4}];",                          # 4 * elements
         f"ld.shared.b64 pf4, [{SMB}+{SM_PF}];",                         # bytes (4-byte view) between a thread's iterations
         "setp.eq.u32 pq, r3, 0;", "@pq bra L_ADV;",
-        # the chunk `depth` iterations ahead starts depth * pf4 bytes (4-byte view) further; staged if complete
-        "cvt.u64.u32 d1, r3;", "mul.lo.u64 d1, d1, pf4;", f"add.u64 d0, {OFF4}, d1;", "add.u64 d1, d0, 32;",
+        # the chunk `depth` iterations ahead, as a byte offset in the 4-byte view; staged if complete
+        f"ld.shared.b64 d1, [{SMB}+{SM_DPF}];", f"add.u64 d0, {OFF4}, d1;", "add.u64 d1, d0, 32;",
         "setp.gt.u64 p, d1, d2;", f"and.b32 x0, {TAIL}, 2;", "setp.ne.u32 pq, x0, 0;", "or.pred p, p, pq;",
         "@p bra L_COMMIT;",
-        "shr.u64 d0, d0, 2;",                                            # first element of that chunk
-        f"ld.shared.b32 r8, [{SMB}+{L + 60}];",                         # number of staged inputs
+        f"ld.shared.b32 r9, [{SMB}+{L + 60}];",                         # staged inputs per element size
         f"add.u32 sa, {SMB}, {SM_STG};",
-        "L_STG_LOOP:",
-        "ld.shared.v4.b32 {x0, x1, x2, x3}, [sa];",                      # ptr lo, hi, dst offset, log2(bytes)
-        "mov.b64 ptr, {x0, x1};", "shl.b64 d1, d0, x3;", "add.u64 ptr, ptr, d1;", f"add.u32 x2, x2, {STG};",
-        "setp.eq.u32 p, x3, 0;", "@p cp.async.ca.shared.global [x2], [ptr], 8;",
-        "@!p cp.async.cg.shared.global [x2], [ptr], 16;",
-        "setp.eq.u32 p, x3, 2;", f"@p cp.async.cg.shared.global [x2+{STAGE_PIECE}], [ptr+16], 16;",
-        "add.u32 sa, sa, 16;", "sub.u32 r8, r8, 1;", "setp.ne.u32 p, r8, 0;", "@p bra L_STG_LOOP;",
+    ]
+    lines += stage_loop("4", 0, 2) + stage_loop("2", 8, 1) + stage_loop("1", 16, 0)
+    lines += [
         "L_COMMIT:",
         "cp.async.commit_group;",
         # next staging buffer of this thread (a ring of `depth` buffers)
         f"add.u32 {STG}, {STG}, r4;", "mov.u32 x0, %tid.x;", "shl.b32 x0, x0, 4;", "add.u32 x0, x0, r6;",
         "add.u32 x0, x0, r5;", f"setp.ge.u32 p, {STG}, x0;", f"@p sub.u32 {STG}, {STG}, r5;",
         # the copies of the next chunk are the oldest group still in flight
-        "setp.eq.u32 p, r3, 3;", "@p cp.async.wait_group 2;", "setp.eq.u32 p, r3, 4;", "@p cp.async.wait_group 3;",
-        "setp.eq.u32 p, r3, 2;", "@p cp.async.wait_group 1;", "setp.eq.u32 p, r3, 1;", "@p cp.async.wait_group 0;",
+        "@pd3 cp.async.wait_group 2;", "@pd4 cp.async.wait_group 3;", "@pd2 cp.async.wait_group 1;",
+        "@pd1 cp.async.wait_group 0;",
         "L_ADV:",
         f"add.u32 {CHUNK}, {CHUNK}, r0;", f"setp.ge.u32 p, {CHUNK}, r1;", "@p bra L_ESC;",
-        "setp.eq.u32 p, r7, 2;", "@p bra L_ROWS;",
+        "and.b32 x0, r7, 3;", "setp.eq.u32 p, x0, 2;", "@p bra L_FIXED;",
         f"ld.shared.v4.b32 {{r4, r5, r6, r9}}, [{SMB}+{L + 32}];",      # rowcol, cpr, div_mul, div_sh1
         "setp.ne.u32 p, r4, 0;", "@p bra L_ROWCOL;",
         # flat chunks: the next chunk of this thread is pf4 bytes further
         f"add.u64 {OFF4}, {OFF4}, pf4;", f"cvt.u32.u64 {COFF4}, {OFF4};", f"add.u64 d1, {OFF4}, 32;",
         "setp.gt.u64 ptail, d1, d2;", "bra L_COORD_DONE;",
-        "L_ROWS:",
-        # row kernel: same columns, a block of rows further; absent once past the last row
+        "L_FIXED:",
+        # same columns, a fixed distance further (blocks of rows; elementwise rows when the chunk stride is a
+        # multiple of the chunks per row); absent once past the last element
         f"add.u64 {OFF4}, {OFF4}, pf4;", f"setp.ge.u64 ptail, {OFF4}, d2;", f"and.b32 x0, {TAIL}, 2;",
         "setp.ne.u32 pq, x0, 0;", "or.pred ptail, ptail, pq;", "bra L_COORD_DONE;",
         "L_ROWCOL:",
@@ -413,7 +438,11 @@ def end_body():
         "L_COORD_DONE:",
         f"and.b32 {TAIL}, {TAIL}, 0xFFFFFFFE;", "selp.b32 x0, 1, 0, ptail;", f"or.b32 {TAIL}, {TAIL}, x0;",
         f"add.u32 {PC}, {SMB}, r2;",                                    # restart after the once-per-thread part
-    ] + entry_code()[2:] + [f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];"]
+        # L2 prefetch is off whenever inputs are staged: only then is pnext worth recomputing
+        "and.b32 x0, r7, 256;", "setp.eq.u32 pnext, x0, 0;", "@pnext bra L_NO_PF;",
+    ] + next_chunk_predicate() + ["bra L_RESTART;", "L_NO_PF:", "setp.ne.u32 pnext, x0, 0;", "L_RESTART:",
+                                  f"ld.shared.v2.b32 {{nop, nimm}}, [{PC}];"]
+    return lines
 
 
 def inline_rows_guard():
@@ -535,7 +564,7 @@ def build(flavour: str) -> list[str]:
     out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3, r0, r1, r2, r3, r4, r5, r6, r7, r8, r9;")
     out.append(".reg .b32 " + ", ".join(X + ["y0", "y1", "m0", "m1"]) + ";")
     out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2, d0, d1, d2, pf4;")
-    out.append(".reg .pred p, pq, ptail, pnext;")
+    out.append(".reg .pred p, pq, ptail, pnext, pd1, pd2, pd3, pd4;")
     table = ", ".join(f"L_{i}" if i in bodies else "L_ESC" for i in range(limit))
     out.append(f"TBL: .branchtargets {table};")
     out += entry_code()

@@ -611,8 +611,9 @@ __device__ __forceinline__ void cp_async_wait(uint32_t pending) {  // at most `p
 
 // Starts the copies of one future chunk (first element e0) of every staged input into staging buffer `buf`.
 __device__ __forceinline__ void stage_chunk(const LtLoop &lp, uint64_t e0, uint32_t buf) {
+    const uint32_t total = (lp.stg_n & 0xffu) + ((lp.stg_n >> 8) & 0xffu) + ((lp.stg_n >> 16) & 0xffu);  // counts per element size
 #pragma unroll 1
-    for (uint32_t k = 0; k < lp.stg_n; ++k) {
+    for (uint32_t k = 0; k < total && k < LT_VM_MAX_PTR; ++k) {
         const uint32_t sh = lp.stg[k].shift;
         const char *src = reinterpret_cast<const char *>(((uint64_t)lp.stg[k].ptr_hi << 32) | lp.stg[k].ptr_lo) + (e0 << sh);
         const uint32_t dst = buf + lp.stg[k].dst;
@@ -622,6 +623,30 @@ __device__ __forceinline__ void stage_chunk(const LtLoop &lp, uint64_t e0, uint3
             if (sh == 2) cp_async16(dst + LT_VM_STAGE_PIECE, src + 16);
         }
     }
+}
+
+// Builds LtLoop::stg: the staged inputs sorted by element size (4-, 2-, 1-byte), counts packed in stg_n.
+template <class PtrOf>
+__device__ __forceinline__ void fill_stage_list(LtLoop &lp, const uint8_t *io_stage, const uint8_t *io_dtype, uint32_t n_slots,
+                                                PtrOf ptr_of) {
+    uint32_t k = 0, counts = 0;
+    for (uint32_t pass = 0; pass < 3; ++pass) {  // pass 0: 4-byte elements, 1: 2-byte, 2: 1-byte
+        uint32_t n = 0;
+        for (uint32_t s = 0; s < n_slots; ++s) {
+            if (io_stage[s] == 0xffu) continue;
+            const uint32_t sz = io_dtype[s] == LT_ST_BF16 ? 1u : io_dtype[s] == LT_ST_U8 ? 2u : 0u;
+            if (sz != pass) continue;
+            const uint64_t p = ptr_of(s);
+            lp.stg[k].ptr_lo = (uint32_t)p;
+            lp.stg[k].ptr_hi = (uint32_t)(p >> 32);
+            lp.stg[k].dst = io_stage[s] * LT_VM_STAGE_PIECE;
+            lp.stg[k].shift = 2u - sz;
+            ++k;
+            ++n;
+        }
+        counts |= n << (8 * pass);
+    }
+    lp.stg_n = counts;
 }
 
 // Fills the loop constants shared by the elementwise and row kernels (thread 0, before the link step).
@@ -635,7 +660,7 @@ __device__ __forceinline__ void fill_loop(LtLoop &lp, const LtKParams &P, uint32
     lp.buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
     lp.buf_total = depth * lp.buf_bytes;
     lp.stage_base = stage_base;
-    lp.inloop = mode;
+    lp.inloop = mode | ((prefetch && !depth) ? 256u : 0u);
     lp.rowcol = P.rowcol;
     lp.cpr = P.cpr;
     lp.div_mul = P.div_mul;
@@ -651,17 +676,11 @@ __device__ __forceinline__ void fill_loop(LtLoop &lp, const LtKParams &P, uint32
     // row-wise opcodes run inside the core when every thread of a row group owns a complete chunk
     const bool regular = (P.cols % V) == 0 && (mode != 2 || P.group * V == P.cols);
     lp.inline_rows = (regular && P.n < (1ull << 32)) ? 1u : 0u;
-    uint32_t k = 0;
-    if (depth)
-        for (uint32_t s = 0; s < LT_VM_MAX_PTR; ++s)
-            if (P.io_stage[s] != 0xffu) {
-                lp.stg[k].ptr_lo = (uint32_t)P.ptr[s];
-                lp.stg[k].ptr_hi = (uint32_t)(P.ptr[s] >> 32);
-                lp.stg[k].dst = P.io_stage[s] * LT_VM_STAGE_PIECE;
-                lp.stg[k].shift = 2u - (P.io_dtype[s] == LT_ST_BF16 ? 1u : P.io_dtype[s] == LT_ST_U8 ? 2u : 0u);
-                ++k;
-            }
-    lp.stg_n = k;
+    const uint64_t dpf = (uint64_t)depth * step4;
+    lp.dpf_lo = (uint32_t)dpf;
+    lp.dpf_hi = (uint32_t)(dpf >> 32);
+    lp.stg_n = 0;
+    if (depth) fill_stage_list(lp, P.io_stage, P.io_dtype, LT_VM_MAX_PTR, [&P](uint32_t s) { return P.ptr[s]; });
 }
 
 __device__ __forceinline__ Chunk ew_chunk(const LtKParams &P, uint32_t c) {
@@ -704,8 +723,11 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
         S.ptr[threadIdx.x] = flag_pointer(P.ptr[threadIdx.x], P.io_dtype[threadIdx.x], linear);
         if (depth && P.io_stage[threadIdx.x] != 0xffu) S.soff[threadIdx.x] = P.io_stage[threadIdx.x] * LT_VM_STAGE_PIECE;
     }
+    // rows that are a multiple of the chunk and a chunk stride that is a multiple of the chunks per row: a
+    // thread's next chunk is a fixed distance ahead in the same columns, no coordinates to recompute
+    const bool fixed_cols = P.rowcol && linear && (stride % P.cpr) == 0;
     if (threadIdx.x == 0)
-        fill_loop(S.loop, P, 1, stride, n_chunks, (uint64_t)stride * (V * 4), stage_base, linear);
+        fill_loop(S.loop, P, fixed_cols ? 2 : 1, stride, n_chunks, (uint64_t)stride * (V * 4), stage_base, linear);
     __syncthreads();
     link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
     __syncthreads();
@@ -828,25 +850,17 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
             lp.buf_bytes = buf_bytes;
             lp.buf_total = depth * buf_bytes;
             lp.stage_base = stage_base;
-            lp.inloop = 1;
+            lp.inloop = 1u | (depth ? 0u : 256u);
             lp.rowcol = 0;
             lp.prefetch = depth ? 0u : 1u;
             lp.pf_lo = LT_EW_THREADS * V * 4;
             lp.pf_hi = 0;
+            lp.dpf_lo = depth * LT_EW_THREADS * V * 4;
+            lp.dpf_hi = 0;
             lp.n4_lo = numel * 4u;
             lp.n4_hi = numel >> 30;
-            uint32_t k = 0;
-            if (depth)
-                for (uint32_t s = 0; s < P.n_slots; ++s)
-                    if (P.io_stage[s] != 0xffu) {
-                        const uint64_t ptr = E.ptr(s);
-                        lp.stg[k].ptr_lo = (uint32_t)ptr;
-                        lp.stg[k].ptr_hi = (uint32_t)(ptr >> 32);
-                        lp.stg[k].dst = P.io_stage[s] * LT_VM_STAGE_PIECE;
-                        lp.stg[k].shift = 2u - (P.io_dtype[s] == LT_ST_BF16 ? 1u : P.io_dtype[s] == LT_ST_U8 ? 2u : 0u);
-                        ++k;
-                    }
-            lp.stg_n = k;
+            lp.stg_n = 0;
+            if (depth) fill_stage_list(lp, P.io_stage, P.io_dtype, P.n_slots, [&E](uint32_t s) { return E.ptr(s); });
         }
         __syncthreads();
         const uint32_t c0 = chunk_first + threadIdx.x;

@@ -25,7 +25,7 @@
 #define LT_VM_SM_SOFF 1184  // per-slot offset inside a staging buffer, or 0xFFFFFFFF
 #define LT_VM_SM_LOOP 1232  // struct LtLoop: constants of the chunk loop the PTX core runs by itself
 #define LT_VM_SM_STG 1296   // LtLoop::stg, the list of inputs staged by asynchronous copies
-#define LT_VM_SM_RED 1512   // 64 floats: cross-warp exchange of the row reductions (two alternating halves)
+#define LT_VM_SM_RED 1520   // 64 floats: cross-warp exchange of the row reductions (two alternating halves)
 #define LT_VM_STAGE_PIECE 4096  // bytes one 16-byte piece of a staged input takes per stage (256 threads x 16)
 
 #define LT_MULTI_MAX_INS 64
@@ -94,8 +94,11 @@ static_assert(OP_MOV_ACC_S < OP_ST && OP_C_NZI < OP_LD, "opcode map");
 // Per-CTA constants of the chunk loop, in shared memory (read by the PTX core with broadcast loads).
 struct LtLoop {
     uint32_t stride, n_chunks, body_off, depth;          // chunks between a thread's iterations; total; byte offset of the per-chunk part of the program; staging depth
-    uint32_t buf_bytes, buf_total, stage_base, inloop;   // one staging buffer; all of them; shared address of the first; core loops by itself: 1 = over chunks (elementwise), 2 = over blocks of rows
+    // one staging buffer; all of them; shared address of the first; inloop bits 0-1: the core loops by itself, 1 = over
+    // chunks recomputing coordinates, 2 = a fixed distance ahead with unchanged columns; bit 8 = L2 prefetch on
+    uint32_t buf_bytes, buf_total, stage_base, inloop;
     uint32_t rowcol, cpr, div_mul, div_sh1;
+    // stg_n: staged inputs by element size, 4-byte | 2-byte << 8 | 1-byte << 16 (the list is sorted that way)
     uint32_t div_sh2, cols, prefetch, stg_n;             // prefetch: 1 = L2-prefetch the next chunk of full-class loads
     struct {
         uint32_t ptr_lo, ptr_hi, dst, shift;             // source pointer, offset inside a staging buffer, log2(element bytes)
@@ -103,6 +106,7 @@ struct LtLoop {
     uint32_t pf_lo, pf_hi;                               // byte distance (4-byte elements) between a thread's iterations
     uint32_t n4_lo, n4_hi;                               // 4 * number of elements
     uint32_t group, inline_rows;                         // row kernel: threads per row; 1 = reductions / row index / random bits run in the core
+    uint32_t dpf_lo, dpf_hi;                             // depth * pf: distance to the chunk whose inputs are staged next
 };
 
 // Kernel parameter block of the elementwise and row-reduction kernels.  It is passed by
