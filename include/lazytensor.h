@@ -154,9 +154,10 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * evaluation bit for bit, at about ten more instructions per element and op),
  * "waves" (1 default: grid size of the persistent kernels in waves of resident thread blocks; every
  * block pays a fixed set-up -- program staging and linking -- so one wave measured fastest),
- * "stage" (1 default: inputs are copied asynchronously into shared-memory staging buffers a few chunks
- * ahead of their use; 0 = loads go straight to registers),
- * "horizontal" (1 default: bundle isomorphic independent groups into multi-tensor launches),
+ * "stage" (3 default: inputs are copied asynchronously into per-thread shared-memory staging buffers a few
+ * chunks ahead of their use when at least this many buffers fit in 64 KB per block -- fewer measured slower than
+ * loading at first use with L2 prefetch; launches that give a thread one or two chunks stage anyway, to fetch all
+ * inputs in parallel; 0 = never stage),
  * "cache_capacity" (0 = unbounded).  Options are part of the cache key.
  * Unknown key: LT_ERR_INVALID_ARG.  The environment variables LT_FUSION, LT_VERIFY,
  * LT_FAST_MATH, LT_HORIZONTAL preset the same options at context creation.

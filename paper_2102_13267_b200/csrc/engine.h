@@ -146,7 +146,7 @@ struct Plan {
 };
 
 struct Options {
-    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 1, stage = 1;
+    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 1, stage = 3;
 };
 
 struct HashKey {

@@ -137,9 +137,9 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     const uint32_t buf = pieces * LT_VM_STAGE_PIECE;
                     uint32_t depth = (96u * 1024u + (uint32_t)c->occ_multi * buf - 1) / ((uint32_t)c->occ_multi * buf);
                     depth = std::min(4u, std::max(2u, depth));
-                    while (depth >= 2 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
-                    // two buffers (one chunk of look-ahead) measured slower than L2 prefetch: need three
-                    if (depth >= 3) P.stage_depth = depth;
+                    while (depth >= 1 && depth * buf > LT_MAX_STAGE_BYTES) --depth;
+                    // with fewer than three buffers the kernel also prefetches one chunk further into L2
+                    if (depth >= (uint32_t)std::max<int64_t>(1, c->opt.stage)) P.stage_depth = depth;
                     else {
                         P.stage_pieces = 0;
                         for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;
@@ -192,8 +192,8 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     const uint64_t resident = (uint64_t)c->sm_count * occ * waves;
                     const uint64_t iters = (units + resident - 1) / resident;
                     if (iters <= 2 && depth >= 1) depth = (uint32_t)std::min<uint64_t>(depth, iters);
-                    // two buffers (one chunk of look-ahead) measured slower than L2 prefetch: need three
-                    if (depth >= 3 || (depth >= 1 && iters <= 2)) P.stage_depth = depth;
+                    // with fewer than three buffers the kernel also prefetches one chunk further into L2
+                    if (depth >= (uint32_t)std::max<int64_t>(1, c->opt.stage) || (depth >= 1 && iters <= 2)) P.stage_depth = depth;
                     else {
                         P.stage_pieces = 0;
                         for (size_t s = 0; s < LT_VM_MAX_PTR; ++s) P.io_stage[s] = 0xff;

@@ -368,12 +368,13 @@ def next_chunk_predicate():
 
 
 def stage_loop(label: str, count_shift: int, shift: int):
-    """Copies of the staged inputs of one element size (list entries: pointer lo, hi, offset in the buffer)."""
+    """Copies of the staged inputs of one element size (list entries: pointer lo, hi, offset in the buffer).
+    With few staging buffers the chunk after the staged one is also pulled into L2 (ppf)."""
     lines = [f"bfe.u32 r8, r9, {count_shift}, 8;", "setp.eq.u32 p, r8, 0;", f"@p bra L_STG_END{label};"]
     if shift == 2:
-        lines.append("mov.b64 d1, d0;")
+        lines += ["mov.b64 d1, d0;", "mov.b64 d3, pf4;"]
     else:
-        lines.append(f"shr.u64 d1, d0, {2 - shift};")       # byte offset for this element size
+        lines += [f"shr.u64 d1, d0, {2 - shift};", f"shr.u64 d3, pf4, {2 - shift};"]   # byte offsets for this element size
     lines += [f"L_STG_LOOP{label}:", "ld.shared.v4.b32 {x0, x1, x2, x3}, [sa];", "mov.b64 ptr, {x0, x1};",
               "add.u64 ptr, ptr, d1;", f"add.u32 x2, x2, {STG};"]
     if shift == 0:
@@ -382,6 +383,7 @@ def stage_loop(label: str, count_shift: int, shift: int):
         lines.append("cp.async.cg.shared.global [x2], [ptr], 16;")
         if shift == 2:
             lines.append(f"cp.async.cg.shared.global [x2+{STAGE_PIECE}], [ptr+16], 16;")
+    lines += ["@ppf add.u64 ptr, ptr, d3;", "@ppf prefetch.global.L2 [ptr];"]
     lines += ["add.u32 sa, sa, 16;", "sub.u32 r8, r8, 1;", "setp.ne.u32 p, r8, 0;", f"@p bra L_STG_LOOP{label};",
               f"L_STG_END{label}:"]
     return lines
@@ -402,6 +404,9 @@ def end_body():
         f"ld.shared.b64 d1, [{SMB}+{SM_DPF}];", f"add.u64 d0, {OFF4}, d1;", "add.u64 d1, d0, 32;",
         "setp.gt.u64 p, d1, d2;", f"and.b32 x0, {TAIL}, 2;", "setp.ne.u32 pq, x0, 0;", "or.pred p, p, pq;",
         "@p bra L_COMMIT;",
+        # inloop bit 9: few staging buffers, so the chunk one iteration further is prefetched into L2 (if complete)
+        "add.u64 d1, d1, pf4;", "setp.le.u64 ppf, d1, d2;", "and.b32 x0, r7, 512;", "setp.ne.u32 p, x0, 0;",
+        "and.pred ppf, ppf, p;",
         f"ld.shared.b32 r9, [{SMB}+{L + 60}];",                         # staged inputs per element size
         f"add.u32 sa, {SMB}, {SM_STG};",
     ]
@@ -563,8 +568,8 @@ def build(flavour: str) -> list[str]:
     out = ["{"]
     out.append(".reg .b32 op, imm, nop, nimm, sa, sv, w0, w1, w2, w3, r0, r1, r2, r3, r4, r5, r6, r7, r8, r9;")
     out.append(".reg .b32 " + ", ".join(X + ["y0", "y1", "m0", "m1"]) + ";")
-    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2, d0, d1, d2, pf4;")
-    out.append(".reg .pred p, pq, ptail, pnext, pd1, pd2, pd3, pd4;")
+    out.append(".reg .b64 ss, ptr, offs, g0, c0, c1, c2, d0, d1, d2, d3, pf4;")
+    out.append(".reg .pred p, pq, ptail, pnext, ppf, pd1, pd2, pd3, pd4;")
     table = ", ".join(f"L_{i}" if i in bodies else "L_ESC" for i in range(limit))
     out.append(f"TBL: .branchtargets {table};")
     out += entry_code()

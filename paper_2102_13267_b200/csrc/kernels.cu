@@ -660,7 +660,8 @@ __device__ __forceinline__ void fill_loop(LtLoop &lp, const LtKParams &P, uint32
     lp.buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
     lp.buf_total = depth * lp.buf_bytes;
     lp.stage_base = stage_base;
-    lp.inloop = mode | ((prefetch && !depth) ? 256u : 0u);
+    // bit 8: L2 prefetch by the loads (no staging); bit 9: L2 prefetch behind a short staging ring
+    lp.inloop = mode | ((prefetch && !depth) ? 256u : 0u) | ((depth && depth < 3) ? 512u : 0u);
     lp.rowcol = P.rowcol;
     lp.cpr = P.cpr;
     lp.div_mul = P.div_mul;
@@ -850,7 +851,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
             lp.buf_bytes = buf_bytes;
             lp.buf_total = depth * buf_bytes;
             lp.stage_base = stage_base;
-            lp.inloop = 1u | (depth ? 0u : 256u);
+            lp.inloop = 1u | (depth ? 0u : 256u) | ((depth && depth < 3) ? 512u : 0u);
             lp.rowcol = 0;
             lp.prefetch = depth ? 0u : 1u;
             lp.pf_lo = LT_EW_THREADS * V * 4;
