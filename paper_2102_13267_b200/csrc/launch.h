@@ -12,7 +12,9 @@
 cudaError_t lt_launch_ew(const LtKParams &p, int flavour, unsigned grid, cudaStream_t stream);
 cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream);
 cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, cudaStream_t stream);
-#define LT_MAX_STAGE_BYTES (64u * 1024u)  // staging buffers per thread block
+#ifndef LT_MAX_STAGE_BYTES
+#define LT_MAX_STAGE_BYTES (64u * 1024u)
+#endif  // staging buffers per thread block
 
 // once per device: allow up to `max_stage_bytes` of dynamic shared memory for the staging buffers
 cudaError_t lt_kernel_setup(size_t max_stage_bytes);
