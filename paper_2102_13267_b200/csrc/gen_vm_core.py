@@ -493,12 +493,18 @@ def red_body(kind: int):
 
 
 def iota_row_body():
-    """ACC = (row / scal[imm]) % scal[imm+1]; the row is recovered from the chunk's byte offsets."""
+    """ACC = (row / scal[imm]) % scal[imm+1]; the row is recovered from the chunk's byte offsets: rows are a
+    multiple of the chunk here, so row = (chunks before this row's start) / (chunks per row), by multiply-shift."""
+    L = SM_LOOP
     return inline_rows_guard() + [
-        f"cvt.u64.u32 d0, {COFF4};", f"sub.u64 d0, {OFF4}, d0;", "shr.u64 d0, d0, 2;", "cvt.u32.u64 x0, d0;",   # row * cols (< 2^32)
-        f"ld.shared.b32 x1, [{SMB}+{SM_LOOP + 52}];", "div.u32 x0, x0, x1;",                                   # row
+        f"cvt.u64.u32 d0, {COFF4};", f"sub.u64 d0, {OFF4}, d0;", "shr.u64 d0, d0, 5;", "cvt.u32.u64 x0, d0;",   # row * chunks per row
+        f"ld.shared.v2.b32 {{x1, x2}}, [{SMB}+{L + 40}];", f"ld.shared.b32 x3, [{SMB}+{L + 48}];",              # div_mul, div_sh1, div_sh2
+        "mul.hi.u32 x4, x1, x0;", "sub.u32 x5, x0, x4;", "shr.u32 x5, x5, x2;", "add.u32 x4, x4, x5;", "shr.u32 x0, x4, x3;",  # row
         "shl.b32 sa, imm, 2;", f"add.u32 sa, sa, {SMB};", f"ld.shared.b32 x1, [sa+{SM_SCAL}];",
-        f"ld.shared.b32 x2, [sa+{SM_SCAL + 4}];", "div.u32 x0, x0, x1;", "rem.u32 x0, x0, x2;",
+        f"ld.shared.b32 x2, [sa+{SM_SCAL + 4}];",   # two loads: the slot pair need not be 8-byte aligned
+        "setp.ne.u32 p, x1, 1;", "@p div.u32 x0, x0, x1;",
+        "sub.u32 x3, x2, 1;", "and.b32 x4, x3, x2;", "setp.eq.u32 p, x4, 0;",                                   # extent a power of two?
+        "@p and.b32 x0, x0, x3;", "@!p rem.u32 x0, x0, x2;",
     ] + [f"mov.b64 {a}, {{x0, x0}};" for a in A]
 
 
