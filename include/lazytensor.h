@@ -221,6 +221,34 @@ lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
 lt_status lt_barrier(lt_ctx *ctx, int blocking);
 
 /*
+ * Barrier that obtains no device memory.  (The paper has no counterpart: its runtime always
+ * allocates through the framework.)  For callers that cannot allocate while they run: a control
+ * loop whose latency budget has no room for an allocator call that may synchronise the device, a
+ * plug-in confined to buffers its host application handed it, a process started after another
+ * framework claimed the rest of the GPU.  It does what lt_barrier does with the same kernels, but
+ *   - values that pass from one kernel of the flush to a later one (the plan's temporaries) are
+ *     placed in a static array in device memory of LT_STATIC_SCRATCH_MAX_BYTES bytes that every
+ *     GPU using the library holds until the process exits; a graph whose temporaries (each
+ *     rounded up to 256 bytes) need more is refused with LT_ERR_UNSUPPORTED;
+ *   - every result must overwrite one of the graph's own inputs: lt_assign it to a tensor made
+ *     by lt_tensor_from_device that the graph reads and that no other tensor names (the buffer
+ *     is then written in place, Section 4.3 -- an in-place update such as x := f(x, ...)).  A
+ *     result without such a buffer, or an input in memory the library owns
+ *     (lt_tensor_from_host, a result of an earlier lt_barrier), is refused with
+ *     LT_ERR_UNSUPPORTED;
+ *   - neither the allocator callbacks nor cudaMalloc / cudaFree (or their Async forms) are called.
+ * A refused call leaves the pending graph in place, so lt_barrier can still flush it.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before starting any stream capture.
+ * All calls, from all contexts on a device, share the one array, which keeps the previous call's
+ * contents: two flushes that may overlap on the GPU (different streams, no ordering) race on it
+ * and must be ordered by the caller.  No kernel of the library reads a temporary before writing
+ * it; `clear_first` non-zero zero-fills the array on the stream before the flush all the same.
+ */
+#define LT_STATIC_SCRATCH_MAX_BYTES (32u << 20)
+lt_status lt_barrier_static_scratch(lt_ctx *ctx, int blocking, int clear_first);
+
+/*
  * IR-incompatible read-out (Section 3): runs a blocking barrier if `t` is pending, then
  * copies the tensor to `host_dst` (host).  `nbytes` must equal the tensor's byte size.
  */

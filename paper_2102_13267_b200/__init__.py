@@ -77,6 +77,7 @@ _SIGNATURES = {
     "lt_release": [_vp, _u64],
     "lt_release_many": [_vp, _P(_u64), ctypes.c_size_t],
     "lt_barrier": [_vp, _int],
+    "lt_barrier_static_scratch": [_vp, _int, _int],
     "lt_fetch": [_vp, _u64, _vp, ctypes.c_size_t],
     "lt_device_ptr": [_vp, _u64, _P(_vp)],
     "lt_tensor_info": [_vp, _u64, _P(_int), _P(_int), _P(_i64), _P(_int)],
@@ -341,6 +342,17 @@ class LazyContext:
             self._flush_dead()
         keeps, self._keeps = self._keeps, []
         st = _lib.lt_barrier(self._ctx, 1 if blocking else 0)
+        if st:
+            self._keeps.extend(keeps)
+            self._check(st)
+
+    def barrier_static_scratch(self, blocking: bool = False, clear_first: bool = False) -> None:
+        """lt_barrier_static_scratch: the flush for callers that may not allocate device memory (results go to
+        caller buffers via `assign`, temporaries to the library's fixed scratch array)."""
+        if self._dead:
+            self._flush_dead()
+        keeps, self._keeps = self._keeps, []
+        st = _lib.lt_barrier_static_scratch(self._ctx, 1 if blocking else 0, 1 if clear_first else 0)
         if st:
             self._keeps.extend(keeps)
             self._check(st)

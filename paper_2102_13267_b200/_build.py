@@ -12,7 +12,7 @@ OBJ = HERE / "_build"
 LIB = HERE / "liblazytensor.so"
 CUDA_HOME = Path(os.environ.get("CUDA_HOME", "/usr/local/cuda"))
 
-CU_SOURCES = ["kernels.cu"]
+CU_SOURCES = ["kernels.cu", "static_scratch.cu"]
 CPP_SOURCES = ["engine.cpp", "canon.cpp", "planner.cpp", "executor.cpp"]
 HEADERS = ["engine.h", "vm.h", "launch.h", "vm_core.inc", "../../include/lazytensor.h"]
 

@@ -192,6 +192,12 @@ struct lt_ctx {
     std::string last_plan_text;  // dump of a plan that has since been evicted
     std::string error;
 
+    // set only for the duration of lt_barrier_static_scratch: temporaries are carved out of this
+    // fixed device range and nothing may be obtained from, or returned to, the allocator
+    bool static_mode = false;
+    void *static_base = nullptr;
+    size_t static_cap = 0;
+
     bool timing = false;
     std::vector<lt::TimedLaunch> timed;
     std::vector<cudaEvent_t> event_pool;

@@ -2,6 +2,7 @@
 // and launches its kernels on the context's stream.
 #include <cmath>
 #include <cstring>
+#include <string>
 
 #include "engine.h"
 #include "launch.h"
@@ -60,7 +61,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
 
     auto release_all = [&](bool outputs_too) {
         for (void *&p : c->temp_ptr) {
-            if (p) ctx_free(c, p);
+            if (p && !c->static_mode) ctx_free(c, p);
             p = nullptr;
         }
         if (outputs_too)
@@ -71,6 +72,25 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 }
     };
 
+    if (c->static_mode) {
+        // Allocation-free flush: every result must land in a buffer the caller handed in, every
+        // parameter must be caller memory (so that nothing is returned to the allocator when the
+        // graph is dropped), and the temporaries must fit the fixed scratch range.
+        for (size_t k = 0; k < n_out; ++k)
+            if (plan.outputs[k].donated_param < 0)
+                return fail(c, LT_ERR_UNSUPPORTED,
+                            "lt_barrier_static_scratch: a result has no caller buffer to go to (lt_assign it to an "
+                            "input of the graph made by lt_tensor_from_device that no other tensor names)");
+        for (uint32_t i = 0; i < plan.n_params; ++i)
+            if (c->buffers[c->nodes[cg.param_node[i]].buffer].owned)
+                return fail(c, LT_ERR_UNSUPPORTED, "lt_barrier_static_scratch: an input lives in library-owned memory");
+        size_t need = 0;
+        for (size_t t = 0; t < plan.temp_bytes.size(); ++t) need += (plan.temp_bytes[t] + 255u) & ~(size_t)255u;
+        if (need > c->static_cap)
+            return fail(c, LT_ERR_UNSUPPORTED, "lt_barrier_static_scratch: the graph needs " + std::to_string(need) +
+                                                   " bytes of temporaries, the static scratch array holds " +
+                                                   std::to_string(c->static_cap));
+    }
     uint64_t donated = 0, allocated = 0;
     for (size_t k = 0; k < n_out; ++k) {
         const OutputPlan &o = plan.outputs[k];
@@ -86,7 +106,13 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             ++allocated;
         }
     }
+    size_t static_used = 0;
     for (size_t t = 0; t < plan.temp_bytes.size(); ++t) {
+        if (c->static_mode) {
+            c->temp_ptr[t] = (char *)c->static_base + static_used;
+            static_used += (plan.temp_bytes[t] + 255u) & ~(size_t)255u;
+            continue;
+        }
         c->temp_ptr[t] = ctx_alloc(c, plan.temp_bytes[t]);
         if (!c->temp_ptr[t]) {
             release_all(true);

@@ -1,0 +1,81 @@
+// lt_barrier_static_scratch: a barrier for callers that cannot obtain device memory while
+// they run -- control loops with a latency budget that has no room for an allocator call (which
+// may synchronise the device), plug-ins that were handed a fixed carve-out of a GPU whose
+// remaining memory belongs to the host application, processes started after another framework
+// has already claimed the device's memory.  The kernels launched are the same ones lt_barrier
+// launches; only the placement of the values that pass between two kernels of one flush differs:
+// they live in the array below instead of memory taken from the context's allocator.
+#include <cuda_runtime.h>
+
+#include <mutex>
+#include <string>
+
+#include "engine.h"
+
+#ifndef LT_STATIC_SCRATCH_BYTES
+#define LT_STATIC_SCRATCH_BYTES (32u << 20)  // keep equal to the figure documented in lazytensor.h
+#endif
+static_assert(LT_STATIC_SCRATCH_BYTES == LT_STATIC_SCRATCH_MAX_BYTES, "header and array disagree");
+
+// One copy per GPU that loads the library, held until the process exits.  In host code this name
+// is only a handle for cudaGetSymbolAddress; kernels get the address that call returns.
+static __device__ __align__(256) unsigned char lt_static_scratch[LT_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_setup_lock;
+void *g_scratch_addr[kMaxDevices];  // per device ordinal, filled on first use
+
+// Writes zeros over the first `n` 16-byte words of the array (device code may name it directly).
+__global__ void lt_static_scratch_clear(size_t n) {
+    uint4 *p = reinterpret_cast<uint4 *>(lt_static_scratch);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        p[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Device address of the array on `device`, looked up once per device with that device current.
+cudaError_t scratch_address(int device, void **out) {
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> hold(g_setup_lock);
+    if (!g_scratch_addr[device]) {
+        int previous = -1;
+        cudaError_t e = cudaGetDevice(&previous);
+        if (e == cudaSuccess && previous != device) e = cudaSetDevice(device);
+        void *p = nullptr;
+        if (e == cudaSuccess) e = cudaGetSymbolAddress(&p, lt_static_scratch);
+        if (previous >= 0 && previous != device) cudaSetDevice(previous);
+        if (e != cudaSuccess) return e;
+        g_scratch_addr[device] = p;
+    }
+    *out = g_scratch_addr[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) lt_status lt_barrier_static_scratch(lt_ctx *c, int blocking,
+                                                                                      int clear_first) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    if (c->device == LT_DEVICE_NONE)
+        return lt::fail(c, LT_ERR_DEVICE, "lt_barrier_static_scratch needs a context on a CUDA device");
+    void *base = nullptr;
+    cudaError_t e = scratch_address(c->device, &base);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return lt::fail(c, LT_ERR_CUDA, std::string("cudaGetSymbolAddress(static scratch): ") + cudaGetErrorString(e));
+    }
+    if (clear_first) {
+        // The array still holds what the previous flush left there.  No kernel of this library reads
+        // a temporary before writing it, so clearing is only for callers that want a known state.
+        lt_static_scratch_clear<<<148, 256, 0, c->stream>>>(LT_STATIC_SCRATCH_BYTES / 16u);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return lt::fail(c, LT_ERR_CUDA, std::string("clearing the static scratch: ") + cudaGetErrorString(e));
+    }
+    c->static_base = base;
+    c->static_cap = LT_STATIC_SCRATCH_BYTES;
+    c->static_mode = true;
+    const lt_status s = lt_barrier(c, blocking);
+    c->static_mode = false;
+    return s;
+}
