@@ -124,6 +124,7 @@ typedef struct {
     uint64_t ns_plan;            /* fusion planning + program generation (misses only)       */
     uint64_t ns_bind_launch;     /* argument binding, allocation and kernel launches         */
     uint64_t ns_rebind;          /* turning roots into device-data leaves, freeing IR        */
+    uint64_t launches_compiled;  /* of kernels_launched: ahead-of-time compiled programs     */
 } lt_stats;
 
 /* Device time per kernel family, measured with CUDA events when kernel timing is on. */

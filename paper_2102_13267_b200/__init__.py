@@ -54,7 +54,8 @@ class lt_stats(ctypes.Structure):
         "nodes_recorded", "barriers", "compiles", "cache_hits", "kernels_launched",
         "launches_elementwise", "launches_row", "launches_multi", "bytes_planned",
         "outputs_donated", "outputs_allocated", "temporaries_allocated",
-        "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind")]
+        "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind",
+        "launches_compiled")]
 
 
 class lt_kernel_timing(ctypes.Structure):

@@ -1,0 +1,680 @@
+// Ahead-of-time compiled programs.
+//
+// The planner's register programs (vm.h) are normally interpreted.  For the programs listed in
+// compiled_programs.inc the same per-lane operations are instantiated at build time over the
+// program itself: the instruction stream is a template parameter, every opcode test is resolved
+// by the compiler, and what remains is the straight-line kernel one would write by hand for that
+// fusion group -- no dispatch, no program fetch, registers allocated by ptxas.  The planner looks a
+// group's program up in this table (exact match of instructions, slot dtypes and classes); a group
+// that is not listed, or a launch whose pointers or extents do not allow 128-bit accesses, runs on
+// the interpreter instead.  Immediates, pointers and extents stay run-time parameters, so one
+// entry serves every shape and every value of the dynamic scalars.
+//
+// Three shells, as for the interpreter:
+//   lt_c_ew     grid-stride over chunks of 8 elements, U chunks in flight per thread
+//   lt_c_row    a power-of-two group of threads owns a row and keeps it in registers (U chunks of
+//               8 elements per thread) across the row reductions; groups of up to 32 threads reduce
+//               with shuffles alone, larger ones exchange warp partials through shared memory
+//   lt_c_multi  one program over many tensors; a CTA takes super-chunks of 16384 elements and
+//               finds the owning tensor by binary search over a prefix table in the parameters
+// Every global access is a 128-bit (64-bit for one-byte types) access of a full chunk; full-class
+// inputs are all requested at the top of an iteration, before any arithmetic or store.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "compiled.h"
+#include "vm.h"
+#include "vm_ops.cuh"
+
+namespace {
+
+constexpr int V = LT_VM_V;
+constexpr int NT = LT_VM_NT;
+constexpr int C_THREADS = 256;     // elementwise and multi-tensor shells
+constexpr int C_ROW_THREADS = 128; // row shell (or the row's group size, if larger)
+
+// ------------------------------------------------------------------ program introspection
+template <class PG>
+struct Info {
+    static constexpr __host__ __device__ bool is_ld(uint32_t op) { return op >= OP_LD && op < OP_LD + LT_VM_ND; }
+    static constexpr __host__ __device__ bool is_f2m(uint32_t op) { return op >= OP_F2M && op < OP_F2M + F2M_COUNT; }
+    // ordinal among the instructions that read a slot, or -1
+    static constexpr __host__ __device__ int load_ordinal(int i) {
+        int n = 0;
+        for (int k = PG::n_pro; k < i; ++k)
+            if (is_ld(PG::ins[k].op) || is_f2m(PG::ins[k].op)) ++n;
+        return n;
+    }
+    static constexpr __host__ __device__ int n_loads() { return load_ordinal(PG::n_ins); }
+    // slot a reserved (prologue-loaded) temporary stands for, or -1
+    static constexpr __host__ __device__ int pro_slot(int t) {
+        for (int k = 0; k < PG::n_pro; ++k)
+            if ((int)(PG::ins[k].op - OP_LD) == t) return (int)PG::ins[k].imm;
+        return -1;
+    }
+    static constexpr __host__ __device__ bool needs_coords() {
+        for (int k = 0; k < PG::n_ins; ++k) {
+            const uint32_t op = PG::ins[k].op;
+            if (op == OP_IOTA_COL || op == OP_IOTA_ROW) return true;
+        }
+        for (int s = 0; s < PG::n_slots; ++s)
+            if (PG::cls[s] != LT_CLS_FULL) return true;
+        return false;
+    }
+};
+
+// ------------------------------------------------------------------ per-lane operations
+template <int OP, int FLAV>
+__device__ __forceinline__ float f2c(float a, float b) {
+    if constexpr (OP == F2_DIV || OP == F2_RDIV) {
+        const float n = OP == F2_DIV ? a : b, d = OP == F2_DIV ? b : a;
+        float r;
+        if constexpr (FLAV == 0) asm("div.approx.f32 %0, %1, %2;" : "=f"(r) : "f"(n), "f"(d));
+        else if constexpr (FLAV == 1) asm("div.full.f32 %0, %1, %2;" : "=f"(r) : "f"(n), "f"(d));
+        else r = __fdiv_rn(n, d);
+        return r;
+    } else {
+        return f2<OP, false>(a, b);
+    }
+}
+
+template <int OP, int FLAV>
+__device__ __forceinline__ float unc(float x) {
+    constexpr bool FAST = FLAV == 0;
+    if constexpr (OP == OP_U_SQRT) return FLAV == 2 ? __fsqrt_rn(x) : sqrt_approx(x);
+    else if constexpr (OP == OP_U_RSQRT) {
+        float r;
+        asm("rsqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+        return r;
+    } else if constexpr (OP == OP_U_RECIP) {
+        if constexpr (FLAV == 2) return __frcp_rn(x);
+        else if constexpr (FLAV == 0) return rcp_approx(x);
+        else {
+            float r;
+            asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+            return r;
+        }
+    } else if constexpr (FAST && OP == OP_U_EXP) {
+        float r;
+        const float y = __fmul_rn(x, 1.4426950408889634f);
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y));
+        return r;
+    } else if constexpr (FAST && OP == OP_U_LOG) {
+        float r;
+        asm("lg2.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+        return __fmul_rn(r, 0.6931471805599453f);
+    } else if constexpr (FAST && OP == OP_U_SIGMOID) {
+        float r;
+        const float y = __fmul_rn(x, -1.4426950408889634f);
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y));
+        return rcp_approx(__fadd_rn(r, 1.0f));
+    } else if constexpr (FAST && OP == OP_U_GELU) {
+        // 0.5 x (1 + tanh(k (x + c x^3))) with the polynomial in Horner form
+        const float k = 0.7978845608028654f, kc = 0.7978845608028654f * 0.044715f;
+        const float inner = __fmul_rn(fmaf(__fmul_rn(x, x), kc, k), x);
+        const float h = __fmul_rn(x, 0.5f);
+        return fmaf(h, tanh_approx(inner), h);
+    } else {
+        return un<OP, FAST>(x);
+    }
+}
+
+// ------------------------------------------------------------------ chunk memory access
+struct Raw {  // a chunk in storage format: 32 bytes of 4-byte elements, 16 of 2-byte, 8 of 1-byte
+    uint4 a, b;
+};
+
+template <int DT>
+__device__ __forceinline__ void raw_load(Raw &r, const char *p, bool streaming) {
+    if constexpr (DT == LT_ST_BF16) {
+        r.a = streaming ? __ldcs(reinterpret_cast<const uint4 *>(p)) : __ldg(reinterpret_cast<const uint4 *>(p));
+    } else if constexpr (DT == LT_ST_U8) {
+        const uint2 w = streaming ? __ldcs(reinterpret_cast<const uint2 *>(p)) : __ldg(reinterpret_cast<const uint2 *>(p));
+        r.a.x = w.x;
+        r.a.y = w.y;
+    } else {
+        const uint4 *q = reinterpret_cast<const uint4 *>(p);
+        r.a = streaming ? __ldcs(q) : __ldg(q);
+        r.b = streaming ? __ldcs(q + 1) : __ldg(q + 1);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ void raw_widen(float (&d)[V], const Raw &r) {
+    if constexpr (DT == LT_ST_BF16) {
+        const uint32_t w[4] = {r.a.x, r.a.y, r.a.z, r.a.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            d[2 * j] = u2f(w[j] << 16);
+            d[2 * j + 1] = u2f(w[j] & 0xffff0000u);
+        }
+    } else if constexpr (DT == LT_ST_U8) {
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            d[b] = u2f((r.a.x >> (8 * b)) & 0xffu);
+            d[4 + b] = u2f((r.a.y >> (8 * b)) & 0xffu);
+        }
+    } else {
+        d[0] = u2f(r.a.x); d[1] = u2f(r.a.y); d[2] = u2f(r.a.z); d[3] = u2f(r.a.w);
+        d[4] = u2f(r.b.x); d[5] = u2f(r.b.y); d[6] = u2f(r.b.z); d[7] = u2f(r.b.w);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ void chunk_store(const float (&a)[V], char *p) {
+    if constexpr (DT == LT_ST_BF16) {
+        uint4 w;
+        __nv_bfloat162 h;
+        h = __floats2bfloat162_rn(a[0], a[1]); w.x = *reinterpret_cast<uint32_t *>(&h);
+        h = __floats2bfloat162_rn(a[2], a[3]); w.y = *reinterpret_cast<uint32_t *>(&h);
+        h = __floats2bfloat162_rn(a[4], a[5]); w.z = *reinterpret_cast<uint32_t *>(&h);
+        h = __floats2bfloat162_rn(a[6], a[7]); w.w = *reinterpret_cast<uint32_t *>(&h);
+        __stcs(reinterpret_cast<uint4 *>(p), w);
+    } else if constexpr (DT == LT_ST_U8) {
+        uint2 w;
+        w.x = (f2u(a[0]) & 0xffu) | ((f2u(a[1]) & 0xffu) << 8) | ((f2u(a[2]) & 0xffu) << 16) | (f2u(a[3]) << 24);
+        w.y = (f2u(a[4]) & 0xffu) | ((f2u(a[5]) & 0xffu) << 8) | ((f2u(a[6]) & 0xffu) << 16) | (f2u(a[7]) << 24);
+        __stcs(reinterpret_cast<uint2 *>(p), w);
+    } else {
+        __stcs(reinterpret_cast<uint4 *>(p), make_uint4(f2u(a[0]), f2u(a[1]), f2u(a[2]), f2u(a[3])));
+        __stcs(reinterpret_cast<uint4 *>(p) + 1, make_uint4(f2u(a[4]), f2u(a[5]), f2u(a[6]), f2u(a[7])));
+    }
+}
+
+constexpr __host__ __device__ int esz_shift(int dt) { return dt == LT_ST_BF16 ? 1 : (dt == LT_ST_U8 ? 0 : 2); }
+
+// Coordinates of the U chunks a thread works on in one iteration.
+template <int U>
+struct Coords {
+    uint64_t flat0[U];  // flat index of lane 0
+    uint32_t col0[U];   // column of lane 0
+    uint32_t row[U];
+    bool ok[U];         // the chunk exists
+};
+
+// No row reductions in this shell.
+struct NoReduce {
+    template <int KIND, int U>
+    __device__ __forceinline__ void operator()(float (&)[U][V], const bool (&)[U]) const {}
+};
+
+// Row reductions of a thread group of `group` threads (power of two) inside a CTA.
+struct GroupReduce {
+    float *smem;     // 2 x 32 floats, alternating between consecutive reductions
+    uint32_t group;  // threads per row
+    uint32_t phase;
+    template <int KIND, int U>
+    __device__ __forceinline__ void operator()(float (&acc)[U][V], const bool (&ok)[U]) {
+        const float ident = KIND == 0 ? 0.0f : (KIND == 1 ? -INFINITY : INFINITY);
+        float part[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            // pairwise over the eight lanes, then over the chunks
+            float l0 = red_comb<KIND>(acc[u][0], acc[u][1]), l1 = red_comb<KIND>(acc[u][2], acc[u][3]);
+            float l2 = red_comb<KIND>(acc[u][4], acc[u][5]), l3 = red_comb<KIND>(acc[u][6], acc[u][7]);
+            part[u] = ok[u] ? red_comb<KIND>(red_comb<KIND>(l0, l1), red_comb<KIND>(l2, l3)) : ident;
+        }
+#pragma unroll
+        for (int s = 1; s < U; s <<= 1)
+#pragma unroll
+            for (int u = 0; u + s < U; u += 2 * s) part[u] = red_comb<KIND>(part[u], part[u + s]);
+        float r = part[0];
+        const uint32_t width = group < 32u ? group : 32u;
+        for (uint32_t off = width >> 1; off > 0; off >>= 1) r = red_comb<KIND>(r, __shfl_xor_sync(0xffffffffu, r, off));
+        if (group > 32u) {
+            float *buf = smem + (phase & 1u) * 32u;
+            ++phase;
+            const uint32_t warp = threadIdx.x >> 5;
+            if ((threadIdx.x & 31u) == 0) buf[warp] = r;
+            __syncthreads();
+            const uint32_t wpr = group >> 5;
+            const uint32_t first = (warp / wpr) * wpr;
+            r = buf[first];
+            for (uint32_t w = 1; w < wpr; ++w) r = red_comb<KIND>(r, buf[first + w]);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[u][i] = r;
+    }
+    template <int KIND>
+    static __device__ __forceinline__ float red_comb(float a, float b) {
+        if constexpr (KIND == 0) return __fadd_rn(a, b);
+        else if constexpr (KIND == 1) return max_nan(a, b);
+        else return min_nan(a, b);
+    }
+};
+
+// ------------------------------------------------------------------ the machine
+// State and straight-line execution of program PG on U chunks at once.  `Ptr` gives the base
+// pointer of a slot, `Scal` the 32-bit immediates.
+template <class PG, int U, class Ptr, class Scal, class Red>
+struct Machine {
+    using I = Info<PG>;
+    static constexpr int FLAV = PG::flavour;
+    static constexpr int NL = I::n_loads() > 0 ? I::n_loads() : 1;
+
+    float acc[U][V];
+    float t[NT][U][V];
+    Raw raw[NL][U];  // storage-format chunks requested at the top of the iteration
+    const Ptr &ptr;
+    const Scal &scal;
+    Red &red;
+    const Coords<U> &ck;
+
+    __device__ __forceinline__ Machine(const Ptr &p, const Scal &s, Red &r, const Coords<U> &c) : ptr(p), scal(s), red(r), ck(c) {}
+
+    template <int SLOT>
+    __device__ __forceinline__ const char *address(int u) const {
+        constexpr int cls = PG::cls[SLOT], sh = esz_shift(PG::dtype[SLOT]);
+        const char *base = reinterpret_cast<const char *>(ptr(SLOT));
+        if constexpr (cls == LT_CLS_FULL) return base + (ck.flat0[u] << sh);
+        else if constexpr (cls == LT_CLS_COLVEC) return base + ((uint64_t)ck.col0[u] << sh);
+        else if constexpr (cls == LT_CLS_ROWVEC) return base + ((uint64_t)ck.row[u] << sh);
+        else return base;
+    }
+
+    // widened chunk of a slot read at the point of use (column vectors, broadcast elements)
+    template <int SLOT>
+    __device__ __forceinline__ void load_now(float (&d)[V], int u) const {
+        constexpr int cls = PG::cls[SLOT], dt = PG::dtype[SLOT];
+        const char *p = address<SLOT>(u);
+        if constexpr (cls <= LT_CLS_COLVEC) {
+            Raw r;
+            raw_load<dt>(r, p, false);
+            raw_widen<dt>(d, r);
+        } else {
+            float x;
+            if constexpr (dt == LT_ST_BF16) x = u2f((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(p)) << 16);
+            else if constexpr (dt == LT_ST_U8) x = u2f((uint32_t)__ldg(reinterpret_cast<const unsigned char *>(p)));
+            else x = __ldg(reinterpret_cast<const float *>(p));
+#pragma unroll
+            for (int i = 0; i < V; ++i) d[i] = x;
+        }
+    }
+
+    // requests every full-class input of the iteration
+    template <int K = PG::n_pro>
+    __device__ __forceinline__ void issue_loads() {
+        if constexpr (K < PG::n_ins) {
+            constexpr uint32_t op = PG::ins[K].op;
+            if constexpr (I::is_ld(op) || I::is_f2m(op)) {
+                constexpr int slot = PG::ins[K].imm;
+                if constexpr (PG::cls[slot] == LT_CLS_FULL) {
+                    constexpr int dt = PG::dtype[slot];
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+                        if (ck.ok[u]) raw_load<dt>(raw[I::load_ordinal(K)][u], address<slot>(u), true);
+                }
+            }
+            issue_loads<K + 1>();
+        }
+    }
+
+    // value of the slot instruction K reads, widened
+    template <int K>
+    __device__ __forceinline__ void operand_of(float (&d)[V], int u) const {
+        constexpr int slot = PG::ins[K].imm;
+        if constexpr (PG::cls[slot] == LT_CLS_FULL) {
+            constexpr int dt = PG::dtype[slot];
+            raw_widen<dt>(d, raw[I::load_ordinal(K)][u]);
+        } else {
+            load_now<slot>(d, u);
+        }
+    }
+
+    // second operand of a two-operand opcode: a temporary (a reserved one is read from its column
+    // vector here) or a broadcast immediate
+    template <int SRC, int IMM>
+    __device__ __forceinline__ void source(float (&d)[V], int u) const {
+        if constexpr (SRC == LT_VM_SRC_S) {
+            const float s = u2f(scal(IMM));
+#pragma unroll
+            for (int i = 0; i < V; ++i) d[i] = s;
+        } else if constexpr (I::pro_slot(SRC) >= 0) {
+            load_now<I::pro_slot(SRC)>(d, u);
+        } else {
+#pragma unroll
+            for (int i = 0; i < V; ++i) d[i] = t[SRC][u][i];
+        }
+    }
+
+    template <int K>
+    __device__ __forceinline__ void step() {
+        constexpr uint32_t op = PG::ins[K].op;
+        constexpr uint32_t imm = PG::ins[K].imm;
+        if constexpr (op >= OP_MOV_T_ACC && op < OP_MOV_T_ACC + NT) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int i = 0; i < V; ++i) t[op - OP_MOV_T_ACC][u][i] = acc[u][i];
+        } else if constexpr (op >= OP_MOV_ACC_T && op < OP_MOV_ACC_T + NT) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) source<op - OP_MOV_ACC_T, 0>(acc[u], u);
+        } else if constexpr (op == OP_MOV_ACC_S) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) source<LT_VM_SRC_S, imm>(acc[u], u);
+        } else if constexpr (op == OP_ST) {
+            static_assert(PG::cls[imm] == LT_CLS_FULL, "compiled programs store full-class results only");
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (ck.ok[u]) chunk_store<PG::dtype[imm]>(acc[u], const_cast<char *>(address<imm>(u)));
+        } else if constexpr (op == OP_IOTA_COL) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = u2f(ck.col0[u] + i);
+        } else if constexpr (op == OP_IOTA_ROW) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t r = (ck.row[u] / scal(imm)) % scal(imm + 1);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = u2f(r);
+            }
+        } else if constexpr (op == OP_PHILOX) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                // chunks start on a multiple of eight elements: two counter blocks, four words each
+                const uint64_t q = ck.flat0[u] >> 2;
+                uint32_t a[4], b[4];
+                philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), scal(imm + 2), scal(imm + 3), scal(imm), scal(imm + 1), a);
+                philox4x32_10((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), scal(imm + 2), scal(imm + 3), scal(imm), scal(imm + 1), b);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[u][i] = u2f(a[i]);
+                    acc[u][4 + i] = u2f(b[i]);
+                }
+            }
+        } else if constexpr (op >= OP_RED_SUM && op <= OP_RED_MIN) {
+            red.template operator()<op - OP_RED_SUM, U>(acc, ck.ok);
+        } else if constexpr (op >= OP_U_NEG && op <= OP_C_NZI) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = unc<op, FLAV>(acc[u][i]);
+        } else if constexpr (I::is_ld(op)) {
+            constexpr int d = op - OP_LD;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if constexpr (d < NT) operand_of<K>(t[d][u], u);
+                else operand_of<K>(acc[u], u);
+            }
+        } else if constexpr (I::is_f2m(op)) {
+            constexpr int k = op - OP_F2M;
+            constexpr int f = k == F2M_ADD ? F2_ADD : k == F2M_SUB ? F2_SUB : k == F2M_RSUB ? F2_RSUB : F2_MUL;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float m[V];
+                operand_of<K>(m, u);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = f2c<f, FLAV>(acc[u][i], m[i]);
+            }
+        } else if constexpr (op >= OP_F2 && op < OP_I2) {
+            constexpr int idx = (op - OP_F2) / LT_VM_NSRC, src = (op - OP_F2) % LT_VM_NSRC;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float m[V];
+                source<src, imm>(m, u);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = f2c<idx, FLAV>(acc[u][i], m[i]);
+            }
+        } else if constexpr (op >= OP_I2 && op < OP_CMP) {
+            constexpr int idx = (op - OP_I2) / LT_VM_NSRC, src = (op - OP_I2) % LT_VM_NSRC;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float m[V];
+                source<src, imm>(m, u);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = i2<idx>(acc[u][i], m[i]);
+            }
+        } else if constexpr (op >= OP_CMP && op < OP_WHERE_A) {
+            constexpr int idx = (op - OP_CMP) / LT_VM_NSRC, src = (op - OP_CMP) % LT_VM_NSRC;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float m[V];
+                source<src, imm>(m, u);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[u][i] = cmp<idx>(acc[u][i], m[i]);
+            }
+        } else if constexpr (op >= OP_WHERE_A && op < OP_LIMIT) {
+            constexpr bool variant_b = op >= OP_WHERE_B;
+            constexpr int rel = variant_b ? op - OP_WHERE_B : op - OP_WHERE_A;
+            constexpr int mt = rel / LT_VM_NSRC, src = rel % LT_VM_NSRC;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float m[V], msk[V];
+                source<src, imm>(m, u);
+                source<mt, 0>(msk, u);
+#pragma unroll
+                for (int i = 0; i < V; ++i) {
+                    const bool on = f2u(msk[i]) != 0u;
+                    acc[u][i] = variant_b ? (on ? m[i] : acc[u][i]) : (on ? acc[u][i] : m[i]);
+                }
+            }
+        } else {
+            static_assert(op == OP_END, "opcode not handled by the compiled shells");
+        }
+    }
+
+    template <int K = PG::n_pro>
+    __device__ __forceinline__ void run() {
+        if constexpr (K < PG::n_ins) {
+            step<K>();
+            run<K + 1>();
+        }
+    }
+};
+
+struct ScalK {
+    const LtKParams &P;
+    __device__ __forceinline__ uint32_t operator()(uint32_t i) const { return P.scal[i]; }
+};
+struct PtrK {
+    const LtKParams &P;
+    __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[s]; }
+};
+struct ScalM {
+    const LtMultiParams &P;
+    __device__ __forceinline__ uint32_t operator()(uint32_t i) const { return P.scal[i]; }
+};
+struct PtrM {
+    const LtMultiParams &P;
+    uint32_t base;
+    __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[base + s]; }
+};
+
+// ------------------------------------------------------------------ shells
+// Elementwise: chunk c of U-tuples strides through the tensor; rows are a multiple of the chunk.
+template <class PG, int U>
+__global__ void __launch_bounds__(C_THREADS) lt_c_ew(const __grid_constant__ LtKParams P) {
+    const uint32_t n_chunks = (uint32_t)P.n_chunks;
+    const uint32_t stride = gridDim.x * C_THREADS;
+    const PtrK ptr{P};
+    const ScalK scal{P};
+    NoReduce red;
+    for (uint32_t c = blockIdx.x * C_THREADS + threadIdx.x; c < n_chunks; c += U * stride) {
+        Coords<U> ck;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t cu = c + u * stride;
+            ck.ok[u] = cu < n_chunks;
+            ck.flat0[u] = (uint64_t)cu * V;
+            if (Info<PG>::needs_coords() && P.rowcol) {
+                const uint32_t q = __umulhi(P.div_mul, cu);
+                const uint32_t row = (q + ((cu - q) >> P.div_sh1)) >> P.div_sh2;
+                ck.row[u] = row;
+                ck.col0[u] = (cu - row * P.cpr) * V;
+            } else {
+                ck.row[u] = 0;
+                ck.col0[u] = cu * V;
+            }
+        }
+        Machine<PG, U, PtrK, ScalK, NoReduce> m(ptr, scal, red, ck);
+        m.issue_loads();
+        m.run();
+    }
+}
+
+// Row reductions: thread `gl` of a row's group owns chunks gl, gl + group, ... of the row.
+template <class PG, int U>
+__global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant__ LtKParams P, uint32_t group, uint32_t group_log2) {
+    __shared__ float red_buf[64];
+    const PtrK ptr{P};
+    const ScalK scal{P};
+    GroupReduce red{red_buf, group, 0u};
+    const uint32_t rows_per_cta = blockDim.x >> group_log2;
+    const uint32_t row_blocks = (P.rows + rows_per_cta - 1u) / rows_per_cta;
+    const uint32_t sub = threadIdx.x >> group_log2, gl = threadIdx.x & (group - 1u);
+    for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
+        const uint32_t row = rb * rows_per_cta + sub;
+        Coords<U> ck;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            ck.row[u] = row;
+            ck.col0[u] = (u * group + gl) * V;
+            ck.ok[u] = row < P.rows && ck.col0[u] < P.cols;
+            ck.flat0[u] = (uint64_t)row * P.cols + ck.col0[u];
+        }
+        Machine<PG, U, PtrK, ScalK, GroupReduce> m(ptr, scal, red, ck);
+        m.issue_loads();
+        m.run();
+    }
+}
+
+// Multi-tensor: every tensor is a flat range of chunks; a super-chunk is 2048 consecutive chunks.
+template <class PG, int U>
+__global__ void __launch_bounds__(C_THREADS) lt_c_multi(const __grid_constant__ LtMultiParams P) {
+    const ScalM scal{P};
+    NoReduce red;
+    constexpr uint32_t PER_SUPER = LT_EW_THREADS * LT_MULTI_SUB;
+    static_assert(LT_EW_THREADS == C_THREADS && LT_MULTI_SUB % U == 0, "super-chunk walk");
+    for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
+        uint32_t lo = 0, hi = P.n_inst;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (P.super_prefix[mid] <= sc) lo = mid; else hi = mid;
+        }
+        const PtrM ptr{P, lo * P.n_slots};
+        const uint32_t chunks_all = P.numel[lo] / V;
+        const uint32_t first = (sc - P.super_prefix[lo]) * PER_SUPER + threadIdx.x;
+#pragma unroll 1
+        for (uint32_t k = 0; k < LT_MULTI_SUB; k += U) {
+            Coords<U> ck;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t cu = first + (k + u) * C_THREADS;
+                ck.ok[u] = cu < chunks_all;
+                ck.flat0[u] = (uint64_t)cu * V;
+                ck.row[u] = 0;
+                ck.col0[u] = cu * V;
+            }
+            if (!ck.ok[0]) break;
+            Machine<PG, U, PtrM, ScalM, NoReduce> m(ptr, scal, red, ck);
+            m.issue_loads();
+            m.run();
+        }
+    }
+}
+
+// ------------------------------------------------------------------ table
+#include "compiled_programs.inc"
+
+template <class PG>
+bool same_program(const LtIns *ins, uint32_t n_ins, uint32_t n_pro, const uint8_t *dtype, const uint8_t *cls, uint32_t n_slots) {
+    if (n_ins != (uint32_t)PG::n_ins || n_pro != (uint32_t)PG::n_pro || n_slots != (uint32_t)PG::n_slots) return false;
+    for (int i = 0; i < PG::n_ins; ++i)
+        if (ins[i].op != PG::ins[i].op || ins[i].imm != PG::ins[i].imm) return false;
+    for (int s = 0; s < PG::n_slots; ++s)
+        if (dtype[s] != PG::dtype[s] || cls[s] != PG::cls[s]) return false;
+    return true;
+}
+
+template <class PG>
+cudaError_t launch_one(const void *params, int u, unsigned grid, unsigned threads, unsigned group, unsigned group_log2,
+                       cudaStream_t stream) {
+    if constexpr (PG::kind == 0) {
+        const LtKParams &P = *static_cast<const LtKParams *>(params);
+        if (u >= 2) lt_c_ew<PG, 2><<<grid, C_THREADS, 0, stream>>>(P);
+        else lt_c_ew<PG, 1><<<grid, C_THREADS, 0, stream>>>(P);
+    } else if constexpr (PG::kind == 1) {
+        const LtKParams &P = *static_cast<const LtKParams *>(params);
+        if (u >= 8) lt_c_row<PG, 8><<<grid, threads, 0, stream>>>(P, group, group_log2);
+        else if (u >= 4) lt_c_row<PG, 4><<<grid, threads, 0, stream>>>(P, group, group_log2);
+        else if (u >= 2) lt_c_row<PG, 2><<<grid, threads, 0, stream>>>(P, group, group_log2);
+        else lt_c_row<PG, 1><<<grid, threads, 0, stream>>>(P, group, group_log2);
+    } else {
+        const LtMultiParams &P = *static_cast<const LtMultiParams *>(params);
+        if (u >= 2) lt_c_multi<PG, 2><<<grid, C_THREADS, 0, stream>>>(P);
+        else lt_c_multi<PG, 1><<<grid, C_THREADS, 0, stream>>>(P);
+    }
+    return cudaGetLastError();
+}
+
+template <class PG>
+cudaError_t occupancy_one(int u, int threads, int *blocks) {
+    if constexpr (PG::kind == 0) {
+        return u >= 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_ew<PG, 2>, C_THREADS, 0)
+                      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_ew<PG, 1>, C_THREADS, 0);
+    } else if constexpr (PG::kind == 1) {
+        if (u >= 8) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 8>, threads, 0);
+        if (u >= 4) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 4>, threads, 0);
+        if (u >= 2) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 2>, threads, 0);
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 1>, threads, 0);
+    } else {
+        return u >= 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_multi<PG, 2>, C_THREADS, 0)
+                      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_multi<PG, 1>, C_THREADS, 0);
+    }
+}
+
+}  // namespace
+
+int lt_compiled_find(int kind, int flavour, const LtIns *ins, uint32_t n_ins, uint32_t n_pro, const uint8_t *dtype,
+                     const uint8_t *cls, uint32_t n_slots) {
+    int id = 0;
+#define LT_X(PG)                                                                                                  \
+    if (PG::kind == kind && PG::flavour == flavour && same_program<PG>(ins, n_ins, n_pro, dtype, cls, n_slots)) return id; \
+    ++id;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return -1;
+}
+
+int lt_compiled_count(void) {
+    int n = 0;
+#define LT_X(PG) ++n;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return n;
+}
+
+const char *lt_compiled_name(int id) {
+    int k = 0;
+#define LT_X(PG)                 \
+    if (k == id) return PG::name; \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return "";
+}
+
+cudaError_t lt_compiled_launch(int id, const void *params, int u, unsigned grid, unsigned threads, unsigned group,
+                               unsigned group_log2, cudaStream_t stream) {
+    int k = 0;
+#define LT_X(PG)                                                                                \
+    if (k == id) return launch_one<PG>(params, u, grid, threads, group, group_log2, stream); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t lt_compiled_occupancy(int id, int u, int threads, int *blocks) {
+    int k = 0;
+#define LT_X(PG)                                                  \
+    if (k == id) return occupancy_one<PG>(u, threads, blocks); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}

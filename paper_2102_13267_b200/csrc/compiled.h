@@ -1,0 +1,19 @@
+// Table of ahead-of-time compiled programs (compiled.cu): lookup by exact program, launch by index.
+#pragma once
+#include <cuda_runtime_api.h>
+#include <stdint.h>
+
+#include "vm.h"
+
+// Index of the table entry whose kernel family (0 elementwise, 1 row, 2 multi-tensor), flavour, instructions,
+// prologue length and slot dtypes / classes equal the arguments, or -1.
+int lt_compiled_find(int kind, int flavour, const LtIns *ins, uint32_t n_ins, uint32_t n_pro, const uint8_t *dtype,
+                     const uint8_t *cls, uint32_t n_slots);
+int lt_compiled_count(void);
+const char *lt_compiled_name(int id);
+// `u`: chunks of eight elements a thread keeps in flight (elementwise, multi: 1 or 2; row: 1, 2, 4 or 8).
+// `params` points at the LtKParams (elementwise, row) or LtMultiParams block.  Row launches: `threads` per
+// CTA and the power-of-two `group` of threads that owns a row.
+cudaError_t lt_compiled_launch(int id, const void *params, int u, unsigned grid, unsigned threads, unsigned group,
+                               unsigned group_log2, cudaStream_t stream);
+cudaError_t lt_compiled_occupancy(int id, int u, int threads, int *blocks_per_sm);

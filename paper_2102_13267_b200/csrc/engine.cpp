@@ -337,6 +337,8 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "ieee")) c->opt.ieee = value;
     else if (!strcmp(key, "waves")) c->opt.waves = value;
     else if (!strcmp(key, "stage")) c->opt.stage = value;
+    else if (!strcmp(key, "compiled")) c->opt.compiled = value;
+    else if (!strcmp(key, "compiled_u")) c->opt.compiled_u = value;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
 }

@@ -123,6 +123,8 @@ struct Launch {
     std::vector<uint32_t> groups;   // one group, or the instances of a multi-tensor launch
     uint64_t bytes = 0;
     unsigned threads = LT_EW_THREADS;
+    int compiled = -1;                   // entry of the ahead-of-time compiled table (compiled.h), or -1
+    int compiled_blocks[4] = {0, 0, 0, 0};  // resident blocks per SM of that entry's kernels, by log2(chunks in flight); 0 = not asked yet
     std::unique_ptr<LtKParams> kp;       // K_EW / K_ROW parameter block (static parts prefilled)
     std::unique_ptr<LtMultiParams> mp;   // K_MULTI
 };
@@ -147,6 +149,8 @@ struct Plan {
 
 struct Options {
     int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 1, stage = 3;
+    int64_t compiled = 1;  // use the ahead-of-time compiled kernel of a program when the table has one
+    int64_t compiled_u = 0;  // chunks in flight per thread in compiled elementwise / multi kernels (0 = default)
 };
 
 struct HashKey {

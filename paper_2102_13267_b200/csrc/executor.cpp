@@ -4,6 +4,7 @@
 #include <cstring>
 #include <string>
 
+#include "compiled.h"
 #include "engine.h"
 #include "launch.h"
 
@@ -46,6 +47,23 @@ cudaEvent_t take_event(lt_ctx *c) {
     cudaEvent_t e = nullptr;
     cudaEventCreate(&e);
     return e;
+}
+
+bool aligned_for(uint64_t p, uint8_t dtype) { return (p & (dtype == LT_U8 ? 7u : 15u)) == 0; }
+
+// resident blocks per SM of a compiled kernel variant, asked once per plan launch
+int compiled_blocks(Launch &L, int u, int threads) {
+    int lg = 0;
+    while ((1 << lg) < u) ++lg;
+    if (L.compiled_blocks[lg] == 0) {
+        int b = 0;
+        if (lt_compiled_occupancy(L.compiled, u, threads, &b) != cudaSuccess || b < 1) {
+            cudaGetLastError();
+            b = 1;
+        }
+        L.compiled_blocks[lg] = b;
+    }
+    return L.compiled_blocks[lg];
 }
 
 }  // namespace
@@ -172,7 +190,27 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     }
                 }
             }
-            if (!dry) {
+            bool done = false;
+            if (!dry && c->opt.compiled && L.compiled >= 0) {
+                // compiled kernel: needs 128-bit accesses everywhere (aligned pointers, whole chunks)
+                bool ok = true;
+                for (size_t k = 0; k < L.groups.size() && ok; ++k) {
+                    ok = (P.numel[k] % LT_VM_V) == 0;
+                    for (size_t s = 0; s < slots && ok; ++s) ok = aligned_for(P.ptr[k * slots + s], g0.io[s].dtype);
+                }
+                if (ok) {
+                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 1;
+                    const int occ = compiled_blocks(L, u, LT_EW_THREADS);
+                    unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * waves);
+                    if (grid < 1) grid = 1;
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, c->stream);
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                    c->stats.launches_compiled++;
+                    done = true;
+                }
+            }
+            if (!dry && !done) {
                 unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * c->occ_multi * waves);
                 if (grid < 1) grid = 1;
                 if (ev0) cudaEventRecord(ev0, c->stream);
@@ -226,7 +264,45 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     }
                 }
             }
-            if (L.kind == K_EW) {
+            bool done = false;
+            if (!dry && c->opt.compiled && L.compiled >= 0) {
+                // compiled kernel: needs 128-bit accesses everywhere (aligned pointers, whole chunks)
+                bool ok = (L.kind == K_EW && !P.rowcol) ? (P.n % LT_VM_V) == 0 : (P.cols % LT_VM_V) == 0;
+                ok = ok && P.n_chunks < (1ull << 31);
+                for (size_t s = 0; s < g.io.size() && ok; ++s)
+                    if (g.io[s].cls <= LT_CLS_COLVEC) ok = aligned_for(P.ptr[s], g.io[s].dtype);
+                if (ok && L.kind == K_EW) {
+                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 1;
+                    const int occ = compiled_blocks(L, u, LT_EW_THREADS);
+                    const uint64_t need = (P.n_chunks + (uint64_t)LT_EW_THREADS * u - 1) / ((uint64_t)LT_EW_THREADS * u);
+                    unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * occ * waves);
+                    if (grid < 1) grid = 1;
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, c->stream);
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                    done = true;
+                } else if (ok && P.cpr <= 8u * 1024u) {
+                    // a row lives in the registers of its thread group: up to 8 chunks per thread, one warp per row if it fits
+                    int u = 1;
+                    while (u < 8 && P.cpr > 32u * u) u *= 2;
+                    unsigned grp = 1, lg = 0;
+                    while (grp * u < P.cpr) grp <<= 1, ++lg;
+                    const unsigned threads = grp > 128 ? grp : 128;
+                    const int occ = compiled_blocks(L, u, (int)threads);
+                    const uint64_t blocks = ((uint64_t)P.rows + threads / grp - 1) / (threads / grp);
+                    unsigned grid = (unsigned)std::min<uint64_t>(blocks, (uint64_t)c->sm_count * occ * waves);
+                    if (grid < 1) grid = 1;
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    e = lt_compiled_launch(L.compiled, &P, u, grid, threads, grp, lg, c->stream);
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                    done = true;
+                }
+                if (done) c->stats.launches_compiled++;
+            }
+            if (done) {
+                if (L.kind == K_EW) c->stats.launches_elementwise++;
+                else c->stats.launches_row++;
+            } else if (L.kind == K_EW) {
                 if (!dry) {
                     uint64_t need = (P.n_chunks + LT_EW_THREADS - 1) / LT_EW_THREADS;
                     uint64_t want = std::min<uint64_t>(need, (uint64_t)c->sm_count * c->occ_ew * waves);

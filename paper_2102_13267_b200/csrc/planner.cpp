@@ -8,6 +8,7 @@
 #include <cstring>
 #include <map>
 
+#include "compiled.h"
 #include "engine.h"
 
 namespace lt {
@@ -1134,6 +1135,16 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             }
         }
     }
+    // ---- ahead-of-time compiled kernels: exact lookup of each launch's program
+    for (Launch &L : plan.launches) {
+        const Group &g = groups[L.groups[0]];
+        uint8_t dt[LT_VM_MAX_PTR] = {0}, cl[LT_VM_MAX_PTR] = {0};
+        for (size_t s = 0; s < g.io.size() && s < LT_VM_MAX_PTR; ++s) {
+            dt[s] = g.io[s].dtype;
+            cl[s] = L.kind == K_MULTI ? (uint8_t)LT_CLS_FULL : g.io[s].cls;
+        }
+        L.compiled = lt_compiled_find(L.kind, L.flavour, g.ins.data(), (uint32_t)g.ins.size(), g.n_pro, dt, cl, (uint32_t)g.io.size());
+    }
     return LT_OK;
 }
 
@@ -1158,6 +1169,17 @@ std::string describe_plan(const Plan &plan) {
                  L.flavour == 0 ? "fast" : (L.flavour == 1 ? "precise" : "ieee"), L.groups.size(), (unsigned long long)g.rows, (unsigned long long)g.cols,
                  g.rowcol ? "rowcol" : "flat", (unsigned long long)L.bytes);
         s += buf;
+        {
+            // the exact identity of the program: what the table of compiled programs is keyed on
+            std::string key = "  key: " + std::to_string(L.kind) + " " + std::to_string(L.flavour) + " " + std::to_string(g.n_pro) + " |";
+            for (const IoRef &io : g.io) key += " " + std::to_string(io.dtype);
+            key += " |";
+            for (const IoRef &io : g.io) key += " " + std::to_string(L.kind == K_MULTI ? 0 : io.cls);
+            key += " |";
+            for (const LtIns &in : g.ins) key += " " + std::to_string(in.op) + ":" + std::to_string(in.imm);
+            s += key + "\n";
+            s += std::string("  compiled: ") + (L.compiled >= 0 ? lt_compiled_name(L.compiled) : "no") + "\n";
+        }
         for (size_t q = 0; q < g.io.size(); ++q) {
             const IoRef &io = g.io[q];
             snprintf(buf, sizeof(buf), "  p%zu: %s %s %s %s%u\n", q, io.is_store ? "store" : "load", dtype_name(io.dtype),

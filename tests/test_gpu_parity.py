@@ -20,9 +20,13 @@ def lt():
     return lt
 
 
-@pytest.fixture()
-def ctx(lt):
+@pytest.fixture(params=["compiled", "interpreted"])
+def ctx(lt, request):
+    """Every case runs twice: with the ahead-of-time compiled kernels allowed (the default; launches whose
+    extents or pointers rule out 128-bit accesses still fall to the interpreter) and on the interpreter alone."""
     c = lt.LazyContext(device=0)
+    c.set_option("compiled", 1 if request.param == "compiled" else 0)
+    c.compiled_allowed = request.param == "compiled"
     yield c
     c.close()
 
@@ -62,6 +66,8 @@ def test_c2_mlp_epilogue(ctx, shape, primitive):
     out = traces.mlp_epilogue(ctx, *gl, primitive_gelu=primitive)
     ctx.barrier()
     assert ctx.stats()["kernels_launched"] == 1
+    if shape[1] % 8 == 0 and shape[0] > 1:  # (a one-row input is not a broadcast: another program)
+        assert ctx.stats()["launches_compiled"] == (1 if ctx.compiled_allowed else 0)
     assert_matches(ctx.fetch(out), ref.array, "bf16", f"c2 {shape}")
 
 
@@ -79,6 +85,8 @@ def test_c3_residual_dropout_layernorm(ctx, shape, out_dtype):
     z, k = traces.residual_dropout_layernorm(ctx, *gl, **kw)
     ctx.barrier()
     assert ctx.stats()["kernels_launched"] == 1
+    if shape[-1] % 8 == 0:
+        assert ctx.stats()["launches_compiled"] == (1 if ctx.compiled_allowed else 0)
     assert_matches(ctx.fetch(k), kr.array, "u8", f"c3 mask {shape}")
     assert_matches(ctx.fetch(z), zr.array, out_dtype, f"c3 z {shape}")
     # a new offset gives a new mask without a recompile
@@ -104,6 +112,8 @@ def test_c4_causal_softmax(ctx, shape, out_dtype):
     y = traces.causal_softmax(ctx, *gl, **kw)
     ctx.barrier()
     assert ctx.stats()["kernels_launched"] == 1
+    if shape[-1] % 8 == 0:
+        assert ctx.stats()["launches_compiled"] == (1 if ctx.compiled_allowed else 0)
     got = ctx.fetch(y)
     assert_matches(got, ref.array, out_dtype, f"c4 {shape}")
     # masked entries are exactly +0
@@ -144,6 +154,7 @@ def test_c5_adam_small(ctx):
 def test_c5_adam_full_shapes(ctx):
     s = _adam_case(ctx, parameter_shapes(), steps=3, check_every=3)
     assert s["kernels_launched"] == 3 and s["launches_multi"] == 3
+    assert s["launches_compiled"] == (3 if ctx.compiled_allowed else 0)
     assert s["bytes_planned"] == 3 * 715_596_896
 
 
