@@ -28,6 +28,7 @@ def _stale(target: Path, deps) -> bool:
     return any(Path(d).stat().st_mtime > t for d in deps)
 
 
+PER_SOURCE_FLAGS: dict = {}
 EXTRA_NVCC = os.environ.get("LT_NVCC_FLAGS", "").split()  # e.g. -DLT_EW_MIN_BLOCKS=2 for tuning experiments
 
 
@@ -37,7 +38,7 @@ def _compile(src: str) -> Path:
     deps = [path] + [CSRC / h for h in HEADERS]
     if _stale(obj, deps):
         if src.endswith(".cu"):
-            cmd = [str(CUDA_HOME / "bin" / "nvcc"), *NVCC_FLAGS, *EXTRA_NVCC, "-c", str(path), "-o", str(obj)]
+            cmd = [str(CUDA_HOME / "bin" / "nvcc"), *NVCC_FLAGS, *PER_SOURCE_FLAGS.get(src, []), *EXTRA_NVCC, "-c", str(path), "-o", str(obj)]
         else:
             cmd = ["g++", *CXX_FLAGS, "-c", str(path), "-o", str(obj)]
         subprocess.check_call(cmd)

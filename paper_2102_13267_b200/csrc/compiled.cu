@@ -53,6 +53,27 @@ struct Info {
             if ((int)(PG::ins[k].op - OP_LD) == t) return (int)PG::ins[k].imm;
         return -1;
     }
+    // Staging layout of one pipeline stage (row shell): the full-class inputs of an iteration, load
+    // ordinal by load ordinal; every thread owns U chunks of each.  Byte offset of load `ord`:
+    static constexpr __host__ __device__ int chunk_bytes(int slot) { return PG::dtype[slot] == LT_ST_BF16 ? 16 : PG::dtype[slot] == LT_ST_U8 ? 8 : 32; }
+    static constexpr __host__ __device__ int stage_offset(int ord, int u_count, int threads) {
+        int off = 0, n = 0;
+        for (int k = PG::n_pro; k < PG::n_ins; ++k)
+            if (is_ld(PG::ins[k].op) || is_f2m(PG::ins[k].op)) {
+                if (n == ord) return off;
+                if (PG::cls[PG::ins[k].imm] == LT_CLS_FULL) off += chunk_bytes(PG::ins[k].imm) * u_count * threads;
+                ++n;
+            }
+        return off;
+    }
+    static constexpr __host__ __device__ int stage_bytes(int u_count, int threads) { return stage_offset(1 << 20, u_count, threads); }
+    // Programs that generate random bits are bound by integer issue, not by the wait for their inputs:
+    // the staging copies would only add instructions.
+    static constexpr __host__ __device__ bool integer_heavy() {
+        for (int k = 0; k < PG::n_ins; ++k)
+            if (PG::ins[k].op == OP_PHILOX) return true;
+        return false;
+    }
     static constexpr __host__ __device__ bool needs_coords() {
         for (int k = 0; k < PG::n_ins; ++k) {
             const uint32_t op = PG::ins[k].op;
@@ -70,12 +91,33 @@ __device__ __forceinline__ float f2c(float a, float b) {
     if constexpr (OP == F2_DIV || OP == F2_RDIV) {
         const float n = OP == F2_DIV ? a : b, d = OP == F2_DIV ? b : a;
         float r;
-        if constexpr (FLAV == 0) asm("div.approx.f32 %0, %1, %2;" : "=f"(r) : "f"(n), "f"(d));
+        // fast: numerator times approximate reciprocal (what div.approx computes); written as two operations
+        // so that the reciprocal of a broadcast divisor (a row sum) is formed once, not once per lane
+        if constexpr (FLAV == 0) r = __fmul_rn(n, rcp_approx(d));
         else if constexpr (FLAV == 1) asm("div.full.f32 %0, %1, %2;" : "=f"(r) : "f"(n), "f"(d));
         else r = __fdiv_rn(n, d);
         return r;
     } else {
         return f2<OP, false>(a, b);
+    }
+}
+
+// Two lanes at once.  Multiplications run as one packed mul.rn.f32x2 (each lane rounded separately, as
+// in the scalar form).  Additions and subtractions stay scalar on purpose: ptxas 12.9 fuses a packed
+// multiply that feeds a packed add into one packed fused multiply-add despite the explicit .rn on
+// both (measured: results equal fmaf, not the two roundings), which would break the one-rounding-
+// per-traced-op rule; a packed multiply feeding scalar adds is left alone.
+template <int OP, int FLAV>
+__device__ __forceinline__ void f2c_pair(float &a0, float &a1, float b0, float b1) {
+    if constexpr (OP == F2_MUL) {
+        uint64_t a, b, r;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
+        asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(b0), "f"(b1));
+        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(r));
+    } else {
+        a0 = f2c<OP, FLAV>(a0, b0);
+        a1 = f2c<OP, FLAV>(a1, b1);
     }
 }
 
@@ -182,6 +224,21 @@ __device__ __forceinline__ void chunk_store(const float (&a)[V], char *p) {
     }
 }
 
+// Asynchronous copies global -> shared, completion tracked per thread in commit groups.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait(uint32_t pending) {  // at most `pending` newest groups still in flight
+    if (pending == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");
+    else if (pending == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else if (pending == 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+    else asm volatile("cp.async.wait_group 3;" ::: "memory");
+}
+
 constexpr __host__ __device__ int esz_shift(int dt) { return dt == LT_ST_BF16 ? 1 : (dt == LT_ST_U8 ? 0 : 2); }
 
 // Coordinates of the U chunks a thread works on in one iteration.
@@ -195,7 +252,7 @@ struct Coords {
 
 // No row reductions in this shell.
 struct NoReduce {
-    template <int KIND, int U>
+    template <int KIND, int U, bool GUARD>
     __device__ __forceinline__ void operator()(float (&)[U][V], const bool (&)[U]) const {}
 };
 
@@ -204,7 +261,7 @@ struct GroupReduce {
     float *smem;     // 2 x 32 floats, alternating between consecutive reductions
     uint32_t group;  // threads per row
     uint32_t phase;
-    template <int KIND, int U>
+    template <int KIND, int U, bool GUARD>
     __device__ __forceinline__ void operator()(float (&acc)[U][V], const bool (&ok)[U]) {
         const float ident = KIND == 0 ? 0.0f : (KIND == 1 ? -INFINITY : INFINITY);
         float part[U];
@@ -213,7 +270,7 @@ struct GroupReduce {
             // pairwise over the eight lanes, then over the chunks
             float l0 = red_comb<KIND>(acc[u][0], acc[u][1]), l1 = red_comb<KIND>(acc[u][2], acc[u][3]);
             float l2 = red_comb<KIND>(acc[u][4], acc[u][5]), l3 = red_comb<KIND>(acc[u][6], acc[u][7]);
-            part[u] = ok[u] ? red_comb<KIND>(red_comb<KIND>(l0, l1), red_comb<KIND>(l2, l3)) : ident;
+            part[u] = (!GUARD || ok[u]) ? red_comb<KIND>(red_comb<KIND>(l0, l1), red_comb<KIND>(l2, l3)) : ident;
         }
 #pragma unroll
         for (int s = 1; s < U; s <<= 1)
@@ -249,7 +306,8 @@ struct GroupReduce {
 // ------------------------------------------------------------------ the machine
 // State and straight-line execution of program PG on U chunks at once.  `Ptr` gives the base
 // pointer of a slot, `Scal` the 32-bit immediates.
-template <class PG, int U, class Ptr, class Scal, class Red>
+// GUARD false: every chunk of every iteration exists, so validity tests disappear.
+template <class PG, int U, class Ptr, class Scal, class Red, bool GUARD = true>
 struct Machine {
     using I = Info<PG>;
     static constexpr int FLAV = PG::flavour;
@@ -305,10 +363,67 @@ struct Machine {
                     constexpr int dt = PG::dtype[slot];
 #pragma unroll
                     for (int u = 0; u < U; ++u)
-                        if (ck.ok[u]) raw_load<dt>(raw[I::load_ordinal(K)][u], address<slot>(u), true);
+                        if (!GUARD || ck.ok[u]) raw_load<dt>(raw[I::load_ordinal(K)][u], address<slot>(u), true);
                 }
             }
             issue_loads<K + 1>();
+        }
+    }
+
+    // Pipeline stage of the row shell.  stage_issue starts the asynchronous copies of an iteration's
+    // full-class inputs into the stage at shared address `stage`; stage_fetch moves a landed stage into
+    // the registers issue_loads would have filled.  A thread reads back only what it copied itself.
+    template <int THREADS, int K = PG::n_pro>
+    static __device__ __forceinline__ void stage_issue(const Ptr &ptr, const uint64_t (&flat0)[U], const bool (&ok)[U], uint32_t stage) {
+        if constexpr (K < PG::n_ins) {
+            constexpr uint32_t op = PG::ins[K].op;
+            if constexpr (I::is_ld(op) || I::is_f2m(op)) {
+                constexpr int slot = PG::ins[K].imm;
+                if constexpr (PG::cls[slot] == LT_CLS_FULL) {
+                    constexpr int cb = I::chunk_bytes(slot), sh = esz_shift(PG::dtype[slot]);
+                    constexpr int off = I::stage_offset(I::load_ordinal(K), U, THREADS);
+                    const char *base = reinterpret_cast<const char *>(ptr(slot));
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (GUARD && !ok[u]) continue;
+                        const char *src = base + (flat0[u] << sh);
+                        if constexpr (cb == 8) {
+                            cp_async8(stage + off + (u * THREADS + threadIdx.x) * 8, src);
+                        } else {
+                            cp_async16(stage + off + (u * THREADS + threadIdx.x) * 16, src);
+                            if constexpr (cb == 32) cp_async16(stage + off + ((U + u) * THREADS + threadIdx.x) * 16, src + 16);
+                        }
+                    }
+                }
+            }
+            stage_issue<THREADS, K + 1>(ptr, flat0, ok, stage);
+        }
+    }
+
+    template <int THREADS, int K = PG::n_pro>
+    __device__ __forceinline__ void stage_fetch(const unsigned char *stage) {
+        if constexpr (K < PG::n_ins) {
+            constexpr uint32_t op = PG::ins[K].op;
+            if constexpr (I::is_ld(op) || I::is_f2m(op)) {
+                constexpr int slot = PG::ins[K].imm;
+                if constexpr (PG::cls[slot] == LT_CLS_FULL) {
+                    constexpr int cb = I::chunk_bytes(slot);
+                    constexpr int ord = I::load_ordinal(K);
+                    const unsigned char *b = stage + I::stage_offset(ord, U, THREADS);
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if constexpr (cb == 8) {
+                            const uint2 w = *reinterpret_cast<const uint2 *>(b + (u * THREADS + threadIdx.x) * 8);
+                            raw[ord][u].a.x = w.x;
+                            raw[ord][u].a.y = w.y;
+                        } else {
+                            raw[ord][u].a = *reinterpret_cast<const uint4 *>(b + (u * THREADS + threadIdx.x) * 16);
+                            if constexpr (cb == 32) raw[ord][u].b = *reinterpret_cast<const uint4 *>(b + ((U + u) * THREADS + threadIdx.x) * 16);
+                        }
+                    }
+                }
+            }
+            stage_fetch<THREADS, K + 1>(stage);
         }
     }
 
@@ -359,7 +474,7 @@ struct Machine {
             static_assert(PG::cls[imm] == LT_CLS_FULL, "compiled programs store full-class results only");
 #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (ck.ok[u]) chunk_store<PG::dtype[imm]>(acc[u], const_cast<char *>(address<imm>(u)));
+                if (!GUARD || ck.ok[u]) chunk_store<PG::dtype[imm]>(acc[u], const_cast<char *>(address<imm>(u)));
         } else if constexpr (op == OP_IOTA_COL) {
 #pragma unroll
             for (int u = 0; u < U; ++u)
@@ -373,21 +488,48 @@ struct Machine {
                 for (int i = 0; i < V; ++i) acc[u][i] = u2f(r);
             }
         } else if constexpr (op == OP_PHILOX) {
+            // Philox4x32-10 (Salmon et al., SC'11).  A chunk starts on a multiple of eight elements, so it
+            // takes the four words of counter blocks flat0/4 and flat0/4 + 1.  All 2U blocks of the thread
+            // advance round by round together: they share the key schedule and give the scheduler 2U
+            // independent multiply chains.
+            uint32_t c[2 * U][4];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                // chunks start on a multiple of eight elements: two counter blocks, four words each
                 const uint64_t q = ck.flat0[u] >> 2;
-                uint32_t a[4], b[4];
-                philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), scal(imm + 2), scal(imm + 3), scal(imm), scal(imm + 1), a);
-                philox4x32_10((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), scal(imm + 2), scal(imm + 3), scal(imm), scal(imm + 1), b);
+                c[2 * u][0] = (uint32_t)q; c[2 * u][1] = (uint32_t)(q >> 32);
+                c[2 * u + 1][0] = (uint32_t)(q + 1); c[2 * u + 1][1] = (uint32_t)((q + 1) >> 32);
+                c[2 * u][2] = c[2 * u + 1][2] = scal(imm + 2);
+                c[2 * u][3] = c[2 * u + 1][3] = scal(imm + 3);
+            }
+            uint32_t k0 = scal(imm), k1 = scal(imm + 1);
+#pragma unroll
+            for (int r = 0; r < 10; ++r) {
+#pragma unroll
+                for (int b = 0; b < 2 * U; ++b) {
+                    const uint32_t hi0 = __umulhi(0xD2511F53u, c[b][0]), lo0 = 0xD2511F53u * c[b][0];
+                    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c[b][2]), lo1 = 0xCD9E8D57u * c[b][2];
+                    c[b][0] = hi1 ^ c[b][1] ^ k0;
+                    c[b][1] = lo1;
+                    c[b][2] = hi0 ^ c[b][3] ^ k1;
+                    c[b][3] = lo0;
+                }
+                k0 += 0x9E3779B9u;
+                k1 += 0xBB67AE85u;
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    acc[u][i] = u2f(a[i]);
-                    acc[u][4 + i] = u2f(b[i]);
+                    acc[u][i] = u2f(c[2 * u][i]);
+                    acc[u][4 + i] = u2f(c[2 * u + 1][i]);
                 }
-            }
         } else if constexpr (op >= OP_RED_SUM && op <= OP_RED_MIN) {
-            red.template operator()<op - OP_RED_SUM, U>(acc, ck.ok);
+            red.template operator()<op - OP_RED_SUM, U, GUARD>(acc, ck.ok);
+        } else if constexpr (op == OP_U_SQUARE) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int i = 0; i < V; i += 2) f2c_pair<F2_MUL, FLAV>(acc[u][i], acc[u][i + 1], acc[u][i], acc[u][i + 1]);
         } else if constexpr (op >= OP_U_NEG && op <= OP_C_NZI) {
 #pragma unroll
             for (int u = 0; u < U; ++u)
@@ -408,7 +550,7 @@ struct Machine {
                 float m[V];
                 operand_of<K>(m, u);
 #pragma unroll
-                for (int i = 0; i < V; ++i) acc[u][i] = f2c<f, FLAV>(acc[u][i], m[i]);
+                for (int i = 0; i < V; i += 2) f2c_pair<f, FLAV>(acc[u][i], acc[u][i + 1], m[i], m[i + 1]);
             }
         } else if constexpr (op >= OP_F2 && op < OP_I2) {
             constexpr int idx = (op - OP_F2) / LT_VM_NSRC, src = (op - OP_F2) % LT_VM_NSRC;
@@ -417,7 +559,7 @@ struct Machine {
                 float m[V];
                 source<src, imm>(m, u);
 #pragma unroll
-                for (int i = 0; i < V; ++i) acc[u][i] = f2c<idx, FLAV>(acc[u][i], m[i]);
+                for (int i = 0; i < V; i += 2) f2c_pair<idx, FLAV>(acc[u][i], acc[u][i + 1], m[i], m[i + 1]);
             }
         } else if constexpr (op >= OP_I2 && op < OP_CMP) {
             constexpr int idx = (op - OP_I2) / LT_VM_NSRC, src = (op - OP_I2) % LT_VM_NSRC;
@@ -484,6 +626,9 @@ struct PtrM {
     __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[base + s]; }
 };
 
+struct TrueTag { static constexpr bool value = true; };
+struct FalseTag { static constexpr bool value = false; };
+
 // ------------------------------------------------------------------ shells
 // Elementwise: chunk c of U-tuples strides through the tensor; rows are a multiple of the chunk.
 template <class PG, int U>
@@ -517,18 +662,23 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_ew(const __grid_constant__ LtK
 }
 
 // Row reductions: thread `gl` of a row's group owns chunks gl, gl + group, ... of the row.
+// With `depth` > 0 the full-class inputs of the CTA's next `depth` blocks of rows are in flight as
+// asynchronous copies into a ring of shared-memory stages while the current block is computed.
 template <class PG, int U>
-__global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant__ LtKParams P, uint32_t group, uint32_t group_log2) {
+__global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant__ LtKParams P, uint32_t group, uint32_t group_log2,
+                                                          uint32_t depth) {
     __shared__ float red_buf[64];
+    extern __shared__ __align__(16) unsigned char stage_mem[];
+    using M = Machine<PG, U, PtrK, ScalK, GroupReduce>;
+    constexpr uint32_t STAGE = Info<PG>::stage_bytes(U, C_ROW_THREADS);
     const PtrK ptr{P};
     const ScalK scal{P};
     GroupReduce red{red_buf, group, 0u};
     const uint32_t rows_per_cta = blockDim.x >> group_log2;
     const uint32_t row_blocks = (P.rows + rows_per_cta - 1u) / rows_per_cta;
     const uint32_t sub = threadIdx.x >> group_log2, gl = threadIdx.x & (group - 1u);
-    for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
+    auto coords_of = [&](uint32_t rb, Coords<U> &ck) {
         const uint32_t row = rb * rows_per_cta + sub;
-        Coords<U> ck;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             ck.row[u] = row;
@@ -536,10 +686,50 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
             ck.ok[u] = row < P.rows && ck.col0[u] < P.cols;
             ck.flat0[u] = (uint64_t)row * P.cols + ck.col0[u];
         }
-        Machine<PG, U, PtrK, ScalK, GroupReduce> m(ptr, scal, red, ck);
-        m.issue_loads();
-        m.run();
+    };
+    const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(stage_mem);
+    if (depth) {  // requires blockDim.x == C_ROW_THREADS
+        uint32_t rb = blockIdx.x;
+        for (uint32_t d = 0; d < depth; ++d, rb += gridDim.x) {
+            if (rb < row_blocks) {
+                Coords<U> nx;
+                coords_of(rb, nx);
+                M::template stage_issue<C_ROW_THREADS>(ptr, nx.flat0, nx.ok, stage0 + d * STAGE);
+            }
+            cp_async_commit();
+        }
     }
+    // every thread owns U whole chunks of an existing row in every iteration: no validity tests
+    const bool full = (P.rows % rows_per_cta) == 0 && group * U * V == P.cols;
+    uint32_t s = 0;
+    auto iterate = [&](auto guard_tag) {
+        constexpr bool GUARD = decltype(guard_tag)::value;
+        using MG = Machine<PG, U, PtrK, ScalK, GroupReduce, GUARD>;
+        for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
+            Coords<U> ck;
+            coords_of(rb, ck);
+            MG m(ptr, scal, red, ck);
+            if (depth) {
+                cp_async_wait(depth - 1);
+                m.template stage_fetch<C_ROW_THREADS>(stage_mem + s * STAGE);
+                // the stage just read is refilled with the block `depth` iterations ahead
+                const uint32_t rn = rb + depth * gridDim.x;
+                if (rn < row_blocks) {
+                    Coords<U> nx;
+                    coords_of(rn, nx);
+                    MG::template stage_issue<C_ROW_THREADS>(ptr, nx.flat0, nx.ok, stage0 + s * STAGE);
+                }
+                cp_async_commit();
+                s = s + 1 == depth ? 0 : s + 1;
+            } else {
+                m.issue_loads();
+            }
+            m.run();
+        }
+    };
+    if (full) iterate(FalseTag{});
+    else iterate(TrueTag{});
+    if (depth) cp_async_wait(0);
 }
 
 // Multi-tensor: every tensor is a flat range of chunks; a super-chunk is 2048 consecutive chunks.
@@ -590,19 +780,35 @@ bool same_program(const LtIns *ins, uint32_t n_ins, uint32_t n_pro, const uint8_
     return true;
 }
 
+inline cudaError_t row_smem_attr(const void *kernel, size_t dyn) {
+    // opt in to more than 48 KB of dynamic shared memory; per kernel, cheap enough to repeat per launch
+    return dyn > 32u * 1024u ? cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) : cudaSuccess;
+}
+
+
+template <class PG, int U>
+cudaError_t launch_row(const LtKParams &P, unsigned grid, unsigned threads, unsigned group, unsigned group_log2, unsigned depth,
+                       cudaStream_t stream) {
+    const size_t dyn = (size_t)depth * Info<PG>::stage_bytes(U, C_ROW_THREADS);
+    cudaError_t e = row_smem_attr((const void *)lt_c_row<PG, U>, dyn);
+    if (e != cudaSuccess) return e;
+    lt_c_row<PG, U><<<grid, threads, dyn, stream>>>(P, group, group_log2, depth);
+    return cudaGetLastError();
+}
+
 template <class PG>
 cudaError_t launch_one(const void *params, int u, unsigned grid, unsigned threads, unsigned group, unsigned group_log2,
-                       cudaStream_t stream) {
+                       unsigned depth, cudaStream_t stream) {
     if constexpr (PG::kind == 0) {
         const LtKParams &P = *static_cast<const LtKParams *>(params);
         if (u >= 2) lt_c_ew<PG, 2><<<grid, C_THREADS, 0, stream>>>(P);
         else lt_c_ew<PG, 1><<<grid, C_THREADS, 0, stream>>>(P);
     } else if constexpr (PG::kind == 1) {
         const LtKParams &P = *static_cast<const LtKParams *>(params);
-        if (u >= 8) lt_c_row<PG, 8><<<grid, threads, 0, stream>>>(P, group, group_log2);
-        else if (u >= 4) lt_c_row<PG, 4><<<grid, threads, 0, stream>>>(P, group, group_log2);
-        else if (u >= 2) lt_c_row<PG, 2><<<grid, threads, 0, stream>>>(P, group, group_log2);
-        else lt_c_row<PG, 1><<<grid, threads, 0, stream>>>(P, group, group_log2);
+        if (u >= 8) return launch_row<PG, 8>(P, grid, threads, group, group_log2, depth, stream);
+        if (u >= 4) return launch_row<PG, 4>(P, grid, threads, group, group_log2, depth, stream);
+        if (u >= 2) return launch_row<PG, 2>(P, grid, threads, group, group_log2, depth, stream);
+        return launch_row<PG, 1>(P, grid, threads, group, group_log2, depth, stream);
     } else {
         const LtMultiParams &P = *static_cast<const LtMultiParams *>(params);
         if (u >= 2) lt_c_multi<PG, 2><<<grid, C_THREADS, 0, stream>>>(P);
@@ -611,16 +817,23 @@ cudaError_t launch_one(const void *params, int u, unsigned grid, unsigned thread
     return cudaGetLastError();
 }
 
+template <class PG, int U>
+cudaError_t row_occupancy(int threads, size_t dyn, int *blocks) {
+    cudaError_t e = row_smem_attr((const void *)lt_c_row<PG, U>, dyn);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, U>, threads, dyn);
+}
+
 template <class PG>
-cudaError_t occupancy_one(int u, int threads, int *blocks) {
+cudaError_t occupancy_one(int u, int threads, size_t dyn, int *blocks) {
     if constexpr (PG::kind == 0) {
         return u >= 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_ew<PG, 2>, C_THREADS, 0)
                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_ew<PG, 1>, C_THREADS, 0);
     } else if constexpr (PG::kind == 1) {
-        if (u >= 8) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 8>, threads, 0);
-        if (u >= 4) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 4>, threads, 0);
-        if (u >= 2) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 2>, threads, 0);
-        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_row<PG, 1>, threads, 0);
+        if (u >= 8) return row_occupancy<PG, 8>(threads, dyn, blocks);
+        if (u >= 4) return row_occupancy<PG, 4>(threads, dyn, blocks);
+        if (u >= 2) return row_occupancy<PG, 2>(threads, dyn, blocks);
+        return row_occupancy<PG, 1>(threads, dyn, blocks);
     } else {
         return u >= 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_multi<PG, 2>, C_THREADS, 0)
                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_multi<PG, 1>, C_THREADS, 0);
@@ -640,12 +853,34 @@ int lt_compiled_find(int kind, int flavour, const LtIns *ins, uint32_t n_ins, ui
     return -1;
 }
 
+int lt_compiled_prefers_staging(int id) {
+    int k = 0;
+#define LT_X(PG)                                            \
+    if (k == id) return Info<PG>::integer_heavy() ? 0 : 1; \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return 0;
+}
+
 int lt_compiled_count(void) {
     int n = 0;
 #define LT_X(PG) ++n;
     LT_COMPILED_LIST(LT_X)
 #undef LT_X
     return n;
+}
+
+size_t lt_compiled_row_stage_bytes(int id, int u) {
+    int k = 0;
+#define LT_X(PG)                                                                                                        \
+    if (k == id)                                                                                                        \
+        return (size_t)(u >= 8 ? Info<PG>::stage_bytes(8, C_ROW_THREADS) : u >= 4 ? Info<PG>::stage_bytes(4, C_ROW_THREADS) \
+                        : u >= 2 ? Info<PG>::stage_bytes(2, C_ROW_THREADS) : Info<PG>::stage_bytes(1, C_ROW_THREADS)); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return 0;
 }
 
 const char *lt_compiled_name(int id) {
@@ -659,20 +894,20 @@ const char *lt_compiled_name(int id) {
 }
 
 cudaError_t lt_compiled_launch(int id, const void *params, int u, unsigned grid, unsigned threads, unsigned group,
-                               unsigned group_log2, cudaStream_t stream) {
+                               unsigned group_log2, unsigned depth, cudaStream_t stream) {
     int k = 0;
 #define LT_X(PG)                                                                                \
-    if (k == id) return launch_one<PG>(params, u, grid, threads, group, group_log2, stream); \
+    if (k == id) return launch_one<PG>(params, u, grid, threads, group, group_log2, depth, stream); \
     ++k;
     LT_COMPILED_LIST(LT_X)
 #undef LT_X
     return cudaErrorInvalidValue;
 }
 
-cudaError_t lt_compiled_occupancy(int id, int u, int threads, int *blocks) {
+cudaError_t lt_compiled_occupancy(int id, int u, int threads, size_t dyn_smem, int *blocks) {
     int k = 0;
 #define LT_X(PG)                                                  \
-    if (k == id) return occupancy_one<PG>(u, threads, blocks); \
+    if (k == id) return occupancy_one<PG>(u, threads, dyn_smem, blocks); \
     ++k;
     LT_COMPILED_LIST(LT_X)
 #undef LT_X

@@ -14,6 +14,11 @@ const char *lt_compiled_name(int id);
 // `u`: chunks of eight elements a thread keeps in flight (elementwise, multi: 1 or 2; row: 1, 2, 4 or 8).
 // `params` points at the LtKParams (elementwise, row) or LtMultiParams block.  Row launches: `threads` per
 // CTA and the power-of-two `group` of threads that owns a row.
+// `depth`: row launches with 128-thread CTAs may keep the inputs of the next `depth` (1..4) blocks of rows in
+// flight in shared memory (depth x lt_compiled_row_stage_bytes of dynamic shared memory); 0 = load directly.
 cudaError_t lt_compiled_launch(int id, const void *params, int u, unsigned grid, unsigned threads, unsigned group,
-                               unsigned group_log2, cudaStream_t stream);
-cudaError_t lt_compiled_occupancy(int id, int u, int threads, int *blocks_per_sm);
+                               unsigned group_log2, unsigned depth, cudaStream_t stream);
+cudaError_t lt_compiled_occupancy(int id, int u, int threads, size_t dyn_smem, int *blocks_per_sm);
+size_t lt_compiled_row_stage_bytes(int id, int u);
+// 1 if the entry's row kernel gains from the shared-memory staging pipeline (0: issue-bound programs).
+int lt_compiled_prefers_staging(int id);

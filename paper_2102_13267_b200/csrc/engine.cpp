@@ -1,4 +1,5 @@
 // Recorder, liveness arena and the C ABI (lazytensor.h).
+#include "compiled.h"
 #include "engine.h"
 #include "launch.h"
 
@@ -339,6 +340,8 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "stage")) c->opt.stage = value;
     else if (!strcmp(key, "compiled")) c->opt.compiled = value;
     else if (!strcmp(key, "compiled_u")) c->opt.compiled_u = value;
+    else if (!strcmp(key, "compiled_row_u")) c->opt.compiled_row_u = value;
+    else if (!strcmp(key, "compiled_depth")) c->opt.compiled_depth = value;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
 }

@@ -148,8 +148,10 @@ struct Plan {
 };
 
 struct Options {
-    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 1, stage = 3;
+    int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 0, stage = 3;  // waves: 0 = each kernel's default (1; compiled multi-tensor 2)
     int64_t compiled = 1;  // use the ahead-of-time compiled kernel of a program when the table has one
+    int64_t compiled_row_u = 0;  // chunks per thread in compiled row kernels (0 = one warp per row where it fits)
+    int64_t compiled_depth = -1;  // staging depth of compiled row kernels (-1 = default, 0 = direct loads)
     int64_t compiled_u = 0;  // chunks in flight per thread in compiled elementwise / multi kernels (0 = default)
 };
 

@@ -52,12 +52,12 @@ cudaEvent_t take_event(lt_ctx *c) {
 bool aligned_for(uint64_t p, uint8_t dtype) { return (p & (dtype == LT_U8 ? 7u : 15u)) == 0; }
 
 // resident blocks per SM of a compiled kernel variant, asked once per plan launch
-int compiled_blocks(Launch &L, int u, int threads) {
+int compiled_blocks(Launch &L, int u, int threads, size_t dyn = 0) {
     int lg = 0;
     while ((1 << lg) < u) ++lg;
     if (L.compiled_blocks[lg] == 0) {
         int b = 0;
-        if (lt_compiled_occupancy(L.compiled, u, threads, &b) != cudaSuccess || b < 1) {
+        if (lt_compiled_occupancy(L.compiled, u, threads, dyn, &b) != cudaSuccess || b < 1) {
             cudaGetLastError();
             b = 1;
         }
@@ -199,12 +199,15 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     for (size_t s = 0; s < slots && ok; ++s) ok = aligned_for(P.ptr[k * slots + s], g0.io[s].dtype);
                 }
                 if (ok) {
-                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 1;
+                    // two chunks in flight per thread and two waves of blocks measured best for wide programs
+                    // (four input streams) over many tensors of uneven size
+                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 2;
                     const int occ = compiled_blocks(L, u, LT_EW_THREADS);
-                    unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * waves);
+                    const unsigned mwaves = c->opt.waves > 0 ? waves : 2u;
+                    unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * mwaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, c->stream);
+                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, 0, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     c->stats.launches_compiled++;
                     done = true;
@@ -278,22 +281,30 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * occ * waves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, c->stream);
+                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, 0, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     done = true;
                 } else if (ok && P.cpr <= 8u * 1024u) {
                     // a row lives in the registers of its thread group: up to 8 chunks per thread, one warp per row if it fits
                     int u = 1;
                     while (u < 8 && P.cpr > 32u * u) u *= 2;
+                    if (c->opt.compiled_row_u > 0) u = (int)c->opt.compiled_row_u;
+                    while (u < 8 && P.cpr > 128u * u) u *= 2;  // a row's group is at most one CTA of 128 threads
                     unsigned grp = 1, lg = 0;
                     while (grp * u < P.cpr) grp <<= 1, ++lg;
                     const unsigned threads = grp > 128 ? grp : 128;
-                    const int occ = compiled_blocks(L, u, (int)threads);
+                    // pipeline depth: stages of the next blocks' inputs in shared memory, within ~72 KB per CTA
+                    const size_t stage = lt_compiled_row_stage_bytes(L.compiled, u);
+                    unsigned depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth
+                                                                       : (lt_compiled_prefers_staging(L.compiled) ? 2u : 0u);
+                    while (depth > 0 && depth * stage > 72u * 1024u) --depth;
+                    if (stage == 0 || threads != 128 || depth < 2) depth = 0;
+                    const int occ = compiled_blocks(L, u, (int)threads, depth * stage);
                     const uint64_t blocks = ((uint64_t)P.rows + threads / grp - 1) / (threads / grp);
                     unsigned grid = (unsigned)std::min<uint64_t>(blocks, (uint64_t)c->sm_count * occ * waves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch(L.compiled, &P, u, grid, threads, grp, lg, c->stream);
+                    e = lt_compiled_launch(L.compiled, &P, u, grid, threads, grp, lg, depth, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     done = true;
                 }
