@@ -67,13 +67,6 @@ struct Info {
         return off;
     }
     static constexpr __host__ __device__ int stage_bytes(int u_count, int threads) { return stage_offset(1 << 20, u_count, threads); }
-    // Programs that generate random bits are bound by integer issue, not by the wait for their inputs:
-    // the staging copies would only add instructions.
-    static constexpr __host__ __device__ bool integer_heavy() {
-        for (int k = 0; k < PG::n_ins; ++k)
-            if (PG::ins[k].op == OP_PHILOX) return true;
-        return false;
-    }
     static constexpr __host__ __device__ bool needs_coords() {
         for (int k = 0; k < PG::n_ins; ++k) {
             const uint32_t op = PG::ins[k].op;
@@ -851,16 +844,6 @@ int lt_compiled_find(int kind, int flavour, const LtIns *ins, uint32_t n_ins, ui
     LT_COMPILED_LIST(LT_X)
 #undef LT_X
     return -1;
-}
-
-int lt_compiled_prefers_staging(int id) {
-    int k = 0;
-#define LT_X(PG)                                            \
-    if (k == id) return Info<PG>::integer_heavy() ? 0 : 1; \
-    ++k;
-    LT_COMPILED_LIST(LT_X)
-#undef LT_X
-    return 0;
 }
 
 int lt_compiled_count(void) {

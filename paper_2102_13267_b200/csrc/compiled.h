@@ -20,5 +20,3 @@ cudaError_t lt_compiled_launch(int id, const void *params, int u, unsigned grid,
                                unsigned group_log2, unsigned depth, cudaStream_t stream);
 cudaError_t lt_compiled_occupancy(int id, int u, int threads, size_t dyn_smem, int *blocks_per_sm);
 size_t lt_compiled_row_stage_bytes(int id, int u);
-// 1 if the entry's row kernel gains from the shared-memory staging pipeline (0: issue-bound programs).
-int lt_compiled_prefers_staging(int id);

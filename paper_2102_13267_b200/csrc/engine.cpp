@@ -237,8 +237,11 @@ void buffer_unref(lt_ctx *c, uint32_t b) {
     c->free_buffers.push_back(b);
 }
 
-void *ctx_alloc(lt_ctx *c, size_t bytes) {
-    if (bytes == 0) bytes = 16;
+// Device memory of the context.  Blocks the library has released are kept in a per-size pool (up to
+// `pool_bytes` in total) and handed out again before the allocator is asked: everything runs on one
+// stream, so a block freed after the last kernel using it was enqueued can be reused by the next
+// flush at once.  In steady state (same graph every step) a flush makes no allocator call at all.
+static void *raw_alloc(lt_ctx *c, size_t bytes) {
     if (c->has_alloc) return c->alloc.alloc(bytes, (void *)c->stream, c->alloc.user);
     if (c->device == LT_DEVICE_NONE) return malloc(bytes);
     void *p = nullptr;
@@ -249,11 +252,54 @@ void *ctx_alloc(lt_ctx *c, size_t bytes) {
     return p;
 }
 
-void ctx_free(lt_ctx *c, void *p) {
-    if (!p) return;
+static void raw_free(lt_ctx *c, void *p) {
     if (c->has_alloc) c->alloc.free(p, (void *)c->stream, c->alloc.user);
     else if (c->device == LT_DEVICE_NONE) free(p);
     else cudaFreeAsync(p, c->stream);
+}
+
+void pool_trim(lt_ctx *c, size_t keep_bytes) {
+    for (auto it = c->pool.begin(); it != c->pool.end() && c->pool_held > keep_bytes;) {
+        std::vector<void *> &v = it->second;
+        while (!v.empty() && c->pool_held > keep_bytes) {
+            c->block_size.erase(v.back());
+            raw_free(c, v.back());
+            v.pop_back();
+            c->pool_held -= it->first;
+        }
+        it = v.empty() ? c->pool.erase(it) : std::next(it);
+    }
+}
+
+void *ctx_alloc(lt_ctx *c, size_t bytes) {
+    if (bytes == 0) bytes = 16;
+    bytes = (bytes + 511u) & ~(size_t)511u;
+    auto it = c->pool.find(bytes);
+    if (it != c->pool.end() && !it->second.empty()) {
+        void *p = it->second.back();
+        it->second.pop_back();
+        c->pool_held -= bytes;
+        return p;
+    }
+    void *p = raw_alloc(c, bytes);
+    if (!p && c->pool_held) {  // give the pooled blocks back and try once more
+        pool_trim(c, 0);
+        p = raw_alloc(c, bytes);
+    }
+    if (p) c->block_size[p] = bytes;
+    return p;
+}
+
+void ctx_free(lt_ctx *c, void *p) {
+    if (!p) return;
+    auto it = c->block_size.find(p);
+    if (it != c->block_size.end() && c->opt.pool_bytes > 0 && c->pool_held + it->second <= (size_t)c->opt.pool_bytes) {
+        c->pool[it->second].push_back(p);
+        c->pool_held += it->second;
+        return;
+    }
+    if (it != c->block_size.end()) c->block_size.erase(it);
+    raw_free(c, p);
 }
 
 }  // namespace lt
@@ -324,6 +370,7 @@ lt_status lt_ctx_destroy(lt_ctx *c) {
     for (auto e : c->event_pool) cudaEventDestroy(e);
     for (auto &b : c->buffers)
         if (b.owned && b.ptr && b.refs > 0) ctx_free(c, b.ptr);
+    pool_trim(c, 0);
     delete c;
     return LT_OK;
 }
@@ -338,6 +385,10 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "ieee")) c->opt.ieee = value;
     else if (!strcmp(key, "waves")) c->opt.waves = value;
     else if (!strcmp(key, "stage")) c->opt.stage = value;
+    else if (!strcmp(key, "pool_bytes")) {
+        c->opt.pool_bytes = value;
+        pool_trim(c, value > 0 ? (size_t)value : 0);
+    }
     else if (!strcmp(key, "compiled")) c->opt.compiled = value;
     else if (!strcmp(key, "compiled_u")) c->opt.compiled_u = value;
     else if (!strcmp(key, "compiled_row_u")) c->opt.compiled_row_u = value;

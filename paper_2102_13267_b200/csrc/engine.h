@@ -149,6 +149,7 @@ struct Plan {
 
 struct Options {
     int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 0, stage = 3;  // waves: 0 = each kernel's default (1; compiled multi-tensor 2)
+    int64_t pool_bytes = 4ll << 30;  // released device blocks the context keeps for reuse (0 = return every block at once)
     int64_t compiled = 1;  // use the ahead-of-time compiled kernel of a program when the table has one
     int64_t compiled_row_u = 0;  // chunks per thread in compiled row kernels (0 = one warp per row where it fits)
     int64_t compiled_depth = -1;  // staging depth of compiled row kernels (-1 = default, 0 = direct loads)
@@ -208,6 +209,11 @@ struct lt_ctx {
     std::vector<lt::TimedLaunch> timed;
     std::vector<cudaEvent_t> event_pool;
 
+    // released device blocks by (rounded) size, and the size of every block obtained from the allocator
+    std::unordered_map<size_t, std::vector<void *>> pool;
+    std::unordered_map<void *, size_t> block_size;
+    size_t pool_held = 0;
+
     // scratch reused across barriers
     lt::Canonical canon;
     std::vector<uint32_t> roots_scratch, stack_scratch;
@@ -231,6 +237,7 @@ const char *op_name(int op);
 int64_t shape_numel(const int64_t *dims, int rank);
 lt_status fail(lt_ctx *c, lt_status s, const std::string &msg);
 void *ctx_alloc(lt_ctx *c, size_t bytes);
+void pool_trim(lt_ctx *c, size_t keep_bytes);
 void ctx_free(lt_ctx *c, void *p);
 
 // canonicaliser (canon.cpp)

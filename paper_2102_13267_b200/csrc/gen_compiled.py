@@ -66,6 +66,18 @@ def programs():
         g, be = (d.leaf((64,), "f32") for _ in range(2))
         keep = traces.residual_dropout_layernorm(d.ctx, x, h, g, be, shape=(16, 64), p=0.1, eps=1e-5, seed=1, offset=0, out_dtype=od)
         out.append((f"residual_dropout_layernorm_{od}", d.keys()))
+    # the same normalisation without dropout (evaluation mode)
+    d = Dry()
+    x, h = (d.leaf((16, 64), "bf16") for _ in range(2))
+    g, be = (d.leaf((64,), "f32") for _ in range(2))
+    t = d.ctx.op("add", d.ctx.op("convert", x, dtype="f32"), d.ctx.op("convert", h, dtype="f32"))
+    inv_c = d.ctx.scalar(1.0 / 64)
+    dev = d.ctx.op("sub", t, d.ctx.op("mul", d.ctx.op("row_sum", t), inv_c))
+    var = d.ctx.op("mul", d.ctx.op("row_sum", d.ctx.op("mul", dev, dev)), inv_c)
+    z = d.ctx.op("mul", dev, d.ctx.op("rsqrt", d.ctx.op("add", var, d.ctx.scalar(1e-5))))
+    keep = d.ctx.op("convert", d.ctx.op("add", d.ctx.op("mul", z, g), be), dtype="bf16")
+    del t, dev, var, z
+    out.append(("residual_layernorm_bf16", d.keys()))
     for od in ("bf16", "f32"):
         d = Dry()
         keep = traces.causal_softmax(d.ctx, d.leaf((2, 64, 64), "bf16"), shape=(2, 64, 64), scale=1 / math.sqrt(128), out_dtype=od)

@@ -43,6 +43,11 @@ def main() -> None:
     def bf16(shape, std=1.0):
         return (torch.randn(shape, device=dev) * std).to(torch.bfloat16)
 
+    def hold_gpu(ms=4.0):
+        """Keeps the stream busy for a few milliseconds so that the flushes recorded next queue up behind it and
+        then run back to back: the per-launch event brackets then hold kernel time, not the host's pace."""
+        torch.cuda._sleep(int(ms * 1e-3 * 1.9e9))
+
     def report(name, nbytes, ctx):
         kt = ctx.kernel_timing()
         ms = sum(v["ms"] for v in kt.values()) / args.iters
@@ -61,6 +66,7 @@ def main() -> None:
         torch.cuda.synchronize()
         ctx.set_kernel_timing(True)
         ctx.kernel_timing()
+        hold_gpu()
         for i in range(args.iters):
             keep[i % nsets] = trace(ctx, sets[i % nsets])
             ctx.barrier()
@@ -100,6 +106,7 @@ def main() -> None:
         ctx.set_kernel_timing(True)
         ctx.kernel_timing()
         for _ in range(args.iters):
+            hold_gpu(8.0)  # recording a step of 161 tensors takes the host a few milliseconds
             step += 1
             traces.adam_step(ctx, P, G, M, V, step=step)
             ctx.barrier()
