@@ -98,6 +98,18 @@ def test_c3_residual_dropout_layernorm(ctx, shape, out_dtype):
     assert (s["compiles"], s["cache_hits"]) == (1, 1)
 
 
+@pytest.mark.parametrize("shape", [(32, 256), (7, 48), (3, 1000), (5, 2048), (3, 8192), (2048, 1024)])
+def test_residual_layernorm_without_dropout(ctx, shape):
+    x, h, g, b = configs.c3_inputs(13, shape)
+    O, ol, gl = both(ctx, [(x, "bf16"), (h, "bf16"), (g, "f32"), (b, "f32")])
+    zr = traces.residual_layernorm(O, *ol, shape=shape, eps=1e-5)
+    z = traces.residual_layernorm(ctx, *gl, shape=shape, eps=1e-5)
+    ctx.barrier()
+    st = ctx.stats()
+    assert st["kernels_launched"] == 1 and st["launches_compiled"] == (1 if ctx.compiled_allowed else 0)
+    assert_matches(ctx.fetch(z), zr.array, "bf16", f"layernorm {shape}")
+
+
 # ------------------------------------------------------------------ C4
 @pytest.mark.parametrize("shape", [(2, 64, 64), (1, 130, 130), (3, 24, 24), (1, 8, 8), (2, 1000, 1000), (1, 4, 2048),
                                    (16, 2048, 2048)])

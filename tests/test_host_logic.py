@@ -360,3 +360,32 @@ def test_failed_allocation_leaves_the_graph_flushable():
     lib.lt_ctx_destroy.argtypes = [ctypes.c_void_p]
     assert lib.lt_ctx_destroy(c) == 0
     assert not live  # the output buffer went back through the free callback
+
+
+# ------------------------------------------------------------------ ahead-of-time compiled programs
+def test_compiled_table_is_what_the_planner_emits_today():
+    """The committed table of compiled programs equals what its generator derives from the planner now
+    (a planner change that alters a listed program must be followed by regenerating the table), and
+    planning a listed graph finds its entry."""
+    import importlib.util
+
+    path = os.path.join(ROOT, "paper_2102_13267_b200", "csrc", "gen_compiled.py")
+    spec = importlib.util.spec_from_file_location("gen_compiled", path)
+    gen = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(gen)
+    text, names = gen.render()
+    committed = open(os.path.join(ROOT, "paper_2102_13267_b200", "csrc", "compiled_programs.inc")).read()
+    assert text == committed, "run paper_2102_13267_b200/csrc/gen_compiled.py and rebuild"
+    assert len(names) >= 8
+    d = gen.Dry()
+    a, b, c, e = (d.leaf((64, 64), "f32") for _ in range(4))
+    keep = gen.traces.elementwise_chain(d.ctx, a, b, c, e)
+    d.ctx.barrier()
+    assert "compiled: elementwise_chain" in d.ctx.dump_plan()
+    # a graph that is not listed stays on the interpreter
+    d = gen.Dry()
+    a, b = (d.leaf((64, 64), "f32") for _ in range(2))
+    keep = d.ctx.op("max", d.ctx.op("sub", a, b), d.ctx.op("exp", b))
+    d.ctx.barrier()
+    assert "compiled: no" in d.ctx.dump_plan()
+    del keep

@@ -74,6 +74,20 @@ def residual_dropout_layernorm(B, x, h, gamma, beta, *, shape, p: float, eps: fl
     return z, keep
 
 
+def residual_layernorm(B, x, h, gamma, beta, *, shape, eps: float, out_dtype: str = "bf16"):
+    """z = LayerNorm(x + h) * gamma + beta over the last dim: the normalisation above without dropout."""
+    cols = shape[-1]
+    t = B.op("add", B.op("convert", x, dtype="f32"), B.op("convert", h, dtype="f32"))
+    inv_c = B.scalar(1.0 / cols)
+    d = B.op("sub", t, B.op("mul", B.op("row_sum", t), inv_c))
+    var = B.op("mul", B.op("row_sum", B.op("mul", d, d)), inv_c)
+    z = B.op("mul", d, B.op("rsqrt", B.op("add", var, B.scalar(eps))))
+    z = B.op("add", B.op("mul", z, gamma), beta)
+    if out_dtype != "f32":
+        z = B.op("convert", z, dtype=out_dtype)
+    return z
+
+
 def causal_softmax(B, scores, *, shape, scale: float, out_dtype: str = "bf16"):
     """softmax over the last dim of scores*scale with columns > row masked to -inf ([heads, q, k] input)."""
     s = B.op("convert", scores, dtype="f32")
