@@ -125,6 +125,7 @@ typedef struct {
     uint64_t ns_bind_launch;     /* argument binding, allocation and kernel launches         */
     uint64_t ns_rebind;          /* turning roots into device-data leaves, freeing IR        */
     uint64_t launches_compiled;  /* of kernels_launched: ahead-of-time compiled programs     */
+    uint64_t replays;            /* lt_replay calls that ran a plan                          */
 } lt_stats;
 
 /* Device time per kernel family, measured with CUDA events when kernel timing is on. */
@@ -220,6 +221,41 @@ lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
  * has pending computation.  With `blocking` non-zero, return after the stream has drained.
  */
 lt_status lt_barrier(lt_ctx *ctx, int blocking);
+
+/*
+ * Replay (Section 8, future work: "provide users with a way to guarantee that the underlying
+ * computation of a tensor is going to remain the same across steps", so that "the IR graph
+ * construction" can be skipped "after constructing it in the usual way during the first
+ * iteration").  lt_replay runs the graph of the previous successful lt_barrier again -- no
+ * recording, canonicalising or hashing -- as if the caller had issued the same lt_op / lt_assign
+ * calls on the same tensor handles once more:
+ *   - every input is the current value of the tensor that supplied it last time (for an in-place
+ *     update x := f(x, ...), the value the previous flush or replay left in x);
+ *   - every tensor that received a result receives the new result (in place where the previous
+ *     flush wrote in place, otherwise in fresh memory; its previous value is released);
+ *   - run-time scalars (lt_scalar with a value other than 0 or 1, lt_scalar_dynamic) are read again
+ *     from their tensors, so lt_scalar_set changes them between replays; the other run-time slots
+ *     (seed and offset of philox_bits) keep their values unless set with lt_replay_set_slot.
+ * LT_ERR_INVALID_ARG if operations are pending, if there is nothing to replay, or if one of those
+ * tensors has been released or no longer has the recorded shape; LT_ERR_UNSUPPORTED if an input of
+ * the previous flush was not named by any tensor (nothing to read the new value from) or an in-place
+ * result would now overwrite memory another tensor names.  Nothing has run in those cases: record
+ * the step with lt_op and flush it with lt_barrier instead.
+ */
+lt_status lt_replay(lt_ctx *ctx, int blocking);
+
+/* New value of a run-time scalar tensor (see lt_replay).  LT_ERR_INVALID_ARG for a handle that is not
+ * a run-time scalar, or while pending operations read it (flush them first). */
+lt_status lt_scalar_set(lt_ctx *ctx, lt_tensor scalar, double value);
+
+/* Number of run-time slots of the graph lt_replay would run (0 if none), in canonical order: each
+ * run-time scalar is one slot, each philox_bits op two (seed, offset). */
+lt_status lt_replay_slots(lt_ctx *ctx, uint32_t *n_slots);
+
+/* Sets run-time slot `slot` for the following replays: `as_integer` non-zero stores `ivalue` (64-bit
+ * patterns: seeds, offsets), else `dvalue`.  A slot supplied by a live scalar tensor is read from the
+ * tensor instead (use lt_scalar_set). */
+lt_status lt_replay_set_slot(lt_ctx *ctx, uint32_t slot, int as_integer, double dvalue, int64_t ivalue);
 
 /*
  * Barrier that obtains no device memory.  (The paper has no counterpart: its runtime always

@@ -55,7 +55,7 @@ class lt_stats(ctypes.Structure):
         "launches_elementwise", "launches_row", "launches_multi", "bytes_planned",
         "outputs_donated", "outputs_allocated", "temporaries_allocated",
         "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind",
-        "launches_compiled")]
+        "launches_compiled", "replays")]
 
 
 class lt_kernel_timing(ctypes.Structure):
@@ -79,6 +79,10 @@ _SIGNATURES = {
     "lt_release_many": [_vp, _P(_u64), ctypes.c_size_t],
     "lt_barrier": [_vp, _int],
     "lt_barrier_static_scratch": [_vp, _int, _int],
+    "lt_replay": [_vp, _int],
+    "lt_scalar_set": [_vp, _u64, ctypes.c_double],
+    "lt_replay_slots": [_vp, _P(ctypes.c_uint32)],
+    "lt_replay_set_slot": [_vp, ctypes.c_uint32, _int, ctypes.c_double, _i64],
     "lt_fetch": [_vp, _u64, _vp, ctypes.c_size_t],
     "lt_device_ptr": [_vp, _u64, _P(_vp)],
     "lt_tensor_info": [_vp, _u64, _P(_int), _P(_int), _P(_i64), _P(_int)],
@@ -346,6 +350,24 @@ class LazyContext:
         if st:
             self._keeps.extend(keeps)
             self._check(st)
+
+    def replay(self, blocking: bool = False) -> None:
+        """lt_replay: run the previously flushed graph again on the same tensors, without recording it."""
+        self._check(_lib.lt_replay(self._ctx, 1 if blocking else 0))
+
+    def scalar_set(self, scalar: LazyTensor, value: float) -> None:
+        self._check(_lib.lt_scalar_set(self._ctx, scalar.handle, float(value)))
+
+    def replay_slots(self) -> int:
+        n = ctypes.c_uint32()
+        self._check(_lib.lt_replay_slots(self._ctx, ctypes.byref(n)))
+        return n.value
+
+    def replay_set_slot(self, slot: int, value, integer: bool = False) -> None:
+        iv = int(value) if integer else 0
+        if iv >= (1 << 63):
+            iv -= 1 << 64
+        self._check(_lib.lt_replay_set_slot(self._ctx, slot, 1 if integer else 0, 0.0 if integer else float(value), iv))
 
     def barrier_static_scratch(self, blocking: bool = False, clear_first: bool = False) -> None:
         """lt_barrier_static_scratch: the flush for callers that may not allocate device memory (results go to

@@ -116,6 +116,54 @@ void release_donors(lt_ctx *c, const std::vector<uint32_t> &roots) {
     }
 }
 
+// Remembers, for lt_replay, which tensors the graph being flushed reads and writes.  Called after the
+// launches, while the root tensors still name their IR and their lt_assign donors.
+void record_replay(lt_ctx *c, Plan *plan, const Canonical &cg, const std::vector<uint32_t> &roots) {
+    ReplayRecord &r = c->replay;
+    r.plan = plan;
+    r.why_not.clear();
+    r.dyn = cg.dyn;
+    r.params.assign(cg.param_node.size(), ReplayRecord::ParamRef());
+    r.dyn_scalar.assign(cg.dyn.size(), ReplayRecord::Ref());
+    r.roots.clear();
+    // arena node -> a live tensor naming it (leaves read as they are, run-time scalars)
+    std::vector<uint32_t> &by_node = c->stack_scratch;  // reused as a map: node -> slot + 1
+    by_node.assign(c->nodes.size(), 0);
+    for (uint32_t slot = 0; slot < c->tensors.size(); ++slot)
+        if (c->tensors[slot].live) by_node[c->tensors[slot].node] = slot + 1;
+    auto ref_of = [c](uint32_t slot, ReplayRecord::Ref &ref) {
+        ref.slot = slot;
+        ref.gen = c->tensors[slot].gen;
+    };
+    for (size_t i = 0; i < cg.param_node.size(); ++i) {
+        const Node &leaf = c->nodes[cg.param_node[i]];
+        ReplayRecord::ParamRef &pr = r.params[i];
+        pr.dtype = leaf.dtype;
+        pr.rank = leaf.rank;
+        memcpy(pr.dims, leaf.dims, sizeof(pr.dims));
+        if (by_node[cg.param_node[i]]) {
+            ref_of(by_node[cg.param_node[i]] - 1, pr);
+            continue;
+        }
+        // an in-place update: the tensor that named this buffer before lt_assign
+        for (uint32_t slot : roots)
+            if (c->tensors[slot].donor == leaf.buffer) {
+                ref_of(slot, pr);
+                break;
+            }
+        if (pr.slot == NONE && r.why_not.empty()) r.why_not = "an input of the flushed graph was not named by any tensor";
+    }
+    for (const CNode &cn : cg.nodes)
+        if (cn.op == N_SCALAR && cn.dyn >= 0 && by_node[cn.arena]) ref_of(by_node[cn.arena] - 1, r.dyn_scalar[cn.dyn]);
+    for (uint32_t slot : roots) {
+        ReplayRecord::Root root;
+        ref_of(slot, root);
+        root.output = cg.nodes[c->nodes[c->tensors[slot].node].canon].output;
+        r.roots.push_back(root);
+    }
+    by_node.clear();
+}
+
 void put_text(const std::string &s, char *buf, size_t cap, size_t *need) {
     if (need) *need = s.size() + 1;
     if (buf && cap) {
@@ -760,8 +808,10 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
             if (!c->opt.verify ||
                 (p->canon_bytes.size() == cg.bytes.size() && !memcmp(p->canon_bytes.data(), cg.bytes.data(), cg.bytes.size())))
                 plan = p;
-            else
+            else {
+                if (c->replay.plan == p) c->replay.plan = nullptr;
                 c->cache.erase(it);  // a colliding entry: replace it below
+            }
         }
     }
     if (plan) {
@@ -783,6 +833,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
                 c->last_plan_text = describe_plan(*c->last_plan);
                 c->last_plan = nullptr;
             }
+            if (c->replay.plan == victim->second.get()) c->replay.plan = nullptr;
             c->cache.erase(victim);
         }
         plan = np.get();
@@ -819,6 +870,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
             new_nodes[k] = n;
         }
         gather_roots(c, roots, true);
+        record_replay(c, plan, cg, roots);
         for (uint32_t slot : roots) {
             TensorRec &t = c->tensors[slot];
             const Node &old = c->nodes[t.node];
@@ -838,6 +890,127 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
         cudaError_t e = cudaStreamSynchronize(c->stream);
         if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
     }
+    return LT_OK;
+}
+
+lt_status lt_replay(lt_ctx *c, int blocking) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    ReplayRecord &r = c->replay;
+    if (!r.plan) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: no flushed graph to replay");
+    if (!r.why_not.empty()) return fail(c, LT_ERR_UNSUPPORTED, "lt_replay: " + r.why_not);
+    std::vector<uint32_t> &roots = c->roots_scratch;
+    gather_roots(c, roots, false);
+    if (!roots.empty()) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: operations are pending; flush them with lt_barrier");
+    Plan *plan = r.plan;
+    auto live = [c](const ReplayRecord::Ref &ref) {
+        return ref.slot < c->tensors.size() && c->tensors[ref.slot].live && c->tensors[ref.slot].gen == ref.gen;
+    };
+    // parameters: the current value of the tensors that supplied them
+    Canonical &cg = c->canon;
+    cg.param_node.resize(r.params.size());
+    for (size_t i = 0; i < r.params.size(); ++i) {
+        const ReplayRecord::ParamRef &pr = r.params[i];
+        if (!live(pr)) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: an input tensor of the recorded step has been released");
+        const uint32_t n = c->tensors[pr.slot].node;
+        const Node &nd = c->nodes[n];
+        bool same = nd.op == N_DEVICE_DATA && nd.dtype == pr.dtype && nd.rank == pr.rank;
+        for (int k = 0; same && k < pr.rank; ++k) same = nd.dims[k] == pr.dims[k];
+        if (!same) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: an input tensor no longer has the recorded dtype and shape");
+        cg.param_node[i] = n;
+    }
+    for (const ReplayRecord::Root &root : r.roots)
+        if (!live(root)) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: a result tensor of the recorded step has been released");
+    // in-place results: the buffer must still be named by the receiving tensor alone
+    for (size_t k = 0; k < plan->outputs.size(); ++k) {
+        const int32_t p = plan->outputs[k].donated_param;
+        if (p < 0) continue;
+        const Node &leaf = c->nodes[cg.param_node[p]];
+        bool ok = leaf.tensor_refs == 1 && c->buffers[leaf.buffer].refs == 1;
+        bool receives = false;
+        for (const ReplayRecord::Root &root : r.roots)
+            if (root.output == (int32_t)k && root.slot == r.params[p].slot) receives = true;
+        if (!ok || !receives)
+            return fail(c, LT_ERR_UNSUPPORTED, "lt_replay: an in-place result would overwrite memory another tensor names");
+    }
+    // run-time values: scalars from their tensors, the rest as recorded or set
+    for (size_t k = 0; k < r.dyn.size(); ++k)
+        if (r.dyn_scalar[k].slot != NONE && live(r.dyn_scalar[k])) {
+            const Node &sn = c->nodes[c->tensors[r.dyn_scalar[k].slot].node];
+            if (sn.op == N_SCALAR) r.dyn[k].d = sn.sval;
+        }
+    cg.dyn = r.dyn;
+    plan->last_used = ++c->use_clock;
+    c->last_plan = plan;
+    {
+        Timer tm(c->stats.ns_bind_launch);
+        lt_status s = execute_plan(c, *plan, cg);
+        if (s) return s;
+    }
+    {
+        Timer tm(c->stats.ns_rebind);
+        const size_t n_out = plan->outputs.size();
+        std::vector<uint32_t> new_nodes(n_out);
+        for (size_t k = 0; k < n_out; ++k) {
+            const OutputPlan &op = plan->outputs[k];
+            uint32_t n = node_new(c);
+            Node &nd = c->nodes[n];
+            nd.op = N_DEVICE_DATA;
+            nd.dtype = op.dtype;
+            nd.rank = op.rank;
+            memcpy(nd.dims, op.dims, sizeof(nd.dims));
+            if (op.donated_param >= 0) {
+                uint32_t b = c->nodes[cg.param_node[op.donated_param]].buffer;
+                c->buffers[b].refs++;
+                nd.buffer = b;
+            } else {
+                nd.buffer = buffer_new(c, c->out_ptr[k], op.bytes, true);
+            }
+            nd.refs = 1;
+            new_nodes[k] = n;
+        }
+        for (const ReplayRecord::Root &root : r.roots) {
+            TensorRec &t = c->tensors[root.slot];
+            const uint32_t nn = new_nodes[root.output], old_id = t.node;
+            t.node = nn;
+            node_ref(c, nn);
+            c->nodes[nn].tensor_refs++;
+            c->nodes[old_id].tensor_refs--;
+            node_unref(c, old_id);
+        }
+        for (uint32_t n : new_nodes) node_unref(c, n);
+    }
+    c->stats.replays++;
+    if (blocking && c->device != LT_DEVICE_NONE) {
+        cudaError_t e = cudaStreamSynchronize(c->stream);
+        if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
+    }
+    return LT_OK;
+}
+
+lt_status lt_scalar_set(lt_ctx *c, lt_tensor scalar, double value) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    uint32_t slot;
+    lt_status s = lookup(c, scalar, &slot);
+    if (s) return s;
+    Node &nd = c->nodes[c->tensors[slot].node];
+    if (nd.op != N_SCALAR || !(nd.flags & NF_DYNAMIC))
+        return fail(c, LT_ERR_INVALID_ARG, "lt_scalar_set: not a run-time scalar (0 and 1 are part of the graph; use lt_scalar_dynamic)");
+    if (nd.refs != nd.tensor_refs) return fail(c, LT_ERR_INVALID_ARG, "lt_scalar_set: pending operations read this scalar; flush them first");
+    nd.sval = value;
+    return LT_OK;
+}
+
+lt_status lt_replay_slots(lt_ctx *c, uint32_t *n_slots) {
+    if (!c || !n_slots) return LT_ERR_INVALID_ARG;
+    *n_slots = c->replay.plan ? (uint32_t)c->replay.dyn.size() : 0u;
+    return LT_OK;
+}
+
+lt_status lt_replay_set_slot(lt_ctx *c, uint32_t slot, int as_integer, double dvalue, int64_t ivalue) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    if (!c->replay.plan || slot >= c->replay.dyn.size()) return fail(c, LT_ERR_INVALID_ARG, "lt_replay_set_slot: no such run-time slot");
+    if (as_integer) c->replay.dyn[slot].i = ivalue;
+    else c->replay.dyn[slot].d = dvalue;
     return LT_OK;
 }
 

@@ -164,6 +164,27 @@ struct HashKeyHasher {
     size_t operator()(const HashKey &k) const { return (size_t)(k.h[0] ^ (k.h[1] * 0x9E3779B97F4A7C15ull)); }
 };
 
+// What lt_replay needs to run the last flushed graph again without recording it: the plan, and which
+// tensors supplied its parameters and run-time scalars and received its results.
+struct ReplayRecord {
+    Plan *plan = nullptr;
+    struct Ref {
+        uint32_t slot = NONE, gen = 0;
+    };
+    struct ParamRef : Ref {
+        uint8_t dtype = 0, rank = 0;
+        int64_t dims[LT_MAX_RANK] = {0};
+    };
+    std::vector<ParamRef> params;   // tensor whose current value is parameter i
+    std::vector<Ref> dyn_scalar;    // scalar tensor that supplies run-time slot k (slot == NONE: value stays as recorded)
+    std::vector<DynValue> dyn;      // run-time values (recorded, or set since)
+    struct Root : Ref {
+        int32_t output = -1;
+    };
+    std::vector<Root> roots;        // tensors that receive the outputs
+    std::string why_not;            // non-empty: the last flush cannot be replayed, with the reason
+};
+
 struct TimedLaunch {
     cudaEvent_t start, stop;
     uint8_t kind;
@@ -204,6 +225,8 @@ struct lt_ctx {
     bool static_mode = false;
     void *static_base = nullptr;
     size_t static_cap = 0;
+
+    lt::ReplayRecord replay;
 
     bool timing = false;
     std::vector<lt::TimedLaunch> timed;
