@@ -405,7 +405,59 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
     keep.clear()
     del usets
     un.close()
+    # replay: the same step without recording, canonicalising or hashing (one lt_replay call per step)
+    X, H, Bv = sets[0]
+    o = traces.mlp_epilogue(ctx, X, H, Bv, primitive_gelu=False)
+    ctx.barrier()
+    ms_r = timed(n, lambda i: ctx.replay())
+    out["c2_replay_gbs"] = nbytes * n / (ms_r / 1e3) / 1e9
+    del o
+    out.update(adam_steps(lt, torch, ctx.device))
     return out
+
+
+def adam_steps(lt, torch, device: int) -> dict:
+    """C5: 100 Adam steps over the 161 ResNet-50 parameter tensors, one flush per step; traced every step
+    (1 compile + 99 cache hits) against traced once and replayed 99 times.  Wall-clock per step, host included."""
+    import math as _m
+
+    from workloads import configs, traces
+    from workloads.resnet50 import parameter_shapes
+
+    shapes = parameter_shapes()
+    nbytes = configs.algorithmic_bytes("c5")
+    dev = torch.device("cuda", device)
+    res = {}
+    for mode in ("traced", "replayed"):
+        ctx = lt.LazyContext(device=device)
+        P, G, M, V = ([ctx.from_torch(torch.randn(s, device=dev) * 0.05) for s in shapes] for _ in range(4))
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        if mode == "traced":
+            for step in range(1, 101):
+                traces.adam_step(ctx, P, G, M, V, step=step)
+                ctx.barrier()
+        else:
+            s = traces.AdamScalars(ctx, step=1)
+            for p, g, m, v in zip(P, G, M, V):
+                traces.adam_update(ctx, p, g, m, v, s)
+            ctx.barrier()
+            for step in range(2, 101):
+                ctx.scalar_set(s.sqrt_bc2, _m.sqrt(1.0 - 0.999 ** step))
+                ctx.scalar_set(s.step_size, 1e-3 / (1.0 - 0.9 ** step))
+                ctx.replay()
+        torch.cuda.synchronize()
+        sec = time.perf_counter() - t0
+        st = ctx.stats()
+        res[f"c5_adam_100_steps_{mode}_ms_per_step"] = 10.0 * sec
+        res[f"c5_adam_100_steps_{mode}_gbs"] = nbytes * 100 / sec / 1e9
+        res[f"c5_adam_{mode}_cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "replays": st["replays"],
+                                         "kernels": st["kernels_launched"]}
+        if mode == "traced":
+            res["c5_host_us_per_barrier"] = {k: st[k] / 1e3 / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
+        del P, G, M, V
+        ctx.close()
+    return res
 
 
 def main() -> None:

@@ -948,36 +948,36 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
     }
     {
         Timer tm(c->stats.ns_rebind);
+        // A result written in place already lives where its tensor's leaf points (checked above: that
+        // tensor alone names the buffer): nothing to rebind.  Fresh results get a new leaf.
         const size_t n_out = plan->outputs.size();
-        std::vector<uint32_t> new_nodes(n_out);
+        std::vector<uint32_t> fresh(n_out, NONE);
         for (size_t k = 0; k < n_out; ++k) {
             const OutputPlan &op = plan->outputs[k];
+            if (op.donated_param >= 0) continue;
             uint32_t n = node_new(c);
             Node &nd = c->nodes[n];
             nd.op = N_DEVICE_DATA;
             nd.dtype = op.dtype;
             nd.rank = op.rank;
             memcpy(nd.dims, op.dims, sizeof(nd.dims));
-            if (op.donated_param >= 0) {
-                uint32_t b = c->nodes[cg.param_node[op.donated_param]].buffer;
-                c->buffers[b].refs++;
-                nd.buffer = b;
-            } else {
-                nd.buffer = buffer_new(c, c->out_ptr[k], op.bytes, true);
-            }
+            nd.buffer = buffer_new(c, c->out_ptr[k], op.bytes, true);
             nd.refs = 1;
-            new_nodes[k] = n;
+            fresh[k] = n;
         }
         for (const ReplayRecord::Root &root : r.roots) {
+            const uint32_t nn = fresh[root.output];
+            if (nn == NONE) continue;
             TensorRec &t = c->tensors[root.slot];
-            const uint32_t nn = new_nodes[root.output], old_id = t.node;
+            const uint32_t old_id = t.node;
             t.node = nn;
             node_ref(c, nn);
             c->nodes[nn].tensor_refs++;
             c->nodes[old_id].tensor_refs--;
             node_unref(c, old_id);
         }
-        for (uint32_t n : new_nodes) node_unref(c, n);
+        for (uint32_t n : fresh)
+            if (n != NONE) node_unref(c, n);
     }
     c->stats.replays++;
     if (blocking && c->device != LT_DEVICE_NONE) {

@@ -22,7 +22,7 @@ HERE = Path(__file__).resolve().parent
 sys.path.insert(0, str(HERE.parent.parent))
 
 import paper_2102_13267_b200 as lt  # noqa: E402
-from workloads import traces  # noqa: E402
+from workloads import idioms, traces  # noqa: E402
 
 NT = 3          # LT_VM_NT
 OP_MOV_T_ACC = 1
@@ -81,6 +81,17 @@ def programs():
     P, G, M, V = ([d.leaf(s, "f32") for s in shapes] for _ in range(4))
     traces.adam_step(d.ctx, P, G, M, V, step=1)
     out.append(("adam_step", d.keys()))
+    # common fusion groups beyond the benchmark's (workloads/idioms.py)
+    for name, kinds, trace in idioms.ALL:
+        d = Dry()
+        ins = [d.leaf((16, 64) if k.startswith("mat") else (64,), k.split(":")[1]) for k in kinds]
+        keep = trace(d.ctx, ins, 64)
+        out.append((name, d.keys()))
+    d = Dry()
+    shapes = [(64,), (128,)]
+    P, G, Bf = ([d.leaf(s, "f32") for s in shapes] for _ in range(3))
+    idioms.sgd_momentum(d.ctx, P, G, Bf)
+    out.append(("sgd_momentum", d.keys()))
     del keep
     return out
 

@@ -188,3 +188,51 @@ def test_unfused_matches_oracle(ctx):
     ref = traces.causal_softmax(O, *ol, shape=(2, 40, 40), scale=0.1)
     y = traces.causal_softmax(ctx, *gl, shape=(2, 40, 40), scale=0.1)
     assert_matches(ctx.fetch(y), ref.array, "bf16", "unfused softmax")
+
+
+# ------------------------------------------------------------------ common fusion groups (workloads/idioms.py)
+def _idiom_inputs(kinds, shape, seed):
+    g = rng.generator(seed, 9)
+    arrs = []
+    for k in kinds:
+        what, dt = k.split(":")
+        shp = shape if what == "mat" else (shape[-1],)
+        a = rng.normal_f32(g, shp, 1.0, 1.0 if what == "vec" else 0.0)
+        arrs.append((rng.to_bf16_bits(a) if dt == "bf16" else a, dt))
+    return arrs
+
+
+@pytest.mark.parametrize("shape", [(24, 64), (7, 1000), (5, 2048), (3, 40), (300, 1024)])
+@pytest.mark.parametrize("idiom", [e[0] for e in __import__("workloads.idioms", fromlist=["ALL"]).ALL])
+def test_common_fusion_groups(ctx, idiom, shape):
+    from workloads import idioms
+
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == idiom)
+    O, ol, gl = both(ctx, _idiom_inputs(kinds, shape, 31))
+    ref = trace(O, ol, shape[-1])
+    out = trace(ctx, gl, shape[-1])
+    ctx.barrier()
+    st = ctx.stats()
+    assert st["kernels_launched"] == 1 and st["launches_compiled"] == (1 if ctx.compiled_allowed else 0)
+    dt = "f32" if name.endswith("f32") else "bf16"
+    assert_matches(ctx.fetch(out), ref.array, dt, f"{name} {shape}")
+
+
+def test_sgd_momentum_many_tensors(ctx):
+    from workloads import idioms
+
+    shapes = parameter_shapes()[:10] + [(1000,)]
+    g = rng.generator(32, 9)
+    host = [[rng.normal_f32(g, s, 0.1) for s in shapes] for _ in range(3)]
+    O = EagerOracle()
+    op, og, ob = ([O.leaf(a, "f32") for a in arrs] for arrs in host)
+    gp, gg, gb = ([ctx.leaf(a, "f32") for a in arrs] for arrs in host)
+    for _ in range(3):
+        idioms.sgd_momentum(O, op, og, ob)
+        idioms.sgd_momentum(ctx, gp, gg, gb)
+        ctx.barrier()
+    st = ctx.stats()
+    assert st["kernels_launched"] == 3 and st["launches_multi"] == 3
+    assert st["launches_compiled"] == (3 if ctx.compiled_allowed else 0)
+    for a, r in zip(gp + gb, op + ob):
+        assert_matches(ctx.fetch(a), r.array, "f32", "sgd momentum", exact=True)

@@ -1,0 +1,84 @@
+"""Traced programs of common fusion groups beyond the five benchmark configurations.
+
+Same conventions as traces.py: a backend `B` with `scalar`, `op`, `assign`; nothing here computes a value.
+Each entry of ALL is (name, kinds of its inputs, trace function); input kinds are
+"mat:<dtype>" for a [rows, cols] operand and "vec:<dtype>" for a [cols] operand.  The library ships an
+ahead-of-time compiled kernel for every one of them; the parity tests run each against the oracle.
+"""
+from __future__ import annotations
+
+
+def _f32(B, t, dtype):
+    return t if dtype == "f32" else B.op("convert", t, dtype="f32")
+
+
+def _out(B, t, dtype):
+    return t if dtype == "f32" else B.op("convert", t, dtype=dtype)
+
+
+def bias_relu(B, x, bias, *, cols, dtype="bf16"):
+    """out = relu(x + bias)."""
+    return _out(B, B.op("relu", B.op("add", _f32(B, x, dtype), _f32(B, bias, dtype))), dtype)
+
+
+def bias_gelu(B, x, bias, *, cols, dtype="bf16"):
+    """out = GELU_tanh(x + bias)."""
+    return _out(B, B.op("gelu_tanh", B.op("add", _f32(B, x, dtype), _f32(B, bias, dtype))), dtype)
+
+
+def residual_add(B, x, y, *, cols, dtype="bf16"):
+    """out = x + y."""
+    return _out(B, B.op("add", _f32(B, x, dtype), _f32(B, y, dtype)), dtype)
+
+
+def swiglu(B, gate, up, *, cols, dtype="bf16"):
+    """out = gate * sigmoid(gate) * up."""
+    g = _f32(B, gate, dtype)
+    return _out(B, B.op("mul", B.op("mul", g, B.op("sigmoid", g)), _f32(B, up, dtype)), dtype)
+
+
+def softmax(B, x, *, cols, dtype="bf16"):
+    """Row softmax with the row maximum subtracted."""
+    s = _f32(B, x, dtype)
+    e = B.op("exp", B.op("sub", s, B.op("row_max", s)))
+    return _out(B, B.op("div", e, B.op("row_sum", e)), dtype)
+
+
+def layernorm(B, x, gamma, beta, *, cols, dtype="bf16", eps=1e-5):
+    """LayerNorm over the last dim, biased two-pass variance, f32 gamma / beta."""
+    t = _f32(B, x, dtype)
+    inv_c = B.scalar(1.0 / cols)
+    d = B.op("sub", t, B.op("mul", B.op("row_sum", t), inv_c))
+    var = B.op("mul", B.op("row_sum", B.op("mul", d, d)), inv_c)
+    z = B.op("mul", d, B.op("rsqrt", B.op("add", var, B.scalar(eps))))
+    return _out(B, B.op("add", B.op("mul", z, gamma), beta), dtype)
+
+
+def rmsnorm(B, x, gamma, *, cols, dtype="bf16", eps=1e-6):
+    """x * rsqrt(mean(x^2) + eps) * gamma."""
+    t = _f32(B, x, dtype)
+    ms = B.op("mul", B.op("row_sum", B.op("mul", t, t)), B.scalar(1.0 / cols))
+    return _out(B, B.op("mul", B.op("mul", t, B.op("rsqrt", B.op("add", ms, B.scalar(eps)))), gamma), dtype)
+
+
+def sgd_momentum(B, params, grads, bufs, *, lr=0.1, momentum=0.9):
+    """For every tensor: buf := momentum * buf + g; p := p - lr * buf (in place).  The two scalars are
+    shared by all tensors, so the updates are one program over many tensors."""
+    lr_s, mom_s = B.scalar(lr), B.scalar(momentum)
+    for p, g, buf in zip(params, grads, bufs):
+        nb = B.op("add", B.op("mul", buf, mom_s), g)
+        B.assign(buf, nb)
+        B.assign(p, B.op("sub", p, B.op("mul", nb, lr_s)))
+
+
+ALL = [
+    ("bias_relu_bf16", ("mat:bf16", "vec:bf16"), lambda B, ins, cols: bias_relu(B, *ins, cols=cols)),
+    ("bias_gelu_bf16", ("mat:bf16", "vec:bf16"), lambda B, ins, cols: bias_gelu(B, *ins, cols=cols)),
+    ("residual_add_bf16", ("mat:bf16", "mat:bf16"), lambda B, ins, cols: residual_add(B, *ins, cols=cols)),
+    ("residual_add_f32", ("mat:f32", "mat:f32"), lambda B, ins, cols: residual_add(B, *ins, cols=cols, dtype="f32")),
+    ("swiglu_bf16", ("mat:bf16", "mat:bf16"), lambda B, ins, cols: swiglu(B, *ins, cols=cols)),
+    ("softmax_bf16", ("mat:bf16",), lambda B, ins, cols: softmax(B, *ins, cols=cols)),
+    ("softmax_f32", ("mat:f32",), lambda B, ins, cols: softmax(B, *ins, cols=cols, dtype="f32")),
+    ("layernorm_bf16", ("mat:bf16", "vec:f32", "vec:f32"), lambda B, ins, cols: layernorm(B, *ins, cols=cols)),
+    ("rmsnorm_bf16", ("mat:bf16", "vec:f32"), lambda B, ins, cols: rmsnorm(B, *ins, cols=cols)),
+]
