@@ -8,8 +8,10 @@
  * it up in a compile cache and executes it (Section 4); in-place updates are a
  * substitution of the destination's computation, with input buffers donated to
  * outputs at the barrier (Section 4.3).  Where the paper hands the graph to the
- * XLA compiler, this library cuts it into fusion groups and runs each group as
- * one hand-written CUDA kernel that interprets a small register program.
+ * XLA compiler, this library cuts it into fusion groups, emits a small register
+ * program per group and runs the group as one hand-written CUDA kernel: a kernel
+ * instantiated at build time over the program itself when the program is in the
+ * library's table of compiled programs, an interpreter of the program otherwise.
  *
  * Conventions
  *   - Every call returns an lt_status; LT_OK is 0.  A human-readable message for the
@@ -154,13 +156,21 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * "ieee" (0 default: in groups storing f32, division, square root and reciprocal are accurate to
  * 2 ulp; 1 = correctly rounded, so that a graph of + - * / sqrt matches an op-by-op binary32
  * evaluation bit for bit, at about ten more instructions per element and op),
- * "waves" (1 default: grid size of the persistent kernels in waves of resident thread blocks; every
- * block pays a fixed set-up -- program staging and linking -- so one wave measured fastest),
+ * "waves" (0 default = each kernel's own choice: one wave of resident thread blocks, two for the compiled
+ * multi-tensor kernel; every interpreter block pays a fixed set-up -- program staging and linking),
  * "stage" (3 default: inputs are copied asynchronously into per-thread shared-memory staging buffers a few
  * chunks ahead of their use when at least this many buffers fit in 64 KB per block -- fewer measured slower than
  * loading at first use with L2 prefetch; launches that give a thread one or two chunks stage anyway, to fetch all
  * inputs in parallel; 0 = never stage),
- * "cache_capacity" (0 = unbounded).  Options are part of the cache key.
+ * "cache_capacity" (0 = unbounded),
+ * "compiled" (1 default: a launch whose program is in the table of ahead-of-time compiled programs, whose
+ * pointers are 16-byte aligned and whose rows are a multiple of 8 elements runs on that kernel; 0 = always
+ * interpret), "compiled_u" / "compiled_row_u" / "compiled_depth" (0 / 0 / -1 default = the library's choice:
+ * chunks of 8 elements in flight per thread in compiled elementwise and multi-tensor kernels, chunks per thread
+ * in compiled row kernels, depth of their shared-memory staging ring -- tuning knobs for measurements),
+ * "pool_bytes" (4 GiB default: device blocks the library has released are kept, up to this total, and reused
+ * by later flushes before the allocator is asked; 0 = return every block at once).
+ * fusion, fast_math, horizontal and ieee are part of the cache key; the others act at launch time.
  * Unknown key: LT_ERR_INVALID_ARG.  The environment variables LT_FUSION, LT_VERIFY,
  * LT_FAST_MATH, LT_HORIZONTAL preset the same options at context creation.
  */
