@@ -112,7 +112,7 @@ def measured_peak() -> tuple[float, str]:
 
 # DRAM bytes of one launch of the dominant kernel on this workload, from the ncu capture summarised in
 # profiles/lt_c_ew_c2_mlp_epilogue.md, with the hash of the kernel sources it was taken on.
-NCU_TRAFFIC = {"bytes": 0, "sources_sha256": ""}
+NCU_TRAFFIC = {"bytes": 162635776, "sources_sha256": "d6b37667622b4bb593556f5220ce2a133aa1ad83d6d7e645e5c4a86413dccf7d"}
 KERNEL_SOURCES = ("paper_2102_13267_b200/csrc/compiled.cu", "paper_2102_13267_b200/csrc/compiled_programs.inc",
                   "paper_2102_13267_b200/csrc/vm_ops.cuh", "paper_2102_13267_b200/csrc/vm.h")
 

@@ -284,7 +284,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, 0, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     done = true;
-                } else if (ok && P.cpr <= 8u * 1024u) {
+                } else if (ok && P.cpr <= 8u * 128u) {  // a row's group of threads is at most one CTA of 128
                     // a row lives in the registers of its thread group: up to 8 chunks per thread, one warp per row if it fits
                     int u = 1;
                     while (u < 8 && P.cpr > 32u * u) u *= 2;
@@ -300,7 +300,11 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     if (stage == 0 || threads != 128 || depth < 2) depth = 0;
                     const int occ = compiled_blocks(L, u, (int)threads, depth * stage);
                     const uint64_t blocks = ((uint64_t)P.rows + threads / grp - 1) / (threads / grp);
-                    unsigned grid = (unsigned)std::min<uint64_t>(blocks, (uint64_t)c->sm_count * occ * waves);
+                    // one wave of persistent CTAs; with many blocks of rows per CTA, four waves balance the tail
+                    // better (measured on [32768 x 2048]: 49.6 us against 54.5)
+                    const uint64_t resident = (uint64_t)c->sm_count * occ;
+                    const unsigned rwaves = c->opt.waves > 0 ? waves : (blocks >= 16 * resident ? 4u : 1u);
+                    unsigned grid = (unsigned)std::min<uint64_t>(blocks, resident * rwaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
                     e = lt_compiled_launch(L.compiled, &P, u, grid, threads, grp, lg, depth, c->stream);

@@ -1,6 +1,6 @@
 """Kernel-only timing of the five benchmark configurations (also the driver for ncu captures).
 
-    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5] [--iters N] [--sets K] [key=value ...]
+    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5,idioms] [--iters N] [--sets K] [key=value ...]
 
 For each configuration: traces the graph, flushes it `iters` times over rotating buffer sets
 (larger than L2 together) with per-launch CUDA events, and prints microseconds per flush and
@@ -52,7 +52,7 @@ def main() -> None:
         kt = ctx.kernel_timing()
         ms = sum(v["ms"] for v in kt.values()) / args.iters
         n = sum(v["launches"] for v in kt.values()) / args.iters
-        print(f"{name:4s} {1e3 * ms:9.1f} us/flush {nbytes / ms / 1e6:8.1f} GB/s  {n:.0f} launches/flush", flush=True)
+        print(f"{name:18s} {1e3 * ms:9.1f} us/flush {nbytes / ms / 1e6:8.1f} GB/s  {n:.0f} launches/flush", flush=True)
 
     def run(name, cfg, make, trace):
         nbytes = configs.algorithmic_bytes(cfg)
@@ -93,6 +93,41 @@ def main() -> None:
         shape = configs.FULL["c4"]
         run("c4", "c4", lambda c: (c.from_torch(bf16(shape, 4.0)),),
             lambda c, s: traces.causal_softmax(c, *s, shape=shape, scale=1 / math.sqrt(128)))
+    # common fusion groups (workloads/idioms.py) on [16384 x 1024]: name, bytes per element moved
+    from workloads import idioms
+
+    ishape = (16384, 1024)
+    for name, kinds, trace in idioms.ALL:
+        if name not in which and "idioms" not in which:
+            continue
+        per_elem = sum((2 if k.endswith("bf16") else 4) for k in kinds if k.startswith("mat")) + (4 if name.endswith("f32") else 2)
+        nbytes = per_elem * ishape[0] * ishape[1]
+
+        def make(c, kinds=kinds):
+            out = []
+            for k in kinds:
+                shp = ishape if k.startswith("mat") else (ishape[1],)
+                t = torch.randn(shp, device=dev)
+                out.append(c.from_torch(t.to(torch.bfloat16) if k.endswith("bf16") else t))
+            return out
+
+        nsets = args.sets or max(2, math.ceil(1.2e9 / nbytes))
+        ctx = context()
+        sets = [make(ctx) for _ in range(nsets)]
+        keep = [None] * nsets
+        for i in range(5):
+            keep[i % nsets] = trace(ctx, sets[i % nsets], ishape[1])
+            ctx.barrier()
+        torch.cuda.synchronize()
+        ctx.set_kernel_timing(True)
+        ctx.kernel_timing()
+        hold_gpu()
+        for i in range(args.iters):
+            keep[i % nsets] = trace(ctx, sets[i % nsets], ishape[1])
+            ctx.barrier()
+        report(name[:18], nbytes, ctx)
+        del keep, sets
+        ctx.close()
     if "c5" in which:
         shapes = parameter_shapes()
         ctx = context()
