@@ -635,8 +635,9 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_ew(const __grid_constant__ LtK
         Coords<U> ck;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t cu = c + u * stride;
-            ck.ok[u] = cu < n_chunks;
+            const uint32_t cx = c + u * stride;
+            ck.ok[u] = cx < n_chunks;
+            const uint32_t cu = ck.ok[u] ? cx : 0u;  // a chunk past the end takes the coordinates of chunk 0 (see lt_c_row)
             ck.flat0[u] = (uint64_t)cu * V;
             if (Info<PG>::needs_coords() && P.rowcol) {
                 const uint32_t q = __umulhi(P.div_mul, cu);
@@ -674,10 +675,14 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
         const uint32_t row = rb * rows_per_cta + sub;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            ck.row[u] = row;
-            ck.col0[u] = (u * group + gl) * V;
-            ck.ok[u] = row < P.rows && ck.col0[u] < P.cols;
-            ck.flat0[u] = (uint64_t)row * P.cols + ck.col0[u];
+            // a chunk past the end of the row, or a row past the last, takes the coordinates of an existing
+            // one: broadcast operands are read at use without a validity test and must stay in bounds
+            const uint32_t col = (u * group + gl) * V;
+            const bool in_row = col < P.cols, in_rows = row < P.rows;
+            ck.row[u] = in_rows ? row : 0u;
+            ck.col0[u] = in_row ? col : 0u;
+            ck.ok[u] = in_rows && in_row;
+            ck.flat0[u] = (uint64_t)ck.row[u] * P.cols + ck.col0[u];
         }
     };
     const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(stage_mem);
