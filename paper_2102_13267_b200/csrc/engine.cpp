@@ -161,6 +161,11 @@ void record_replay(lt_ctx *c, Plan *plan, const Canonical &cg, const std::vector
         root.output = cg.nodes[c->nodes[c->tensors[slot].node].canon].output;
         r.roots.push_back(root);
     }
+    r.in_place_ok.assign(plan->outputs.size(), 0);
+    for (const ReplayRecord::Root &root : r.roots) {
+        const int32_t p = plan->outputs[root.output].donated_param;
+        if (p >= 0 && r.params[p].slot == root.slot) r.in_place_ok[root.output] = 1;
+    }
     by_node.clear();
 }
 
@@ -925,11 +930,8 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
         const int32_t p = plan->outputs[k].donated_param;
         if (p < 0) continue;
         const Node &leaf = c->nodes[cg.param_node[p]];
-        bool ok = leaf.tensor_refs == 1 && c->buffers[leaf.buffer].refs == 1;
-        bool receives = false;
-        for (const ReplayRecord::Root &root : r.roots)
-            if (root.output == (int32_t)k && root.slot == r.params[p].slot) receives = true;
-        if (!ok || !receives)
+        const bool ok = leaf.tensor_refs == 1 && c->buffers[leaf.buffer].refs == 1;
+        if (!ok || !r.in_place_ok[k])
             return fail(c, LT_ERR_UNSUPPORTED, "lt_replay: an in-place result would overwrite memory another tensor names");
     }
     // run-time values: scalars from their tensors, the rest as recorded or set

@@ -182,6 +182,7 @@ struct ReplayRecord {
         int32_t output = -1;
     };
     std::vector<Root> roots;        // tensors that receive the outputs
+    std::vector<uint8_t> in_place_ok;  // per output written in place: 1 if the tensor receiving it is the one that supplies the buffer
     std::string why_not;            // non-empty: the last flush cannot be replayed, with the reason
 };
 
