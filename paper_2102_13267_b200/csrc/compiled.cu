@@ -270,8 +270,12 @@ struct GroupReduce {
 #pragma unroll
             for (int u = 0; u + s < U; u += 2 * s) part[u] = red_comb<KIND>(part[u], part[u + s]);
         float r = part[0];
-        const uint32_t width = group < 32u ? group : 32u;
-        for (uint32_t off = width >> 1; off > 0; off >>= 1) r = red_comb<KIND>(r, __shfl_xor_sync(0xffffffffu, r, off));
+        if (group >= 32u) {  // the usual case, a whole warp (or more) per row: five fixed butterfly steps
+#pragma unroll
+            for (uint32_t off = 16; off > 0; off >>= 1) r = red_comb<KIND>(r, __shfl_xor_sync(0xffffffffu, r, off));
+        } else {
+            for (uint32_t off = group >> 1; off > 0; off >>= 1) r = red_comb<KIND>(r, __shfl_xor_sync(0xffffffffu, r, off));
+        }
         if (group > 32u) {
             float *buf = smem + (phase & 1u) * 32u;
             ++phase;
