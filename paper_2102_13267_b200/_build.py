@@ -61,5 +61,15 @@ def build(force: bool = False) -> Path:
     return LIB
 
 
+def build_host_bench() -> Path:
+    """Compile csrc/host_bench.cpp (host cost of record / flush / replay through the C ABI, no Python) against the library."""
+    exe = HERE / "lt_host_bench"
+    src = CSRC / "host_bench.cpp"
+    if _stale(exe, [src, LIB]):
+        subprocess.check_call(["g++", "-O2", "-std=c++17", f"-I{HERE.parent / 'include'}", str(src), f"-L{HERE}", "-llazytensor",
+                               f"-Wl,-rpath,{HERE}", "-o", str(exe)])
+    return exe
+
+
 if __name__ == "__main__":
     print(build())

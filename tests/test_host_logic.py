@@ -389,3 +389,19 @@ def test_compiled_table_is_what_the_planner_emits_today():
     d.ctx.barrier()
     assert "compiled: no" in d.ctx.dump_plan()
     del keep
+
+
+def test_host_bench_driver_runs_without_python_in_the_loop():
+    """The C++ driver records, flushes and replays three of the configurations through the C ABI alone."""
+    import importlib.util
+    import subprocess
+
+    spec = importlib.util.spec_from_file_location("_lt_build", os.path.join(ROOT, "paper_2102_13267_b200", "_build.py"))
+    b = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(b)
+    out = subprocess.run([str(b.build_host_bench())], capture_output=True, text=True, timeout=120, check=True).stdout
+    lines = out.strip().splitlines()
+    assert len(lines) == 4
+    assert "compiles 1, hits 19999" in lines[0] and "compiles 1, hits 19999" in lines[1]
+    assert "compiles 1, hits 99," in lines[2]
+    assert "replays 99" in lines[3]
