@@ -362,6 +362,55 @@ def test_failed_allocation_leaves_the_graph_flushable():
     assert not live  # the output buffer went back through the free callback
 
 
+def test_released_blocks_are_reused_before_the_allocator_is_asked():
+    """Steady state makes no allocator call: the block of a released result serves the next flush of the
+    same size; `pool_bytes` = 0 hands every block back at once; closing the context returns the rest."""
+    lib = ctypes.CDLL(str(lt.LIB_PATH))
+    calls = {"alloc": 0, "free": 0}
+    live = {}
+
+    def alloc(nbytes, stream, user):
+        calls["alloc"] += 1
+        buf = ctypes.create_string_buffer(max(int(nbytes), 16))
+        live[ctypes.addressof(buf)] = buf
+        return ctypes.addressof(buf)
+
+    def free(ptr, stream, user):
+        calls["free"] += 1
+        live.pop(ptr, None)
+
+    a_fn, f_fn = lt.ALLOC_FN(alloc), lt.FREE_FN(free)
+    st = lt.lt_allocator(a_fn, f_fn, None)
+    c = ctypes.c_void_p()
+    assert lib.lt_ctx_create(-1, None, ctypes.byref(st), ctypes.byref(c)) == 0
+    for name in ("lt_tensor_from_device", "lt_op", "lt_barrier", "lt_release", "lt_ctx_set_option", "lt_ctx_destroy"):
+        getattr(lib, name).argtypes = lt._SIGNATURES[name]
+    shape = (ctypes.c_int64 * 2)(64, 64)
+    a, b, y = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    assert lib.lt_tensor_from_device(c, ctypes.c_void_p(1 << 20), 0, 2, shape, ctypes.byref(a)) == 0
+    assert lib.lt_tensor_from_device(c, ctypes.c_void_p(2 << 20), 0, 2, shape, ctypes.byref(b)) == 0
+
+    def step():
+        ins = (ctypes.c_uint64 * 2)(a.value, b.value)
+        assert lib.lt_op(c, 1, ins, 2, None, 0, ctypes.byref(y)) == 0
+        assert lib.lt_barrier(c, 0) == 0
+        assert lib.lt_release(c, y.value) == 0
+
+    for _ in range(5):
+        step()
+    assert calls == {"alloc": 1, "free": 0}  # one block, recycled four times
+    assert lib.lt_ctx_set_option(c, b"pool_bytes", 0) == 0  # gives the pooled block back ...
+    assert calls["free"] == 1 and not live
+    for _ in range(3):
+        step()                                               # ... and from now on every flush allocates and frees
+    assert calls == {"alloc": 4, "free": 4}
+    assert lib.lt_ctx_set_option(c, b"pool_bytes", 1 << 20) == 0
+    step()
+    assert calls == {"alloc": 5, "free": 4} and len(live) == 1
+    assert lib.lt_ctx_destroy(c) == 0
+    assert calls["free"] == 5 and not live
+
+
 # ------------------------------------------------------------------ ahead-of-time compiled programs
 def test_compiled_table_is_what_the_planner_emits_today():
     """The committed table of compiled programs equals what its generator derives from the planner now
