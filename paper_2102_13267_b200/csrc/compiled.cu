@@ -468,10 +468,23 @@ struct Machine {
 #pragma unroll
             for (int u = 0; u < U; ++u) source<LT_VM_SRC_S, imm>(acc[u], u);
         } else if constexpr (op == OP_ST) {
-            static_assert(PG::cls[imm] == LT_CLS_FULL, "compiled programs store full-class results only");
+            static_assert(PG::cls[imm] == LT_CLS_FULL || PG::cls[imm] == LT_CLS_ROWVEC, "results are full-class or one value per row");
+            if constexpr (PG::cls[imm] == LT_CLS_FULL) {
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (!GUARD || ck.ok[u]) chunk_store<PG::dtype[imm]>(acc[u], const_cast<char *>(address<imm>(u)));
+                for (int u = 0; u < U; ++u)
+                    if (!GUARD || ck.ok[u]) chunk_store<PG::dtype[imm]>(acc[u], const_cast<char *>(address<imm>(u)));
+            } else {
+                // one value per row (a reduction's result): written by the thread that owns the row's first chunk
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if ((!GUARD || ck.ok[u]) && ck.col0[u] == 0) {
+                        char *p = const_cast<char *>(address<imm>(u));
+                        constexpr int dt = PG::dtype[imm];
+                        if constexpr (dt == LT_ST_BF16) *reinterpret_cast<__nv_bfloat16 *>(p) = __float2bfloat16_rn(acc[u][0]);
+                        else if constexpr (dt == LT_ST_U8) *reinterpret_cast<unsigned char *>(p) = (unsigned char)f2u(acc[u][0]);
+                        else *reinterpret_cast<float *>(p) = acc[u][0];
+                    }
+            }
         } else if constexpr (op == OP_IOTA_COL) {
 #pragma unroll
             for (int u = 0; u < U; ++u)

@@ -92,8 +92,40 @@ def programs():
     P, G, Bf = ([d.leaf(s, "f32") for s in shapes] for _ in range(3))
     idioms.sgd_momentum(d.ctx, P, G, Bf)
     out.append(("sgd_momentum", d.keys()))
+    # every single-op program of the five configurations traced with fusion off: the unfused baseline
+    # ("one kernel per traced op") then runs compiled kernels too, not the interpreter
+    for name, record in unfused_traces():
+        d = Dry(fusion=0)
+        keep = record(d)
+        out.append((name, d.keys()))
     del keep
     return out
+
+
+def unfused_traces():
+    def c1(d):
+        return traces.elementwise_chain(d.ctx, *(d.leaf((64, 64), "f32") for _ in range(4)))
+
+    def c2(d, prim):
+        x, h = (d.leaf((16, 64), "bf16") for _ in range(2))
+        return traces.mlp_epilogue(d.ctx, x, h, d.leaf((64,), "bf16"), primitive_gelu=prim)
+
+    def c3(d):
+        x, h = (d.leaf((16, 64), "bf16") for _ in range(2))
+        g, be = (d.leaf((64,), "f32") for _ in range(2))
+        return traces.residual_dropout_layernorm(d.ctx, x, h, g, be, shape=(16, 64), p=0.1, eps=1e-5, seed=1, offset=0)
+
+    def c4(d):
+        return traces.causal_softmax(d.ctx, d.leaf((2, 64, 64), "bf16"), shape=(2, 64, 64), scale=0.1)
+
+    def c5(d):
+        shapes = [(64,), (128,)]
+        P, G, M, V = ([d.leaf(s, "f32") for s in shapes] for _ in range(4))
+        traces.adam_step(d.ctx, P, G, M, V, step=1)
+        return P
+
+    return [("op_c1", c1), ("op_c2", lambda d: c2(d, False)), ("op_c2p", lambda d: c2(d, True)), ("op_c3", c3),
+            ("op_c4", c4), ("op_c5", c5)]
 
 
 def parse(key: str):
@@ -113,7 +145,7 @@ def check(name, kind, n_pro, cls, ins):
         assert not (OP_MOV_T_ACC <= op < OP_MOV_T_ACC + NT and op - OP_MOV_T_ACC in reserved), f"{name}: reserved temporary overwritten"
         assert not (OP_LD <= op < OP_LD + NT and op - OP_LD in reserved), f"{name}: reserved temporary overwritten"
         if op == OP_ST:
-            assert cls[imm] == 0, f"{name}: compiled kernels store full-class results only"
+            assert cls[imm] in (0, 2), f"{name}: compiled kernels store full-class results or one value per row"
 
 
 def render() -> tuple[str, list[str]]:
