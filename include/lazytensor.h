@@ -331,6 +331,15 @@ lt_status lt_get_kernel_timing(lt_ctx *ctx, lt_kernel_timing *out);
 lt_status lt_dump_ir(lt_ctx *ctx, char *buf, size_t cap, size_t *need);
 lt_status lt_dump_plan(lt_ctx *ctx, char *buf, size_t cap, size_t *need);
 
+/*
+ * Debug builds only (library compiled with -DLT_DEBUG_BOUNDS; the release build answers
+ * LT_ERR_UNSUPPORTED): the ahead-of-time compiled kernels check every address they form against the
+ * extent of the tensor it belongs to; an access that would leave it is redirected inside the buffer and
+ * counted.  Returns the count since the library was loaded (0 is the only acceptable value).
+ * Synchronises the device.
+ */
+lt_status lt_debug_bounds_violations(lt_ctx *ctx, uint64_t *out);
+
 const char *lt_last_error(lt_ctx *ctx);
 const char *lt_version(void);
 

@@ -79,6 +79,7 @@ _SIGNATURES = {
     "lt_release_many": [_vp, _P(_u64), ctypes.c_size_t],
     "lt_barrier": [_vp, _int],
     "lt_barrier_static_scratch": [_vp, _int, _int],
+    "lt_debug_bounds_violations": [_vp, _P(_u64)],
     "lt_replay": [_vp, _int],
     "lt_scalar_set": [_vp, _u64, ctypes.c_double],
     "lt_replay_slots": [_vp, _P(ctypes.c_uint32)],
@@ -350,6 +351,15 @@ class LazyContext:
         if st:
             self._keeps.extend(keeps)
             self._check(st)
+
+    def debug_bounds_violations(self) -> int | None:
+        """Out-of-bounds accesses the compiled kernels caught (debug build), or None in a release build."""
+        n = _u64()
+        st = _lib.lt_debug_bounds_violations(self._ctx, ctypes.byref(n))
+        if st == STATUS_NAMES.index("LT_ERR_UNSUPPORTED"):
+            return None
+        self._check(st)
+        return n.value
 
     def replay(self, blocking: bool = False) -> None:
         """lt_replay: run the previously flushed graph again on the same tensors, without recording it."""

@@ -234,6 +234,23 @@ __device__ __forceinline__ void cp_async_wait(uint32_t pending) {  // at most `p
 
 constexpr __host__ __device__ int esz_shift(int dt) { return dt == LT_ST_BF16 ? 1 : (dt == LT_ST_U8 ? 0 : 2); }
 
+// Debug build (-DLT_DEBUG_BOUNDS): every address the shells form is checked against the extent of its slot;
+// an access that would leave it is counted in a device word the host can read, and redirected to element 0 so
+// that it stays inside the buffer.  The release build contains none of this.
+#ifdef LT_DEBUG_BOUNDS
+__device__ unsigned long long lt_c_bounds_violations = 0;
+__device__ __forceinline__ uint64_t bounds_checked(uint64_t first, uint32_t count, uint64_t extent) {
+    if (first + count > extent) {
+        atomicAdd(&lt_c_bounds_violations, 1ull);
+        return 0;
+    }
+    return first;
+}
+#define LT_CHECKED(first, count, extent) bounds_checked((first), (count), (extent))
+#else
+#define LT_CHECKED(first, count, extent) (first)
+#endif
+
 // Coordinates of the U chunks a thread works on in one iteration.
 template <int U>
 struct Coords {
@@ -324,9 +341,9 @@ struct Machine {
     __device__ __forceinline__ const char *address(int u) const {
         constexpr int cls = PG::cls[SLOT], sh = esz_shift(PG::dtype[SLOT]);
         const char *base = reinterpret_cast<const char *>(ptr(SLOT));
-        if constexpr (cls == LT_CLS_FULL) return base + (ck.flat0[u] << sh);
-        else if constexpr (cls == LT_CLS_COLVEC) return base + ((uint64_t)ck.col0[u] << sh);
-        else if constexpr (cls == LT_CLS_ROWVEC) return base + ((uint64_t)ck.row[u] << sh);
+        if constexpr (cls == LT_CLS_FULL) return base + (LT_CHECKED(ck.flat0[u], V, ptr.extent(cls)) << sh);
+        else if constexpr (cls == LT_CLS_COLVEC) return base + (LT_CHECKED((uint64_t)ck.col0[u], V, ptr.extent(cls)) << sh);
+        else if constexpr (cls == LT_CLS_ROWVEC) return base + (LT_CHECKED((uint64_t)ck.row[u], 1, ptr.extent(cls)) << sh);
         else return base;
     }
 
@@ -383,7 +400,7 @@ struct Machine {
 #pragma unroll
                     for (int u = 0; u < U; ++u) {
                         if (GUARD && !ok[u]) continue;
-                        const char *src = base + (flat0[u] << sh);
+                        const char *src = base + (LT_CHECKED(flat0[u], V, ptr.extent(LT_CLS_FULL)) << sh);
                         if constexpr (cb == 8) {
                             cp_async8(stage + off + (u * THREADS + threadIdx.x) * 8, src);
                         } else {
@@ -625,6 +642,10 @@ struct ScalK {
 struct PtrK {
     const LtKParams &P;
     __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[s]; }
+    // elements a slot of the class holds (bounds checks of the debug build)
+    __device__ __forceinline__ uint64_t extent(int cls) const {
+        return cls == LT_CLS_FULL ? P.n : cls == LT_CLS_COLVEC ? P.cols : cls == LT_CLS_ROWVEC ? P.rows : 1;
+    }
 };
 struct ScalM {
     const LtMultiParams &P;
@@ -633,7 +654,9 @@ struct ScalM {
 struct PtrM {
     const LtMultiParams &P;
     uint32_t base;
+    uint32_t numel;
     __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[base + s]; }
+    __device__ __forceinline__ uint64_t extent(int) const { return numel; }
 };
 
 struct TrueTag { static constexpr bool value = true; };
@@ -760,7 +783,7 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_multi(const __grid_constant__ 
             const uint32_t mid = (lo + hi) >> 1;
             if (P.super_prefix[mid] <= sc) lo = mid; else hi = mid;
         }
-        const PtrM ptr{P, lo * P.n_slots};
+        const PtrM ptr{P, lo * P.n_slots, P.numel[lo]};
         const uint32_t chunks_all = P.numel[lo] / V;
         const uint32_t first = (sc - P.super_prefix[lo]) * PER_SUPER + threadIdx.x;
 #pragma unroll 1
@@ -866,6 +889,15 @@ int lt_compiled_find(int kind, int flavour, const LtIns *ins, uint32_t n_ins, ui
     LT_COMPILED_LIST(LT_X)
 #undef LT_X
     return -1;
+}
+
+int lt_compiled_bounds_violations(unsigned long long *out) {
+#ifdef LT_DEBUG_BOUNDS
+    return cudaMemcpyFromSymbol(out, lt_c_bounds_violations, sizeof(*out)) == cudaSuccess ? 0 : -1;
+#else
+    (void)out;
+    return 1;  // not a debug build
+#endif
 }
 
 int lt_compiled_count(void) {

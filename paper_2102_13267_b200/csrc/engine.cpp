@@ -1016,6 +1016,20 @@ lt_status lt_replay_set_slot(lt_ctx *c, uint32_t slot, int as_integer, double dv
     return LT_OK;
 }
 
+lt_status lt_debug_bounds_violations(lt_ctx *c, uint64_t *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_DEVICE, "lt_debug_bounds_violations needs a context on a CUDA device");
+    unsigned long long n = 0;
+    const int r = lt_compiled_bounds_violations(&n);
+    if (r == 1) return fail(c, LT_ERR_UNSUPPORTED, "the library was not built with -DLT_DEBUG_BOUNDS");
+    if (r != 0) {
+        cudaGetLastError();
+        return fail(c, LT_ERR_CUDA, "reading the bounds-violation counter failed");
+    }
+    *out = n;
+    return LT_OK;
+}
+
 lt_status lt_fetch(lt_ctx *c, lt_tensor t, void *host_dst, size_t nbytes) {
     if (!c) return LT_ERR_INVALID_ARG;
     uint32_t slot;
