@@ -61,6 +61,34 @@ def rmsnorm(B, x, gamma, *, cols, dtype="bf16", eps=1e-6):
     return _out(B, B.op("mul", B.op("mul", t, B.op("rsqrt", B.op("add", ms, B.scalar(eps)))), gamma), dtype)
 
 
+def silu(B, x, *, cols, dtype="bf16"):
+    """out = x * sigmoid(x)."""
+    t = _f32(B, x, dtype)
+    return _out(B, B.op("mul", t, B.op("sigmoid", t)), dtype)
+
+
+def gelu(B, x, *, cols, dtype="bf16"):
+    """out = GELU_tanh(x)."""
+    return _out(B, B.op("gelu_tanh", _f32(B, x, dtype)), dtype)
+
+
+def add_relu(B, x, y, *, cols, dtype="bf16"):
+    """out = relu(x + y)."""
+    return _out(B, B.op("relu", B.op("add", _f32(B, x, dtype), _f32(B, y, dtype))), dtype)
+
+
+def scale_to_f32(B, x, *, cols, scale=0.125):
+    """out (f32) = x (bf16) * scale."""
+    return B.op("mul", B.op("convert", x, dtype="f32"), B.scalar(scale))
+
+
+def scaled_softmax(B, x, *, cols, dtype="bf16", scale=0.0884):
+    """Row softmax of x * scale."""
+    s = B.op("mul", _f32(B, x, dtype), B.scalar(scale))
+    e = B.op("exp", B.op("sub", s, B.op("row_max", s)))
+    return _out(B, B.op("div", e, B.op("row_sum", e)), dtype)
+
+
 def sgd_momentum(B, params, grads, bufs, *, lr=0.1, momentum=0.9):
     """For every tensor: buf := momentum * buf + g; p := p - lr * buf (in place).  The two scalars are
     shared by all tensors, so the updates are one program over many tensors."""
@@ -81,4 +109,10 @@ ALL = [
     ("softmax_f32", ("mat:f32",), lambda B, ins, cols: softmax(B, *ins, cols=cols, dtype="f32")),
     ("layernorm_bf16", ("mat:bf16", "vec:f32", "vec:f32"), lambda B, ins, cols: layernorm(B, *ins, cols=cols)),
     ("rmsnorm_bf16", ("mat:bf16", "vec:f32"), lambda B, ins, cols: rmsnorm(B, *ins, cols=cols)),
+    ("layernorm_f32", ("mat:f32", "vec:f32", "vec:f32"), lambda B, ins, cols: layernorm(B, *ins, cols=cols, dtype="f32")),
+    ("silu_bf16", ("mat:bf16",), lambda B, ins, cols: silu(B, *ins, cols=cols)),
+    ("gelu_bf16", ("mat:bf16",), lambda B, ins, cols: gelu(B, *ins, cols=cols)),
+    ("add_relu_bf16", ("mat:bf16", "mat:bf16"), lambda B, ins, cols: add_relu(B, *ins, cols=cols)),
+    ("scale_to_f32", ("mat:bf16",), lambda B, ins, cols: scale_to_f32(B, *ins, cols=cols)),
+    ("scaled_softmax_bf16", ("mat:bf16",), lambda B, ins, cols: scaled_softmax(B, *ins, cols=cols)),
 ]
