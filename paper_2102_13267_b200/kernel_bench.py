@@ -1,11 +1,13 @@
-"""Kernel-only timing of the five benchmark configurations (also the driver for ncu captures).
+"""Kernel-only timing of the benchmark configurations and of the common fusion groups (also the driver for ncu captures).
 
     python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5,idioms] [--iters N] [--sets K] [key=value ...]
 
-For each configuration: traces the graph, flushes it `iters` times over rotating buffer sets
-(larger than L2 together) with per-launch CUDA events, and prints microseconds per flush and
-algorithmic GB/s.  `key=value` pairs are context options (e.g. fusion=0, stage=0, ieee=1).
-With `--iters 4 --sets 1` it is the small workload used for `ncu --set full` captures.
+For each configuration: traces the graph and flushes it `iters` times over rotating buffer sets (larger than L2
+together), queued behind a busy stream so that the GPU, not the host, sets the pace.  Two figures are printed:
+every launch between its own two CUDA events (`lt_set_kernel_timing`), and "back to back": one pair of events around
+all the launches, kernel timing off (for C5 the steps are replayed, the host cannot record 161 tensors that fast).
+`key=value` pairs are context options (e.g. fusion=0, compiled=0, ieee=1).  With `--iters 4 --sets 1` it is the
+small workload used for `ncu --set full` captures.
 """
 from __future__ import annotations
 
