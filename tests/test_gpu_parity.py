@@ -236,3 +236,24 @@ def test_sgd_momentum_many_tensors(ctx):
     assert st["launches_compiled"] == (3 if ctx.compiled_allowed else 0)
     for a, r in zip(gp + gb, op + ob):
         assert_matches(ctx.fetch(a), r.array, "f32", "sgd momentum", exact=True)
+
+
+@pytest.mark.parametrize("idiom", ["softmax_bf16", "residual_add_bf16"])
+def test_in_place_update_through_a_compiled_kernel(ctx, idiom):
+    """x := f(x, ...) with the result donated to x's buffer: the row kernel's staging ring reads blocks of rows
+    ahead of the block being written, the elementwise kernel requests its inputs before it stores."""
+    from workloads import idioms
+
+    shape = (3000, 1024)  # more blocks of rows than resident CTAs, a ragged last wave
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == idiom)
+    O, ol, gl = both(ctx, _idiom_inputs(kinds, shape, 35))
+    ptr = ctx.device_ptr(gl[0])
+    for _ in range(2):
+        O_out = trace(O, ol, shape[-1])
+        ol[0] = O_out
+        ctx.assign(gl[0], trace(ctx, gl, shape[-1]))
+        ctx.barrier()
+    st = ctx.stats()
+    assert st["outputs_donated"] == 2 and st["outputs_allocated"] == 0 and ctx.device_ptr(gl[0]) == ptr
+    assert st["launches_compiled"] == (2 if ctx.compiled_allowed else 0)
+    assert_matches(ctx.fetch(gl[0]), ol[0].array, "bf16", f"in-place {name}")
