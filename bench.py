@@ -444,7 +444,73 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
     out["c2_replay_gbs"] = nbytes * n / (ms_r / 1e3) / 1e9
     del o
     out.update(adam_steps(lt, torch, ctx.device))
+    out["other_configs"] = other_configs(lt, torch, ctx.device)
     return out
+
+
+def other_configs(lt, torch, device: int) -> dict:
+    """C1, C3, C4: fused and unfused GB/s, 40 flushes over rotating buffer sets (> 1 GB together) queued behind
+    a busy stream and timed between two events (kernel time including the gap to the next launch)."""
+    import math as _m
+
+    from workloads import configs, traces
+
+    dev = torch.device("cuda", device)
+    peak, _ = measured_peak()
+
+    def bf16(shape, std=1.0):
+        return (torch.randn(shape, device=dev) * std).to(torch.bfloat16)
+
+    def c1_make(c):
+        return [c.from_torch(torch.rand(configs.FULL["c1"], device=dev) * 2 - 1) for _ in range(4)]
+
+    def c3_make(c):
+        sh = configs.FULL["c3"]
+        return (c.from_torch(bf16(sh)), c.from_torch(bf16(sh)), c.from_torch(1 + 0.02 * torch.randn(sh[1], device=dev)),
+                c.from_torch(0.02 * torch.randn(sh[1], device=dev)))
+
+    def c4_make(c):
+        return (c.from_torch(bf16(configs.FULL["c4"], 4.0)),)
+
+    cases = {
+        "c1": (c1_make, lambda c, s: traces.elementwise_chain(c, *s)),
+        "c3": (c3_make, lambda c, s: traces.residual_dropout_layernorm(c, *s, shape=configs.FULL["c3"], p=0.1, eps=1e-5,
+                                                                        seed=1, offset=0)),
+        "c4": (c4_make, lambda c, s: traces.causal_softmax(c, *s, shape=configs.FULL["c4"], scale=1 / _m.sqrt(128))),
+    }
+    res = {}
+    for name, (make, trace) in cases.items():
+        nbytes = configs.algorithmic_bytes(name)
+        nsets = max(2, _m.ceil(1.2e9 / nbytes))
+        entry = {}
+        for mode, iters in (("fused", 40), ("unfused", 10)):
+            c = lt.LazyContext(device=device)
+            if mode == "unfused":
+                c.set_option("fusion", 0)
+            sets = [make(c) for _ in range(nsets)]
+            keep = [None] * nsets
+            for i in range(3):
+                keep[i % nsets] = trace(c, sets[i % nsets])
+                c.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(int(4e-3 * 1.9e9))  # the flushes queue up behind this and then run back to back
+            e0.record()
+            for i in range(iters):
+                keep[i % nsets] = trace(c, sets[i % nsets])
+                c.barrier()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / iters
+            entry[f"{mode}_us"] = 1e3 * ms
+            entry[f"{mode}_gbs"] = nbytes / ms / 1e6
+            entry[f"{mode}_launches"] = c.stats()["kernels_launched"] // (iters + 3)
+            del keep, sets
+            c.close()
+        entry["frac_of_measured_peak"] = entry["fused_gbs"] / peak
+        entry["speedup_vs_unfused"] = entry["unfused_us"] / entry["fused_us"]
+        res[name] = entry
+    return res
 
 
 def adam_steps(lt, torch, device: int) -> dict:
