@@ -168,6 +168,8 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * interpret), "compiled_u" / "compiled_row_u" / "compiled_depth" (0 / 0 / -1 default = the library's choice:
  * chunks of 8 elements in flight per thread in compiled elementwise and multi-tensor kernels, chunks per thread
  * in compiled row kernels, depth of their shared-memory staging ring -- tuning knobs for measurements),
+ * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
+ * line per flush and per replay; preset by the environment variable LT_LOG),
  * "pool_bytes" (4 GiB default: device blocks the library has released are kept, up to this total, and reused
  * by later flushes before the allocator is asked; 0 = return every block at once).
  * fusion, fast_math, horizontal and ieee are part of the cache key; the others act at launch time.

@@ -391,6 +391,7 @@ lt_status lt_ctx_create(int device, void *cuda_stream, const lt_allocator *alloc
     env_opt("LT_VERIFY", &c->opt.verify);
     env_opt("LT_FAST_MATH", &c->opt.fast_math);
     env_opt("LT_HORIZONTAL", &c->opt.horizontal);
+    env_opt("LT_LOG", &c->opt.log);
     if (device != LT_DEVICE_NONE) {
         cudaError_t e = cudaSetDevice(device);
         int sms = 0;
@@ -438,6 +439,7 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "ieee")) c->opt.ieee = value;
     else if (!strcmp(key, "waves")) c->opt.waves = value;
     else if (!strcmp(key, "stage")) c->opt.stage = value;
+    else if (!strcmp(key, "log")) c->opt.log = value;
     else if (!strcmp(key, "pool_bytes")) {
         c->opt.pool_bytes = value;
         pool_trim(c, value > 0 ? (size_t)value : 0);
@@ -802,6 +804,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
         return LT_OK;
     }
     c->stats.barriers++;
+    const uint64_t hits_before = c->stats.cache_hits;
     Plan *plan = nullptr;
     {
         Timer tm(c->stats.ns_hash_lookup);
@@ -846,6 +849,14 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
     }
     plan->last_used = ++c->use_clock;
     c->last_plan = plan;
+    const bool was_hit = c->stats.cache_hits != hits_before;
+    if (c->opt.log >= 2 || (c->opt.log >= 1 && !was_hit)) {
+        size_t compiled = 0;
+        for (const Launch &L : plan->launches) compiled += L.compiled >= 0 ? 1 : 0;
+        fprintf(stderr, "[lazytensor] barrier %llu: %zu nodes, hash %016llx%016llx, %s, %zu launches (%zu with a compiled kernel), %zu outputs, %zu temporaries\n",
+                (unsigned long long)c->stats.barriers, cg.nodes.size(), (unsigned long long)cg.hash[0], (unsigned long long)cg.hash[1],
+                was_hit ? "cache hit" : "planned", plan->launches.size(), compiled, plan->outputs.size(), plan->temp_bytes.size());
+    }
     {
         Timer tm(c->stats.ns_bind_launch);
         lt_status s = execute_plan(c, *plan, cg);
@@ -982,6 +993,9 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
             if (n != NONE) node_unref(c, n);
     }
     c->stats.replays++;
+    if (c->opt.log >= 2)
+        fprintf(stderr, "[lazytensor] replay %llu: %zu launches, %zu run-time slots\n", (unsigned long long)c->stats.replays,
+                plan->launches.size(), r.dyn.size());
     if (blocking && c->device != LT_DEVICE_NONE) {
         cudaError_t e = cudaStreamSynchronize(c->stream);
         if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));

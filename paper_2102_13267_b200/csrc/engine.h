@@ -149,6 +149,7 @@ struct Plan {
 
 struct Options {
     int64_t fusion = 1, verify = 1, fast_math = 1, horizontal = 1, cache_capacity = 0, ieee = 0, waves = 0, stage = 3;  // waves: 0 = each kernel's default (1; compiled multi-tensor 2)
+    int64_t log = 0;  // 1: one line on stderr per planned graph (cache miss); 2: also per flush and replay
     int64_t pool_bytes = 4ll << 30;  // released device blocks the context keeps for reuse (0 = return every block at once)
     int64_t compiled = 1;  // use the ahead-of-time compiled kernel of a program when the table has one
     int64_t compiled_row_u = 0;  // chunks per thread in compiled row kernels (0 = one warp per row where it fits)
