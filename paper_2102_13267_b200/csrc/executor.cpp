@@ -199,11 +199,11 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     for (size_t s = 0; s < slots && ok; ++s) ok = aligned_for(P.ptr[k * slots + s], g0.io[s].dtype);
                 }
                 if (ok) {
-                    // two chunks in flight per thread and two waves of blocks measured best for wide programs
+                    // two chunks in flight per thread and eight waves of blocks measured best for wide programs
                     // (four input streams) over many tensors of uneven size
                     const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 2;
                     const int occ = compiled_blocks(L, u, LT_EW_THREADS);
-                    const unsigned mwaves = c->opt.waves > 0 ? waves : 2u;
+                    const unsigned mwaves = c->opt.waves > 0 ? waves : 8u;  // C5: 116 us against 121 with two waves
                     unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * mwaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
@@ -278,7 +278,10 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 1;
                     const int occ = compiled_blocks(L, u, LT_EW_THREADS);
                     const uint64_t need = (P.n_chunks + (uint64_t)LT_EW_THREADS * u - 1) / ((uint64_t)LT_EW_THREADS * u);
-                    unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * occ * waves);
+                    // a compiled CTA has no set-up to amortise: many short CTAs, scheduled by the hardware as others
+                    // retire, beat one wave of persistent ones (C2: 31.3 us against 33.5; no change beyond 8 waves)
+                    const unsigned ewaves = c->opt.waves > 0 ? waves : 16u;
+                    unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * occ * ewaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
                     e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, 0, c->stream);
