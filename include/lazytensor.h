@@ -156,8 +156,9 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * "ieee" (0 default: in groups storing f32, division, square root and reciprocal are accurate to
  * 2 ulp; 1 = correctly rounded, so that a graph of + - * / sqrt matches an op-by-op binary32
  * evaluation bit for bit, at about ten more instructions per element and op),
- * "waves" (0 default = each kernel's own choice: one wave of resident thread blocks, two for the compiled
- * multi-tensor kernel; every interpreter block pays a fixed set-up -- program staging and linking),
+ * "waves" (0 default = each kernel's own choice of grid size, in waves of resident thread blocks: one for the
+ * interpreter kernels, whose blocks pay a fixed set-up -- program staging and linking; up to 16 for compiled
+ * elementwise kernels, 8 for compiled multi-tensor kernels, 1 or 4 for compiled row kernels),
  * "stage" (3 default: inputs are copied asynchronously into per-thread shared-memory staging buffers a few
  * chunks ahead of their use when at least this many buffers fit in 64 KB per block -- fewer measured slower than
  * loading at first use with L2 prefetch; launches that give a thread one or two chunks stage anyway, to fetch all
