@@ -20,6 +20,8 @@ cudaError_t lt_compiled_launch(int id, const void *params, int u, unsigned grid,
                                unsigned group_log2, unsigned depth, cudaStream_t stream);
 cudaError_t lt_compiled_occupancy(int id, int u, int threads, size_t dyn_smem, int *blocks_per_sm);
 size_t lt_compiled_row_stage_bytes(int id, int u);
+// 1 if the entry's row kernel gains from the staging ring, 0 for issue-bound programs (random-bit generation).
+int lt_compiled_prefers_staging(int id);
 // Accesses the compiled shells found outside their slots since the library was loaded (debug build with
 // -DLT_DEBUG_BOUNDS only): 0 = *out is valid, 1 = not a debug build, -1 = the read failed.  Synchronises the device.
 int lt_compiled_bounds_violations(unsigned long long *out);

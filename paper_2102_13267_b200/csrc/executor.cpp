@@ -298,7 +298,8 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                     const unsigned threads = grp > 128 ? grp : 128;
                     // pipeline depth: stages of the next blocks' inputs in shared memory, within ~72 KB per CTA
                     const size_t stage = lt_compiled_row_stage_bytes(L.compiled, u);
-                    unsigned depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth : 2u;
+                    unsigned depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth
+                                                                       : (lt_compiled_prefers_staging(L.compiled) ? 2u : 0u);
                     while (depth > 0 && depth * stage > 72u * 1024u) --depth;
                     if (stage == 0 || threads != 128 || depth < 2) depth = 0;
                     const int occ = compiled_blocks(L, u, (int)threads, depth * stage);
