@@ -11,10 +11,14 @@
 // entry serves every shape and every value of the dynamic scalars.
 //
 // Three shells, as for the interpreter:
-//   lt_c_ew     grid-stride over chunks of 8 elements, U chunks in flight per thread
+//   lt_c_ew     chunks of 8 elements strided over the grid, U chunks in flight per thread; many short CTAs
+//               (a compiled CTA has no set-up to amortise)
 //   lt_c_row    a power-of-two group of threads owns a row and keeps it in registers (U chunks of
 //               8 elements per thread) across the row reductions; groups of up to 32 threads reduce
-//               with shuffles alone, larger ones exchange warp partials through shared memory
+//               with shuffles alone, larger ones exchange warp partials through shared memory.
+//               Persistent CTAs; the inputs of the next blocks of rows travel through a cp.async
+//               staging ring (not for programs bound by integer issue), small column vectors are
+//               loaded once per thread
 //   lt_c_multi  one program over many tensors; a CTA takes super-chunks of 16384 elements and
 //               finds the owning tensor by binary search over a prefix table in the parameters
 // Every global access is a 128-bit (64-bit for one-byte types) access of a full chunk; full-class
