@@ -43,14 +43,17 @@ import pynvml as nv
 nv.nvmlInit()
 h = nv.nvmlDeviceGetHandleByIndex(int(sys.argv[1]))
 mx = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
-print("max", mx, flush=True)
-while True:
+def sample():
     try:
         r = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
     except Exception:
         r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
-    print(time.time(), nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM), int(r), flush=True)
-    time.sleep(0.004)
+    return time.time(), nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM), int(r)
+sample()  # the first query of each kind can take a long time: get it over with before reporting ready
+print("max", mx, flush=True)
+while True:
+    print(*sample(), flush=True)
+    time.sleep(0.0005)
 """
 
 _REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
@@ -269,24 +272,54 @@ def run_ours(args) -> None:
         torch.cuda.synchronize()
         return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
+    # Every rotating set is flushed before anything is timed, whatever --warmup says: the first flush on a set
+    # obtains its output block from the allocator (a cudaMalloc of 64 MiB takes milliseconds), later ones reuse
+    # the block the context's pool got back when the previous output of that set was dropped.
+    for i in range(N_SETS + 2):
+        step(i)
     for i in range(max(args.warmup, 3)):
         step(i)
     sampler = ClockSampler(local) if rank == 0 else None
     sync_all()
     ctx.reset_stats()
+    host_s = [0.0]
+
+    def timed_steps(n_steps: int) -> float:
+        """Exactly n_steps steps between two events.  A short spin kernel ahead of the first event lets the host
+        get a few steps ahead, as it is in the steady state of a long run, so that a 20-step region is not
+        dominated by the first launch's latency; the spin itself ends before the first event is recorded."""
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(1.0e-3 * 1.9e9))
+        e0.record()
+        n_host = min(n_steps, 200)  # the host's own pace: taken while the launch queue cannot be full yet
+        h0 = time.perf_counter()
+        for i in range(n_host):
+            step(i)
+        host_s[0] = (time.perf_counter() - h0) / max(n_host, 1)
+        for i in range(n_host, n_steps):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
+
     w0 = time.time()
-    ms = timed(args.steps, step)
-    w1 = time.time()
+    ms = timed_steps(args.steps)
     st = ctx.stats()
-    clocks = sampler.stop(w0, w1) if sampler else None
+    host_us_per_step = 1e6 * host_s[0]
     value = aggregate_gbs(nbytes, args.steps, world, ms)
     ms_local = ms  # (max over ranks; at one GPU this rank's own time)
-    # second pass with every launch bracketed by its own pair of events (costs ~2 us per step on the stream)
+    # second pass with every launch bracketed by its own pair of events (costs ~2 us per step on the stream);
+    # long enough (>= 2000 launches of the same kernel on the same buffers) for the clock sampler to see the load
     ctx.set_kernel_timing(True)
     ctx.kernel_timing()
-    timed(min(args.steps, 1000), step)
+    timed(max(min(args.steps, 4000), 2000), step)
     kt = ctx.kernel_timing()
     ctx.set_kernel_timing(False)
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1) if sampler else None
+    if clocks is not None:
+        clocks["window"] = "timed region + the bracketed pass that follows it (same kernel, same buffers)"
 
     # ---- end to end through the C ABI with host buffers: H2D of the inputs and D2H of the result every step
     e2e_steps = max(3, min(args.steps, 30))
@@ -358,7 +391,10 @@ def run_ours(args) -> None:
     achieved = nbytes / (avg_ms / 1e3) / 1e9 if avg_ms > 0 else 0.0
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": ncu_traffic(), "peak_source": peak_src, "kernel": kernel_name,
-                "launch_us": 1e3 * avg_ms, "bytes_per_launch": nbytes, "frac_of_8TBs_nominal": achieved / 8000.0,
+                "launch_us": 1e3 * avg_ms, "host_us_per_step": host_us_per_step,
+                "paced_by": "gpu" if host_us_per_step < 1e3 * avg_ms else "host (the figure is not the kernel's rate)",
+                "allocator_calls_in_timed_region": int(st["allocator_calls"]),
+                "bytes_per_launch": nbytes, "frac_of_8TBs_nominal": achieved / 8000.0,
                 "timing": "events around the timed region / launches (one launch per step, back to back)",
                 "launch_us_bracketed": 1e3 * bracket_ms,
                 "frac_bracketed": (nbytes / (bracket_ms / 1e3) / 1e9 / peak) if bracket_ms > 0 else None}
@@ -401,7 +437,7 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
     out = {}
     n = 200
     # the same graph traced from primitive ops (16 ops) instead of the gelu_tanh op
-    for i in range(5):
+    for i in range(len(sets) + 2):
         step(i, True)
     ms = timed(n, lambda i: step(i, True))
     out["c2_primitive_trace_gbs"] = nbytes * n / (ms / 1e3) / 1e9
@@ -417,7 +453,7 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
         un.barrier()
 
     for prim, key in ((False, "c2_unfused_gbs"), (True, "c2_primitive_unfused_gbs")):
-        for i in range(3):
+        for i in range(len(usets) + 2):
             ustep(i, prim)
         ms = timed(50, lambda i: ustep(i, prim))
         out[key] = nbytes * 50 / (ms / 1e3) / 1e9
@@ -426,7 +462,7 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
     out["c2_fused_gbs"] = nbytes * n / (ms_f / 1e3) / 1e9
     # the same fused graph on the interpreter kernel (ahead-of-time compiled kernels switched off)
     ctx.set_option("compiled", 0)
-    for i in range(3):
+    for i in range(len(sets) + 2):
         step(i)
     ms_i = timed(n, step)
     ctx.set_option("compiled", 1)
@@ -489,10 +525,12 @@ def other_configs(lt, torch, device: int) -> dict:
                 c.set_option("fusion", 0)
             sets = [make(c) for _ in range(nsets)]
             keep = [None] * nsets
-            for i in range(3):
+            warm = nsets + 2  # every set flushed once: no allocator call is left for the timed flushes
+            for i in range(warm):
                 keep[i % nsets] = trace(c, sets[i % nsets])
                 c.barrier()
             torch.cuda.synchronize()
+            c.reset_stats()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda._sleep(int(4e-3 * 1.9e9))  # the flushes queue up behind this and then run back to back
             e0.record()
@@ -504,7 +542,8 @@ def other_configs(lt, torch, device: int) -> dict:
             ms = e0.elapsed_time(e1) / iters
             entry[f"{mode}_us"] = 1e3 * ms
             entry[f"{mode}_gbs"] = nbytes / ms / 1e6
-            entry[f"{mode}_launches"] = c.stats()["kernels_launched"] // (iters + 3)
+            entry[f"{mode}_launches"] = c.stats()["kernels_launched"] // iters
+            entry[f"{mode}_allocator_calls"] = c.stats()["allocator_calls"]
             del keep, sets
             c.close()
         entry["frac_of_measured_peak"] = entry["fused_gbs"] / peak

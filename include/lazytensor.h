@@ -128,6 +128,9 @@ typedef struct {
     uint64_t ns_rebind;          /* turning roots into device-data leaves, freeing IR        */
     uint64_t launches_compiled;  /* of kernels_launched: ahead-of-time compiled programs     */
     uint64_t replays;            /* lt_replay calls that ran a plan                          */
+    uint64_t allocator_calls;    /* calls of the allocator's alloc and free (or cudaMallocAsync /
+                                    cudaFreeAsync); 0 over a span means every block came from and
+                                    went back to the context's own pool of released blocks          */
 } lt_stats;
 
 /* Device time per kernel family, measured with CUDA events when kernel timing is on. */

@@ -16,7 +16,7 @@ CU_SOURCES = ["kernels.cu", "compiled.cu", "static_scratch.cu"]
 CPP_SOURCES = ["engine.cpp", "canon.cpp", "planner.cpp", "executor.cpp"]
 HEADERS = ["engine.h", "vm.h", "launch.h", "vm_core.inc", "vm_ops.cuh", "compiled.h", "compiled_programs.inc", "../../include/lazytensor.h"]
 
-NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-diag-suppress", "177",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 CXX_FLAGS = ["-O2", "-std=c++17", "-fPIC", "-Wall", "-Wno-unused-function", f"-I{CUDA_HOME}/include"]
 

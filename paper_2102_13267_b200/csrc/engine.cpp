@@ -295,6 +295,7 @@ void buffer_unref(lt_ctx *c, uint32_t b) {
 // stream, so a block freed after the last kernel using it was enqueued can be reused by the next
 // flush at once.  In steady state (same graph every step) a flush makes no allocator call at all.
 static void *raw_alloc(lt_ctx *c, size_t bytes) {
+    c->stats.allocator_calls++;
     if (c->has_alloc) return c->alloc.alloc(bytes, (void *)c->stream, c->alloc.user);
     if (c->device == LT_DEVICE_NONE) return malloc(bytes);
     void *p = nullptr;
@@ -306,6 +307,7 @@ static void *raw_alloc(lt_ctx *c, size_t bytes) {
 }
 
 static void raw_free(lt_ctx *c, void *p) {
+    c->stats.allocator_calls++;
     if (c->has_alloc) c->alloc.free(p, (void *)c->stream, c->alloc.user);
     else if (c->device == LT_DEVICE_NONE) free(p);
     else cudaFreeAsync(p, c->stream);

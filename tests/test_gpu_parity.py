@@ -58,8 +58,6 @@ def test_c1_chain(ctx, shape):
 @pytest.mark.parametrize("shape", [(33, 40), (17, 36), (1, 8), (5, 7), (128, 4096), (8192, 4096)])
 @pytest.mark.parametrize("primitive", [True, False])
 def test_c2_mlp_epilogue(ctx, shape, primitive):
-    if shape == (8192, 4096) and not primitive:
-        pytest.skip("full size runs the primitive trace")
     x, h, b = configs.c2_inputs(2, shape)
     O, ol, gl = both(ctx, [(x, "bf16"), (h, "bf16"), (b, "bf16")])
     ref = traces.mlp_epilogue(O, *ol, primitive_gelu=primitive)
@@ -76,8 +74,6 @@ def test_c2_mlp_epilogue(ctx, shape, primitive):
                                    (4, 3, 64), (16384, 1024)])
 @pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
 def test_c3_residual_dropout_layernorm(ctx, shape, out_dtype):
-    if shape == (16384, 1024) and out_dtype == "f32":
-        pytest.skip("full size runs the bf16 variant")
     x, h, g, b = configs.c3_inputs(3, shape)
     O, ol, gl = both(ctx, [(x, "bf16"), (h, "bf16"), (g, "f32"), (b, "f32")])
     kw = dict(shape=shape, p=0.1, eps=1e-5, seed=0xDEADBEEF12345, offset=7, out_dtype=out_dtype)
@@ -115,8 +111,6 @@ def test_residual_layernorm_without_dropout(ctx, shape):
                                    (16, 2048, 2048)])
 @pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
 def test_c4_causal_softmax(ctx, shape, out_dtype):
-    if shape == (16, 2048, 2048) and out_dtype == "f32":
-        pytest.skip("full size runs the bf16 variant")
     s = configs.c4_inputs(4, shape)
     O, ol, gl = both(ctx, [(s, "bf16")])
     kw = dict(shape=shape, scale=1.0 / math.sqrt(128.0), out_dtype=out_dtype)
@@ -161,6 +155,31 @@ def test_c5_adam_small(ctx):
     shapes = parameter_shapes()[:14] + [(1000,), (7,), (3, 5, 1, 1)]
     s = _adam_case(ctx, shapes, steps=4)
     assert s["kernels_launched"] == 4  # one multi-tensor launch per step
+
+
+def test_c5_adam_100_steps(ctx):
+    """The workload as specified: 100 steps, one barrier per step, 1 compile + 99 cache hits, on a reduced set of
+    the parameter shapes (the oracle runs every step too).  Three tensors are compared after every step, all of them
+    after the last."""
+    shapes = parameter_shapes()[:14] + [(1000,), (7,), (3, 5, 1, 1)]
+    params, grads, ms, vs = configs.c5_inputs(55, shapes)
+    O = EagerOracle()
+    op, og, om, ov = ([O.leaf(a, "f32") for a in arrs] for arrs in (params, grads, ms, vs))
+    gp, gg, gm, gv = ([ctx.leaf(a, "f32") for a in arrs] for arrs in (params, grads, ms, vs))
+    ptrs = [ctx.device_ptr(t) for t in gp + gm + gv]
+    watch = (0, 7, len(shapes) - 2)
+    for step in range(1, 101):
+        traces.adam_step(O, op, og, om, ov, step=step)
+        traces.adam_step(ctx, gp, gg, gm, gv, step=step)
+        ctx.barrier()
+        for i in (watch if step < 100 else range(len(shapes))):
+            for name, a, b in (("p", gp[i], op[i]), ("m", gm[i], om[i]), ("v", gv[i], ov[i])):
+                assert_matches(ctx.fetch(a), b.array, "f32", f"c5 step {step} {name}[{i}] {shapes[i]}")
+    assert [ctx.device_ptr(t) for t in gp + gm + gv] == ptrs
+    s = ctx.stats()
+    assert (s["compiles"], s["cache_hits"]) == (1, 99)
+    assert s["kernels_launched"] == 100 and s["launches_multi"] == 100
+    assert s["outputs_allocated"] == 0 and s["outputs_donated"] == 3 * len(shapes) * 100
 
 
 def test_c5_adam_full_shapes(ctx):

@@ -175,6 +175,113 @@ def test_integer_and_mask_ops_bruteforce(B):
     np.testing.assert_array_equal(B.op("where", m1, x, B.scalar(0.0)).array, f32(1, 0, 3, 0))
 
 
+def test_bitwise_ops_hand_table_and_numpy(B):
+    # hand table, one byte: a mistake that swaps | and ^ (or & and |) fails on 0b1100 / 0b1010
+    m1 = leaf(B, np.array([0b1100, 0xFF, 0x00, 0x5A], dtype=np.uint8), "u8")
+    m2 = leaf(B, np.array([0b1010, 0x0F, 0x00, 0xA5], dtype=np.uint8), "u8")
+    np.testing.assert_array_equal(B.op("and", m1, m2).array, [0b1000, 0x0F, 0x00, 0x00])
+    np.testing.assert_array_equal(B.op("or", m1, m2).array, [0b1110, 0xFF, 0x00, 0xFF])
+    np.testing.assert_array_equal(B.op("xor", m1, m2).array, [0b0110, 0xF0, 0x00, 0xFF])
+    # 32-bit lanes: every byte of the word takes part (a one-byte element size would leave the upper bytes alone)
+    g = rng.generator(21)
+    for dt, npdt in (("i32", np.int32), ("u32", np.uint32)):
+        a = g.integers(0, 2**32, size=(13, 9), dtype=np.uint64).astype(np.uint32).view(npdt)
+        b = g.integers(0, 2**32, size=(13, 9), dtype=np.uint64).astype(np.uint32).view(npdt)
+        a.flat[:3] = np.array([0x0F0F0F0F, 0xFFFFFFFF, 0x80000000], dtype=np.uint32).view(npdt)
+        b.flat[:3] = np.array([0x00FF00FF, 0x00000000, 0x80000001], dtype=np.uint32).view(npdt)
+        for name, fn in (("and", np.bitwise_and), ("or", np.bitwise_or), ("xor", np.bitwise_xor)):
+            got = B.op(name, leaf(B, a, dt), leaf(B, b, dt)).array
+            np.testing.assert_array_equal(got, fn(a, b), err_msg=f"{name} {dt}")
+        assert B.op("and", leaf(B, a, dt), leaf(B, b, dt)).array.flat[0] == 0x000F000F
+        assert B.op("or", leaf(B, a, dt), leaf(B, b, dt)).array.view(np.uint32).flat[0] == 0x0FFF0FFF
+        assert B.op("xor", leaf(B, a, dt), leaf(B, b, dt)).array.view(np.uint32).flat[0] == 0x0FF00FF0
+    # unsigned arithmetic and unsigned max/min (the top bit is magnitude, not sign)
+    ua = np.array([0, 1, 0xFFFFFFFF, 0x80000000, 7], dtype=np.uint32)
+    ub = np.array([5, 0xFFFFFFFF, 2, 0x7FFFFFFF, 7], dtype=np.uint32)
+    with np.errstate(over="ignore"):
+        for name, fn in (("add", np.add), ("sub", np.subtract), ("mul", np.multiply), ("max", np.maximum),
+                         ("min", np.minimum)):
+            np.testing.assert_array_equal(B.op(name, leaf(B, ua, "u32"), leaf(B, ub, "u32")).array, fn(ua, ub),
+                                          err_msg=f"{name} u32")
+    assert list(B.op("max", leaf(B, ua, "u32"), leaf(B, ub, "u32")).array[2:4]) == [0xFFFFFFFF, 0x80000000]
+
+
+def test_integer_neg_abs_hand_cases(B):
+    a = np.array([0, 1, -1, 5, -5, 2**31 - 1, -(2**31) + 1, -(2**31)], dtype=np.int32)
+    A = leaf(B, a, "i32")
+    # two's complement: the most negative value is its own negation and its own absolute value
+    np.testing.assert_array_equal(B.op("neg", A).array,
+                                  np.array([0, -1, 1, -5, 5, -(2**31) + 1, 2**31 - 1, -(2**31)], dtype=np.int32))
+    np.testing.assert_array_equal(B.op("abs", A).array,
+                                  np.array([0, 1, 1, 5, 5, 2**31 - 1, 2**31 - 1, -(2**31)], dtype=np.int32))
+    g = rng.generator(22)
+    r = g.integers(-(2**31) + 1, 2**31, size=1000, dtype=np.int64).astype(np.int32)
+    np.testing.assert_array_equal(B.op("neg", leaf(B, r, "i32")).array, -r)
+    np.testing.assert_array_equal(B.op("abs", leaf(B, r, "i32")).array, np.abs(r))
+
+
+def test_integer_converts_hand_cases(B):
+    u8 = np.array([0, 1, 2, 127, 128, 255], dtype=np.uint8)
+    # u8 -> i32 / u32 zero-extends (128..255 stay positive)
+    np.testing.assert_array_equal(B.op("convert", leaf(B, u8, "u8"), dtype="i32").array,
+                                  np.array([0, 1, 2, 127, 128, 255], dtype=np.int32))
+    np.testing.assert_array_equal(B.op("convert", leaf(B, u8, "u8"), dtype="u32").array,
+                                  np.array([0, 1, 2, 127, 128, 255], dtype=np.uint32))
+    # i32 <-> u32 keeps the bit pattern
+    i = np.array([0, 1, -1, -(2**31), 2**31 - 1, -256], dtype=np.int32)
+    np.testing.assert_array_equal(B.op("convert", leaf(B, i, "i32"), dtype="u32").array,
+                                  np.array([0, 1, 2**32 - 1, 2**31, 2**31 - 1, 2**32 - 256], dtype=np.uint32))
+    u = np.array([0, 1, 2**32 - 1, 2**31, 2**31 - 1, 2**32 - 256], dtype=np.uint32)
+    np.testing.assert_array_equal(B.op("convert", leaf(B, u, "u32"), dtype="i32").array, i)
+    # integers -> u8 is (x != 0), not truncation: 256 and 0x80000000 have a zero low byte and still give 1
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, np.array([0, 1, -1, 256, -(2**31), 65536], np.int32), "i32"), dtype="u8").array,
+        [0, 1, 1, 1, 1, 1])
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, np.array([0, 3, 256, 2**31, 2**32 - 1], np.uint32), "u32"), dtype="u8").array,
+        [0, 1, 1, 1, 1])
+    np.testing.assert_array_equal(
+        B.op("convert", leaf(B, np.array([0, 1, 2, 128, 255], np.uint8), "u8"), dtype="u8").array, [0, 1, 1, 1, 1])
+    # same-width identity converts
+    np.testing.assert_array_equal(B.op("convert", leaf(B, i, "i32"), dtype="i32").array, i)
+    np.testing.assert_array_equal(B.op("convert", leaf(B, u, "u32"), dtype="u32").array, u)
+
+
+def test_compare_on_u8_bruteforce(B):
+    vals = np.array([0, 1, 2, 127, 128, 255], dtype=np.uint8)
+    a, b = np.meshgrid(vals, vals, indexing="ij")  # every ordered pair; 128 > 127 fails a signed-char compare
+    a, b = np.ascontiguousarray(a), np.ascontiguousarray(b)
+    for name, fn in (("gt", np.greater), ("ge", np.greater_equal), ("lt", np.less), ("le", np.less_equal),
+                     ("eq", np.equal), ("ne", np.not_equal)):
+        got = B.op(name, leaf(B, a, "u8"), leaf(B, b, "u8")).array
+        np.testing.assert_array_equal(got, fn(a.astype(np.int64), b.astype(np.int64)).astype(np.uint8), err_msg=name)
+    assert B.op("gt", leaf(B, np.array([128], np.uint8), "u8"), leaf(B, np.array([127], np.uint8), "u8")).array[0] == 1
+
+
+def test_where_on_narrow_and_integer_elements(B):
+    m = np.array([1, 0, 2, 0, 255, 0, 1], dtype=np.uint8)  # any non-zero byte selects the first branch
+    M = leaf(B, m, "u8")
+    sel = m != 0
+    # bf16 (2-byte elements): distinct bit patterns in both bytes, so a 1-byte or 4-byte copy shows
+    xa = np.array([0x3F80, 0xC000, 0x4049, 0x7F80, 0x0001, 0x8000, 0x1234], dtype=np.uint16)
+    xb = np.array([0xBF80, 0x4000, 0xC049, 0xFF80, 0x8001, 0x0000, 0x4321], dtype=np.uint16)
+    np.testing.assert_array_equal(B.op("where", M, leaf(B, xa, "bf16"), leaf(B, xb, "bf16")).array,
+                                  np.where(sel, xa, xb))
+    # u8 (1-byte elements)
+    ua = np.arange(10, 17, dtype=np.uint8)
+    ub = np.arange(200, 207, dtype=np.uint8)
+    np.testing.assert_array_equal(B.op("where", M, leaf(B, ua, "u8"), leaf(B, ub, "u8")).array, np.where(sel, ua, ub))
+    assert list(B.op("where", M, leaf(B, ua, "u8"), leaf(B, ub, "u8")).array) == [10, 201, 12, 203, 14, 205, 16]
+    # i32 / u32 (4-byte elements) with the mask broadcast along rows
+    ia = np.arange(14, dtype=np.int32).reshape(2, 7) - 5
+    ib = -ia * 1000 - 1
+    np.testing.assert_array_equal(B.op("where", M, leaf(B, ia, "i32"), leaf(B, ib, "i32")).array,
+                                  np.where(sel[None, :], ia, ib))
+    np.testing.assert_array_equal(
+        B.op("where", M, leaf(B, ia.view(np.uint32), "u32"), leaf(B, ib.view(np.uint32), "u32")).array,
+        np.where(sel[None, :], ia, ib).view(np.uint32))
+
+
 def test_float_compare_nan(B):
     a, b = leaf(B, f32(float("nan"), 1.0)), leaf(B, f32(1.0, 1.0))
     assert list(B.op("eq", a, b).array) == [0, 1]
