@@ -20,7 +20,9 @@
  *     leaves the pending graph in place so it can be flushed again.
  *   - "host" pointers are ordinary process memory; "device" pointers are CUDA global
  *     memory on the context's device.
- *   - A context and its tensors may be used by one thread at a time.
+ *   - A context and its tensors may be used by one thread at a time.  Calls that touch the device make the
+ *     context's device current for their duration and restore the caller's; the stream given to
+ *     lt_ctx_create must belong to that device.
  *   - Tensors are dense, row-major, contiguous.  Rank is at most LT_MAX_RANK.
  *   - Handles belong to the context that made them; a handle used with another
  *     context gives LT_ERR_DEVICE (Section 4.1: no implicit cross-device transfers).
@@ -52,7 +54,9 @@ typedef enum {
     LT_ERR_UNSUPPORTED = 5,   /* op or shape outside what the kernels implement          */
     LT_ERR_OOM = 6,           /* the allocator callback returned NULL                    */
     LT_ERR_CUDA = 7,          /* a CUDA runtime call failed (message has the CUDA text)  */
-    LT_ERR_DEVICE_TIMEOUT = 8 /* a bounded device-side wait gave up                      */
+    LT_ERR_DEVICE_TIMEOUT = 8 /* a bounded device-side wait gave up: reported by the first blocking call
+                                 (lt_barrier with blocking set, lt_fetch) after a kernel that stages long
+                                 rows through shared memory ran out of polls on a copy's completion      */
 } lt_status;
 
 typedef enum { LT_F32 = 0, LT_BF16 = 1, LT_U8 = 2, LT_I32 = 3, LT_U32 = 4 } lt_dtype;
@@ -159,24 +163,17 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * "ieee" (0 default: in groups storing f32, division, square root and reciprocal are accurate to
  * 2 ulp; 1 = correctly rounded, so that a graph of + - * / sqrt matches an op-by-op binary32
  * evaluation bit for bit, at about ten more instructions per element and op),
- * "waves" (0 default = each kernel's own choice of grid size, in waves of resident thread blocks: one for the
- * interpreter kernels, whose blocks pay a fixed set-up -- program staging and linking; up to 16 for compiled
- * elementwise kernels, 8 for compiled multi-tensor kernels, 1 or 4 for compiled row kernels),
- * "stage" (3 default: inputs are copied asynchronously into per-thread shared-memory staging buffers a few
- * chunks ahead of their use when at least this many buffers fit in 64 KB per block -- fewer measured slower than
- * loading at first use with L2 prefetch; launches that give a thread one or two chunks stage anyway, to fetch all
- * inputs in parallel; 0 = never stage),
  * "cache_capacity" (0 = unbounded),
  * "compiled" (1 default: a launch whose program is in the table of ahead-of-time compiled programs, whose
  * pointers are 16-byte aligned and whose rows are a multiple of 8 elements runs on that kernel; 0 = always
- * interpret), "compiled_u" / "compiled_row_u" / "compiled_depth" (0 / 0 / -1 default = the library's choice:
- * chunks of 8 elements in flight per thread in compiled elementwise and multi-tensor kernels, chunks per thread
- * in compiled row kernels, depth of their shared-memory staging ring -- tuning knobs for measurements),
+ * interpret),
  * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
  * line per flush and per replay; preset by the environment variable LT_LOG),
  * "pool_bytes" (4 GiB default: device blocks the library has released are kept, up to this total, and reused
  * by later flushes before the allocator is asked; 0 = return every block at once).
  * fusion, fast_math, horizontal and ieee are part of the cache key; the others act at launch time.
+ * Keys that start with "debug." select launch shapes for measurements (grid size in waves, chunks in flight
+ * per thread, staging depth); they never change a result, are not part of the interface and may vanish.
  * Unknown key: LT_ERR_INVALID_ARG.  The environment variables LT_FUSION, LT_VERIFY,
  * LT_FAST_MATH, LT_HORIZONTAL preset the same options at context creation.
  */
@@ -239,11 +236,10 @@ lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
 lt_status lt_barrier(lt_ctx *ctx, int blocking);
 
 /*
- * Replay (Section 8, future work: "provide users with a way to guarantee that the underlying
- * computation of a tensor is going to remain the same across steps", so that "the IR graph
- * construction" can be skipped "after constructing it in the usual way during the first
- * iteration").  lt_replay runs the graph of the previous successful lt_barrier again -- no
- * recording, canonicalising or hashing -- as if the caller had issued the same lt_op / lt_assign
+ * Replay (Section 7, future work, proposes it: when the user can promise that a step's computation
+ * stays the same from one iteration to the next, the graph only has to be built during the first one).
+ * lt_replay runs the graph of the previous successful lt_barrier again -- no recording,
+ * canonicalising or hashing -- as if the caller had issued the same lt_op / lt_assign
  * calls on the same tensor handles once more:
  *   - every input is the current value of the tensor that supplied it last time (for an in-place
  *     update x := f(x, ...), the value the previous flush or replay left in x);

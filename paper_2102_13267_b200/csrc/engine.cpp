@@ -296,6 +296,7 @@ void buffer_unref(lt_ctx *c, uint32_t b) {
 // flush at once.  In steady state (same graph every step) a flush makes no allocator call at all.
 static void *raw_alloc(lt_ctx *c, size_t bytes) {
     c->stats.allocator_calls++;
+    DeviceScope on_device(c->has_alloc ? LT_DEVICE_NONE : c->device);
     if (c->has_alloc) return c->alloc.alloc(bytes, (void *)c->stream, c->alloc.user);
     if (c->device == LT_DEVICE_NONE) return malloc(bytes);
     void *p = nullptr;
@@ -308,6 +309,7 @@ static void *raw_alloc(lt_ctx *c, size_t bytes) {
 
 static void raw_free(lt_ctx *c, void *p) {
     c->stats.allocator_calls++;
+    DeviceScope on_device(c->has_alloc ? LT_DEVICE_NONE : c->device);
     if (c->has_alloc) c->alloc.free(p, (void *)c->stream, c->alloc.user);
     else if (c->device == LT_DEVICE_NONE) free(p);
     else cudaFreeAsync(p, c->stream);
@@ -395,7 +397,8 @@ lt_status lt_ctx_create(int device, void *cuda_stream, const lt_allocator *alloc
     env_opt("LT_HORIZONTAL", &c->opt.horizontal);
     env_opt("LT_LOG", &c->opt.log);
     if (device != LT_DEVICE_NONE) {
-        cudaError_t e = cudaSetDevice(device);
+        DeviceScope on_device(device);  // the caller's current device is put back when the call returns
+        cudaError_t e = on_device.ok() ? cudaSuccess : cudaErrorInvalidDevice;
         int sms = 0;
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
         if (e == cudaSuccess) e = lt_kernel_setup(LT_MAX_STAGE_BYTES);
@@ -418,6 +421,7 @@ lt_status lt_ctx_create(int device, void *cuda_stream, const lt_allocator *alloc
 
 lt_status lt_ctx_destroy(lt_ctx *c) {
     if (!c) return LT_ERR_INVALID_ARG;
+    DeviceScope on_device(c->device);
     if (c->device != LT_DEVICE_NONE) cudaStreamSynchronize(c->stream);
     for (auto &t : c->timed) {
         cudaEventDestroy(t.start);
@@ -439,17 +443,17 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "horizontal")) c->opt.horizontal = value;
     else if (!strcmp(key, "cache_capacity")) c->opt.cache_capacity = value;
     else if (!strcmp(key, "ieee")) c->opt.ieee = value;
-    else if (!strcmp(key, "waves")) c->opt.waves = value;
-    else if (!strcmp(key, "stage")) c->opt.stage = value;
+    else if (!strcmp(key, "debug.waves")) c->opt.waves = value;
+    else if (!strcmp(key, "debug.stage")) c->opt.stage = value;
     else if (!strcmp(key, "log")) c->opt.log = value;
     else if (!strcmp(key, "pool_bytes")) {
         c->opt.pool_bytes = value;
         pool_trim(c, value > 0 ? (size_t)value : 0);
     }
     else if (!strcmp(key, "compiled")) c->opt.compiled = value;
-    else if (!strcmp(key, "compiled_u")) c->opt.compiled_u = value;
-    else if (!strcmp(key, "compiled_row_u")) c->opt.compiled_row_u = value;
-    else if (!strcmp(key, "compiled_depth")) c->opt.compiled_depth = value;
+    else if (!strcmp(key, "debug.compiled_u")) c->opt.compiled_u = value;
+    else if (!strcmp(key, "debug.compiled_row_u")) c->opt.compiled_row_u = value;
+    else if (!strcmp(key, "debug.compiled_depth")) c->opt.compiled_depth = value;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
 }
@@ -488,6 +492,8 @@ lt_status lt_tensor_from_host(lt_ctx *c, const void *hptr, lt_dtype dtype, int r
     lt_status s = check_shape(c, rank, shape);
     if (s) return s;
     if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    DeviceScope on_device(c->device);
+    if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
     size_t bytes = (size_t)shape_numel(shape, rank) * dtype_size(dtype);
     if (!hptr && bytes) return fail(c, LT_ERR_INVALID_ARG, "host pointer is null");
     void *d = ctx_alloc(c, bytes);
@@ -790,6 +796,8 @@ lt_status lt_release_many(lt_ctx *c, const lt_tensor *handles, size_t n) {
 
 lt_status lt_barrier(lt_ctx *c, int blocking) {
     if (!c) return LT_ERR_INVALID_ARG;
+    DeviceScope on_device(c->device);
+    if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
     std::vector<uint32_t> &roots = c->roots_scratch;
     Canonical &cg = c->canon;
     {
@@ -913,6 +921,8 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
 
 lt_status lt_replay(lt_ctx *c, int blocking) {
     if (!c) return LT_ERR_INVALID_ARG;
+    DeviceScope on_device(c->device);
+    if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
     ReplayRecord &r = c->replay;
     if (!r.plan) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: no flushed graph to replay");
     if (!r.why_not.empty()) return fail(c, LT_ERR_UNSUPPORTED, "lt_replay: " + r.why_not);
@@ -1035,6 +1045,7 @@ lt_status lt_replay_set_slot(lt_ctx *c, uint32_t slot, int as_integer, double dv
 lt_status lt_debug_bounds_violations(lt_ctx *c, uint64_t *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
     if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_DEVICE, "lt_debug_bounds_violations needs a context on a CUDA device");
+    DeviceScope on_device(c->device);
     unsigned long long n = 0;
     const int r = lt_compiled_bounds_violations(&n);
     if (r == 1) return fail(c, LT_ERR_UNSUPPORTED, "the library was not built with -DLT_DEBUG_BOUNDS");
@@ -1053,6 +1064,8 @@ lt_status lt_fetch(lt_ctx *c, lt_tensor t, void *host_dst, size_t nbytes) {
     if (s) return s;
     if (!host_dst && nbytes) return fail(c, LT_ERR_INVALID_ARG, "host destination is null");
     if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    DeviceScope on_device(c->device);
+    if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
     if (!is_leaf(c->nodes[c->tensors[slot].node])) {
         s = lt_barrier(c, 1);
         if (s) return s;
@@ -1131,6 +1144,7 @@ lt_status lt_get_kernel_timing(lt_ctx *c, lt_kernel_timing *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
     memset(out, 0, sizeof(*out));
     if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    DeviceScope on_device(c->device);
     cudaError_t e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
     for (auto &t : c->timed) {

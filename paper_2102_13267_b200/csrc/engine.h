@@ -225,6 +225,7 @@ struct lt_ctx {
     // set only for the duration of lt_barrier_static_scratch: temporaries are carved out of this
     // fixed device range and nothing may be obtained from, or returned to, the allocator
     bool static_mode = false;
+    bool static_clear = false;  // zero-fill the range on the stream once the flush has passed its checks
     void *static_base = nullptr;
     size_t static_cap = 0;
 
@@ -264,6 +265,31 @@ lt_status fail(lt_ctx *c, lt_status s, const std::string &msg);
 void *ctx_alloc(lt_ctx *c, size_t bytes);
 void pool_trim(lt_ctx *c, size_t keep_bytes);
 void ctx_free(lt_ctx *c, void *p);
+
+// Makes `device` the calling thread's current CUDA device for the scope and puts the previous one back
+// afterwards: every entry point that enqueues work or touches device memory runs inside one, so a caller
+// that has switched devices since lt_ctx_create still launches on the context's stream's device.
+struct DeviceScope {
+    int previous = -1;
+    bool switched = false, good = true;
+    explicit DeviceScope(int device) {
+        if (device < 0) return;
+        if (cudaGetDevice(&previous) != cudaSuccess) {
+            good = false;
+            return;
+        }
+        if (previous != device) {
+            good = cudaSetDevice(device) == cudaSuccess;
+            switched = good;
+        }
+    }
+    ~DeviceScope() {
+        if (switched) cudaSetDevice(previous);
+    }
+    bool ok() const { return good; }
+    DeviceScope(const DeviceScope &) = delete;
+    DeviceScope &operator=(const DeviceScope &) = delete;
+};
 
 // canonicaliser (canon.cpp)
 void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonical &out);

@@ -108,6 +108,10 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             return fail(c, LT_ERR_UNSUPPORTED, "lt_barrier_static_scratch: the graph needs " + std::to_string(need) +
                                                    " bytes of temporaries, the static scratch array holds " +
                                                    std::to_string(c->static_cap));
+        if (c->static_clear && !dry) {
+            cudaError_t ce = lt_static_scratch_clear_enqueue(c->static_base, c->static_cap, c->sm_count, c->stream);
+            if (ce != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("clearing the static scratch: ") + cudaGetErrorString(ce));
+        }
     }
     uint64_t donated = 0, allocated = 0;
     for (size_t k = 0; k < n_out; ++k) {

@@ -19,3 +19,6 @@ cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, 
 // once per device: allow up to `max_stage_bytes` of dynamic shared memory for the staging buffers
 cudaError_t lt_kernel_setup(size_t max_stage_bytes);
 cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_256, int *multi_blocks_per_sm);
+
+// static_scratch.cu: zero-fills `bytes` of the fixed scratch array at `base` on `stream`
+cudaError_t lt_static_scratch_clear_enqueue(void *base, size_t bytes, int sm_count, cudaStream_t stream);

@@ -27,9 +27,8 @@ constexpr int kMaxDevices = 64;
 std::mutex g_setup_lock;
 void *g_scratch_addr[kMaxDevices];  // per device ordinal, filled on first use
 
-// Writes zeros over the first `n` 16-byte words of the array (device code may name it directly).
-__global__ void lt_static_scratch_clear(size_t n) {
-    uint4 *p = reinterpret_cast<uint4 *>(lt_static_scratch);
+// Writes zeros over `n` 16-byte words starting at `p` (the array's device address on the launching device).
+__global__ void lt_static_scratch_clear(uint4 *p, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
@@ -52,7 +51,28 @@ cudaError_t scratch_address(int device, void **out) {
     return cudaSuccess;
 }
 
+// Restores what the call changed on the context, whichever way the call ends.
+struct StaticModeScope {
+    lt_ctx *c;
+    StaticModeScope(lt_ctx *ctx, void *base) : c(ctx) {
+        c->static_base = base;
+        c->static_cap = LT_STATIC_SCRATCH_BYTES;
+        c->static_mode = true;
+    }
+    ~StaticModeScope() {
+        c->static_mode = false;
+        c->static_clear = false;
+    }
+};
+
 }  // namespace
+
+// Called by the executor once a flush in static mode has passed its checks (every result has a caller
+// buffer, the temporaries fit), just before the first kernel: a refused call leaves the array untouched.
+cudaError_t lt_static_scratch_clear_enqueue(void *base, size_t bytes, int sm_count, cudaStream_t stream) {
+    lt_static_scratch_clear<<<sm_count > 0 ? sm_count : 1, 256, 0, stream>>>(reinterpret_cast<uint4 *>(base), bytes / 16u);
+    return cudaGetLastError();
+}
 
 extern "C" __attribute__((visibility("default"))) lt_status lt_barrier_static_scratch(lt_ctx *c, int blocking,
                                                                                       int clear_first) {
@@ -65,17 +85,12 @@ extern "C" __attribute__((visibility("default"))) lt_status lt_barrier_static_sc
         cudaGetLastError();
         return lt::fail(c, LT_ERR_CUDA, std::string("cudaGetSymbolAddress(static scratch): ") + cudaGetErrorString(e));
     }
-    if (clear_first) {
-        // The array still holds what the previous flush left there.  No kernel of this library reads
-        // a temporary before writing it, so clearing is only for callers that want a known state.
-        lt_static_scratch_clear<<<148, 256, 0, c->stream>>>(LT_STATIC_SCRATCH_BYTES / 16u);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return lt::fail(c, LT_ERR_CUDA, std::string("clearing the static scratch: ") + cudaGetErrorString(e));
-    }
-    c->static_base = base;
-    c->static_cap = LT_STATIC_SCRATCH_BYTES;
-    c->static_mode = true;
-    const lt_status s = lt_barrier(c, blocking);
-    c->static_mode = false;
-    return s;
+    // The array still holds what the previous flush left there.  No kernel of this library reads a
+    // temporary before writing it, so clearing is only for callers that want a known state; the executor
+    // enqueues it after the graph has passed the checks of this mode.
+    lt::DeviceScope on_device(c->device);
+    if (!on_device.ok()) return lt::fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
+    StaticModeScope mode(c, base);
+    c->static_clear = clear_first != 0;
+    return lt_barrier(c, blocking);
 }

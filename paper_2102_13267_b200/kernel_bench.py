@@ -6,7 +6,7 @@ For each configuration: traces the graph and flushes it `iters` times over rotat
 together), queued behind a busy stream so that the GPU, not the host, sets the pace.  Two figures are printed:
 every launch between its own two CUDA events (`lt_set_kernel_timing`), and "back to back": one pair of events around
 all the launches, kernel timing off (for C5 the steps are replayed, the host cannot record 161 tensors that fast).
-`key=value` pairs are context options (e.g. fusion=0, compiled=0, ieee=1).  With `--iters 4 --sets 1` it is the
+`key=value` pairs are context options (e.g. fusion=0, compiled=0, ieee=1, debug.waves=2).  With `--iters 4 --sets 1` it is the
 small workload used for `ncu --set full` captures.
 """
 from __future__ import annotations
@@ -75,7 +75,7 @@ def main() -> None:
         ctx = context()
         sets = [make(ctx) for _ in range(nsets)]
         keep = [None] * nsets
-        for i in range(min(5, args.iters)):
+        for i in range(nsets + 2):  # every set flushed once: no allocator call is left for the timed flushes
             keep[i % nsets] = trace(ctx, sets[i % nsets])
             ctx.barrier()
         torch.cuda.synchronize()
@@ -139,7 +139,7 @@ def main() -> None:
         ctx = context()
         sets = [make(ctx) for _ in range(nsets)]
         keep = [None] * nsets
-        for i in range(5):
+        for i in range(nsets + 2):
             keep[i % nsets] = trace(ctx, sets[i % nsets], ishape[1])
             ctx.barrier()
         torch.cuda.synchronize()

@@ -6,8 +6,8 @@ buffers its host application handed it, a process that starts after another fram
 the rest of the GPU.  For them the library has one flush that places the values passed between
 its kernels in a fixed device array and writes every result over an input.  The test runs a graph
 that needs such in-between values (an unfused RMS-style normalisation, updated in place) through
-both flushes and compares them, twice in a row because the array keeps the previous call's data.
-The file sorts last so that a failure here cannot hide one elsewhere.
+both flushes and compares them with each other and with the CPU oracle's evaluation of the same
+ops, twice in a row because the array keeps the previous call's data.  The file sorts last so that a failure here cannot hide one elsewhere.
 """
 import numpy as np
 import pytest
@@ -63,13 +63,47 @@ def _run(static: bool, steps: int):
     return outs
 
 
+def _oracle(steps: int):
+    """The same ops, one at a time, on the CPU oracle."""
+    from oracle.eager import EagerOracle
+
+    O = EagerOracle()
+    xh, gh = _inputs()
+    x, g = O.leaf(xh, "f32"), O.leaf(gh, "f32")
+    outs = []
+    for _ in range(steps):
+        _record_update(O, x, g)
+        outs.append(O.fetch(x))
+    return outs
+
+
 def test_static_scratch_flush_matches_the_allocating_flush_twice_in_a_row():
     ref = _run(static=False, steps=2)
     got = _run(static=True, steps=2)
-    for r, g in zip(ref, got):
+    want = _oracle(steps=2)
+    for r, g, w in zip(ref, got, want):
         np.testing.assert_allclose(g, r, rtol=1e-5, atol=1e-6)
         assert np.array_equal(g, r)  # same kernels, same order: in fact identical
+        np.testing.assert_allclose(g, w, rtol=1e-5, atol=1e-6)  # and both agree with the op-by-op evaluation
+        np.testing.assert_allclose(r, w, rtol=1e-5, atol=1e-6)
     assert not np.array_equal(ref[0], ref[1])  # the second step really computed something new
+
+
+def test_static_scratch_flush_with_clear_first_and_another_current_device_setting():
+    """`clear_first` zero-fills the array after the checks and before the kernels; the result is unchanged."""
+    import torch
+
+    import paper_2102_13267_b200 as lt
+
+    ctx = lt.LazyContext(device=0)
+    ctx.set_option("fusion", 0)
+    xh, gh = _inputs()
+    xd, gd = torch.from_numpy(xh).cuda(), torch.from_numpy(gh).cuda()
+    x, g = ctx.from_torch(xd), ctx.from_torch(gd)
+    _record_update(ctx, x, g)
+    ctx.barrier_static_scratch(blocking=True, clear_first=True)
+    np.testing.assert_allclose(xd.cpu().numpy(), _oracle(steps=1)[0], rtol=1e-5, atol=1e-6)
+    ctx.close()
 
 
 def test_static_scratch_flush_refuses_what_it_cannot_place():
