@@ -14,7 +14,7 @@ CUDA_HOME = Path(os.environ.get("CUDA_HOME", "/usr/local/cuda"))
 
 CU_SOURCES = ["kernels.cu", "compiled.cu", "static_scratch.cu"]
 CPP_SOURCES = ["engine.cpp", "canon.cpp", "planner.cpp", "executor.cpp"]
-HEADERS = ["engine.h", "vm.h", "launch.h", "vm_core.inc", "vm_ops.cuh", "compiled.h", "compiled_programs.inc", "../../include/lazytensor.h"]
+HEADERS = ["engine.h", "vm.h", "launch.h", "vm_core.inc", "vm_ops.cuh", "compiled.h", "compiled_programs.inc", "pdl.cuh", "../../include/lazytensor.h"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-diag-suppress", "177",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

@@ -28,6 +28,7 @@
 #include <stdint.h>
 
 #include "compiled.h"
+#include "pdl.cuh"
 #include "vm.h"
 #include "vm_ops.cuh"
 
@@ -384,20 +385,25 @@ struct Machine {
     }
 
     // requests every full-class input of the iteration
+    __device__ __forceinline__ void issue_loads() { request<PG::n_pro>(ptr, ck, raw); }
+
+    // the same for the chunks `c` (this or a later iteration's), into `dst`
     template <int K = PG::n_pro>
-    __device__ __forceinline__ void issue_loads() {
+    static __device__ __forceinline__ void request(const Ptr &ptr, const Coords<U> &c, Raw (&dst)[NL][U]) {
         if constexpr (K < PG::n_ins) {
             constexpr uint32_t op = PG::ins[K].op;
             if constexpr (I::is_ld(op) || I::is_f2m(op)) {
                 constexpr int slot = PG::ins[K].imm;
                 if constexpr (PG::cls[slot] == LT_CLS_FULL) {
-                    constexpr int dt = PG::dtype[slot];
+                    constexpr int dt = PG::dtype[slot], sh = esz_shift(dt);
+                    const char *base = reinterpret_cast<const char *>(ptr(slot));
 #pragma unroll
                     for (int u = 0; u < U; ++u)
-                        if (!GUARD || ck.ok[u]) raw_load<dt>(raw[I::load_ordinal(K)][u], address<slot>(u), true);
+                        if (!GUARD || c.ok[u])
+                            raw_load<dt>(dst[I::load_ordinal(K)][u], base + (LT_CHECKED(c.flat0[u], V, ptr.extent(LT_CLS_FULL)) << sh), true);
                 }
             }
-            issue_loads<K + 1>();
+            request<K + 1>(ptr, c, dst);
         }
     }
 
@@ -704,6 +710,8 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_ew(const __grid_constant__ LtK
     const PtrK ptr{P};
     const ScalK scal{P};
     NoReduce red;
+    pdl_release();
+    pdl_wait();
     for (uint32_t c = blockIdx.x * C_THREADS + threadIdx.x; c < n_chunks; c += U * stride) {
         Coords<U> ck;
 #pragma unroll
@@ -759,6 +767,8 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
         }
     };
     const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(stage_mem);
+    pdl_release();
+    pdl_wait();
     if (depth) {  // requires blockDim.x == C_ROW_THREADS
         uint32_t rb = blockIdx.x;
         for (uint32_t d = 0; d < depth; ++d, rb += gridDim.x) {
@@ -824,6 +834,8 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_multi(const __grid_constant__ 
     NoReduce red;
     constexpr uint32_t PER_SUPER = LT_EW_THREADS * LT_MULTI_SUB;
     static_assert(LT_EW_THREADS == C_THREADS && LT_MULTI_SUB % U == 0, "super-chunk walk");
+    pdl_release();
+    pdl_wait();
     for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
         uint32_t lo = 0, hi = P.n_inst;
         while (hi - lo > 1) {
@@ -877,8 +889,7 @@ cudaError_t launch_row(const LtKParams &P, unsigned grid, unsigned threads, unsi
     const size_t dyn = (size_t)depth * Info<PG>::stage_bytes(U, C_ROW_THREADS);
     cudaError_t e = row_smem_attr((const void *)lt_c_row<PG, U>, dyn);
     if (e != cudaSuccess) return e;
-    lt_c_row<PG, U><<<grid, threads, dyn, stream>>>(P, group, group_log2, depth);
-    return cudaGetLastError();
+    return launch_pdl(lt_c_row<PG, U>, grid, threads, dyn, stream, P, (uint32_t)group, (uint32_t)group_log2, (uint32_t)depth);
 }
 
 template <class PG>
@@ -886,8 +897,7 @@ cudaError_t launch_one(const void *params, int u, unsigned grid, unsigned thread
                        unsigned depth, cudaStream_t stream) {
     if constexpr (PG::kind == 0) {
         const LtKParams &P = *static_cast<const LtKParams *>(params);
-        if (u >= 2) lt_c_ew<PG, 2><<<grid, C_THREADS, 0, stream>>>(P);
-        else lt_c_ew<PG, 1><<<grid, C_THREADS, 0, stream>>>(P);
+        return u >= 2 ? launch_pdl(lt_c_ew<PG, 2>, grid, C_THREADS, 0, stream, P) : launch_pdl(lt_c_ew<PG, 1>, grid, C_THREADS, 0, stream, P);
     } else if constexpr (PG::kind == 1) {
         const LtKParams &P = *static_cast<const LtKParams *>(params);
         if (u >= 8) return launch_row<PG, 8>(P, grid, threads, group, group_log2, depth, stream);
@@ -896,10 +906,8 @@ cudaError_t launch_one(const void *params, int u, unsigned grid, unsigned thread
         return launch_row<PG, 1>(P, grid, threads, group, group_log2, depth, stream);
     } else {
         const LtMultiParams &P = *static_cast<const LtMultiParams *>(params);
-        if (u >= 2) lt_c_multi<PG, 2><<<grid, C_THREADS, 0, stream>>>(P);
-        else lt_c_multi<PG, 1><<<grid, C_THREADS, 0, stream>>>(P);
+        return u >= 2 ? launch_pdl(lt_c_multi<PG, 2>, grid, C_THREADS, 0, stream, P) : launch_pdl(lt_c_multi<PG, 1>, grid, C_THREADS, 0, stream, P);
     }
-    return cudaGetLastError();
 }
 
 template <class PG, int U>

@@ -205,7 +205,8 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 if (ok) {
                     // two chunks in flight per thread and eight waves of blocks measured best for wide programs
                     // (four input streams) over many tensors of uneven size
-                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 2;
+                    // (one chunk with correctly rounded division and square root: their slow paths cost registers)
+                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : (L.flavour == 2 ? 1 : 2);
                     const int occ = compiled_blocks(L, u, LT_EW_THREADS);
                     const unsigned mwaves = c->opt.waves > 0 ? waves : 8u;  // C5: 116 us against 121 with two waves
                     unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * mwaves);

@@ -76,11 +76,18 @@ def programs():
         d = Dry()
         keep = traces.causal_softmax(d.ctx, d.leaf((2, 64, 64), "bf16"), shape=(2, 64, 64), scale=1 / math.sqrt(128), out_dtype=od)
         out.append((f"causal_softmax_{od}", d.keys()))
-    d = Dry()
-    shapes = [(64,), (128,)]
-    P, G, M, V = ([d.leaf(s, "f32") for s in shapes] for _ in range(4))
-    traces.adam_step(d.ctx, P, G, M, V, step=1)
-    out.append(("adam_step", d.keys()))
+    # Adam with the default arithmetic (division and square root within 2 ulp) and with ieee=1 (correctly rounded:
+    # bit-identical to an op-by-op binary32 evaluation)
+    for opts, suffix in (({}, ""), ({"ieee": 1}, "_ieee")):
+        d = Dry(**opts)
+        shapes = [(64,), (128,)]
+        P, G, M, V = ([d.leaf(s, "f32") for s in shapes] for _ in range(4))
+        traces.adam_step(d.ctx, P, G, M, V, step=1)
+        out.append(("adam_step" + suffix, d.keys()))
+    d = Dry(ieee=1)
+    a, b, c, e = (d.leaf((64, 64), "f32") for _ in range(4))
+    keep = traces.elementwise_chain(d.ctx, a, b, c, e)
+    out.append(("elementwise_chain_ieee", d.keys()))
     # common fusion groups beyond the benchmark's (workloads/idioms.py)
     for name, kinds, trace in idioms.ALL:
         d = Dry()

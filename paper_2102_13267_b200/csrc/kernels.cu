@@ -13,6 +13,7 @@
 #include <cstddef>
 
 #include "launch.h"
+#include "pdl.cuh"
 #include "vm.h"
 #include "vm_core.inc"
 #include "vm_ops.cuh"
@@ -584,6 +585,7 @@ __device__ __forceinline__ Chunk ew_chunk(const LtKParams &P, uint32_t c) {
 // ------------------------------------------------------------------ kernels
 template <int FLAV>
 __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(const __grid_constant__ LtKParams P) {
+    pdl_release();
     __shared__ __align__(16) Staged S;
     extern __shared__ __align__(16) unsigned char stage_mem[];
     const EnvK E{P};
@@ -607,6 +609,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
     __syncthreads();
     link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
     __syncthreads();
+    pdl_wait();  // everything above read only the parameter block
     const uint32_t c0 = blockIdx.x * blockDim.x + threadIdx.x;
     if (c0 >= n_chunks) return;
     // Software pipeline: the full-class inputs of the thread's next `depth` chunks are in flight as
@@ -627,6 +630,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_ew_kernel(
 
 template <int FLAV, int MAXT>
 __global__ void __launch_bounds__(MAXT, MAXT == 256 ? LT_EW_MIN_BLOCKS : 1) lt_row_kernel(const __grid_constant__ LtKParams P) {
+    pdl_release();
     __shared__ __align__(16) Staged S;
     extern __shared__ __align__(16) unsigned char stage_mem[];
     const EnvK E{P};
@@ -646,6 +650,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? LT_EW_MIN_BLOCKS : 1) lt_r
     __syncthreads();
     link_program(S, P.n_ins, P.io_dtype, P.io_class, false);
     __syncthreads();
+    pdl_wait();  // everything above read only the parameter block
     RowCtx rc;
     rc.smem = S.red;
     rc.phase = 0;
@@ -688,6 +693,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? LT_EW_MIN_BLOCKS : 1) lt_r
 
 template <int FLAV>
 __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kernel(const __grid_constant__ LtMultiParams P) {
+    pdl_release();
     __shared__ __align__(16) Staged S;
     extern __shared__ __align__(16) unsigned char stage_mem[];
     stage_program(S, P);
@@ -703,6 +709,7 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
     const uint32_t buf_bytes = P.stage_pieces * LT_VM_STAGE_PIECE;
     const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage_mem);
     const uint32_t buf0 = stage_base + threadIdx.x * 16u;
+    pdl_wait();  // everything above read only the parameter block
     for (uint32_t sc = blockIdx.x; sc < P.total_super; sc += gridDim.x) {
         // instance that owns super-chunk sc: last i with super_prefix[i] <= sc
         uint32_t lo = 0, hi = P.n_inst;
@@ -770,10 +777,9 @@ __global__ void __launch_bounds__(LT_EW_THREADS, LT_EW_MIN_BLOCKS) lt_multi_kern
 
 cudaError_t lt_launch_ew(const LtKParams &p, int flavour, unsigned grid, cudaStream_t stream) {
     const size_t dyn = (size_t)p.stage_depth * p.stage_pieces * LT_VM_STAGE_PIECE;
-    if (flavour == 0) lt_ew_kernel<0><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
-    else if (flavour == 1) lt_ew_kernel<1><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
-    else lt_ew_kernel<2><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
-    return cudaGetLastError();
+    if (flavour == 0) return launch_pdl(lt_ew_kernel<0>, grid, LT_EW_THREADS, dyn, stream, p);
+    else if (flavour == 1) return launch_pdl(lt_ew_kernel<1>, grid, LT_EW_THREADS, dyn, stream, p);
+    return launch_pdl(lt_ew_kernel<2>, grid, LT_EW_THREADS, dyn, stream, p);
 }
 
 cudaError_t lt_kernel_setup(size_t max_stage_bytes) {
@@ -792,23 +798,20 @@ cudaError_t lt_kernel_setup(size_t max_stage_bytes) {
 cudaError_t lt_launch_row(const LtKParams &p, int flavour, unsigned grid, unsigned threads, cudaStream_t stream) {
     const size_t dyn = (size_t)p.stage_depth * p.stage_pieces * LT_VM_STAGE_PIECE;
     if (threads <= 256) {
-        if (flavour == 0) lt_row_kernel<0, 256><<<grid, threads, dyn, stream>>>(p);
-        else if (flavour == 1) lt_row_kernel<1, 256><<<grid, threads, dyn, stream>>>(p);
-        else lt_row_kernel<2, 256><<<grid, threads, dyn, stream>>>(p);
-    } else {
-        if (flavour == 0) lt_row_kernel<0, 1024><<<grid, threads, 0, stream>>>(p);
-        else if (flavour == 1) lt_row_kernel<1, 1024><<<grid, threads, 0, stream>>>(p);
-        else lt_row_kernel<2, 1024><<<grid, threads, 0, stream>>>(p);
+        if (flavour == 0) return launch_pdl(lt_row_kernel<0, 256>, grid, threads, dyn, stream, p);
+        else if (flavour == 1) return launch_pdl(lt_row_kernel<1, 256>, grid, threads, dyn, stream, p);
+        return launch_pdl(lt_row_kernel<2, 256>, grid, threads, dyn, stream, p);
     }
-    return cudaGetLastError();
+    if (flavour == 0) return launch_pdl(lt_row_kernel<0, 1024>, grid, threads, (size_t)0, stream, p);
+    else if (flavour == 1) return launch_pdl(lt_row_kernel<1, 1024>, grid, threads, (size_t)0, stream, p);
+    return launch_pdl(lt_row_kernel<2, 1024>, grid, threads, (size_t)0, stream, p);
 }
 
 cudaError_t lt_launch_multi(const LtMultiParams &p, int flavour, unsigned grid, cudaStream_t stream) {
     const size_t dyn = (size_t)p.stage_depth * p.stage_pieces * LT_VM_STAGE_PIECE;
-    if (flavour == 0) lt_multi_kernel<0><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
-    else if (flavour == 1) lt_multi_kernel<1><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
-    else lt_multi_kernel<2><<<grid, LT_EW_THREADS, dyn, stream>>>(p);
-    return cudaGetLastError();
+    if (flavour == 0) return launch_pdl(lt_multi_kernel<0>, grid, LT_EW_THREADS, dyn, stream, p);
+    else if (flavour == 1) return launch_pdl(lt_multi_kernel<1>, grid, LT_EW_THREADS, dyn, stream, p);
+    return launch_pdl(lt_multi_kernel<2>, grid, LT_EW_THREADS, dyn, stream, p);
 }
 
 cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_256, int *multi_blocks_per_sm) {
