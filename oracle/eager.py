@@ -60,6 +60,8 @@ def lib():
         _lib.orc_iota.argtypes = [ctypes.c_int, P]
         _lib.orc_philox_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint64, P]
         _lib.orc_row_reduce.argtypes = [ctypes.c_char_p, P, P]
+        _lib.orc_col_reduce.argtypes = [ctypes.c_char_p, P, P]
+        _lib.orc_all_reduce.argtypes = [ctypes.c_char_p, P, P]
         _lib.orc_set_threads.argtypes = [ctypes.c_int]
         _lib.orc_philox4x32_10.argtypes = [ctypes.POINTER(ctypes.c_uint32)] * 3
         _lib.orc_philox4x32_10.restype = None
@@ -117,6 +119,8 @@ _COMPARE = {"gt", "ge", "lt", "le", "eq", "ne"}
 _UNARY = {"neg", "abs", "relu", "exp", "log", "tanh", "sqrt", "rsqrt", "recip", "square",
           "sigmoid", "gelu_tanh", "not"}
 _REDUCE = {"row_sum", "row_max", "row_min"}
+_COL_REDUCE = {"col_sum", "col_max", "col_min"}
+_ALL_REDUCE = {"all_sum", "all_max", "all_min"}
 
 
 class _Scalar:
@@ -206,6 +210,15 @@ class EagerOracle:
             (a,) = inputs
             out = self._new(a.shape[:-1] + (1,), a.dtype)
             self._check(L.orc_row_reduce(name.encode(), a._c(), out._c()), name)
+        elif name in _COL_REDUCE:
+            (a,) = inputs
+            out = self._new((1,) * (len(a.shape) - 1) + a.shape[-1:], a.dtype)
+            self._check(L.orc_col_reduce(name.encode(), a._c(), out._c()), name)
+        elif name in _ALL_REDUCE:
+            (a,) = inputs
+            out = self._new((), a.dtype)
+            self._check(L.orc_all_reduce(name.encode(), a._c(), out._c()), name)
+            out.array = out.array.reshape(())  # rank 0, like the traced op's result
         else:
             raise ValueError(f"unknown op {name!r}")
         return out

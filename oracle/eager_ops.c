@@ -414,6 +414,70 @@ int orc_iota(int dim, orc_array *out) {
     return ORC_OK;
 }
 
+/*
+ * Reductions over the other axes (the row reductions' siblings).
+ * "col_*": reduce over every dimension but the last; `a` is viewed as
+ * [rows, cols] with cols = its last extent, `out` has the same rank with all
+ * leading extents 1.  "all_*": reduce over every element; `out` holds one element (rank 0 or [1]).
+ * Sums accumulate in binary64 in index order and round once; max / min
+ * propagate NaN.  Float dtypes only.
+ */
+static int reduce_kind(const char *op, const char *prefix) {
+    size_t n = strlen(prefix);
+    if (strncmp(op, prefix, n) != 0) return -1;
+    return strcmp(op + n, "sum") == 0 ? 0 : strcmp(op + n, "max") == 0 ? 1 : strcmp(op + n, "min") == 0 ? 2 : -1;
+}
+
+int orc_col_reduce(const char *op, const orc_array *a, orc_array *out) {
+    int kind = reduce_kind(op, "col_");
+    if (kind < 0) return ORC_ERR_OP;
+    if (!is_float(a->dtype) || a->dtype != out->dtype) return ORC_ERR_DTYPE;
+    if (a->rank < 1 || out->rank != a->rank || out->shape[a->rank - 1] != a->shape[a->rank - 1]) return ORC_ERR_SHAPE;
+    for (int d = 0; d + 1 < a->rank; ++d)
+        if (out->shape[d] != 1) return ORC_ERR_SHAPE;
+    int64_t cols = a->shape[a->rank - 1];
+    int64_t rows = cols ? numel(a) / cols : 0;
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+    for (int64_t c = 0; c < cols; ++c) {
+        float res;
+        if (kind == 0) {
+            double acc = 0.0;
+            for (int64_t r = 0; r < rows; ++r) acc += (double)load_f(a, r * cols + c);
+            res = (float)acc;
+        } else {
+            res = kind == 1 ? -INFINITY : INFINITY;
+            for (int64_t r = 0; r < rows; ++r) {
+                float x = load_f(a, r * cols + c);
+                res = kind == 1 ? max_nan(res, x) : min_nan(res, x);
+            }
+        }
+        store_f(out, c, res);
+    }
+    return ORC_OK;
+}
+
+int orc_all_reduce(const char *op, const orc_array *a, orc_array *out) {
+    int kind = reduce_kind(op, "all_");
+    if (kind < 0) return ORC_ERR_OP;
+    if (!is_float(a->dtype) || a->dtype != out->dtype) return ORC_ERR_DTYPE;
+    if (out->rank > 1 || numel(out) != 1) return ORC_ERR_SHAPE;
+    int64_t n = numel(a);
+    float res;
+    if (kind == 0) {
+        double acc = 0.0;
+        for (int64_t i = 0; i < n; ++i) acc += (double)load_f(a, i);
+        res = (float)acc;
+    } else {
+        res = kind == 1 ? -INFINITY : INFINITY;
+        for (int64_t i = 0; i < n; ++i) {
+            float x = load_f(a, i);
+            res = kind == 1 ? max_nan(res, x) : min_nan(res, x);
+        }
+    }
+    store_f(out, 0, res);
+    return ORC_OK;
+}
+
 /* ---------------------------------------------------------------- Philox */
 
 /*

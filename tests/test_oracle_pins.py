@@ -349,6 +349,48 @@ def test_row_max_min(B):
     np.testing.assert_array_equal(B.op("row_max", leaf(B, f32(-np.inf, -np.inf).reshape(1, 2))).array, [[-np.inf]])
 
 
+def test_col_and_all_reductions(B):
+    g = rng.generator(12)
+    x = rng.normal_f32(g, (23, 5, 31), 50.0)
+    flat = x.reshape(-1, 31)
+    got = B.op("col_sum", leaf(B, x)).array
+    assert got.shape == (1, 1, 31)
+    for c in range(31):
+        exact = math.fsum(float(v) for v in flat[:, c])  # correctly rounded double sum
+        assert abs(float(got[0, 0, c]) - exact) <= abs(exact) * 2**-24 + 1e-30
+    np.testing.assert_array_equal(B.op("col_max", leaf(B, x)).array.reshape(-1), flat.max(axis=0))
+    np.testing.assert_array_equal(B.op("col_min", leaf(B, x)).array.reshape(-1), flat.min(axis=0))
+    # which axis: a matrix whose rows and columns sum differently
+    m = f32(1, 2, 3, 10, 20, 30).reshape(2, 3)
+    np.testing.assert_array_equal(B.op("col_sum", leaf(B, m)).array, f32(11, 22, 33).reshape(1, 3))
+    np.testing.assert_array_equal(B.op("row_sum", leaf(B, m)).array, f32(6, 60).reshape(2, 1))
+    np.testing.assert_array_equal(B.op("col_max", leaf(B, f32(1, 9, 7, 2).reshape(2, 2))).array, f32(7, 9).reshape(1, 2))
+    # whole-tensor reductions
+    s = B.op("all_sum", leaf(B, x)).array
+    assert s.shape == ()
+    exact = math.fsum(float(v) for v in x.reshape(-1))
+    assert abs(float(s) - exact) <= abs(exact) * 2**-24 + 1e-30
+    assert float(B.op("all_max", leaf(B, x)).array) == x.max() and float(B.op("all_min", leaf(B, x)).array) == x.min()
+    assert float(B.op("all_sum", leaf(B, m)).array) == 66.0
+    # cancellation a binary32 accumulator would lose; NaN propagation; bf16 results round once
+    col = np.array([[2.0**25]] + [[1.0]] * 16 + [[-(2.0**25)]], dtype=F32)
+    assert B.op("col_sum", leaf(B, col)).array[0, 0] == 16.0 and float(B.op("all_sum", leaf(B, col)).array) == 16.0
+    n = f32(1, float("nan"), 3, 4).reshape(2, 2)
+    assert np.isnan(B.op("col_max", leaf(B, n)).array[0, 1]) and B.op("col_max", leaf(B, n)).array[0, 0] == 3.0
+    assert np.isnan(float(B.op("all_min", leaf(B, n)).array))
+    xb = rng.to_bf16_bits(rng.normal_f32(g, (64, 9), 1.0))
+    want = rng.to_bf16_bits(rng.bf16_bits_to_f32(xb).astype(np.float64).sum(axis=0).astype(F32))
+    np.testing.assert_array_equal(B.op("col_sum", OTensor(xb, "bf16")).array.reshape(-1), want)
+
+
+def test_outer_broadcast_matches_numpy(B):
+    g = rng.generator(13)
+    r, c = rng.normal_f32(g, (7, 1)), rng.normal_f32(g, (1, 5))
+    np.testing.assert_array_equal(B.op("mul", leaf(B, r), leaf(B, c)).array, r * c)
+    np.testing.assert_array_equal(B.op("sub", leaf(B, c), leaf(B, r)).array, c - r)
+    np.testing.assert_array_equal(B.op("sub", leaf(B, r), leaf(B, rng.normal_f32(rng.generator(14), (5,)))).array.shape, (7, 5))
+
+
 # ---------------------------------------------------------------------- GELU
 
 def test_gelu_closed_forms(B):
