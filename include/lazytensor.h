@@ -69,7 +69,8 @@ typedef enum { LT_F32 = 0, LT_BF16 = 1, LT_U8 = 2, LT_I32 = 3, LT_U32 = 4 } lt_d
  * kernels implement): an operand either has the result's shape, or is rank 0, or
  * has every dimension 1 except a last dimension equal to the result's ("column
  * vector", e.g. [C] or [1,C]), or equals the result's shape except for a last
- * dimension of 1 ("row scalar", e.g. [R,1]).  Anything else is LT_ERR_SHAPE.
+ * dimension of 1 ("row scalar", e.g. [R,1]).  The operands need not include one of the result's shape:
+ * [R,1] with [1,C] gives [R,C] (an outer product when the op is MUL).  Anything else is LT_ERR_SHAPE.
  * Operands share one dtype; a rank-0 scalar adopts the dtype of the tensor it meets.
  */
 typedef enum {
@@ -95,8 +96,13 @@ typedef enum {
        (lo32(i/4), hi32(i/4), lo32(offset), hi32(offset)) and key (lo32(seed), hi32(seed)).
        seed and offset are run-time parameters: they do not enter the graph hash. */
     LT_OP_PHILOX_BITS = 42,
-    /* reductions over the last dimension, kept with extent 1; float dtypes */
-    LT_OP_ROW_SUM = 50, LT_OP_ROW_MAX = 51, LT_OP_ROW_MIN = 52
+    /* reductions over the last dimension, kept with extent 1; float dtypes; rows of any length (rows of more
+       than 8192 elements take a kernel that walks the row in slices, see lt_barrier) */
+    LT_OP_ROW_SUM = 50, LT_OP_ROW_MAX = 51, LT_OP_ROW_MIN = 52,
+    /* reductions over every dimension but the last: [d0, .., dk, C] -> [1, .., 1, C]; float dtypes */
+    LT_OP_COL_SUM = 53, LT_OP_COL_MAX = 54, LT_OP_COL_MIN = 55,
+    /* reductions over every element -> rank 0; float dtypes */
+    LT_OP_ALL_SUM = 56, LT_OP_ALL_MAX = 57, LT_OP_ALL_MIN = 58
 } lt_opcode;
 
 /*
@@ -132,6 +138,8 @@ typedef struct {
     uint64_t ns_rebind;          /* turning roots into device-data leaves, freeing IR        */
     uint64_t launches_compiled;  /* of kernels_launched: ahead-of-time compiled programs     */
     uint64_t replays;            /* lt_replay calls that ran a plan                          */
+    uint64_t launches_reduce;    /* reductions run as kernels of their own: over columns, over a whole tensor,
+                                    over rows of more than 8192 elements outside a fused long-row kernel          */
     uint64_t allocator_calls;    /* calls of the allocator's alloc and free (or cudaMallocAsync /
                                     cudaFreeAsync); 0 over a span means every block came from and
                                     went back to the context's own pool of released blocks          */
@@ -169,6 +177,8 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * interpret),
  * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
  * line per flush and per replay; preset by the environment variable LT_LOG),
+ * "wait_limit_ms" (2000 default: how long a kernel that stages long rows through shared memory waits for one of
+ * its asynchronous copies before it gives up, see LT_ERR_DEVICE_TIMEOUT),
  * "pool_bytes" (4 GiB default: device blocks the library has released are kept, up to this total, and reused
  * by later flushes before the allocator is asked; 0 = return every block at once).
  * fusion, fast_math, horizontal and ieee are part of the cache key; the others act at launch time.
@@ -232,6 +242,10 @@ lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
 /*
  * Barrier (Section 4; mark_step / LazyTensorBarrier): materialise every live tensor that
  * has pending computation.  With `blocking` non-zero, return after the stream has drained.
+ * Row reductions over more than 8192 columns: a group whose program has a kernel instantiated at build time
+ * (softmax, LayerNorm, RMSNorm and the other listed groups) runs fused, one thread block per row walking it in
+ * slices, when its inputs are 16-byte aligned and the row is a multiple of 8 elements; any other such graph runs
+ * with each long reduction as a kernel of its own and the surrounding arithmetic as elementwise kernels.
  */
 lt_status lt_barrier(lt_ctx *ctx, int blocking);
 
@@ -341,6 +355,14 @@ lt_status lt_dump_plan(lt_ctx *ctx, char *buf, size_t cap, size_t *need);
  * Synchronises the device.
  */
 lt_status lt_debug_bounds_violations(lt_ctx *ctx, uint64_t *out);
+
+/*
+ * Exercises the one device-side wait the library has, without touching any tensor: enqueues a one-warp kernel
+ * that waits at most `limit_ns` nanoseconds for a completion nothing delivers, gives up and raises the device
+ * status word.  The next blocking call on the context (lt_barrier with blocking set, lt_fetch) then returns
+ * LT_ERR_DEVICE_TIMEOUT and clears the word; the context stays usable.
+ */
+lt_status lt_debug_wait_probe(lt_ctx *ctx, uint64_t limit_ns);
 
 const char *lt_last_error(lt_ctx *ctx);
 const char *lt_version(void);

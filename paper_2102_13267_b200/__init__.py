@@ -37,6 +37,7 @@ OPCODES = {
     "neg": 20, "abs": 21, "relu": 22, "exp": 23, "log": 24, "tanh": 25, "sqrt": 26, "rsqrt": 27,
     "recip": 28, "square": 29, "sigmoid": 30, "gelu_tanh": 31, "not": 32,
     "convert": 40, "iota": 41, "philox_bits": 42, "row_sum": 50, "row_max": 51, "row_min": 52,
+    "col_sum": 53, "col_max": 54, "col_min": 55, "all_sum": 56, "all_max": 57, "all_min": 58,
 }
 STATUS_NAMES = ["LT_OK", "LT_ERR_INVALID_ARG", "LT_ERR_SHAPE", "LT_ERR_DTYPE", "LT_ERR_DEVICE",
                 "LT_ERR_UNSUPPORTED", "LT_ERR_OOM", "LT_ERR_CUDA", "LT_ERR_DEVICE_TIMEOUT"]
@@ -55,7 +56,7 @@ class lt_stats(ctypes.Structure):
         "launches_elementwise", "launches_row", "launches_multi", "bytes_planned",
         "outputs_donated", "outputs_allocated", "temporaries_allocated",
         "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind",
-        "launches_compiled", "replays", "allocator_calls")]
+        "launches_compiled", "replays", "launches_reduce", "allocator_calls")]
 
 
 class lt_kernel_timing(ctypes.Structure):
@@ -80,6 +81,7 @@ _SIGNATURES = {
     "lt_barrier": [_vp, _int],
     "lt_barrier_static_scratch": [_vp, _int, _int],
     "lt_debug_bounds_violations": [_vp, _P(_u64)],
+    "lt_debug_wait_probe": [_vp, _u64],
     "lt_replay": [_vp, _int],
     "lt_scalar_set": [_vp, _u64, ctypes.c_double],
     "lt_replay_slots": [_vp, _P(ctypes.c_uint32)],
@@ -360,6 +362,10 @@ class LazyContext:
             return None
         self._check(st)
         return n.value
+
+    def debug_wait_probe(self, limit_ns: int) -> None:
+        """lt_debug_wait_probe: enqueue a kernel whose bounded wait runs out (see LT_ERR_DEVICE_TIMEOUT)."""
+        self._check(_lib.lt_debug_wait_probe(self._ctx, int(limit_ns)))
 
     def replay(self, blocking: bool = False) -> None:
         """lt_replay: run the previously flushed graph again on the same tensors, without recording it."""

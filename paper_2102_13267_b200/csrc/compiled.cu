@@ -27,6 +27,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "compiled.h"
 #include "pdl.cuh"
 #include "vm.h"
@@ -79,6 +81,32 @@ struct Info {
             if (PG::ins[k].op == OP_PHILOX) return true;
         return false;
     }
+    static constexpr __host__ __device__ bool is_red(uint32_t op) { return op >= OP_RED_SUM && op <= OP_RED_MIN; }
+    // row reductions of the program: how many, how many before instruction i, and the kind (0 sum, 1 max, 2 min) of the r-th
+    static constexpr __host__ __device__ int red_ordinal(int i) {
+        int n = 0;
+        for (int k = PG::n_pro; k < i; ++k)
+            if (is_red(PG::ins[k].op)) ++n;
+        return n;
+    }
+    static constexpr __host__ __device__ int n_reds() { return red_ordinal(PG::n_ins); }
+    static constexpr __host__ __device__ int red_kind(int r) {
+        int n = 0;
+        for (int k = PG::n_pro; k < PG::n_ins; ++k)
+            if (is_red(PG::ins[k].op)) {
+                if (n == r) return (int)(PG::ins[k].op - OP_RED_SUM);
+                ++n;
+            }
+        return 0;
+    }
+    // is slot s a full-class input (read by a load or a memory operand of the per-chunk program)?
+    static constexpr __host__ __device__ bool full_input(int s) {
+        if (PG::cls[s] != LT_CLS_FULL) return false;
+        for (int k = PG::n_pro; k < PG::n_ins; ++k)
+            if ((is_ld(PG::ins[k].op) || is_f2m(PG::ins[k].op)) && (int)PG::ins[k].imm == s) return true;
+        return false;
+    }
+    static constexpr __host__ __device__ int elem_bytes(int s) { return PG::dtype[s] == LT_ST_BF16 ? 2 : PG::dtype[s] == LT_ST_U8 ? 1 : 4; }
     static constexpr __host__ __device__ int n_reserved() {
         int n = 0;
         for (int t = 0; t < LT_VM_NT; ++t) n += pro_slot(t) >= 0 ? 1 : 0;
@@ -661,6 +689,77 @@ struct Machine {
             run<K + 1>();
         }
     }
+
+    // Long rows (see lt_c_longrow): the program is run once per reduction plus once more.  In pass PHASE every
+    // reduction before the PHASE-th yields its known result (red.val), the PHASE-th folds this thread's lanes into
+    // red.part and ends the pass, and stores happen only in the last pass (the compiler drops whatever a pass
+    // computes without using it).
+    template <int PHASE, int K = PG::n_pro>
+    __device__ __forceinline__ void run_phase() {
+        if constexpr (K < PG::n_ins) {
+            constexpr uint32_t op = PG::ins[K].op;
+            if constexpr (I::is_red(op)) {
+                constexpr int ord = I::red_ordinal(K);
+                if constexpr (ord < PHASE) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int i = 0; i < V; ++i) acc[u][i] = red.val[ord];
+                    run_phase<PHASE, K + 1>();
+                } else {
+                    constexpr int KIND = op - OP_RED_SUM;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const float l0 = GroupReduce::red_comb<KIND>(acc[u][0], acc[u][1]), l1 = GroupReduce::red_comb<KIND>(acc[u][2], acc[u][3]);
+                        const float l2 = GroupReduce::red_comb<KIND>(acc[u][4], acc[u][5]), l3 = GroupReduce::red_comb<KIND>(acc[u][6], acc[u][7]);
+                        const float c = GroupReduce::red_comb<KIND>(GroupReduce::red_comb<KIND>(l0, l1), GroupReduce::red_comb<KIND>(l2, l3));
+                        if (!GUARD || ck.ok[u]) red.part = GroupReduce::red_comb<KIND>(red.part, c);
+                    }
+                }
+            } else if constexpr (op == OP_ST && PHASE < I::n_reds()) {
+                run_phase<PHASE, K + 1>();
+            } else {
+                step<K>();
+                run_phase<PHASE, K + 1>();
+            }
+        }
+    }
+
+    // storage-format chunks of the full-class inputs from a row staged in shared memory; soff[s] is the byte
+    // offset of slot s's row inside the stage
+    template <int K = PG::n_pro>
+    __device__ __forceinline__ void fetch_row(const unsigned char *stage, const uint32_t (&soff)[PG::n_slots]) {
+        if constexpr (K < PG::n_ins) {
+            constexpr uint32_t op = PG::ins[K].op;
+            if constexpr (I::is_ld(op) || I::is_f2m(op)) {
+                constexpr int slot = PG::ins[K].imm;
+                if constexpr (PG::cls[slot] == LT_CLS_FULL) {
+                    constexpr int cb = I::chunk_bytes(slot), sh = esz_shift(PG::dtype[slot]);
+                    constexpr int ord = I::load_ordinal(K);
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (GUARD && !ck.ok[u]) continue;
+                        const unsigned char *b = stage + soff[slot] + ((size_t)ck.col0[u] << sh);
+                        if constexpr (cb == 8) {
+                            const uint2 w = *reinterpret_cast<const uint2 *>(b);
+                            raw[ord][u].a.x = w.x;
+                            raw[ord][u].a.y = w.y;
+                        } else {
+                            raw[ord][u].a = *reinterpret_cast<const uint4 *>(b);
+                            if constexpr (cb == 32) raw[ord][u].b = *reinterpret_cast<const uint4 *>(b + 16);
+                        }
+                    }
+                }
+            }
+            fetch_row<K + 1>(stage, soff);
+        }
+    }
+};
+
+// State of the reductions of a long row: results so far, and this thread's share of the one being formed.
+struct LongRed {
+    float val[4];
+    float part;
 };
 
 struct ScalK {
@@ -864,6 +963,201 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_multi(const __grid_constant__ 
     }
 }
 
+
+// ------------------------------------------------------------------ long rows
+// A word the host reads after a blocking call: bit 0 = a bounded wait for an asynchronous copy gave up.
+__device__ unsigned int lt_device_status = 0;
+
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Waits until the phase of the mbarrier at shared address `bar` with parity `parity` has completed, for at most
+// `limit_ns` nanoseconds.  Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (global_ns() - t0 > limit_ns) return false;
+    }
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One-dimensional bulk asynchronous copy global -> this CTA's shared memory (no multicast); both addresses and the
+// size are multiples of 16 bytes.  Completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+                 "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+constexpr int C_LONG_THREADS = 256;
+constexpr int C_LONG_U = 2;
+constexpr uint32_t C_LONG_MAX_BULK = 1u << 19;  // keeps a stage's byte count inside the mbarrier's transaction counter
+
+// compile-time walks over the slots of a program (the program tables are not addressable at run time in device code)
+template <class PG, int S = 0>
+__device__ __forceinline__ void long_offsets(uint32_t cols, uint32_t (&soff)[PG::n_slots], uint32_t off) {
+    if constexpr (S < PG::n_slots) {
+        soff[S] = off;
+        if constexpr (Info<PG>::full_input(S)) off += (cols * Info<PG>::elem_bytes(S) + 15u) & ~15u;
+        long_offsets<PG, S + 1>(cols, soff, off);
+    }
+}
+template <class PG, int S = 0>
+__device__ __forceinline__ uint32_t long_row_bytes(uint32_t cols) {
+    if constexpr (S < PG::n_slots) {
+        uint32_t here = 0;
+        if constexpr (Info<PG>::full_input(S)) here = cols * Info<PG>::elem_bytes(S);
+        return here + long_row_bytes<PG, S + 1>(cols);
+    } else {
+        return 0u;
+    }
+}
+template <class PG, int S = 0, class Ptr>
+__device__ __forceinline__ void long_issue(const Ptr &ptr, uint32_t cols, uint32_t row, uint32_t stage, const uint32_t (&soff)[PG::n_slots],
+                                           uint32_t bar) {
+    if constexpr (S < PG::n_slots) {
+        if constexpr (Info<PG>::full_input(S)) {
+            const uint32_t bytes = cols * Info<PG>::elem_bytes(S);
+            const char *src = reinterpret_cast<const char *>(ptr(S)) + (uint64_t)row * bytes;
+            for (uint32_t done = 0; done < bytes; done += C_LONG_MAX_BULK) {
+                const uint32_t n = bytes - done < C_LONG_MAX_BULK ? bytes - done : C_LONG_MAX_BULK;
+                bulk_copy_g2s(stage + soff[S] + done, src + done, n, bar);
+            }
+        }
+        long_issue<PG, S + 1>(ptr, cols, row, stage, soff, bar);
+    }
+}
+
+template <int KIND>
+__device__ __forceinline__ float long_cta_reduce(float v, float *buf) {
+#pragma unroll
+    for (uint32_t off = 16; off > 0; off >>= 1) v = GroupReduce::red_comb<KIND>(v, __shfl_xor_sync(0xffffffffu, v, off));
+    __syncthreads();  // buf may still be read from the previous reduction
+    if ((threadIdx.x & 31u) == 0) buf[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = buf[0];
+#pragma unroll
+    for (int w = 1; w < C_LONG_THREADS / 32; ++w) r = GroupReduce::red_comb<KIND>(r, buf[w]);
+    return r;
+}
+
+// Rows too long for a thread group's registers: a CTA owns a row and walks it in slices of 256 x 2 chunks.  A program
+// with n reductions makes n + 1 passes over the row (Machine::run_phase).  With `depth` > 0 the row's full-class
+// inputs are brought into shared memory once, by one-dimensional bulk asynchronous copies that complete on an
+// mbarrier, `depth` rows ahead; every pass then reads the staged row.  With depth 0 the passes read global memory
+// (the row was just read by this CTA and sits in L2).  The wait for a stage is bounded: when it gives up the CTA
+// raises bit 0 of lt_device_status, waits (again bounded) for the copies it still has in flight and returns.
+template <class PG>
+__global__ void __launch_bounds__(C_LONG_THREADS) lt_c_longrow(const __grid_constant__ LtKParams P, uint32_t depth, uint32_t stage_bytes,
+                                                               uint64_t limit_ns) {
+    constexpr int U = C_LONG_U, T = C_LONG_THREADS, NR = Info<PG>::n_reds();
+    static_assert(NR <= 4, "at most four reductions per long-row program");
+    using M = Machine<PG, U, PtrK, ScalK, LongRed, true>;
+    __shared__ float red_buf[T / 32];
+    __shared__ __align__(8) uint64_t bars[2];
+    extern __shared__ __align__(128) unsigned char stage_mem[];
+    const PtrK ptr{P};
+    const ScalK scal{P};
+    LongRed red;
+    const uint32_t cpr = P.cpr, n_slices = (cpr + T * U - 1) / (T * U);
+    // byte offset of every staged slot's row inside a stage
+    uint32_t soff[PG::n_slots];
+    long_offsets<PG>(P.cols, soff, 0u);
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&bars[0]);
+    const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(stage_mem);
+    if (depth && threadIdx.x == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    pdl_release();
+    pdl_wait();
+    __syncthreads();
+    auto issue = [&](uint32_t row, uint32_t s) {  // thread 0: start the copies of `row` into stage s
+        mbar_expect_tx(bar0 + 8 * s, long_row_bytes<PG>(P.cols));
+        long_issue<PG>(ptr, P.cols, row, stage0 + s * stage_bytes, soff, bar0 + 8 * s);
+    };
+    if (depth && threadIdx.x == 0) {
+        uint32_t row = blockIdx.x;
+        for (uint32_t d = 0; d < depth; ++d, row += gridDim.x)
+            if (row < P.rows) issue(row, d);
+    }
+    uint32_t k = 0;
+    for (uint32_t row = blockIdx.x; row < P.rows; row += gridDim.x, ++k) {
+        const uint32_t s = depth ? k % depth : 0u;
+        const unsigned char *stage = stage_mem + (size_t)s * stage_bytes;
+        if (depth) {
+            const bool landed = mbar_wait_bounded(bar0 + 8 * s, (k / depth) & 1u, limit_ns);
+            if (__syncthreads_or(landed ? 0 : 1)) {
+                if (threadIdx.x == 0) atomicOr(&lt_device_status, 1u);
+                // copies this CTA still has in flight write into its shared memory: give them the same time once more
+                for (uint32_t d = 0; d < depth; ++d) mbar_wait_bounded(bar0 + 8 * d, ((k + (d >= s ? 0u : 1u)) / depth) & 1u, limit_ns);
+                return;
+            }
+        }
+        auto pass = [&](auto phase_tag) {
+            constexpr int PHASE = decltype(phase_tag)::value;
+            if constexpr (PHASE < NR) red.part = Info<PG>::red_kind(PHASE) == 0 ? 0.0f : (Info<PG>::red_kind(PHASE) == 1 ? -INFINITY : INFINITY);
+            for (uint32_t sl = 0; sl < n_slices; ++sl) {
+                Coords<U> ck;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t chunk = (sl * U + u) * T + threadIdx.x;
+                    ck.ok[u] = chunk < cpr;
+                    ck.row[u] = row;
+                    ck.col0[u] = ck.ok[u] ? chunk * V : 0u;  // a chunk past the end takes the coordinates of the first
+                    ck.flat0[u] = (uint64_t)row * P.cols + ck.col0[u];
+                }
+                M m(ptr, scal, red, ck);
+                if (depth) m.fetch_row(stage, soff);
+                else m.issue_loads();
+                m.template run_phase<PHASE>();
+            }
+            if constexpr (PHASE < NR) red.val[PHASE] = long_cta_reduce<Info<PG>::red_kind(PHASE)>(red.part, red_buf);
+        };
+        pass(std::integral_constant<int, 0>{});
+        if constexpr (NR >= 1) pass(std::integral_constant<int, 1>{});
+        if constexpr (NR >= 2) pass(std::integral_constant<int, 2>{});
+        if constexpr (NR >= 3) pass(std::integral_constant<int, 3>{});
+        if constexpr (NR >= 4) pass(std::integral_constant<int, 4>{});
+        if (depth) {
+            __syncthreads();  // every thread has finished reading stage s
+            const uint32_t next = row + depth * gridDim.x;
+            if (threadIdx.x == 0 && next < P.rows) issue(next, s);
+        }
+    }
+}
+
+// A kernel that waits, bounded, for an mbarrier phase nothing completes: exercises the give-up path of
+// mbar_wait_bounded and the status word without any copy in flight.
+__global__ void lt_wait_probe(uint64_t limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (!mbar_wait_bounded(b, 0, limit_ns) && threadIdx.x == 0) atomicOr(&lt_device_status, 1u);
+}
+
 // ------------------------------------------------------------------ table
 #include "compiled_programs.inc"
 
@@ -944,6 +1238,100 @@ int lt_compiled_find(int kind, int flavour, const LtIns *ins, uint32_t n_ins, ui
     LT_COMPILED_LIST(LT_X)
 #undef LT_X
     return -1;
+}
+
+namespace {
+
+template <class PG, int S = 0>
+size_t long_stage_bytes(uint32_t cols) {
+    if constexpr (S < PG::n_slots) {
+        constexpr bool in = Info<PG>::full_input(S);
+        constexpr int eb = Info<PG>::elem_bytes(S);
+        return (in ? (((size_t)cols * eb + 15u) & ~(size_t)15u) : 0) + long_stage_bytes<PG, S + 1>(cols);
+    } else {
+        return 0;
+    }
+}
+
+template <class PG, int S = 0>
+bool long_stage_allowed(uint32_t cols) {  // every staged row a multiple of 16 bytes
+    if constexpr (S < PG::n_slots) {
+        constexpr bool in = Info<PG>::full_input(S);
+        constexpr int eb = Info<PG>::elem_bytes(S);
+        return !(in && ((size_t)cols * eb) % 16u) && long_stage_allowed<PG, S + 1>(cols);
+    } else {
+        return true;
+    }
+}
+
+template <class PG>
+cudaError_t launch_long(const LtKParams &P, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns, cudaStream_t stream) {
+    if constexpr (PG::kind == 1 && Info<PG>::n_reds() <= 4) {
+        const size_t dyn = (size_t)depth * stage_bytes;
+        cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG>, dyn);
+        if (e != cudaSuccess) return e;
+        return launch_pdl(lt_c_longrow<PG>, grid, C_LONG_THREADS, dyn, stream, P, (uint32_t)depth, (uint32_t)stage_bytes, limit_ns);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+}
+
+template <class PG>
+cudaError_t long_occupancy(size_t dyn, int *blocks) {
+    if constexpr (PG::kind == 1 && Info<PG>::n_reds() <= 4) {
+        cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG>, dyn);
+        if (e != cudaSuccess) return e;
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_longrow<PG>, C_LONG_THREADS, dyn);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+size_t lt_compiled_long_stage_bytes(int id, uint32_t cols) {
+    int k = 0;
+#define LT_X(PG)                                                                  \
+    if (k == id) return long_stage_allowed<PG>(cols) ? long_stage_bytes<PG>(cols) : 0; \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return 0;
+}
+
+cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns,
+                                    cudaStream_t stream) {
+    int k = 0;
+#define LT_X(PG)                                                                                                              \
+    if (k == id) return launch_long<PG>(*static_cast<const LtKParams *>(params), grid, depth, stage_bytes, limit_ns, stream); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t lt_compiled_long_occupancy(int id, size_t dyn_smem, int *blocks) {
+    int k = 0;
+#define LT_X(PG)                                        \
+    if (k == id) return long_occupancy<PG>(dyn_smem, blocks); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t lt_device_status_read(unsigned int *out, int clear) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, lt_device_status, sizeof(*out));
+    if (e == cudaSuccess && clear && *out) {
+        const unsigned int zero = 0;
+        e = cudaMemcpyToSymbol(lt_device_status, &zero, sizeof(zero));
+    }
+    return e;
+}
+
+cudaError_t lt_wait_probe_launch(uint64_t limit_ns, cudaStream_t stream) {
+    lt_wait_probe<<<1, 32, 0, stream>>>(limit_ns);
+    return cudaGetLastError();
 }
 
 int lt_compiled_bounds_violations(unsigned long long *out) {

@@ -25,3 +25,17 @@ int lt_compiled_prefers_staging(int id);
 // Accesses the compiled shells found outside their slots since the library was loaded (debug build with
 // -DLT_DEBUG_BOUNDS only): 0 = *out is valid, 1 = not a debug build, -1 = the read failed.  Synchronises the device.
 int lt_compiled_bounds_violations(unsigned long long *out);
+
+// Long rows (more columns than a row's thread group keeps in registers): a CTA walks the row in slices, one pass
+// per reduction plus one.  lt_compiled_long_stage_bytes: shared memory one staged row of the entry's full-class
+// inputs takes at `cols` columns, 0 when they cannot be staged (a row that is not a multiple of 16 bytes).
+// `depth` 0 = passes read global memory, 1 or 2 = rows staged that far ahead by bulk asynchronous copies whose
+// completion the kernel awaits for at most `limit_ns` nanoseconds.
+size_t lt_compiled_long_stage_bytes(int id, uint32_t cols);
+cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns,
+                                    cudaStream_t stream);
+cudaError_t lt_compiled_long_occupancy(int id, size_t dyn_smem, int *blocks);
+// Device status word (bit 0: a bounded wait gave up); synchronises the device.  `clear` resets it when set.
+cudaError_t lt_device_status_read(unsigned int *out, int clear);
+// Launches a one-warp kernel that waits `limit_ns` for an mbarrier phase nothing completes and then raises bit 0.
+cudaError_t lt_wait_probe_launch(uint64_t limit_ns, cudaStream_t stream);

@@ -118,9 +118,10 @@ void release_donors(lt_ctx *c, const std::vector<uint32_t> &roots) {
 
 // Remembers, for lt_replay, which tensors the graph being flushed reads and writes.  Called after the
 // launches, while the root tensors still name their IR and their lt_assign donors.
-void record_replay(lt_ctx *c, Plan *plan, const Canonical &cg, const std::vector<uint32_t> &roots) {
+void record_replay(lt_ctx *c, Plan *cached, Plan *plan, const Canonical &cg, const std::vector<uint32_t> &roots) {
     ReplayRecord &r = c->replay;
-    r.plan = plan;
+    r.plan = cached;
+    r.exec = plan;
     r.why_not.clear();
     r.dyn = cg.dyn;
     r.params.assign(cg.param_node.size(), ReplayRecord::ParamRef());
@@ -167,6 +168,22 @@ void record_replay(lt_ctx *c, Plan *plan, const Canonical &cg, const std::vector
         if (p >= 0 && r.params[p].slot == root.slot) r.in_place_ok[root.output] = 1;
     }
     by_node.clear();
+}
+
+// Drains the stream; afterwards, if a kernel with bounded device-side waits has run since the last look, reads the
+// device status word: a wait that gave up is reported (and the word cleared) here.
+lt_status sync_and_check(lt_ctx *c) {
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
+    if (c->status_pending) {
+        c->status_pending = false;
+        unsigned int word = 0;
+        e = lt_device_status_read(&word, 1);
+        if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("reading the device status word: ") + cudaGetErrorString(e));
+        if (word & 1u)
+            return fail(c, LT_ERR_DEVICE_TIMEOUT, "a kernel gave up waiting for an asynchronous copy into shared memory; results of that flush are incomplete");
+    }
+    return LT_OK;
 }
 
 void put_text(const std::string &s, char *buf, size_t cap, size_t *need) {
@@ -216,6 +233,8 @@ const char *op_name(int op) {
     case LT_OP_CONVERT: return "convert"; case LT_OP_IOTA: return "iota";
     case LT_OP_PHILOX_BITS: return "philox_bits";
     case LT_OP_ROW_SUM: return "row_sum"; case LT_OP_ROW_MAX: return "row_max"; case LT_OP_ROW_MIN: return "row_min";
+    case LT_OP_COL_SUM: return "col_sum"; case LT_OP_COL_MAX: return "col_max"; case LT_OP_COL_MIN: return "col_min";
+    case LT_OP_ALL_SUM: return "all_sum"; case LT_OP_ALL_MAX: return "all_max"; case LT_OP_ALL_MIN: return "all_min";
     case N_DEVICE_DATA: return "device_data"; case N_SCALAR: return "constant";
     default: return "?";
     }
@@ -454,6 +473,7 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "debug.compiled_u")) c->opt.compiled_u = value;
     else if (!strcmp(key, "debug.compiled_row_u")) c->opt.compiled_row_u = value;
     else if (!strcmp(key, "debug.compiled_depth")) c->opt.compiled_depth = value;
+    else if (!strcmp(key, "wait_limit_ms")) c->wait_limit_ns = value > 0 ? value * 1000000ll : 1;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
 }
@@ -630,6 +650,8 @@ lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int6
     const bool is_compare = opcode >= LT_OP_GT && opcode <= LT_OP_NE;
     const bool is_unary = opcode >= LT_OP_NEG && opcode <= LT_OP_NOT;
     const bool is_reduce = opcode >= LT_OP_ROW_SUM && opcode <= LT_OP_ROW_MIN;
+    const bool is_col_reduce = opcode >= LT_OP_COL_SUM && opcode <= LT_OP_COL_MIN;
+    const bool is_all_reduce = opcode >= LT_OP_ALL_SUM && opcode <= LT_OP_ALL_MIN;
 
     if (is_binary || is_compare) {
         if (n_in != 2) return fail(c, LT_ERR_INVALID_ARG, "binary op takes 2 inputs");
@@ -702,11 +724,22 @@ lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int6
         if (n_in != 1) return fail(c, LT_ERR_INVALID_ARG, "reduction takes 1 input");
         if (!float_dtype(ops[0]->dtype)) return fail(c, LT_ERR_DTYPE, "row reductions need a float dtype");
         if (ops[0]->rank < 1) return fail(c, LT_ERR_SHAPE, "row reduction needs rank >= 1");
-        if (ops[0]->dims[ops[0]->rank - 1] > (int64_t)LT_VM_V * 1024)
-            return fail(c, LT_ERR_UNSUPPORTED, "row reductions support rows of at most 8192 elements");
         orank = ops[0]->rank;
         memcpy(od, ops[0]->dims, sizeof(od));
         od[orank - 1] = 1;
+        odtype = ops[0]->dtype;
+    } else if (is_col_reduce || is_all_reduce) {
+        if (n_in != 1) return fail(c, LT_ERR_INVALID_ARG, "reduction takes 1 input");
+        if (ops[0]->op == N_SCALAR) return fail(c, LT_ERR_INVALID_ARG, "reduction of a constant");
+        if (!float_dtype(ops[0]->dtype)) return fail(c, LT_ERR_DTYPE, "reductions need a float dtype");
+        if (is_col_reduce) {
+            if (ops[0]->rank < 1) return fail(c, LT_ERR_SHAPE, "column reduction needs rank >= 1");
+            orank = ops[0]->rank;
+            for (int i = 0; i + 1 < orank; ++i) od[i] = 1;
+            od[orank - 1] = ops[0]->dims[orank - 1];
+        } else {
+            orank = 0;
+        }
         odtype = ops[0]->dtype;
     } else {
         return fail(c, LT_ERR_UNSUPPORTED, "unknown opcode " + std::to_string(opcode));
@@ -808,8 +841,8 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
     if (roots.empty()) {
         gather_roots(c, roots, true);
         if (blocking && c->device != LT_DEVICE_NONE) {
-            cudaError_t e = cudaStreamSynchronize(c->stream);
-            if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
+            lt_status st = sync_and_check(c);
+            if (st) return st;
         }
         return LT_OK;
     }
@@ -827,7 +860,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
                 (p->canon_bytes.size() == cg.bytes.size() && !memcmp(p->canon_bytes.data(), cg.bytes.data(), cg.bytes.size())))
                 plan = p;
             else {
-                if (c->replay.plan == p) c->replay.plan = nullptr;
+                if (c->replay.plan == p) c->replay.plan = c->replay.exec = nullptr;
                 c->cache.erase(it);  // a colliding entry: replace it below
             }
         }
@@ -851,7 +884,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
                 c->last_plan_text = describe_plan(*c->last_plan);
                 c->last_plan = nullptr;
             }
-            if (c->replay.plan == victim->second.get()) c->replay.plan = nullptr;
+            if (c->replay.plan == victim->second.get()) c->replay.plan = c->replay.exec = nullptr;
             c->cache.erase(victim);
         }
         plan = np.get();
@@ -867,9 +900,10 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
                 (unsigned long long)c->stats.barriers, cg.nodes.size(), (unsigned long long)cg.hash[0], (unsigned long long)cg.hash[1],
                 was_hit ? "cache hit" : "planned", plan->launches.size(), compiled, plan->outputs.size(), plan->temp_bytes.size());
     }
+    Plan *ran = plan;  // the cached plan, or its split variant when that is what this flush needed
     {
         Timer tm(c->stats.ns_bind_launch);
-        lt_status s = execute_plan(c, *plan, cg);
+        lt_status s = run_plan(c, plan, cg, &ran);
         if (s) return s;  // nothing was rebound: the graph can be flushed again
     }
     {
@@ -878,7 +912,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
         const size_t n_out = cg.outputs.size();
         std::vector<uint32_t> new_nodes(n_out);
         for (size_t k = 0; k < n_out; ++k) {
-            const OutputPlan &op = plan->outputs[k];
+            const OutputPlan &op = ran->outputs[k];
             uint32_t n = node_new(c);
             Node &nd = c->nodes[n];
             nd.op = N_DEVICE_DATA;
@@ -896,7 +930,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
             new_nodes[k] = n;
         }
         gather_roots(c, roots, true);
-        record_replay(c, plan, cg, roots);
+        record_replay(c, plan, ran, cg, roots);
         for (uint32_t slot : roots) {
             TensorRec &t = c->tensors[slot];
             const Node &old = c->nodes[t.node];
@@ -912,10 +946,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
         release_donors(c, roots);
         for (uint32_t n : new_nodes) node_unref(c, n);
     }
-    if (blocking && c->device != LT_DEVICE_NONE) {
-        cudaError_t e = cudaStreamSynchronize(c->stream);
-        if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
-    }
+    if (blocking && c->device != LT_DEVICE_NONE) return sync_and_check(c);
     return LT_OK;
 }
 
@@ -929,7 +960,7 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
     std::vector<uint32_t> &roots = c->roots_scratch;
     gather_roots(c, roots, false);
     if (!roots.empty()) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: operations are pending; flush them with lt_barrier");
-    Plan *plan = r.plan;
+    Plan *plan = r.exec;
     auto live = [c](const ReplayRecord::Ref &ref) {
         return ref.slot < c->tensors.size() && c->tensors[ref.slot].live && c->tensors[ref.slot].gen == ref.gen;
     };
@@ -964,8 +995,8 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
             if (sn.op == N_SCALAR) r.dyn[k].d = sn.sval;
         }
     cg.dyn = r.dyn;
-    plan->last_used = ++c->use_clock;
-    c->last_plan = plan;
+    r.plan->last_used = ++c->use_clock;
+    c->last_plan = r.plan;
     {
         Timer tm(c->stats.ns_bind_launch);
         lt_status s = execute_plan(c, *plan, cg);
@@ -1008,10 +1039,7 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
     if (c->opt.log >= 2)
         fprintf(stderr, "[lazytensor] replay %llu: %zu launches, %zu run-time slots\n", (unsigned long long)c->stats.replays,
                 plan->launches.size(), r.dyn.size());
-    if (blocking && c->device != LT_DEVICE_NONE) {
-        cudaError_t e = cudaStreamSynchronize(c->stream);
-        if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("cudaStreamSynchronize: ") + cudaGetErrorString(e));
-    }
+    if (blocking && c->device != LT_DEVICE_NONE) return sync_and_check(c);
     return LT_OK;
 }
 
@@ -1057,6 +1085,16 @@ lt_status lt_debug_bounds_violations(lt_ctx *c, uint64_t *out) {
     return LT_OK;
 }
 
+lt_status lt_debug_wait_probe(lt_ctx *c, uint64_t limit_ns) {
+    if (!c) return LT_ERR_INVALID_ARG;
+    if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_DEVICE, "lt_debug_wait_probe needs a context on a CUDA device");
+    DeviceScope on_device(c->device);
+    cudaError_t e = lt_wait_probe_launch(limit_ns, c->stream);
+    if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("probe launch: ") + cudaGetErrorString(e));
+    c->status_pending = true;
+    return LT_OK;
+}
+
 lt_status lt_fetch(lt_ctx *c, lt_tensor t, void *host_dst, size_t nbytes) {
     if (!c) return LT_ERR_INVALID_ARG;
     uint32_t slot;
@@ -1086,9 +1124,8 @@ lt_status lt_fetch(lt_ctx *c, lt_tensor t, void *host_dst, size_t nbytes) {
         return LT_OK;
     }
     cudaError_t e = cudaMemcpyAsync(host_dst, c->buffers[nd.buffer].ptr, bytes, cudaMemcpyDeviceToHost, c->stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) return fail(c, LT_ERR_CUDA, std::string("device to host copy: ") + cudaGetErrorString(e));
-    return LT_OK;
+    return sync_and_check(c);
 }
 
 lt_status lt_device_ptr(lt_ctx *c, lt_tensor t, void **dptr) {

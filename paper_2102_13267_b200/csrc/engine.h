@@ -102,7 +102,7 @@ struct IoRef {
     uint32_t cnode;   // canonical node the slot carries
 };
 
-enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2 };
+enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2, K_RED = 3 };  // K_RED: a reduction that runs as a kernel of its own (reduce.cu)
 
 struct Group {
     uint8_t kind = K_EW;
@@ -115,6 +115,10 @@ struct Group {
     std::vector<IoRef> io;
     std::vector<Imm> imms;
     uint64_t bytes = 0;
+    bool long_row = false;          // K_ROW with more columns than a row's thread group keeps in registers
+    uint8_t red_axis = 0;           // K_RED: 0 rows, 1 columns, 2 everything
+    uint8_t red_kind = 0;           // K_RED: 0 sum, 1 max, 2 min
+    int32_t scratch_temp = -1;      // K_RED: temporary that holds the partial results, or -1
 };
 
 struct Launch {
@@ -145,6 +149,9 @@ struct Plan {
     std::vector<Group> groups;
     std::vector<Launch> launches;
     uint64_t last_used = 0;
+    // The same graph planned with every long row reduction as a kernel of its own: built when a fused long-row
+    // launch cannot run on the pointers at hand (alignment), and used for that flush instead.
+    std::unique_ptr<Plan> split;
 };
 
 struct Options {
@@ -168,7 +175,8 @@ struct HashKeyHasher {
 // What lt_replay needs to run the last flushed graph again without recording it: the plan, and which
 // tensors supplied its parameters and run-time scalars and received its results.
 struct ReplayRecord {
-    Plan *plan = nullptr;
+    Plan *plan = nullptr;   // the cached plan of the flushed graph (null once evicted)
+    Plan *exec = nullptr;   // what ran and runs again: `plan`, or the split variant it owns
     struct Ref {
         uint32_t slot = NONE, gen = 0;
     };
@@ -230,6 +238,8 @@ struct lt_ctx {
     size_t static_cap = 0;
 
     lt::ReplayRecord replay;
+    bool status_pending = false;      // a kernel with bounded device-side waits ran since the status word was last read
+    int64_t wait_limit_ns = 2000000000ll;  // how long such a wait may last
 
     bool timing = false;
     std::vector<lt::TimedLaunch> timed;
@@ -296,12 +306,13 @@ void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonica
 void hash_bytes(const uint8_t *data, size_t n, uint64_t out[2]);
 
 // planner (planner.cpp)
-lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan);
+lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_long_rows = false);
 std::string describe_plan(const Plan &plan);
 int broadcast_class(const int64_t *dims, int rank, uint64_t rows, uint64_t cols);
 
 // executor (executor.cpp)
-lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg);
+lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_split = nullptr);
+lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran);
 void fastdiv_make(uint32_t d, uint32_t *mul, uint32_t *sh1, uint32_t *sh2);
 
 }  // namespace lt

@@ -1,7 +1,9 @@
 // Executor: binds this trace's pointers and run-time scalars into a plan's parameter blocks
 // and launches its kernels on the context's stream.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <memory>
 #include <string>
 
 #include "compiled.h"
@@ -68,12 +70,49 @@ int compiled_blocks(Launch &L, int u, int threads, size_t dyn = 0) {
 
 }  // namespace
 
-lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
+// Runs `plan`, or -- when one of its fused long-row launches cannot run on the pointers of this flush -- the
+// same graph planned with every long row reduction as a kernel of its own.  *ran is the plan that was executed
+// (its outputs' placement is what the caller binds).
+lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran) {
+    bool needs_split = false;
+    *ran = plan;
+    lt_status s = execute_plan(c, *plan, cg, &needs_split);
+    if (!needs_split) return s;
+    if (!plan->split) {
+        std::unique_ptr<Plan> sp(new Plan());
+        s = build_plan(c, cg, *sp, true);
+        if (s) return s;
+        plan->split = std::move(sp);
+    }
+    *ran = plan->split.get();
+    return execute_plan(c, *plan->split, cg, nullptr);
+}
+
+lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_split) {
     const bool dry = c->device == LT_DEVICE_NONE;
     const size_t n_out = plan.outputs.size();
     c->param_ptr.resize(plan.n_params);
     for (uint32_t i = 0; i < plan.n_params; ++i)
         c->param_ptr[i] = c->buffers[c->nodes[cg.param_node[i]].buffer].ptr;
+    // A fused long-row launch runs only on its compiled kernel, which needs 128-bit accesses: whole chunks per row
+    // and 16-byte aligned inputs (results and temporaries come from the allocator, aligned).  Checked before
+    // anything is obtained or enqueued, so that the caller can fall back to the split plan.
+    if (!dry)
+        for (const Launch &L : plan.launches) {
+            const Group &g = plan.groups[L.groups[0]];
+            if (L.kind != K_ROW || !g.long_row) continue;
+            bool ok = c->opt.compiled && L.compiled >= 0 && (g.cols % LT_VM_V) == 0;
+            for (size_t q = 0; q < g.io.size() && ok; ++q)
+                if (g.io[q].kind == IO_PARAM && g.io[q].cls <= LT_CLS_COLVEC)
+                    ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index], g.io[q].dtype);
+            if (!ok) {
+                if (needs_split) {
+                    *needs_split = true;
+                    return LT_OK;
+                }
+                return fail(c, LT_ERR_UNSUPPORTED, "a fused reduction over rows of more than 8192 elements needs 16-byte aligned inputs and rows that are a multiple of 8 elements");
+            }
+        }
     c->out_ptr.assign(n_out, nullptr);
     c->temp_ptr.assign(plan.temp_bytes.size(), nullptr);
 
@@ -155,7 +194,19 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             ev0 = take_event(c);
             ev1 = take_event(c);
         }
-        if (L.kind == K_MULTI) {
+        if (L.kind == K_RED) {
+            const Group &g = plan.groups[L.groups[0]];
+            unsigned launched = 1;
+            if (!dry) {
+                void *scratch = g.scratch_temp >= 0 ? c->temp_ptr[g.scratch_temp] : nullptr;
+                if (ev0) cudaEventRecord(ev0, c->stream);
+                e = lt_launch_reduce(g.red_axis, g.red_kind, g.io[0].dtype, (const void *)(uintptr_t)resolve(g.io[0]),
+                                     (void *)(uintptr_t)resolve(g.io[1]), scratch, g.rows, g.cols, c->sm_count, c->stream, &launched);
+                if (ev1) cudaEventRecord(ev1, c->stream);
+            }
+            c->stats.launches_reduce += 1;
+            if (launched > 1) c->stats.kernels_launched += launched - 1;
+        } else if (L.kind == K_MULTI) {
             LtMultiParams &P = *L.mp;
             const Group &g0 = plan.groups[L.groups[0]];
             for (size_t q = 0; q < g0.imms.size(); ++q) P.scal[q] = encode_imm(g0.imms[q], cg.dyn);
@@ -231,7 +282,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
             const Group &g = plan.groups[L.groups[0]];
             for (size_t q = 0; q < g.imms.size(); ++q) P.scal[q] = encode_imm(g.imms[q], cg.dyn);
             for (size_t s = 0; s < g.io.size(); ++s) P.ptr[s] = resolve(g.io[s]);
-            {
+            if (!g.long_row) {
                 // Staging plan: aligned full-class inputs are copied asynchronously into per-thread
                 // shared-memory buffers a few chunks ahead.  Needs rows that are a multiple of the chunk
                 // (chunk c starts at element 8c) and 256-thread blocks (the buffer layout).
@@ -273,7 +324,30 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 }
             }
             bool done = false;
-            if (!dry && c->opt.compiled && L.compiled >= 0) {
+            if (g.long_row) {
+                // a CTA per row, walking it in slices; rows staged in shared memory `depth` ahead when they fit
+                // (feasibility was checked on entry)
+                if (!dry) {
+                    const size_t cap = 200u * 1024u;
+                    const size_t stage = lt_compiled_long_stage_bytes(L.compiled, P.cols);
+                    unsigned depth = stage == 0 ? 0u : (unsigned)std::min<size_t>(2, cap / stage);
+                    if (c->opt.compiled_depth >= 0) depth = std::min<unsigned>(depth, (unsigned)c->opt.compiled_depth);
+                    int occ = 1;
+                    if (lt_compiled_long_occupancy(L.compiled, depth * stage, &occ) != cudaSuccess || occ < 1) {
+                        cudaGetLastError();
+                        occ = 1;
+                    }
+                    unsigned grid = (unsigned)std::min<uint64_t>(P.rows, (uint64_t)c->sm_count * occ);
+                    if (grid < 1) grid = 1;
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    e = lt_compiled_launch_long(L.compiled, &P, grid, depth, stage, (uint64_t)c->wait_limit_ns, c->stream);
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                    if (depth) c->status_pending = true;
+                }
+                c->stats.launches_compiled++;
+                done = true;
+            }
+            if (!done && !dry && c->opt.compiled && L.compiled >= 0) {
                 // compiled kernel: needs 128-bit accesses everywhere (aligned pointers, whole chunks)
                 bool ok = (L.kind == K_EW && !P.rowcol) ? (P.n % LT_VM_V) == 0 : (P.cols % LT_VM_V) == 0;
                 ok = ok && P.n_chunks < (1ull << 31);
@@ -358,7 +432,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg) {
                 c->stats.launches_row++;
             }
         }
-        if (ev0) c->timed.push_back(TimedLaunch{ev0, ev1, L.kind, L.bytes});
+        if (ev0) c->timed.push_back(TimedLaunch{ev0, ev1, (uint8_t)(L.kind == K_RED ? K_ROW : L.kind), L.bytes});
         if (e != cudaSuccess) {
             release_all(true);
             return fail(c, LT_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e));

@@ -4,6 +4,7 @@
 #pragma once
 #include <cuda_runtime_api.h>
 #include <stddef.h>
+#include <stdint.h>
 
 #include "vm.h"
 
@@ -22,3 +23,11 @@ cudaError_t lt_kernel_occupancy(int *ew_blocks_per_sm, int *row_blocks_per_sm_25
 
 // static_scratch.cu: zero-fills `bytes` of the fixed scratch array at `base` on `stream`
 cudaError_t lt_static_scratch_clear_enqueue(void *base, size_t bytes, int sm_count, cudaStream_t stream);
+
+// reduce.cu: reductions that run as kernels of their own.  axis 0: rows of [rows, cols] -> out[rows]; 1: columns ->
+// out[cols]; 2: everything -> out[1].  kind 0 sum, 1 max, 2 min; dtype 0 f32, 1 bf16 (input and result).
+// The column and whole-tensor forms need lt_reduce_scratch_bytes of scratch memory (0 for small inputs).
+// *launched receives the number of kernels enqueued (1 or 2).
+size_t lt_reduce_scratch_bytes(int axis, uint64_t rows, uint64_t cols, int sm_count);
+cudaError_t lt_launch_reduce(int axis, int kind, int dtype, const void *in, void *out, void *scratch, uint64_t rows, uint64_t cols,
+                             int sm_count, cudaStream_t stream, unsigned *launched);

@@ -10,6 +10,7 @@
 
 #include "compiled.h"
 #include "engine.h"
+#include "launch.h"
 
 namespace lt {
 
@@ -23,12 +24,16 @@ struct PNode {
     bool leaf = false;   // device data or scalar
     bool absorbed = false;
     bool reduce = false;
+    bool foreign = false;  // runs as a kernel of its own (column / whole-tensor reduction, isolated long row reduction)
     bool needs_store = false;
     int temp = -1;       // temporary buffer index when stored but not an output
     std::vector<uint32_t> consumers;
 };
 
 inline bool is_reduce(uint16_t op) { return op >= LT_OP_ROW_SUM && op <= LT_OP_ROW_MIN; }
+inline bool is_col_reduce(uint16_t op) { return op >= LT_OP_COL_SUM && op <= LT_OP_COL_MIN; }
+inline bool is_all_reduce(uint16_t op) { return op >= LT_OP_ALL_SUM && op <= LT_OP_ALL_MIN; }
+constexpr uint64_t MAX_RESIDENT_COLS = (uint64_t)LT_VM_V * 1024;  // longest row a thread group keeps in registers
 inline bool is_factory(uint16_t op) { return op == LT_OP_IOTA || op == LT_OP_PHILOX_BITS; }
 inline bool is_float(uint8_t dt) { return dt == LT_F32 || dt == LT_BF16; }
 
@@ -696,7 +701,7 @@ int broadcast_class(const int64_t *dims, int rank, uint64_t rows, uint64_t cols)
     return class_in(c ? ne / c : 0, c, ne, rows, cols);
 }
 
-lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
+lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_long_rows) {
     const size_t N = cg.nodes.size();
     std::vector<PNode> pn(N);
     const bool fuse = c->opt.fusion != 0;
@@ -706,9 +711,14 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
         domain_of(n, &pn[i].rows, &pn[i].cols, &pn[i].numel);
         pn[i].leaf = n.op == N_DEVICE_DATA || n.op == N_SCALAR;
         pn[i].reduce = is_reduce(n.op);
+        pn[i].foreign = is_col_reduce(n.op) || is_all_reduce(n.op);
         for (int k = 0; k < n.n_in; ++k) pn[n.in[k]].consumers.push_back((uint32_t)i);
         if (pn[i].numel == 0) return fail(c, LT_ERR_UNSUPPORTED, "empty tensors cannot be part of a flushed graph");
     }
+
+    if (isolate_long_rows)
+        for (size_t i = 0; i < N; ++i)
+            if (pn[i].reduce && pn[cg.nodes[i].in[0]].cols > MAX_RESIDENT_COLS) pn[i].foreign = true;
 
     // ---- absorbed nodes: cheap producers recomputed inside every consumer group instead of
     // being materialised (index/random factories, and computations on broadcast operands)
@@ -716,19 +726,19 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
         for (size_t i = 0; i < N; ++i) {
             const CNode &n = cg.nodes[i];
             PNode &p = pn[i];
-            if (p.leaf || p.reduce || n.output >= 0 || p.consumers.empty()) continue;
+            if (p.leaf || p.reduce || p.foreign || n.output >= 0 || p.consumers.empty()) continue;
             bool okc = true;
             if (is_factory(n.op)) {
                 for (uint32_t cidx : p.consumers) {
                     const PNode &q = pn[cidx];
                     uint64_t qr = q.rows, qc = q.cols;
                     if (q.reduce) { qr = p.rows; qc = p.cols; }
-                    if (qr != p.rows || qc != p.cols) okc = false;
+                    if (qr != p.rows || qc != p.cols || q.foreign) okc = false;
                 }
             } else {
                 for (uint32_t cidx : p.consumers) {
                     const PNode &q = pn[cidx];
-                    if (q.reduce || q.numel <= p.numel) okc = false;
+                    if (q.reduce || q.foreign || q.numel <= p.numel) okc = false;
                 }
                 for (int k = 0; okc && k < n.n_in; ++k)
                     if (!pn[n.in[k]].leaf && !pn[n.in[k]].absorbed) okc = false;
@@ -767,14 +777,18 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             dr = pn[n.in[0]].rows;
             dc = pn[n.in[0]].cols;
         }
+        if (p.foreign) {
+            dr = pn[n.in[0]].rows;
+            dc = pn[n.in[0]].cols;
+        }
         native_deps((uint32_t)i, deps);
         int gmin = -1;
         for (uint32_t d : deps) gmin = std::max(gmin, pn[d].group);
         int target = -1;
-        if (fuse) {
+        if (fuse && !p.foreign) {
             auto joinable = [&](int gi) -> bool {
                 const Group &g = groups[gi];
-                if ((int)g.members.size() >= MAX_GROUP_NODES) return false;
+                if (g.kind == K_RED || (int)g.members.size() >= MAX_GROUP_NODES) return false;
                 if (g.rows == dr && g.cols == dc) return true;
                 // an [R,1] computation on row scalars of a wider group stays with that group
                 if (!p.reduce && p.cols == 1 && p.rows == g.rows && g.cols > 1) {
@@ -792,7 +806,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                     if (a == target || a < 0) continue;
                     Group &ga = groups[a];
                     Group &gb = groups[target];
-                    if (ga.rows != gb.rows || ga.cols != gb.cols) continue;
+                    if (ga.kind == K_RED || ga.rows != gb.rows || ga.cols != gb.cols) continue;
                     if (ga.members.size() + gb.members.size() >= (size_t)MAX_GROUP_NODES) continue;
                     bool legal = true;
                     for (uint32_t m : ga.members) {
@@ -819,7 +833,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                 const int lo = std::max(gmin + 1, (int)groups.size() - 8);
                 for (int gi = (int)groups.size() - 1; gi >= lo && target < 0; --gi) {
                     const Group &g = groups[gi];
-                    if (g.rows != dr || g.cols != dc || (int)g.members.size() >= MAX_GROUP_NODES) continue;
+                    if (g.kind == K_RED || g.rows != dr || g.cols != dc || (int)g.members.size() >= MAX_GROUP_NODES) continue;
                     for (int k = 0; k < n.n_in && target < 0; ++k) {
                         const uint32_t o = n.in[k];
                         if (cg.nodes[o].op != N_DEVICE_DATA) continue;
@@ -837,6 +851,12 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             target = (int)groups.size() - 1;
             groups[target].rows = dr;
             groups[target].cols = dc;
+            if (p.foreign) {
+                Group &g = groups[target];
+                g.kind = K_RED;
+                g.red_axis = is_col_reduce(n.op) ? 1 : (is_all_reduce(n.op) ? 2 : 0);
+                g.red_kind = (uint8_t)((n.op - LT_OP_ROW_SUM) % 3);
+            }
         }
         groups[target].members.push_back((uint32_t)i);
         p.group = target;
@@ -879,6 +899,32 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
                         else if (pn[q].group != (int)gi) pn[m].needs_store = true;
                     }
                 }
+            }
+            if (g.kind == K_RED) {
+                // a kernel of its own: slot 0 = the input, slot 1 = the result; no register program
+                const uint32_t m = g.members[0];
+                const uint32_t src = cg.nodes[m].in[0];
+                pn[m].needs_store = true;
+                g.ins.clear();
+                g.io.clear();
+                g.imms.clear();
+                auto slot_for = [&](uint32_t v, bool store) {
+                    const CNode &vn = cg.nodes[v];
+                    IoRef io;
+                    io.is_store = store ? 1 : 0;
+                    io.dtype = vn.dtype;
+                    io.cls = store ? (uint8_t)(g.red_axis == 0 ? LT_CLS_ROWVEC : g.red_axis == 1 ? LT_CLS_COLVEC : LT_CLS_SCALAR) : (uint8_t)LT_CLS_FULL;
+                    io.cnode = v;
+                    if (vn.op == N_DEVICE_DATA) io.kind = IO_PARAM, io.index = (uint32_t)vn.param;
+                    else if (vn.output >= 0) io.kind = IO_OUTPUT, io.index = (uint32_t)vn.output;
+                    else io.kind = IO_TEMP, io.index = 0;
+                    g.io.push_back(io);
+                };
+                slot_for(src, false);
+                slot_for(m, true);
+                g.flavour = 1;
+                for (uint32_t nn : emit) in_emit[nn] = 0;
+                break;
             }
             int n_inputs = 0;
             {
@@ -945,8 +991,15 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
         }
         g.bytes = 0;
         for (const IoRef &io : g.io) g.bytes += io_bytes(g, io);
-        if (g.kind == K_ROW && g.cols > (uint64_t)LT_VM_V * 1024)
-            return fail(c, LT_ERR_UNSUPPORTED, "row-reduction groups support rows of at most 8192 elements");
+        if (g.kind == K_RED) {
+            const size_t scratch = lt_reduce_scratch_bytes(g.red_axis, g.rows, g.cols, c->sm_count);
+            if (scratch) {
+                g.scratch_temp = (int32_t)plan.temp_bytes.size();
+                plan.temp_bytes.push_back(scratch);
+            }
+        }
+        g.long_row = g.kind == K_ROW && g.cols > MAX_RESIDENT_COLS;
+        if (g.long_row && g.cols >= (1ull << 28)) return fail(c, LT_ERR_UNSUPPORTED, "rows of a fused reduction are limited to 2^28 elements");
         if (g.kind == K_EW && g.rowcol) {
             uint64_t cpr = (g.cols + LT_VM_V - 1) / LT_VM_V;
             if (g.rows * cpr >= (1ull << 31) || g.rows >= (1ull << 31) || g.cols >= (1ull << 31))
@@ -1106,7 +1159,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             }
             P.super_prefix[L.groups.size()] = acc;
             P.total_super = acc;
-        } else {
+        } else if (L.kind != K_RED) {
             L.kp.reset(new LtKParams());
             LtKParams &P = *L.kp;
             memset(&P, 0, sizeof(P));
@@ -1125,7 +1178,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
             P.cpr = (uint32_t)((g.cols + LT_VM_V - 1) / LT_VM_V);
             fastdiv_make(P.cpr ? P.cpr : 1, &P.div_mul, &P.div_sh1, &P.div_sh2);
             P.n_chunks = g.rowcol ? (uint64_t)g.rows * P.cpr : (P.n + LT_VM_V - 1) / LT_VM_V;
-            if (g.kind == K_ROW) {
+            if (g.kind == K_ROW && !g.long_row) {
                 uint32_t grp = 1, lg = 0;
                 while (grp < P.cpr) grp <<= 1, ++lg;
                 P.group = grp;
@@ -1136,14 +1189,28 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan) {
         }
     }
     // ---- ahead-of-time compiled kernels: exact lookup of each launch's program
+    bool unfused_long_row = false;
     for (Launch &L : plan.launches) {
         const Group &g = groups[L.groups[0]];
+        if (L.kind == K_RED) continue;
         uint8_t dt[LT_VM_MAX_PTR] = {0}, cl[LT_VM_MAX_PTR] = {0};
         for (size_t s = 0; s < g.io.size() && s < LT_VM_MAX_PTR; ++s) {
             dt[s] = g.io[s].dtype;
             cl[s] = L.kind == K_MULTI ? (uint8_t)LT_CLS_FULL : g.io[s].cls;
         }
         L.compiled = lt_compiled_find(L.kind, L.flavour, g.ins.data(), (uint32_t)g.ins.size(), g.n_pro, dt, cl, (uint32_t)g.io.size());
+        if (g.long_row && (L.compiled < 0 || !c->opt.compiled)) unfused_long_row = true;
+    }
+    if (unfused_long_row) {
+        // Only the kernels instantiated at build time walk a long row in slices.  A long-row group without one is
+        // planned again with each of its reductions as a kernel of its own; what surrounds them becomes elementwise
+        // groups that read the reductions' results as one value per row.
+        if (isolate_long_rows) return fail(c, LT_ERR_UNSUPPORTED, "a long-row group could not be planned");
+        plan.groups.clear();
+        plan.launches.clear();
+        plan.temp_bytes.clear();
+        plan.outputs.clear();
+        return build_plan(c, cg, plan, true);
     }
     return LT_OK;
 }
@@ -1159,7 +1226,7 @@ std::string describe_plan(const Plan &plan) {
             snprintf(buf, sizeof(buf), "  output %zu donated param %d\n", k, plan.outputs[k].donated_param);
             s += buf;
         }
-    static const char *kind[] = {"elementwise", "row", "multi"};
+    static const char *kind[] = {"elementwise", "row", "multi", "reduce"};
     static const char *cls[] = {"full", "colvec", "rowvec", "scalar"};
     static const char *iok[] = {"param", "output", "temp"};
     for (size_t li = 0; li < plan.launches.size(); ++li) {
@@ -1169,7 +1236,11 @@ std::string describe_plan(const Plan &plan) {
                  L.flavour == 0 ? "fast" : (L.flavour == 1 ? "precise" : "ieee"), L.groups.size(), (unsigned long long)g.rows, (unsigned long long)g.cols,
                  g.rowcol ? "rowcol" : "flat", (unsigned long long)L.bytes);
         s += buf;
-        {
+        if (L.kind == K_RED) {
+            static const char *axis[] = {"rows", "columns", "all"}, *what[] = {"sum", "max", "min"};
+            snprintf(buf, sizeof(buf), "  reduction kernel: %s over %s%s\n", what[g.red_kind], axis[g.red_axis], g.scratch_temp >= 0 ? ", two stages" : "");
+            s += buf;
+        } else {
             // the exact identity of the program: what the table of compiled programs is keyed on
             std::string key = "  key: " + std::to_string(L.kind) + " " + std::to_string(L.flavour) + " " + std::to_string(g.n_pro) + " |";
             for (const IoRef &io : g.io) key += " " + std::to_string(io.dtype);
@@ -1200,6 +1271,7 @@ std::string describe_plan(const Plan &plan) {
             s += "\n";
         }
     }
+    if (plan.split) s += "-- the same graph with long row reductions as kernels of their own (used when the fused kernel cannot run):\n" + describe_plan(*plan.split);
     return s;
 }
 

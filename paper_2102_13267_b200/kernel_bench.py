@@ -1,6 +1,6 @@
 """Kernel-only timing of the benchmark configurations and of the common fusion groups (also the driver for ncu captures).
 
-    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5,idioms] [--iters N] [--sets K] [key=value ...]
+    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5,idioms,long,reduce] [--iters N] [--sets K] [key=value ...]
 
 For each configuration: traces the graph and flushes it `iters` times over rotating buffer sets (larger than L2
 together), queued behind a busy stream so that the GPU, not the host, sets the pace.  Two figures are printed:
@@ -161,6 +161,56 @@ def main() -> None:
         report(name[:18], nbytes, kt, region)
         del keep, sets
         ctx.close()
+    # rows longer than a thread group's registers (fused long-row kernels), and reductions over columns / everything
+    def generic(name, nbytes, make, trace):
+        nsets = args.sets or max(2, math.ceil(1.2e9 / nbytes))
+        ctx = context()
+        sets = [make(ctx) for _ in range(nsets)]
+        keep = [None] * nsets
+        for i in range(nsets + 2):
+            keep[i % nsets] = trace(ctx, sets[i % nsets])
+            ctx.barrier()
+        torch.cuda.synchronize()
+        ctx.set_kernel_timing(True)
+        ctx.kernel_timing()
+        hold_gpu()
+        for i in range(args.iters):
+            keep[i % nsets] = trace(ctx, sets[i % nsets])
+            ctx.barrier()
+        kt = ctx.kernel_timing()
+        ctx.set_kernel_timing(False)
+
+        def flush_all():
+            for i in range(args.iters):
+                keep[i % nsets] = trace(ctx, sets[i % nsets])
+                ctx.barrier()
+
+        region = back_to_back(flush_all) if args.iters >= 20 else None
+        report(name[:18], nbytes, kt, region)
+        del keep, sets
+        ctx.close()
+
+    if "long" in which:
+        for rows, cols in ((8192, 16384), (2048, 65536)):
+            for iname in ("softmax_bf16", "layernorm_bf16", "softmax_f32"):
+                _, kinds, trace = next(e for e in idioms.ALL if e[0] == iname)
+                es = 4 if iname.endswith("f32") else 2
+
+                def make(c, kinds=kinds, rows=rows, cols=cols):
+                    out = []
+                    for k in kinds:
+                        t = torch.randn((rows, cols) if k.startswith("mat") else (cols,), device=dev)
+                        out.append(c.from_torch(t.to(torch.bfloat16) if k.endswith("bf16") else t))
+                    return out
+
+                generic(f"{iname[:10]} {cols}", 2 * es * rows * cols, make, lambda c, s_, trace=trace, cols=cols: trace(c, s_, cols))
+    if "reduce" in which:
+        for rows, cols in ((16384, 4096), (1 << 20, 64)):
+            for op in ("col_sum", "all_sum", "row_sum"):
+                generic(f"{op} {rows}x{cols}", 4 * rows * cols, lambda c, rows=rows, cols=cols: [c.from_torch(torch.randn((rows, cols), device=dev))],
+                        lambda c, s_, op=op: c.op(op, s_[0]))
+        generic("row_sum 4096x65536", 4 * 4096 * 65536, lambda c: [c.from_torch(torch.randn((4096, 65536), device=dev))],
+                lambda c, s_: c.op("row_sum", s_[0]))
     if "c5" in which:
         shapes = parameter_shapes()
         ctx = context()

@@ -1,0 +1,208 @@
+"""GPU parity of the wider reduction shapes against the CPU eager oracle: rows longer than a thread group keeps
+in registers (fused long-row kernels and the split plan), column and whole-tensor reductions, outer broadcasts,
+and the bounded device-side wait."""
+import math
+
+import numpy as np
+import pytest
+
+from helpers import assert_matches
+from oracle.eager import EagerOracle, max_threads, set_threads
+from workloads import configs, idioms, rng, traces
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lt():
+    import paper_2102_13267_b200 as lt
+    set_threads(max_threads())
+    return lt
+
+
+@pytest.fixture()
+def ctx(lt):
+    c = lt.LazyContext(device=0)
+    yield c
+    c.close()
+
+
+def _idiom_inputs(kinds, shape, seed):
+    g = rng.generator(seed, 9)
+    arrs = []
+    for k in kinds:
+        what, dt = k.split(":")
+        shp = shape if what == "mat" else (shape[-1],)
+        a = rng.normal_f32(g, shp, 1.0, 1.0 if what == "vec" else 0.0)
+        arrs.append((rng.to_bf16_bits(a) if dt == "bf16" else a, dt))
+    return arrs
+
+
+LONG_IDIOMS = ["softmax_bf16", "softmax_f32", "scaled_softmax_bf16", "layernorm_bf16", "layernorm_f32", "rmsnorm_bf16"]
+
+
+@pytest.mark.parametrize("shape", [(5, 16384), (3, 65536), (4, 10000), (2, 8200), (300, 16384), (2, 3, 12288)])
+@pytest.mark.parametrize("idiom", LONG_IDIOMS)
+def test_listed_groups_on_long_rows_run_fused(ctx, idiom, shape):
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == idiom)
+    arrs = _idiom_inputs(kinds, shape, 61)
+    O = EagerOracle()
+    ref = trace(O, [O.leaf(a, d) for a, d in arrs], shape[-1])
+    out = trace(ctx, [ctx.leaf(a, d) for a, d in arrs], shape[-1])
+    ctx.barrier()
+    st = ctx.stats()
+    assert st["kernels_launched"] == 1 and st["launches_row"] == 1 and st["launches_compiled"] == 1, st
+    assert_matches(ctx.fetch(out), ref.array, "f32" if name.endswith("f32") else "bf16", f"{name} {shape}")
+
+
+@pytest.mark.parametrize("depth", [0, 1, 2])
+def test_long_row_staging_depths_agree(lt, depth):
+    """Rows staged in shared memory two ahead, one ahead, or read from global memory in every pass."""
+    shape = (37, 16384)
+    c = lt.LazyContext(device=0)
+    c.set_option("debug.compiled_depth", depth)
+    x, h, g, b = configs.c3_inputs(62, shape)
+    O = EagerOracle()
+    kw = dict(shape=shape, p=0.1, eps=1e-5, seed=0xABCDEF, offset=3)
+    zr, kr = traces.residual_dropout_layernorm(O, O.leaf(x, "bf16"), O.leaf(h, "bf16"), O.leaf(g, "f32"), O.leaf(b, "f32"), **kw)
+    z, k = traces.residual_dropout_layernorm(c, c.leaf(x, "bf16"), c.leaf(h, "bf16"), c.leaf(g, "f32"), c.leaf(b, "f32"), **kw)
+    c.barrier()
+    st = c.stats()
+    assert st["kernels_launched"] == 1 and st["launches_compiled"] == 1
+    assert_matches(c.fetch(k), kr.array, "u8", "long c3 mask")
+    assert_matches(c.fetch(z), zr.array, "bf16", "long c3 z")
+    c.close()
+
+
+def test_causal_softmax_on_long_rows(ctx):
+    shape = (1, 20, 16384)
+    s = configs.c4_inputs(63, shape)
+    O = EagerOracle()
+    ref = traces.causal_softmax(O, O.leaf(s, "bf16"), shape=shape, scale=1 / math.sqrt(128))
+    y = traces.causal_softmax(ctx, ctx.leaf(s, "bf16"), shape=shape, scale=1 / math.sqrt(128))
+    ctx.barrier()
+    assert ctx.stats()["launches_compiled"] == 1
+    got = ctx.fetch(y)
+    assert_matches(got, ref.array, "bf16", "long causal softmax")
+    assert (got[0, 3, 4:] == 0).all()
+
+
+def test_in_place_softmax_on_long_rows(ctx):
+    shape = (150, 16384)
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == "softmax_bf16")
+    arrs = _idiom_inputs(kinds, shape, 64)
+    O = EagerOracle()
+    ol, gl = [O.leaf(a, d) for a, d in arrs], [ctx.leaf(a, d) for a, d in arrs]
+    ptr = ctx.device_ptr(gl[0])
+    for _ in range(2):
+        ol[0] = trace(O, ol, shape[-1])
+        ctx.assign(gl[0], trace(ctx, gl, shape[-1]))
+        ctx.barrier()
+    st = ctx.stats()
+    assert st["outputs_donated"] == 2 and st["outputs_allocated"] == 0 and ctx.device_ptr(gl[0]) == ptr
+    assert_matches(ctx.fetch(gl[0]), ol[0].array, "bf16", "in-place long softmax")
+
+
+def _unlisted(B, z):
+    """A row-normalisation no kernel was instantiated for: |z - max| / (sum |z - max| + 3)."""
+    d = B.op("abs", B.op("sub", z, B.op("row_max", z)))
+    return B.op("div", d, B.op("add", B.op("row_sum", d), B.scalar(3.0)))
+
+
+@pytest.mark.parametrize("shape", [(6, 16384), (3, 9001), (2, 70000), (40, 8193)])
+def test_unlisted_long_row_graph_runs_split(ctx, shape):
+    z = rng.normal_f32(rng.generator(65), shape, 1.0)
+    O = EagerOracle()
+    ref = _unlisted(O, O.leaf(z, "f32"))
+    out = _unlisted(ctx, ctx.leaf(z, "f32"))
+    ctx.barrier()
+    st = ctx.stats()
+    assert st["launches_reduce"] == 2 and st["launches_row"] == 0, st
+    assert_matches(ctx.fetch(out), ref.array, "f32", f"split long rows {shape}")
+
+
+def test_listed_group_with_unaligned_input_falls_back_to_the_split_plan(ctx):
+    import torch
+
+    shape = (7, 16384)
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == "softmax_f32")
+    (x, _), = _idiom_inputs(kinds, shape, 66)
+    store = torch.zeros(x.size + 8, dtype=torch.float32, device="cuda:0")
+    view = store[1:1 + x.size]  # 4-byte aligned only
+    view.copy_(torch.from_numpy(x.reshape(-1)).to("cuda:0"))
+    t = ctx.from_device_ptr(view.data_ptr(), "f32", shape, keep=store)
+    O = EagerOracle()
+    ref = trace(O, [O.leaf(x, "f32")], shape[-1])
+    out = trace(ctx, [t], shape[-1])
+    ctx.barrier()
+    st = ctx.stats()
+    assert st["launches_reduce"] == 2 and st["launches_row"] == 0, st
+    assert "kernels of their own" in ctx.dump_plan()
+    assert_matches(ctx.fetch(out), ref.array, "f32", "split fallback")
+    # the same graph on an aligned input afterwards: the cached plan's fused kernel
+    t2 = ctx.leaf(x, "f32")
+    out2 = trace(ctx, [t2], shape[-1])
+    ctx.barrier()
+    st2 = ctx.stats()
+    assert st2["cache_hits"] == 1 and st2["launches_row"] == 1
+    assert_matches(ctx.fetch(out2), ref.array, "f32", "fused after fallback")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 1), (3, 5), (1000, 7), (257, 96), (4, 3, 130), (5000,), (20000, 33), (64, 4096)])
+def test_column_and_whole_tensor_reductions(ctx, dtype, shape):
+    x = rng.normal_f32(rng.generator(67), shape, 2.0)
+    a = x if dtype == "f32" else rng.to_bf16_bits(x)
+    O = EagerOracle()
+    ox, gx = O.leaf(a, dtype), ctx.leaf(a, dtype)
+    names = ["col_sum", "col_max", "col_min", "all_sum", "all_max", "all_min"]
+    outs = [ctx.op(n, gx) for n in names]
+    ctx.barrier()
+    assert ctx.stats()["launches_reduce"] == 6
+    for n, t in zip(names, outs):
+        ref = O.op(n, ox)
+        assert_matches(ctx.fetch(t), ref.array, dtype, f"{n} {dtype} {shape}")
+
+
+def test_reduction_results_feed_later_groups(ctx):
+    shape = (300, 72)
+    x = rng.normal_f32(rng.generator(68), shape, 1.0)
+    O = EagerOracle()
+
+    def graph(B, t):
+        centred = B.op("sub", t, B.op("mul", B.op("col_sum", t), B.scalar(1.0 / shape[0])))      # column means removed
+        scaled = B.op("div", centred, B.op("add", B.op("all_max", B.op("abs", centred)), B.scalar(1.0)))  # global scale
+        return B.op("add", scaled, B.op("row_max", scaled))
+
+    ref = graph(O, O.leaf(x, "f32"))
+    out = graph(ctx, ctx.leaf(x, "f32"))
+    ctx.barrier()
+    assert ctx.stats()["launches_reduce"] == 2
+    assert_matches(ctx.fetch(out), ref.array, "f32", "reductions feeding groups")
+
+
+def test_outer_broadcast(ctx):
+    g = rng.generator(69)
+    r, cv = rng.normal_f32(g, (37, 1)), rng.normal_f32(g, (1, 100))
+    O = EagerOracle()
+    for name in ("mul", "sub", "max"):
+        ref = O.op(name, O.leaf(r, "f32"), O.leaf(cv, "f32"))
+        got = ctx.fetch(ctx.op(name, ctx.leaf(r, "f32"), ctx.leaf(cv, "f32")))
+        assert_matches(got, ref.array, "f32", f"outer {name}", exact=True)
+        ref = O.op(name, O.leaf(cv.reshape(100), "f32"), O.leaf(r, "f32"))
+        got = ctx.fetch(ctx.op(name, ctx.leaf(cv.reshape(100), "f32"), ctx.leaf(r, "f32")))
+        assert_matches(got, ref.array, "f32", f"outer {name} swapped", exact=True)
+
+
+def test_bounded_wait_gives_up_and_is_reported(lt):
+    """The kernel that stages long rows waits for its copies with a time limit.  Here the limit runs out on a wait
+    nothing can satisfy (no copy is involved): the next blocking call reports it, and the context stays usable."""
+    c = lt.LazyContext(device=0)
+    x = c.leaf(np.arange(64, dtype=np.float32).reshape(8, 8), "f32")
+    c.debug_wait_probe(2_000_000)  # 2 ms
+    with pytest.raises(lt.LazyTensorError) as err:
+        c.barrier(blocking=True)
+    assert err.value.status == lt.STATUS_NAMES.index("LT_ERR_DEVICE_TIMEOUT")
+    c.barrier(blocking=True)  # reported once
+    np.testing.assert_array_equal(c.fetch(x + 1.0), np.arange(64, dtype=np.float32).reshape(8, 8) + 1)
+    c.close()

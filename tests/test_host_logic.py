@@ -301,8 +301,8 @@ def test_error_paths(ctx):
         ctx.op("add", fake(ctx, (4, 8), "i32"), ctx.scalar(0.5))
     assert e.value.status == 3
     with pytest.raises(lt.LazyTensorError) as e:
-        ctx.op("row_sum", fake(ctx, (2, 8200)))
-    assert e.value.status == 5  # LT_ERR_UNSUPPORTED
+        ctx.op("col_sum", fake(ctx, (4, 8), "i32"))
+    assert e.value.status == 3
     with pytest.raises(lt.LazyTensorError) as e:
         ctx.op("exp", fake(ctx, (4,), "i32"))
     assert e.value.status == 3
@@ -454,3 +454,64 @@ def test_host_bench_driver_runs_without_python_in_the_loop():
     assert "compiles 1, hits 19999" in lines[0] and "compiles 1, hits 19999" in lines[1]
     assert "compiles 1, hits 99," in lines[2]
     assert "replays 99" in lines[3]
+
+
+# ------------------------------------------------------------------ long rows and the other reduction shapes
+def test_long_row_groups_fused_when_listed_and_split_otherwise():
+    from workloads import idioms
+
+    ctx = lt.LazyContext(device=None)
+    x = fake(ctx, (4, 16384), "bf16")
+    y = idioms.softmax(ctx, x, cols=16384)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("launch ") == 1 and "compiled: softmax_bf16" in plan and "rows=4 cols=16384" in plan
+    # a graph with no kernel instantiated for it: each long reduction becomes a kernel of its own, the arithmetic
+    # around it elementwise kernels that read one value per row
+    z = fake(ctx, (4, 16384))
+    d = ctx.op("sub", z, ctx.op("row_max", z))
+    w = ctx.op("div", ctx.op("abs", d), ctx.op("add", ctx.op("row_sum", ctx.op("abs", d)), ctx.scalar(3.0)))
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("reduction kernel: max over rows") == 1 and plan.count("reduction kernel: sum over rows") == 1
+    assert "launch 0: reduce" in plan and "rowvec" in plan
+    st = ctx.stats()
+    assert st["launches_reduce"] == 2
+    # the same graph at 8192 columns stays one fused row kernel
+    z = fake(ctx, (4, 8192))
+    d = ctx.op("sub", z, ctx.op("row_max", z))
+    w2 = ctx.op("div", ctx.op("abs", d), ctx.op("add", ctx.op("row_sum", ctx.op("abs", d)), ctx.scalar(3.0)))
+    ctx.barrier()
+    assert ctx.dump_plan().count("launch ") == 1
+    del y, w, w2
+
+
+def test_column_and_whole_tensor_reductions_plan_as_their_own_kernels():
+    ctx = lt.LazyContext(device=None)
+    x = fake(ctx, (512, 96))
+    s = ctx.op("col_sum", ctx.op("mul", x, x))          # the product is materialised, then reduced
+    t = ctx.op("all_max", x)
+    u = ctx.op("sub", x, ctx.op("col_max", x))           # result read back as a column vector
+    v = ctx.op("mul", x, t)                              # rank-0 result read back as a broadcast scalar
+    assert s.shape == (1, 96) and t.shape == () and u.shape == (512, 96)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("reduction kernel: sum over columns") == 1
+    assert plan.count("reduction kernel: max over all") == 1
+    assert plan.count("reduction kernel: max over columns") == 1
+    assert "colvec" in plan and "scalar" in plan
+    assert ctx.stats()["launches_reduce"] == 3
+    with pytest.raises(lt.LazyTensorError):
+        ctx.op("all_sum", ctx.scalar(2.0))
+    del s, t, u, v
+
+
+def test_outer_broadcast_of_row_scalars_and_column_vector():
+    ctx = lt.LazyContext(device=None)
+    r, cvec = fake(ctx, (7, 1)), fake(ctx, (1, 40))
+    y = ctx.op("mul", r, cvec)
+    assert y.shape == (7, 40)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("launch ") == 1 and "rowvec" in plan and "colvec" in plan
+    del y
