@@ -1006,8 +1006,7 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uin
                  : "memory");
 }
 
-constexpr int C_LONG_THREADS = 256;
-constexpr int C_LONG_U = 2;
+constexpr int C_LONG_U = 2;  // chunks per thread and slice; CTAs of 256 threads, or 512 when only one fits an SM
 constexpr uint32_t C_LONG_MAX_BULK = 1u << 19;  // keeps a stage's byte count inside the mbarrier's transaction counter
 
 // compile-time walks over the slots of a program (the program tables are not addressable at run time in device code)
@@ -1045,7 +1044,24 @@ __device__ __forceinline__ void long_issue(const Ptr &ptr, uint32_t cols, uint32
     }
 }
 
-template <int KIND>
+// Asks for `bytes` (a multiple of 16) at `src` to be brought into L2; nothing waits for it.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+template <class PG, int S = 0, class Ptr>
+__device__ __forceinline__ void long_prefetch(const Ptr &ptr, uint32_t cols, uint32_t row) {
+    if constexpr (S < PG::n_slots) {
+        if constexpr (Info<PG>::full_input(S)) {
+            const uint32_t bytes = cols * Info<PG>::elem_bytes(S);
+            const char *src = reinterpret_cast<const char *>(ptr(S)) + (uint64_t)row * bytes;
+            for (uint32_t done = 0; done < bytes; done += C_LONG_MAX_BULK)
+                bulk_prefetch_l2(src + done, bytes - done < C_LONG_MAX_BULK ? bytes - done : C_LONG_MAX_BULK);
+        }
+        long_prefetch<PG, S + 1>(ptr, cols, row);
+    }
+}
+
+template <int KIND, int T>
 __device__ __forceinline__ float long_cta_reduce(float v, float *buf) {
 #pragma unroll
     for (uint32_t off = 16; off > 0; off >>= 1) v = GroupReduce::red_comb<KIND>(v, __shfl_xor_sync(0xffffffffu, v, off));
@@ -1054,20 +1070,22 @@ __device__ __forceinline__ float long_cta_reduce(float v, float *buf) {
     __syncthreads();
     float r = buf[0];
 #pragma unroll
-    for (int w = 1; w < C_LONG_THREADS / 32; ++w) r = GroupReduce::red_comb<KIND>(r, buf[w]);
+    for (int w = 1; w < T / 32; ++w) r = GroupReduce::red_comb<KIND>(r, buf[w]);
     return r;
 }
 
-// Rows too long for a thread group's registers: a CTA owns a row and walks it in slices of 256 x 2 chunks.  A program
+// Rows too long for a thread group's registers: a CTA of T threads owns a row and walks it in slices of T x 2 chunks.  A program
 // with n reductions makes n + 1 passes over the row (Machine::run_phase).  With `depth` > 0 the row's full-class
 // inputs are brought into shared memory once, by one-dimensional bulk asynchronous copies that complete on an
 // mbarrier, `depth` rows ahead; every pass then reads the staged row.  With depth 0 the passes read global memory
 // (the row was just read by this CTA and sits in L2).  The wait for a stage is bounded: when it gives up the CTA
 // raises bit 0 of lt_device_status, waits (again bounded) for the copies it still has in flight and returns.
-template <class PG>
-__global__ void __launch_bounds__(C_LONG_THREADS) lt_c_longrow(const __grid_constant__ LtKParams P, uint32_t depth, uint32_t stage_bytes,
-                                                               uint64_t limit_ns) {
-    constexpr int U = C_LONG_U, T = C_LONG_THREADS, NR = Info<PG>::n_reds();
+// `l2_ahead` (when the rows are multiples of 16 bytes): while a row is processed, the row the CTA stages or reads
+// next is requested into L2, so that HBM keeps streaming during the passes that read no global memory.
+template <class PG, int T>
+__global__ void __launch_bounds__(T) lt_c_longrow(const __grid_constant__ LtKParams P, uint32_t depth, uint32_t stage_bytes,
+                                                  uint64_t limit_ns, uint32_t l2_ahead) {
+    constexpr int U = C_LONG_U, NR = Info<PG>::n_reds();
     static_assert(NR <= 4, "at most four reductions per long-row program");
     using M = Machine<PG, U, PtrK, ScalK, LongRed, true>;
     __shared__ float red_buf[T / 32];
@@ -1103,6 +1121,10 @@ __global__ void __launch_bounds__(C_LONG_THREADS) lt_c_longrow(const __grid_cons
     for (uint32_t row = blockIdx.x; row < P.rows; row += gridDim.x, ++k) {
         const uint32_t s = depth ? k % depth : 0u;
         const unsigned char *stage = stage_mem + (size_t)s * stage_bytes;
+        if (l2_ahead && threadIdx.x == 0) {
+            const uint32_t ahead = row + (depth ? depth : 1u) * gridDim.x;  // not yet requested by a copy into shared memory
+            if (ahead < P.rows) long_prefetch<PG>(ptr, P.cols, ahead);
+        }
         if (depth) {
             const bool landed = mbar_wait_bounded(bar0 + 8 * s, (k / depth) & 1u, limit_ns);
             if (__syncthreads_or(landed ? 0 : 1)) {
@@ -1130,7 +1152,7 @@ __global__ void __launch_bounds__(C_LONG_THREADS) lt_c_longrow(const __grid_cons
                 else m.issue_loads();
                 m.template run_phase<PHASE>();
             }
-            if constexpr (PHASE < NR) red.val[PHASE] = long_cta_reduce<Info<PG>::red_kind(PHASE)>(red.part, red_buf);
+            if constexpr (PHASE < NR) red.val[PHASE] = long_cta_reduce<Info<PG>::red_kind(PHASE), T>(red.part, red_buf);
         };
         pass(std::integral_constant<int, 0>{});
         if constexpr (NR >= 1) pass(std::integral_constant<int, 1>{});
@@ -1264,24 +1286,38 @@ bool long_stage_allowed(uint32_t cols) {  // every staged row a multiple of 16 b
     }
 }
 
+template <class PG, int T>
+cudaError_t launch_long_t(const LtKParams &P, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns, bool l2_ahead,
+                          cudaStream_t stream) {
+    const size_t dyn = (size_t)depth * stage_bytes;
+    cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG, T>, dyn);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(lt_c_longrow<PG, T>, grid, (unsigned)T, dyn, stream, P, (uint32_t)depth, (uint32_t)stage_bytes, limit_ns,
+                      (uint32_t)(l2_ahead ? 1 : 0));
+}
+
 template <class PG>
-cudaError_t launch_long(const LtKParams &P, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns, cudaStream_t stream) {
+cudaError_t launch_long(const LtKParams &P, unsigned grid, unsigned threads, unsigned depth, size_t stage_bytes, uint64_t limit_ns,
+                        bool l2_ahead, cudaStream_t stream) {
     if constexpr (PG::kind == 1 && Info<PG>::n_reds() <= 4) {
-        const size_t dyn = (size_t)depth * stage_bytes;
-        cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG>, dyn);
-        if (e != cudaSuccess) return e;
-        return launch_pdl(lt_c_longrow<PG>, grid, C_LONG_THREADS, dyn, stream, P, (uint32_t)depth, (uint32_t)stage_bytes, limit_ns);
+        return threads >= 512 ? launch_long_t<PG, 512>(P, grid, depth, stage_bytes, limit_ns, l2_ahead, stream)
+                              : launch_long_t<PG, 256>(P, grid, depth, stage_bytes, limit_ns, l2_ahead, stream);
     } else {
         return cudaErrorInvalidValue;
     }
 }
 
 template <class PG>
-cudaError_t long_occupancy(size_t dyn, int *blocks) {
+cudaError_t long_occupancy(unsigned threads, size_t dyn, int *blocks) {
     if constexpr (PG::kind == 1 && Info<PG>::n_reds() <= 4) {
-        cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG>, dyn);
+        if (threads >= 512) {
+            cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG, 512>, dyn);
+            if (e != cudaSuccess) return e;
+            return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_longrow<PG, 512>, 512, dyn);
+        }
+        cudaError_t e = row_smem_attr((const void *)lt_c_longrow<PG, 256>, dyn);
         if (e != cudaSuccess) return e;
-        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_longrow<PG>, C_LONG_THREADS, dyn);
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_longrow<PG, 256>, 256, dyn);
     } else {
         return cudaErrorInvalidValue;
     }
@@ -1299,21 +1335,22 @@ size_t lt_compiled_long_stage_bytes(int id, uint32_t cols) {
     return 0;
 }
 
-cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns,
-                                    cudaStream_t stream) {
+cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned threads, unsigned depth, size_t stage_bytes,
+                                    uint64_t limit_ns, int l2_ahead, cudaStream_t stream) {
     int k = 0;
-#define LT_X(PG)                                                                                                              \
-    if (k == id) return launch_long<PG>(*static_cast<const LtKParams *>(params), grid, depth, stage_bytes, limit_ns, stream); \
+#define LT_X(PG)                                                                                                                  \
+    if (k == id)                                                                                                                  \
+        return launch_long<PG>(*static_cast<const LtKParams *>(params), grid, threads, depth, stage_bytes, limit_ns, l2_ahead != 0, stream); \
     ++k;
     LT_COMPILED_LIST(LT_X)
 #undef LT_X
     return cudaErrorInvalidValue;
 }
 
-cudaError_t lt_compiled_long_occupancy(int id, size_t dyn_smem, int *blocks) {
+cudaError_t lt_compiled_long_occupancy(int id, unsigned threads, size_t dyn_smem, int *blocks) {
     int k = 0;
-#define LT_X(PG)                                        \
-    if (k == id) return long_occupancy<PG>(dyn_smem, blocks); \
+#define LT_X(PG)                                                  \
+    if (k == id) return long_occupancy<PG>(threads, dyn_smem, blocks); \
     ++k;
     LT_COMPILED_LIST(LT_X)
 #undef LT_X

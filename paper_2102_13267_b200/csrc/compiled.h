@@ -32,9 +32,10 @@ int lt_compiled_bounds_violations(unsigned long long *out);
 // `depth` 0 = passes read global memory, 1 or 2 = rows staged that far ahead by bulk asynchronous copies whose
 // completion the kernel awaits for at most `limit_ns` nanoseconds.
 size_t lt_compiled_long_stage_bytes(int id, uint32_t cols);
-cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned depth, size_t stage_bytes, uint64_t limit_ns,
-                                    cudaStream_t stream);
-cudaError_t lt_compiled_long_occupancy(int id, size_t dyn_smem, int *blocks);
+// `threads`: 256 or 512 per CTA.  `l2_ahead` non-zero: the row a CTA takes next is requested into L2 while it works.
+cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned threads, unsigned depth, size_t stage_bytes,
+                                    uint64_t limit_ns, int l2_ahead, cudaStream_t stream);
+cudaError_t lt_compiled_long_occupancy(int id, unsigned threads, size_t dyn_smem, int *blocks);
 // Device status word (bit 0: a bounded wait gave up); synchronises the device.  `clear` resets it when set.
 cudaError_t lt_device_status_read(unsigned int *out, int clear);
 // Launches a one-warp kernel that waits `limit_ns` for an mbarrier phase nothing completes and then raises bit 0.

@@ -473,6 +473,7 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "debug.compiled_u")) c->opt.compiled_u = value;
     else if (!strcmp(key, "debug.compiled_row_u")) c->opt.compiled_row_u = value;
     else if (!strcmp(key, "debug.compiled_depth")) c->opt.compiled_depth = value;
+    else if (!strcmp(key, "debug.long_l2_ahead")) c->opt.long_l2_ahead = value;
     else if (!strcmp(key, "wait_limit_ms")) c->wait_limit_ns = value > 0 ? value * 1000000ll : 1;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;

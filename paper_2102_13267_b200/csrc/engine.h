@@ -162,6 +162,7 @@ struct Options {
     int64_t compiled_row_u = 0;  // chunks per thread in compiled row kernels (0 = one warp per row where it fits)
     int64_t compiled_depth = -1;  // staging depth of compiled row kernels (-1 = default, 0 = direct loads)
     int64_t compiled_u = 0;  // chunks in flight per thread in compiled elementwise / multi kernels (0 = default)
+    int64_t long_l2_ahead = -1;  // long-row kernels: request the next row into L2 (-1 = the library's choice)
 };
 
 struct HashKey {

@@ -328,19 +328,39 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                 // a CTA per row, walking it in slices; rows staged in shared memory `depth` ahead when they fit
                 // (feasibility was checked on entry)
                 if (!dry) {
+                    // Staging and CTA size: the row a CTA works on is staged when it fits; several CTAs per SM overlap one
+                    // another's passes; when a staged row leaves room for one CTA only, that CTA has 512 threads.
                     const size_t cap = 200u * 1024u;
                     const size_t stage = lt_compiled_long_stage_bytes(L.compiled, P.cols);
-                    unsigned depth = stage == 0 ? 0u : (unsigned)std::min<size_t>(2, cap / stage);
-                    if (c->opt.compiled_depth >= 0) depth = std::min<unsigned>(depth, (unsigned)c->opt.compiled_depth);
-                    int occ = 1;
-                    if (lt_compiled_long_occupancy(L.compiled, depth * stage, &occ) != cudaSuccess || occ < 1) {
-                        cudaGetLastError();
-                        occ = 1;
+                    const unsigned deepest = stage == 0 ? 0u : (unsigned)std::min<size_t>(2, cap / stage);
+                    auto blocks_at = [&](unsigned threads, unsigned d) {
+                        int b = 0;
+                        if (lt_compiled_long_occupancy(L.compiled, threads, d * stage, &b) != cudaSuccess || b < 1) {
+                            cudaGetLastError();
+                            b = 1;
+                        }
+                        return b;
+                    };
+                    // (one row ahead: two measured no faster, and the shared memory it takes is L1 the column vectors miss)
+                    unsigned depth = std::min(deepest, 1u), threads = 256;
+                    int occ = blocks_at(256, depth);
+                    if (occ < 2 && depth >= 1) {
+                        threads = 512;
+                        occ = blocks_at(512, depth);
+                    }
+                    if (c->opt.compiled_depth >= 0 && (unsigned)c->opt.compiled_depth <= deepest) {
+                        depth = (unsigned)c->opt.compiled_depth;
+                        threads = c->opt.compiled_row_u == 512 ? 512 : 256;
+                        occ = blocks_at(threads, depth);
                     }
                     unsigned grid = (unsigned)std::min<uint64_t>(P.rows, (uint64_t)c->sm_count * occ);
                     if (grid < 1) grid = 1;
+                    // rows are multiples of 16 bytes when they can be staged; the request pays off when one CTA per SM
+                    // leaves HBM idle during the passes that read shared memory only
+                    bool l2_ahead = stage != 0 && occ < 2 && depth >= 1;
+                    if (c->opt.long_l2_ahead >= 0) l2_ahead = stage != 0 && c->opt.long_l2_ahead != 0;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch_long(L.compiled, &P, grid, depth, stage, (uint64_t)c->wait_limit_ns, c->stream);
+                    e = lt_compiled_launch_long(L.compiled, &P, grid, threads, depth, stage, (uint64_t)c->wait_limit_ns, l2_ahead ? 1 : 0, c->stream);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     if (depth) c->status_pending = true;
                 }

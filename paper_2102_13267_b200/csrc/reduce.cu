@@ -76,33 +76,67 @@ __global__ void __launch_bounds__(RT) lt_reduce_rows(const void *in, void *out, 
     }
 }
 
-// Column reduction, one stage: CTA (bx, by) reduces rows [by * rows_per, ...) of the 32 columns bx * 32 ..;
-// thread (x, y) of the 32 x 8 CTA walks rows y, y + 8, ...  The result goes to dst[by * cols + col].
-template <int DT_IN, int DT_OUT, int KIND>
+// W consecutive elements starting at element i (W = 4: i is a multiple of 4 and the array 16-byte aligned)
+template <int DT, int W>
+__device__ __forceinline__ void load_vec(const void *p, uint64_t i, double (&v)[W]) {
+    if constexpr (W == 1) {
+        v[0] = load_as_double<DT>(p, i);
+    } else if constexpr (DT == 0) {
+        const float4 f = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p) + i));
+        v[0] = f.x, v[1] = f.y, v[2] = f.z, v[3] = f.w;
+    } else if constexpr (DT == 1) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const unsigned short *>(p) + i));
+        v[0] = __uint_as_float(w.x << 16), v[1] = __uint_as_float(w.x & 0xffff0000u);
+        v[2] = __uint_as_float(w.y << 16), v[3] = __uint_as_float(w.y & 0xffff0000u);
+    } else {
+        const double2 a = reinterpret_cast<const double2 *>(reinterpret_cast<const double *>(p) + i)[0];
+        const double2 b = reinterpret_cast<const double2 *>(reinterpret_cast<const double *>(p) + i)[1];
+        v[0] = a.x, v[1] = a.y, v[2] = b.x, v[3] = b.y;
+    }
+}
+
+// Column reduction, one stage: CTA (bx, by) reduces rows [by * rows_per, ...) of the 32 * W columns bx * 32 * W ..;
+// thread (x, y) of the 32 x 8 CTA owns W adjacent columns and walks rows y, y + 8, ...  The result goes to
+// dst[by * cols + col].  W = 4 needs cols % 4 == 0 and a 16-byte aligned input.
+template <int DT_IN, int DT_OUT, int KIND, int W>
 __global__ void __launch_bounds__(RT) lt_reduce_cols(const void *in, void *dst, uint64_t rows, uint64_t cols, uint64_t rows_per) {
-    __shared__ double smem[8][33];
+    __shared__ double smem[8][32 * W + 1];
     pdl_release();
     pdl_wait();
     const uint32_t x = threadIdx.x & 31u, y = threadIdx.x >> 5;
-    const uint64_t col = (uint64_t)blockIdx.x * 32u + x;
+    const uint64_t col = ((uint64_t)blockIdx.x * 32u + x) * W;
     const uint64_t r0 = (uint64_t)blockIdx.y * rows_per;
     const uint64_t r1 = r0 + rows_per < rows ? r0 + rows_per : rows;
-    double a0 = ident<KIND>(), a1 = ident<KIND>();
+    double a0[W], a1[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) a0[w] = a1[w] = ident<KIND>();
     if (col < cols) {
         uint64_t r = r0 + y;
         for (; r + 8 < r1; r += 16) {
-            a0 = comb<KIND>(a0, load_as_double<DT_IN>(in, r * cols + col));
-            a1 = comb<KIND>(a1, load_as_double<DT_IN>(in, (r + 8) * cols + col));
-        }
-        if (r < r1) a0 = comb<KIND>(a0, load_as_double<DT_IN>(in, r * cols + col));
-    }
-    smem[y][x] = comb<KIND>(a0, a1);
-    __syncthreads();
-    if (y == 0 && col < cols) {
-        double v = smem[0][x];
+            double v0[W], v1[W];
+            load_vec<DT_IN, W>(in, r * cols + col, v0);
+            load_vec<DT_IN, W>(in, (r + 8) * cols + col, v1);
 #pragma unroll
-        for (int k = 1; k < 8; ++k) v = comb<KIND>(v, smem[k][x]);
-        store_from_double<DT_OUT>(dst, (uint64_t)blockIdx.y * cols + col, v);
+            for (int w = 0; w < W; ++w) a0[w] = comb<KIND>(a0[w], v0[w]), a1[w] = comb<KIND>(a1[w], v1[w]);
+        }
+        if (r < r1) {
+            double v0[W];
+            load_vec<DT_IN, W>(in, r * cols + col, v0);
+#pragma unroll
+            for (int w = 0; w < W; ++w) a0[w] = comb<KIND>(a0[w], v0[w]);
+        }
+    }
+#pragma unroll
+    for (int w = 0; w < W; ++w) smem[y][x * W + w] = comb<KIND>(a0[w], a1[w]);
+    __syncthreads();
+    // thread t of the first 32 * W finishes column bx * 32 * W + t
+    for (uint32_t t = threadIdx.x; t < 32u * W; t += RT) {
+        const uint64_t cc = (uint64_t)blockIdx.x * 32u * W + t;
+        if (cc >= cols) continue;
+        double v = smem[0][t];
+#pragma unroll
+        for (int k = 1; k < 8; ++k) v = comb<KIND>(v, smem[k][t]);
+        store_from_double<DT_OUT>(dst, (uint64_t)blockIdx.y * cols + cc, v);
     }
 }
 
@@ -134,17 +168,23 @@ cudaError_t launch_typed(int axis, const void *in, void *out, void *scratch, uin
         return launch_pdl(lt_reduce_rows<DT, KIND>, grid, RT, (size_t)0, stream, in, out, (uint32_t)rows, cols);
     }
     if (axis == 1) {
-        const unsigned gx = (unsigned)((cols + 31) / 32);
+        const bool wide = (cols % 4) == 0 && ((uintptr_t)in % 16) == 0;
+        const unsigned gx = (unsigned)((cols + (wide ? 127 : 31)) / (wide ? 128 : 32));
+        const unsigned gx2 = (unsigned)((cols + ((cols % 4) == 0 ? 127 : 31)) / ((cols % 4) == 0 ? 128 : 32));
         if (parts <= 1) {
             *launched = 1;
-            return launch_pdl_grid(lt_reduce_cols<DT, DT, KIND>, dim3(gx, 1), RT, stream, in, out, rows, cols, rows);
+            return wide ? launch_pdl_grid(lt_reduce_cols<DT, DT, KIND, 4>, dim3(gx, 1), RT, stream, in, out, rows, cols, rows)
+                        : launch_pdl_grid(lt_reduce_cols<DT, DT, KIND, 1>, dim3(gx, 1), RT, stream, in, out, rows, cols, rows);
         }
         const uint64_t rows_per = (rows + parts - 1) / parts;
-        cudaError_t e = launch_pdl_grid(lt_reduce_cols<DT, F64, KIND>, dim3(gx, parts), RT, stream, in, scratch, rows, cols, rows_per);
+        cudaError_t e = wide ? launch_pdl_grid(lt_reduce_cols<DT, F64, KIND, 4>, dim3(gx, parts), RT, stream, in, scratch, rows, cols, rows_per)
+                             : launch_pdl_grid(lt_reduce_cols<DT, F64, KIND, 1>, dim3(gx, parts), RT, stream, in, scratch, rows, cols, rows_per);
         if (e != cudaSuccess) return e;
         *launched = 2;
-        return launch_pdl_grid(lt_reduce_cols<F64, DT, KIND>, dim3(gx, 1), RT, stream, (const void *)scratch, out, (uint64_t)parts, cols,
-                               (uint64_t)parts);
+        // the partial results: binary64, 256-byte aligned scratch
+        return (cols % 4) == 0
+                   ? launch_pdl_grid(lt_reduce_cols<F64, DT, KIND, 4>, dim3(gx2, 1), RT, stream, (const void *)scratch, out, (uint64_t)parts, cols, (uint64_t)parts)
+                   : launch_pdl_grid(lt_reduce_cols<F64, DT, KIND, 1>, dim3(gx2, 1), RT, stream, (const void *)scratch, out, (uint64_t)parts, cols, (uint64_t)parts);
     }
     const uint64_t n = rows * cols;
     if (parts <= 1) {
@@ -171,7 +211,7 @@ unsigned lt_reduce_parts(int axis, uint64_t rows, uint64_t cols, int sm_count) {
     if (axis == 0) return 0;
     if (axis == 1) {
         // enough CTAs to fill the device a few times over, at least 64 rows each
-        const uint64_t gx = (cols + 31) / 32;
+        const uint64_t gx = (cols + 127) / 128;
         uint64_t want = ((uint64_t)sm_count * 8 + gx - 1) / gx;
         const uint64_t most = (rows + 63) / 64;
         if (want > most) want = most;
