@@ -102,7 +102,15 @@ typedef enum {
     /* reductions over every dimension but the last: [d0, .., dk, C] -> [1, .., 1, C]; float dtypes */
     LT_OP_COL_SUM = 53, LT_OP_COL_MAX = 54, LT_OP_COL_MIN = 55,
     /* reductions over every element -> rank 0; float dtypes */
-    LT_OP_ALL_SUM = 56, LT_OP_ALL_MAX = 57, LT_OP_ALL_MIN = 58
+    LT_OP_ALL_SUM = 56, LT_OP_ALL_MAX = 57, LT_OP_ALL_MIN = 58,
+    /* Shape operations as pure functions of their inputs (Section 4.4, Fig. 3: the IR has no aliasing; the view
+       calls below are built from these).  Any dtype.
+       RESHAPE: attrs = {rank, d0, ..}: same elements in row-major order under another shape.
+       NARROW: attrs = {dim, start, length}: the slice [start, start + length) along dim.
+       PERMUTE: attrs = {p0, .., p(rank-1)}: result dimension i is input dimension p_i.
+       UPDATE_SLICE: 2 inputs (base, update), attrs = {dim, start}: base with the slice of update's extent along
+       dim, starting at start, replaced by update -- the inverse of NARROW. */
+    LT_OP_RESHAPE = 60, LT_OP_NARROW = 61, LT_OP_PERMUTE = 62, LT_OP_UPDATE_SLICE = 63
 } lt_opcode;
 
 /*
@@ -140,6 +148,8 @@ typedef struct {
     uint64_t replays;            /* lt_replay calls that ran a plan                          */
     uint64_t launches_reduce;    /* reductions run as kernels of their own: over columns, over a whole tensor,
                                     over rows of more than 8192 elements outside a fused long-row kernel          */
+    uint64_t launches_view;      /* shape operations run as copy kernels (narrow, permute, update_slice, and
+                                    reshape where it is not folded into a program or a shared buffer)            */
     uint64_t allocator_calls;    /* calls of the allocator's alloc and free (or cudaMallocAsync /
                                     cudaFreeAsync); 0 over a span means every block came from and
                                     went back to the context's own pool of released blocks          */
@@ -232,6 +242,23 @@ lt_status lt_op(lt_ctx *ctx, int opcode, const lt_tensor *in, int n_in, const in
  * kernel that overwrites it, at the same element index, or by an earlier kernel.
  */
 lt_status lt_assign(lt_ctx *ctx, lt_tensor dst, lt_tensor src);
+
+/*
+ * Views (Section 4.4, "In-place operations on views").  The result shares its value with `t` the way a view shares
+ * storage in an eager framework, although the IR has no mutation:
+ *   - an in-place update of the view (lt_assign with the view as destination) records the forward sequence -- the
+ *     view's new computation -- and the backward sequence: the inverse of every view operation between it and its
+ *     base, applied in reverse order (RESHAPE back to the base's shape, PERMUTE with the inverse permutation,
+ *     UPDATE_SLICE for NARROW), which becomes the base's new computation (Fig. 3);
+ *   - an in-place update of the base is seen by its views: a view is derived again from the base's current
+ *     computation the next time it is used.
+ * Views of views work the same way, link by link.  Releasing the base leaves the view a tensor of its own.
+ * Shapes and argument ranges as for LT_OP_RESHAPE / LT_OP_NARROW / LT_OP_PERMUTE.  Reshaping materialised data
+ * shares the buffer; the other view operations copy at the next barrier.
+ */
+lt_status lt_view_reshape(lt_ctx *ctx, lt_tensor t, int rank, const int64_t *shape, lt_tensor *out);
+lt_status lt_view_narrow(lt_ctx *ctx, lt_tensor t, int dim, int64_t start, int64_t length, lt_tensor *out);
+lt_status lt_view_permute(lt_ctx *ctx, lt_tensor t, const int *perm, lt_tensor *out);
 
 /* UnregisterTensor: the handle dies; a pending computation nobody names is never run.
    lt_release_many releases `n` handles in one call (language bindings batch the handles their

@@ -62,6 +62,10 @@ def lib():
         _lib.orc_row_reduce.argtypes = [ctypes.c_char_p, P, P]
         _lib.orc_col_reduce.argtypes = [ctypes.c_char_p, P, P]
         _lib.orc_all_reduce.argtypes = [ctypes.c_char_p, P, P]
+        _lib.orc_reshape.argtypes = [P, P]
+        _lib.orc_narrow.argtypes = [P, ctypes.c_int, ctypes.c_int64, P]
+        _lib.orc_permute.argtypes = [P, ctypes.POINTER(ctypes.c_int), P]
+        _lib.orc_update_slice.argtypes = [P, P, ctypes.c_int, ctypes.c_int64, P]
         _lib.orc_set_threads.argtypes = [ctypes.c_int]
         _lib.orc_philox4x32_10.argtypes = [ctypes.POINTER(ctypes.c_uint32)] * 3
         _lib.orc_philox4x32_10.restype = None
@@ -81,20 +85,31 @@ def max_threads() -> int:
 
 
 class OTensor:
-    """A value of the eager oracle: a numpy array plus its dtype tag."""
+    """A value of the eager oracle: a numpy array plus its dtype tag.
 
-    __slots__ = ("array", "dtype")
+    A tensor made by one of the `view_*` calls holds a numpy view of its base's storage (`shares` is set on
+    both): in-place updates of either then write into that storage, which is numpy's own aliasing and not
+    something this module computes."""
 
-    def __init__(self, array: np.ndarray, dtype: str):
+    __slots__ = ("array", "dtype", "shares")
+
+    def __init__(self, array: np.ndarray, dtype: str, view: bool = False):
         assert array.dtype == _NP[dtype], (array.dtype, dtype)
-        self.array = np.ascontiguousarray(array)
+        self.array = array if view else np.ascontiguousarray(array)
         self.dtype = dtype
+        self.shares = view
 
     @property
     def shape(self):
         return tuple(self.array.shape)
 
     def _c(self) -> _Arr:
+        if not self.array.flags["C_CONTIGUOUS"]:
+            # an op reads a strided view: hand the C routine a dense copy (kept alive on the instance below)
+            dense = OTensor(np.ascontiguousarray(self.array), self.dtype)
+            a = dense._c()
+            a._keep = dense
+            return a
         a = _Arr()
         a.data = self.array.ctypes.data
         a.dtype = DTYPES[self.dtype]
@@ -206,6 +221,25 @@ class EagerOracle:
         elif name == "philox_bits":
             out = self._new(tuple(attrs["shape"]), "u32")
             self._check(L.orc_philox_bits(int(attrs["seed"]), int(attrs["offset"]), out._c()), name)
+        elif name == "reshape":
+            (a,) = inputs
+            out = self._new(tuple(attrs["shape"]), a.dtype)
+            self._check(L.orc_reshape(a._c(), out._c()), name)
+            out.array = out.array.reshape(tuple(attrs["shape"]))
+        elif name == "narrow":
+            (a,) = inputs
+            d = int(attrs["dim"])
+            out = self._new(a.shape[:d] + (int(attrs["length"]),) + a.shape[d + 1:], a.dtype)
+            self._check(L.orc_narrow(a._c(), d, int(attrs["start"]), out._c()), name)
+        elif name == "permute":
+            (a,) = inputs
+            perm = [int(p) for p in attrs["perm"]]
+            out = self._new(tuple(a.shape[p] for p in perm), a.dtype)
+            self._check(L.orc_permute(a._c(), (ctypes.c_int * len(perm))(*perm), out._c()), name)
+        elif name == "update_slice":
+            base, upd = inputs
+            out = self._new(base.shape, base.dtype)
+            self._check(L.orc_update_slice(base._c(), upd._c(), int(attrs["dim"]), int(attrs["start"]), out._c()), name)
         elif name in _REDUCE:
             (a,) = inputs
             out = self._new(a.shape[:-1] + (1,), a.dtype)
@@ -223,11 +257,36 @@ class EagerOracle:
             raise ValueError(f"unknown op {name!r}")
         return out
 
+    # -- views (paper Section 4.4): numpy views of the base's storage
+    def _own_storage(self, t: OTensor) -> None:
+        if not t.shares:
+            t.array = np.array(t.array, copy=True)  # storage no other value refers to
+            t.shares = True
+
+    def view_reshape(self, t: OTensor, shape) -> OTensor:
+        self._own_storage(t)
+        v = t.array.view()
+        v.shape = tuple(shape)  # raises instead of copying when the storage cannot be seen under that shape
+        return OTensor(v, t.dtype, view=True)
+
+    def view_narrow(self, t: OTensor, dim: int, start: int, length: int) -> OTensor:
+        self._own_storage(t)
+        index = [slice(None)] * t.array.ndim
+        index[dim] = slice(start, start + length)
+        return OTensor(t.array[tuple(index)], t.dtype, view=True)
+
+    def view_permute(self, t: OTensor, perm) -> OTensor:
+        self._own_storage(t)
+        return OTensor(np.transpose(t.array, tuple(perm)), t.dtype, view=True)
+
     # -- in-place update: the destination takes over the source's value (paper Section 4.3)
     def assign(self, dst: OTensor, src: OTensor) -> None:
         if dst.shape != src.shape or dst.dtype != src.dtype:
             raise ValueError("assign needs equal shape and dtype")
-        dst.array = src.array
+        if dst.shares:
+            dst.array[...] = src.array  # written into the storage its views (or its base) see
+        else:
+            dst.array = src.array
 
     def release(self, t) -> None:
         pass

@@ -478,6 +478,101 @@ int orc_all_reduce(const char *op, const orc_array *a, orc_array *out) {
     return ORC_OK;
 }
 
+/* ------------------------------------------------------------------ views */
+
+static size_t elem_size(int dt) { return dt == ORC_BF16 ? 2 : dt == ORC_U8 ? 1 : 4; }
+
+/* Row-major strides (in elements) of `a`. */
+static void strides_of(const orc_array *a, int64_t *st) {
+    int64_t s = 1;
+    for (int d = a->rank - 1; d >= 0; --d) {
+        st[d] = s;
+        s *= a->shape[d];
+    }
+}
+
+/* Coordinates of flat index i in an array of `rank` dimensions `shape`. */
+static void unravel(int64_t i, const int64_t *shape, int rank, int64_t *idx) {
+    for (int d = rank - 1; d >= 0; --d) {
+        idx[d] = shape[d] ? i % shape[d] : 0;
+        i = shape[d] ? i / shape[d] : 0;
+    }
+}
+
+/* out = a with another shape of the same element count; element order (row-major) is kept. */
+int orc_reshape(const orc_array *a, orc_array *out) {
+    if (a->dtype != out->dtype) return ORC_ERR_DTYPE;
+    if (numel(a) != numel(out)) return ORC_ERR_SHAPE;
+    memcpy(out->data, a->data, (size_t)numel(a) * elem_size(a->dtype));
+    return ORC_OK;
+}
+
+/* out[.., k, ..] = a[.., start + k, ..] along dimension `dim`; out's extent there is the slice length. */
+int orc_narrow(const orc_array *a, int dim, int64_t start, orc_array *out) {
+    if (a->dtype != out->dtype) return ORC_ERR_DTYPE;
+    if (a->rank != out->rank || dim < 0 || dim >= a->rank) return ORC_ERR_SHAPE;
+    for (int d = 0; d < a->rank; ++d)
+        if (d != dim && a->shape[d] != out->shape[d]) return ORC_ERR_SHAPE;
+    if (start < 0 || start + out->shape[dim] > a->shape[dim]) return ORC_ERR_SHAPE;
+    int64_t st[ORC_MAX_RANK], idx[ORC_MAX_RANK];
+    strides_of(a, st);
+    size_t es = elem_size(a->dtype);
+    int64_t n = numel(out);
+    for (int64_t i = 0; i < n; ++i) {
+        unravel(i, out->shape, out->rank, idx);
+        idx[dim] += start;
+        int64_t src = 0;
+        for (int d = 0; d < a->rank; ++d) src += idx[d] * st[d];
+        memcpy((char *)out->data + (size_t)i * es, (const char *)a->data + (size_t)src * es, es);
+    }
+    return ORC_OK;
+}
+
+/* out dimension i is a's dimension perm[i]: out[j0, j1, ..] = a[i0, i1, ..] with i[perm[k]] = j[k]. */
+int orc_permute(const orc_array *a, const int *perm, orc_array *out) {
+    if (a->dtype != out->dtype) return ORC_ERR_DTYPE;
+    if (a->rank != out->rank) return ORC_ERR_SHAPE;
+    int seen[ORC_MAX_RANK] = {0};
+    for (int k = 0; k < a->rank; ++k) {
+        if (perm[k] < 0 || perm[k] >= a->rank || seen[perm[k]]) return ORC_ERR_SHAPE;
+        seen[perm[k]] = 1;
+        if (out->shape[k] != a->shape[perm[k]]) return ORC_ERR_SHAPE;
+    }
+    int64_t st[ORC_MAX_RANK], idx[ORC_MAX_RANK];
+    strides_of(a, st);
+    size_t es = elem_size(a->dtype);
+    int64_t n = numel(out);
+    for (int64_t i = 0; i < n; ++i) {
+        unravel(i, out->shape, out->rank, idx);
+        int64_t src = 0;
+        for (int k = 0; k < a->rank; ++k) src += idx[k] * st[perm[k]];
+        memcpy((char *)out->data + (size_t)i * es, (const char *)a->data + (size_t)src * es, es);
+    }
+    return ORC_OK;
+}
+
+/* out = base with the slice [start, start + upd.shape[dim]) along `dim` replaced by upd. */
+int orc_update_slice(const orc_array *base, const orc_array *upd, int dim, int64_t start, orc_array *out) {
+    if (base->dtype != out->dtype || upd->dtype != out->dtype) return ORC_ERR_DTYPE;
+    if (!same_shape(base, out) || upd->rank != base->rank || dim < 0 || dim >= base->rank) return ORC_ERR_SHAPE;
+    for (int d = 0; d < base->rank; ++d)
+        if (d != dim && upd->shape[d] != base->shape[d]) return ORC_ERR_SHAPE;
+    if (start < 0 || start + upd->shape[dim] > base->shape[dim]) return ORC_ERR_SHAPE;
+    size_t es = elem_size(out->dtype);
+    memcpy(out->data, base->data, (size_t)numel(base) * es);
+    int64_t st[ORC_MAX_RANK], idx[ORC_MAX_RANK];
+    strides_of(out, st);
+    int64_t n = numel(upd);
+    for (int64_t i = 0; i < n; ++i) {
+        unravel(i, upd->shape, upd->rank, idx);
+        idx[dim] += start;
+        int64_t dst = 0;
+        for (int d = 0; d < out->rank; ++d) dst += idx[d] * st[d];
+        memcpy((char *)out->data + (size_t)dst * es, (const char *)upd->data + (size_t)i * es, es);
+    }
+    return ORC_OK;
+}
+
 /* ---------------------------------------------------------------- Philox */
 
 /*

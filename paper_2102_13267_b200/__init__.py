@@ -38,6 +38,7 @@ OPCODES = {
     "recip": 28, "square": 29, "sigmoid": 30, "gelu_tanh": 31, "not": 32,
     "convert": 40, "iota": 41, "philox_bits": 42, "row_sum": 50, "row_max": 51, "row_min": 52,
     "col_sum": 53, "col_max": 54, "col_min": 55, "all_sum": 56, "all_max": 57, "all_min": 58,
+    "reshape": 60, "narrow": 61, "permute": 62, "update_slice": 63,
 }
 STATUS_NAMES = ["LT_OK", "LT_ERR_INVALID_ARG", "LT_ERR_SHAPE", "LT_ERR_DTYPE", "LT_ERR_DEVICE",
                 "LT_ERR_UNSUPPORTED", "LT_ERR_OOM", "LT_ERR_CUDA", "LT_ERR_DEVICE_TIMEOUT"]
@@ -56,7 +57,7 @@ class lt_stats(ctypes.Structure):
         "launches_elementwise", "launches_row", "launches_multi", "bytes_planned",
         "outputs_donated", "outputs_allocated", "temporaries_allocated",
         "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind",
-        "launches_compiled", "replays", "launches_reduce", "allocator_calls")]
+        "launches_compiled", "replays", "launches_reduce", "launches_view", "allocator_calls")]
 
 
 class lt_kernel_timing(ctypes.Structure):
@@ -76,6 +77,9 @@ _SIGNATURES = {
     "lt_scalar_dynamic": [_vp, ctypes.c_double, _int, _P(_u64)],
     "lt_op": [_vp, _int, _P(_u64), _int, _P(_i64), _int, _P(_u64)],
     "lt_assign": [_vp, _u64, _u64],
+    "lt_view_reshape": [_vp, _u64, _int, _P(_i64), _P(_u64)],
+    "lt_view_narrow": [_vp, _u64, _int, _i64, _i64, _P(_u64)],
+    "lt_view_permute": [_vp, _u64, _P(_int), _P(_u64)],
     "lt_release": [_vp, _u64],
     "lt_release_many": [_vp, _P(_u64), ctypes.c_size_t],
     "lt_barrier": [_vp, _int],
@@ -312,6 +316,15 @@ class LazyContext:
         if attrs:
             if name == "convert":
                 a = [DTYPES[attrs["dtype"]]]
+            elif name == "reshape":
+                shp = tuple(attrs["shape"])
+                a = [len(shp), *shp]
+            elif name == "narrow":
+                a = [int(attrs["dim"]), int(attrs["start"]), int(attrs["length"])]
+            elif name == "permute":
+                a = [int(p) for p in attrs["perm"]]
+            elif name == "update_slice":
+                a = [int(attrs["dim"]), int(attrs["start"])]
             elif name == "iota":
                 shp = tuple(attrs["shape"])
                 a = [int(attrs["dim"]), len(shp), *shp]
@@ -337,6 +350,21 @@ class LazyContext:
 
     def is_materialised(self, t: LazyTensor) -> bool:
         return self._info(t.handle)[3]
+
+    # ---- views (paper Section 4.4): results that follow, and are followed by, in-place updates of their base
+    def view_reshape(self, t: LazyTensor, shape) -> LazyTensor:
+        shp = (_i64 * max(len(shape), 1))(*shape)
+        self._check(_lib.lt_view_reshape(self._ctx, t.handle, len(shape), shp, ctypes.byref(self._h)))
+        return LazyTensor(self, self._h.value, keep=t._keep)
+
+    def view_narrow(self, t: LazyTensor, dim: int, start: int, length: int) -> LazyTensor:
+        self._check(_lib.lt_view_narrow(self._ctx, t.handle, int(dim), int(start), int(length), ctypes.byref(self._h)))
+        return LazyTensor(self, self._h.value, keep=t._keep)
+
+    def view_permute(self, t: LazyTensor, perm) -> LazyTensor:
+        p = (_int * max(len(perm), 1))(*perm)
+        self._check(_lib.lt_view_permute(self._ctx, t.handle, p, ctypes.byref(self._h)))
+        return LazyTensor(self, self._h.value, keep=t._keep)
 
     def assign(self, dst: LazyTensor, src: LazyTensor) -> None:
         self._check(_lib.lt_assign(self._ctx, dst.handle, src.handle))

@@ -12,7 +12,7 @@ OBJ = HERE / "_build"
 LIB = HERE / "liblazytensor.so"
 CUDA_HOME = Path(os.environ.get("CUDA_HOME", "/usr/local/cuda"))
 
-CU_SOURCES = ["kernels.cu", "compiled.cu", "static_scratch.cu", "reduce.cu"]
+CU_SOURCES = ["kernels.cu", "compiled.cu", "static_scratch.cu", "reduce.cu", "views.cu"]
 CPP_SOURCES = ["engine.cpp", "canon.cpp", "planner.cpp", "executor.cpp"]
 HEADERS = ["engine.h", "vm.h", "launch.h", "vm_core.inc", "vm_ops.cuh", "compiled.h", "compiled_programs.inc", "pdl.cuh", "../../include/lazytensor.h"]
 

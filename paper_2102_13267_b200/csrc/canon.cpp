@@ -96,6 +96,7 @@ void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonica
         cn.dyn = -1;
         cn.sval = 0.0;
         cn.attr0 = 0;
+        cn.attr1 = 0;
         cn.output = -1;
         cn.arena = id;
         if (n.op == N_DEVICE_DATA) {
@@ -124,6 +125,9 @@ void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonica
             cg.dyn.push_back(v);
         } else if (n.op == LT_OP_CONVERT || n.op == LT_OP_IOTA) {
             cn.attr0 = n.attr[0];
+        } else if (n.op >= LT_OP_RESHAPE && n.op <= LT_OP_UPDATE_SLICE) {
+            cn.attr0 = n.attr[0];
+            cn.attr1 = n.attr[1];
         }
         cg.nodes.push_back(cn);
     };
@@ -199,6 +203,10 @@ void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonica
             for (int i = 0; i < n.n_in; ++i) put<uint32_t>(b, n.in[i]);
             if (n.op == LT_OP_PHILOX_BITS) put<int32_t>(b, n.dyn);
             if (n.op == LT_OP_CONVERT || n.op == LT_OP_IOTA) put<int64_t>(b, n.attr0);
+            if (n.op >= LT_OP_RESHAPE && n.op <= LT_OP_UPDATE_SLICE) {
+                put<int64_t>(b, n.attr0);
+                put<int64_t>(b, n.attr1);
+            }
         }
     }
     put<uint32_t>(b, (uint32_t)cg.outputs.size());

@@ -34,6 +34,8 @@ inline lt_tensor make_handle(const lt_ctx *c, uint32_t slot) {
     return ((uint64_t)c->tag << 48) | ((uint64_t)(c->tensors[slot].gen & 0xffffu) << 32) | (uint64_t)(slot + 1);
 }
 
+lt_status sync_view_of(lt_ctx *c, uint32_t slot);
+
 lt_status lookup(lt_ctx *c, lt_tensor h, uint32_t *slot) {
     if ((uint16_t)(h >> 48) != c->tag) return fail(c, LT_ERR_DEVICE, "tensor handle belongs to another context");
     uint32_t s = (uint32_t)(h & 0xffffffffu);
@@ -43,6 +45,7 @@ lt_status lookup(lt_ctx *c, lt_tensor h, uint32_t *slot) {
     if (!t.live || (t.gen & 0xffffu) != (uint32_t)((h >> 32) & 0xffffu))
         return fail(c, LT_ERR_INVALID_ARG, "tensor handle was released");
     *slot = s;
+    if (t.view_base != NONE) return sync_view_of(c, s);  // a view first catches up with its base
     return LT_OK;
 }
 
@@ -62,6 +65,10 @@ uint32_t tensor_new(lt_ctx *c, uint32_t node) {
     t.seq = c->next_seq++;
     t.live = true;
     t.queued = false;
+    t.view_base = NONE;
+    t.view_op = 0;
+    t.version = 0;
+    t.base_seen = 0;
     node_ref(c, node);
     c->nodes[node].tensor_refs++;
     return slot;
@@ -235,6 +242,8 @@ const char *op_name(int op) {
     case LT_OP_ROW_SUM: return "row_sum"; case LT_OP_ROW_MAX: return "row_max"; case LT_OP_ROW_MIN: return "row_min";
     case LT_OP_COL_SUM: return "col_sum"; case LT_OP_COL_MAX: return "col_max"; case LT_OP_COL_MIN: return "col_min";
     case LT_OP_ALL_SUM: return "all_sum"; case LT_OP_ALL_MAX: return "all_max"; case LT_OP_ALL_MIN: return "all_min";
+    case LT_OP_RESHAPE: return "reshape"; case LT_OP_NARROW: return "narrow"; case LT_OP_PERMUTE: return "permute";
+    case LT_OP_UPDATE_SLICE: return "update_slice";
     case N_DEVICE_DATA: return "device_data"; case N_SCALAR: return "constant";
     default: return "?";
     }
@@ -607,6 +616,213 @@ static bool scalar_fits(const Node &s, int dtype) {
     return v >= 0 && v <= 4294967295.0;
 }
 
+
+// ---- shape operations (pure IR nodes) and views (Section 4.4)
+
+static uint64_t pack_perm(const int *perm, int rank) {
+    uint64_t v = 0;
+    for (int i = 0; i < rank; ++i) v |= (uint64_t)(perm[i] & 0xf) << (4 * i);
+    return v;
+}
+
+// Appends the node `opcode`(src [, upd]) with the given attributes; shapes are validated here.  For RESHAPE of
+// materialised data no operation is recorded: the result is another leaf over the same buffer.
+static lt_status record_shape_op(lt_ctx *c, int opcode, uint32_t src, uint32_t upd, int64_t a0, int64_t a1, int rank,
+                                 const int64_t *dims, uint32_t *out_node) {
+    const Node s = c->nodes[src];  // copy: the arena may grow below
+    if (s.op == N_SCALAR) return fail(c, LT_ERR_INVALID_ARG, "shape operations need a tensor, not a constant");
+    int64_t od[LT_MAX_RANK] = {0};
+    int orank = s.rank;
+    if (opcode == LT_OP_RESHAPE) {
+        lt_status st = check_shape(c, rank, dims);
+        if (st) return st;
+        if (shape_numel(dims, rank) != shape_numel(s.dims, s.rank)) return fail(c, LT_ERR_SHAPE, "reshape must keep the number of elements");
+        orank = rank;
+        for (int i = 0; i < rank; ++i) od[i] = dims[i];
+        if (s.op == N_DEVICE_DATA) {
+            uint32_t n = node_new(c);
+            Node &nd = c->nodes[n];
+            nd.op = N_DEVICE_DATA;
+            nd.dtype = s.dtype;
+            nd.rank = (uint8_t)orank;
+            for (int i = 0; i < orank; ++i) nd.dims[i] = od[i];
+            nd.buffer = s.buffer;
+            c->buffers[s.buffer].refs++;
+            *out_node = n;
+            return LT_OK;
+        }
+    } else if (opcode == LT_OP_NARROW) {
+        const int64_t dim = a0, start = a1, len = rank;  // (length travels in `rank`)
+        if (dim < 0 || dim >= s.rank) return fail(c, LT_ERR_INVALID_ARG, "narrow: dimension out of range");
+        if (start < 0 || len < 1 || start + len > s.dims[dim]) return fail(c, LT_ERR_SHAPE, "narrow: slice outside the dimension");
+        memcpy(od, s.dims, sizeof(od));
+        od[dim] = len;
+    } else if (opcode == LT_OP_PERMUTE) {
+        bool seen[LT_MAX_RANK] = {false};
+        for (int i = 0; i < s.rank; ++i) {
+            const int p = (int)((a0 >> (4 * i)) & 0xf);
+            if (p >= s.rank || seen[p]) return fail(c, LT_ERR_INVALID_ARG, "permute: not a permutation of the dimensions");
+            seen[p] = true;
+            od[i] = s.dims[p];
+        }
+    } else {  // UPDATE_SLICE
+        const Node &u = c->nodes[upd];
+        const int64_t dim = a0, start = a1;
+        if (u.op == N_SCALAR || u.dtype != s.dtype || u.rank != s.rank) return fail(c, LT_ERR_SHAPE, "update_slice: update must match the base's dtype and rank");
+        if (dim < 0 || dim >= s.rank) return fail(c, LT_ERR_INVALID_ARG, "update_slice: dimension out of range");
+        for (int i = 0; i < s.rank; ++i)
+            if (i != dim && u.dims[i] != s.dims[i]) return fail(c, LT_ERR_SHAPE, "update_slice: update must match the base outside the sliced dimension");
+        if (start < 0 || start + u.dims[dim] > s.dims[dim]) return fail(c, LT_ERR_SHAPE, "update_slice: slice outside the dimension");
+        memcpy(od, s.dims, sizeof(od));
+    }
+    uint32_t n = node_new(c);
+    Node &nd = c->nodes[n];
+    nd.op = (uint16_t)opcode;
+    nd.dtype = s.dtype;
+    nd.rank = (uint8_t)orank;
+    for (int i = 0; i < orank; ++i) nd.dims[i] = od[i];
+    nd.attr[0] = a0;
+    nd.attr[1] = a1;
+    nd.n_in = opcode == LT_OP_UPDATE_SLICE ? 2 : 1;
+    nd.in[0] = src;
+    node_ref(c, src);
+    if (opcode == LT_OP_UPDATE_SLICE) {
+        nd.in[1] = upd;
+        node_ref(c, upd);
+    }
+    c->stats.nodes_recorded++;
+    *out_node = n;
+    return LT_OK;
+}
+
+// `slot` from now on denotes the computation `node` (the core of lt_assign).
+static void repoint_tensor(lt_ctx *c, uint32_t slot, uint32_t node, bool keep_donor) {
+    TensorRec &d = c->tensors[slot];
+    if (d.node == node) return;
+    const Node &dn = c->nodes[d.node];
+    if (keep_donor && dn.op == N_DEVICE_DATA && dn.buffer != NONE) {
+        if (d.donor != NONE) buffer_unref(c, d.donor);
+        d.donor = dn.buffer;
+        c->buffers[d.donor].refs++;
+    }
+    const uint32_t old = d.node;
+    d.node = node;
+    node_ref(c, node);
+    c->nodes[node].tensor_refs++;
+    c->nodes[old].tensor_refs--;
+    node_unref(c, old);
+    queue_pending(c, slot);
+}
+
+static bool view_base_alive(const lt_ctx *c, const TensorRec &t) {
+    return t.view_base != NONE && t.view_base < c->tensors.size() && c->tensors[t.view_base].live &&
+           c->tensors[t.view_base].gen == t.view_base_gen;
+}
+
+// the view operation of tensor `t` applied to `src`
+static lt_status apply_view_op(lt_ctx *c, const TensorRec &t, uint32_t src, uint32_t *out_node) {
+    const Node &cur = c->nodes[t.node];  // the view's shape does not change
+    if (t.view_op == LT_OP_RESHAPE) {
+        int64_t dims[LT_MAX_RANK];
+        memcpy(dims, cur.dims, sizeof(dims));
+        return record_shape_op(c, LT_OP_RESHAPE, src, NONE, 0, 0, cur.rank, dims, out_node);
+    }
+    if (t.view_op == LT_OP_NARROW) return record_shape_op(c, LT_OP_NARROW, src, NONE, t.view_a0, t.view_a1, (int)cur.dims[t.view_a0], nullptr, out_node);
+    return record_shape_op(c, LT_OP_PERMUTE, src, NONE, t.view_a0, 0, 0, nullptr, out_node);
+}
+
+// A view follows its base: if the base has been updated in place since the view's computation was derived, derive
+// it again from the base's current computation (the base is brought up to date first when it is a view itself).
+static lt_status sync_view(lt_ctx *c, uint32_t slot) {
+    TensorRec &t0 = c->tensors[slot];
+    if (t0.view_base == NONE) return LT_OK;
+    if (!view_base_alive(c, t0)) {
+        t0.view_base = NONE;  // the base is gone: a tensor of its own from here on
+        return LT_OK;
+    }
+    const uint32_t b = t0.view_base;
+    lt_status st = sync_view(c, b);
+    if (st) return st;
+    if (c->tensors[b].version == c->tensors[slot].base_seen) return LT_OK;
+    uint32_t n = NONE;
+    st = apply_view_op(c, c->tensors[slot], c->tensors[b].node, &n);
+    if (st) return st;
+    c->nodes[n].refs++;  // held across the repointing
+    repoint_tensor(c, slot, n, false);
+    node_unref(c, n);
+    TensorRec &t = c->tensors[slot];
+    t.base_seen = c->tensors[b].version;
+    t.version++;
+    return LT_OK;
+}
+
+// An in-place update of a view (Section 4.4): the backward sequence.  Starting from the updated value of the view,
+// the inverse of each view operation gives the updated value of the next base up the chain.
+static lt_status propagate_to_bases(lt_ctx *c, uint32_t slot) {
+    uint32_t cur = slot;
+    while (c->tensors[cur].view_base != NONE) {
+        if (!view_base_alive(c, c->tensors[cur])) {
+            c->tensors[cur].view_base = NONE;
+            break;
+        }
+        const uint32_t b = c->tensors[cur].view_base;
+        lt_status st = sync_view(c, b);
+        if (st) return st;
+        const TensorRec &t = c->tensors[cur];
+        const Node base_node = c->nodes[c->tensors[b].node];
+        uint32_t inv = NONE;
+        if (t.view_op == LT_OP_RESHAPE) {
+            int64_t dims[LT_MAX_RANK];
+            memcpy(dims, base_node.dims, sizeof(dims));
+            st = record_shape_op(c, LT_OP_RESHAPE, t.node, NONE, 0, 0, base_node.rank, dims, &inv);
+        } else if (t.view_op == LT_OP_PERMUTE) {
+            int inverse[LT_MAX_RANK] = {0};
+            for (int i = 0; i < base_node.rank; ++i) inverse[(t.view_a0 >> (4 * i)) & 0xf] = i;
+            st = record_shape_op(c, LT_OP_PERMUTE, t.node, NONE, (int64_t)pack_perm(inverse, base_node.rank), 0, 0, nullptr, &inv);
+        } else {
+            st = record_shape_op(c, LT_OP_UPDATE_SLICE, c->tensors[b].node, t.node, t.view_a0, t.view_a1, 0, nullptr, &inv);
+        }
+        if (st) return st;
+        c->nodes[inv].refs++;
+        repoint_tensor(c, b, inv, true);
+        node_unref(c, inv);
+        c->tensors[b].version++;
+        c->tensors[cur].base_seen = c->tensors[b].version;  // this view is what the base was updated from
+        cur = b;
+    }
+    return LT_OK;
+}
+
+static lt_status make_view(lt_ctx *c, lt_tensor t, int opcode, int64_t a0, int64_t a1, int rank, const int64_t *dims, lt_tensor *out) {
+    if (!c || !out) return LT_ERR_INVALID_ARG;
+    Timer tm(c->stats.ns_record);
+    uint32_t bs;
+    lt_status st = lookup(c, t, &bs);
+    if (st) return st;
+    uint32_t n = NONE;
+    st = record_shape_op(c, opcode, c->tensors[bs].node, NONE, a0, a1, rank, dims, &n);
+    if (st) return st;
+    const uint32_t slot = tensor_new(c, n);
+    TensorRec &v = c->tensors[slot];
+    const TensorRec &b = c->tensors[bs];
+    v.view_base = bs;
+    v.view_base_gen = b.gen;
+    v.view_op = (uint16_t)opcode;
+    v.view_a0 = a0;
+    v.view_a1 = a1;
+    v.base_seen = b.version;
+    c->view_slots.push_back(slot);
+    if (c->nodes[n].op != N_DEVICE_DATA) queue_pending(c, slot);
+    *out = make_handle(c, slot);
+    return LT_OK;
+}
+
+}  // extern "C"
+namespace {
+lt_status sync_view_of(lt_ctx *c, uint32_t slot) { return sync_view(c, slot); }
+}
+extern "C" {
+
 lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int64_t *attrs, int n_attrs,
                 lt_tensor *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
@@ -647,6 +863,42 @@ lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int6
         return true;
     };
 
+    if (opcode >= LT_OP_RESHAPE && opcode <= LT_OP_UPDATE_SLICE) {
+        if (n_in < 1) return fail(c, LT_ERR_INVALID_ARG, std::string(op_name(opcode)) + ": wrong number of inputs or attributes");
+        const Node &src = c->nodes[ids[0]];
+        int64_t a0 = 0, a1 = 0;
+        int rank = 0;
+        const int64_t *dims = nullptr;
+        bool ok = false;
+        if (opcode == LT_OP_RESHAPE) {
+            ok = n_in == 1 && n_attrs >= 1 && attrs[0] >= 0 && attrs[0] <= LT_MAX_RANK && n_attrs == 1 + attrs[0];
+            if (ok) rank = (int)attrs[0], dims = attrs + 1;
+        } else if (opcode == LT_OP_NARROW) {
+            ok = n_in == 1 && n_attrs == 3 && attrs[2] <= 0x7fffffffLL;
+            if (ok) a0 = attrs[0], a1 = attrs[1], rank = (int)attrs[2];
+        } else if (opcode == LT_OP_PERMUTE) {
+            ok = n_in == 1 && n_attrs == src.rank;
+            if (ok) {
+                int perm[LT_MAX_RANK];
+                for (int i = 0; i < n_attrs; ++i) {
+                    if (attrs[i] < 0 || attrs[i] >= src.rank) return fail(c, LT_ERR_INVALID_ARG, "permute: not a permutation of the dimensions");
+                    perm[i] = (int)attrs[i];
+                }
+                a0 = (int64_t)pack_perm(perm, n_attrs);
+            }
+        } else {
+            ok = n_in == 2 && n_attrs == 2;
+            if (ok) a0 = attrs[0], a1 = attrs[1];
+        }
+        if (!ok) return fail(c, LT_ERR_INVALID_ARG, std::string(op_name(opcode)) + ": wrong number of inputs or attributes");
+        uint32_t n = NONE;
+        lt_status st = record_shape_op(c, opcode, ids[0], ids[1], a0, a1, rank, dims, &n);
+        if (st) return st;
+        const uint32_t slot = tensor_new(c, n);
+        if (c->nodes[n].op != N_DEVICE_DATA) queue_pending(c, slot);
+        *out = make_handle(c, slot);
+        return LT_OK;
+    }
     const bool is_binary = opcode >= LT_OP_ADD && opcode <= LT_OP_XOR;
     const bool is_compare = opcode >= LT_OP_GT && opcode <= LT_OP_NE;
     const bool is_unary = opcode >= LT_OP_NEG && opcode <= LT_OP_NOT;
@@ -784,19 +1036,31 @@ lt_status lt_assign(lt_ctx *c, lt_tensor dst, lt_tensor src) {
     if (!same) return fail(c, LT_ERR_SHAPE, "lt_assign needs equal shape and dtype");
     // Section 4.3: the destination's computation is replaced by the source's; the buffer it
     // named is remembered so the barrier can write the new value in place.
-    if (dn.op == N_DEVICE_DATA && dn.buffer != NONE) {
-        if (d.donor != NONE) buffer_unref(c, d.donor);
-        d.donor = dn.buffer;
-        c->buffers[d.donor].refs++;
-    }
-    uint32_t old = d.node;
-    d.node = sr.node;
-    node_ref(c, d.node);
-    c->nodes[d.node].tensor_refs++;
-    c->nodes[old].tensor_refs--;
-    node_unref(c, old);
-    queue_pending(c, ds);
+    repoint_tensor(c, ds, sr.node, true);
+    c->tensors[ds].version++;
+    // Section 4.4: an update of a view also updates what it is a view of
+    if (c->tensors[ds].view_base != NONE) return propagate_to_bases(c, ds);
     return LT_OK;
+}
+
+lt_status lt_view_reshape(lt_ctx *c, lt_tensor t, int rank, const int64_t *shape, lt_tensor *out) {
+    return make_view(c, t, LT_OP_RESHAPE, 0, 0, rank, shape, out);
+}
+
+lt_status lt_view_narrow(lt_ctx *c, lt_tensor t, int dim, int64_t start, int64_t length, lt_tensor *out) {
+    if (length < 1 || length > 0x7fffffffLL) return c ? fail(c, LT_ERR_SHAPE, "narrow: slice outside the dimension") : LT_ERR_INVALID_ARG;
+    return make_view(c, t, LT_OP_NARROW, dim, start, (int)length, nullptr, out);
+}
+
+lt_status lt_view_permute(lt_ctx *c, lt_tensor t, const int *perm, lt_tensor *out) {
+    if (!c || !perm) return LT_ERR_INVALID_ARG;
+    uint32_t bs;
+    lt_status st = lookup(c, t, &bs);
+    if (st) return st;
+    const int rank = c->nodes[c->tensors[bs].node].rank;
+    for (int i = 0; i < rank; ++i)
+        if (perm[i] < 0 || perm[i] >= rank) return fail(c, LT_ERR_INVALID_ARG, "permute: not a permutation of the dimensions");
+    return make_view(c, t, LT_OP_PERMUTE, (int64_t)pack_perm(perm, rank), 0, 0, nullptr, out);
 }
 
 lt_status lt_release(lt_ctx *c, lt_tensor t) {
@@ -834,6 +1098,18 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
     if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
     std::vector<uint32_t> &roots = c->roots_scratch;
     Canonical &cg = c->canon;
+    if (!c->view_slots.empty()) {
+        // live views catch up with in-place updates of their bases before the graph is closed
+        size_t w = 0;
+        for (size_t k = 0; k < c->view_slots.size(); ++k) {
+            const uint32_t slot = c->view_slots[k];
+            if (slot >= c->tensors.size() || !c->tensors[slot].live || c->tensors[slot].view_base == NONE) continue;
+            lt_status st = sync_view_of(c, slot);
+            if (st) return st;
+            if (c->tensors[slot].view_base != NONE) c->view_slots[w++] = slot;
+        }
+        c->view_slots.resize(w);
+    }
     {
         Timer tm(c->stats.ns_canonicalise);
         gather_roots(c, roots, false);
@@ -1226,6 +1502,12 @@ lt_status lt_dump_ir(lt_ctx *c, char *buf, size_t cap, size_t *need) {
             }
             if (n.op == LT_OP_CONVERT) s += std::string(", dtype=") + dtype_name((int)n.attr0);
             if (n.op == LT_OP_IOTA) s += ", dim=" + std::to_string(n.attr0);
+            if (n.op == LT_OP_NARROW || n.op == LT_OP_UPDATE_SLICE) s += ", dim=" + std::to_string(n.attr0) + ", start=" + std::to_string(n.attr1);
+            if (n.op == LT_OP_PERMUTE) {
+                s += ", dims=(";
+                for (int k = 0; k < n.rank; ++k) s += (k ? ", " : "") + std::to_string((n.attr0 >> (4 * k)) & 0xf);
+                s += ")";
+            }
             if (n.output >= 0) s += ", ROOT=" + std::to_string(n.output);
             s += "\n";
         }

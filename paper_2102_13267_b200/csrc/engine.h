@@ -50,6 +50,13 @@ struct TensorRec {
     uint64_t seq = 0;       // creation order
     bool live = false;
     bool queued = false;    // already in the pending list
+    // Views (Section 4.4): the tensor this one is a view of, the view operation, and how far it has followed the
+    // base's in-place updates.
+    uint32_t view_base = NONE, view_base_gen = 0;
+    uint16_t view_op = 0;           // LT_OP_RESHAPE / NARROW / PERMUTE
+    int64_t view_a0 = 0, view_a1 = 0;
+    uint64_t version = 0;           // in-place updates this tensor has received
+    uint64_t base_seen = 0;         // version of the base its current computation was derived from
 };
 
 // ---------------------------------------------------------------- canonical form
@@ -61,7 +68,8 @@ struct CNode {
     int32_t param;   // N_DEVICE_DATA: parameter ordinal
     int32_t dyn;     // first run-time slot (scalar: 1 slot; philox: 2 slots), else -1
     double sval;     // static scalar value
-    int64_t attr0;   // CONVERT dtype / IOTA dim
+    int64_t attr0;   // CONVERT dtype / IOTA dim / NARROW, UPDATE_SLICE dim / PERMUTE packed permutation
+    int64_t attr1;   // NARROW, UPDATE_SLICE start
     int32_t output;  // index in the output list, else -1
     uint32_t arena;  // arena node (not part of the hashed bytes)
 };
@@ -102,7 +110,7 @@ struct IoRef {
     uint32_t cnode;   // canonical node the slot carries
 };
 
-enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2, K_RED = 3 };  // K_RED: a reduction that runs as a kernel of its own (reduce.cu)
+enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2, K_RED = 3, K_VIEW = 4 };  // K_RED: a reduction that runs as a kernel of its own (reduce.cu); K_VIEW: a shape operation (views.cu)
 
 struct Group {
     uint8_t kind = K_EW;
@@ -119,6 +127,10 @@ struct Group {
     uint8_t red_axis = 0;           // K_RED: 0 rows, 1 columns, 2 everything
     uint8_t red_kind = 0;           // K_RED: 0 sum, 1 max, 2 min
     int32_t scratch_temp = -1;      // K_RED: temporary that holds the partial results, or -1
+    uint16_t view_op = 0;           // K_VIEW: LT_OP_RESHAPE / NARROW / PERMUTE / UPDATE_SLICE
+    uint8_t view_rank = 0;
+    int64_t view_a0 = 0, view_a1 = 0;
+    int64_t view_in_dims[LT_MAX_RANK] = {0}, view_out_dims[LT_MAX_RANK] = {0};  // of the (first) input and of the result
 };
 
 struct Launch {
@@ -220,6 +232,7 @@ struct lt_ctx {
     std::vector<lt::TensorRec> tensors;
     std::vector<uint32_t> free_tensors;
     std::vector<uint32_t> pending;  // tensor slots that may have pending IR
+    std::vector<uint32_t> view_slots;  // tensor slots that are (or were) views
     uint64_t next_seq = 1;
     uint32_t stamp = 0;
 

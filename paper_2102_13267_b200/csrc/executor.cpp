@@ -194,7 +194,23 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
             ev0 = take_event(c);
             ev1 = take_event(c);
         }
-        if (L.kind == K_RED) {
+        if (L.kind == K_VIEW) {
+            const Group &g = plan.groups[L.groups[0]];
+            unsigned launched = 1;
+            if (!dry) {
+                const IoRef &res = g.io.back();
+                const bool upd = g.view_op == LT_OP_UPDATE_SLICE;
+                const bool in_place = upd && res.kind == IO_OUTPUT && plan.outputs[res.index].donated_param >= 0 &&
+                                      resolve(res) == resolve(g.io[0]);
+                if (ev0) cudaEventRecord(ev0, c->stream);
+                e = lt_launch_view(g.view_op, (int)dtype_size(res.dtype), g.view_rank, g.view_in_dims, g.view_out_dims, g.view_a0, g.view_a1,
+                                   (const void *)(uintptr_t)resolve(g.io[0]), upd ? (const void *)(uintptr_t)resolve(g.io[1]) : nullptr,
+                                   (void *)(uintptr_t)resolve(res), in_place ? 1 : 0, c->sm_count, c->stream, &launched);
+                if (ev1) cudaEventRecord(ev1, c->stream);
+            }
+            c->stats.launches_view += 1;
+            if (launched > 1) c->stats.kernels_launched += launched - 1;
+        } else if (L.kind == K_RED) {
             const Group &g = plan.groups[L.groups[0]];
             unsigned launched = 1;
             if (!dry) {
@@ -452,7 +468,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                 c->stats.launches_row++;
             }
         }
-        if (ev0) c->timed.push_back(TimedLaunch{ev0, ev1, (uint8_t)(L.kind == K_RED ? K_ROW : L.kind), L.bytes});
+        if (ev0) c->timed.push_back(TimedLaunch{ev0, ev1, (uint8_t)(L.kind == K_RED ? K_ROW : L.kind == K_VIEW ? K_EW : L.kind), L.bytes});
         if (e != cudaSuccess) {
             release_all(true);
             return fail(c, LT_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e));

@@ -31,3 +31,10 @@ cudaError_t lt_static_scratch_clear_enqueue(void *base, size_t bytes, int sm_cou
 size_t lt_reduce_scratch_bytes(int axis, uint64_t rows, uint64_t cols, int sm_count);
 cudaError_t lt_launch_reduce(int axis, int kind, int dtype, const void *in, void *out, void *scratch, uint64_t rows, uint64_t cols,
                              int sm_count, cudaStream_t stream, unsigned *launched);
+
+// views.cu: copy kernels of the shape operations.  `op` is the lt_opcode (reshape 60, narrow 61, permute 62,
+// update_slice 63); in_dims is the (first) input's shape (reshape: {numel}), out_dims the result's (update_slice:
+// the update's); a0 / a1 as recorded (dimension and start; packed permutation).  `in_place` non-zero: update_slice
+// whose result already holds the base.  *launched receives the number of kernels enqueued.
+cudaError_t lt_launch_view(int op, int elem_bytes, int rank, const int64_t *in_dims, const int64_t *out_dims, int64_t a0, int64_t a1,
+                           const void *in, const void *upd, void *out, int in_place, int sm_count, cudaStream_t stream, unsigned *launched);

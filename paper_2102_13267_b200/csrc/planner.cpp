@@ -33,6 +33,7 @@ struct PNode {
 inline bool is_reduce(uint16_t op) { return op >= LT_OP_ROW_SUM && op <= LT_OP_ROW_MIN; }
 inline bool is_col_reduce(uint16_t op) { return op >= LT_OP_COL_SUM && op <= LT_OP_COL_MIN; }
 inline bool is_all_reduce(uint16_t op) { return op >= LT_OP_ALL_SUM && op <= LT_OP_ALL_MIN; }
+inline bool is_shape_op(uint16_t op) { return op >= LT_OP_RESHAPE && op <= LT_OP_UPDATE_SLICE; }
 constexpr uint64_t MAX_RESIDENT_COLS = (uint64_t)LT_VM_V * 1024;  // longest row a thread group keeps in registers
 inline bool is_factory(uint16_t op) { return op == LT_OP_IOTA || op == LT_OP_PHILOX_BITS; }
 inline bool is_float(uint8_t dt) { return dt == LT_F32 || dt == LT_BF16; }
@@ -312,7 +313,7 @@ struct CodeGen {
             if (tainted[rep_or_self(cn.in[i])] || tainted[cn.in[i]]) tainted[n] = 1;
         if (approx_sensitive(op)) tainted[n] = 1;
 
-        if (op == LT_OP_CONVERT && convert_is_alias(cg.nodes[cn.in[0]].dtype, cn.dtype)) {
+        if ((op == LT_OP_CONVERT && convert_is_alias(cg.nodes[cn.in[0]].dtype, cn.dtype)) || op == LT_OP_RESHAPE) {
             int x = rep_or_self(cn.in[0]);
             if (cg.nodes[cn.in[0]].op == N_SCALAR) { ok = false; return; }
             rep[n] = x;
@@ -716,6 +717,13 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
         if (pn[i].numel == 0) return fail(c, LT_ERR_UNSUPPORTED, "empty tensors cannot be part of a flushed graph");
     }
 
+    for (size_t i = 0; i < N; ++i) {
+        const CNode &n = cg.nodes[i];
+        if (!is_shape_op(n.op)) continue;
+        const PNode &src = pn[n.in[0]];
+        const bool same_domain = n.op == LT_OP_RESHAPE && src.rows == pn[i].rows && src.cols == pn[i].cols;
+        pn[i].foreign = !(same_domain && fuse);
+    }
     if (isolate_long_rows)
         for (size_t i = 0; i < N; ++i)
             if (pn[i].reduce && pn[cg.nodes[i].in[0]].cols > MAX_RESIDENT_COLS) pn[i].foreign = true;
@@ -777,7 +785,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             dr = pn[n.in[0]].rows;
             dc = pn[n.in[0]].cols;
         }
-        if (p.foreign) {
+        if (p.foreign && !is_shape_op(n.op)) {
             dr = pn[n.in[0]].rows;
             dc = pn[n.in[0]].cols;
         }
@@ -788,7 +796,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
         if (fuse && !p.foreign) {
             auto joinable = [&](int gi) -> bool {
                 const Group &g = groups[gi];
-                if (g.kind == K_RED || (int)g.members.size() >= MAX_GROUP_NODES) return false;
+                if (g.kind >= K_RED || (int)g.members.size() >= MAX_GROUP_NODES) return false;
                 if (g.rows == dr && g.cols == dc) return true;
                 // an [R,1] computation on row scalars of a wider group stays with that group
                 if (!p.reduce && p.cols == 1 && p.rows == g.rows && g.cols > 1) {
@@ -806,7 +814,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                     if (a == target || a < 0) continue;
                     Group &ga = groups[a];
                     Group &gb = groups[target];
-                    if (ga.kind == K_RED || ga.rows != gb.rows || ga.cols != gb.cols) continue;
+                    if (ga.kind >= K_RED || ga.rows != gb.rows || ga.cols != gb.cols) continue;
                     if (ga.members.size() + gb.members.size() >= (size_t)MAX_GROUP_NODES) continue;
                     bool legal = true;
                     for (uint32_t m : ga.members) {
@@ -833,7 +841,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                 const int lo = std::max(gmin + 1, (int)groups.size() - 8);
                 for (int gi = (int)groups.size() - 1; gi >= lo && target < 0; --gi) {
                     const Group &g = groups[gi];
-                    if (g.kind == K_RED || g.rows != dr || g.cols != dc || (int)g.members.size() >= MAX_GROUP_NODES) continue;
+                    if (g.kind >= K_RED || g.rows != dr || g.cols != dc || (int)g.members.size() >= MAX_GROUP_NODES) continue;
                     for (int k = 0; k < n.n_in && target < 0; ++k) {
                         const uint32_t o = n.in[k];
                         if (cg.nodes[o].op != N_DEVICE_DATA) continue;
@@ -851,7 +859,21 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             target = (int)groups.size() - 1;
             groups[target].rows = dr;
             groups[target].cols = dc;
-            if (p.foreign) {
+            if (p.foreign && is_shape_op(n.op)) {
+                Group &g = groups[target];
+                g.kind = K_VIEW;
+                g.rows = p.rows;  // the result's own domain
+                g.cols = p.cols;
+                g.view_op = n.op;
+                g.view_a0 = n.attr0;
+                g.view_a1 = n.attr1;
+                const CNode &src = cg.nodes[n.in[0]];
+                g.view_rank = src.rank;
+                memcpy(g.view_in_dims, src.dims, sizeof(g.view_in_dims));
+                memcpy(g.view_out_dims, n.dims, sizeof(g.view_out_dims));
+                if (n.op == LT_OP_UPDATE_SLICE) memcpy(g.view_out_dims, cg.nodes[n.in[1]].dims, sizeof(g.view_out_dims));  // the slice's extent
+                if (n.op == LT_OP_RESHAPE) g.view_rank = 1, g.view_in_dims[0] = g.view_out_dims[0] = (int64_t)p.numel;
+            } else if (p.foreign) {
                 Group &g = groups[target];
                 g.kind = K_RED;
                 g.red_axis = is_col_reduce(n.op) ? 1 : (is_all_reduce(n.op) ? 2 : 0);
@@ -899,6 +921,31 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                         else if (pn[q].group != (int)gi) pn[m].needs_store = true;
                     }
                 }
+            }
+            if (g.kind == K_VIEW) {
+                // a copy kernel: the inputs in order, then the result; all dense buffers
+                const uint32_t m = g.members[0];
+                pn[m].needs_store = true;
+                g.ins.clear();
+                g.io.clear();
+                g.imms.clear();
+                auto slot_for = [&](uint32_t v, bool store) {
+                    const CNode &vn = cg.nodes[v];
+                    IoRef io;
+                    io.is_store = store ? 1 : 0;
+                    io.dtype = vn.dtype;
+                    io.cls = LT_CLS_FULL;
+                    io.cnode = v;
+                    if (vn.op == N_DEVICE_DATA) io.kind = IO_PARAM, io.index = (uint32_t)vn.param;
+                    else if (vn.output >= 0) io.kind = IO_OUTPUT, io.index = (uint32_t)vn.output;
+                    else io.kind = IO_TEMP, io.index = 0;
+                    g.io.push_back(io);
+                };
+                for (int k = 0; k < cg.nodes[m].n_in; ++k) slot_for(cg.nodes[m].in[k], false);
+                slot_for(m, true);
+                g.flavour = 1;
+                for (uint32_t nn : emit) in_emit[nn] = 0;
+                break;
             }
             if (g.kind == K_RED) {
                 // a kernel of its own: slot 0 = the input, slot 1 = the result; no register program
@@ -991,6 +1038,10 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
         }
         g.bytes = 0;
         for (const IoRef &io : g.io) g.bytes += io_bytes(g, io);
+        if (g.kind == K_VIEW) {
+            g.bytes = 0;
+            for (const IoRef &io : g.io) g.bytes += pn[io.cnode].numel * dtype_size(io.dtype);
+        }
         if (g.kind == K_RED) {
             const size_t scratch = lt_reduce_scratch_bytes(g.red_axis, g.rows, g.cols, c->sm_count);
             if (scratch) {
@@ -1114,7 +1165,11 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                 bool safe = true;
                 for (auto &rd : readers[p]) {
                     const uint32_t rg = rd.first;
-                    if (rg == gi) {
+                    if (rg == gi && g.kind == K_VIEW) {
+                        // update_slice rewrites only the slice of its base: in place when the base (slot 0) is the one
+                        // read of the buffer; the other shape operations move every element
+                        if (g.view_op != LT_OP_UPDATE_SLICE || rd.second != 0) { safe = false; break; }
+                    } else if (rg == gi) {
                         const IoRef &ld = groups[rg].io[rd.second];
                         if (ld.cls != LT_CLS_FULL) { safe = false; break; }
                         // the load must come before the store in program order
@@ -1159,7 +1214,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             }
             P.super_prefix[L.groups.size()] = acc;
             P.total_super = acc;
-        } else if (L.kind != K_RED) {
+        } else if (L.kind < K_RED) {
             L.kp.reset(new LtKParams());
             LtKParams &P = *L.kp;
             memset(&P, 0, sizeof(P));
@@ -1192,7 +1247,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
     bool unfused_long_row = false;
     for (Launch &L : plan.launches) {
         const Group &g = groups[L.groups[0]];
-        if (L.kind == K_RED) continue;
+        if (L.kind >= K_RED) continue;
         uint8_t dt[LT_VM_MAX_PTR] = {0}, cl[LT_VM_MAX_PTR] = {0};
         for (size_t s = 0; s < g.io.size() && s < LT_VM_MAX_PTR; ++s) {
             dt[s] = g.io[s].dtype;
@@ -1226,7 +1281,7 @@ std::string describe_plan(const Plan &plan) {
             snprintf(buf, sizeof(buf), "  output %zu donated param %d\n", k, plan.outputs[k].donated_param);
             s += buf;
         }
-    static const char *kind[] = {"elementwise", "row", "multi", "reduce"};
+    static const char *kind[] = {"elementwise", "row", "multi", "reduce", "view"};
     static const char *cls[] = {"full", "colvec", "rowvec", "scalar"};
     static const char *iok[] = {"param", "output", "temp"};
     for (size_t li = 0; li < plan.launches.size(); ++li) {
@@ -1236,7 +1291,10 @@ std::string describe_plan(const Plan &plan) {
                  L.flavour == 0 ? "fast" : (L.flavour == 1 ? "precise" : "ieee"), L.groups.size(), (unsigned long long)g.rows, (unsigned long long)g.cols,
                  g.rowcol ? "rowcol" : "flat", (unsigned long long)L.bytes);
         s += buf;
-        if (L.kind == K_RED) {
+        if (L.kind == K_VIEW) {
+            snprintf(buf, sizeof(buf), "  copy kernel: %s\n", op_name(g.view_op));
+            s += buf;
+        } else if (L.kind == K_RED) {
             static const char *axis[] = {"rows", "columns", "all"}, *what[] = {"sum", "max", "min"};
             snprintf(buf, sizeof(buf), "  reduction kernel: %s over %s%s\n", what[g.red_kind], axis[g.red_axis], g.scratch_temp >= 0 ? ", two stages" : "");
             s += buf;

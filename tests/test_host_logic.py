@@ -515,3 +515,86 @@ def test_outer_broadcast_of_row_scalars_and_column_vector():
     plan = ctx.dump_plan()
     assert plan.count("launch ") == 1 and "rowvec" in plan and "colvec" in plan
     del y
+
+
+# ------------------------------------------------------------------ views (paper Section 4.4, Fig. 3)
+def test_in_place_update_of_a_view_records_forward_and_backward_sequences(ctx):
+    x = fake(ctx, (2, 3, 4))
+    v = ctx.view_permute(x, (1, 2, 0))
+    assert v.shape == (3, 4, 2)
+    ctx.assign(v, ctx.op("add", v, ctx.scalar(42.0)))
+    ctx.release(v)  # the figure shows the base's computation alone
+    lines = [ln.strip() for ln in ctx.dump_ir().splitlines()[1:-1]]
+    golden = [ln for ln in open(os.path.join(ROOT, "tests", "golden", "fig3_inplace_on_view.txt")) if not ln.startswith("#")]
+    assert len(lines) == len(golden) == 5
+    order = {}  # node number in the dump -> position in the golden list (the dump numbers operands first-visit)
+    parsed = []
+    for ln in lines:
+        m = re.match(r"%(\d+) = f32\[([\d,]*)\] lt::(\w+)\(([^)]*)\)(.*)", ln)
+        parsed.append((int(m.group(1)), m.group(2), m.group(3), [int(t.strip()[1:]) for t in m.group(4).split(",") if t.strip()], m.group(5)))
+    by_op = lambda name, k=0: [p for p in parsed if p[2] == name][k]
+    want = [tuple(f.strip() for f in g.split("|")) for g in golden]
+    got_nodes = [by_op("scalar_data"), by_op("device_data"), by_op("permute", 0), by_op("add"), by_op("permute", 1)]
+    for pos, node in enumerate(got_nodes):
+        order[node[0]] = pos
+    for (shape, op, operands, dims, root), node in zip(want, got_nodes):
+        assert "[" + node[1] + "]" == shape and node[2] == op
+        assert sorted(order[o] for o in node[3]) == sorted(int(t) for t in operands.split() if t != "-")
+        if dims != "-":
+            assert f"dims={dims}" in node[4]
+        assert ("ROOT=0" in node[4]) == (root == "ROOT")
+    # the forward permutation feeds the add, the inverse one consumes it
+    assert got_nodes[3][3].count(got_nodes[2][0]) == 1 and got_nodes[4][3] == [got_nodes[3][0]]
+
+
+def test_views_follow_their_base_and_bases_follow_their_views(ctx):
+    x = fake(ctx, (4, 8))
+    v = ctx.view_narrow(x, 1, 2, 4)
+    w = ctx.view_reshape(x, (8, 4))
+    assert v.shape == (4, 4) and w.shape == (8, 4)
+    # the base is updated in place: both views are derived again from its new computation
+    ctx.assign(x, ctx.op("mul", x, ctx.scalar(3.0)))
+    ctx.release(w)
+    text = ctx.dump_ir()
+    assert text.count("lt::narrow(") == 1 and "dim=1, start=2" in text and text.count("ROOT=") == 2
+    # the view is updated in place: the base becomes update_slice(base, view)
+    ctx.assign(v, ctx.op("neg", v))
+    text = ctx.dump_ir()
+    assert text.count("lt::update_slice(") == 1 and text.count("lt::neg(") == 1
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert "copy kernel: narrow" in plan and "copy kernel: update_slice" in plan
+    # a chain of views: permute of a narrow; the update walks back through both
+    y = fake(ctx, (2, 3, 4))
+    n = ctx.view_narrow(y, 2, 1, 2)
+    p = ctx.view_permute(n, (2, 0, 1))
+    assert p.shape == (2, 2, 3)
+    ctx.assign(p, ctx.op("add", p, ctx.scalar(1.0)))
+    text = ctx.dump_ir()
+    assert text.count("lt::permute(") == 2 and "dims=(1, 2, 0)" in text and text.count("lt::update_slice(") == 1
+    assert text.count("ROOT=") == 3  # the permuted view, the narrowed view and the base
+    ctx.barrier()
+    # reshaping materialised data records nothing and shares the buffer
+    z = fake(ctx, (6, 4))
+    r = ctx.view_reshape(z, (2, 12))
+    assert ctx.is_materialised(r) and ctx.dump_ir().count("lt::") == 0
+
+
+def test_shape_op_errors(ctx):
+    x = fake(ctx, (4, 8))
+    for bad in (lambda: ctx.view_narrow(x, 1, 6, 4), lambda: ctx.view_narrow(x, 2, 0, 1), lambda: ctx.view_reshape(x, (5, 7)),
+                lambda: ctx.view_permute(x, (0, 0)), lambda: ctx.op("update_slice", x, fake(ctx, (4, 9)), dim=1, start=0),
+                lambda: ctx.op("update_slice", x, fake(ctx, (4, 4)), dim=1, start=5)):
+        with pytest.raises(lt.LazyTensorError):
+            bad()
+
+
+def test_reshape_that_keeps_rows_and_columns_is_folded_into_the_program(ctx):
+    x = fake(ctx, (2, 3, 8))
+    y = ctx.op("add", ctx.op("reshape", ctx.op("mul", x, x), shape=(6, 8)), ctx.scalar(2.0))
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1 and ctx.stats()["launches_view"] == 0
+    z = ctx.op("add", ctx.op("reshape", ctx.op("mul", x, x), shape=(4, 12)), ctx.scalar(2.0))
+    ctx.barrier()
+    assert ctx.stats()["launches_view"] == 1
+    del y, z

@@ -391,6 +391,52 @@ def test_outer_broadcast_matches_numpy(B):
     np.testing.assert_array_equal(B.op("sub", leaf(B, r), leaf(B, rng.normal_f32(rng.generator(14), (5,)))).array.shape, (7, 5))
 
 
+def test_shape_ops_match_numpy(B):
+    g = rng.generator(15)
+    x = rng.normal_f32(g, (3, 4, 5))
+    X = leaf(B, x)
+    np.testing.assert_array_equal(B.op("reshape", X, shape=(6, 10)).array, x.reshape(6, 10))
+    for dim, start, length in ((0, 1, 2), (1, 0, 3), (2, 2, 3), (2, 4, 1)):
+        index = [slice(None)] * 3
+        index[dim] = slice(start, start + length)
+        np.testing.assert_array_equal(B.op("narrow", X, dim=dim, start=start, length=length).array, x[tuple(index)])
+        upd = rng.normal_f32(g, x[tuple(index)].shape)
+        want = x.copy()
+        want[tuple(index)] = upd
+        np.testing.assert_array_equal(B.op("update_slice", X, leaf(B, upd), dim=dim, start=start).array, want)
+    for perm in ((0, 1, 2), (1, 2, 0), (2, 0, 1), (2, 1, 0), (0, 2, 1)):
+        np.testing.assert_array_equal(B.op("permute", X, perm=perm).array, np.transpose(x, perm))
+    # a permutation and its inverse compose to the identity (Fig. 3: (1,2,0) then (2,0,1))
+    back = B.op("permute", B.op("permute", X, perm=(1, 2, 0)), perm=(2, 0, 1)).array
+    np.testing.assert_array_equal(back, x)
+    # narrow and update_slice are inverse to each other
+    sl = B.op("narrow", X, dim=1, start=1, length=2)
+    np.testing.assert_array_equal(B.op("update_slice", X, sl, dim=1, start=1).array, x)
+    # other element sizes
+    xb = rng.to_bf16_bits(x)
+    np.testing.assert_array_equal(B.op("permute", OTensor(xb, "bf16"), perm=(2, 0, 1)).array, np.transpose(xb, (2, 0, 1)))
+    m = (x > 0).astype(np.uint8)
+    np.testing.assert_array_equal(B.op("narrow", OTensor(m, "u8"), dim=2, start=1, length=3).array, m[:, :, 1:4])
+    with pytest.raises(ValueError):
+        B.op("narrow", X, dim=1, start=3, length=2)
+
+
+def test_views_share_storage_like_numpy(B):
+    x0 = np.arange(24, dtype=F32).reshape(2, 3, 4)
+    x = leaf(B, x0)
+    v = B.view_permute(x, (1, 2, 0))
+    B.assign(v, B.op("add", v, B.scalar(42.0)))       # the paper's example
+    np.testing.assert_array_equal(x.array, x0 + 42)
+    n = B.view_narrow(x, 2, 1, 2)
+    B.assign(x, B.op("mul", x, B.scalar(2.0)))         # the base changes: the view sees it
+    np.testing.assert_array_equal(n.array, ((x0 + 42) * 2)[:, :, 1:3])
+    B.assign(n, B.op("neg", n))                        # the view changes: the base sees it
+    want = (x0 + 42) * 2
+    want[:, :, 1:3] *= -1
+    np.testing.assert_array_equal(x.array, want)
+    np.testing.assert_array_equal(v.array, np.transpose(want, (1, 2, 0)))
+
+
 # ---------------------------------------------------------------------- GELU
 
 def test_gelu_closed_forms(B):
