@@ -369,6 +369,7 @@ def run_ours(args) -> None:
         c.close()
     e2e_value = aggregate_gbs(nbytes, e2e_steps, world, e2e_ms)
 
+    dp_adam = None if args.no_extra else data_parallel_adam(lt, torch, local, world)  # collective: every rank takes part
     if rank != 0:
         if world > 1:
             dist.barrier()
@@ -404,6 +405,7 @@ def run_ours(args) -> None:
         extra = extra_measurements(ctx, lt, torch, timed, step, sets, nbytes)
         extra["host_ns_per_barrier"] = {k: st[k] / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
         extra["cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "barriers": st["barriers"]}
+        extra["c5_data_parallel_adam_step"] = dp_adam
     cpu = cpu_baseline() if world == 1 and not args.no_cpu else None
 
     line = {
@@ -482,6 +484,36 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
     out.update(adam_steps(lt, torch, ctx.device))
     out["other_configs"] = other_configs(lt, torch, ctx.device)
     return out
+
+
+def data_parallel_adam(lt, torch, device: int, world: int, steps: int = 50) -> dict:
+    """Second workload at any N: the synchronous data-parallel Adam step over the 161 ResNet-50 tensors -- the
+    gradient buffer all-reduced over the ranks bucket by bucket (NCCL; nothing to exchange at N = 1), then the
+    fused multi-tensor update, recorded once and replayed.  Device time per step, maximum over ranks."""
+    from paper_2102_13267_b200.data_parallel import DataParallelAdam
+    from workloads import configs
+    from workloads.resnet50 import parameter_shapes
+
+    ctx = lt.LazyContext(device=device)
+    dp = DataParallelAdam(ctx, parameter_shapes())
+    dp.flat["p"].normal_(0.0, 0.05)
+    dp.flat["g"].normal_(0.0, 1e-3)
+    for _ in range(3):
+        dp.step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        dp.step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, torch.device("cuda", device)) / steps
+    st = ctx.stats()
+    nbytes = configs.algorithmic_bytes("c5")
+    res = {"ms_per_step": ms, "adam_gbs_all_ranks": world * nbytes / ms / 1e6, "all_reduce_bytes_per_rank": 4 * dp.total,
+           "buckets": len(dp.buckets), "compiles": st["compiles"], "replays": st["replays"], "world": world}
+    ctx.close()
+    return res
 
 
 def other_configs(lt, torch, device: int) -> dict:

@@ -84,6 +84,15 @@ def programs():
         P, G, M, V = ([d.leaf(s, "f32") for s in shapes] for _ in range(4))
         traces.adam_step(d.ctx, P, G, M, V, step=1)
         out.append(("adam_step" + suffix, d.keys()))
+    # the data-parallel step: the summed gradient is scaled by a run-time 1 / world size inside the same program
+    d = Dry()
+    shapes = [(64,), (128,)]
+    P, G, M, V = ([d.leaf(s, "f32") for s in shapes] for _ in range(4))
+    sc = traces.AdamScalars(d.ctx, step=1)
+    inv = d.ctx.scalar(0.5, dynamic=True)
+    for p_, g_, m_, v_ in zip(P, G, M, V):
+        traces.adam_update(d.ctx, p_, d.ctx.op("mul", g_, inv), m_, v_, sc)
+    out.append(("adam_step_data_parallel", d.keys()))
     d = Dry(ieee=1)
     a, b, c, e = (d.leaf((64, 64), "f32") for _ in range(4))
     keep = traces.elementwise_chain(d.ctx, a, b, c, e)

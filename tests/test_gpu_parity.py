@@ -189,6 +189,34 @@ def test_c5_adam_full_shapes(ctx):
     assert s["bytes_planned"] == 3 * 715_596_896
 
 
+def test_data_parallel_adam_step_on_one_rank(ctx):
+    """The data-parallel step with a world of one (no exchange): flat buffers, the averaging scalar folded into the
+    graph, recorded once and replayed."""
+    from paper_2102_13267_b200.data_parallel import DataParallelAdam
+
+    shapes = parameter_shapes()[:12] + [(1000,), (7,)]
+    params, grads, ms, vs = configs.c5_inputs(56, shapes)
+    dp = DataParallelAdam(ctx, shapes)
+    import torch
+    for i in range(len(shapes)):
+        dp.view("p", i).copy_(torch.from_numpy(params[i]))
+        dp.view("g", i).copy_(torch.from_numpy(grads[i]))
+    O = EagerOracle()
+    op, og, om, ov = ([O.leaf(a, "f32") for a in arrs] for arrs in (params, grads, ms, vs))
+    for step in range(1, 6):
+        s = traces.AdamScalars(O, step=step)
+        for p, g, m, v in zip(op, og, om, ov):
+            traces.adam_update(O, p, O.op("mul", g, O.scalar(1.0)), m, v, s)
+        dp.step()
+    st = ctx.stats()
+    assert (st["compiles"], st["replays"], st["launches_multi"]) == (1, 4, 5)
+    assert st["launches_compiled"] == (5 if ctx.compiled_allowed else 0)
+    torch.cuda.synchronize()
+    for i in range(len(shapes)):
+        for which, ref in (("p", op[i]), ("m", om[i]), ("v", ov[i])):
+            assert_matches(dp.view(which, i).cpu().numpy(), ref.array, "f32", f"dp adam {which}[{i}]")
+
+
 # ------------------------------------------------------------------ unfused baseline
 def test_unfused_matches_oracle(ctx):
     ctx.set_option("fusion", 0)
