@@ -150,6 +150,8 @@ typedef struct {
                                     over rows of more than 8192 elements outside a fused long-row kernel          */
     uint64_t launches_view;      /* shape operations run as copy kernels (narrow, permute, update_slice, and
                                     reshape where it is not folded into a program or a shared buffer)            */
+    uint64_t programs_specialised; /* programs handed to the run-time specialiser (see the "specialise" option)    */
+    uint64_t launches_specialised; /* of launches_compiled: kernels the run-time specialiser built                */
     uint64_t allocator_calls;    /* calls of the allocator's alloc and free (or cudaMallocAsync /
                                     cudaFreeAsync); 0 over a span means every block came from and
                                     went back to the context's own pool of released blocks          */
@@ -185,6 +187,11 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * "compiled" (1 default: a launch whose program is in the table of ahead-of-time compiled programs, whose
  * pointers are 16-byte aligned and whose rows are a multiple of 8 elements runs on that kernel; 0 = always
  * interpret),
+ * "specialise" (2 default: a program that has no kernel in the table and keeps being flushed gets one built at run
+ * time -- the same kernels, instantiated over the program by the CUDA run-time compiler on a worker thread while the
+ * interpreter keeps serving the flushes; 1 = build it when the graph is planned and wait for it; 0 = never.  Absent,
+ * silently, when the run-time compiler library cannot be loaded), "specialise_after" (3 default: flushes of a plan
+ * before mode 2 asks for the kernel),
  * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
  * line per flush and per replay; preset by the environment variable LT_LOG),
  * "wait_limit_ms" (2000 default: how long a kernel that stages long rows through shared memory waits for one of

@@ -27,13 +27,6 @@ inline uint64_t avalanche(uint64_t x) {
     return x;
 }
 
-template <class T>
-inline void put(std::vector<uint8_t> &b, T v) {
-    size_t at = b.size();
-    b.resize(at + sizeof(T));
-    memcpy(b.data() + at, &v, sizeof(T));
-}
-
 }  // namespace
 
 // 128-bit non-cryptographic hash: two 64-bit lanes, each absorbing every 8-byte word with
@@ -179,41 +172,47 @@ void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonica
         }
     }
 
-    // serialise
+    // serialise (into a buffer sized for the worst case, trimmed afterwards)
     std::vector<uint8_t> &b = cg.bytes;
-    b.reserve(cg.nodes.size() * 48 + 64);
-    put<uint32_t>(b, 0x4c5a5431u);  // format tag
-    put<int64_t>(b, c->opt.fusion);
-    put<int64_t>(b, c->opt.fast_math);
-    put<int64_t>(b, c->opt.horizontal);
-    put<int64_t>(b, c->opt.ieee);
-    put<uint32_t>(b, (uint32_t)cg.nodes.size());
+    b.resize(cg.nodes.size() * (4 + 8 * LT_MAX_RANK + 1 + 12 + 4 + 16) + cg.outputs.size() * 8 + 64);
+    uint8_t *w = b.data();
+    auto put = [&w](auto v) {
+        memcpy(w, &v, sizeof(v));
+        w += sizeof(v);
+    };
+    put((uint32_t)0x4c5a5431u);  // format tag
+    put((int64_t)c->opt.fusion);
+    put((int64_t)c->opt.fast_math);
+    put((int64_t)c->opt.horizontal);
+    put((int64_t)c->opt.ieee);
+    put((uint32_t)cg.nodes.size());
     for (const CNode &n : cg.nodes) {
-        put<uint16_t>(b, n.op);
-        put<uint8_t>(b, n.dtype);
-        put<uint8_t>(b, n.rank);
-        for (int i = 0; i < n.rank; ++i) put<int64_t>(b, n.dims[i]);
+        put((uint16_t)n.op);
+        put((uint8_t)n.dtype);
+        put((uint8_t)n.rank);
+        for (int i = 0; i < n.rank; ++i) put((int64_t)n.dims[i]);
         if (n.op == N_DEVICE_DATA) {
-            put<int32_t>(b, n.param);
+            put((int32_t)n.param);
         } else if (n.op == N_SCALAR) {
-            put<int32_t>(b, n.dyn);
-            if (n.dyn < 0) put<double>(b, n.sval);
+            put((int32_t)n.dyn);
+            if (n.dyn < 0) put((double)n.sval);
         } else {
-            put<uint8_t>(b, n.n_in);
-            for (int i = 0; i < n.n_in; ++i) put<uint32_t>(b, n.in[i]);
-            if (n.op == LT_OP_PHILOX_BITS) put<int32_t>(b, n.dyn);
-            if (n.op == LT_OP_CONVERT || n.op == LT_OP_IOTA) put<int64_t>(b, n.attr0);
+            put((uint8_t)n.n_in);
+            for (int i = 0; i < n.n_in; ++i) put((uint32_t)n.in[i]);
+            if (n.op == LT_OP_PHILOX_BITS) put((int32_t)n.dyn);
+            if (n.op == LT_OP_CONVERT || n.op == LT_OP_IOTA) put((int64_t)n.attr0);
             if (n.op >= LT_OP_RESHAPE && n.op <= LT_OP_UPDATE_SLICE) {
-                put<int64_t>(b, n.attr0);
-                put<int64_t>(b, n.attr1);
+                put((int64_t)n.attr0);
+                put((int64_t)n.attr1);
             }
         }
     }
-    put<uint32_t>(b, (uint32_t)cg.outputs.size());
+    put((uint32_t)cg.outputs.size());
     for (size_t k = 0; k < cg.outputs.size(); ++k) {
-        put<uint32_t>(b, cg.outputs[k]);
-        put<int32_t>(b, cg.donor_param[k]);
+        put((uint32_t)cg.outputs[k]);
+        put((int32_t)cg.donor_param[k]);
     }
+    b.resize((size_t)(w - b.data()));
 }
 
 }  // namespace lt

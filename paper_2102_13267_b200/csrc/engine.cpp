@@ -23,11 +23,26 @@ inline uint64_t now_ns() {
         .count();
 }
 
+// Host-time accounting of lt_stats.  The per-call cost matters: lt_op is timed, and recording a node takes little
+// more than a hundred nanoseconds.  On x86-64 the time-stamp counter is read (a few nanoseconds) and the ticks are
+// scaled to nanoseconds when the statistics are read; elsewhere the steady clock is used directly.
+#if defined(__x86_64__)
+inline uint64_t ticks_now() { return __builtin_ia32_rdtsc(); }
+const uint64_t g_tick0 = ticks_now(), g_ns0 = now_ns();
+inline double ns_per_tick() {
+    const uint64_t dt = ticks_now() - g_tick0, dn = now_ns() - g_ns0;
+    return dt && dn > 1000000 ? (double)dn / (double)dt : 0.4;  // (before a millisecond has passed: a nominal 2.5 GHz)
+}
+#else
+inline uint64_t ticks_now() { return now_ns(); }
+inline double ns_per_tick() { return 1.0; }
+#endif
+
 struct Timer {
     uint64_t &acc;
     uint64_t t0;
-    explicit Timer(uint64_t &a) : acc(a), t0(now_ns()) {}
-    ~Timer() { acc += now_ns() - t0; }
+    explicit Timer(uint64_t &a) : acc(a), t0(ticks_now()) {}
+    ~Timer() { acc += ticks_now() - t0; }
 };
 
 inline lt_tensor make_handle(const lt_ctx *c, uint32_t slot) {
@@ -113,6 +128,12 @@ void gather_roots(lt_ctx *c, std::vector<uint32_t> &roots, bool consume) {
     }
 }
 
+// The pending list has been turned into roots: forget it.
+void consume_pending(lt_ctx *c) {
+    for (uint32_t slot : c->pending) c->tensors[slot].queued = false;
+    c->pending.clear();
+}
+
 void release_donors(lt_ctx *c, const std::vector<uint32_t> &roots) {
     for (uint32_t slot : roots) {
         TensorRec &t = c->tensors[slot];
@@ -139,6 +160,11 @@ void record_replay(lt_ctx *c, Plan *cached, Plan *plan, const Canonical &cg, con
     by_node.assign(c->nodes.size(), 0);
     for (uint32_t slot = 0; slot < c->tensors.size(); ++slot)
         if (c->tensors[slot].live) by_node[c->tensors[slot].node] = slot + 1;
+    // buffer -> the first root (in creation order) that named it before lt_assign
+    std::vector<uint32_t> &by_donor = c->donor_scratch;
+    by_donor.assign(c->buffers.size(), 0);
+    for (size_t k = roots.size(); k-- > 0;)
+        if (c->tensors[roots[k]].donor != NONE) by_donor[c->tensors[roots[k]].donor] = roots[k] + 1;
     auto ref_of = [c](uint32_t slot, ReplayRecord::Ref &ref) {
         ref.slot = slot;
         ref.gen = c->tensors[slot].gen;
@@ -154,11 +180,7 @@ void record_replay(lt_ctx *c, Plan *cached, Plan *plan, const Canonical &cg, con
             continue;
         }
         // an in-place update: the tensor that named this buffer before lt_assign
-        for (uint32_t slot : roots)
-            if (c->tensors[slot].donor == leaf.buffer) {
-                ref_of(slot, pr);
-                break;
-            }
+        if (leaf.buffer < by_donor.size() && by_donor[leaf.buffer]) ref_of(by_donor[leaf.buffer] - 1, pr);
         if (pr.slot == NONE && r.why_not.empty()) r.why_not = "an input of the flushed graph was not named by any tensor";
     }
     for (const CNode &cn : cg.nodes)
@@ -483,6 +505,9 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "debug.compiled_row_u")) c->opt.compiled_row_u = value;
     else if (!strcmp(key, "debug.compiled_depth")) c->opt.compiled_depth = value;
     else if (!strcmp(key, "debug.long_l2_ahead")) c->opt.long_l2_ahead = value;
+    else if (!strcmp(key, "debug.ignore_table")) c->opt.ignore_table = value;
+    else if (!strcmp(key, "specialise")) c->opt.specialise = value;
+    else if (!strcmp(key, "specialise_after")) c->opt.specialise_after = value;
     else if (!strcmp(key, "wait_limit_ms")) c->wait_limit_ns = value > 0 ? value * 1000000ll : 1;
     else return fail(c, LT_ERR_INVALID_ARG, std::string("unknown option ") + key);
     return LT_OK;
@@ -1206,7 +1231,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
             nd.refs = 1;  // held by this loop until the tensors are repointed
             new_nodes[k] = n;
         }
-        gather_roots(c, roots, true);
+        consume_pending(c);  // `roots` still holds what the first pass gathered: nothing was recorded in between
         record_replay(c, plan, ran, cg, roots);
         for (uint32_t slot : roots) {
             TensorRec &t = c->tensors[slot];
@@ -1432,6 +1457,9 @@ lt_status lt_tensor_info(lt_ctx *c, lt_tensor t, int *dtype, int *rank, int64_t 
 lt_status lt_get_stats(lt_ctx *c, lt_stats *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
     *out = c->stats;
+    const double k = ns_per_tick();  // the time fields accumulate ticks
+    for (uint64_t *f : {&out->ns_record, &out->ns_canonicalise, &out->ns_hash_lookup, &out->ns_plan, &out->ns_bind_launch, &out->ns_rebind})
+        *f = (uint64_t)((double)*f * k);
     return LT_OK;
 }
 

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "../../include/lazytensor.h"
+#include "jit.h"
 #include "vm.h"
 
 namespace lt {
@@ -141,6 +142,12 @@ struct Launch {
     unsigned threads = LT_EW_THREADS;
     int compiled = -1;                   // entry of the ahead-of-time compiled table (compiled.h), or -1
     int compiled_blocks[4] = {0, 0, 0, 0};  // resident blocks per SM of that entry's kernels, by log2(chunks in flight); 0 = not asked yet
+    // run-time specialisation (jit.h) of a program without a table entry: requested once the plan has run a few
+    // times, used as soon as the machine code is ready
+    std::unique_ptr<JitProgram> jit_program;  // null: not eligible
+    std::shared_ptr<JitKernel> jit;
+    bool jit_failed = false;
+    uint32_t runs = 0;
     std::unique_ptr<LtKParams> kp;       // K_EW / K_ROW parameter block (static parts prefilled)
     std::unique_ptr<LtMultiParams> mp;   // K_MULTI
 };
@@ -174,6 +181,9 @@ struct Options {
     int64_t compiled_row_u = 0;  // chunks per thread in compiled row kernels (0 = one warp per row where it fits)
     int64_t compiled_depth = -1;  // staging depth of compiled row kernels (-1 = default, 0 = direct loads)
     int64_t compiled_u = 0;  // chunks in flight per thread in compiled elementwise / multi kernels (0 = default)
+    int64_t specialise = 2;        // run-time specialisation: 0 off, 1 at planning time (blocking), 2 on a worker thread
+    int64_t specialise_after = 3;  // ... once a plan has run this many times (mode 2)
+    int64_t ignore_table = 0;      // measurements: plan as if the build-time table were empty (everything specialised or interpreted)
     int64_t long_l2_ahead = -1;  // long-row kernels: request the next row into L2 (-1 = the library's choice)
 };
 
@@ -266,7 +276,7 @@ struct lt_ctx {
 
     // scratch reused across barriers
     lt::Canonical canon;
-    std::vector<uint32_t> roots_scratch, stack_scratch;
+    std::vector<uint32_t> roots_scratch, stack_scratch, donor_scratch;
     std::vector<void *> param_ptr, out_ptr, temp_ptr;
     std::vector<uint32_t> buf_stamp;
     std::vector<int32_t> buf_param;

@@ -2,6 +2,7 @@
 // and launches its kernels on the context's stream.
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <cstring>
 #include <memory>
 #include <string>
@@ -53,19 +54,66 @@ cudaEvent_t take_event(lt_ctx *c) {
 
 bool aligned_for(uint64_t p, uint8_t dtype) { return (p & (dtype == LT_U8 ? 7u : 15u)) == 0; }
 
+// The straight-line kernel of a launch comes from the build-time table (L.compiled) or from the run-time
+// specialiser (L.jit, once its machine code is ready and loaded); the helpers below hide which.
+bool specialised(const Launch &L) { return L.compiled < 0; }
+
 // resident blocks per SM of a compiled kernel variant, asked once per plan launch
-int compiled_blocks(Launch &L, int u, int threads, size_t dyn = 0) {
+int compiled_blocks(lt_ctx *c, Launch &L, int u, int threads, size_t dyn = 0) {
     int lg = 0;
     while ((1 << lg) < u) ++lg;
     if (L.compiled_blocks[lg] == 0) {
         int b = 0;
-        if (lt_compiled_occupancy(L.compiled, u, threads, dyn, &b) != cudaSuccess || b < 1) {
+        if (specialised(L)) b = jit_occupancy(*L.jit, c->device, 0, threads, dyn);
+        else if (lt_compiled_occupancy(L.compiled, u, threads, dyn, &b) != cudaSuccess || b < 1) {
             cudaGetLastError();
             b = 1;
         }
         L.compiled_blocks[lg] = b;
     }
     return L.compiled_blocks[lg];
+}
+
+cudaError_t fast_launch(lt_ctx *c, Launch &L, const void *params, int u, unsigned grid, unsigned threads, unsigned group, unsigned group_log2,
+                        unsigned depth, size_t dyn) {
+    if (!specialised(L)) return lt_compiled_launch(L.compiled, params, u, grid, threads, group, group_log2, depth, c->stream);
+    uint32_t a1 = group, a2 = group_log2, a3 = depth;
+    void *args[4] = {const_cast<void *>(params), &a1, &a2, &a3};
+    std::string err;
+    if (!jit_launch(*L.jit, c->device, 0, grid, threads, dyn, (void *)c->stream, args, &err)) {
+        c->error = err;
+        return cudaErrorLaunchFailure;
+    }
+    c->stats.launches_specialised++;
+    return cudaSuccess;
+}
+
+// Is there a straight-line kernel for this launch right now?  Requests the specialisation when the plan has run
+// often enough, and loads its machine code when it has arrived.
+bool fast_kernel_ready(lt_ctx *c, Launch &L) {
+    if (!c->opt.compiled) return false;
+    if (L.compiled >= 0) return true;
+    if (!L.jit_program || L.jit_failed || !c->opt.specialise) return false;
+    ++L.runs;
+    if (!L.jit) {
+        const bool now = c->opt.specialise == 1;
+        if (!now && (int64_t)L.runs < c->opt.specialise_after) return false;
+        L.jit = jit_request(*L.jit_program, now);
+        if (!L.jit) {
+            L.jit_failed = true;
+            return false;
+        }
+        c->stats.programs_specialised++;
+    }
+    const int st = L.jit->state.load();
+    if (st == 0) return false;  // still being compiled: the interpreter serves this flush
+    std::string err;
+    if (st < 0 || !jit_load(*L.jit, c->device, &err)) {
+        L.jit_failed = true;
+        if (c->opt.log >= 1) fprintf(stderr, "[lazytensor] run-time specialisation failed: %s\n%s\n", err.c_str(), L.jit->log.c_str());
+        return false;
+    }
+    return true;
 }
 
 }  // namespace
@@ -101,7 +149,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
         for (const Launch &L : plan.launches) {
             const Group &g = plan.groups[L.groups[0]];
             if (L.kind != K_ROW || !g.long_row) continue;
-            bool ok = c->opt.compiled && L.compiled >= 0 && (g.cols % LT_VM_V) == 0;
+            bool ok = c->opt.compiled && (L.compiled >= 0 || (L.jit && !L.jit_failed)) && (g.cols % LT_VM_V) == 0;
             for (size_t q = 0; q < g.io.size() && ok; ++q)
                 if (g.io[q].kind == IO_PARAM && g.io[q].cls <= LT_CLS_COLVEC)
                     ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index], g.io[q].dtype);
@@ -262,7 +310,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                 }
             }
             bool done = false;
-            if (!dry && c->opt.compiled && L.compiled >= 0) {
+            if (!dry && fast_kernel_ready(c, L)) {
                 // compiled kernel: needs 128-bit accesses everywhere (aligned pointers, whole chunks)
                 bool ok = true;
                 for (size_t k = 0; k < L.groups.size() && ok; ++k) {
@@ -273,13 +321,13 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     // two chunks in flight per thread and eight waves of blocks measured best for wide programs
                     // (four input streams) over many tensors of uneven size
                     // (one chunk with correctly rounded division and square root: their slow paths cost registers)
-                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : (L.flavour == 2 ? 1 : 2);
-                    const int occ = compiled_blocks(L, u, LT_EW_THREADS);
+                    const int u = (c->opt.compiled_u > 0 && !specialised(L)) ? (int)c->opt.compiled_u : (L.flavour == 2 ? 1 : 2);
+                    const int occ = compiled_blocks(c, L, u, LT_EW_THREADS);
                     const unsigned mwaves = c->opt.waves > 0 ? waves : 8u;  // C5: 116 us against 121 with two waves
                     unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * mwaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, 0, c->stream);
+                    e = fast_launch(c, L, &P, u, grid, LT_EW_THREADS, 0, 0, 0, 0);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     c->stats.launches_compiled++;
                     done = true;
@@ -347,11 +395,19 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     // Staging and CTA size: the row a CTA works on is staged when it fits; several CTAs per SM overlap one
                     // another's passes; when a staged row leaves room for one CTA only, that CTA has 512 threads.
                     const size_t cap = 200u * 1024u;
-                    const size_t stage = lt_compiled_long_stage_bytes(L.compiled, P.cols);
+                    if (specialised(L)) {
+                        std::string err;
+                        if (!jit_load(*L.jit, c->device, &err)) {
+                            release_all(true);
+                            return fail(c, LT_ERR_CUDA, err);
+                        }
+                    }
+                    const size_t stage = specialised(L) ? jit_long_stage_bytes(*L.jit_program, P.cols) : lt_compiled_long_stage_bytes(L.compiled, P.cols);
                     const unsigned deepest = stage == 0 ? 0u : (unsigned)std::min<size_t>(2, cap / stage);
                     auto blocks_at = [&](unsigned threads, unsigned d) {
                         int b = 0;
-                        if (lt_compiled_long_occupancy(L.compiled, threads, d * stage, &b) != cudaSuccess || b < 1) {
+                        if (specialised(L)) b = jit_occupancy(*L.jit, c->device, threads >= 512 ? 1 : 0, (int)threads, d * stage);
+                        else if (lt_compiled_long_occupancy(L.compiled, threads, d * stage, &b) != cudaSuccess || b < 1) {
                             cudaGetLastError();
                             b = 1;
                         }
@@ -376,22 +432,35 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     bool l2_ahead = stage != 0 && occ < 2 && depth >= 1;
                     if (c->opt.long_l2_ahead >= 0) l2_ahead = stage != 0 && c->opt.long_l2_ahead != 0;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch_long(L.compiled, &P, grid, threads, depth, stage, (uint64_t)c->wait_limit_ns, l2_ahead ? 1 : 0, c->stream);
+                    if (specialised(L)) {
+                        uint32_t a1 = depth, a2 = (uint32_t)stage, a4 = l2_ahead ? 1u : 0u;
+                        uint64_t a3 = (uint64_t)c->wait_limit_ns;
+                        void *args[5] = {&P, &a1, &a2, &a3, &a4};
+                        std::string err;
+                        if (!jit_launch(*L.jit, c->device, threads >= 512 ? 1 : 0, grid, threads, depth * stage, (void *)c->stream, args, &err)) {
+                            c->error = err;
+                            e = cudaErrorLaunchFailure;
+                        } else {
+                            c->stats.launches_specialised++;
+                        }
+                    } else {
+                        e = lt_compiled_launch_long(L.compiled, &P, grid, threads, depth, stage, (uint64_t)c->wait_limit_ns, l2_ahead ? 1 : 0, c->stream);
+                    }
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     if (depth) c->status_pending = true;
                 }
                 c->stats.launches_compiled++;
                 done = true;
             }
-            if (!done && !dry && c->opt.compiled && L.compiled >= 0) {
+            if (!done && !dry && fast_kernel_ready(c, L)) {
                 // compiled kernel: needs 128-bit accesses everywhere (aligned pointers, whole chunks)
                 bool ok = (L.kind == K_EW && !P.rowcol) ? (P.n % LT_VM_V) == 0 : (P.cols % LT_VM_V) == 0;
                 ok = ok && P.n_chunks < (1ull << 31);
                 for (size_t s = 0; s < g.io.size() && ok; ++s)
                     if (g.io[s].cls <= LT_CLS_COLVEC) ok = aligned_for(P.ptr[s], g.io[s].dtype);
                 if (ok && L.kind == K_EW) {
-                    const int u = c->opt.compiled_u > 0 ? (int)c->opt.compiled_u : 1;
-                    const int occ = compiled_blocks(L, u, LT_EW_THREADS);
+                    const int u = (c->opt.compiled_u > 0 && !specialised(L)) ? (int)c->opt.compiled_u : 1;
+                    const int occ = compiled_blocks(c, L, u, LT_EW_THREADS);
                     const uint64_t need = (P.n_chunks + (uint64_t)LT_EW_THREADS * u - 1) / ((uint64_t)LT_EW_THREADS * u);
                     // a compiled CTA has no set-up to amortise: many short CTAs, scheduled by the hardware as others
                     // retire, beat one wave of persistent ones (C2: 31.3 us against 33.5; no change beyond 8 waves)
@@ -399,25 +468,25 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * occ * ewaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch(L.compiled, &P, u, grid, LT_EW_THREADS, 0, 0, 0, c->stream);
+                    e = fast_launch(c, L, &P, u, grid, LT_EW_THREADS, 0, 0, 0, 0);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     done = true;
                 } else if (ok && P.cpr <= 8u * 128u) {  // a row's group of threads is at most one CTA of 128
                     // a row lives in the registers of its thread group: up to 8 chunks per thread, one warp per row if it fits
                     int u = 1;
                     while (u < 8 && P.cpr > 32u * u) u *= 2;
-                    if (c->opt.compiled_row_u > 0) u = (int)c->opt.compiled_row_u;
+                    if (c->opt.compiled_row_u > 0 && !specialised(L)) u = (int)c->opt.compiled_row_u;
                     while (u < 8 && P.cpr > 128u * u) u *= 2;  // a row's group is at most one CTA of 128 threads
                     unsigned grp = 1, lg = 0;
                     while (grp * u < P.cpr) grp <<= 1, ++lg;
                     const unsigned threads = grp > 128 ? grp : 128;
                     // pipeline depth: stages of the next blocks' inputs in shared memory, within ~72 KB per CTA
-                    const size_t stage = lt_compiled_row_stage_bytes(L.compiled, u);
-                    unsigned depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth
-                                                                       : (lt_compiled_prefers_staging(L.compiled) ? 2u : 0u);
+                    const size_t stage = specialised(L) ? jit_row_stage_bytes(*L.jit_program, u, 128) : lt_compiled_row_stage_bytes(L.compiled, u);
+                    const bool wants_ring = specialised(L) ? !jit_integer_heavy(*L.jit_program) : lt_compiled_prefers_staging(L.compiled) != 0;
+                    unsigned depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth : (wants_ring ? 2u : 0u);
                     while (depth > 0 && depth * stage > 72u * 1024u) --depth;
                     if (stage == 0 || threads != 128 || depth < 2) depth = 0;
-                    const int occ = compiled_blocks(L, u, (int)threads, depth * stage);
+                    const int occ = compiled_blocks(c, L, u, (int)threads, depth * stage);
                     const uint64_t blocks = ((uint64_t)P.rows + threads / grp - 1) / (threads / grp);
                     // one wave of persistent CTAs; with many blocks of rows per CTA, four waves balance the tail
                     // better (measured on [32768 x 2048]: 49.6 us against 54.5)
@@ -426,7 +495,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     unsigned grid = (unsigned)std::min<uint64_t>(blocks, resident * rwaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
-                    e = lt_compiled_launch(L.compiled, &P, u, grid, threads, grp, lg, depth, c->stream);
+                    e = fast_launch(c, L, &P, u, grid, threads, grp, lg, depth, depth * stage);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     done = true;
                 }

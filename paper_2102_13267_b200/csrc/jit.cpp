@@ -1,0 +1,379 @@
+// Run-time specialisation: the kernels of compiled_shells.cuh, built for a program that has no entry in the
+// build-time table.
+//
+// The paper's runtime compiles a traced graph once and caches the executable (Section 4).  This library normally
+// needs no compiler at run time -- programs in the table have kernels, everything else is interpreted -- but a graph
+// that keeps coming back deserves the straight-line kernel too.  For such a program the same hand-written shells
+// are instantiated over the program by the CUDA run-time compiler (NVRTC, loaded with dlopen; if it or the driver
+// library cannot be loaded the feature is simply absent), on a worker thread, while the interpreter keeps
+// serving the flushes; once the machine code is there the launches switch over.  Nothing is generated but the
+// program's table entry (a struct of constants): the kernels are the ones in compiled_shells.cuh.
+#include "jit.h"
+
+#include <cuda.h>
+#include <dlfcn.h>
+#include <nvrtc.h>
+
+#include <condition_variable>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <map>
+#include <mutex>
+#include <thread>
+
+namespace lt {
+
+namespace {
+
+#include "jit_sources.inc"  // the text of vm.h, vm_ops.cuh, pdl.cuh and compiled_shells.cuh
+
+struct Api {
+    bool ok = false;
+    // NVRTC
+    nvrtcResult (*CreateProgram)(nvrtcProgram *, const char *, const char *, int, const char *const *, const char *const *) = nullptr;
+    nvrtcResult (*DestroyProgram)(nvrtcProgram *) = nullptr;
+    nvrtcResult (*CompileProgram)(nvrtcProgram, int, const char *const *) = nullptr;
+    nvrtcResult (*AddNameExpression)(nvrtcProgram, const char *) = nullptr;
+    nvrtcResult (*GetLoweredName)(nvrtcProgram, const char *, const char **) = nullptr;
+    nvrtcResult (*GetCUBINSize)(nvrtcProgram, size_t *) = nullptr;
+    nvrtcResult (*GetCUBIN)(nvrtcProgram, char *) = nullptr;
+    nvrtcResult (*GetProgramLogSize)(nvrtcProgram, size_t *) = nullptr;
+    nvrtcResult (*GetProgramLog)(nvrtcProgram, char *) = nullptr;
+    // driver
+    CUresult (*ModuleLoadData)(CUmodule *, const void *) = nullptr;
+    CUresult (*ModuleGetFunction)(CUfunction *, CUmodule, const char *) = nullptr;
+    CUresult (*LaunchKernelEx)(const CUlaunchConfig *, CUfunction, void **, void **) = nullptr;
+    CUresult (*FuncSetAttribute)(CUfunction, CUfunction_attribute, int) = nullptr;
+    CUresult (*OccupancyMaxActiveBlocksPerMultiprocessor)(int *, CUfunction, int, size_t) = nullptr;
+    CUresult (*GetErrorString)(CUresult, const char **) = nullptr;
+};
+
+template <class F>
+bool sym(void *lib, const char *name, F &fn) {
+    fn = reinterpret_cast<F>(dlsym(lib, name));
+    return fn != nullptr;
+}
+
+const Api &api() {
+    static Api a = [] {
+        Api x;
+        void *rtc = nullptr;
+        for (const char *n : {"libnvrtc.so.12", "libnvrtc.so"})
+            if (!rtc) rtc = dlopen(n, RTLD_NOW | RTLD_LOCAL);
+        void *drv = nullptr;
+        for (const char *n : {"libcuda.so.1", "libcuda.so"})
+            if (!drv) drv = dlopen(n, RTLD_NOW | RTLD_LOCAL);
+        if (!rtc) return x;
+        bool ok = sym(rtc, "nvrtcCreateProgram", x.CreateProgram) && sym(rtc, "nvrtcDestroyProgram", x.DestroyProgram) &&
+                  sym(rtc, "nvrtcCompileProgram", x.CompileProgram) && sym(rtc, "nvrtcAddNameExpression", x.AddNameExpression) &&
+                  sym(rtc, "nvrtcGetLoweredName", x.GetLoweredName) && sym(rtc, "nvrtcGetCUBINSize", x.GetCUBINSize) &&
+                  sym(rtc, "nvrtcGetCUBIN", x.GetCUBIN) && sym(rtc, "nvrtcGetProgramLogSize", x.GetProgramLogSize) &&
+                  sym(rtc, "nvrtcGetProgramLog", x.GetProgramLog);
+        // without the driver library (a machine with no GPU) programs can still be compiled, not loaded
+        if (drv)
+            sym(drv, "cuModuleLoadData", x.ModuleLoadData), sym(drv, "cuModuleGetFunction", x.ModuleGetFunction),
+                sym(drv, "cuLaunchKernelEx", x.LaunchKernelEx), sym(drv, "cuFuncSetAttribute", x.FuncSetAttribute),
+                sym(drv, "cuOccupancyMaxActiveBlocksPerMultiprocessor", x.OccupancyMaxActiveBlocksPerMultiprocessor),
+                sym(drv, "cuGetErrorString", x.GetErrorString);
+        x.ok = ok;
+        return x;
+    }();
+    return a;
+}
+
+std::string program_struct(const JitProgram &p) {
+    std::string s = "#include \"compiled_shells.cuh\"\nnamespace {\nstruct JP {\n    static constexpr const char *name = \"specialised\";\n";
+    s += "    static constexpr int kind = " + std::to_string(p.kind) + ", flavour = " + std::to_string(p.flavour) + ", n_pro = " +
+         std::to_string(p.n_pro) + ", n_ins = " + std::to_string(p.ins.size()) + ", n_slots = " + std::to_string(p.dtype.size()) + ";\n";
+    s += "    static constexpr LtIns ins[" + std::to_string(p.ins.size()) + "] = {";
+    for (size_t i = 0; i < p.ins.size(); ++i) s += (i ? ", {" : "{") + std::to_string(p.ins[i].op) + ", " + std::to_string(p.ins[i].imm) + "}";
+    s += "};\n    static constexpr uint8_t dtype[" + std::to_string(p.dtype.size()) + "] = {";
+    for (size_t i = 0; i < p.dtype.size(); ++i) s += (i ? ", " : "") + std::to_string(p.dtype[i]);
+    s += "};\n    static constexpr uint8_t cls[" + std::to_string(p.cls.size()) + "] = {";
+    for (size_t i = 0; i < p.cls.size(); ++i) s += (i ? ", " : "") + std::to_string(p.cls[i]);
+    s += "};\n};\n}\n";
+    return s;
+}
+
+// kernel instantiations one program needs: (name expression, slot in JitKernel::fn)
+std::vector<std::pair<std::string, int>> variants_of(const JitProgram &p) {
+    std::vector<std::pair<std::string, int>> v;
+    if (p.kind == 0) v.push_back({"lt_c_ew<JP, 1>", 0});
+    else if (p.kind == 2) v.push_back({std::string("lt_c_multi<JP, ") + (p.flavour == 2 ? "1" : "2") + ">", 0});
+    else if (p.long_row) {
+        v.push_back({"lt_c_longrow<JP, 256>", 0});
+        v.push_back({"lt_c_longrow<JP, 512>", 1});
+    } else {
+        v.push_back({"lt_c_row<JP, " + std::to_string(p.row_u) + ">", 0});
+    }
+    return v;
+}
+
+void compile(JitKernel &k) {
+    const Api &a = api();
+    const std::string src = program_struct(k.program);
+    const char *names[] = {"vm.h", "vm_ops.cuh", "pdl.cuh", "compiled_shells.cuh"};
+    const char *texts[] = {kSrcVm, kSrcVmOps, kSrcPdl, kSrcShells};
+    nvrtcProgram prog = nullptr;
+    if (a.CreateProgram(&prog, src.c_str(), "specialised.cu", 4, texts, names) != NVRTC_SUCCESS) {
+        k.log = "nvrtcCreateProgram failed";
+        k.state.store(-1);
+        return;
+    }
+    const auto variants = variants_of(k.program);
+    for (auto &v : variants) a.AddNameExpression(prog, v.first.c_str());
+    const char *opts[] = {"--gpu-architecture=sm_100a", "-std=c++17", "-default-device", "-diag-suppress=177"};
+    const nvrtcResult r = a.CompileProgram(prog, 4, opts);
+    size_t n = 0;
+    if (a.GetProgramLogSize(prog, &n) == NVRTC_SUCCESS && n > 1) {
+        k.log.resize(n);
+        a.GetProgramLog(prog, &k.log[0]);
+    }
+    bool ok = r == NVRTC_SUCCESS;
+    if (ok) {
+        for (auto &v : variants) {
+            const char *low = nullptr;
+            ok = ok && a.GetLoweredName(prog, v.first.c_str(), &low) == NVRTC_SUCCESS && low;
+            if (ok) k.entry[v.second] = low;
+        }
+        ok = ok && a.GetCUBINSize(prog, &n) == NVRTC_SUCCESS && n > 0;
+        if (ok) {
+            k.cubin.resize(n);
+            ok = a.GetCUBIN(prog, k.cubin.data()) == NVRTC_SUCCESS;
+        }
+    }
+    a.DestroyProgram(&prog);
+    k.state.store(ok ? 1 : -1);
+}
+
+// One worker thread for the whole process; jobs only produce machine code, so they outlive no context.
+struct Worker {
+    std::mutex m;
+    std::condition_variable cv;
+    std::deque<std::shared_ptr<JitKernel>> queue;
+    std::map<std::string, std::shared_ptr<JitKernel>> cache;  // by program identity
+    std::thread th;
+    bool stop = false;
+    ~Worker() {
+        {
+            std::lock_guard<std::mutex> g(m);
+            stop = true;
+            queue.clear();
+        }
+        cv.notify_all();
+        if (th.joinable()) th.join();
+    }
+    void run() {
+        for (;;) {
+            std::shared_ptr<JitKernel> job;
+            {
+                std::unique_lock<std::mutex> g(m);
+                cv.wait(g, [&] { return stop || !queue.empty(); });
+                if (stop) return;
+                job = queue.front();
+                queue.pop_front();
+            }
+            compile(*job);
+        }
+    }
+};
+
+Worker &worker() {
+    static Worker w;
+    return w;
+}
+
+std::string identity(const JitProgram &p) {
+    std::string s;
+    s.push_back((char)p.kind);
+    s.push_back((char)p.flavour);
+    s.push_back((char)p.long_row);
+    s.push_back((char)p.row_u);
+    s.append((const char *)&p.n_pro, sizeof(p.n_pro));
+    s.append((const char *)p.ins.data(), p.ins.size() * sizeof(LtIns));
+    s.append((const char *)p.dtype.data(), p.dtype.size());
+    s.append((const char *)p.cls.data(), p.cls.size());
+    return s;
+}
+
+}  // namespace
+
+bool jit_available() { return api().ok; }
+
+std::shared_ptr<JitKernel> jit_request(const JitProgram &p, bool synchronous) {
+    if (!api().ok) return nullptr;
+    Worker &w = worker();
+    std::shared_ptr<JitKernel> k;
+    bool fresh = false;
+    {
+        std::lock_guard<std::mutex> g(w.m);
+        auto it = w.cache.find(identity(p));
+        if (it != w.cache.end()) k = it->second;
+        else {
+            k = std::make_shared<JitKernel>();
+            k->program = p;
+            w.cache[identity(p)] = k;
+            fresh = true;
+            if (!synchronous) {
+                if (!w.th.joinable()) w.th = std::thread([&w] { w.run(); });
+                w.queue.push_back(k);
+            }
+        }
+    }
+    if (fresh && synchronous) compile(*k);
+    else if (fresh) w.cv.notify_one();
+    else if (synchronous)
+        while (k->state.load() == 0) std::this_thread::yield();  // someone else is compiling it: wait for them
+    return k;
+}
+
+// ---- loading and launching (on the thread, and with the device, of the caller)
+
+static const char *cu_text(CUresult r) {
+    const char *s = nullptr;
+    if (api().GetErrorString) api().GetErrorString(r, &s);
+    return s ? s : "driver error";
+}
+
+bool jit_load(JitKernel &k, int device, std::string *err) {
+    if (k.state.load() != 1) return false;
+    std::lock_guard<std::mutex> g(k.load_lock);
+    auto it = k.loaded.find(device);
+    if (it != k.loaded.end()) return it->second.ok;
+    JitKernel::Loaded L;
+    const Api &a = api();
+    if (!a.ModuleLoadData || !a.LaunchKernelEx) {
+        if (err) *err = "the CUDA driver library is not available";
+        k.loaded[device] = L;
+        return false;
+    }
+    CUmodule mod = nullptr;
+    CUresult r = a.ModuleLoadData(&mod, k.cubin.data());
+    if (r == CUDA_SUCCESS) {
+        L.ok = true;
+        for (int v = 0; v < 2 && L.ok; ++v)
+            if (!k.entry[v].empty()) {
+                CUfunction f = nullptr;
+                r = a.ModuleGetFunction(&f, mod, k.entry[v].c_str());
+                L.ok = r == CUDA_SUCCESS;
+                L.fn[v] = f;
+            }
+    }
+    if (!L.ok && err) *err = std::string("loading a specialised kernel: ") + cu_text(r);
+    k.loaded[device] = L;
+    return L.ok;
+}
+
+static void *fn_of(JitKernel &k, int device, int variant) {
+    auto it = k.loaded.find(device);
+    return it == k.loaded.end() || !it->second.ok ? nullptr : it->second.fn[variant];
+}
+
+int jit_occupancy(JitKernel &k, int device, int variant, int threads, size_t dyn_smem) {
+    CUfunction f = (CUfunction)fn_of(k, device, variant);
+    if (!f) return 1;
+    const Api &a = api();
+    if (dyn_smem > 32u * 1024u) a.FuncSetAttribute(f, CU_FUNC_ATTRIBUTE_MAX_DYNAMIC_SHARED_SIZE_BYTES, (int)dyn_smem);
+    int n = 0;
+    if (a.OccupancyMaxActiveBlocksPerMultiprocessor(&n, f, threads, dyn_smem) != CUDA_SUCCESS || n < 1) n = 1;
+    return n;
+}
+
+bool jit_launch(JitKernel &k, int device, int variant, unsigned grid, unsigned threads, size_t dyn_smem, void *stream, void **args,
+                std::string *err) {
+    CUfunction f = (CUfunction)fn_of(k, device, variant);
+    if (!f) {
+        if (err) *err = "specialised kernel not loaded";
+        return false;
+    }
+    const Api &a = api();
+    if (dyn_smem > 32u * 1024u) {
+        const CUresult r = a.FuncSetAttribute(f, CU_FUNC_ATTRIBUTE_MAX_DYNAMIC_SHARED_SIZE_BYTES, (int)dyn_smem);
+        if (r != CUDA_SUCCESS) {
+            if (err) *err = std::string("cuFuncSetAttribute: ") + cu_text(r);
+            return false;
+        }
+    }
+    CUlaunchConfig cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDimX = grid;
+    cfg.gridDimY = cfg.gridDimZ = 1;
+    cfg.blockDimX = threads;
+    cfg.blockDimY = cfg.blockDimZ = 1;
+    cfg.sharedMemBytes = (unsigned)dyn_smem;
+    cfg.hStream = (CUstream)stream;
+    CUlaunchAttribute attr[1];
+    memset(attr, 0, sizeof(attr));
+    attr[0].id = CU_LAUNCH_ATTRIBUTE_PROGRAMMATIC_STREAM_SERIALIZATION;  // see pdl.cuh
+    attr[0].value.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const CUresult r = a.LaunchKernelEx(&cfg, f, args, nullptr);
+    if (r != CUDA_SUCCESS) {
+        if (err) *err = std::string("cuLaunchKernelEx: ") + cu_text(r);
+        return false;
+    }
+    return true;
+}
+
+// ---- what the executor needs to know about a program without instantiating anything (cf. Info<> in the shells)
+
+static bool reads_slot(const LtIns &in) {
+    return (in.op >= OP_LD && in.op < OP_LD + LT_VM_ND) || (in.op >= OP_F2M && in.op < OP_F2M + F2M_COUNT);
+}
+
+static size_t chunk_bytes(uint8_t dtype) { return dtype == LT_ST_BF16 ? 16 : dtype == LT_ST_U8 ? 8 : 32; }
+
+size_t jit_row_stage_bytes(const JitProgram &p, int u, int threads) {
+    size_t off = 0;
+    for (size_t k = p.n_pro; k < p.ins.size(); ++k)
+        if (reads_slot(p.ins[k]) && p.cls[p.ins[k].imm] == LT_CLS_FULL) off += chunk_bytes(p.dtype[p.ins[k].imm]) * (size_t)u * threads;
+    return off;
+}
+
+bool jit_integer_heavy(const JitProgram &p) {
+    for (const LtIns &in : p.ins)
+        if (in.op == OP_PHILOX) return true;
+    return false;
+}
+
+size_t jit_long_stage_bytes(const JitProgram &p, uint32_t cols) {
+    size_t off = 0;
+    for (size_t s = 0; s < p.dtype.size(); ++s) {
+        if (p.cls[s] != LT_CLS_FULL) continue;
+        bool in = false;
+        for (size_t k = p.n_pro; k < p.ins.size() && !in; ++k) in = reads_slot(p.ins[k]) && p.ins[k].imm == s;
+        if (!in) continue;
+        const size_t es = p.dtype[s] == LT_ST_BF16 ? 2 : p.dtype[s] == LT_ST_U8 ? 1 : 4;
+        if (((size_t)cols * es) % 16u) return 0;
+        off += ((size_t)cols * es + 15u) & ~(size_t)15u;
+    }
+    return off;
+}
+
+int jit_reductions(const JitProgram &p) {
+    int n = 0;
+    for (size_t k = p.n_pro; k < p.ins.size(); ++k) n += p.ins[k].op >= OP_RED_SUM && p.ins[k].op <= OP_RED_MIN;
+    return n;
+}
+
+// What the shells can express (cf. the checks of the table generator): broadcast operands loaded in the prologue into
+// temporaries that nothing overwrites, results that are full-class or one value per row.
+bool jit_supported(const JitProgram &p) {
+    bool reserved[LT_VM_NT] = {false};
+    for (uint32_t k = 0; k < p.n_pro; ++k) {
+        const int d = (int)p.ins[k].op - OP_LD;
+        if (d < 0 || d >= LT_VM_NT || p.cls[p.ins[k].imm] == LT_CLS_FULL) return false;
+        reserved[d] = true;
+    }
+    for (size_t k = p.n_pro; k < p.ins.size(); ++k) {
+        const uint32_t op = p.ins[k].op;
+        if (op >= OP_MOV_T_ACC && op < OP_MOV_T_ACC + LT_VM_NT && reserved[op - OP_MOV_T_ACC]) return false;
+        if (op >= OP_LD && op < OP_LD + LT_VM_NT && reserved[op - OP_LD]) return false;
+        if (op == OP_ST && p.cls[p.ins[k].imm] != LT_CLS_FULL && p.cls[p.ins[k].imm] != LT_CLS_ROWVEC) return false;
+    }
+    return jit_reductions(p) <= 4;
+}
+
+}  // namespace lt

@@ -6,9 +6,11 @@
 // depend on the overlap.  pdl_release() lets the next kernel on the stream be scheduled as soon as this one
 // leaves room.  Without a kernel directly ahead on the stream both are no-ops.
 #pragma once
+#ifndef __CUDACC_RTC__
 #include <cuda_runtime.h>
 
 #include <utility>
+#endif
 
 #ifndef LT_PDL
 #define LT_PDL 1
@@ -17,6 +19,7 @@
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+#ifndef __CUDACC_RTC__
 template <class... KArgs, class... Args>
 cudaError_t launch_pdl_grid(void (*kernel)(KArgs...), dim3 grid, unsigned threads, cudaStream_t stream, Args &&...args);
 
@@ -49,3 +52,4 @@ cudaError_t launch_pdl_grid(void (*kernel)(KArgs...), dim3 grid, unsigned thread
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
+#endif  // !__CUDACC_RTC__

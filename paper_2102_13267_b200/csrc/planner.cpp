@@ -1253,8 +1253,32 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             dt[s] = g.io[s].dtype;
             cl[s] = L.kind == K_MULTI ? (uint8_t)LT_CLS_FULL : g.io[s].cls;
         }
-        L.compiled = lt_compiled_find(L.kind, L.flavour, g.ins.data(), (uint32_t)g.ins.size(), g.n_pro, dt, cl, (uint32_t)g.io.size());
-        if (g.long_row && (L.compiled < 0 || !c->opt.compiled)) unfused_long_row = true;
+        L.compiled = c->opt.ignore_table ? -1 : lt_compiled_find(L.kind, L.flavour, g.ins.data(), (uint32_t)g.ins.size(), g.n_pro, dt, cl, (uint32_t)g.io.size());
+        if (L.compiled < 0 && c->opt.compiled && c->opt.specialise && jit_available()) {
+            // no table entry: describe the program for the run-time specialiser
+            std::unique_ptr<JitProgram> jp(new JitProgram());
+            jp->kind = L.kind;
+            jp->flavour = L.flavour;
+            jp->n_pro = g.n_pro;
+            jp->ins = g.ins;
+            jp->dtype.assign(dt, dt + g.io.size());
+            jp->cls.assign(cl, cl + g.io.size());
+            jp->long_row = g.long_row;
+            if (L.kind == K_ROW && !g.long_row) {
+                const uint32_t cpr = (uint32_t)((g.cols + LT_VM_V - 1) / LT_VM_V);
+                int u = 1;
+                while (u < 8 && cpr > 32u * u) u *= 2;  // (the executor's choice: one warp per row where it fits)
+                jp->row_u = u;
+            }
+            if (jit_supported(*jp)) L.jit_program = std::move(jp);
+            // a long-row group is only worth keeping fused if its kernel is there when the flush runs
+            if (L.jit_program && g.long_row && c->opt.specialise == 1) {
+                L.jit = jit_request(*L.jit_program, true);
+                if (!L.jit || L.jit->state.load() != 1) L.jit_failed = true;
+            }
+        }
+        const bool long_ok = L.compiled >= 0 || (L.jit && !L.jit_failed);
+        if (g.long_row && (!long_ok || !c->opt.compiled)) unfused_long_row = true;
     }
     if (unfused_long_row) {
         // Only the kernels instantiated at build time walk a long row in slices.  A long-row group without one is
@@ -1308,6 +1332,10 @@ std::string describe_plan(const Plan &plan) {
             for (const LtIns &in : g.ins) key += " " + std::to_string(in.op) + ":" + std::to_string(in.imm);
             s += key + "\n";
             s += std::string("  compiled: ") + (L.compiled >= 0 ? lt_compiled_name(L.compiled) : "no") + "\n";
+            if (L.jit_program) {
+                const int st = L.jit ? L.jit->state.load() : 2;
+                s += std::string("  specialised at run time: ") + (L.jit_failed || st < 0 ? "failed" : st == 1 ? "ready" : st == 0 ? "being compiled" : "not requested yet") + "\n";
+            }
         }
         for (size_t q = 0; q < g.io.size(); ++q) {
             const IoRef &io = g.io[q];

@@ -8,7 +8,17 @@
 // reaches straight-line code that names its registers statically -- a register file
 // indexed at run time would live in local memory.
 #pragma once
+#ifdef __CUDACC_RTC__
+// the run-time compiler has no standard headers: the fixed-width names this file and the shells use
+typedef unsigned char uint8_t;
+typedef unsigned short uint16_t;
+typedef unsigned int uint32_t;
+typedef unsigned long long uint64_t;
+typedef int int32_t;
+typedef long long int64_t;
+#else
 #include <stdint.h>
+#endif
 
 #define LT_VM_V 8          // lanes per chunk
 #define LT_EW_THREADS 256  // CTA size of the elementwise and multi-tensor kernels

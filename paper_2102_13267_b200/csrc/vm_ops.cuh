@@ -1,17 +1,28 @@
 // Per-lane arithmetic of the register machine (vm.h), shared by the interpreter kernels and the
 // ahead-of-time compiled programs: one function per opcode family, one rounding per traced op.
 #pragma once
-#include <cuda_bf16.h>
+#ifndef __CUDACC_RTC__
 #include <cuda_runtime.h>
 #include <stdint.h>
+#endif
 
 #include "vm.h"
+
+#define LT_INF __int_as_float(0x7f800000)
 
 namespace {
 
 // ---------------------------------------------------------------------- math
 __device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
 __device__ __forceinline__ uint32_t f2u(float f) { return __float_as_uint(f); }
+
+// binary32 -> bfloat16, round to nearest even (the conversion instruction; NaN stays NaN)
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float round_bf16(float x) { return __uint_as_float(pack_bf16x2(0.0f, x) & 0xffff0000u); }
 
 __device__ __forceinline__ float max_nan(float a, float b) {
     float r;
@@ -107,7 +118,7 @@ __device__ __forceinline__ float un(float x) {
         float inner = k * fmaf(0.044715f * x, x * x, x);
         float th = FAST ? tanh_approx(inner) : tanhf(inner);
         return 0.5f * x * (1.0f + th);
-    } else if constexpr (OP == OP_U_RBF16) return __bfloat162float(__float2bfloat16_rn(x));
+    } else if constexpr (OP == OP_U_RBF16) return round_bf16(x);
     else if constexpr (OP == OP_U_INEG) return u2f(0u - f2u(x));
     else if constexpr (OP == OP_U_IABS) return u2f((uint32_t)abs((int32_t)f2u(x)));
     else if constexpr (OP == OP_U_NOT) return u2f(f2u(x) == 0u ? 1u : 0u);

@@ -461,6 +461,7 @@ def test_long_row_groups_fused_when_listed_and_split_otherwise():
     from workloads import idioms
 
     ctx = lt.LazyContext(device=None)
+    ctx.set_option("specialise", 0)
     x = fake(ctx, (4, 16384), "bf16")
     y = idioms.softmax(ctx, x, cols=16384)
     ctx.barrier()
@@ -598,3 +599,30 @@ def test_reshape_that_keeps_rows_and_columns_is_folded_into_the_program(ctx):
     ctx.barrier()
     assert ctx.stats()["launches_view"] == 1
     del y, z
+
+
+# ------------------------------------------------------------------ run-time specialisation
+def test_run_time_specialiser_builds_the_shells_for_an_unlisted_program():
+    """With specialise=1 a long-row group that has no kernel in the table stays fused, because its kernel is built
+    while the graph is planned.  The run-time compiler needs no GPU, so this runs here: it shows that the device
+    headers are self-contained and that the program's table entry is generated correctly."""
+    ctx = lt.LazyContext(device=None)
+    ctx.set_option("specialise", 1)
+    z = fake(ctx, (4, 16384))
+    d = ctx.op("abs", ctx.op("sub", z, ctx.op("row_max", z)))
+    w = ctx.op("div", d, ctx.op("add", ctx.op("row_sum", d), ctx.scalar(3.0)))
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    if "specialised at run time" not in plan:
+        pytest.skip("the run-time compiler library is not installed")
+    assert plan.count("launch ") == 1 and "launch 0: row" in plan and "specialised at run time: ready" in plan, plan
+    assert ctx.stats()["launches_reduce"] == 0
+    # with specialise=0 the same graph is split
+    other = lt.LazyContext(device=None)
+    other.set_option("specialise", 0)
+    z = fake(other, (4, 16384))
+    d = other.op("abs", other.op("sub", z, other.op("row_max", z)))
+    w2 = other.op("div", d, other.op("add", other.op("row_sum", d), other.scalar(3.0)))
+    other.barrier()
+    assert other.stats()["launches_reduce"] == 2
+    del w, w2
