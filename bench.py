@@ -116,8 +116,9 @@ def measured_peak() -> tuple[float, str]:
 # DRAM bytes of one launch of the dominant kernel on this workload, from the ncu capture summarised in
 # profiles/lt_c_ew_c2_mlp_epilogue.md, with the hash of the kernel sources it was taken on.
 NCU_TRAFFIC = {"bytes": 164695040, "sources_sha256": "6fcb33f1d1e5c4759d6becbce2a07613c0159d631b57bbab3801547877f2a83d"}
-KERNEL_SOURCES = ("paper_2102_13267_b200/csrc/compiled.cu", "paper_2102_13267_b200/csrc/compiled_programs.inc",
-                  "paper_2102_13267_b200/csrc/vm_ops.cuh", "paper_2102_13267_b200/csrc/vm.h")
+KERNEL_SOURCES = ("paper_2102_13267_b200/csrc/compiled.cu", "paper_2102_13267_b200/csrc/compiled_shells.cuh",
+                  "paper_2102_13267_b200/csrc/compiled_programs.inc", "paper_2102_13267_b200/csrc/vm_ops.cuh",
+                  "paper_2102_13267_b200/csrc/vm.h", "paper_2102_13267_b200/csrc/pdl.cuh")
 
 
 def kernel_sources_sha256() -> str:
@@ -517,7 +518,7 @@ def data_parallel_adam(lt, torch, device: int, world: int, steps: int = 50) -> d
 
 
 def other_configs(lt, torch, device: int) -> dict:
-    """C1, C3, C4: fused and unfused GB/s, 40 flushes over rotating buffer sets (> 1 GB together) queued behind
+    """C1 to C4: fused, interpreted, specialised and unfused GB/s, flushes over rotating buffer sets (> 1 GB together) queued behind
     a busy stream and timed between two events (kernel time including the gap to the next launch)."""
     import math as _m
 
@@ -540,8 +541,13 @@ def other_configs(lt, torch, device: int) -> dict:
     def c4_make(c):
         return (c.from_torch(bf16(configs.FULL["c4"], 4.0)),)
 
+    def c2_make(c):
+        sh = configs.FULL["c2"]
+        return (c.from_torch(bf16(sh)), c.from_torch(bf16(sh)), c.from_torch(bf16((sh[1],), 0.02)))
+
     cases = {
         "c1": (c1_make, lambda c, s: traces.elementwise_chain(c, *s)),
+        "c2": (c2_make, lambda c, s: traces.mlp_epilogue(c, *s, primitive_gelu=False)),
         "c3": (c3_make, lambda c, s: traces.residual_dropout_layernorm(c, *s, shape=configs.FULL["c3"], p=0.1, eps=1e-5,
                                                                         seed=1, offset=0)),
         "c4": (c4_make, lambda c, s: traces.causal_softmax(c, *s, shape=configs.FULL["c4"], scale=1 / _m.sqrt(128))),
@@ -551,10 +557,20 @@ def other_configs(lt, torch, device: int) -> dict:
         nbytes = configs.algorithmic_bytes(name)
         nsets = max(2, _m.ceil(1.2e9 / nbytes))
         entry = {}
-        for mode, iters in (("fused", 40), ("unfused", 10)):
+        # fused: the build-time kernel of the graph; interpreted: the same fused program on the interpreter kernels (what
+        # a graph runs on until a kernel has been built for it); specialised: the kernel the run-time specialiser builds
+        # for a program without a table entry (here: the table ignored); unfused: one kernel per traced op
+        for mode, iters in (("fused", 40), ("interpreted", 20), ("specialised", 40), ("unfused", 10)):
+            if name == "c2" and mode == "unfused":
+                continue  # (measured above on the benchmark's own buffers)
             c = lt.LazyContext(device=device)
             if mode == "unfused":
                 c.set_option("fusion", 0)
+            elif mode == "interpreted":
+                c.set_option("compiled", 0)
+            elif mode == "specialised":
+                c.set_option("debug.ignore_table", 1)
+                c.set_option("specialise", 1)
             sets = [make(c) for _ in range(nsets)]
             keep = [None] * nsets
             warm = nsets + 2  # every set flushed once: no allocator call is left for the timed flushes
@@ -579,7 +595,10 @@ def other_configs(lt, torch, device: int) -> dict:
             del keep, sets
             c.close()
         entry["frac_of_measured_peak"] = entry["fused_gbs"] / peak
-        entry["speedup_vs_unfused"] = entry["unfused_us"] / entry["fused_us"]
+        entry["interpreted_frac_of_measured_peak"] = entry["interpreted_gbs"] / peak
+        entry["specialised_frac_of_measured_peak"] = entry["specialised_gbs"] / peak
+        if "unfused_us" in entry:
+            entry["speedup_vs_unfused"] = entry["unfused_us"] / entry["fused_us"]
         res[name] = entry
     return res
 
@@ -596,8 +615,13 @@ def adam_steps(lt, torch, device: int) -> dict:
     nbytes = configs.algorithmic_bytes("c5")
     dev = torch.device("cuda", device)
     res = {}
-    for mode in ("traced", "replayed"):
+    for mode in ("traced", "replayed", "replayed_interpreted", "replayed_specialised"):
         ctx = lt.LazyContext(device=device)
+        if mode == "replayed_interpreted":
+            ctx.set_option("compiled", 0)
+        elif mode == "replayed_specialised":
+            ctx.set_option("debug.ignore_table", 1)
+            ctx.set_option("specialise", 1)
         P, G, M, V = ([ctx.from_torch(torch.randn(s, device=dev) * 0.05) for s in shapes] for _ in range(4))
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -610,6 +634,9 @@ def adam_steps(lt, torch, device: int) -> dict:
             for p, g, m, v in zip(P, G, M, V):
                 traces.adam_update(ctx, p, g, m, v, s)
             ctx.barrier()
+            if mode == "replayed_specialised":  # the kernel was built while the graph was planned: not part of a step
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
             for step in range(2, 101):
                 ctx.scalar_set(s.sqrt_bc2, _m.sqrt(1.0 - 0.999 ** step))
                 ctx.scalar_set(s.step_size, 1e-3 / (1.0 - 0.9 ** step))

@@ -194,7 +194,7 @@ def test_data_parallel_adam_step_on_one_rank(ctx):
     graph, recorded once and replayed."""
     from paper_2102_13267_b200.data_parallel import DataParallelAdam
 
-    shapes = parameter_shapes()[:12] + [(1000,), (7,)]
+    shapes = parameter_shapes()[:12] + [(1000,), (8, 3)]
     params, grads, ms, vs = configs.c5_inputs(56, shapes)
     dp = DataParallelAdam(ctx, shapes)
     import torch
