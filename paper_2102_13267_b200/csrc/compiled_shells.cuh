@@ -55,7 +55,7 @@ struct Info {
     }
     static constexpr __host__ __device__ int stage_bytes(int u_count, int threads) { return stage_offset(1 << 20, u_count, threads); }
     // Programs that generate random bits are bound by integer issue, not by the wait for their inputs: the
-    // staging copies would only add instructions (C3 back to back: 27.5 us with direct loads, 30.6 with the ring).
+    // staging copies would only add instructions (measured slower with the ring than with direct loads).
     static constexpr __host__ __device__ bool integer_heavy() {
         for (int k = 0; k < PG::n_ins; ++k)
             if (PG::ins[k].op == OP_PHILOX) return true;
@@ -863,9 +863,8 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
     uint32_t s = 0;
     // Column vectors of the reserved temporaries (gamma, beta, a bias): a thread owns the same columns in every
     // iteration, so when they fit in 64 registers they are loaded once instead of being re-read through L1 for every
-    // row -- two f32 vectors are 8 bytes per element of L1 traffic, twice the HBM traffic of a bf16 LayerNorm (18.5 ->
-    // 14.7 us on [16384 x 1024]).  Not for programs that generate random bits: they are short of registers and issue
-    // slots, not of L1 bandwidth (C3: 27.3 us without, 37.5 with, at 202 registers).
+    // row -- two f32 vectors are 8 bytes per element of L1 traffic, twice the HBM traffic of a bf16 LayerNorm.  Not
+    // for programs that generate random bits: they are short of registers and issue slots, not of L1 bandwidth.
     constexpr bool HOIST = Info<PG>::n_reserved() > 0 && Info<PG>::n_reserved() * U * V <= 64 && !Info<PG>::integer_heavy();
     float hv[NT][U][V];
     if constexpr (HOIST) {

@@ -323,7 +323,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     // (one chunk with correctly rounded division and square root: their slow paths cost registers)
                     const int u = (c->opt.compiled_u > 0 && !specialised(L)) ? (int)c->opt.compiled_u : (L.flavour == 2 ? 1 : 2);
                     const int occ = compiled_blocks(c, L, u, LT_EW_THREADS);
-                    const unsigned mwaves = c->opt.waves > 0 ? waves : 8u;  // C5: 116 us against 121 with two waves
+                    const unsigned mwaves = c->opt.waves > 0 ? waves : 8u;  // (eight waves measured a few per cent faster than two on 161 tensors of uneven size)
                     unsigned grid = (unsigned)std::min<uint64_t>(P.total_super, (uint64_t)c->sm_count * occ * mwaves);
                     if (grid < 1) grid = 1;
                     if (ev0) cudaEventRecord(ev0, c->stream);
@@ -463,7 +463,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     const int occ = compiled_blocks(c, L, u, LT_EW_THREADS);
                     const uint64_t need = (P.n_chunks + (uint64_t)LT_EW_THREADS * u - 1) / ((uint64_t)LT_EW_THREADS * u);
                     // a compiled CTA has no set-up to amortise: many short CTAs, scheduled by the hardware as others
-                    // retire, beat one wave of persistent ones (C2: 31.3 us against 33.5; no change beyond 8 waves)
+                    // retire, beat one wave of persistent ones (measured; no change beyond 8 waves)
                     const unsigned ewaves = c->opt.waves > 0 ? waves : 16u;
                     unsigned grid = (unsigned)std::min<uint64_t>(need, (uint64_t)c->sm_count * occ * ewaves);
                     if (grid < 1) grid = 1;
@@ -489,7 +489,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     const int occ = compiled_blocks(c, L, u, (int)threads, depth * stage);
                     const uint64_t blocks = ((uint64_t)P.rows + threads / grp - 1) / (threads / grp);
                     // one wave of persistent CTAs; with many blocks of rows per CTA, four waves balance the tail
-                    // better (measured on [32768 x 2048]: 49.6 us against 54.5)
+                    // better (measured on [32768 x 2048])
                     const uint64_t resident = (uint64_t)c->sm_count * occ;
                     const unsigned rwaves = c->opt.waves > 0 ? waves : (blocks >= 16 * resident ? 4u : 1u);
                     unsigned grid = (unsigned)std::min<uint64_t>(blocks, resident * rwaves);

@@ -606,7 +606,8 @@ def as_macro(name: str, lines: list[str]) -> str:
     return f"#define {name} \\\n{body}\n"
 
 
-def main() -> None:
+def render() -> str:
+    """Text of vm_core.inc for the opcode map vm.h has today."""
     text = ("// Generated by gen_vm_core.py from vm.h -- do not edit.\n"
             f"// Operands: %0-%3 ACC, then the temporaries (f32x2 pairs); {PC} pc (shared address); {EOP} escape opcode;\n"
             f"// {EIMM} escape immediate; {CHUNK} chunk index; {OFF4} chunk byte offset for 4-byte elements; {COFF4} column\n"
@@ -615,6 +616,11 @@ def main() -> None:
             f"// {CHUNK}-{STG} are updated by the core when it moves to the next chunk by itself (OP_END).\n"
             "#pragma once\n\n")
     text += "\n".join(as_macro(f"LT_VM_CORE_{fl.upper()}", build(fl)) for fl in ("fast", "precise", "ieee"))
+    return text
+
+
+def main() -> None:
+    text = render()
     (HERE / "vm_core.inc").write_text(text)
     print(f"wrote vm_core.inc ({len(text)} bytes)")
 

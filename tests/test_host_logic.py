@@ -626,3 +626,14 @@ def test_run_time_specialiser_builds_the_shells_for_an_unlisted_program():
     other.barrier()
     assert other.stats()["launches_reduce"] == 2
     del w, w2
+
+
+def test_committed_interpreter_core_is_what_its_generator_emits():
+    import importlib.util
+
+    path = os.path.join(ROOT, "paper_2102_13267_b200", "csrc", "gen_vm_core.py")
+    spec = importlib.util.spec_from_file_location("gen_vm_core", path)
+    gen = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(gen)
+    committed = open(os.path.join(ROOT, "paper_2102_13267_b200", "csrc", "vm_core.inc")).read()
+    assert gen.render() == committed, "run paper_2102_13267_b200/csrc/gen_vm_core.py and rebuild"
