@@ -367,6 +367,7 @@ struct Machine {
         constexpr int cls = PG::cls[SLOT], sh = esz_shift(PG::dtype[SLOT]);
         const char *base = reinterpret_cast<const char *>(ptr(SLOT));
         if constexpr (cls == LT_CLS_FULL) return base + (LT_CHECKED(ck.flat0[u], V, ptr.extent(cls)) << sh);
+        else if constexpr (cls == LT_CLS_PITCHED) return base + (((uint64_t)ck.row[u] * ptr.pitch(SLOT) + ck.col0[u]) << sh);
         else if constexpr (cls == LT_CLS_COLVEC) return base + (LT_CHECKED((uint64_t)ck.col0[u], V, ptr.extent(cls)) << sh);
         else if constexpr (cls == LT_CLS_ROWVEC) return base + (LT_CHECKED((uint64_t)ck.row[u], 1, ptr.extent(cls)) << sh);
         else return base;
@@ -377,9 +378,9 @@ struct Machine {
     __device__ __forceinline__ void load_now(float (&d)[V], int u) const {
         constexpr int cls = PG::cls[SLOT], dt = PG::dtype[SLOT];
         const char *p = address<SLOT>(u);
-        if constexpr (cls <= LT_CLS_COLVEC) {
+        if constexpr (cls <= LT_CLS_COLVEC || cls == LT_CLS_PITCHED) {
             Raw r;
-            raw_load<dt>(r, p, false);
+            raw_load<dt>(r, p, cls == LT_CLS_PITCHED);  // (a slice is streamed like any full-class operand)
             raw_widen<dt>(d, r);
         } else {
             float x;
@@ -748,6 +749,7 @@ struct ScalK {
 struct PtrK {
     const LtKParams &P;
     __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[s]; }
+    __device__ __forceinline__ uint32_t pitch(uint32_t s) const { return P.pitch[s]; }
     // elements a slot of the class holds (bounds checks of the debug build)
     __device__ __forceinline__ uint64_t extent(int cls) const {
         return cls == LT_CLS_FULL ? P.n : cls == LT_CLS_COLVEC ? P.cols : cls == LT_CLS_ROWVEC ? P.rows : 1;
@@ -762,6 +764,7 @@ struct PtrM {
     uint32_t base;
     uint32_t numel;
     __device__ __forceinline__ uint64_t operator()(uint32_t s) const { return P.ptr[base + s]; }
+    __device__ __forceinline__ uint32_t pitch(uint32_t) const { return 0; }
     __device__ __forceinline__ uint64_t extent(int) const { return numel; }
 };
 

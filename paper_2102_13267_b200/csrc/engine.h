@@ -109,6 +109,8 @@ struct IoRef {
     uint8_t cls;
     uint32_t index;   // parameter ordinal / output index / temporary index
     uint32_t cnode;   // canonical node the slot carries
+    uint32_t pitch = 0;    // LT_CLS_PITCHED: elements between rows of the buffer the slice is read from
+    uint64_t offset = 0;   // elements from the start of the buffer to the operand's first element (a slice read in place)
 };
 
 enum : uint8_t { K_EW = 0, K_ROW = 1, K_MULTI = 2, K_RED = 3, K_VIEW = 4 };  // K_RED: a reduction that runs as a kernel of its own (reduce.cu); K_VIEW: a shape operation (views.cu)

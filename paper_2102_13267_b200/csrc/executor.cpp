@@ -151,8 +151,9 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
             if (L.kind != K_ROW || !g.long_row) continue;
             bool ok = c->opt.compiled && (L.compiled >= 0 || (L.jit && !L.jit_failed)) && (g.cols % LT_VM_V) == 0;
             for (size_t q = 0; q < g.io.size() && ok; ++q)
-                if (g.io[q].kind == IO_PARAM && g.io[q].cls <= LT_CLS_COLVEC)
-                    ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index], g.io[q].dtype);
+                if (g.io[q].kind == IO_PARAM && (g.io[q].cls <= LT_CLS_COLVEC || g.io[q].cls == LT_CLS_PITCHED))
+                    ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index] + g.io[q].offset * dtype_size(g.io[q].dtype), g.io[q].dtype) &&
+                         aligned_for((uint64_t)g.io[q].pitch * dtype_size(g.io[q].dtype), g.io[q].dtype);
             if (!ok) {
                 if (needs_split) {
                     *needs_split = true;
@@ -231,7 +232,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
 
     auto resolve = [&](const IoRef &io) -> uint64_t {
         void *p = io.kind == IO_PARAM ? c->param_ptr[io.index] : io.kind == IO_OUTPUT ? c->out_ptr[io.index] : c->temp_ptr[io.index];
-        return (uint64_t)(uintptr_t)p;
+        return (uint64_t)(uintptr_t)p + io.offset * dtype_size(io.dtype);  // (offset: a slice read in place)
     };
 
     const unsigned waves = (unsigned)std::max<int64_t>(1, c->opt.waves);
@@ -456,8 +457,10 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                 // compiled kernel: needs 128-bit accesses everywhere (aligned pointers, whole chunks)
                 bool ok = (L.kind == K_EW && !P.rowcol) ? (P.n % LT_VM_V) == 0 : (P.cols % LT_VM_V) == 0;
                 ok = ok && P.n_chunks < (1ull << 31);
-                for (size_t s = 0; s < g.io.size() && ok; ++s)
-                    if (g.io[s].cls <= LT_CLS_COLVEC) ok = aligned_for(P.ptr[s], g.io[s].dtype);
+                for (size_t s = 0; s < g.io.size() && ok; ++s) {
+                    if (g.io[s].cls <= LT_CLS_COLVEC || g.io[s].cls == LT_CLS_PITCHED) ok = aligned_for(P.ptr[s], g.io[s].dtype);
+                    if (ok && g.io[s].cls == LT_CLS_PITCHED) ok = aligned_for((uint64_t)g.io[s].pitch * dtype_size(g.io[s].dtype), g.io[s].dtype);
+                }
                 if (ok && L.kind == K_EW) {
                     const int u = (c->opt.compiled_u > 0 && !specialised(L)) ? (int)c->opt.compiled_u : 1;
                     const int occ = compiled_blocks(c, L, u, LT_EW_THREADS);

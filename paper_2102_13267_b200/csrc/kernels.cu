@@ -50,6 +50,7 @@ struct EnvK {
     __device__ __forceinline__ uint64_t ptr(uint32_t s) const { return P.ptr[s]; }
     __device__ __forceinline__ uint32_t dtype(uint32_t s) const { return P.io_dtype[s]; }
     __device__ __forceinline__ uint32_t cls(uint32_t s) const { return P.io_class[s]; }
+    __device__ __forceinline__ uint32_t pitch(uint32_t s) const { return P.pitch[s]; }
 };
 
 struct EnvM {
@@ -59,6 +60,7 @@ struct EnvM {
     __device__ __forceinline__ uint64_t ptr(uint32_t s) const { return P.ptr[base + s]; }
     __device__ __forceinline__ uint32_t dtype(uint32_t s) const { return P.io_dtype[s]; }
     __device__ __forceinline__ uint32_t cls(uint32_t) const { return LT_CLS_FULL; }
+    __device__ __forceinline__ uint32_t pitch(uint32_t) const { return 0; }
 };
 
 // Random bits of the V lanes whose flat indices start at flat0 (element i uses word i mod 4 of
@@ -119,7 +121,7 @@ template <class Env>
 __device__ __forceinline__ void load_raw(float (&d)[V], const Env &E, uint32_t slot, const Chunk &ck) {
     const uint32_t dt = E.dtype(slot), cls = E.cls(slot);
     const char *base = reinterpret_cast<const char *>(E.ptr(slot));
-    if (cls >= LT_CLS_ROWVEC) {  // one element, replicated in storage format
+    if (cls == LT_CLS_ROWVEC || cls == LT_CLS_SCALAR) {  // one element, replicated in storage format
         const uint64_t idx = cls == LT_CLS_ROWVEC ? (ck.row_ok ? ck.row : 0) : 0;
         if (dt == LT_ST_BF16) {
             uint32_t h = __ldg(reinterpret_cast<const unsigned short *>(base) + idx);
@@ -138,7 +140,8 @@ __device__ __forceinline__ void load_raw(float (&d)[V], const Env &E, uint32_t s
         return;
     }
     const bool colvec = cls == LT_CLS_COLVEC;
-    const uint64_t idx = colvec ? (uint64_t)ck.col0 : ck.flat0;
+    // (pitched: a slice of wider rows read in place -- row * pitch + column)
+    const uint64_t idx = colvec ? (uint64_t)ck.col0 : cls == LT_CLS_PITCHED ? (uint64_t)(ck.row_ok ? ck.row : 0) * E.pitch(slot) + ck.col0 : ck.flat0;
     const char *p = base + (idx << esz_log2(dt));
     const uintptr_t need = dt == LT_ST_U8 ? 7u : 15u;
     if (ck.nvalid == V && (reinterpret_cast<uintptr_t>(p) & need) == 0) {

@@ -24,6 +24,7 @@ struct PNode {
     bool leaf = false;   // device data or scalar
     bool absorbed = false;
     bool reduce = false;
+    bool in_place_slice = false;  // a narrow of a device-data leaf that its consumers read in place (pitched / offset loads)
     bool foreign = false;  // runs as a kernel of its own (column / whole-tensor reduction, isolated long row reduction)
     bool needs_store = false;
     int temp = -1;       // temporary buffer index when stored but not an output
@@ -134,7 +135,24 @@ struct CodeGen {
         io.dtype = n.dtype;
         io.cls = (uint8_t)cls_of(v);
         io.cnode = v;
-        if (n.op == N_DEVICE_DATA) {
+        if (n.op == LT_OP_NARROW && pn[v].in_place_slice) {
+            // a slice read in place: the parameter it is cut from, an offset, and a row pitch when rows are not contiguous
+            const CNode &base = cg.nodes[n.in[0]];
+            io.kind = IO_PARAM;
+            io.index = (uint32_t)base.param;
+            const uint64_t base_cols = (uint64_t)base.dims[base.rank - 1];
+            if (n.attr0 == n.rank - 1 && n.rank > 0 && (uint64_t)n.dims[n.rank - 1] != base_cols) {
+                io.offset = (uint64_t)n.attr1;
+                if (io.cls == LT_CLS_FULL && g.rows > 1) {
+                    io.cls = LT_CLS_PITCHED;
+                    io.pitch = (uint32_t)base_cols;
+                }
+            } else {
+                uint64_t inner = 1;
+                for (int d = 1; d < n.rank; ++d) inner *= (uint64_t)n.dims[d];
+                io.offset = (uint64_t)n.attr1 * inner;
+            }
+        } else if (n.op == N_DEVICE_DATA) {
             io.kind = IO_PARAM;
             io.index = (uint32_t)n.param;
         } else if (n.output >= 0) {
@@ -144,7 +162,7 @@ struct CodeGen {
             io.kind = IO_TEMP;
             io.index = 0;  // patched once temporaries are numbered
         }
-        if (io.cls == LT_CLS_COLVEC || io.cls == LT_CLS_ROWVEC) needs_rowcol = true;
+        if (io.cls == LT_CLS_COLVEC || io.cls == LT_CLS_ROWVEC || io.cls == LT_CLS_PITCHED) needs_rowcol = true;
         slot_of[v] = (int)g.io.size();
         g.io.push_back(io);
         return slot_of[v];
@@ -619,7 +637,7 @@ void emission_list(const Canonical &cg, const std::vector<PNode> &pn, const Grou
 uint64_t io_bytes(const Group &g, const IoRef &io) {
     uint64_t es = dtype_size(io.dtype);
     switch (io.cls) {
-    case LT_CLS_FULL: return g.rows * g.cols * es;
+    case LT_CLS_FULL: case LT_CLS_PITCHED: return g.rows * g.cols * es;
     case LT_CLS_COLVEC: return g.cols * es;
     case LT_CLS_ROWVEC: return g.rows * es;
     default: return es;
@@ -723,6 +741,24 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
         const PNode &src = pn[n.in[0]];
         const bool same_domain = n.op == LT_OP_RESHAPE && src.rows == pn[i].rows && src.cols == pn[i].cols;
         pn[i].foreign = !(same_domain && fuse);
+        // A slice of materialised data along the last or the first dimension is a block of rows at a fixed pitch (or one
+        // contiguous range): consumers that compute over the slice's own [rows, cols] read it in place.
+        if (fuse && n.op == LT_OP_NARROW && cg.nodes[n.in[0]].op == N_DEVICE_DATA && n.output < 0 && !pn[i].consumers.empty() &&
+            (n.attr0 == n.rank - 1 || n.attr0 == 0) && src.cols < (1ull << 32)) {
+            bool all = true;
+            for (uint32_t q : pn[i].consumers) {
+                const CNode &qn = cg.nodes[q];
+                const bool elementwise = (qn.op >= LT_OP_ADD && qn.op <= LT_OP_NOT) || qn.op == LT_OP_CONVERT || is_reduce(qn.op);
+                uint64_t qr = pn[q].rows, qc = pn[q].cols;
+                if (is_reduce(qn.op)) qr = pn[i].rows, qc = pn[i].cols;
+                if (!elementwise || qr != pn[i].rows || qc != pn[i].cols) all = false;
+            }
+            if (all) {
+                pn[i].in_place_slice = true;
+                pn[i].foreign = false;
+                pn[i].leaf = true;  // nothing computes it: it is an input like the buffer it points into
+            }
+        }
     }
     if (isolate_long_rows)
         for (size_t i = 0; i < N; ++i)
@@ -1171,7 +1207,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                         if (g.view_op != LT_OP_UPDATE_SLICE || rd.second != 0) { safe = false; break; }
                     } else if (rg == gi) {
                         const IoRef &ld = groups[rg].io[rd.second];
-                        if (ld.cls != LT_CLS_FULL) { safe = false; break; }
+                        if (ld.cls != LT_CLS_FULL || ld.offset != 0) { safe = false; break; }  // (a slice reads other elements than the store's)
                         // the load must come before the store in program order
                         int ld_pos = -1, st_pos = -1;
                         for (size_t q = 0; q < g.ins.size(); ++q) {
@@ -1225,6 +1261,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             for (size_t s = 0; s < g.io.size(); ++s) {
                 P.io_dtype[s] = g.io[s].dtype;
                 P.io_class[s] = g.io[s].cls;
+                P.pitch[s] = g.io[s].pitch;
             }
             P.n = g.rows * g.cols;
             P.rowcol = g.rowcol ? 1u : 0u;
@@ -1306,7 +1343,7 @@ std::string describe_plan(const Plan &plan) {
             s += buf;
         }
     static const char *kind[] = {"elementwise", "row", "multi", "reduce", "view"};
-    static const char *cls[] = {"full", "colvec", "rowvec", "scalar"};
+    static const char *cls[] = {"full", "colvec", "rowvec", "scalar", "pitched"};
     static const char *iok[] = {"param", "output", "temp"};
     for (size_t li = 0; li < plan.launches.size(); ++li) {
         const Launch &L = plan.launches[li];

@@ -50,7 +50,8 @@ struct LtIns {
 };
 
 // element classes of a pointer slot relative to the group's [rows, cols] domain
-enum { LT_CLS_FULL = 0, LT_CLS_COLVEC = 1, LT_CLS_ROWVEC = 2, LT_CLS_SCALAR = 3 };
+// LT_CLS_PITCHED: a full-class operand whose rows lie `pitch` elements apart (a slice of wider rows, read in place)
+enum { LT_CLS_FULL = 0, LT_CLS_COLVEC = 1, LT_CLS_ROWVEC = 2, LT_CLS_SCALAR = 3, LT_CLS_PITCHED = 4 };
 // storage dtypes (same numbering as lt_dtype)
 enum { LT_ST_F32 = 0, LT_ST_BF16 = 1, LT_ST_U8 = 2, LT_ST_I32 = 3, LT_ST_U32 = 4 };
 
@@ -129,6 +130,7 @@ struct LtKParams {
     uint8_t io_dtype[LT_VM_MAX_PTR];
     uint8_t io_class[LT_VM_MAX_PTR];
     uint8_t io_stage[LT_VM_MAX_PTR];  // first 16-byte piece of the slot in a staging buffer, 0xFF = not staged
+    uint32_t pitch[LT_VM_MAX_PTR];    // LT_CLS_PITCHED slots: elements between the starts of consecutive rows
     uint32_t stage_depth;   // staging buffers per thread (0 = loads go straight to registers)
     uint32_t stage_pieces;  // 16-byte pieces per staging buffer
     uint32_t n_ins;

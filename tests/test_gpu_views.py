@@ -147,3 +147,36 @@ def test_reshape_views(ctx):
     want = x0.reshape(4, 24)
     want = (want - want.max(axis=1, keepdims=True)).reshape(8, 12)
     np.testing.assert_array_equal(ox.array, want)
+
+
+@pytest.mark.parametrize("mode", ["interpreted", "specialised"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape,dim,start,length", [((64, 256), 1, 64, 128), ((37, 100), 1, 3, 40), ((64, 256), 0, 16, 8),
+                                                     ((5, 6, 64), 2, 8, 32), ((300, 1024), 1, 512, 256)])
+def test_slices_read_in_place_by_fused_groups(lt, mode, dtype, shape, dim, start, length):
+    """A narrow of materialised data feeding elementwise work and a row reduction: read with pitched (or offset) loads
+    inside the fused kernel, on the interpreter and on the run-time specialised shells."""
+    c = lt.LazyContext(device=0)
+    if mode == "interpreted":
+        c.set_option("compiled", 0)
+    else:
+        c.set_option("specialise", 1)
+    a = _data(shape, dtype, 77)
+    sl_shape = shape[:dim] + (length,) + shape[dim + 1:]
+    b = _data(sl_shape, dtype, 78)
+    O = EagerOracle()
+
+    def graph(B, x, y):
+        s = B.op("narrow", x, dim=dim, start=start, length=length)
+        t = B.op("convert", B.op("mul", s, y), dtype="f32")
+        return B.op("sub", t, B.op("row_max", t))
+
+    ref = graph(O, O.leaf(a, dtype), O.leaf(b, dtype))
+    out = graph(c, c.leaf(a, dtype), c.leaf(b, dtype))
+    c.barrier()
+    st = c.stats()
+    assert st["kernels_launched"] == 1 and st["launches_view"] == 0, (st, c.dump_plan())
+    if mode == "specialised" and "specialised at run time" in c.dump_plan() and sl_shape[-1] % 8 == 0 and (start * (2 if dtype == "bf16" else 4)) % 16 == 0:
+        assert st["launches_specialised"] == 1, c.dump_plan()
+    assert_matches(c.fetch(out), ref.array, "f32", f"in-place slice {shape} {dim} {start} {length} {dtype} {mode}")
+    c.close()

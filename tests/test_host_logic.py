@@ -637,3 +637,22 @@ def test_committed_interpreter_core_is_what_its_generator_emits():
     spec.loader.exec_module(gen)
     committed = open(os.path.join(ROOT, "paper_2102_13267_b200", "csrc", "vm_core.inc")).read()
     assert gen.render() == committed, "run paper_2102_13267_b200/csrc/gen_vm_core.py and rebuild"
+
+
+def test_slices_of_materialised_data_are_read_in_place(ctx):
+    x = fake(ctx, (64, 256))
+    y = fake(ctx, (64, 128))
+    out = ctx.op("mul", ctx.op("narrow", x, dim=1, start=64, length=128), y)       # columns 64..191 of every row
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("launch ") == 1 and "pitched param0" in plan and "copy kernel" not in plan, plan
+    head = ctx.op("add", ctx.op("narrow", x, dim=0, start=16, length=8), ctx.scalar(1.0))   # rows 16..23: one contiguous range
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("launch ") == 1 and "load f32 full param0" in plan and "copy kernel" not in plan, plan
+    # a slice that is itself a result, or that feeds a reduction kernel of its own, is copied
+    s = ctx.op("narrow", x, dim=1, start=0, length=8)
+    t = ctx.op("col_sum", ctx.op("narrow", x, dim=1, start=8, length=8))
+    ctx.barrier()
+    assert ctx.dump_plan().count("copy kernel: narrow") == 2
+    del out, head, s, t
