@@ -266,6 +266,7 @@ bool jit_load(JitKernel &k, int device, std::string *err) {
 }
 
 static void *fn_of(JitKernel &k, int device, int variant) {
+    std::lock_guard<std::mutex> g(k.load_lock);  // (contexts on other threads may be loading the same kernel on their device)
     auto it = k.loaded.find(device);
     return it == k.loaded.end() || !it->second.ok ? nullptr : it->second.fn[variant];
 }
