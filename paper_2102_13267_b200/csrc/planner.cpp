@@ -312,6 +312,7 @@ struct CodeGen {
             io.kind = IO_TEMP;
             io.index = 0;
         }
+        if (io.cls == LT_CLS_SCALAR && g.rows == 1) io.cls = LT_CLS_ROWVEC;  // the one value of a one-row group: row 0's
         if (io.cls == LT_CLS_COLVEC || io.cls == LT_CLS_SCALAR) {
             ok = false;  // native members are FULL or ROWVEC by construction
             return;

@@ -206,3 +206,57 @@ def test_bounded_wait_gives_up_and_is_reported(lt):
     c.barrier(blocking=True)  # reported once
     np.testing.assert_array_equal(c.fetch(x + 1.0), np.arange(64, dtype=np.float32).reshape(8, 8) + 1)
     c.close()
+
+
+def test_degenerate_and_mixed_cases(ctx):
+    O = EagerOracle()
+    g = rng.generator(90)
+    # a single long row; a long row next to short work in the same flush
+    x = rng.normal_f32(g, (1, 20000), 1.0)
+    y = rng.normal_f32(g, (33, 64), 1.0)
+    ox, gx, oy, gy = O.leaf(x, "f32"), ctx.leaf(x, "f32"), O.leaf(y, "f32"), ctx.leaf(y, "f32")
+    outs_o = [O.op("row_sum", ox), O.op("sub", ox, O.op("row_max", ox)), O.op("exp", oy), O.op("all_min", oy)]
+    outs_g = [ctx.op("row_sum", gx), ctx.op("sub", gx, ctx.op("row_max", gx)), ctx.op("exp", gy), ctx.op("all_min", gy)]
+    ctx.barrier()
+    for k, (r, t) in enumerate(zip(outs_o, outs_g)):
+        assert_matches(ctx.fetch(t), r.array, "f32", f"mixed flush output {k}")
+    # reductions of reductions, and a rank-0 result used twice
+    m = ctx.op("all_max", ctx.op("col_sum", gy))
+    mo = O.op("all_max", O.op("col_sum", oy))
+    z = ctx.op("mul", ctx.op("sub", gy, m), m)
+    zo = O.op("mul", O.op("sub", oy, mo), mo)
+    assert_matches(ctx.fetch(z), zo.array, "f32", "rank-0 result used twice")
+    assert_matches(ctx.fetch(m), mo.array, "f32", "rank-0 result fetched")
+
+
+def test_replay_of_a_graph_with_reduction_kernels_and_a_view(lt):
+    """lt_replay re-runs a plan that holds a column reduction (two stages through a plan temporary) and an in-place
+    update through a narrow."""
+    import torch
+
+    c = lt.LazyContext(device=0)
+    shape = (2000, 96)
+    x0 = rng.normal_f32(rng.generator(91), shape, 1.0)
+    xd = torch.from_numpy(x0).cuda()
+    x = c.from_torch(xd)
+    O = EagerOracle()
+    ox = O.leaf(x0, "f32")
+
+    def step(B, t):
+        centred = B.op("sub", t, B.op("mul", B.op("col_sum", t), B.scalar(1.0 / shape[0])))
+        v = B.view_narrow(t, 1, 32, 32)
+        B.assign(t, B.op("mul", centred, B.scalar(0.5)))
+        B.assign(v, B.op("add", v, B.scalar(1.0)))
+        return v
+
+    keep = step(c, x)
+    c.barrier()
+    ok = step(O, ox)
+    for _ in range(3):
+        c.replay()
+        step(O, ox)
+    st = c.stats()
+    assert st["replays"] == 3 and st["compiles"] == 1
+    assert_matches(c.fetch(x), ox.array, "f32", "base after three replays")
+    assert_matches(c.fetch(keep), np.ascontiguousarray(ok.array), "f32", "view after three replays")
+    c.close()

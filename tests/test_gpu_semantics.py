@@ -118,7 +118,7 @@ def test_iota_philox_and_reductions(ctx):
         got = ctx.fetch(ctx.op("philox_bits", shape=shape, seed=2**63 + 5, offset=2**40 + 3))
         assert_matches(got, ref.array, "u32", f"philox {shape}")
     g = rng.generator(24)
-    for shape in [(4, 8), (3, 40), (2, 3, 100), (5, 1), (2, 2048)]:
+    for shape in [(4, 8), (3, 40), (2, 3, 100), (5, 1), (2, 2048), (1, 64), (1, 1), (64,), (1, 9000)]:
         x = rng.normal_f32(g, shape, 3.0)
         ox, gx = both(ctx, O, x, "f32")
         for name in ("row_sum", "row_max", "row_min"):

@@ -133,3 +133,25 @@ def test_static_scratch_flush_refuses_what_it_cannot_place():
     ctx.barrier(blocking=True)
     assert float(bd[0]) == -2.0
     ctx.close()
+
+
+def test_static_scratch_holds_the_partials_of_a_reduction_kernel():
+    """A whole-tensor reduction runs in two stages through a temporary: with the allocation-free flush that temporary
+    lives in the fixed array too."""
+    import torch
+
+    import paper_2102_13267_b200 as lt
+    from oracle.eager import EagerOracle
+
+    ctx = lt.LazyContext(device=0)
+    xh, _ = _inputs()
+    xd = torch.from_numpy(xh).cuda()
+    x = ctx.from_torch(xd)
+    O = EagerOracle()
+    ox = O.leaf(xh, "f32")
+    for B, t in ((O, ox), (ctx, x)):
+        B.assign(t, B.op("sub", t, B.op("all_max", t)))
+    ctx.barrier_static_scratch(blocking=True)
+    assert ctx.device_ptr(x) == xd.data_ptr() and ctx.stats()["launches_reduce"] == 1
+    np.testing.assert_allclose(xd.cpu().numpy(), ox.array, rtol=1e-5, atol=1e-6)
+    ctx.close()
