@@ -16,6 +16,7 @@
 
 #include <condition_variable>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <deque>
 #include <map>
@@ -110,9 +111,66 @@ std::vector<std::pair<std::string, int>> variants_of(const JitProgram &p) {
     return v;
 }
 
+// ---- optional on-disk cache of the machine code (environment variable LT_KERNEL_CACHE = a directory)
+//
+// A file per (program, library sources): "<hash>.ltk" = magic, the two lowered kernel names, the machine code.  The
+// hash covers the program's generated table entry and the text of the device headers, so a rebuilt library with
+// changed shells never picks up stale code.  Files are written to a temporary name and renamed.
+
+uint64_t fnv1a(const std::string &s, uint64_t h = 1469598103934665603ull) {
+    for (unsigned char c : s) h = (h ^ c) * 1099511628211ull;
+    return h;
+}
+
+std::string cache_path(const std::string &src, const JitProgram &p) {
+    const char *dir = getenv("LT_KERNEL_CACHE");
+    if (!dir || !*dir) return "";
+    uint64_t h = fnv1a(src);
+    for (const char *t : {kSrcVm, kSrcVmOps, kSrcPdl, kSrcShells}) h = fnv1a(t, h);
+    h = fnv1a(std::string(p.long_row ? "L" : "R") + std::to_string(p.row_u), h);
+    char name[64];
+    snprintf(name, sizeof(name), "/%016llx.ltk", (unsigned long long)h);
+    return std::string(dir) + name;
+}
+
+bool cache_read(const std::string &path, JitKernel &k) {
+    FILE *f = fopen(path.c_str(), "rb");
+    if (!f) return false;
+    bool ok = false;
+    uint32_t head[4] = {0, 0, 0, 0};  // magic, length of name 0, of name 1, of the machine code
+    if (fread(head, sizeof(head), 1, f) == 1 && head[0] == 0x4b544c31u && head[1] < 4096 && head[2] < 4096 && head[3] > 0 &&
+        head[3] < (64u << 20)) {
+        k.entry[0].resize(head[1]);
+        k.entry[1].resize(head[2]);
+        k.cubin.resize(head[3]);
+        ok = (head[1] == 0 || fread(&k.entry[0][0], head[1], 1, f) == 1) && (head[2] == 0 || fread(&k.entry[1][0], head[2], 1, f) == 1) &&
+             fread(k.cubin.data(), head[3], 1, f) == 1;
+    }
+    fclose(f);
+    return ok;
+}
+
+void cache_write(const std::string &path, const JitKernel &k) {
+    const std::string tmp = path + ".tmp" + std::to_string((unsigned long long)(uintptr_t)&k);
+    FILE *f = fopen(tmp.c_str(), "wb");
+    if (!f) return;
+    const uint32_t head[4] = {0x4b544c31u, (uint32_t)k.entry[0].size(), (uint32_t)k.entry[1].size(), (uint32_t)k.cubin.size()};
+    bool ok = fwrite(head, sizeof(head), 1, f) == 1 && (k.entry[0].empty() || fwrite(k.entry[0].data(), k.entry[0].size(), 1, f) == 1) &&
+              (k.entry[1].empty() || fwrite(k.entry[1].data(), k.entry[1].size(), 1, f) == 1) && fwrite(k.cubin.data(), k.cubin.size(), 1, f) == 1;
+    ok = fclose(f) == 0 && ok;
+    if (ok) rename(tmp.c_str(), path.c_str());
+    else remove(tmp.c_str());
+}
+
 void compile(JitKernel &k) {
     const Api &a = api();
     const std::string src = program_struct(k.program);
+    const std::string cached = cache_path(src, k.program);
+    if (!cached.empty() && cache_read(cached, k)) {
+        k.log = "(machine code from " + cached + ")";
+        k.state.store(1);
+        return;
+    }
     const char *names[] = {"vm.h", "vm_ops.cuh", "pdl.cuh", "compiled_shells.cuh"};
     const char *texts[] = {kSrcVm, kSrcVmOps, kSrcPdl, kSrcShells};
     nvrtcProgram prog = nullptr;
@@ -144,6 +202,7 @@ void compile(JitKernel &k) {
         }
     }
     a.DestroyProgram(&prog);
+    if (ok && !cached.empty()) cache_write(cached, k);
     k.state.store(ok ? 1 : -1);
 }
 

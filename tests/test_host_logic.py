@@ -656,3 +656,35 @@ def test_slices_of_materialised_data_are_read_in_place(ctx):
     ctx.barrier()
     assert ctx.dump_plan().count("copy kernel: narrow") == 2
     del out, head, s, t
+
+
+def test_kernel_cache_directory_is_written_and_read(tmp_path, monkeypatch):
+    """LT_KERNEL_CACHE: the specialiser stores the machine code of a program in the directory and a later request
+    (here: another program identity is needed, so a second process is what really reuses it) finds the file."""
+    import subprocess
+    import sys
+
+    code = (
+        "import sys; sys.path.insert(0, %r)\n"
+        "import paper_2102_13267_b200 as lt\n"
+        "c = lt.LazyContext(device=None); c.set_option('specialise', 1)\n"
+        "z = c.from_device_ptr(1 << 30, 'f32', (4, 16384))\n"
+        "d = c.op('abs', c.op('sub', z, c.op('row_min', z)))\n"
+        "w = c.op('div', d, c.op('add', c.op('row_sum', d), c.scalar(5.0)))\n"
+        "c.barrier(); p = c.dump_plan()\n"
+        "print('READY' if 'specialised at run time: ready' in p else ('ABSENT' if 'specialised at run time' not in p else 'FAILED'))\n"
+    ) % ROOT
+    env = dict(os.environ, LT_KERNEL_CACHE=str(tmp_path))
+    import time
+    t0 = time.time()
+    first = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+    t1 = time.time()
+    if "ABSENT" in first.stdout:
+        pytest.skip("the run-time compiler library is not installed")
+    assert "READY" in first.stdout, first.stdout + first.stderr
+    files = list(tmp_path.glob("*.ltk"))
+    assert len(files) == 1 and files[0].stat().st_size > 10000
+    stamp = files[0].stat().st_mtime_ns
+    second = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+    assert "READY" in second.stdout, second.stdout + second.stderr
+    assert files[0].stat().st_mtime_ns == stamp and len(list(tmp_path.glob("*"))) == 1  # read, not rewritten
