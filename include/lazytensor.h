@@ -191,7 +191,10 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * time -- the same kernels, instantiated over the program by the CUDA run-time compiler on a worker thread while the
  * interpreter keeps serving the flushes; 1 = build it when the graph is planned and wait for it; 0 = never.  Absent,
  * silently, when the run-time compiler library cannot be loaded.  With the environment variable LT_KERNEL_CACHE set to a
- * directory, the machine code is also kept there and found again by later processes), "specialise_after" (3 default:
+ * directory, the machine code is also kept there and found again by later processes.  Of several installed copies of
+ * the run-time compiler the newest one whose code the driver can load is used; LT_NVRTC names a file instead.
+ * LT_KERNEL_LOG set: the compiler's log, with registers and shared memory of every kernel, goes to stderr),
+ * "specialise_after" (3 default:
  * flushes of a plan before mode 2 asks for the kernel),
  * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
  * line per flush and per replay; preset by the environment variable LT_LOG),

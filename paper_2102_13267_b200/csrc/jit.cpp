@@ -21,7 +21,9 @@
 #include <deque>
 #include <map>
 #include <mutex>
+#include <string>
 #include <thread>
+#include <vector>
 
 namespace lt {
 
@@ -31,6 +33,7 @@ namespace {
 
 struct Api {
     bool ok = false;
+    int compiler_version = 0;  // major * 1000 + minor * 10
     // NVRTC
     nvrtcResult (*CreateProgram)(nvrtcProgram *, const char *, const char *, int, const char *const *, const char *const *) = nullptr;
     nvrtcResult (*DestroyProgram)(nvrtcProgram *) = nullptr;
@@ -59,13 +62,41 @@ bool sym(void *lib, const char *name, F &fn) {
 const Api &api() {
     static Api a = [] {
         Api x;
-        void *rtc = nullptr;
-        for (const char *n : {"libnvrtc.so.12", "libnvrtc.so"})
-            if (!rtc) rtc = dlopen(n, RTLD_NOW | RTLD_LOCAL);
         void *drv = nullptr;
         for (const char *n : {"libcuda.so.1", "libcuda.so"})
             if (!drv) drv = dlopen(n, RTLD_NOW | RTLD_LOCAL);
+        int driver_version = 0;  // e.g. 12090; 0 = unknown (no driver here: anything may compile, nothing is loaded)
+        CUresult (*driver_get_version)(int *) = nullptr;
+        if (drv && sym(drv, "cuDriverGetVersion", driver_get_version)) driver_get_version(&driver_version);
+        // Several copies of the compiler can be installed (a toolkit's, and one bundled with a Python package that is
+        // already mapped under the same soname, which a bare name would resolve to).  Their register allocation
+        // differs measurably, so take the newest one the driver can load code from: LT_NVRTC names a file outright,
+        // else the toolkit directories are tried by path before the bare names.
+        std::vector<std::string> candidates;
+        if (const char *e = getenv("LT_NVRTC")) candidates.push_back(e);
+        else {
+            for (const char *var : {"CUDA_HOME", "CUDA_PATH"})
+                if (const char *e = getenv(var)) candidates.push_back(std::string(e) + "/lib64/libnvrtc.so.12");
+            candidates.push_back("/usr/local/cuda/lib64/libnvrtc.so.12");
+            candidates.push_back("libnvrtc.so.12");
+            candidates.push_back("libnvrtc.so");
+        }
+        void *rtc = nullptr;
+        int best = -1;
+        for (const std::string &n : candidates) {
+            void *h = dlopen(n.c_str(), RTLD_NOW | RTLD_LOCAL);
+            if (!h) continue;
+            nvrtcResult (*version)(int *, int *) = nullptr;
+            int major = 0, minor = 0;
+            const bool known = sym(h, "nvrtcVersion", version) && version(&major, &minor) == NVRTC_SUCCESS;
+            const int v = known ? major * 1000 + minor * 10 : 0;
+            if (v > best && (driver_version == 0 || v <= driver_version)) {
+                if (rtc) dlclose(rtc);
+                rtc = h, best = v;
+            } else dlclose(h);
+        }
         if (!rtc) return x;
+        x.compiler_version = best;
         bool ok = sym(rtc, "nvrtcCreateProgram", x.CreateProgram) && sym(rtc, "nvrtcDestroyProgram", x.DestroyProgram) &&
                   sym(rtc, "nvrtcCompileProgram", x.CompileProgram) && sym(rtc, "nvrtcAddNameExpression", x.AddNameExpression) &&
                   sym(rtc, "nvrtcGetLoweredName", x.GetLoweredName) && sym(rtc, "nvrtcGetCUBINSize", x.GetCUBINSize) &&
@@ -127,7 +158,7 @@ std::string cache_path(const std::string &src, const JitProgram &p) {
     if (!dir || !*dir) return "";
     uint64_t h = fnv1a(src);
     for (const char *t : {kSrcVm, kSrcVmOps, kSrcPdl, kSrcShells}) h = fnv1a(t, h);
-    h = fnv1a(std::string(p.long_row ? "L" : "R") + std::to_string(p.row_u), h);
+    h = fnv1a(std::string(p.long_row ? "L" : "R") + std::to_string(p.row_u) + "/" + std::to_string(api().compiler_version), h);
     char name[64];
     snprintf(name, sizeof(name), "/%016llx.ltk", (unsigned long long)h);
     return std::string(dir) + name;
@@ -181,8 +212,9 @@ void compile(JitKernel &k) {
     }
     const auto variants = variants_of(k.program);
     for (auto &v : variants) a.AddNameExpression(prog, v.first.c_str());
-    const char *opts[] = {"--gpu-architecture=sm_100a", "-std=c++17", "-default-device", "-diag-suppress=177"};
-    const nvrtcResult r = a.CompileProgram(prog, 4, opts);
+    // the log then carries the assembler's resource lines (registers, spills, shared memory) of every kernel
+    const char *opts[] = {"--gpu-architecture=sm_100a", "-std=c++17", "-default-device", "-diag-suppress=177", "--ptxas-options=-v"};
+    const nvrtcResult r = a.CompileProgram(prog, 5, opts);
     size_t n = 0;
     if (a.GetProgramLogSize(prog, &n) == NVRTC_SUCCESS && n > 1) {
         k.log.resize(n);
@@ -202,6 +234,7 @@ void compile(JitKernel &k) {
         }
     }
     a.DestroyProgram(&prog);
+    if (getenv("LT_KERNEL_LOG")) fprintf(stderr, "[lazytensor] specialised %s (compiler %d):\n%s\n", variants.empty() ? "" : variants[0].first.c_str(), a.compiler_version, k.log.c_str());
     if (ok && !cached.empty()) cache_write(cached, k);
     k.state.store(ok ? 1 : -1);
 }
