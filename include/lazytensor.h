@@ -55,8 +55,9 @@ typedef enum {
     LT_ERR_OOM = 6,           /* the allocator callback returned NULL                    */
     LT_ERR_CUDA = 7,          /* a CUDA runtime call failed (message has the CUDA text)  */
     LT_ERR_DEVICE_TIMEOUT = 8 /* a bounded device-side wait gave up: reported by the first blocking call
-                                 (lt_barrier with blocking set, lt_fetch) after a kernel that stages long
-                                 rows through shared memory ran out of polls on a copy's completion      */
+                                 (lt_barrier with blocking set, lt_fetch) after a long-row kernel ran out
+                                 of time waiting for a copy into shared memory, or for the partial results
+                                 of the other thread blocks of its cluster                                */
 } lt_status;
 
 typedef enum { LT_F32 = 0, LT_BF16 = 1, LT_U8 = 2, LT_I32 = 3, LT_U32 = 4 } lt_dtype;
@@ -198,8 +199,8 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * flushes of a plan before mode 2 asks for the kernel),
  * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
  * line per flush and per replay; preset by the environment variable LT_LOG),
- * "wait_limit_ms" (2000 default: how long a kernel that stages long rows through shared memory waits for one of
- * its asynchronous copies before it gives up, see LT_ERR_DEVICE_TIMEOUT),
+ * "wait_limit_ms" (2000 default: how long a long-row kernel waits for one of its asynchronous copies into shared
+ * memory, or for the other thread blocks of its cluster, before it gives up, see LT_ERR_DEVICE_TIMEOUT),
  * "pool_bytes" (4 GiB default: device blocks the library has released are kept, up to this total, and reused
  * by later flushes before the allocator is asked; 0 = return every block at once).
  * fusion, fast_math, horizontal and ieee are part of the cache key; the others act at launch time.
@@ -281,8 +282,9 @@ lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
  * Barrier (Section 4; mark_step / LazyTensorBarrier): materialise every live tensor that
  * has pending computation.  With `blocking` non-zero, return after the stream has drained.
  * Row reductions over more than 8192 columns: a group whose program has a kernel instantiated at build time
- * (softmax, LayerNorm, RMSNorm and the other listed groups) runs fused, one thread block per row walking it in
- * slices, when its inputs are 16-byte aligned and the row is a multiple of 8 elements; any other such graph runs
+ * (softmax, LayerNorm, RMSNorm and the other listed groups), or built by the run-time specialiser in mode 1, runs
+ * fused -- up to 65536 columns with a thread-block cluster holding the row in registers, beyond that one thread block
+ * per row walking it in slices -- when its inputs are 16-byte aligned and the row is a multiple of 8 elements; any other such graph runs
  * with each long reduction as a kernel of its own and the surrounding arithmetic as elementwise kernels.
  */
 lt_status lt_barrier(lt_ctx *ctx, int blocking);

@@ -174,7 +174,89 @@ cudaError_t long_occupancy(unsigned threads, size_t dyn, int *blocks) {
     }
 }
 
+// Cluster row kernel: launched with the cluster dimension and the programmatic-launch attribute; with no parameter
+// block, answers how many clusters the device holds at once instead
+template <class PG, int U, bool HS>
+cudaError_t rowc_do(const LtKParams *P, unsigned clusters, unsigned cluster_size, unsigned depth, uint64_t limit_ns, cudaStream_t stream,
+                    int *max_clusters) {
+    const size_t dyn = (size_t)depth * Info<PG>::stage_bytes(U, C_ROW_THREADS) + (HS ? (size_t)Info<PG>::n_reserved() * U * C_ROW_THREADS * 32u : 0u);
+    cudaError_t e = row_smem_attr((const void *)lt_c_rowc<PG, U, HS>, dyn);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((clusters ? clusters : 1u) * cluster_size);
+    cfg.blockDim = dim3(C_ROW_THREADS);
+    cfg.dynamicSmemBytes = dyn;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = LT_PDL;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (!P) {
+        cfg.numAttrs = 1;  // the occupancy query takes the cluster dimension only
+        return cudaOccupancyMaxActiveClusters(max_clusters, lt_c_rowc<PG, U, HS>, &cfg);
+    }
+    return cudaLaunchKernelEx(&cfg, lt_c_rowc<PG, U, HS>, *P, (uint32_t)depth, limit_ns);
+}
+
+// `shared_vectors`: column vectors of the program kept in shared memory (only instantiated for programs that have some)
+template <class PG>
+cudaError_t rowc_one(const LtKParams *P, int u, bool shared_vectors, unsigned clusters, unsigned cluster_size, unsigned depth, uint64_t limit_ns,
+                     cudaStream_t stream, int *max_clusters) {
+    if constexpr (PG::kind == 1) {
+        if constexpr (Info<PG>::n_reserved() > 0) {
+            if (shared_vectors) {
+                if (u >= 8) return rowc_do<PG, 8, true>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+                if (u >= 4) return rowc_do<PG, 4, true>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+                if (u >= 2) return rowc_do<PG, 2, true>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+                return rowc_do<PG, 1, true>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+            }
+        }
+        if (u >= 8) return rowc_do<PG, 8, false>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+        if (u >= 4) return rowc_do<PG, 4, false>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+        if (u >= 2) return rowc_do<PG, 2, false>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+        return rowc_do<PG, 1, false>(P, clusters, cluster_size, depth, limit_ns, stream, max_clusters);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace
+
+size_t lt_compiled_cluster_vector_bytes(int id, int u) {
+    int k = 0;
+#define LT_X(PG)                                                                          \
+    if (k == id) return (size_t)Info<PG>::n_reserved() * (size_t)u * C_ROW_THREADS * 32u; \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return 0;
+}
+
+cudaError_t lt_compiled_launch_cluster(int id, const void *params, int u, int shared_vectors, unsigned clusters, unsigned cluster_size,
+                                       unsigned depth, uint64_t limit_ns, cudaStream_t stream) {
+    int k = 0;
+#define LT_X(PG)                                                                                                                        \
+    if (k == id) return rowc_one<PG>(static_cast<const LtKParams *>(params), u, shared_vectors != 0, clusters, cluster_size, depth, limit_ns, stream, nullptr); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t lt_compiled_cluster_occupancy(int id, int u, int shared_vectors, unsigned cluster_size, unsigned depth, int *max_clusters) {
+    int k = 0;
+#define LT_X(PG)                                                                                  \
+    if (k == id) return rowc_one<PG>(nullptr, u, shared_vectors != 0, 0, cluster_size, depth, 0, nullptr, max_clusters); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}
 
 size_t lt_compiled_long_stage_bytes(int id, uint32_t cols) {
     int k = 0;

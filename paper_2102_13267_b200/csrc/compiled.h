@@ -36,6 +36,17 @@ size_t lt_compiled_long_stage_bytes(int id, uint32_t cols);
 cudaError_t lt_compiled_launch_long(int id, const void *params, unsigned grid, unsigned threads, unsigned depth, size_t stage_bytes,
                                     uint64_t limit_ns, int l2_ahead, cudaStream_t stream);
 cudaError_t lt_compiled_long_occupancy(int id, unsigned threads, size_t dyn_smem, int *blocks);
+// Rows of up to 8 x 128 x 8 chunks whose thread group is a thread-block cluster of `cluster_size` (2, 4 or 8) CTAs of
+// 128 threads, `u` (1, 2, 4 or 8) chunks per thread, the row in registers: `clusters` clusters share the rows.
+// `depth` as for lt_compiled_launch (stages of lt_compiled_row_stage_bytes each); `limit_ns` bounds the wait of a
+// reduction for the other CTAs' parts.  lt_compiled_cluster_occupancy: how many such clusters the device holds at once.
+// `shared_vectors` non-zero: the program's column vectors (a thread's columns of gamma, beta, a bias) are kept in
+// lt_compiled_cluster_vector_bytes of shared memory for the whole launch instead of being re-read for every row; zero:
+// in registers when they fit 64 of them, else re-read.
+cudaError_t lt_compiled_launch_cluster(int id, const void *params, int u, int shared_vectors, unsigned clusters, unsigned cluster_size,
+                                       unsigned depth, uint64_t limit_ns, cudaStream_t stream);
+cudaError_t lt_compiled_cluster_occupancy(int id, int u, int shared_vectors, unsigned cluster_size, unsigned depth, int *max_clusters);
+size_t lt_compiled_cluster_vector_bytes(int id, int u);
 // Device status word (bit 0: a bounded wait gave up); synchronises the device.  `clear` resets it when set.
 cudaError_t lt_device_status_read(unsigned int *out, int clear);
 // Launches a one-warp kernel that waits `limit_ns` for an mbarrier phase nothing completes and then raises bit 0.

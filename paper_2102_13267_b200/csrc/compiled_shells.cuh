@@ -87,6 +87,11 @@ struct Info {
         return false;
     }
     static constexpr __host__ __device__ int elem_bytes(int s) { return PG::dtype[s] == LT_ST_BF16 ? 2 : PG::dtype[s] == LT_ST_U8 ? 1 : 4; }
+    static constexpr __host__ __device__ int reserved_ordinal(int t) {  // position of reserved temporary t among the reserved ones
+        int n = 0;
+        for (int k = 0; k < t; ++k) n += pro_slot(k) >= 0 ? 1 : 0;
+        return n;
+    }
     static constexpr __host__ __device__ int n_reserved() {
         int n = 0;
         for (int t = 0; t < LT_VM_NT; ++t) n += pro_slot(t) >= 0 ? 1 : 0;
@@ -345,7 +350,7 @@ struct GroupReduce {
 // State and straight-line execution of program PG on U chunks at once.  `Ptr` gives the base
 // pointer of a slot, `Scal` the 32-bit immediates.
 // GUARD false: every chunk of every iteration exists, so validity tests disappear.
-template <class PG, int U, class Ptr, class Scal, class Red, bool GUARD = true, bool HOISTED = false>
+template <class PG, int U, class Ptr, class Scal, class Red, bool GUARD = true, int HOISTED = 0>
 struct Machine {
     using I = Info<PG>;
     static constexpr int FLAV = PG::flavour;
@@ -358,7 +363,8 @@ struct Machine {
     const Scal &scal;
     Red &red;
     const Coords<U> &ck;
-    const float (*hoisted)[U][V] = nullptr;  // HOISTED: the reserved temporaries' column vectors, loaded once per thread
+    const float (*hoisted)[U][V] = nullptr;  // HOISTED 1: the reserved temporaries' column vectors, loaded once per thread
+    const float *hoisted_shared = nullptr;   // HOISTED 2: the same in shared memory, [reserved ordinal][u][thread][V] (128-thread CTAs)
 
     __device__ __forceinline__ Machine(const Ptr &p, const Scal &s, Red &r, const Coords<U> &c) : ptr(p), scal(s), red(r), ck(c) {}
 
@@ -493,9 +499,13 @@ struct Machine {
 #pragma unroll
             for (int i = 0; i < V; ++i) d[i] = s;
         } else if constexpr (I::pro_slot(SRC) >= 0) {
-            if constexpr (HOISTED) {
+            if constexpr (HOISTED == 1) {
 #pragma unroll
                 for (int i = 0; i < V; ++i) d[i] = hoisted[SRC][u][i];
+            } else if constexpr (HOISTED == 2) {
+                const float4 *q = reinterpret_cast<const float4 *>(hoisted_shared + ((I::reserved_ordinal(SRC) * U + u) * C_ROW_THREADS + threadIdx.x) * V);
+                const float4 a = q[0], b = q[1];
+                d[0] = a.x, d[1] = a.y, d[2] = a.z, d[3] = a.w, d[4] = b.x, d[5] = b.y, d[6] = b.z, d[7] = b.w;
             } else {
                 load_now<I::pro_slot(SRC)>(d, u);
             }
@@ -779,6 +789,23 @@ __device__ __forceinline__ void hoist_colvecs(const M &m, float (&hv)[NT][U][V])
     }
 }
 
+template <class PG, int U, int T = 0, class M>
+__device__ __forceinline__ void hoist_to_shared(const M &m, float *base) {
+    if constexpr (T < NT) {
+        if constexpr (Info<PG>::pro_slot(T) >= 0) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float d[V];
+                m.template load_now<Info<PG>::pro_slot(T)>(d, u);
+                float4 *q = reinterpret_cast<float4 *>(base + ((Info<PG>::reserved_ordinal(T) * U + u) * C_ROW_THREADS + threadIdx.x) * V);
+                q[0] = make_float4(d[0], d[1], d[2], d[3]);
+                q[1] = make_float4(d[4], d[5], d[6], d[7]);
+            }
+        }
+        hoist_to_shared<PG, U, T + 1>(m, base);
+    }
+}
+
 struct TrueTag { static constexpr bool value = true; };
 struct FalseTag { static constexpr bool value = false; };
 
@@ -878,7 +905,7 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
     }
     auto iterate = [&](auto guard_tag) {
         constexpr bool GUARD = decltype(guard_tag)::value;
-        using MG = Machine<PG, U, PtrK, ScalK, GroupReduce, GUARD, HOIST>;
+        using MG = Machine<PG, U, PtrK, ScalK, GroupReduce, GUARD, HOIST ? 1 : 0>;
         for (uint32_t rb = blockIdx.x; rb < row_blocks; rb += gridDim.x) {
             Coords<U> ck;
             coords_of(rb, ck);
@@ -1146,6 +1173,211 @@ __global__ void __launch_bounds__(T) lt_c_longrow(const __grid_constant__ LtKPar
             if (threadIdx.x == 0 && next < P.rows) issue(next, s);
         }
     }
+}
+
+// ------------------------------------------------------------------ long rows in the registers of a thread-block cluster
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_count_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+// The cluster's hardware barrier (all threads of all its CTAs arrive; like bar.sync it completes by itself under
+// uniform control flow).  Used at the two ends of the kernel only: its release semantics wait for every earlier
+// global store of the thread, far too expensive per row.
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// A 32-bit store into the shared memory of CTA `cta_rank` of the cluster (distributed shared memory) that, when it
+// lands, counts four bytes on an mbarrier of that CTA: whoever sees the barrier's phase complete sees the value.
+// `slot` and `bar` are this CTA's shared-window addresses of the word and the barrier; the peer's are at the same
+// offsets.  No fence is involved, so earlier global stores of the thread stay in flight.
+__device__ __forceinline__ void store_remote_signal(uint32_t slot, uint32_t bar, uint32_t cta_rank, float v) {
+    uint32_t rs, rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rs) : "r"(slot), "r"(cta_rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(bar), "r"(cta_rank));
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(rs), "f"(v), "r"(rb) : "memory");
+}
+
+constexpr int C_MAX_CLUSTER = 8;                     // portable cluster size
+constexpr int C_ROW_WARPS = C_ROW_THREADS / 32;
+
+// Row reductions of a thread group that spans all threads of all CTAs of a cluster.  Lanes, chunks and the warp are
+// folded as in GroupReduce.  Then lane k of every warp sends the warp's partial to CTA k of the cluster, into slot
+// [sender's rank][warp] of one of two exchange buffers, as a store that signals an mbarrier there; a thread waits
+// (bounded) until its CTA's barrier has counted the bytes of all warps of all CTAs and folds the slots in index
+// order -- the same order everywhere, so every thread of the row holds the same bits.  No CTA-wide or cluster-wide
+// barrier per reduction.  Buffers and barriers alternate between consecutive reductions; a buffer is written again
+// two reductions later, and a CTA sends for reduction n + 2 only after it has received every CTA's part of n + 1,
+// which each sent after all its threads had finished reading n.
+struct ClusterReduce {
+    const float *slots;   // 2 x (C_MAX_CLUSTER x C_ROW_WARPS) floats
+    uint32_t slots_addr;  // shared-window address of `slots`
+    uint32_t bar_addr;    // ... of the two mbarriers
+    uint32_t nctas, rank, phase;
+    uint64_t limit_ns;
+    bool gave_up;
+    template <int KIND, int U, bool GUARD>
+    __device__ __forceinline__ void operator()(float (&acc)[U][V], const bool (&ok)[U]) {
+        const float ident = KIND == 0 ? 0.0f : (KIND == 1 ? -LT_INF : LT_INF);
+        float part[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float l0 = GroupReduce::red_comb<KIND>(acc[u][0], acc[u][1]), l1 = GroupReduce::red_comb<KIND>(acc[u][2], acc[u][3]);
+            float l2 = GroupReduce::red_comb<KIND>(acc[u][4], acc[u][5]), l3 = GroupReduce::red_comb<KIND>(acc[u][6], acc[u][7]);
+            part[u] = (!GUARD || ok[u]) ? GroupReduce::red_comb<KIND>(GroupReduce::red_comb<KIND>(l0, l1), GroupReduce::red_comb<KIND>(l2, l3)) : ident;
+        }
+#pragma unroll
+        for (int s = 1; s < U; s <<= 1)
+#pragma unroll
+            for (int u = 0; u + s < U; u += 2 * s) part[u] = GroupReduce::red_comb<KIND>(part[u], part[u + s]);
+        float r = part[0];
+#pragma unroll
+        for (uint32_t off = 16; off > 0; off >>= 1) r = GroupReduce::red_comb<KIND>(r, __shfl_xor_sync(0xffffffffu, r, off));
+        const uint32_t half = phase & 1u, parity = (phase >> 1) & 1u;
+        ++phase;
+        const uint32_t bar = bar_addr + 8u * half;
+        const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+        if (threadIdx.x == 0) mbar_expect_tx(bar, nctas * C_ROW_WARPS * 4u);
+        if (lane < nctas) store_remote_signal(slots_addr + ((half * C_MAX_CLUSTER + rank) * C_ROW_WARPS + warp) * 4u, bar, lane, r);
+        if (!gave_up && !mbar_wait_bounded(bar, parity, limit_ns)) {
+            gave_up = true;  // results from here on are wrong and the host is told; later waits are skipped
+            atomicOr(&lt_device_status, 1u);
+        }
+        const float4 *x = reinterpret_cast<const float4 *>(slots + half * C_MAX_CLUSTER * C_ROW_WARPS);
+        static_assert(C_ROW_WARPS == 4, "one 128-bit load per CTA's partials");
+        float4 q = x[0];
+        r = GroupReduce::red_comb<KIND>(GroupReduce::red_comb<KIND>(q.x, q.y), GroupReduce::red_comb<KIND>(q.z, q.w));
+        for (uint32_t k = 1; k < nctas; ++k) {
+            q = x[k];
+            r = GroupReduce::red_comb<KIND>(r, GroupReduce::red_comb<KIND>(GroupReduce::red_comb<KIND>(q.x, q.y), GroupReduce::red_comb<KIND>(q.z, q.w)));
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[u][i] = r;
+    }
+};
+
+// Rows longer than one CTA's registers hold, up to 8 CTAs x 128 threads x 8 chunks x 8 elements = 65536 columns: the
+// row's thread group is a thread-block cluster.  Thread t of CTA r (of K) owns chunks (u K + r) 128 + t, u = 0..U-1, of
+// the row its cluster is working on and keeps them in registers across the reductions, exactly as in lt_c_row; only
+// the reductions differ (ClusterReduce).  One pass over the data whatever the number of reductions; a thread owns
+// the same columns for every row, so small column vectors are loaded once.  With `depth` > 0 the CTA's parts of the
+// cluster's next `depth` rows are in flight as asynchronous copies into a ring of shared-memory stages.  All CTAs
+// of a cluster run the same rows and the same program.  The kernel ends with the cluster's barrier: no CTA leaves
+// while another may still write into its shared memory.
+template <class PG, int U, bool HS>
+__global__ void __launch_bounds__(C_ROW_THREADS) lt_c_rowc(const __grid_constant__ LtKParams P, uint32_t depth, uint64_t limit_ns) {
+    __shared__ __align__(16) float slots[2 * C_MAX_CLUSTER * C_ROW_WARPS];
+    __shared__ __align__(8) uint64_t bars[2];
+    extern __shared__ __align__(16) unsigned char stage_mem[];
+    constexpr uint32_t STAGE = Info<PG>::stage_bytes(U, C_ROW_THREADS);
+    const PtrK ptr{P};
+    const ScalK scal{P};
+    const uint32_t nctas = cluster_nctarank(), rank = cluster_ctarank();
+    const uint32_t group = nctas * C_ROW_THREADS, gl = rank * C_ROW_THREADS + threadIdx.x;
+    const uint32_t first = cluster_id_x(), step = cluster_count_x();
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+    ClusterReduce red{slots, (uint32_t)__cvta_generic_to_shared(slots), bar0, nctas, rank, 0u, limit_ns, false};
+    if (threadIdx.x == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    auto coords_of = [&](uint32_t row, Coords<U> &ck) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t col = (u * group + gl) * V;
+            const bool in_row = col < P.cols, in_rows = row < P.rows;  // a chunk that does not exist takes the coordinates of one that does
+            ck.row[u] = in_rows ? row : 0u;
+            ck.col0[u] = in_row ? col : 0u;
+            ck.ok[u] = in_row && in_rows;
+            ck.flat0[u] = (uint64_t)ck.row[u] * P.cols + ck.col0[u];
+        }
+    };
+    // HS: the column vectors of the reserved temporaries (the thread's columns of gamma, beta, a bias) are kept in
+    // shared memory, in front of the stages, instead of in registers: 32 bytes per vector and chunk for each thread
+    constexpr uint32_t HOIST_BYTES = HS ? Info<PG>::n_reserved() * U * C_ROW_THREADS * V * 4 : 0;
+    unsigned char *const ring = stage_mem + HOIST_BYTES;
+    const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(ring);
+    pdl_wait();
+    cluster_sync();  // every CTA of the cluster is running, its barriers initialised, before one writes into another's shared memory
+    using M = Machine<PG, U, PtrK, ScalK, ClusterReduce>;
+    if (depth) {
+        uint32_t row = first;
+        for (uint32_t d = 0; d < depth; ++d, row += step) {
+            if (row < P.rows) {
+                Coords<U> nx;
+                coords_of(row, nx);
+                M::template stage_issue<C_ROW_THREADS>(ptr, nx.flat0, nx.ok, stage0 + d * STAGE);
+            }
+            cp_async_commit();
+        }
+    }
+    const bool full = group * U * V == P.cols;
+    constexpr int HOIST = Info<PG>::n_reserved() == 0 ? 0 : HS ? 2 : (Info<PG>::n_reserved() * U * V <= 64 && !Info<PG>::integer_heavy()) ? 1 : 0;
+    float hv[NT][U][V];
+    if constexpr (HOIST == 1) {
+        Coords<U> c0;
+        coords_of(0, c0);
+        Machine<PG, U, PtrK, ScalK, ClusterReduce, true> m0(ptr, scal, red, c0);
+        hoist_colvecs<PG, U>(m0, hv);
+    } else if constexpr (HOIST == 2) {
+        // every thread copies its own columns and later reads nothing else: no barrier needed
+        Coords<U> c0;
+        coords_of(0, c0);
+        Machine<PG, U, PtrK, ScalK, ClusterReduce, true> m0(ptr, scal, red, c0);
+        hoist_to_shared<PG, U>(m0, reinterpret_cast<float *>(stage_mem));
+    }
+    uint32_t s = 0;
+    auto iterate = [&](auto guard_tag) {
+        constexpr bool GUARD = decltype(guard_tag)::value;
+        using MG = Machine<PG, U, PtrK, ScalK, ClusterReduce, GUARD, HOIST>;
+        for (uint32_t row = first; row < P.rows; row += step) {
+            Coords<U> ck;
+            coords_of(row, ck);
+            MG m(ptr, scal, red, ck);
+            m.hoisted = hv;
+            m.hoisted_shared = reinterpret_cast<const float *>(stage_mem);
+            if (depth) {
+                cp_async_wait(depth - 1);
+                m.template stage_fetch<C_ROW_THREADS>(ring + s * STAGE);
+                const uint32_t rn = row + depth * step;  // the stage just read is refilled with the row `depth` iterations ahead
+                if (rn < P.rows) {
+                    Coords<U> nx;
+                    coords_of(rn, nx);
+                    MG::template stage_issue<C_ROW_THREADS>(ptr, nx.flat0, nx.ok, stage0 + s * STAGE);
+                }
+                cp_async_commit();
+                s = s + 1 == depth ? 0 : s + 1;
+            } else {
+                m.issue_loads();
+            }
+            m.run();
+        }
+    };
+    if (full) iterate(FalseTag{});
+    else iterate(TrueTag{});
+    if (depth) cp_async_wait(0);
+    // the next kernel of the stream may start only now: released at the top, its clusters took the places of this
+    // kernel's retiring ones early and waited there, which measured 10-20 % slower back to back
+    pdl_release();
+    cluster_sync();
 }
 
 // A kernel that waits, bounded, for an mbarrier phase nothing completes: exercises the give-up path of

@@ -506,6 +506,8 @@ lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     else if (!strcmp(key, "debug.compiled_depth")) c->opt.compiled_depth = value;
     else if (!strcmp(key, "debug.long_l2_ahead")) c->opt.long_l2_ahead = value;
     else if (!strcmp(key, "debug.ignore_table")) c->opt.ignore_table = value;
+    else if (!strcmp(key, "debug.cluster")) c->opt.cluster = value;
+    else if (!strcmp(key, "debug.cluster_vectors")) c->opt.cluster_vectors = value;
     else if (!strcmp(key, "specialise")) c->opt.specialise = value;
     else if (!strcmp(key, "specialise_after")) c->opt.specialise_after = value;
     else if (!strcmp(key, "wait_limit_ms")) c->wait_limit_ns = value > 0 ? value * 1000000ll : 1;

@@ -150,6 +150,7 @@ struct Launch {
     std::shared_ptr<JitKernel> jit;
     bool jit_failed = false;
     uint32_t runs = 0;
+    int cluster_max = -1;                // long rows: clusters of the cluster row kernel the device holds at once (-1 = not asked yet)
     std::unique_ptr<LtKParams> kp;       // K_EW / K_ROW parameter block (static parts prefilled)
     std::unique_ptr<LtMultiParams> mp;   // K_MULTI
 };
@@ -187,6 +188,8 @@ struct Options {
     int64_t specialise_after = 3;  // ... once a plan has run this many times (mode 2)
     int64_t ignore_table = 0;      // measurements: plan as if the build-time table were empty (everything specialised or interpreted)
     int64_t long_l2_ahead = -1;  // long-row kernels: request the next row into L2 (-1 = the library's choice)
+    int64_t cluster = 0;  // long rows: CTAs per cluster of the cluster row kernel (0 = the library's choice, 1 = never use it)
+    int64_t cluster_vectors = -1;  // ... its column vectors in shared memory (1), in registers or re-read (0), the library's choice (-1)
 };
 
 struct HashKey {
@@ -326,6 +329,26 @@ struct DeviceScope {
     DeviceScope(const DeviceScope &) = delete;
     DeviceScope &operator=(const DeviceScope &) = delete;
 };
+
+// Long rows of up to 8 x 128 x 8 chunks run with a thread-block cluster as the row's thread group (lt_c_rowc): the
+// cluster size and the chunks per thread for rows of `cpr` chunks; false when the row is too long.  As many chunks
+// per thread as the row needs in the smallest cluster -- eight, or four when the program reads column vectors, which
+// a thread then still keeps in registers (measured: softmax at 16384 columns 90 us in clusters of two against 97 in
+// clusters of four; LayerNorm 129 us in clusters of four against 156 in clusters of two).
+inline bool cluster_shape(uint32_t cpr, bool has_vectors, int64_t want_cluster, int64_t want_u, unsigned *cluster, int *u) {
+    if (cpr > 8u * 128u * 8u || want_cluster == 1) return false;
+    const unsigned prefer = has_vectors ? 4u : 8u;
+    unsigned k = 2;
+    while (k < 8 && (uint64_t)k * 128u * prefer < cpr) k *= 2;
+    if (want_cluster == 2 || want_cluster == 4 || want_cluster == 8) k = (unsigned)want_cluster;
+    int uu = 1;
+    while (uu < 8 && (uint64_t)k * 128u * (unsigned)uu < cpr) uu *= 2;
+    if ((want_u == 1 || want_u == 2 || want_u == 4 || want_u == 8) && (uint64_t)k * 128u * (unsigned)want_u >= cpr) uu = (int)want_u;
+    if ((uint64_t)k * 128u * (unsigned)uu < cpr) return false;
+    *cluster = k;
+    *u = uu;
+    return true;
+}
 
 // canonicaliser (canon.cpp)
 void canonicalise(lt_ctx *c, const std::vector<uint32_t> &root_tensors, Canonical &out);

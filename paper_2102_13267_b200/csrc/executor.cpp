@@ -392,17 +392,72 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
             if (g.long_row) {
                 // a CTA per row, walking it in slices; rows staged in shared memory `depth` ahead when they fit
                 // (feasibility was checked on entry)
-                if (!dry) {
+                if (!dry && specialised(L)) {
+                    std::string err;
+                    if (!jit_load(*L.jit, c->device, &err)) {
+                        release_all(true);
+                        return fail(c, LT_ERR_CUDA, err);
+                    }
+                }
+                // Up to 65536 columns: a thread-block cluster is the row's thread group and the row stays in registers
+                // across the reductions (one pass over the data, column vectors loaded once per thread).
+                unsigned cl_size = 0;
+                int cl_u = 0;
+                bool clustered = !dry && cluster_shape(P.cpr, g.n_pro > 0, c->opt.cluster, c->opt.compiled_row_u, &cl_size, &cl_u) &&
+                                 (!specialised(L) || L.jit_program->cluster_u == cl_u);
+                size_t cl_dyn = 0;
+                unsigned cl_depth = 0;
+                bool cl_shared = false;
+                if (clustered) {
+                    // column vectors that do not fit 64 registers per thread are kept in shared memory rather than re-read for every row
+                    const size_t vec = specialised(L) ? jit_cluster_vector_bytes(*L.jit_program, cl_u) : lt_compiled_cluster_vector_bytes(L.compiled, cl_u);
+                    cl_shared = vec > 0 && vec <= 160u * 1024u && (c->opt.cluster_vectors >= 0 ? c->opt.cluster_vectors != 0 : vec > 128u * 64u * 4u);
+                    // the next rows' inputs travel through a ring of shared-memory stages: not for programs bound by integer
+                    // issue, nor for 4-byte inputs, which measured faster loaded directly (softmax f32 at 65536 columns: 247 us
+                    // against 333 with the ring; the requests of eight chunks per thread are in flight either way)
+                    const size_t stage = specialised(L) ? jit_row_stage_bytes(*L.jit_program, cl_u, 128) : lt_compiled_row_stage_bytes(L.compiled, cl_u);
+                    bool wants_ring = specialised(L) ? !jit_integer_heavy(*L.jit_program) : lt_compiled_prefers_staging(L.compiled) != 0;
+                    for (size_t q = 0; q < g.io.size(); ++q)
+                        if (!g.io[q].is_store && g.io[q].cls == LT_CLS_FULL && dtype_size(g.io[q].dtype) == 4) wants_ring = false;
+                    cl_depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth : (wants_ring ? 2u : 0u);
+                    while (cl_depth > 0 && cl_depth * stage > 72u * 1024u) --cl_depth;
+                    if (stage == 0) cl_depth = 0;
+                    cl_dyn = cl_depth * stage + (cl_shared ? vec : 0);
+                    if (L.cluster_max < 0) {
+                        int n = 0;
+                        if (specialised(L)) n = jit_cluster_occupancy(*L.jit, c->device, cl_shared ? 3 : 2, 128, cl_size, cl_dyn);
+                        else if (lt_compiled_cluster_occupancy(L.compiled, cl_u, cl_shared ? 1 : 0, cl_size, cl_depth, &n) != cudaSuccess) {
+                            cudaGetLastError();
+                            n = 0;
+                        }
+                        L.cluster_max = n;
+                    }
+                    clustered = L.cluster_max >= 1;
+                }
+                if (clustered) {
+                    const unsigned clusters = (unsigned)std::min<uint64_t>(P.rows, (uint64_t)L.cluster_max);
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    if (specialised(L)) {
+                        uint32_t a1 = cl_depth;
+                        uint64_t a2 = (uint64_t)c->wait_limit_ns;
+                        void *args[3] = {&P, &a1, &a2};
+                        std::string err;
+                        if (!jit_launch(*L.jit, c->device, cl_shared ? 3 : 2, clusters * cl_size, 128, cl_dyn, (void *)c->stream, args, &err, cl_size)) {
+                            c->error = err;
+                            e = cudaErrorLaunchFailure;
+                        } else {
+                            c->stats.launches_specialised++;
+                        }
+                    } else {
+                        e = lt_compiled_launch_cluster(L.compiled, &P, cl_u, cl_shared ? 1 : 0, clusters, cl_size, cl_depth, (uint64_t)c->wait_limit_ns, c->stream);
+                    }
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                    c->status_pending = true;
+                }
+                if (!dry && !clustered) {
                     // Staging and CTA size: the row a CTA works on is staged when it fits; several CTAs per SM overlap one
                     // another's passes; when a staged row leaves room for one CTA only, that CTA has 512 threads.
                     const size_t cap = 200u * 1024u;
-                    if (specialised(L)) {
-                        std::string err;
-                        if (!jit_load(*L.jit, c->device, &err)) {
-                            release_all(true);
-                            return fail(c, LT_ERR_CUDA, err);
-                        }
-                    }
                     const size_t stage = specialised(L) ? jit_long_stage_bytes(*L.jit_program, P.cols) : lt_compiled_long_stage_bytes(L.compiled, P.cols);
                     const unsigned deepest = stage == 0 ? 0u : (unsigned)std::min<size_t>(2, cap / stage);
                     auto blocks_at = [&](unsigned threads, unsigned d) {

@@ -51,6 +51,7 @@ struct Api {
     CUresult (*FuncSetAttribute)(CUfunction, CUfunction_attribute, int) = nullptr;
     CUresult (*OccupancyMaxActiveBlocksPerMultiprocessor)(int *, CUfunction, int, size_t) = nullptr;
     CUresult (*GetErrorString)(CUresult, const char **) = nullptr;
+    CUresult (*OccupancyMaxActiveClusters)(int *, CUfunction, const CUlaunchConfig *) = nullptr;
 };
 
 template <class F>
@@ -107,7 +108,7 @@ const Api &api() {
             sym(drv, "cuModuleLoadData", x.ModuleLoadData), sym(drv, "cuModuleGetFunction", x.ModuleGetFunction),
                 sym(drv, "cuLaunchKernelEx", x.LaunchKernelEx), sym(drv, "cuFuncSetAttribute", x.FuncSetAttribute),
                 sym(drv, "cuOccupancyMaxActiveBlocksPerMultiprocessor", x.OccupancyMaxActiveBlocksPerMultiprocessor),
-                sym(drv, "cuGetErrorString", x.GetErrorString);
+                sym(drv, "cuGetErrorString", x.GetErrorString), sym(drv, "cuOccupancyMaxActiveClusters", x.OccupancyMaxActiveClusters);
         x.ok = ok;
         return x;
     }();
@@ -136,6 +137,10 @@ std::vector<std::pair<std::string, int>> variants_of(const JitProgram &p) {
     else if (p.long_row) {
         v.push_back({"lt_c_longrow<JP, 256>", 0});
         v.push_back({"lt_c_longrow<JP, 512>", 1});
+        if (p.cluster_u > 0) {
+            v.push_back({"lt_c_rowc<JP, " + std::to_string(p.cluster_u) + ", false>", 2});
+            if (jit_cluster_vector_bytes(p, 1) > 0) v.push_back({"lt_c_rowc<JP, " + std::to_string(p.cluster_u) + ", true>", 3});
+        }
     } else {
         v.push_back({"lt_c_row<JP, " + std::to_string(p.row_u) + ">", 0});
     }
@@ -144,7 +149,7 @@ std::vector<std::pair<std::string, int>> variants_of(const JitProgram &p) {
 
 // ---- optional on-disk cache of the machine code (environment variable LT_KERNEL_CACHE = a directory)
 //
-// A file per (program, library sources): "<hash>.ltk" = magic, the two lowered kernel names, the machine code.  The
+// A file per (program, library sources): "<hash>.ltk" = magic, the lowered kernel names, the machine code.  The
 // hash covers the program's generated table entry and the text of the device headers, so a rebuilt library with
 // changed shells never picks up stale code.  Files are written to a temporary name and renamed.
 
@@ -158,7 +163,7 @@ std::string cache_path(const std::string &src, const JitProgram &p) {
     if (!dir || !*dir) return "";
     uint64_t h = fnv1a(src);
     for (const char *t : {kSrcVm, kSrcVmOps, kSrcPdl, kSrcShells}) h = fnv1a(t, h);
-    h = fnv1a(std::string(p.long_row ? "L" : "R") + std::to_string(p.row_u) + "/" + std::to_string(api().compiler_version), h);
+    h = fnv1a(std::string(p.long_row ? "L" : "R") + std::to_string(p.row_u) + "C" + std::to_string(p.cluster_u) + "/" + std::to_string(api().compiler_version), h);
     char name[64];
     snprintf(name, sizeof(name), "/%016llx.ltk", (unsigned long long)h);
     return std::string(dir) + name;
@@ -168,14 +173,16 @@ bool cache_read(const std::string &path, JitKernel &k) {
     FILE *f = fopen(path.c_str(), "rb");
     if (!f) return false;
     bool ok = false;
-    uint32_t head[4] = {0, 0, 0, 0};  // magic, length of name 0, of name 1, of the machine code
-    if (fread(head, sizeof(head), 1, f) == 1 && head[0] == 0x4b544c31u && head[1] < 4096 && head[2] < 4096 && head[3] > 0 &&
-        head[3] < (64u << 20)) {
-        k.entry[0].resize(head[1]);
-        k.entry[1].resize(head[2]);
-        k.cubin.resize(head[3]);
-        ok = (head[1] == 0 || fread(&k.entry[0][0], head[1], 1, f) == 1) && (head[2] == 0 || fread(&k.entry[1][0], head[2], 1, f) == 1) &&
-             fread(k.cubin.data(), head[3], 1, f) == 1;
+    uint32_t head[6] = {0, 0, 0, 0, 0, 0};  // magic, lengths of the four kernel names, length of the machine code
+    if (fread(head, sizeof(head), 1, f) == 1 && head[0] == 0x4b544c33u && head[1] < 4096 && head[2] < 4096 && head[3] < 4096 &&
+        head[4] < 4096 && head[5] > 0 && head[5] < (64u << 20)) {
+        ok = true;
+        for (int v = 0; v < 4 && ok; ++v) {
+            k.entry[v].resize(head[1 + v]);
+            ok = head[1 + v] == 0 || fread(&k.entry[v][0], head[1 + v], 1, f) == 1;
+        }
+        k.cubin.resize(head[5]);
+        ok = ok && fread(k.cubin.data(), head[5], 1, f) == 1;
     }
     fclose(f);
     return ok;
@@ -185,9 +192,11 @@ void cache_write(const std::string &path, const JitKernel &k) {
     const std::string tmp = path + ".tmp" + std::to_string((unsigned long long)(uintptr_t)&k);
     FILE *f = fopen(tmp.c_str(), "wb");
     if (!f) return;
-    const uint32_t head[4] = {0x4b544c31u, (uint32_t)k.entry[0].size(), (uint32_t)k.entry[1].size(), (uint32_t)k.cubin.size()};
-    bool ok = fwrite(head, sizeof(head), 1, f) == 1 && (k.entry[0].empty() || fwrite(k.entry[0].data(), k.entry[0].size(), 1, f) == 1) &&
-              (k.entry[1].empty() || fwrite(k.entry[1].data(), k.entry[1].size(), 1, f) == 1) && fwrite(k.cubin.data(), k.cubin.size(), 1, f) == 1;
+    const uint32_t head[6] = {0x4b544c33u, (uint32_t)k.entry[0].size(), (uint32_t)k.entry[1].size(), (uint32_t)k.entry[2].size(),
+                              (uint32_t)k.entry[3].size(), (uint32_t)k.cubin.size()};
+    bool ok = fwrite(head, sizeof(head), 1, f) == 1;
+    for (int v = 0; v < 4 && ok; ++v) ok = k.entry[v].empty() || fwrite(k.entry[v].data(), k.entry[v].size(), 1, f) == 1;
+    ok = ok && fwrite(k.cubin.data(), k.cubin.size(), 1, f) == 1;
     ok = fclose(f) == 0 && ok;
     if (ok) rename(tmp.c_str(), path.c_str());
     else remove(tmp.c_str());
@@ -282,6 +291,7 @@ std::string identity(const JitProgram &p) {
     s.push_back((char)p.flavour);
     s.push_back((char)p.long_row);
     s.push_back((char)p.row_u);
+    s.push_back((char)p.cluster_u);
     s.append((const char *)&p.n_pro, sizeof(p.n_pro));
     s.append((const char *)p.ins.data(), p.ins.size() * sizeof(LtIns));
     s.append((const char *)p.dtype.data(), p.dtype.size());
@@ -344,7 +354,7 @@ bool jit_load(JitKernel &k, int device, std::string *err) {
     CUresult r = a.ModuleLoadData(&mod, k.cubin.data());
     if (r == CUDA_SUCCESS) {
         L.ok = true;
-        for (int v = 0; v < 2 && L.ok; ++v)
+        for (int v = 0; v < 4 && L.ok; ++v)
             if (!k.entry[v].empty()) {
                 CUfunction f = nullptr;
                 r = a.ModuleGetFunction(&f, mod, k.entry[v].c_str());
@@ -373,8 +383,32 @@ int jit_occupancy(JitKernel &k, int device, int variant, int threads, size_t dyn
     return n;
 }
 
+int jit_cluster_occupancy(JitKernel &k, int device, int variant, int threads, unsigned cluster, size_t dyn_smem) {
+    CUfunction f = (CUfunction)fn_of(k, device, variant);
+    const Api &a = api();
+    if (!f || !a.OccupancyMaxActiveClusters) return 0;
+    if (dyn_smem > 32u * 1024u) a.FuncSetAttribute(f, CU_FUNC_ATTRIBUTE_MAX_DYNAMIC_SHARED_SIZE_BYTES, (int)dyn_smem);
+    CUlaunchConfig cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.sharedMemBytes = (unsigned)dyn_smem;
+    cfg.gridDimX = cluster;
+    cfg.gridDimY = cfg.gridDimZ = 1;
+    cfg.blockDimX = (unsigned)threads;
+    cfg.blockDimY = cfg.blockDimZ = 1;
+    CUlaunchAttribute attr[1];
+    memset(attr, 0, sizeof(attr));
+    attr[0].id = CU_LAUNCH_ATTRIBUTE_CLUSTER_DIMENSION;
+    attr[0].value.clusterDim.x = cluster;
+    attr[0].value.clusterDim.y = attr[0].value.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (a.OccupancyMaxActiveClusters(&n, f, &cfg) != CUDA_SUCCESS) n = 0;
+    return n;
+}
+
 bool jit_launch(JitKernel &k, int device, int variant, unsigned grid, unsigned threads, size_t dyn_smem, void *stream, void **args,
-                std::string *err) {
+                std::string *err, unsigned cluster) {
     CUfunction f = (CUfunction)fn_of(k, device, variant);
     if (!f) {
         if (err) *err = "specialised kernel not loaded";
@@ -396,12 +430,18 @@ bool jit_launch(JitKernel &k, int device, int variant, unsigned grid, unsigned t
     cfg.blockDimY = cfg.blockDimZ = 1;
     cfg.sharedMemBytes = (unsigned)dyn_smem;
     cfg.hStream = (CUstream)stream;
-    CUlaunchAttribute attr[1];
+    CUlaunchAttribute attr[2];
     memset(attr, 0, sizeof(attr));
     attr[0].id = CU_LAUNCH_ATTRIBUTE_PROGRAMMATIC_STREAM_SERIALIZATION;  // see pdl.cuh
     attr[0].value.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (cluster) {
+        attr[1].id = CU_LAUNCH_ATTRIBUTE_CLUSTER_DIMENSION;
+        attr[1].value.clusterDim.x = cluster;
+        attr[1].value.clusterDim.y = attr[1].value.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     const CUresult r = a.LaunchKernelEx(&cfg, f, args, nullptr);
     if (r != CUDA_SUCCESS) {
         if (err) *err = std::string("cuLaunchKernelEx: ") + cu_text(r);
@@ -449,6 +489,16 @@ int jit_reductions(const JitProgram &p) {
     int n = 0;
     for (size_t k = p.n_pro; k < p.ins.size(); ++k) n += p.ins[k].op >= OP_RED_SUM && p.ins[k].op <= OP_RED_MIN;
     return n;
+}
+
+size_t jit_cluster_vector_bytes(const JitProgram &p, int u) {
+    bool reserved[LT_VM_NT] = {false};
+    size_t n = 0;
+    for (uint32_t k = 0; k < p.n_pro && k < p.ins.size(); ++k) {
+        const int d = (int)p.ins[k].op - OP_LD;
+        if (d >= 0 && d < LT_VM_NT && !reserved[d]) reserved[d] = true, ++n;
+    }
+    return n * (size_t)u * 128u * 32u;
 }
 
 // What the shells can express (cf. the checks of the table generator): broadcast operands loaded in the prologue into

@@ -1308,6 +1308,11 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                 while (u < 8 && cpr > 32u * u) u *= 2;  // (the executor's choice: one warp per row where it fits)
                 jp->row_u = u;
             }
+            if (L.kind == K_ROW && g.long_row) {
+                unsigned k = 0;
+                int u = 0;
+                if (cluster_shape((uint32_t)((g.cols + LT_VM_V - 1) / LT_VM_V), g.n_pro > 0, c->opt.cluster, c->opt.compiled_row_u, &k, &u)) jp->cluster_u = u;
+            }
             if (jit_supported(*jp)) L.jit_program = std::move(jp);
             // a long-row group is only worth keeping fused if its kernel is there when the flush runs
             if (L.jit_program && g.long_row && c->opt.specialise == 1) {

@@ -30,6 +30,7 @@ def main() -> None:
     ap.add_argument("configs", nargs="?", default="c1,c2,c2p,c3,c4,c5")
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate through (0 = enough for 1 GB)")
+    ap.add_argument("--only", default="", help="of the idioms / long / reduce cases, run those whose name contains this")
     ap.add_argument("options", nargs="*")
     args = ap.parse_args()
     which = args.configs.split(",")
@@ -163,6 +164,8 @@ def main() -> None:
         ctx.close()
     # rows longer than a thread group's registers (fused long-row kernels), and reductions over columns / everything
     def generic(name, nbytes, make, trace):
+        if args.only and args.only not in name:
+            return
         nsets = args.sets or max(2, math.ceil(1.2e9 / nbytes))
         ctx = context()
         sets = [make(ctx) for _ in range(nsets)]
@@ -192,7 +195,7 @@ def main() -> None:
 
     if "long" in which:
         for rows, cols in ((8192, 16384), (2048, 65536)):
-            for iname in ("softmax_bf16", "layernorm_bf16", "softmax_f32"):
+            for iname in ("softmax_bf16", "layernorm_bf16", "softmax_f32", "layernorm_f32"):
                 _, kinds, trace = next(e for e in idioms.ALL if e[0] == iname)
                 es = 4 if iname.endswith("f32") else 2
 
@@ -203,7 +206,7 @@ def main() -> None:
                         out.append(c.from_torch(t.to(torch.bfloat16) if k.endswith("bf16") else t))
                     return out
 
-                generic(f"{iname[:10]} {cols}", 2 * es * rows * cols, make, lambda c, s_, trace=trace, cols=cols: trace(c, s_, cols))
+                generic(f"{iname} {cols}", 2 * es * rows * cols, make, lambda c, s_, trace=trace, cols=cols: trace(c, s_, cols))
     if "reduce" in which:
         for rows, cols in ((16384, 4096), (1 << 20, 64)):
             for op in ("col_sum", "all_sum", "row_sum"):

@@ -55,6 +55,44 @@ def test_listed_groups_on_long_rows_run_fused(ctx, idiom, shape):
     assert_matches(ctx.fetch(out), ref.array, "f32" if name.endswith("f32") else "bf16", f"{name} {shape}")
 
 
+# Rows of up to 65536 columns run with a thread-block cluster as the row's thread group; longer ones, and every long
+# row when that kernel is switched off, are walked in slices by one CTA.  Both against the oracle, every cluster size,
+# with the column vectors in registers / re-read and in shared memory, rows that do and do not fill the group.
+@pytest.mark.parametrize("vectors", [0, 1])
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+@pytest.mark.parametrize("idiom,shape", [("layernorm_bf16", (9, 16384)), ("layernorm_f32", (5, 10000)), ("softmax_bf16", (7, 8200)),
+                                         ("rmsnorm_bf16", (3, 32768)), ("layernorm_bf16", (3, 65536)), ("softmax_f32", (300, 12288))])
+def test_long_rows_in_every_cluster_shape(lt, idiom, shape, cluster, vectors):
+    if cluster * 128 * 8 * 8 < shape[-1] and cluster != 1:
+        pytest.skip("row too long for this cluster size")
+    c = lt.LazyContext(device=0)
+    c.set_option("debug.cluster", cluster)
+    c.set_option("debug.cluster_vectors", vectors)
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == idiom)
+    arrs = _idiom_inputs(kinds, shape, 67)
+    O = EagerOracle()
+    ref = trace(O, [O.leaf(a, d) for a, d in arrs], shape[-1])
+    out = trace(c, [c.leaf(a, d) for a, d in arrs], shape[-1])
+    c.barrier()
+    st = c.stats()
+    assert st["kernels_launched"] == 1 and st["launches_row"] == 1 and st["launches_compiled"] == 1, st
+    assert_matches(c.fetch(out), ref.array, "f32" if name.endswith("f32") else "bf16", f"{name} {shape} cluster {cluster} vectors {vectors}")
+    c.close()
+
+
+def test_rows_beyond_the_cluster_kernel_are_walked_in_slices(ctx):
+    shape = (3, 131072)
+    name, kinds, trace = next(e for e in idioms.ALL if e[0] == "softmax_bf16")
+    arrs = _idiom_inputs(kinds, shape, 68)
+    O = EagerOracle()
+    ref = trace(O, [O.leaf(a, d) for a, d in arrs], shape[-1])
+    out = trace(ctx, [ctx.leaf(a, d) for a, d in arrs], shape[-1])
+    ctx.barrier()
+    st = ctx.stats()
+    assert st["kernels_launched"] == 1 and st["launches_compiled"] == 1, st
+    assert_matches(ctx.fetch(out), ref.array, "bf16", "softmax 131072")
+
+
 @pytest.mark.parametrize("depth", [0, 1, 2])
 def test_long_row_staging_depths_agree(lt, depth):
     """Rows staged in shared memory two ahead, one ahead, or read from global memory in every pass."""

@@ -100,6 +100,16 @@ def test_specialised_long_rows_and_multi_tensor(lt):
     st = c.stats()
     assert st["launches_row"] == 1 and st["launches_reduce"] == 0 and st["launches_specialised"] == 1
     assert_matches(c.fetch(out), ref.array, "f32", "specialised long rows")
+    # the same program on the CTA-per-row kernel, and on every cluster size of the cluster kernel
+    for cluster in (1, 2, 4, 8):
+        k = lt.LazyContext(device=0)
+        k.set_option("specialise", 1)
+        k.set_option("debug.cluster", cluster)
+        got = _row_normalise(k, k.leaf(z, "f32"))
+        k.barrier()
+        assert k.stats()["launches_specialised"] == 1
+        assert_matches(k.fetch(got), ref.array, "f32", f"specialised long rows, cluster {cluster}")
+        k.close()
     # many small tensors, one program that is not in the table: p := p * 0.99 - g * lr, in place
     shapes = [(64, 3, 7, 7), (64,), (1000,), (256, 64), (128,)]
     host = [[rng.normal_f32(rng.generator(84 + k), s, 0.1) for s in shapes] for k in range(2)]
