@@ -139,7 +139,8 @@ typedef struct {
     uint64_t outputs_donated;    /* outputs written into a donated input buffer              */
     uint64_t outputs_allocated;  /* outputs given fresh memory                               */
     uint64_t temporaries_allocated; /* cross-kernel intermediates given scratch memory        */
-    uint64_t ns_record;          /* inside lt_op and the factory calls                       */
+    uint64_t ns_record;          /* inside lt_op, lt_assign, lt_release and the factory calls (estimated: one call
+                                    in eight is timed and counted eight times)                                */
     uint64_t ns_canonicalise;    /* root gathering + post-order serialisation                */
     uint64_t ns_hash_lookup;     /* hashing + cache probe                                    */
     uint64_t ns_plan;            /* fusion planning + program generation (misses only)       */
@@ -156,6 +157,9 @@ typedef struct {
     uint64_t allocator_calls;    /* calls of the allocator's alloc and free (or cudaMallocAsync /
                                     cudaFreeAsync); 0 over a span means every block came from and
                                     went back to the context's own pool of released blocks          */
+    uint64_t traces_matched;     /* of cache_hits: flushes whose trace repeated the previous one call by call and
+                                    was bound to its plan without building the graph (the "trace_match" option)  */
+    uint64_t traces_diverged;    /* traces that started out repeating the previous one and then differed          */
 } lt_stats;
 
 /* Device time per kernel family, measured with CUDA events when kernel timing is on. */

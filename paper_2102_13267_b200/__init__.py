@@ -57,7 +57,7 @@ class lt_stats(ctypes.Structure):
         "launches_elementwise", "launches_row", "launches_multi", "bytes_planned",
         "outputs_donated", "outputs_allocated", "temporaries_allocated",
         "ns_record", "ns_canonicalise", "ns_hash_lookup", "ns_plan", "ns_bind_launch", "ns_rebind",
-        "launches_compiled", "replays", "launches_reduce", "launches_view", "programs_specialised", "launches_specialised", "allocator_calls")]
+        "launches_compiled", "replays", "launches_reduce", "launches_view", "programs_specialised", "launches_specialised", "allocator_calls", "traces_matched", "traces_diverged")]
 
 
 class lt_kernel_timing(ctypes.Structure):

@@ -38,6 +38,17 @@ inline uint64_t ticks_now() { return now_ns(); }
 inline double ns_per_tick() { return 1.0; }
 #endif
 
+// The recording calls are far more frequent than anything else and, once a trace is only matched, cost about as much
+// as two reads of the counter: one call in eight is timed and counted eight times.
+struct RecordTimer {
+    lt_ctx *c;
+    uint64_t t0;
+    explicit RecordTimer(lt_ctx *ctx) : c(ctx), t0((++ctx->record_calls & 7u) ? 0 : ticks_now()) {}
+    ~RecordTimer() {
+        if (t0) c->stats.ns_record += 8 * (ticks_now() - t0);
+    }
+};
+
 struct Timer {
     uint64_t &acc;
     uint64_t t0;
@@ -50,8 +61,12 @@ inline lt_tensor make_handle(const lt_ctx *c, uint32_t slot) {
 }
 
 lt_status sync_view_of(lt_ctx *c, uint32_t slot);
+void trace_materialise(lt_ctx *c);
 
+// Every entry point that looks at a tensor's computation resolves its handles here.  A trace that has so far only
+// been matched against the previous one (its tensors have no IR yet) is first turned into the real thing.
 lt_status lookup(lt_ctx *c, lt_tensor h, uint32_t *slot) {
+    if (c->trace.mode == TM_MATCH && c->trace.cursor) trace_materialise(c);
     if ((uint16_t)(h >> 48) != c->tag) return fail(c, LT_ERR_DEVICE, "tensor handle belongs to another context");
     uint32_t s = (uint32_t)(h & 0xffffffffu);
     if (s == 0 || s > c->tensors.size()) return fail(c, LT_ERR_INVALID_ARG, "unknown tensor handle");
@@ -66,6 +81,17 @@ lt_status lookup(lt_ctx *c, lt_tensor h, uint32_t *slot) {
 
 uint32_t tensor_new(lt_ctx *c, uint32_t node) {
     uint32_t slot;
+    if (c->trace.force_slot != NONE) {
+        // the tensor exists already as a handle without IR (trace matching): it now gets its node
+        slot = c->trace.force_slot;
+        c->trace.force_slot = NONE;
+        TensorRec &t = c->tensors[slot];
+        t.node = node;
+        t.vflags = 0;
+        node_ref(c, node);
+        c->nodes[node].tensor_refs++;
+        return slot;
+    }
     if (!c->free_tensors.empty()) {
         slot = c->free_tensors.back();
         c->free_tensors.pop_back();
@@ -84,6 +110,7 @@ uint32_t tensor_new(lt_ctx *c, uint32_t node) {
     t.view_op = 0;
     t.version = 0;
     t.base_seen = 0;
+    t.vflags = 0;
     node_ref(c, node);
     c->nodes[node].tensor_refs++;
     return slot;
@@ -411,6 +438,679 @@ void ctx_free(lt_ctx *c, void *p) {
 
 }  // namespace lt
 
+// ======================================================================= trace matching
+//
+// Section 7 of the paper names the cost of re-tracing an unchanged program every step as the first thing to remove.
+// lt_replay removes it on request; this removes most of it without being asked.  While a trace is recorded as usual
+// its calls are also logged, operands named relative to the trace (TraceScript).  When the barrier has flushed it,
+// the log is kept with the plan that ran and with where that plan's parameters, run-time values and results come
+// from in the log.  The next trace is then only compared with the log, call by call: a call that repeats the logged
+// one returns a handle that has no IR node behind it.  If the barrier finds the whole log repeated, it binds the plan
+// directly -- nothing is canonicalised, hashed or looked up.  The first call that differs (or any call that wants to
+// look at a tensor's computation) makes the calls matched so far for real, on the same handles, and recording goes on
+// as usual; the trace being built becomes the next log.
+namespace {
+
+constexpr uint32_t TRACE_RELEASED_AT_ONCE = 0xfffffffeu;  // in bind_slot, for a release event
+
+inline bool peek_slot(const lt_ctx *c, lt_tensor h, uint32_t *slot) {
+    if ((uint16_t)(h >> 48) != c->tag) return false;
+    uint32_t s = (uint32_t)(h & 0xffffffffu);
+    if (s == 0 || s > c->tensors.size()) return false;
+    s -= 1;
+    const TensorRec &t = c->tensors[s];
+    if (!t.live || (t.gen & 0xffffu) != (uint32_t)((h >> 32) & 0xffffu)) return false;
+    *slot = s;
+    return true;
+}
+
+// A trace begins: after a barrier that flushed something, or when matching is given up.
+void trace_begin(lt_ctx *c, uint8_t mode) {
+    TraceState &T = c->trace;
+    T.mode = c->opt.trace_match ? mode : (uint8_t)TM_OFF;
+    T.epoch++;
+    T.cursor = 0;
+    T.n_imports = T.n_nodes = 0;
+    T.force_slot = NONE;
+    T.log.clear();
+    T.log_valid = true;
+    T.bind_import_slot.clear();
+    T.bind_node.clear();
+    T.deferred_release.clear();
+    T.virtual_scalars.clear();
+    if (T.mode == TM_MATCH) {
+        // indexed by event and written before they are read: what the last trace left in them does not matter
+        const size_t n = T.script.events.size();
+        T.bind_slot.resize(n);
+        T.bind_val.resize(n);
+        T.bind_val2.resize(n);
+    } else {
+        T.bind_slot.clear();
+        T.bind_val.clear();
+        T.bind_val2.clear();
+    }
+}
+
+inline void trace_unsupported(lt_ctx *c) { c->trace.log_valid = false; }
+
+void trace_forget_plan(lt_ctx *c, const Plan *plan) {
+    if (c->trace.script.plan == plan) {
+        c->trace.script.clear();
+        if (c->trace.mode == TM_MATCH) c->trace.mode = TM_LEARN;  // (only ever reached between traces or while learning)
+    }
+}
+
+// ---- learning: the trace is recorded as usual and logged
+
+// Id of tensor `slot` in the trace being logged.  A tensor from before the trace is described once, when it is
+// first used: what it is, and which of the trace's input nodes it names (two tensors may name the same one).
+uint32_t trace_learn_tid(lt_ctx *c, uint32_t slot) {
+    TraceState &T = c->trace;
+    TensorRec &t = c->tensors[slot];
+    if (t.trace_epoch == T.epoch) return t.trace_id;
+    Node &nd = c->nodes[t.node];
+    TraceImport im;
+    if (!(nd.op == N_DEVICE_DATA || nd.op == N_SCALAR) || t.view_base != NONE) T.log_valid = false;
+    im.op = nd.op;
+    im.dtype = nd.dtype;
+    im.rank = nd.rank;
+    im.flags = nd.flags;
+    memcpy(im.dims, nd.dims, sizeof(im.dims));
+    im.sval = (nd.op == N_SCALAR && !(nd.flags & NF_DYNAMIC)) ? nd.sval : 0.0;
+    if (nd.trace_epoch == T.epoch) {
+        if (nd.trace_ref & TID_IMPORT) im.node_ordinal = nd.trace_ref & ~TID_IMPORT;
+        else T.log_valid = false;  // made in this trace yet named by a tensor that was not: not expressible
+    } else {
+        im.node_ordinal = T.n_nodes++;
+        im.fresh_node = true;
+        nd.trace_epoch = T.epoch;
+        nd.trace_ref = TID_IMPORT | im.node_ordinal;
+    }
+    t.trace_id = TID_IMPORT | (uint32_t)T.log.imports.size();
+    t.trace_epoch = T.epoch;
+    T.log.imports.push_back(im);
+    return t.trace_id;
+}
+
+inline bool trace_learning(const lt_ctx *c) { return c->trace.mode == TM_LEARN && c->trace.log_valid; }
+
+// the tensor in `slot` is the result of the event about to be appended
+void trace_log_result(lt_ctx *c, uint32_t slot) {
+    TraceState &T = c->trace;
+    const uint32_t idx = (uint32_t)T.log.events.size();
+    TensorRec &t = c->tensors[slot];
+    t.trace_id = idx;
+    t.trace_epoch = T.epoch;
+    Node &nd = c->nodes[t.node];
+    nd.trace_ref = idx;
+    nd.trace_epoch = T.epoch;
+    TraceResult res;
+    res.dtype = nd.dtype;
+    res.rank = nd.rank;
+    memcpy(res.dims, nd.dims, sizeof(res.dims));
+    T.log.results.push_back(res);
+}
+
+void trace_log_op(lt_ctx *c, int opcode, const uint32_t *in_slots, int n_in, const int64_t *attrs, int n_attrs, uint32_t out_slot) {
+    TraceState &T = c->trace;
+    if (n_attrs > 64 || T.log.events.size() >= (1u << 24)) {
+        T.log_valid = false;
+        return;
+    }
+    TraceEvent ev;
+    ev.kind = TE_OP;
+    ev.op = (uint16_t)opcode;
+    ev.n_in = (uint8_t)n_in;
+    ev.n_attrs = (uint8_t)n_attrs;
+    for (int i = 0; i < n_in; ++i) ev.in[i] = trace_learn_tid(c, in_slots[i]);
+    ev.attr_off = (uint32_t)T.log.attrs.size();
+    T.log.attrs.insert(T.log.attrs.end(), attrs, attrs + n_attrs);
+    trace_log_result(c, out_slot);
+    T.log.events.push_back(ev);
+}
+
+void trace_log_scalar(lt_ctx *c, uint32_t out_slot) {
+    TraceState &T = c->trace;
+    const Node &nd = c->nodes[c->tensors[out_slot].node];
+    TraceEvent ev;
+    ev.kind = TE_SCALAR;
+    ev.dtype = nd.dtype;
+    ev.flags = nd.flags;
+    ev.sval = (nd.flags & NF_DYNAMIC) ? 0.0 : nd.sval;
+    trace_log_result(c, out_slot);
+    T.log.events.push_back(ev);
+}
+
+void trace_log_leaf(lt_ctx *c, uint32_t out_slot) {
+    TraceState &T = c->trace;
+    const Node &nd = c->nodes[c->tensors[out_slot].node];
+    TraceEvent ev;
+    ev.kind = TE_LEAF;
+    ev.dtype = nd.dtype;
+    ev.rank = nd.rank;
+    ev.n_attrs = nd.rank;
+    ev.attr_off = (uint32_t)T.log.attrs.size();
+    T.log.attrs.insert(T.log.attrs.end(), nd.dims, nd.dims + nd.rank);
+    trace_log_result(c, out_slot);
+    T.log.events.push_back(ev);
+}
+
+void trace_log_pair(lt_ctx *c, uint8_t kind, uint32_t a, uint32_t b) {
+    TraceState &T = c->trace;
+    TraceEvent ev;
+    ev.kind = kind;
+    ev.in[0] = trace_learn_tid(c, a);
+    if (kind == TE_ASSIGN) ev.in[1] = trace_learn_tid(c, b);
+    T.log.events.push_back(ev);
+    T.log.results.emplace_back();
+}
+
+// The barrier has run `ran` for the logged trace: keep the log, with where the plan's inputs and results are in it.
+// Called while the roots still name their IR and `cg` describes it.  Returns false if something cannot be expressed.
+bool trace_seal(lt_ctx *c, Plan *plan, const Plan *ran, const Canonical &cg, const std::vector<uint32_t> &roots) {
+    TraceState &T = c->trace;
+    if (T.mode != TM_LEARN || !T.log_valid || !c->view_slots.empty() || T.log.events.empty()) return false;
+    TraceScript &S = T.log;
+    S.param_src.resize(cg.param_node.size());
+    for (size_t p = 0; p < cg.param_node.size(); ++p) {
+        const Node &nd = c->nodes[cg.param_node[p]];
+        if (nd.trace_epoch != T.epoch) return false;  // an input the trace never touched (pending from earlier)
+        S.param_src[p] = nd.trace_ref;
+    }
+    S.dyn_src.assign(cg.dyn.size(), TraceScript::DynSrc());
+    for (const CNode &cn : cg.nodes) {
+        if (cn.dyn < 0) continue;
+        const Node &nd = c->nodes[cn.arena];
+        if (nd.trace_epoch != T.epoch) return false;
+        S.dyn_src[cn.dyn].ref = nd.trace_ref;
+        if (cn.op == LT_OP_PHILOX_BITS) {
+            S.dyn_src[cn.dyn + 1].ref = nd.trace_ref;
+            S.dyn_src[cn.dyn + 1].which = 1;
+        }
+    }
+    S.roots.clear();
+    for (uint32_t slot : roots) {
+        const TensorRec &t = c->tensors[slot];
+        if (t.trace_epoch != T.epoch) return false;
+        TraceScript::Root r;
+        r.tid = t.trace_id;
+        r.output = cg.nodes[c->nodes[t.node].canon].output;
+        S.roots.push_back(r);
+    }
+    // what lt_replay would need after a flush that only matched this trace
+    const ReplayRecord &R = c->replay;
+    auto tid_of = [&](uint32_t slot) -> uint32_t {
+        if (slot == NONE || c->tensors[slot].trace_epoch != T.epoch) return NONE;
+        return c->tensors[slot].trace_id;
+    };
+    S.replay_why_not = R.why_not;
+    S.replay_param.resize(R.params.size());
+    for (size_t i = 0; i < R.params.size(); ++i) {
+        S.replay_param[i] = tid_of(R.params[i].slot);
+        if (S.replay_param[i] == NONE && S.replay_why_not.empty()) S.replay_why_not = "an input of the flushed graph was not named by a tensor of the trace";
+    }
+    S.replay_dyn_scalar.resize(R.dyn_scalar.size());
+    for (size_t k = 0; k < R.dyn_scalar.size(); ++k) S.replay_dyn_scalar[k] = tid_of(R.dyn_scalar[k].slot);
+    S.replay_in_place_ok = R.in_place_ok;
+    S.n_nodes = T.n_nodes;
+    S.plan = plan;
+    (void)ran;
+    T.script = std::move(T.log);
+    T.log.clear();
+    return true;
+}
+
+// ---- matching
+
+// Does tensor `slot` have id `want` in the trace being followed?  A tensor from before the trace is checked
+// against the description logged at the same point.
+bool trace_match_tid(lt_ctx *c, uint32_t slot, uint32_t want) {
+    TraceState &T = c->trace;
+    TensorRec &t = c->tensors[slot];
+    if (t.trace_epoch == T.epoch) return t.trace_id == want;
+    if (want != (TID_IMPORT | T.n_imports) || T.n_imports >= T.script.imports.size() || t.view_base != NONE || t.node == NONE) return false;
+    const TraceImport &im = T.script.imports[T.n_imports];
+    Node &nd = c->nodes[t.node];
+    if (nd.op != im.op || nd.dtype != im.dtype || nd.rank != im.rank || ((nd.flags ^ im.flags) & NF_DYNAMIC)) return false;
+    for (int i = 0; i < nd.rank; ++i)
+        if (nd.dims[i] != im.dims[i]) return false;
+    if (nd.op == N_SCALAR && !(nd.flags & NF_DYNAMIC) && memcmp(&nd.sval, &im.sval, sizeof(double)) != 0) return false;
+    if (nd.trace_epoch == T.epoch) {
+        if (im.fresh_node || nd.trace_ref != (TID_IMPORT | im.node_ordinal)) return false;
+    } else {
+        if (!im.fresh_node || im.node_ordinal != T.n_nodes) return false;
+        nd.trace_epoch = T.epoch;
+        nd.trace_ref = TID_IMPORT | T.n_nodes;
+        T.bind_node.push_back(t.node);
+        T.n_nodes++;
+    }
+    t.trace_id = want;
+    t.trace_epoch = T.epoch;
+    T.bind_import_slot.push_back(slot);
+    T.n_imports++;
+    return true;
+}
+
+// the result of matched event `index`: a live handle with no node behind it
+uint32_t trace_virtual_tensor(lt_ctx *c, uint32_t index) {
+    uint32_t slot;
+    if (!c->free_tensors.empty()) {
+        slot = c->free_tensors.back();
+        c->free_tensors.pop_back();
+    } else {
+        slot = (uint32_t)c->tensors.size();
+        c->tensors.emplace_back();
+    }
+    TensorRec &t = c->tensors[slot];
+    t.node = NONE;
+    t.gen += 1;
+    t.donor = NONE;
+    t.seq = c->next_seq++;
+    t.live = true;
+    t.queued = false;
+    t.view_base = NONE;
+    t.view_op = 0;
+    t.version = 0;
+    t.base_seen = 0;
+    t.trace_id = index;
+    t.trace_epoch = c->trace.epoch;
+    t.vflags = TV_VIRTUAL;
+    c->trace.bind_slot[index] = slot;
+    return slot;
+}
+
+bool trace_match_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int64_t *attrs, int n_attrs, lt_tensor *out) {
+    TraceState &T = c->trace;
+    if (T.cursor >= T.script.events.size() || n_in < 0 || n_in > 3 || n_attrs < 0) return false;
+    const TraceEvent &ev = T.script.events[T.cursor];
+    if (ev.kind != TE_OP || ev.op != opcode || ev.n_in != n_in || ev.n_attrs != n_attrs || (n_in && !in) || (n_attrs && !attrs)) return false;
+    for (int i = 0; i < n_in; ++i) {
+        uint32_t slot;
+        if (!peek_slot(c, in[i], &slot) || !trace_match_tid(c, slot, ev.in[i])) return false;
+    }
+    const int64_t *want = T.script.attrs.data() + ev.attr_off;
+    int first = 0;
+    if (opcode == LT_OP_PHILOX_BITS && n_attrs >= 2) {  // seed and offset are run-time values
+        T.bind_val[T.cursor].i = attrs[0];
+        T.bind_val2[T.cursor].i = attrs[1];
+        first = 2;
+    }
+    for (int i = first; i < n_attrs; ++i)
+        if (attrs[i] != want[i]) return false;
+    const uint32_t slot = trace_virtual_tensor(c, T.cursor);
+    T.cursor++;
+    c->stats.nodes_recorded++;
+    *out = make_handle(c, slot);
+    return true;
+}
+
+bool trace_match_scalar(lt_ctx *c, double value, lt_dtype dtype, bool force_dynamic, lt_tensor *out) {
+    TraceState &T = c->trace;
+    if (T.cursor >= T.script.events.size()) return false;
+    const TraceEvent &ev = T.script.events[T.cursor];
+    uint64_t bits;
+    memcpy(&bits, &value, 8);
+    const bool dynamic = force_dynamic || !(bits == 0ull || value == 1.0);
+    if (ev.kind != TE_SCALAR || ev.dtype != (uint8_t)dtype || ((ev.flags & NF_DYNAMIC) != 0) != dynamic) return false;
+    if (!dynamic && memcmp(&ev.sval, &value, sizeof(double)) != 0) return false;
+    T.bind_val[T.cursor].d = value;
+    const uint32_t slot = trace_virtual_tensor(c, T.cursor);
+    T.virtual_scalars.push_back(slot);
+    T.cursor++;
+    c->stats.nodes_recorded++;
+    *out = make_handle(c, slot);
+    return true;
+}
+
+bool trace_match_assign(lt_ctx *c, lt_tensor dst, lt_tensor src) {
+    TraceState &T = c->trace;
+    if (T.cursor >= T.script.events.size()) return false;
+    const TraceEvent &ev = T.script.events[T.cursor];
+    uint32_t ds, ss;
+    if (ev.kind != TE_ASSIGN || !peek_slot(c, dst, &ds) || !peek_slot(c, src, &ss)) return false;
+    if (!trace_match_tid(c, ds, ev.in[0]) || !trace_match_tid(c, ss, ev.in[1])) return false;
+    TensorRec &d = c->tensors[ds];
+    if (!(d.vflags & TV_VIRTUAL)) d.vflags |= TV_ASSIGNED;  // still names its old leaf; the barrier gives it the new value
+    T.cursor++;
+    return true;
+}
+
+bool trace_match_release(lt_ctx *c, lt_tensor h) {
+    TraceState &T = c->trace;
+    if (T.cursor >= T.script.events.size()) return false;
+    const TraceEvent &ev = T.script.events[T.cursor];
+    uint32_t slot;
+    if (ev.kind != TE_RELEASE || !peek_slot(c, h, &slot)) return false;
+    const bool untouched = c->tensors[slot].trace_epoch != T.epoch;
+    if (!trace_match_tid(c, slot, ev.in[0])) return false;
+    TensorRec &t = c->tensors[slot];
+    if (untouched) {
+        // a tensor from before the trace that the trace has not used: nothing recorded depends on it, it goes at once
+        t.live = false;
+        t.queued = false;
+        if (t.donor != NONE) {
+            buffer_unref(c, t.donor);
+            t.donor = NONE;
+        }
+        c->nodes[t.node].tensor_refs--;
+        node_unref(c, t.node);
+        t.node = NONE;
+        c->free_tensors.push_back(slot);
+        T.bind_slot[T.cursor] = TRACE_RELEASED_AT_ONCE;
+        T.cursor++;
+        return true;
+    }
+    t.live = false;  // the handle is dead; the slot is kept until the barrier so that the calls can still be made for real
+    t.vflags |= TV_RELEASED;
+    T.deferred_release.push_back(slot);
+    T.cursor++;
+    return true;
+}
+
+bool trace_match_leaf(lt_ctx *c, lt_dtype dtype, int rank, const int64_t *shape) {
+    TraceState &T = c->trace;
+    if (T.cursor >= T.script.events.size()) return false;
+    const TraceEvent &ev = T.script.events[T.cursor];
+    if (ev.kind != TE_LEAF || ev.dtype != (uint8_t)dtype || ev.rank != rank || rank < 0 || (rank && !shape)) return false;
+    const int64_t *want = T.script.attrs.data() + ev.attr_off;
+    for (int i = 0; i < rank; ++i)
+        if (shape[i] != want[i]) return false;
+    return true;
+}
+
+void trace_bind_leaf(lt_ctx *c, uint32_t slot) {  // the (real) leaf just made is the result of the matched event
+    TraceState &T = c->trace;
+    TensorRec &t = c->tensors[slot];
+    t.trace_id = T.cursor;
+    t.trace_epoch = T.epoch;
+    Node &nd = c->nodes[t.node];
+    nd.trace_ref = T.cursor;
+    nd.trace_epoch = T.epoch;
+    T.bind_slot[T.cursor] = slot;
+    T.cursor++;
+}
+
+}  // namespace
+
+extern "C" {
+static lt_status new_scalar(lt_ctx *c, double value, lt_dtype dtype, bool force_dynamic, lt_tensor *out);
+}
+
+namespace {
+
+// Gives up matching: the calls matched so far are made for real, each on the handle it returned.
+void trace_materialise(lt_ctx *c) {
+    TraceState &T = c->trace;
+    if (T.mode != TM_MATCH) return;
+    const uint32_t n = T.cursor;
+    std::vector<TraceEvent> events(T.script.events.begin(), T.script.events.begin() + n);
+    std::vector<int64_t> attrs;
+    attrs.swap(T.script.attrs);
+    std::vector<uint32_t> bslot, bimp, deferred;
+    std::vector<DynValue> bval, bval2;
+    bslot.swap(T.bind_slot);
+    bimp.swap(T.bind_import_slot);
+    bval.swap(T.bind_val);
+    bval2.swap(T.bind_val2);
+    deferred.swap(T.deferred_release);
+    std::vector<TraceImport> old_imports;
+    old_imports.swap(T.script.imports);
+    T.script.clear();
+    if (n) {
+        c->stats.traces_diverged++;
+        if (++T.streak >= 4) T.streak = 0, T.backoff = 16;
+    }
+    trace_begin(c, TM_LEARN);
+    if (!n) return;
+    for (uint32_t slot : deferred) c->tensors[slot].live = true;  // released again below, for real
+    for (uint32_t slot : bimp) c->tensors[slot].vflags = 0;
+    uint64_t counted = 0;
+    auto slot_of = [&](uint32_t tid) { return (tid & TID_IMPORT) ? bimp[tid & ~TID_IMPORT] : bslot[tid]; };
+    lt_status st = LT_OK;
+    for (uint32_t e = 0; e < n && st == LT_OK; ++e) {
+        const TraceEvent &ev = events[e];
+        lt_tensor out = 0;
+        if (ev.kind == TE_OP) {
+            lt_tensor in[3] = {0, 0, 0};
+            for (int i = 0; i < ev.n_in; ++i) in[i] = make_handle(c, slot_of(ev.in[i]));
+            int64_t a[64];
+            for (int i = 0; i < ev.n_attrs; ++i) a[i] = attrs[ev.attr_off + i];
+            if (ev.op == LT_OP_PHILOX_BITS && ev.n_attrs >= 2) a[0] = bval[e].i, a[1] = bval2[e].i;
+            T.force_slot = bslot[e];
+            st = lt_op(c, ev.op, in, ev.n_in, a, ev.n_attrs, &out);
+            ++counted;
+        } else if (ev.kind == TE_SCALAR) {
+            T.force_slot = bslot[e];
+            st = new_scalar(c, bval[e].d, (lt_dtype)ev.dtype, (ev.flags & NF_DYNAMIC) != 0, &out);
+            ++counted;
+        } else if (ev.kind == TE_ASSIGN) {
+            st = lt_assign(c, make_handle(c, slot_of(ev.in[0])), make_handle(c, slot_of(ev.in[1])));
+        } else if (ev.kind == TE_RELEASE) {
+            if (bslot[e] == TRACE_RELEASED_AT_ONCE) {
+                // the tensor is gone already; what the log says about it is what the followed log said
+                if (trace_learning(c)) {
+                    TraceImport im = old_imports[ev.in[0] & ~TID_IMPORT];
+                    if (im.fresh_node) im.node_ordinal = T.n_nodes++;
+                    TraceEvent copy = ev;
+                    copy.in[0] = TID_IMPORT | (uint32_t)T.log.imports.size();
+                    T.log.imports.push_back(im);
+                    T.log.events.push_back(copy);
+                    T.log.results.emplace_back();
+                    T.bind_slot.push_back(NONE);
+                    T.bind_import_slot.push_back(NONE);
+                }
+            } else {
+                st = lt_release(c, make_handle(c, slot_of(ev.in[0])));
+            }
+        } else {  // the leaf exists; it only has to be in the new log
+            if (trace_learning(c)) {
+                trace_log_leaf(c, bslot[e]);
+                T.bind_slot.push_back(bslot[e]);
+            }
+        }
+        T.force_slot = NONE;
+    }
+    c->stats.nodes_recorded -= counted;  // they were counted when they were matched
+    if (st != LT_OK) {
+        // cannot happen for calls that were accepted once; if it does, say so and stop matching for good
+        fprintf(stderr, "[lazytensor] internal error: a matched trace could not be rebuilt (%s)\n", c->error.c_str());
+        c->opt.trace_match = 0;
+        T.mode = TM_OFF;
+    }
+}
+
+inline void trace_materialise_if_started(lt_ctx *c) {
+    if (c->trace.mode == TM_MATCH && c->trace.cursor) trace_materialise(c);
+}
+
+// The barrier of a trace that repeated the logged one to the end: binds and runs the logged plan.
+// False: something differs after all (the caller rebuilds the trace and takes the usual path).
+bool trace_barrier(lt_ctx *c, int blocking, lt_status *result) {
+    TraceState &T = c->trace;
+    TraceScript &S = T.script;
+    if (T.cursor != S.events.size() || !S.plan || T.n_imports != S.imports.size() || T.n_nodes != S.n_nodes) return false;
+    Plan *plan = S.plan;
+    Canonical &cg = c->canon;
+    auto slot_of = [&](uint32_t tid) { return (tid & TID_IMPORT) ? T.bind_import_slot[tid & ~TID_IMPORT] : T.bind_slot[tid]; };
+    cg.param_node.resize(S.param_src.size());
+    for (size_t p = 0; p < S.param_src.size(); ++p) {
+        const uint32_t ref = S.param_src[p];
+        cg.param_node[p] = (ref & TID_IMPORT) ? T.bind_node[ref & ~TID_IMPORT] : c->tensors[T.bind_slot[ref]].node;
+    }
+    // the roots are taken in creation order: the tensors from before the trace must still be in the logged order
+    uint64_t last_seq = 0;
+    for (const TraceScript::Root &r : S.roots) {
+        const TensorRec &t = c->tensors[slot_of(r.tid)];
+        if (!t.live || t.seq <= last_seq) return false;
+        last_seq = t.seq;
+    }
+    Plan *ran = plan;
+    if (!long_rows_runnable(c, *plan, cg)) {
+        if (!plan->split) return false;
+        ran = plan->split.get();
+    }
+    // a result written in place: the tensor that receives it must be the only one naming the buffer (Section 4.3)
+    std::vector<uint8_t> &receiver = c->param_taken;  // per output: a root that names the donated input and was assigned to
+    receiver.assign(plan->outputs.size(), 0);
+    for (const TraceScript::Root &r : S.roots) {
+        const int32_t p = plan->outputs[r.output].donated_param;
+        if (p < 0) continue;
+        const TensorRec &t = c->tensors[slot_of(r.tid)];
+        if (!(t.vflags & TV_VIRTUAL) && (t.vflags & TV_ASSIGNED) && t.node == cg.param_node[p]) receiver[r.output] = 1;
+    }
+    for (size_t k = 0; k < plan->outputs.size(); ++k) {
+        const int32_t p = plan->outputs[k].donated_param;
+        if (p < 0) continue;
+        const Node &leaf = c->nodes[cg.param_node[p]];
+        if (!receiver[k] || leaf.tensor_refs != 1 || c->buffers[leaf.buffer].refs != 1) return false;
+    }
+    cg.dyn.resize(S.dyn_src.size());
+    for (size_t k = 0; k < S.dyn_src.size(); ++k) {
+        const TraceScript::DynSrc &d = S.dyn_src[k];
+        if (d.ref & TID_IMPORT) cg.dyn[k].d = c->nodes[T.bind_node[d.ref & ~TID_IMPORT]].sval;
+        else cg.dyn[k] = d.which ? T.bind_val2[d.ref] : T.bind_val[d.ref];
+    }
+    {
+        Timer tm(c->stats.ns_bind_launch);
+        lt_status s = execute_plan(c, *ran, cg, nullptr);
+        if (s) {
+            *result = s;  // nothing was rebound: the barrier can be called again
+            return true;
+        }
+    }
+    c->stats.barriers++;
+    c->stats.cache_hits++;
+    c->stats.traces_matched++;
+    T.streak = 0;
+    plan->last_used = ++c->use_clock;
+    c->last_plan = plan;
+    if (c->opt.log >= 2)
+        fprintf(stderr, "[lazytensor] barrier %llu: trace matched (%zu calls), %zu launches\n", (unsigned long long)c->stats.barriers,
+                S.events.size(), ran->launches.size());
+    {
+        Timer tm(c->stats.ns_rebind);
+        // what lt_replay needs, while the input leaves are still there
+        ReplayRecord &R = c->replay;
+        auto ref_of = [&](uint32_t tid, ReplayRecord::Ref &ref) {
+            ref.slot = NONE;
+            ref.gen = 0;
+            if (tid == NONE) return;
+            ref.slot = slot_of(tid);
+            ref.gen = c->tensors[ref.slot].gen;
+        };
+        R.plan = plan;
+        R.exec = ran;
+        R.why_not = S.replay_why_not;
+        R.dyn = cg.dyn;
+        R.params.assign(S.replay_param.size(), ReplayRecord::ParamRef());
+        for (size_t i = 0; i < S.replay_param.size(); ++i) {
+            const Node &leaf = c->nodes[cg.param_node[i]];
+            R.params[i].dtype = leaf.dtype;
+            R.params[i].rank = leaf.rank;
+            memcpy(R.params[i].dims, leaf.dims, sizeof(leaf.dims));
+            ref_of(S.replay_param[i], R.params[i]);
+        }
+        R.dyn_scalar.assign(S.replay_dyn_scalar.size(), ReplayRecord::Ref());
+        for (size_t k = 0; k < S.replay_dyn_scalar.size(); ++k) ref_of(S.replay_dyn_scalar[k], R.dyn_scalar[k]);
+        R.roots.clear();
+        for (const TraceScript::Root &r : S.roots) {
+            ReplayRecord::Root root;
+            ref_of(r.tid, root);
+            root.output = r.output;
+            R.roots.push_back(root);
+        }
+        R.in_place_ok = S.replay_in_place_ok;
+        // results: new leaves, as after any flush
+        const size_t n_out = ran->outputs.size();
+        // A result written in place whose only root is the tensor that names the buffer (checked above: alone) already
+        // lives where that tensor's leaf points: the leaf stays, nothing is rebound.
+        std::vector<uint32_t> &sharers = c->stack_scratch;  // per output: how many roots receive it
+        sharers.assign(n_out, 0);
+        for (const TraceScript::Root &r : S.roots) sharers[r.output]++;
+        std::vector<uint32_t> new_nodes(n_out, NONE);
+        for (size_t k = 0; k < n_out; ++k) {
+            const OutputPlan &op = ran->outputs[k];
+            if (op.donated_param >= 0 && sharers[k] == 1) continue;
+            const uint32_t n = node_new(c);
+            Node &nd = c->nodes[n];
+            nd.op = N_DEVICE_DATA;
+            nd.dtype = op.dtype;
+            nd.rank = op.rank;
+            memcpy(nd.dims, op.dims, sizeof(nd.dims));
+            if (op.donated_param >= 0) {
+                const uint32_t b = c->nodes[cg.param_node[op.donated_param]].buffer;
+                c->buffers[b].refs++;
+                nd.buffer = b;
+            } else {
+                nd.buffer = buffer_new(c, c->out_ptr[k], op.bytes, true);
+            }
+            nd.refs = 1;
+            new_nodes[k] = n;
+        }
+        for (const TraceScript::Root &r : S.roots) {
+            TensorRec &t = c->tensors[slot_of(r.tid)];
+            const uint32_t nn = new_nodes[r.output];
+            if (nn == NONE) {
+                t.vflags = 0;
+                t.version++;
+                continue;
+            }
+            const uint32_t old = (t.vflags & TV_VIRTUAL) ? NONE : t.node;
+            t.node = nn;
+            t.vflags = 0;
+            node_ref(c, nn);
+            c->nodes[nn].tensor_refs++;
+            if (old != NONE) {
+                t.version++;
+                c->nodes[old].tensor_refs--;
+                node_unref(c, old);
+            }
+        }
+        // scalars made during the trace and still alive become real constants
+        for (uint32_t slot : T.virtual_scalars) {
+            TensorRec &t = c->tensors[slot];
+            if (!t.live || !(t.vflags & TV_VIRTUAL) || t.trace_epoch != T.epoch) continue;
+            const TraceEvent &ev = S.events[t.trace_id];
+            const uint32_t n = node_new(c);
+            Node &nd = c->nodes[n];
+            nd.op = N_SCALAR;
+            nd.dtype = ev.dtype;
+            nd.rank = 0;
+            nd.flags = ev.flags;
+            nd.sval = T.bind_val[t.trace_id].d;
+            nd.refs = 1;
+            nd.tensor_refs = 1;
+            t.node = n;
+            t.vflags = 0;
+        }
+        // the releases of the trace
+        for (uint32_t slot : T.deferred_release) {
+            TensorRec &t = c->tensors[slot];
+            if (!(t.vflags & TV_VIRTUAL)) {  // a tensor from before the trace that the trace also read: its node goes now, like the rest of the flushed IR
+                if (t.donor != NONE) {
+                    buffer_unref(c, t.donor);
+                    t.donor = NONE;
+                }
+                c->nodes[t.node].tensor_refs--;
+                node_unref(c, t.node);
+            }
+            t.vflags = 0;
+            t.node = NONE;
+            t.queued = false;
+            c->free_tensors.push_back(slot);
+        }
+        for (uint32_t slot : T.bind_import_slot) c->tensors[slot].vflags = 0;
+        for (uint32_t n : new_nodes)
+            if (n != NONE) node_unref(c, n);
+        sharers.clear();
+    }
+    trace_begin(c, TM_MATCH);
+    *result = (blocking && c->device != LT_DEVICE_NONE) ? sync_and_check(c) : LT_OK;
+    return true;
+}
+
+}  // namespace
+
 // ======================================================================= C ABI
 
 extern "C" {
@@ -487,6 +1187,16 @@ lt_status lt_ctx_destroy(lt_ctx *c) {
 
 lt_status lt_ctx_set_option(lt_ctx *c, const char *key, int64_t value) {
     if (!c || !key) return LT_ERR_INVALID_ARG;
+    // a logged trace is tied to the plan made under the options of its time
+    trace_materialise(c);
+    c->trace.script.clear();
+    if (c->trace.mode == TM_MATCH) c->trace.mode = TM_LEARN;
+    if (!strcmp(key, "trace_match")) {
+        c->opt.trace_match = value;
+        c->trace.mode = value ? (uint8_t)TM_LEARN : (uint8_t)TM_OFF;
+        c->trace.log_valid = false;  // (a trace may be half recorded: start logging with the next one)
+        return LT_OK;
+    }
     if (!strcmp(key, "fusion")) c->opt.fusion = value;
     else if (!strcmp(key, "verify")) c->opt.verify = value;
     else if (!strcmp(key, "fast_math")) c->opt.fast_math = value;
@@ -533,13 +1243,26 @@ static lt_status new_device_tensor(lt_ctx *c, void *dptr, bool owned, lt_dtype d
 lt_status lt_tensor_from_device(lt_ctx *c, void *dptr, lt_dtype dtype, int rank, const int64_t *shape,
                                 lt_tensor *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
-    Timer tm(c->stats.ns_record);
+    RecordTimer tm(c);
     if (!valid_dtype(dtype)) return fail(c, LT_ERR_DTYPE, "unknown dtype");
     lt_status s = check_shape(c, rank, shape);
     if (s) return s;
     if (!dptr && shape_numel(shape, rank) > 0) return fail(c, LT_ERR_INVALID_ARG, "device pointer is null");
     c->stats.nodes_recorded++;
-    return new_device_tensor(c, dptr, false, dtype, rank, shape, out);
+    bool matched = false;
+    if (c->trace.mode == TM_MATCH) {
+        matched = trace_match_leaf(c, dtype, rank, shape);
+        if (!matched) trace_materialise(c);
+    }
+    s = new_device_tensor(c, dptr, false, dtype, rank, shape, out);
+    if (s) return s;
+    const uint32_t slot = (uint32_t)(*out & 0xffffffffu) - 1;
+    if (matched) trace_bind_leaf(c, slot);
+    else if (trace_learning(c)) {
+        trace_log_leaf(c, slot);
+        c->trace.bind_slot.push_back(slot);
+    }
+    return LT_OK;
 }
 
 lt_status lt_tensor_from_host(lt_ctx *c, const void *hptr, lt_dtype dtype, int rank, const int64_t *shape,
@@ -549,6 +1272,8 @@ lt_status lt_tensor_from_host(lt_ctx *c, const void *hptr, lt_dtype dtype, int r
     lt_status s = check_shape(c, rank, shape);
     if (s) return s;
     if (c->device == LT_DEVICE_NONE) return fail(c, LT_ERR_UNSUPPORTED, "context has no device");
+    trace_materialise(c);
+    trace_unsupported(c);
     DeviceScope on_device(c->device);
     if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
     size_t bytes = (size_t)shape_numel(shape, rank) * dtype_size(dtype);
@@ -568,8 +1293,12 @@ lt_status lt_tensor_from_host(lt_ctx *c, const void *hptr, lt_dtype dtype, int r
 
 static lt_status new_scalar(lt_ctx *c, double value, lt_dtype dtype, bool force_dynamic, lt_tensor *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
-    Timer tm(c->stats.ns_record);
+    RecordTimer tm(c);
     if (!valid_dtype(dtype)) return fail(c, LT_ERR_DTYPE, "unknown dtype");
+    if (c->trace.mode == TM_MATCH) {
+        if (trace_match_scalar(c, value, dtype, force_dynamic, out)) return LT_OK;
+        trace_materialise(c);
+    }
     uint32_t n = node_new(c);
     Node &nd = c->nodes[n];
     nd.op = N_SCALAR;
@@ -583,6 +1312,10 @@ static lt_status new_scalar(lt_ctx *c, double value, lt_dtype dtype, bool force_
     if (force_dynamic || !special) nd.flags |= NF_DYNAMIC;
     c->stats.nodes_recorded++;
     uint32_t slot = tensor_new(c, n);
+    if (trace_learning(c)) {
+        trace_log_scalar(c, slot);
+        c->trace.bind_slot.push_back(slot);
+    }
     *out = make_handle(c, slot);
     return LT_OK;
 }
@@ -822,8 +1555,10 @@ static lt_status propagate_to_bases(lt_ctx *c, uint32_t slot) {
 
 static lt_status make_view(lt_ctx *c, lt_tensor t, int opcode, int64_t a0, int64_t a1, int rank, const int64_t *dims, lt_tensor *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
-    Timer tm(c->stats.ns_record);
+    RecordTimer tm(c);
     uint32_t bs;
+    trace_materialise(c);
+    trace_unsupported(c);
     lt_status st = lookup(c, t, &bs);
     if (st) return st;
     uint32_t n = NONE;
@@ -853,14 +1588,19 @@ extern "C" {
 lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int64_t *attrs, int n_attrs,
                 lt_tensor *out) {
     if (!c || !out) return LT_ERR_INVALID_ARG;
-    Timer tm(c->stats.ns_record);
+    RecordTimer tm(c);
+    if (c->trace.mode == TM_MATCH) {
+        if (trace_match_op(c, opcode, in, n_in, attrs, n_attrs, out)) return LT_OK;
+        trace_materialise(c);
+    }
     if (n_in < 0 || n_in > 3 || (n_in > 0 && !in) || n_attrs < 0 || (n_attrs > 0 && !attrs))
         return fail(c, LT_ERR_INVALID_ARG, "bad operand or attribute list");
-    uint32_t ids[3] = {NONE, NONE, NONE};
+    uint32_t ids[3] = {NONE, NONE, NONE}, in_slots[3] = {NONE, NONE, NONE};
     for (int i = 0; i < n_in; ++i) {
         uint32_t slot;
         lt_status s = lookup(c, in[i], &slot);
         if (s) return s;
+        in_slots[i] = slot;
         ids[i] = c->tensors[slot].node;
     }
     const Node *ops[3] = {nullptr, nullptr, nullptr};
@@ -922,6 +1662,7 @@ lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int6
         lt_status st = record_shape_op(c, opcode, ids[0], ids[1], a0, a1, rank, dims, &n);
         if (st) return st;
         const uint32_t slot = tensor_new(c, n);
+        trace_unsupported(c);  // shape operations are not logged
         if (c->nodes[n].op != N_DEVICE_DATA) queue_pending(c, slot);
         *out = make_handle(c, slot);
         return LT_OK;
@@ -1041,13 +1782,21 @@ lt_status lt_op(lt_ctx *c, int opcode, const lt_tensor *in, int n_in, const int6
     c->stats.nodes_recorded++;
     uint32_t slot = tensor_new(c, n);
     queue_pending(c, slot);
+    if (trace_learning(c)) {
+        trace_log_op(c, opcode, in_slots, n_in, attrs, n_attrs, slot);
+        c->trace.bind_slot.push_back(slot);
+    }
     *out = make_handle(c, slot);
     return LT_OK;
 }
 
 lt_status lt_assign(lt_ctx *c, lt_tensor dst, lt_tensor src) {
     if (!c) return LT_ERR_INVALID_ARG;
-    Timer tm(c->stats.ns_record);
+    RecordTimer tm(c);
+    if (c->trace.mode == TM_MATCH) {
+        if (trace_match_assign(c, dst, src)) return LT_OK;
+        trace_materialise(c);
+    }
     uint32_t ds, ss;
     lt_status s = lookup(c, dst, &ds);
     if (s) return s;
@@ -1055,6 +1804,11 @@ lt_status lt_assign(lt_ctx *c, lt_tensor dst, lt_tensor src) {
     if (s) return s;
     TensorRec &d = c->tensors[ds];
     const TensorRec &sr = c->tensors[ss];
+    if (d.view_base != NONE || sr.view_base != NONE) trace_unsupported(c);
+    if (trace_learning(c)) {
+        trace_log_pair(c, TE_ASSIGN, ds, ss);
+        c->trace.bind_slot.push_back(NONE);
+    }
     if (d.node == sr.node) return LT_OK;
     const Node &dn = c->nodes[d.node];
     const Node &sn = c->nodes[sr.node];
@@ -1092,10 +1846,19 @@ lt_status lt_view_permute(lt_ctx *c, lt_tensor t, const int *perm, lt_tensor *ou
 
 lt_status lt_release(lt_ctx *c, lt_tensor t) {
     if (!c) return LT_ERR_INVALID_ARG;
-    Timer tm(c->stats.ns_record);
+    RecordTimer tm(c);
+    if (c->trace.mode == TM_MATCH) {
+        if (trace_match_release(c, t)) return LT_OK;
+        trace_materialise(c);
+    }
     uint32_t slot;
     lt_status s = lookup(c, t, &slot);
     if (s) return s;
+    if (c->tensors[slot].view_base != NONE) trace_unsupported(c);
+    if (trace_learning(c)) {
+        trace_log_pair(c, TE_RELEASE, slot, NONE);
+        c->trace.bind_slot.push_back(NONE);
+    }
     TensorRec &tr = c->tensors[slot];
     tr.live = false;
     tr.queued = false;
@@ -1123,6 +1886,11 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
     if (!c) return LT_ERR_INVALID_ARG;
     DeviceScope on_device(c->device);
     if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
+    if (c->trace.mode == TM_MATCH && c->trace.cursor) {
+        lt_status matched = LT_OK;
+        if (trace_barrier(c, blocking, &matched)) return matched;
+        trace_materialise(c);
+    }
     std::vector<uint32_t> &roots = c->roots_scratch;
     Canonical &cg = c->canon;
     if (!c->view_slots.empty()) {
@@ -1165,6 +1933,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
                 plan = p;
             else {
                 if (c->replay.plan == p) c->replay.plan = c->replay.exec = nullptr;
+                trace_forget_plan(c, p);
                 c->cache.erase(it);  // a colliding entry: replace it below
             }
         }
@@ -1189,6 +1958,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
                 c->last_plan = nullptr;
             }
             if (c->replay.plan == victim->second.get()) c->replay.plan = c->replay.exec = nullptr;
+            trace_forget_plan(c, victim->second.get());
             c->cache.erase(victim);
         }
         plan = np.get();
@@ -1235,6 +2005,7 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
         }
         consume_pending(c);  // `roots` still holds what the first pass gathered: nothing was recorded in between
         record_replay(c, plan, ran, cg, roots);
+        const bool sealed = trace_seal(c, plan, ran, cg, roots);
         for (uint32_t slot : roots) {
             TensorRec &t = c->tensors[slot];
             const Node &old = c->nodes[t.node];
@@ -1249,6 +2020,11 @@ lt_status lt_barrier(lt_ctx *c, int blocking) {
         }
         release_donors(c, roots);
         for (uint32_t n : new_nodes) node_unref(c, n);
+        // the next trace is compared with this one if this one could be logged; after several traces in a row that
+        // began like the logged one and then differed, a few are recorded without trying
+        TraceState &T = c->trace;
+        if (T.backoff) --T.backoff;
+        trace_begin(c, sealed && !T.backoff ? TM_MATCH : TM_LEARN);
     }
     if (blocking && c->device != LT_DEVICE_NONE) return sync_and_check(c);
     return LT_OK;
@@ -1258,6 +2034,7 @@ lt_status lt_replay(lt_ctx *c, int blocking) {
     if (!c) return LT_ERR_INVALID_ARG;
     DeviceScope on_device(c->device);
     if (!on_device.ok()) return fail(c, LT_ERR_CUDA, "cudaSetDevice failed for the context's device");
+    trace_materialise_if_started(c);
     ReplayRecord &r = c->replay;
     if (!r.plan) return fail(c, LT_ERR_INVALID_ARG, "lt_replay: no flushed graph to replay");
     if (!r.why_not.empty()) return fail(c, LT_ERR_UNSUPPORTED, "lt_replay: " + r.why_not);
@@ -1402,6 +2179,11 @@ lt_status lt_debug_wait_probe(lt_ctx *c, uint64_t limit_ns) {
 lt_status lt_fetch(lt_ctx *c, lt_tensor t, void *host_dst, size_t nbytes) {
     if (!c) return LT_ERR_INVALID_ARG;
     uint32_t slot;
+    if (c->trace.mode == TM_MATCH && c->trace.cursor && peek_slot(c, t, &slot) && (c->tensors[slot].vflags & (TV_VIRTUAL | TV_ASSIGNED))) {
+        // a result of the trace being matched: flush first (the barrier may still find the trace repeated)
+        lt_status b = lt_barrier(c, 1);
+        if (b) return b;
+    }
     lt_status s = lookup(c, t, &slot);
     if (s) return s;
     if (!host_dst && nbytes) return fail(c, LT_ERR_INVALID_ARG, "host destination is null");
@@ -1446,6 +2228,24 @@ lt_status lt_device_ptr(lt_ctx *c, lt_tensor t, void **dptr) {
 lt_status lt_tensor_info(lt_ctx *c, lt_tensor t, int *dtype, int *rank, int64_t *shape, int *materialised) {
     if (!c) return LT_ERR_INVALID_ARG;
     uint32_t slot;
+    if (c->trace.mode == TM_MATCH && c->trace.cursor && peek_slot(c, t, &slot) && c->tensors[slot].view_base == NONE) {
+        // answered without turning the matched calls into IR: a result of the trace from the log, anything else from its node
+        const TensorRec &tr = c->tensors[slot];
+        if (tr.vflags & TV_VIRTUAL) {
+            const TraceResult &res = c->trace.script.results[tr.trace_id];
+            if (dtype) *dtype = res.dtype;
+            if (rank) *rank = res.rank;
+            if (shape) for (int i = 0; i < res.rank; ++i) shape[i] = res.dims[i];
+            if (materialised) *materialised = 0;
+        } else {
+            const Node &nd = c->nodes[tr.node];
+            if (dtype) *dtype = nd.dtype;
+            if (rank) *rank = nd.rank;
+            if (shape) for (int i = 0; i < nd.rank; ++i) shape[i] = nd.dims[i];
+            if (materialised) *materialised = nd.op == N_DEVICE_DATA && !(tr.vflags & TV_ASSIGNED);
+        }
+        return LT_OK;
+    }
     lt_status s = lookup(c, t, &slot);
     if (s) return s;
     const Node &nd = c->nodes[c->tensors[slot].node];
@@ -1507,6 +2307,7 @@ lt_status lt_get_kernel_timing(lt_ctx *c, lt_kernel_timing *out) {
 
 lt_status lt_dump_ir(lt_ctx *c, char *buf, size_t cap, size_t *need) {
     if (!c) return LT_ERR_INVALID_ARG;
+    trace_materialise_if_started(c);
     std::vector<uint32_t> roots;
     gather_roots(c, roots, false);
     std::string s = "IR {\n";

@@ -35,6 +35,9 @@ struct Node {
     int64_t dims[LT_MAX_RANK] = {0};
     double sval = 0.0;         // N_SCALAR value
     int64_t attr[2] = {0, 0};  // CONVERT: dtype; IOTA: dim; PHILOX: seed, offset
+    // trace matching: where the node entered the trace numbered trace_epoch -- the event that made it, or
+    // TID_IMPORT | the ordinal among the nodes from before the trace that it has read
+    uint32_t trace_ref = 0, trace_epoch = 0;
 };
 
 struct Buffer {
@@ -58,6 +61,10 @@ struct TensorRec {
     int64_t view_a0 = 0, view_a1 = 0;
     uint64_t version = 0;           // in-place updates this tensor has received
     uint64_t base_seen = 0;         // version of the base its current computation was derived from
+    // trace matching: the tensor's id in the trace numbered trace_epoch (the event that made it, or TID_IMPORT |
+    // the ordinal among the tensors from before the trace that it has touched), and what is pending for it
+    uint32_t trace_id = 0, trace_epoch = 0;
+    uint8_t vflags = 0;             // TV_*
 };
 
 // ---------------------------------------------------------------- canonical form
@@ -189,6 +196,7 @@ struct Options {
     int64_t ignore_table = 0;      // measurements: plan as if the build-time table were empty (everything specialised or interpreted)
     int64_t long_l2_ahead = -1;  // long-row kernels: request the next row into L2 (-1 = the library's choice)
     int64_t cluster = 0;  // long rows: CTAs per cluster of the cluster row kernel (0 = the library's choice, 1 = never use it)
+    int64_t trace_match = 1;  // a trace that repeats the previous one call by call is bound to that one's plan without being built (0 = off)
     int64_t cluster_vectors = -1;  // ... its column vectors in shared memory (1), in registers or re-read (0), the library's choice (-1)
 };
 
@@ -223,6 +231,89 @@ struct ReplayRecord {
     std::string why_not;            // non-empty: the last flush cannot be replayed, with the reason
 };
 
+// ---------------------------------------------------------------- trace matching
+// The calls of one trace (from one barrier to the next), operands named relative to the trace, and how the plan
+// that the trace was flushed with takes its inputs from them.  While the next trace repeats these calls one by one
+// nothing is built -- no IR node, no canonical form, no hash: results are handles without a node ("virtual"), and the
+// barrier binds the plan directly.  The first call that differs rebuilds the IR of the calls so far and recording
+// continues as usual.
+enum : uint8_t { TE_OP = 0, TE_SCALAR = 1, TE_ASSIGN = 2, TE_RELEASE = 3, TE_LEAF = 4 };
+enum : uint8_t { TV_VIRTUAL = 1, TV_ASSIGNED = 2, TV_RELEASED = 4 };
+constexpr uint32_t TID_IMPORT = 0x80000000u;
+
+struct TraceEvent {
+    uint8_t kind = 0, n_in = 0, n_attrs = 0, dtype = 0;
+    uint16_t op = 0;
+    uint8_t flags = 0, rank = 0;   // scalar: NF_DYNAMIC
+    uint32_t in[3] = {0, 0, 0};    // tensor ids: operands (op), destination and source (assign), the tensor (release)
+    uint32_t attr_off = 0;         // first of n_attrs words in TraceScript::attrs: an op's attributes as passed, a leaf's dimensions
+    double sval = 0.0;             // static scalar: its value
+};
+
+struct TraceImport {               // a tensor from before the trace, at its first use in it
+    uint32_t node_ordinal = 0;     // which of the distinct nodes read by the trace it names
+    bool fresh_node = false;       // ... and whether it is the first to name it
+    uint16_t op = 0;               // N_DEVICE_DATA or N_SCALAR
+    uint8_t dtype = 0, rank = 0, flags = 0;
+    int64_t dims[LT_MAX_RANK] = {0};
+    double sval = 0.0;
+};
+
+struct TraceResult {               // dtype and shape of what an event made (answers lt_tensor_info while only matching)
+    uint8_t dtype = 0, rank = 0;
+    int64_t dims[LT_MAX_RANK] = {0};
+};
+
+struct TraceScript {
+    std::vector<TraceEvent> events;
+    std::vector<TraceResult> results;  // per event (unused for assign and release)
+    std::vector<int64_t> attrs;
+    std::vector<TraceImport> imports;
+    uint32_t n_nodes = 0;
+    // filled in when the trace is flushed
+    Plan *plan = nullptr;
+    std::vector<uint32_t> param_src;   // per parameter: TID_IMPORT | node ordinal, or the leaf event that made it
+    struct DynSrc {
+        uint32_t ref = 0;              // scalar or random-bits event, or TID_IMPORT | node ordinal of a run-time scalar
+        uint8_t which = 0;             // random bits: 0 seed, 1 offset
+    };
+    std::vector<DynSrc> dyn_src;       // per run-time slot
+    struct Root {
+        uint32_t tid = 0;
+        int32_t output = -1;
+    };
+    std::vector<Root> roots;           // in the order the barrier took them
+    // for lt_replay after a matched flush: the tensors of ReplayRecord, as trace ids
+    std::vector<uint32_t> replay_param, replay_dyn_scalar;
+    std::vector<uint8_t> replay_in_place_ok;
+    std::string replay_why_not;
+    void clear() {
+        events.clear(), results.clear(), attrs.clear(), imports.clear(), param_src.clear(), dyn_src.clear(), roots.clear();
+        replay_param.clear(), replay_dyn_scalar.clear(), replay_in_place_ok.clear(), replay_why_not.clear();
+        n_nodes = 0, plan = nullptr;
+    }
+};
+
+enum : uint8_t { TM_OFF = 0, TM_LEARN = 1, TM_MATCH = 2 };
+
+struct TraceState {
+    uint8_t mode = TM_LEARN;
+    bool log_valid = true;             // TM_LEARN: every call so far can be expressed as an event
+    uint32_t epoch = 1;
+    uint32_t cursor = 0;               // TM_MATCH: next event of `script`
+    uint32_t n_imports = 0, n_nodes = 0;
+    uint32_t force_slot = NONE;        // the next tensor made takes this slot (rebuilding a matched prefix)
+    uint32_t streak = 0, backoff = 0;  // traces in a row that began like the log and then differed; traces left to record without trying
+    TraceScript script;                // what TM_MATCH follows
+    TraceScript log;                   // what TM_LEARN writes
+    std::vector<uint32_t> bind_slot;          // per event of the current trace: slot of the tensor it made
+    std::vector<uint32_t> bind_import_slot;   // per import: the tensor's slot
+    std::vector<uint32_t> bind_node;          // per node ordinal: arena node
+    std::vector<DynValue> bind_val, bind_val2;  // per event: run-time scalar value / seed, offset
+    std::vector<uint32_t> deferred_release;   // TM_MATCH: tensors released since the trace began (slots kept until the barrier)
+    std::vector<uint32_t> virtual_scalars;    // TM_MATCH: slots of the scalars made since the trace began
+};
+
 struct TimedLaunch {
     cudaEvent_t start, stop;
     uint8_t kind;
@@ -253,6 +344,7 @@ struct lt_ctx {
 
     lt::Options opt;
     lt_stats stats{};
+    uint32_t record_calls = 0;  // recording calls so far (one in eight is timed)
     std::unordered_map<lt::HashKey, std::unique_ptr<lt::Plan>, lt::HashKeyHasher> cache;
     uint64_t use_clock = 0;
     lt::Plan *last_plan = nullptr;
@@ -267,6 +359,7 @@ struct lt_ctx {
     size_t static_cap = 0;
 
     lt::ReplayRecord replay;
+    lt::TraceState trace;
     bool status_pending = false;      // a kernel with bounded device-side waits ran since the status word was last read
     int64_t wait_limit_ns = 2000000000ll;  // how long such a wait may last
 
@@ -362,6 +455,7 @@ int broadcast_class(const int64_t *dims, int rank, uint64_t rows, uint64_t cols)
 // executor (executor.cpp)
 lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_split = nullptr);
 lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran);
+bool long_rows_runnable(lt_ctx *c, const Plan &plan, const Canonical &cg);
 void fastdiv_make(uint32_t d, uint32_t *mul, uint32_t *sh1, uint32_t *sh2);
 
 }  // namespace lt

@@ -136,32 +136,37 @@ lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran) {
     return execute_plan(c, *plan->split, cg, nullptr);
 }
 
-lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_split) {
-    const bool dry = c->device == LT_DEVICE_NONE;
-    const size_t n_out = plan.outputs.size();
+// A fused long-row launch runs only on its compiled kernel, which needs 128-bit accesses: whole chunks per row
+// and 16-byte aligned inputs (results and temporaries come from the allocator, aligned).  Fills c->param_ptr.
+bool long_rows_runnable(lt_ctx *c, const Plan &plan, const Canonical &cg) {
     c->param_ptr.resize(plan.n_params);
     for (uint32_t i = 0; i < plan.n_params; ++i)
         c->param_ptr[i] = c->buffers[c->nodes[cg.param_node[i]].buffer].ptr;
-    // A fused long-row launch runs only on its compiled kernel, which needs 128-bit accesses: whole chunks per row
-    // and 16-byte aligned inputs (results and temporaries come from the allocator, aligned).  Checked before
-    // anything is obtained or enqueued, so that the caller can fall back to the split plan.
-    if (!dry)
-        for (const Launch &L : plan.launches) {
-            const Group &g = plan.groups[L.groups[0]];
-            if (L.kind != K_ROW || !g.long_row) continue;
-            bool ok = c->opt.compiled && (L.compiled >= 0 || (L.jit && !L.jit_failed)) && (g.cols % LT_VM_V) == 0;
-            for (size_t q = 0; q < g.io.size() && ok; ++q)
-                if (g.io[q].kind == IO_PARAM && (g.io[q].cls <= LT_CLS_COLVEC || g.io[q].cls == LT_CLS_PITCHED))
-                    ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index] + g.io[q].offset * dtype_size(g.io[q].dtype), g.io[q].dtype) &&
-                         aligned_for((uint64_t)g.io[q].pitch * dtype_size(g.io[q].dtype), g.io[q].dtype);
-            if (!ok) {
-                if (needs_split) {
-                    *needs_split = true;
-                    return LT_OK;
-                }
-                return fail(c, LT_ERR_UNSUPPORTED, "a fused reduction over rows of more than 8192 elements needs 16-byte aligned inputs and rows that are a multiple of 8 elements");
-            }
+    if (c->device == LT_DEVICE_NONE) return true;
+    for (const Launch &L : plan.launches) {
+        const Group &g = plan.groups[L.groups[0]];
+        if (L.kind != K_ROW || !g.long_row) continue;
+        bool ok = c->opt.compiled && (L.compiled >= 0 || (L.jit && !L.jit_failed)) && (g.cols % LT_VM_V) == 0;
+        for (size_t q = 0; q < g.io.size() && ok; ++q)
+            if (g.io[q].kind == IO_PARAM && (g.io[q].cls <= LT_CLS_COLVEC || g.io[q].cls == LT_CLS_PITCHED))
+                ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index] + g.io[q].offset * dtype_size(g.io[q].dtype), g.io[q].dtype) &&
+                     aligned_for((uint64_t)g.io[q].pitch * dtype_size(g.io[q].dtype), g.io[q].dtype);
+        if (!ok) return false;
+    }
+    return true;
+}
+
+lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_split) {
+    const bool dry = c->device == LT_DEVICE_NONE;
+    const size_t n_out = plan.outputs.size();
+    // Checked before anything is obtained or enqueued, so that the caller can fall back to the split plan.
+    if (!long_rows_runnable(c, plan, cg)) {
+        if (needs_split) {
+            *needs_split = true;
+            return LT_OK;
         }
+        return fail(c, LT_ERR_UNSUPPORTED, "a fused reduction over rows of more than 8192 elements needs 16-byte aligned inputs and rows that are a multiple of 8 elements");
+    }
     c->out_ptr.assign(n_out, nullptr);
     c->temp_ptr.assign(plan.temp_bytes.size(), nullptr);
 

@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <initializer_list>
 #include <vector>
 
 #include "lazytensor.h"
@@ -37,16 +38,17 @@ lt_tensor scalar(double v) {
     return t;
 }
 
-lt_tensor op(int code, std::vector<lt_tensor> in, std::vector<int64_t> attrs = {}) {
+// (initializer lists live on the stack: the harness itself allocates nothing per call)
+lt_tensor op(int code, std::initializer_list<lt_tensor> in, std::initializer_list<int64_t> attrs = {}) {
     lt_tensor t;
-    check(lt_op(ctx, code, in.data(), (int)in.size(), attrs.data(), (int)attrs.size(), &t), "lt_op");
+    check(lt_op(ctx, code, in.begin(), (int)in.size(), attrs.size() ? attrs.begin() : nullptr, (int)attrs.size(), &t), "lt_op");
     return t;
 }
 
 // records the op, then releases the operands marked temporary (what a front end's reference counting does)
-lt_tensor op_t(int code, std::vector<lt_tensor> in, std::vector<int> temp, std::vector<int64_t> attrs = {}) {
+lt_tensor op_t(int code, std::initializer_list<lt_tensor> in, std::initializer_list<int> temp, std::initializer_list<int64_t> attrs = {}) {
     lt_tensor t = op(code, in, attrs);
-    for (int i : temp) check(lt_release(ctx, in[i]), "lt_release");
+    for (int i : temp) check(lt_release(ctx, in.begin()[i]), "lt_release");
     return t;
 }
 
@@ -57,10 +59,11 @@ void report(const char *name, int steps, double sec) {
     lt_get_stats(ctx, &st);
     const double b = (double)(st.barriers ? st.barriers : 1);
     printf("%-28s %8.2f us/step | per barrier: record %7.0f ns, canonicalise %7.0f, hash+lookup %6.0f, plan %6.0f, bind+launch %6.0f, "
-           "rebind %6.0f | nodes %llu, compiles %llu, hits %llu, replays %llu\n",
+           "rebind %6.0f | nodes %llu, compiles %llu, hits %llu (%llu by matched trace, %llu traces diverged), replays %llu\n",
            name, 1e6 * sec / steps, st.ns_record / b, st.ns_canonicalise / b, st.ns_hash_lookup / b, st.ns_plan / b,
            st.ns_bind_launch / (b + (double)st.replays), st.ns_rebind / (b + (double)st.replays), (unsigned long long)st.nodes_recorded,
-           (unsigned long long)st.compiles, (unsigned long long)st.cache_hits, (unsigned long long)st.replays);
+           (unsigned long long)st.compiles, (unsigned long long)st.cache_hits, (unsigned long long)st.traces_matched,
+           (unsigned long long)st.traces_diverged, (unsigned long long)st.replays);
 }
 
 void elementwise_chain(int steps) {
@@ -186,8 +189,8 @@ int main() {
     check(lt_ctx_create(LT_DEVICE_NONE, nullptr, nullptr, &ctx), "lt_ctx_create");
     elementwise_chain(20000);
     mlp_epilogue(20000);
-    adam(100, false);
-    adam(100, true);
+    adam(1000, false);
+    adam(1000, true);
     lt_ctx_destroy(ctx);
     return 0;
 }

@@ -452,8 +452,8 @@ def test_host_bench_driver_runs_without_python_in_the_loop():
     lines = out.strip().splitlines()
     assert len(lines) == 4
     assert "compiles 1, hits 19999" in lines[0] and "compiles 1, hits 19999" in lines[1]
-    assert "compiles 1, hits 99," in lines[2]
-    assert "replays 99" in lines[3]
+    assert "compiles 1, hits 999 (998 by matched trace, 0 traces diverged)" in lines[2]
+    assert "replays 999" in lines[3]
 
 
 # ------------------------------------------------------------------ long rows and the other reduction shapes
