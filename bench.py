@@ -647,7 +647,7 @@ def adam_steps(lt, torch, device: int) -> dict:
         res[f"c5_adam_100_steps_{mode}_ms_per_step"] = 10.0 * sec
         res[f"c5_adam_100_steps_{mode}_gbs"] = nbytes * 100 / sec / 1e9
         res[f"c5_adam_{mode}_cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "replays": st["replays"],
-                                         "kernels": st["kernels_launched"]}
+                                         "kernels": st["kernels_launched"], "traces_matched": st["traces_matched"]}
         if mode == "traced":
             res["c5_host_us_per_barrier"] = {k: st[k] / 1e3 / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
         del P, G, M, V

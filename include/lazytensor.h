@@ -201,6 +201,14 @@ lt_status lt_ctx_destroy(lt_ctx *ctx);
  * LT_KERNEL_LOG set: the compiler's log, with registers and shared memory of every kernel, goes to stderr),
  * "specialise_after" (3 default:
  * flushes of a plan before mode 2 asks for the kernel),
+ * "trace_match" (1 default: a trace -- the calls from one barrier to the next -- that repeats the previous trace call
+ * by call, on tensors related to one another in the same way, is bound to the previous trace's plan at the barrier
+ * without its graph being built, canonicalised or hashed (Section 7 of the paper: the cost of tracing again what has
+ * not changed).  Values of run-time scalars, seeds, inputs and their addresses may differ; anything else that differs
+ * makes the library build the graph of the calls so far after all, on the handles already returned, and go on as
+ * usual.  Results, errors and the meaning of every call are the same with 0; only lt_stats.traces_matched and the time
+ * differ.  A tensor released during a matched trace that the trace has read is unregistered at the barrier rather
+ * than at the call),
  * "log" (0 default; 1 = one line on stderr for every graph that is planned, i.e. every cache miss; 2 = also one
  * line per flush and per replay; preset by the environment variable LT_LOG),
  * "wait_limit_ms" (2000 default: how long a long-row kernel waits for one of its asynchronous copies into shared
