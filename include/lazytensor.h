@@ -294,7 +294,7 @@ lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
  * Barrier (Section 4; mark_step / LazyTensorBarrier): materialise every live tensor that
  * has pending computation.  With `blocking` non-zero, return after the stream has drained.
  * Row reductions over more than 8192 columns: a group whose program has a kernel instantiated at build time
- * (softmax, LayerNorm, RMSNorm and the other listed groups), or built by the run-time specialiser in mode 1, runs
+ * (softmax, LayerNorm, RMSNorm and the other listed groups), or built by the run-time specialiser (until then: as below), runs
  * fused -- up to 65536 columns with a thread-block cluster holding the row in registers, beyond that one thread block
  * per row walking it in slices -- when its inputs are 16-byte aligned and the row is a multiple of 8 elements; any other such graph runs
  * with each long reduction as a kernel of its own and the surrounding arithmetic as elementwise kernels.

@@ -455,7 +455,7 @@ int broadcast_class(const int64_t *dims, int rank, uint64_t rows, uint64_t cols)
 // executor (executor.cpp)
 lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_split = nullptr);
 lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran);
-bool long_rows_runnable(lt_ctx *c, const Plan &plan, const Canonical &cg);
+bool long_rows_runnable(lt_ctx *c, Plan &plan, const Canonical &cg);
 void fastdiv_make(uint32_t d, uint32_t *mul, uint32_t *sh1, uint32_t *sh2);
 
 }  // namespace lt

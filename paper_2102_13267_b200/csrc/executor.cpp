@@ -138,15 +138,25 @@ lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran) {
 
 // A fused long-row launch runs only on its compiled kernel, which needs 128-bit accesses: whole chunks per row
 // and 16-byte aligned inputs (results and temporaries come from the allocator, aligned).  Fills c->param_ptr.
-bool long_rows_runnable(lt_ctx *c, const Plan &plan, const Canonical &cg) {
+bool long_rows_runnable(lt_ctx *c, Plan &plan, const Canonical &cg) {
     c->param_ptr.resize(plan.n_params);
     for (uint32_t i = 0; i < plan.n_params; ++i)
         c->param_ptr[i] = c->buffers[c->nodes[cg.param_node[i]].buffer].ptr;
     if (c->device == LT_DEVICE_NONE) return true;
-    for (const Launch &L : plan.launches) {
+    for (Launch &L : plan.launches) {
         const Group &g = plan.groups[L.groups[0]];
         if (L.kind != K_ROW || !g.long_row) continue;
-        bool ok = c->opt.compiled && (L.compiled >= 0 || (L.jit && !L.jit_failed)) && (g.cols % LT_VM_V) == 0;
+        if (L.compiled < 0 && L.jit_program && !L.jit_failed && c->opt.compiled && c->opt.specialise == 2) {
+            // no kernel in the table: ask the specialiser once the plan keeps coming back, and use the kernel when it is there
+            if (!L.jit && (int64_t)++L.runs >= c->opt.specialise_after) {
+                L.jit = jit_request(*L.jit_program, false);
+                if (L.jit) c->stats.programs_specialised++;
+                else L.jit_failed = true;
+            }
+            if (L.jit && L.jit->state.load() < 0) L.jit_failed = true;
+        }
+        const bool have_kernel = L.compiled >= 0 || (L.jit && !L.jit_failed && L.jit->state.load() == 1);
+        bool ok = c->opt.compiled && have_kernel && (g.cols % LT_VM_V) == 0;
         for (size_t q = 0; q < g.io.size() && ok; ++q)
             if (g.io[q].kind == IO_PARAM && (g.io[q].cls <= LT_CLS_COLVEC || g.io[q].cls == LT_CLS_PITCHED))
                 ok = aligned_for((uint64_t)(uintptr_t)c->param_ptr[g.io[q].index] + g.io[q].offset * dtype_size(g.io[q].dtype), g.io[q].dtype) &&

@@ -1320,7 +1320,9 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
                 if (!L.jit || L.jit->state.load() != 1) L.jit_failed = true;
             }
         }
-        const bool long_ok = L.compiled >= 0 || (L.jit && !L.jit_failed);
+        // (in the background mode the group stays fused: until its kernel has been built the executor runs the plan's
+        // split variant instead, as it does when a fused launch meets unaligned pointers)
+        const bool long_ok = L.compiled >= 0 || (L.jit && !L.jit_failed) || (L.jit_program && c->opt.specialise == 2 && c->device != LT_DEVICE_NONE);
         if (g.long_row && (!long_ok || !c->opt.compiled)) unfused_long_row = true;
     }
     if (unfused_long_row) {

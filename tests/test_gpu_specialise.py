@@ -88,6 +88,36 @@ def test_specialised_in_the_background_takes_over_mid_stream(lt):
     c.close()
 
 
+def test_unlisted_long_rows_run_split_until_their_kernel_is_built(lt):
+    """Default mode: a long-row group that is not in the table runs with its reductions as kernels of their own while
+    the specialiser builds the fused kernel in the background, then fused -- every flush against the oracle."""
+    c = lt.LazyContext(device=0)
+    z = rng.normal_f32(rng.generator(85), (64, 16384))
+    O = EagerOracle()
+    ref = _row_normalise(O, O.leaf(z, "f32")).array
+    gz = c.leaf(z, "f32")
+    deadline = time.time() + 90
+    flushes = 0
+    while time.time() < deadline:
+        out = _row_normalise(c, gz)
+        c.barrier()
+        flushes += 1
+        assert_matches(c.fetch(out), ref, "f32", f"flush {flushes}")
+        if flushes == 1:
+            _needs_specialiser(c)
+            assert c.stats()["launches_reduce"] == 2  # the two long reductions on their own
+        if c.stats()["launches_specialised"] >= 2:
+            break
+        time.sleep(0.05)
+    st = c.stats()
+    # (the elementwise pieces of the split variant may have been handed to the specialiser as well)
+    assert st["launches_specialised"] >= 2 and st["compiles"] == 1 and st["programs_specialised"] >= 1, (st, c.dump_plan())
+    split_flushes = st["launches_reduce"] // 2
+    assert 3 <= split_flushes < flushes and st["launches_reduce"] == 2 * split_flushes  # nothing split once the kernel is there
+    assert st["launches_row"] == flushes - split_flushes
+    c.close()
+
+
 def test_specialised_long_rows_and_multi_tensor(lt):
     c = lt.LazyContext(device=0)
     c.set_option("specialise", 1)
