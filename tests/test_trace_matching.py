@@ -309,3 +309,35 @@ def test_random_programs_agree_with_plain_recording():
         matched += on.stats()["traces_matched"]
         diverged += on.stats()["traces_diverged"]
     assert matched > 100 and diverged > 50, (matched, diverged)  # both paths were exercised
+
+
+def test_errors_inside_a_matched_trace_are_the_usual_errors():
+    on, off = pair()
+    out = {}
+    for ctx in (on, off):
+        x, m = fake(ctx, (16, 16)), fake(ctx, (16, 16), "u8")
+        other = lt.LazyContext(device=None)
+        foreign = fake(other, (16, 16))
+        log = []
+        for k in range(5):
+            a = ctx.op("exp", x)
+            if k == 3:
+                for bad in (lambda: ctx.op("add", a, m),            # dtype mismatch
+                            lambda: ctx.op("add", a, foreign),      # a handle of another context
+                            lambda: ctx.op("row_sum", m)):          # not defined for u8
+                    with pytest.raises(lt.LazyTensorError) as err:
+                        bad()
+                    log.append(err.value.args[0] if err.value.args else str(err.value))
+            b = ctx.op("mul", a, a)
+            ctx.release(a)
+            if k >= 3:
+                with pytest.raises(lt.LazyTensorError):
+                    ctx.op("neg", a)                                # released: in a matched trace too
+            before = ctx.stats()
+            ctx.barrier()
+            log.append((delta(ctx, before), ctx.dump_plan(), ctx.is_materialised(b)))
+            del a, b
+        out[ctx] = log
+        other.close()
+    assert out[on] == out[off]
+    assert on.stats()["traces_matched"] >= 1
