@@ -62,7 +62,9 @@ cudaError_t launch_row(const LtKParams &P, unsigned grid, unsigned threads, unsi
 template <class PG>
 cudaError_t launch_one(const void *params, int u, unsigned grid, unsigned threads, unsigned group, unsigned group_log2,
                        unsigned depth, cudaStream_t stream) {
-    if constexpr (PG::kind == 0) {
+    if constexpr (PG::kind == 0 && Info<PG>::accum_slot() >= 0) {
+        return cudaErrorInvalidValue;  // launched through lt_compiled_launch_reduced
+    } else if constexpr (PG::kind == 0) {
         const LtKParams &P = *static_cast<const LtKParams *>(params);
         return u >= 2 ? launch_pdl(lt_c_ew<PG, 2>, grid, C_THREADS, 0, stream, P) : launch_pdl(lt_c_ew<PG, 1>, grid, C_THREADS, 0, stream, P);
     } else if constexpr (PG::kind == 1) {
@@ -86,7 +88,9 @@ cudaError_t row_occupancy(int threads, size_t dyn, int *blocks) {
 
 template <class PG>
 cudaError_t occupancy_one(int u, int threads, size_t dyn, int *blocks) {
-    if constexpr (PG::kind == 0) {
+    if constexpr (PG::kind == 0 && Info<PG>::accum_slot() >= 0) {
+        return cudaErrorInvalidValue;
+    } else if constexpr (PG::kind == 0) {
         return u >= 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_ew<PG, 2>, C_THREADS, 0)
                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, lt_c_ew<PG, 1>, C_THREADS, 0);
     } else if constexpr (PG::kind == 1) {
@@ -226,6 +230,27 @@ cudaError_t rowc_one(const LtKParams *P, int u, bool shared_vectors, unsigned cl
 }
 
 }  // namespace
+
+namespace {
+template <class PG>
+cudaError_t launch_reduced(const LtKParams &P, unsigned gx, unsigned gy, unsigned rows_per, cudaStream_t stream) {
+    if constexpr (PG::kind == 0 && Info<PG>::accum_slot() >= 0) {
+        return launch_pdl_grid(lt_c_ewred<PG>, dim3(gx, gy), (unsigned)C_THREADS, stream, P, (uint32_t)rows_per);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+}
+}  // namespace
+
+cudaError_t lt_compiled_launch_reduced(int id, const void *params, unsigned gx, unsigned gy, unsigned rows_per, cudaStream_t stream) {
+    int k = 0;
+#define LT_X(PG)                                                                                            \
+    if (k == id) return launch_reduced<PG>(*static_cast<const LtKParams *>(params), gx, gy, rows_per, stream); \
+    ++k;
+    LT_COMPILED_LIST(LT_X)
+#undef LT_X
+    return cudaErrorInvalidValue;
+}
 
 size_t lt_compiled_cluster_vector_bytes(int id, int u) {
     int k = 0;

@@ -47,6 +47,11 @@ cudaError_t lt_compiled_launch_cluster(int id, const void *params, int u, int sh
                                        unsigned depth, uint64_t limit_ns, cudaStream_t stream);
 cudaError_t lt_compiled_cluster_occupancy(int id, int u, int shared_vectors, unsigned cluster_size, unsigned depth, int *max_clusters);
 size_t lt_compiled_cluster_vector_bytes(int id, int u);
+// An elementwise entry whose result is reduced instead of stored (a slot of class LT_CLS_REDUCED...): the first stage,
+// a grid of gx x gy CTAs of 256 threads.  Reduction over the rows of every column: gx = ceil(chunks per row / 32), CTA row
+// `by` takes the rows [by * rows_per, ..) and writes cols binary64 partials at partial + by * cols.  Over everything:
+// gy = 1 and gx partials.  The second stage is lt_launch_reduce_final (launch.h).
+cudaError_t lt_compiled_launch_reduced(int id, const void *params, unsigned gx, unsigned gy, unsigned rows_per, cudaStream_t stream);
 // Device status word (bit 0: a bounded wait gave up); synchronises the device.  `clear` resets it when set.
 cudaError_t lt_device_status_read(unsigned int *out, int clear);
 // Launches a one-warp kernel that waits `limit_ns` for an mbarrier phase nothing completes and then raises bit 0.

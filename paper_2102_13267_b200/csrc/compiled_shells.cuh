@@ -97,13 +97,21 @@ struct Info {
         for (int t = 0; t < LT_VM_NT; ++t) n += pro_slot(t) >= 0 ? 1 : 0;
         return n;
     }
+    // the slot whose value the program reduces instead of storing (LT_CLS_REDUCED...), or -1
+    static constexpr __host__ __device__ int accum_slot() {
+        for (int s = 0; s < PG::n_slots; ++s)
+            if (PG::cls[s] >= LT_CLS_REDUCED) return s;
+        return -1;
+    }
+    static constexpr __host__ __device__ int accum_axis() { return accum_slot() < 0 ? 0 : (PG::cls[accum_slot()] - LT_CLS_REDUCED) / 3; }
+    static constexpr __host__ __device__ int accum_kind() { return accum_slot() < 0 ? 0 : (PG::cls[accum_slot()] - LT_CLS_REDUCED) % 3; }
     static constexpr __host__ __device__ bool needs_coords() {
         for (int k = 0; k < PG::n_ins; ++k) {
             const uint32_t op = PG::ins[k].op;
             if (op == OP_IOTA_COL || op == OP_IOTA_ROW) return true;
         }
         for (int s = 0; s < PG::n_slots; ++s)
-            if (PG::cls[s] != LT_CLS_FULL) return true;
+            if (PG::cls[s] != LT_CLS_FULL && PG::cls[s] < LT_CLS_REDUCED) return true;
         return false;
     }
 };
@@ -292,6 +300,59 @@ struct Coords {
 // No row reductions in this shell.
 struct NoReduce {
     template <int KIND, int U, bool GUARD>
+    __device__ __forceinline__ void operator()(float (&)[U][V], const bool (&)[U]) const {}
+};
+
+// An elementwise program whose result is reduced over columns or over everything: the thread keeps one accumulator
+// per lane (a thread owns the same columns throughout, or the lanes are folded at the end).  Sums are kept in binary64
+// and rounded once, when the second stage writes the result; the two chunks a thread computes per iteration are added
+// in binary32 first (one conversion and one binary64 addition per two elements: the conversions, not memory, bound
+// the kernel otherwise), an error of at most 2^-24 of each pair's sum, independent of how many rows there are.  Max
+// and min are exact in binary32 and propagate NaN.
+template <bool B, class X, class Y>
+struct PickType { using type = X; };
+template <class X, class Y>
+struct PickType<false, X, Y> { using type = Y; };
+
+template <int KIND>
+struct AccumReduce {
+    using Acc = typename PickType<KIND == 0, double, float>::type;
+    Acc a[V];
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int i = 0; i < V; ++i) a[i] = KIND == 0 ? (Acc)0 : (KIND == 1 ? (Acc)-LT_INF : (Acc)LT_INF);
+    }
+    static __device__ __forceinline__ double comb(double x, double y) {
+        if constexpr (KIND == 0) return x + y;
+        else if constexpr (KIND == 1) return (x != x || y != y) ? x + y : (x > y ? x : y);
+        else return (x != x || y != y) ? x + y : (x < y ? x : y);
+    }
+    static __device__ __forceinline__ float combf(float x, float y) {
+        if constexpr (KIND == 1) return max_nan(x, y);
+        else return min_nan(x, y);
+    }
+    // the values of the thread's two chunks of this iteration (either may be absent)
+    __device__ __forceinline__ void put(const float (&v0)[V], bool ok0, const float (&v1)[V], bool ok1) {
+        if constexpr (KIND == 0) {
+            if (ok0 && ok1) {
+#pragma unroll
+                for (int i = 0; i < V; ++i) a[i] += (double)__fadd_rn(v0[i], v1[i]);
+            } else if (ok0 || ok1) {
+#pragma unroll
+                for (int i = 0; i < V; ++i) a[i] += (double)(ok0 ? v0[i] : v1[i]);
+            }
+        } else {
+            if (ok0) {
+#pragma unroll
+                for (int i = 0; i < V; ++i) a[i] = combf(a[i], v0[i]);
+            }
+            if (ok1) {
+#pragma unroll
+                for (int i = 0; i < V; ++i) a[i] = combf(a[i], v1[i]);
+            }
+        }
+    }
+    template <int K2, int U, bool GUARD>
     __device__ __forceinline__ void operator()(float (&)[U][V], const bool (&)[U]) const {}
 };
 
@@ -531,8 +592,22 @@ struct Machine {
 #pragma unroll
             for (int u = 0; u < U; ++u) source<LT_VM_SRC_S, imm>(acc[u], u);
         } else if constexpr (op == OP_ST) {
-            static_assert(PG::cls[imm] == LT_CLS_FULL || PG::cls[imm] == LT_CLS_ROWVEC, "results are full-class or one value per row");
-            if constexpr (PG::cls[imm] == LT_CLS_FULL) {
+            static_assert(PG::cls[imm] == LT_CLS_FULL || PG::cls[imm] == LT_CLS_ROWVEC || PG::cls[imm] >= LT_CLS_REDUCED,
+                          "results are full-class, one value per row, or reduced");
+            if constexpr (PG::cls[imm] >= LT_CLS_REDUCED) {
+                // the values, rounded as the store they replace would round them, go into the thread's accumulators
+                static_assert(U == 2, "the reducing shell computes two chunks per iteration");
+                constexpr bool to_bf16 = PG::dtype[imm] == LT_ST_BF16;
+                float v[2][V];
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+#pragma unroll
+                    for (int i = 0; i < V; ++i) {
+                        if constexpr (to_bf16) v[u][i] = round_bf16(acc[u][i]);
+                        else v[u][i] = acc[u][i];
+                    }
+                red.put(v[0], !GUARD || ck.ok[0], v[1], !GUARD || ck.ok[1]);
+            } else if constexpr (PG::cls[imm] == LT_CLS_FULL) {
 #pragma unroll
                 for (int u = 0; u < U; ++u)
                     if (!GUARD || ck.ok[u]) chunk_store<PG::dtype[imm]>(acc[u], const_cast<char *>(address<imm>(u)));
@@ -932,6 +1007,94 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
     if (full) iterate(FalseTag{});
     else iterate(TrueTag{});
     if (depth) cp_async_wait(0);
+}
+
+// An elementwise program whose result is reduced over the rows of every column, or over everything, instead of
+// being stored (LT_CLS_REDUCED): the first of two stages.  Columns: CTA (bx, by) of 32 x 8 threads takes the 32 chunks
+// of columns bx * 256 .. and the rows [by * rows_per, ..); thread (x, y) owns one chunk of eight columns and walks rows
+// y, y + 8, .., two at a time; the eight row lanes meet in shared memory and the CTA writes one binary64 partial per
+// column to partial[by * cols + col].  Everything: chunks strided over the grid, partial[bx] per CTA.  The partials
+// are what lt_reduce_cols / lt_reduce_all of reduce.cu read in their second stage.  Rows are whole chunks.
+template <class PG>
+__global__ void __launch_bounds__(C_THREADS) lt_c_ewred(const __grid_constant__ LtKParams P, uint32_t rows_per) {
+    constexpr int SLOT = Info<PG>::accum_slot(), AXIS = Info<PG>::accum_axis(), KIND = Info<PG>::accum_kind();
+    using R = AccumReduce<KIND>;
+    __shared__ double smem[AXIS == 0 ? 8 * (32 * V + 1) : C_THREADS / 32];
+    const PtrK ptr{P};
+    const ScalK scal{P};
+    R red;
+    red.reset();
+    double *partial = reinterpret_cast<double *>(P.ptr[SLOT]);
+    pdl_release();
+    pdl_wait();
+    if constexpr (AXIS == 0) {
+        const uint32_t x = threadIdx.x & 31u, y = threadIdx.x >> 5;
+        const uint32_t cchunk = blockIdx.x * 32u + x;
+        const uint32_t r0 = blockIdx.y * rows_per;
+        const uint32_t r1 = r0 + rows_per < P.rows ? r0 + rows_per : P.rows;
+        if (cchunk < P.cpr) {
+            for (uint32_t r = r0 + y; r < r1; r += 16) {
+                Coords<2> ck;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const uint32_t row = r + 8u * u;
+                    ck.ok[u] = row < r1;
+                    ck.row[u] = ck.ok[u] ? row : r;
+                    ck.col0[u] = cchunk * V;
+                    ck.flat0[u] = (uint64_t)ck.row[u] * P.cols + ck.col0[u];
+                }
+                Machine<PG, 2, PtrK, ScalK, R, true> m(ptr, scal, red, ck);
+                m.issue_loads();
+                m.run();
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < V; ++i) smem[y * (32 * V + 1) + x * V + i] = (double)red.a[i];
+        __syncthreads();
+        const uint32_t col = blockIdx.x * 32u * V + threadIdx.x;  // 256 threads, 256 columns
+        if (col < P.cols) {
+            double v = smem[threadIdx.x];
+#pragma unroll
+            for (int k = 1; k < 8; ++k) v = R::comb(v, smem[k * (32 * V + 1) + threadIdx.x]);
+            partial[(uint64_t)blockIdx.y * P.cols + col] = v;
+        }
+    } else {
+        const uint32_t n_chunks = (uint32_t)P.n_chunks;
+        const uint32_t stride = gridDim.x * C_THREADS;
+        for (uint32_t c = blockIdx.x * C_THREADS + threadIdx.x; c < n_chunks; c += 2 * stride) {
+            Coords<2> ck;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const uint32_t cx = c + u * stride;
+                ck.ok[u] = cx < n_chunks;
+                const uint32_t cu = ck.ok[u] ? cx : 0u;
+                ck.flat0[u] = (uint64_t)cu * V;
+                if (Info<PG>::needs_coords() && P.rowcol) {
+                    const uint32_t q = __umulhi(P.div_mul, cu);
+                    const uint32_t row = (q + ((cu - q) >> P.div_sh1)) >> P.div_sh2;
+                    ck.row[u] = row;
+                    ck.col0[u] = (cu - row * P.cpr) * V;
+                } else {
+                    ck.row[u] = 0;
+                    ck.col0[u] = cu * V;
+                }
+            }
+            Machine<PG, 2, PtrK, ScalK, R, true> m(ptr, scal, red, ck);
+            m.issue_loads();
+            m.run();
+        }
+        double v = R::comb(R::comb(R::comb((double)red.a[0], (double)red.a[1]), R::comb((double)red.a[2], (double)red.a[3])),
+                           R::comb(R::comb((double)red.a[4], (double)red.a[5]), R::comb((double)red.a[6], (double)red.a[7])));
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v = R::comb(v, __shfl_xor_sync(0xffffffffu, v, off));
+        if ((threadIdx.x & 31u) == 0) smem[threadIdx.x >> 5] = v;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double r = smem[0];
+            for (int w = 1; w < C_THREADS / 32; ++w) r = R::comb(r, smem[w]);
+            partial[blockIdx.x] = r;
+        }
+    }
 }
 
 // Multi-tensor: every tensor is a flat range of chunks; a super-chunk is 2048 consecutive chunks.

@@ -136,8 +136,9 @@ lt_status run_plan(lt_ctx *c, Plan *plan, const Canonical &cg, Plan **ran) {
     return execute_plan(c, *plan->split, cg, nullptr);
 }
 
-// A fused long-row launch runs only on its compiled kernel, which needs 128-bit accesses: whole chunks per row
-// and 16-byte aligned inputs (results and temporaries come from the allocator, aligned).  Fills c->param_ptr.
+// A fused long-row launch, and an elementwise launch that reduces its result, run only on their compiled kernels,
+// which need 128-bit accesses: whole chunks per row and 16-byte aligned inputs (results and temporaries come from
+// the allocator, aligned).  Fills c->param_ptr.
 bool long_rows_runnable(lt_ctx *c, Plan &plan, const Canonical &cg) {
     c->param_ptr.resize(plan.n_params);
     for (uint32_t i = 0; i < plan.n_params; ++i)
@@ -145,7 +146,7 @@ bool long_rows_runnable(lt_ctx *c, Plan &plan, const Canonical &cg) {
     if (c->device == LT_DEVICE_NONE) return true;
     for (Launch &L : plan.launches) {
         const Group &g = plan.groups[L.groups[0]];
-        if (L.kind != K_ROW || !g.long_row) continue;
+        if (!(L.kind == K_ROW && g.long_row) && !(L.kind == K_EW && g.fused_red)) continue;
         if (L.compiled < 0 && L.jit_program && !L.jit_failed && c->opt.compiled && c->opt.specialise == 2) {
             // no kernel in the table: ask the specialiser once the plan keeps coming back, and use the kernel when it is there
             if (!L.jit && (int64_t)++L.runs >= c->opt.specialise_after) {
@@ -280,8 +281,12 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
             if (!dry) {
                 void *scratch = g.scratch_temp >= 0 ? c->temp_ptr[g.scratch_temp] : nullptr;
                 if (ev0) cudaEventRecord(ev0, c->stream);
-                e = lt_launch_reduce(g.red_axis, g.red_kind, g.io[0].dtype, (const void *)(uintptr_t)resolve(g.io[0]),
-                                     (void *)(uintptr_t)resolve(g.io[1]), scratch, g.rows, g.cols, c->sm_count, c->stream, &launched);
+                if (g.from_partials)  // the kernel that computed the input left the first stage's partial results in scratch
+                    e = lt_launch_reduce_final(g.red_axis, g.red_kind, g.io[1].dtype, scratch, (void *)(uintptr_t)resolve(g.io[1]),
+                                               lt_reduce_parts(g.red_axis, g.rows, g.cols, c->sm_count), g.cols, c->stream);
+                else
+                    e = lt_launch_reduce(g.red_axis, g.red_kind, g.io[0].dtype, (const void *)(uintptr_t)resolve(g.io[0]),
+                                         (void *)(uintptr_t)resolve(g.io[1]), scratch, g.rows, g.cols, c->sm_count, c->stream, &launched);
                 if (ev1) cudaEventRecord(ev1, c->stream);
             }
             c->stats.launches_reduce += 1;
@@ -404,7 +409,37 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                 }
             }
             bool done = false;
-            if (g.long_row) {
+            if (g.fused_red) {
+                // the group's kernel reduces one of its results: first stage here, second in the reduction group that follows
+                if (!dry) {
+                    if (specialised(L)) {
+                        std::string err;
+                        if (!jit_load(*L.jit, c->device, &err)) {
+                            release_all(true);
+                            return fail(c, LT_ERR_CUDA, err);
+                        }
+                    }
+                    const unsigned parts = lt_reduce_parts(g.red_axis, g.rows, g.cols, c->sm_count);
+                    const unsigned gx = g.red_axis == 1 ? (P.cpr + 31u) / 32u : parts, gy = g.red_axis == 1 ? parts : 1u;
+                    uint32_t rows_per = (uint32_t)((g.rows + parts - 1) / parts);
+                    if (ev0) cudaEventRecord(ev0, c->stream);
+                    if (specialised(L)) {
+                        void *args[2] = {&P, &rows_per};
+                        std::string err;
+                        if (!jit_launch(*L.jit, c->device, 0, gx, 256, 0, (void *)c->stream, args, &err, 0, gy)) {
+                            c->error = err;
+                            e = cudaErrorLaunchFailure;
+                        } else {
+                            c->stats.launches_specialised++;
+                        }
+                    } else {
+                        e = lt_compiled_launch_reduced(L.compiled, &P, gx, gy, rows_per, c->stream);
+                    }
+                    if (ev1) cudaEventRecord(ev1, c->stream);
+                }
+                c->stats.launches_compiled++;
+                done = true;
+            } else if (g.long_row) {
                 // a CTA per row, walking it in slices; rows staged in shared memory `depth` ahead when they fit
                 // (feasibility was checked on entry)
                 if (!dry && specialised(L)) {

@@ -103,6 +103,15 @@ def programs():
         ins = [d.leaf((16, 64) if k.startswith("mat") else (64,), k.split(":")[1]) for k in kinds]
         keep = trace(d.ctx, ins, 64)
         out.append((name, d.keys()))
+    # reductions of a computed value: the program whose kernel reduces instead of storing (planned as such only when a
+    # kernel for it exists: here the run-time specialiser builds one while planning; shapes large enough for two stages)
+    for name, kinds, trace in idioms.REDUCED:
+        d = Dry(specialise=1)
+        ins = [d.leaf((4096, 64), k.split(":")[1]) for k in kinds]
+        keep = trace(d.ctx, ins, 64)
+        keys = [k for k in d.keys() if any(int(c) >= 8 for c in k.split("|")[2].split())]
+        assert len(keys) == 1, (name, keys)
+        out.append((name, keys))
     d = Dry()
     shapes = [(64,), (128,)]
     P, G, Bf = ([d.leaf(s, "f32") for s in shapes] for _ in range(3))
@@ -161,7 +170,7 @@ def check(name, kind, n_pro, cls, ins):
         assert not (OP_MOV_T_ACC <= op < OP_MOV_T_ACC + NT and op - OP_MOV_T_ACC in reserved), f"{name}: reserved temporary overwritten"
         assert not (OP_LD <= op < OP_LD + NT and op - OP_LD in reserved), f"{name}: reserved temporary overwritten"
         if op == OP_ST:
-            assert cls[imm] in (0, 2), f"{name}: compiled kernels store full-class results or one value per row"
+            assert cls[imm] in (0, 2) or (kind == 0 and cls[imm] >= 8), f"{name}: compiled kernels store full-class results, one value per row, or reduce"
 
 
 def render() -> tuple[str, list[str]]:

@@ -132,7 +132,8 @@ std::string program_struct(const JitProgram &p) {
 // kernel instantiations one program needs: (name expression, slot in JitKernel::fn)
 std::vector<std::pair<std::string, int>> variants_of(const JitProgram &p) {
     std::vector<std::pair<std::string, int>> v;
-    if (p.kind == 0) v.push_back({"lt_c_ew<JP, 1>", 0});
+    if (p.kind == 0 && jit_reduced_slot(p) >= 0) v.push_back({"lt_c_ewred<JP>", 0});
+    else if (p.kind == 0) v.push_back({"lt_c_ew<JP, 1>", 0});
     else if (p.kind == 2) v.push_back({std::string("lt_c_multi<JP, ") + (p.flavour == 2 ? "1" : "2") + ">", 0});
     else if (p.long_row) {
         v.push_back({"lt_c_longrow<JP, 256>", 0});
@@ -408,7 +409,7 @@ int jit_cluster_occupancy(JitKernel &k, int device, int variant, int threads, un
 }
 
 bool jit_launch(JitKernel &k, int device, int variant, unsigned grid, unsigned threads, size_t dyn_smem, void *stream, void **args,
-                std::string *err, unsigned cluster) {
+                std::string *err, unsigned cluster, unsigned grid_y) {
     CUfunction f = (CUfunction)fn_of(k, device, variant);
     if (!f) {
         if (err) *err = "specialised kernel not loaded";
@@ -425,7 +426,8 @@ bool jit_launch(JitKernel &k, int device, int variant, unsigned grid, unsigned t
     CUlaunchConfig cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDimX = grid;
-    cfg.gridDimY = cfg.gridDimZ = 1;
+    cfg.gridDimY = grid_y ? grid_y : 1;
+    cfg.gridDimZ = 1;
     cfg.blockDimX = threads;
     cfg.blockDimY = cfg.blockDimZ = 1;
     cfg.sharedMemBytes = (unsigned)dyn_smem;
@@ -491,6 +493,12 @@ int jit_reductions(const JitProgram &p) {
     return n;
 }
 
+int jit_reduced_slot(const JitProgram &p) {
+    for (size_t s = 0; s < p.cls.size(); ++s)
+        if (p.cls[s] >= LT_CLS_REDUCED) return (int)s;
+    return -1;
+}
+
 size_t jit_cluster_vector_bytes(const JitProgram &p, int u) {
     bool reserved[LT_VM_NT] = {false};
     size_t n = 0;
@@ -514,7 +522,9 @@ bool jit_supported(const JitProgram &p) {
         const uint32_t op = p.ins[k].op;
         if (op >= OP_MOV_T_ACC && op < OP_MOV_T_ACC + LT_VM_NT && reserved[op - OP_MOV_T_ACC]) return false;
         if (op >= OP_LD && op < OP_LD + LT_VM_NT && reserved[op - OP_LD]) return false;
-        if (op == OP_ST && p.cls[p.ins[k].imm] != LT_CLS_FULL && p.cls[p.ins[k].imm] != LT_CLS_ROWVEC) return false;
+        if (op == OP_ST && p.cls[p.ins[k].imm] != LT_CLS_FULL && p.cls[p.ins[k].imm] != LT_CLS_ROWVEC &&
+            !(p.kind == 0 && p.cls[p.ins[k].imm] >= LT_CLS_REDUCED))
+            return false;
     }
     return jit_reductions(p) <= 4;
 }

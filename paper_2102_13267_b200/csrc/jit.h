@@ -49,13 +49,15 @@ bool jit_load(JitKernel &k, int device, std::string *err);
 int jit_occupancy(JitKernel &k, int device, int variant, int threads, size_t dyn_smem);
 // `cluster` > 0: the grid is launched as thread-block clusters of that many CTAs.
 bool jit_launch(JitKernel &k, int device, int variant, unsigned grid, unsigned threads, size_t dyn_smem, void *stream, void **args,
-                std::string *err, unsigned cluster = 0);
+                std::string *err, unsigned cluster = 0, unsigned grid_y = 1);
 // Clusters of `cluster` CTAs of `threads` threads the device holds at once (0: unknown or none).
 int jit_cluster_occupancy(JitKernel &k, int device, int variant, int threads, unsigned cluster, size_t dyn_smem);
 size_t jit_row_stage_bytes(const JitProgram &p, int u, int threads);
 bool jit_integer_heavy(const JitProgram &p);
 size_t jit_long_stage_bytes(const JitProgram &p, uint32_t cols);
 int jit_reductions(const JitProgram &p);
+// The slot an elementwise program reduces instead of storing (class LT_CLS_REDUCED...), or -1.
+int jit_reduced_slot(const JitProgram &p);
 // Shared memory the cluster row kernel needs to keep the program's column vectors at `u` chunks per thread (0: it has none).
 size_t jit_cluster_vector_bytes(const JitProgram &p, int u);
 

@@ -31,6 +31,12 @@ cudaError_t lt_static_scratch_clear_enqueue(void *base, size_t bytes, int sm_cou
 size_t lt_reduce_scratch_bytes(int axis, uint64_t rows, uint64_t cols, int sm_count);
 cudaError_t lt_launch_reduce(int axis, int kind, int dtype, const void *in, void *out, void *scratch, uint64_t rows, uint64_t cols,
                              int sm_count, cudaStream_t stream, unsigned *launched);
+// How many partial results the first stage leaves per column (axis 1) or in all (axis 2); <= 1: one stage, no scratch.
+unsigned lt_reduce_parts(int axis, uint64_t rows, uint64_t cols, int sm_count);
+// The second stage alone: `parts` binary64 partial results per column (axis 1, partials[part * cols + col]) or in all
+// (axis 2) -- what the first stage, or an elementwise kernel that reduces its result (lt_c_ewred), left in scratch.
+cudaError_t lt_launch_reduce_final(int axis, int kind, int dtype, const void *partials, void *out, unsigned parts, uint64_t cols,
+                                   cudaStream_t stream);
 
 // views.cu: copy kernels of the shape operations.  `op` is the lt_opcode (reshape 60, narrow 61, permute 62,
 // update_slice 63); in_dims is the (first) input's shape (reshape: {numel}), out_dims the result's (update_slice:

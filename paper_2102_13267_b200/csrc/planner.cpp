@@ -1098,6 +1098,45 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             return fail(c, LT_ERR_UNSUPPORTED, "tensor too large for 32-bit chunk indexing");
     }
 
+    // ---- a column or whole-tensor reduction whose input is computed by an elementwise group for it alone: the first
+    // stage moves into that group (its kernel reduces the value instead of storing it, lt_c_ewred), the reduction
+    // group keeps the second stage.  The input is never materialised.  Only kernels built for the program can do
+    // this; the split variant of the plan is the graph without it.
+    if (fuse && !isolate_long_rows && c->opt.compiled) {
+        for (size_t g2i = 0; g2i < groups.size(); ++g2i) {
+            Group &g2 = groups[g2i];
+            if (g2.kind != K_RED || g2.red_axis == 0 || g2.scratch_temp < 0 || g2.io.size() != 2 || g2.io[0].kind != IO_TEMP) continue;
+            const uint32_t v = g2.io[0].cnode;
+            const int g1i = pn[v].group;
+            if (g1i < 0 || (size_t)g1i >= g2i) continue;
+            Group &g1 = groups[g1i];
+            if (g1.kind != K_EW || g1.fused_red || g1.rows != g2.rows || g1.cols != g2.cols) continue;
+            if (g2.rows >= (1ull << 31) || g2.cols >= (1ull << 31)) continue;
+            const bool whole_chunks = (g1.rowcol || g2.red_axis == 1) ? (g1.cols % LT_VM_V) == 0 : ((g1.rows * g1.cols) % LT_VM_V) == 0;
+            if (!whole_chunks) continue;
+            size_t readers = 0;
+            for (const Group &g : groups)
+                for (const IoRef &io : g.io)
+                    if (!io.is_store && io.kind == IO_TEMP && io.cnode == v) ++readers;
+            int st = -1;
+            for (size_t q = 0; q < g1.io.size(); ++q)
+                if (g1.io[q].is_store && g1.io[q].kind == IO_TEMP && g1.io[q].cnode == v && g1.io[q].cls == LT_CLS_FULL) st = (int)q;
+            if (readers != 1 || st < 0) continue;
+            plan.temp_bytes[pn[v].temp] = 0;  // nothing is written there any more
+            IoRef &out = g1.io[st];
+            out.cls = (uint8_t)(LT_CLS_REDUCED + 3 * (g2.red_axis - 1) + g2.red_kind);
+            out.index = (uint32_t)g2.scratch_temp;
+            g1.fused_red = true;
+            g1.red_axis = g2.red_axis;
+            g1.red_kind = g2.red_kind;
+            if (g2.red_axis == 1) g1.rowcol = true;  // the kernel walks rows and columns
+            g2.from_partials = true;
+            g2.io[0].index = (uint32_t)g2.scratch_temp;
+            g1.bytes -= g1.rows * g1.cols * dtype_size(out.dtype);
+            g2.bytes = 0;
+        }
+    }
+
     // ---- outputs
     plan.n_params = (uint32_t)cg.param_node.size();
     plan.n_dyn = (uint32_t)cg.dyn.size();
@@ -1315,7 +1354,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             }
             if (jit_supported(*jp)) L.jit_program = std::move(jp);
             // a long-row group is only worth keeping fused if its kernel is there when the flush runs
-            if (L.jit_program && g.long_row && c->opt.specialise == 1) {
+            if (L.jit_program && (g.long_row || g.fused_red) && c->opt.specialise == 1) {
                 L.jit = jit_request(*L.jit_program, true);
                 if (!L.jit || L.jit->state.load() != 1) L.jit_failed = true;
             }
@@ -1323,7 +1362,7 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
         // (in the background mode the group stays fused: until its kernel has been built the executor runs the plan's
         // split variant instead, as it does when a fused launch meets unaligned pointers)
         const bool long_ok = L.compiled >= 0 || (L.jit && !L.jit_failed) || (L.jit_program && c->opt.specialise == 2 && c->device != LT_DEVICE_NONE);
-        if (g.long_row && (!long_ok || !c->opt.compiled)) unfused_long_row = true;
+        if ((g.long_row || g.fused_red) && (!long_ok || !c->opt.compiled)) unfused_long_row = true;
     }
     if (unfused_long_row) {
         // Only the kernels instantiated at build time walk a long row in slices.  A long-row group without one is
@@ -1352,6 +1391,8 @@ std::string describe_plan(const Plan &plan) {
         }
     static const char *kind[] = {"elementwise", "row", "multi", "reduce", "view"};
     static const char *cls[] = {"full", "colvec", "rowvec", "scalar", "pitched"};
+    static const char *reduced[] = {"reduced-over-rows(sum)", "reduced-over-rows(max)", "reduced-over-rows(min)",
+                                    "reduced-over-all(sum)",  "reduced-over-all(max)",  "reduced-over-all(min)"};
     static const char *iok[] = {"param", "output", "temp"};
     for (size_t li = 0; li < plan.launches.size(); ++li) {
         const Launch &L = plan.launches[li];
@@ -1365,7 +1406,8 @@ std::string describe_plan(const Plan &plan) {
             s += buf;
         } else if (L.kind == K_RED) {
             static const char *axis[] = {"rows", "columns", "all"}, *what[] = {"sum", "max", "min"};
-            snprintf(buf, sizeof(buf), "  reduction kernel: %s over %s%s\n", what[g.red_kind], axis[g.red_axis], g.scratch_temp >= 0 ? ", two stages" : "");
+            snprintf(buf, sizeof(buf), "  reduction kernel: %s over %s%s\n", what[g.red_kind], axis[g.red_axis],
+                     g.from_partials ? ", second stage only (the first is in the kernel that computes the input)" : g.scratch_temp >= 0 ? ", two stages" : "");
             s += buf;
         } else {
             // the exact identity of the program: what the table of compiled programs is keyed on
@@ -1385,7 +1427,7 @@ std::string describe_plan(const Plan &plan) {
         for (size_t q = 0; q < g.io.size(); ++q) {
             const IoRef &io = g.io[q];
             snprintf(buf, sizeof(buf), "  p%zu: %s %s %s %s%u\n", q, io.is_store ? "store" : "load", dtype_name(io.dtype),
-                     cls[io.cls], iok[io.kind], io.index);
+                     io.cls >= LT_CLS_REDUCED ? reduced[io.cls - LT_CLS_REDUCED] : cls[io.cls], iok[io.kind], io.index);
             s += buf;
         }
         for (size_t q = 0; q < g.imms.size(); ++q) {

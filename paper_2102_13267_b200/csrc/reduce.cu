@@ -230,6 +230,28 @@ size_t lt_reduce_scratch_bytes(int axis, uint64_t rows, uint64_t cols, int sm_co
     return axis == 1 ? (size_t)parts * cols * sizeof(double) : (size_t)parts * sizeof(double);
 }
 
+namespace {
+template <int DT, int KIND>
+cudaError_t launch_final(int axis, const void *partials, void *out, unsigned parts, uint64_t cols, cudaStream_t stream) {
+    constexpr int F64 = 5;
+    if (axis == 1) {
+        const unsigned gx = (unsigned)((cols + ((cols % 4) == 0 ? 127 : 31)) / ((cols % 4) == 0 ? 128 : 32));
+        return (cols % 4) == 0 ? launch_pdl_grid(lt_reduce_cols<F64, DT, KIND, 4>, dim3(gx, 1), RT, stream, partials, out, (uint64_t)parts, cols, (uint64_t)parts)
+                               : launch_pdl_grid(lt_reduce_cols<F64, DT, KIND, 1>, dim3(gx, 1), RT, stream, partials, out, (uint64_t)parts, cols, (uint64_t)parts);
+    }
+    return launch_pdl(lt_reduce_all<F64, DT, KIND>, 1u, RT, (size_t)0, stream, partials, out, (uint64_t)parts);
+}
+}  // namespace
+
+cudaError_t lt_launch_reduce_final(int axis, int kind, int dtype, const void *partials, void *out, unsigned parts, uint64_t cols, cudaStream_t stream) {
+    if (dtype != 0 && dtype != 1) return cudaErrorInvalidValue;
+#define LT_FINAL(DT)                                                                              \
+    (kind == 0 ? launch_final<DT, 0>(axis, partials, out, parts, cols, stream)                    \
+               : kind == 1 ? launch_final<DT, 1>(axis, partials, out, parts, cols, stream) : launch_final<DT, 2>(axis, partials, out, parts, cols, stream))
+    return dtype == 0 ? LT_FINAL(0) : LT_FINAL(1);
+#undef LT_FINAL
+}
+
 cudaError_t lt_launch_reduce(int axis, int kind, int dtype, const void *in, void *out, void *scratch, uint64_t rows, uint64_t cols,
                              int sm_count, cudaStream_t stream, unsigned *launched) {
     const unsigned parts = lt_reduce_parts(axis, rows, cols, sm_count);

@@ -52,6 +52,10 @@ struct LtIns {
 // element classes of a pointer slot relative to the group's [rows, cols] domain
 // LT_CLS_PITCHED: a full-class operand whose rows lie `pitch` elements apart (a slice of wider rows, read in place)
 enum { LT_CLS_FULL = 0, LT_CLS_COLVEC = 1, LT_CLS_ROWVEC = 2, LT_CLS_SCALAR = 3, LT_CLS_PITCHED = 4 };
+// LT_CLS_REDUCED + 3 * axis + kind: a store slot of an elementwise program whose value is not written but reduced --
+// over the rows of every column (axis 0) or over everything (axis 1); kind 0 sum, 1 max, 2 min -- into binary64
+// partial results that a second, small kernel finishes (compiled shells only)
+enum { LT_CLS_REDUCED = 8 };
 // storage dtypes (same numbering as lt_dtype)
 enum { LT_ST_F32 = 0, LT_ST_BF16 = 1, LT_ST_U8 = 2, LT_ST_I32 = 3, LT_ST_U32 = 4 };
 

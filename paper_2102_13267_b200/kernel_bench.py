@@ -1,6 +1,6 @@
 """Kernel-only timing of the benchmark configurations and of the common fusion groups (also the driver for ncu captures).
 
-    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5,idioms,long,reduce] [--iters N] [--sets K] [key=value ...]
+    python -m paper_2102_13267_b200.kernel_bench [c1,c2,c2p,c3,c4,c5,idioms,long,reduce,reduced] [--iters N] [--sets K] [key=value ...]
 
 For each configuration: traces the graph and flushes it `iters` times over rotating buffer sets (larger than L2
 together), queued behind a busy stream so that the GPU, not the host, sets the pace.  Two figures are printed:
@@ -214,6 +214,31 @@ def main() -> None:
                         lambda c, s_, op=op: c.op(op, s_[0]))
         generic("row_sum 4096x65536", 4 * 4096 * 65536, lambda c: [c.from_torch(torch.randn((4096, 65536), device=dev))],
                 lambda c, s_: c.op("row_sum", s_[0]))
+        # reductions of a computed value, (a - b)^2: the two inputs are all that has to move (run with specialise=1 to have
+        # the fused kernel from the first flush, specialise=0 for the unfused plan)
+        for op in ("col_sum", "all_sum"):
+            for dt, es in (("f32", 4), ("bf16", 2)):
+                def make(c, dt=dt):
+                    ts = [torch.randn((16384, 4096), device=dev) for _ in range(2)]
+                    return [c.from_torch(t.to(torch.bfloat16) if dt == "bf16" else t) for t in ts]
+
+                def trace(c, s_, op=op):
+                    d = c.op("sub", s_[0], s_[1])
+                    return c.op(op, c.op("mul", d, d))
+
+                generic(f"{op} (a-b)^2 {dt}", 2 * es * 16384 * 4096, make, trace)
+    if "reduced" in which:  # reductions of computed values (workloads/idioms.py REDUCED) on [16384 x 4096]: inputs are all that moves
+        for iname, kinds, trace in idioms.REDUCED:
+            nbytes = sum((2 if k.endswith("bf16") else 4) * 16384 * 4096 for k in kinds)
+
+            def make(c, kinds=kinds):
+                out = []
+                for k in kinds:
+                    t = torch.randn((16384, 4096), device=dev)
+                    out.append(c.from_torch(t.to(torch.bfloat16) if k.endswith("bf16") else t))
+                return out
+
+            generic(iname, nbytes, make, lambda c, s_, trace=trace: trace(c, s_, 4096))
     if "c5" in which:
         shapes = parameter_shapes()
         ctx = context()

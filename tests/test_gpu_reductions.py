@@ -298,3 +298,114 @@ def test_replay_of_a_graph_with_reduction_kernels_and_a_view(lt):
     assert_matches(c.fetch(x), ox.array, "f32", "base after three replays")
     assert_matches(c.fetch(keep), np.ascontiguousarray(ok.array), "f32", "view after three replays")
     c.close()
+
+
+# ------------------------------------------------------------------ reductions fused with the computation of their input
+def _sq_diff(B, a, b):
+    d = B.op("sub", a, b)
+    return B.op("mul", d, d)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(4096, 1024), (1000, 264), (33, 8), (5000, 40), (2, 3, 4096), (70000, 16)])
+@pytest.mark.parametrize("name", ["col_sum", "col_max", "col_min", "all_sum", "all_max", "all_min"])
+def test_reduction_of_a_computed_value_runs_inside_the_kernel_that_computes_it(lt, name, shape, dtype):
+    """col / all reduction of an elementwise expression that nothing else reads: the expression's kernel reduces it
+    (first stage) instead of storing it; the reduction group runs only its second stage."""
+    c = lt.LazyContext(device=0)
+    c.set_option("specialise", 1)  # the kernel for this (unlisted) program is built while the graph is planned
+    g = rng.generator(71)
+    a, b = rng.normal_f32(g, shape), rng.normal_f32(g, shape)
+    if dtype == "bf16":
+        a, b = rng.to_bf16_bits(a), rng.to_bf16_bits(b)
+    O = EagerOracle()
+    ref = O.op(name, _sq_diff(O, O.leaf(a, dtype), O.leaf(b, dtype)))
+    out = c.op(name, _sq_diff(c, c.leaf(a, dtype), c.leaf(b, dtype)))
+    c.barrier()
+    if "specialised at run time" not in c.dump_plan():
+        pytest.skip("the run-time compiler library is not installed")
+    plan, st = c.dump_plan(), c.stats()
+    rows = int(np.prod(shape[:-1]))
+    if rows >= 128 or (name.startswith("all") and rows * shape[-1] > 8192):  # large enough for two stages: fused
+        assert "second stage only" in plan and "reduced-over-" in plan, plan
+        assert st["kernels_launched"] == 2 and st["launches_specialised"] == 1 and st["temporaries_allocated"] >= 1, st
+    assert_matches(c.fetch(out), ref.array, dtype, f"fused {name} {dtype} {shape}")
+    c.close()
+
+
+def test_fused_reduction_keeps_other_results_and_nan_semantics(lt):
+    c = lt.LazyContext(device=0)
+    c.set_option("specialise", 1)
+    shape = (777, 512)
+    x = rng.normal_f32(rng.generator(72), shape)
+    x[5, 7] = np.nan
+    O = EagerOracle()
+
+    def graph(B, t):
+        e = B.op("exp", B.op("mul", t, B.scalar(0.5)))          # also a result of its own
+        m = B.op("col_max", B.op("abs", B.op("sub", e, t)))     # NaN in column 7 must come through
+        return e, m
+
+    (re, rm), (ge, gm) = graph(O, O.leaf(x, "f32")), graph(c, c.leaf(x, "f32"))
+    c.barrier()
+    if "specialised at run time" not in c.dump_plan():
+        pytest.skip("the run-time compiler library is not installed")
+    assert "second stage only" in c.dump_plan()
+    assert_matches(c.fetch(ge), re.array, "f32", "value stored next to the reduction")
+    got = c.fetch(gm)
+    assert np.isnan(got[0, 7]) and np.isnan(rm.array[0, 7])
+    assert_matches(got, rm.array, "f32", "column max with a NaN")
+    c.close()
+
+
+def test_fused_reduction_falls_back_when_it_cannot_run(lt):
+    """Rows that are not whole chunks, a value that something else reads, and (default mode) the flushes before the
+    specialiser has built the kernel all run the reduction on a materialised input -- same values."""
+    O = EagerOracle()
+    for shape, extra_reader in (((300, 100), False), ((512, 256), True)):
+        c = lt.LazyContext(device=0)
+        c.set_option("specialise", 1)
+        a = rng.normal_f32(rng.generator(73), shape)
+        oa, ga = O.leaf(a, "f32"), c.leaf(a, "f32")
+        outs = []
+        for B, t in ((O, oa), (c, ga)):
+            sq = B.op("mul", t, t)
+            r = B.op("col_sum", sq)
+            outs.append((r, B.op("row_sum", sq) if extra_reader else None))
+        c.barrier()
+        assert "second stage only" not in c.dump_plan()
+        assert_matches(c.fetch(outs[1][0]), outs[0][0].array, "f32", f"unfused {shape}")
+        c.close()
+    c = lt.LazyContext(device=0)  # default mode
+    a = rng.normal_f32(rng.generator(74), (2048, 512))
+    ref = O.op("all_sum", O.op("mul", O.leaf(a, "f32"), O.leaf(a, "f32"))).array
+    ga = c.leaf(a, "f32")
+    import time
+    deadline, fused_flushes, flushes = time.time() + 90, 0, 0
+    while time.time() < deadline and fused_flushes < 2:
+        out = c.op("all_sum", c.op("mul", ga, ga))
+        before = c.stats()["launches_specialised"]
+        c.barrier()
+        flushes += 1
+        assert_matches(c.fetch(out), ref, "f32", f"flush {flushes}")
+        fused_flushes += c.stats()["launches_specialised"] - before
+        time.sleep(0.05)
+    if "specialised at run time" in c.dump_plan():
+        assert fused_flushes >= 2 and flushes >= 5, (flushes, c.stats())
+    c.close()
+
+
+@pytest.mark.parametrize("shape", [(2048, 1024), (777, 136), (40000, 8)])
+@pytest.mark.parametrize("idiom", [e[0] for e in idioms.REDUCED])
+def test_listed_reductions_of_computed_values(ctx, idiom, shape):
+    """Gradient norms, squared errors, bias gradients, scales: kernels built ahead of time, fused from the first flush."""
+    name, kinds, trace = next(e for e in idioms.REDUCED if e[0] == idiom)
+    arrs = _idiom_inputs(kinds, shape, 75)
+    O = EagerOracle()
+    ref = trace(O, [O.leaf(a, d) for a, d in arrs], shape[-1])
+    out = trace(ctx, [ctx.leaf(a, d) for a, d in arrs], shape[-1])
+    ctx.barrier()
+    plan, st = ctx.dump_plan(), ctx.stats()
+    assert f"compiled: {name}" in plan and "second stage only" in plan, plan
+    assert st["kernels_launched"] == 2 and st["launches_compiled"] == 1 and st["launches_specialised"] == 0, st
+    assert_matches(ctx.fetch(out), ref.array, "f32", f"{name} {shape}")

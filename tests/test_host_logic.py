@@ -688,3 +688,34 @@ def test_kernel_cache_directory_is_written_and_read(tmp_path, monkeypatch):
     second = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
     assert "READY" in second.stdout, second.stdout + second.stderr
     assert files[0].stat().st_mtime_ns == stamp and len(list(tmp_path.glob("*"))) == 1  # read, not rewritten
+
+
+def test_reductions_of_computed_values_are_planned_into_the_computing_kernel(ctx):
+    """col / all reduction of an elementwise value nothing else reads: the value's group reduces it (slot class
+    'reduced-over-...'), the reduction group keeps its second stage -- when a kernel for that program exists."""
+    from workloads import idioms
+
+    x, y = fake(ctx, (4096, 256), "bf16"), fake(ctx, (4096, 256), "bf16")
+    g = idioms.relu_bias_grad(ctx, x, y, cols=256)
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert plan.count("launch ") == 2 and "compiled: relu_bias_grad_bf16" in plan, plan
+    assert "reduced-over-rows(sum)" in plan and "second stage only" in plan
+    assert plan.splitlines()[0].endswith("2 temporaries")  # the value's own (empty) and the partial results
+    # not in the table and no kernel built while planning (no device, background mode): the value is materialised
+    z = ctx.op("col_max", ctx.op("tanh", ctx.op("convert", x, dtype="f32")))
+    ctx.barrier()
+    plan = ctx.dump_plan()
+    assert "second stage only" not in plan and "reduction kernel: max over columns, two stages" in plan, plan
+    # small inputs reduce in one stage: nothing to fuse
+    s = fake(ctx, (4, 64))
+    w = ctx.op("all_sum", ctx.op("mul", s, s))
+    ctx.barrier()
+    assert "second stage only" not in ctx.dump_plan()
+    # a value with another reader, or rows that are not whole chunks, stay as they were
+    a = fake(ctx, (4096, 100))
+    sq = ctx.op("mul", a, a)
+    u = ctx.op("all_sum", sq)
+    ctx.barrier()
+    assert "second stage only" not in ctx.dump_plan()
+    del g, z, w, u, sq

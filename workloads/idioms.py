@@ -116,3 +116,53 @@ ALL = [
     ("scale_to_f32", ("mat:bf16",), lambda B, ins, cols: scale_to_f32(B, *ins, cols=cols)),
     ("scaled_softmax_bf16", ("mat:bf16",), lambda B, ins, cols: scaled_softmax(B, *ins, cols=cols)),
 ]
+
+
+# ---- reductions of a computed value (over the rows of every column, or over everything): the value's kernel does the
+# first stage of the reduction instead of storing it.  Same signature as ALL.
+def _f32(B, t, dtype):
+    return t if dtype == "f32" else B.op("convert", t, dtype="f32")
+
+
+def sum_squares(B, x, *, cols, dtype="f32"):
+    """||x||^2, the gradient-norm building block."""
+    xf = _f32(B, x, dtype)
+    return B.op("all_sum", B.op("mul", xf, xf))
+
+
+def squared_error_sum(B, a, b, *, cols, dtype="f32"):
+    d = B.op("sub", _f32(B, a, dtype), _f32(B, b, dtype))
+    return B.op("all_sum", B.op("mul", d, d))
+
+
+def column_squared_error(B, a, b, *, cols, dtype="f32"):
+    d = B.op("sub", _f32(B, a, dtype), _f32(B, b, dtype))
+    return B.op("col_sum", B.op("mul", d, d))
+
+
+def bias_grad(B, dy, *, cols, dtype="bf16"):
+    """Gradient of a broadcast bias: column sums of dy, accumulated from its f32 values."""
+    return B.op("col_sum", _f32(B, dy, dtype))
+
+
+def relu_bias_grad(B, dy, x, *, cols, dtype="bf16"):
+    """Column sums of dy where the forward input was positive."""
+    g = B.op("where", B.op("gt", _f32(B, x, dtype), B.scalar(0.0)), _f32(B, dy, dtype), B.scalar(0.0))
+    return B.op("col_sum", g)
+
+
+def abs_max(B, x, *, cols, dtype="f32"):
+    """max |x|: the scale of a tensor."""
+    return B.op("all_max", B.op("abs", _f32(B, x, dtype)))
+
+
+REDUCED = [
+    ("sum_squares_f32", ("mat:f32",), lambda B, ins, cols: sum_squares(B, *ins, cols=cols)),
+    ("sum_squares_bf16", ("mat:bf16",), lambda B, ins, cols: sum_squares(B, *ins, cols=cols, dtype="bf16")),
+    ("squared_error_sum_f32", ("mat:f32", "mat:f32"), lambda B, ins, cols: squared_error_sum(B, *ins, cols=cols)),
+    ("column_squared_error_f32", ("mat:f32", "mat:f32"), lambda B, ins, cols: column_squared_error(B, *ins, cols=cols)),
+    ("bias_grad_bf16", ("mat:bf16",), lambda B, ins, cols: bias_grad(B, *ins, cols=cols)),
+    ("relu_bias_grad_bf16", ("mat:bf16", "mat:bf16"), lambda B, ins, cols: relu_bias_grad(B, *ins, cols=cols)),
+    ("abs_max_f32", ("mat:f32",), lambda B, ins, cols: abs_max(B, *ins, cols=cols)),
+    ("abs_max_bf16", ("mat:bf16",), lambda B, ins, cols: abs_max(B, *ins, cols=cols, dtype="bf16")),
+]
