@@ -322,13 +322,14 @@ def test_reduction_of_a_computed_value_runs_inside_the_kernel_that_computes_it(l
     ref = O.op(name, _sq_diff(O, O.leaf(a, dtype), O.leaf(b, dtype)))
     out = c.op(name, _sq_diff(c, c.leaf(a, dtype), c.leaf(b, dtype)))
     c.barrier()
-    if "specialised at run time" not in c.dump_plan():
-        pytest.skip("the run-time compiler library is not installed")
     plan, st = c.dump_plan(), c.stats()
+    listed = "compiled: no" not in plan.split("launch 1:")[0]  # (a - b)^2 summed is one of the listed programs
+    if "specialised at run time" not in plan and not listed:
+        pytest.skip("the run-time compiler library is not installed")
     rows = int(np.prod(shape[:-1]))
     if rows >= 128 or (name.startswith("all") and rows * shape[-1] > 8192):  # large enough for two stages: fused
         assert "second stage only" in plan and "reduced-over-" in plan, plan
-        assert st["kernels_launched"] == 2 and st["launches_specialised"] == 1 and st["temporaries_allocated"] >= 1, st
+        assert st["kernels_launched"] == 2 and st["launches_specialised"] == (0 if listed else 1) and st["launches_compiled"] == 1, st
     assert_matches(c.fetch(out), ref.array, dtype, f"fused {name} {dtype} {shape}")
     c.close()
 
