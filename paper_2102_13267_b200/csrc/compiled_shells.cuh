@@ -104,7 +104,23 @@ struct Info {
         return -1;
     }
     static constexpr __host__ __device__ int accum_axis() { return accum_slot() < 0 ? 0 : (PG::cls[accum_slot()] - LT_CLS_REDUCED) / 3; }
-    static constexpr __host__ __device__ int accum_kind() { return accum_slot() < 0 ? 0 : (PG::cls[accum_slot()] - LT_CLS_REDUCED) % 3; }
+    // a program may reduce several values (all over the same axis): how many, the k-th one's slot, a slot's ordinal and kind
+    static constexpr __host__ __device__ int n_accum() {
+        int n = 0;
+        for (int s = 0; s < PG::n_slots; ++s) n += PG::cls[s] >= LT_CLS_REDUCED ? 1 : 0;
+        return n;
+    }
+    static constexpr __host__ __device__ int accum_slot_at(int k) {
+        for (int s = 0; s < PG::n_slots; ++s)
+            if (PG::cls[s] >= LT_CLS_REDUCED && k-- == 0) return s;
+        return -1;
+    }
+    static constexpr __host__ __device__ int accum_ordinal(int slot) {
+        int n = 0;
+        for (int s = 0; s < slot; ++s) n += PG::cls[s] >= LT_CLS_REDUCED ? 1 : 0;
+        return n;
+    }
+    static constexpr __host__ __device__ int accum_kind_of(int slot) { return (PG::cls[slot] - LT_CLS_REDUCED) % 3; }
     static constexpr __host__ __device__ bool needs_coords() {
         for (int k = 0; k < PG::n_ins; ++k) {
             const uint32_t op = PG::ins[k].op;
@@ -309,19 +325,10 @@ struct NoReduce {
 // in binary32 first (one conversion and one binary64 addition per two elements: the conversions, not memory, bound
 // the kernel otherwise), an error of at most 2^-24 of each pair's sum, independent of how many rows there are.  Max
 // and min are exact in binary32 and propagate NaN.
-template <bool B, class X, class Y>
-struct PickType { using type = X; };
-template <class X, class Y>
-struct PickType<false, X, Y> { using type = Y; };
+constexpr int C_MAX_REDUCED = 3;  // values one elementwise program may reduce
 
 template <int KIND>
-struct AccumReduce {
-    using Acc = typename PickType<KIND == 0, double, float>::type;
-    Acc a[V];
-    __device__ __forceinline__ void reset() {
-#pragma unroll
-        for (int i = 0; i < V; ++i) a[i] = KIND == 0 ? (Acc)0 : (KIND == 1 ? (Acc)-LT_INF : (Acc)LT_INF);
-    }
+struct AccumOps {
     static __device__ __forceinline__ double comb(double x, double y) {
         if constexpr (KIND == 0) return x + y;
         else if constexpr (KIND == 1) return (x != x || y != y) ? x + y : (x > y ? x : y);
@@ -331,24 +338,46 @@ struct AccumReduce {
         if constexpr (KIND == 1) return max_nan(x, y);
         else return min_nan(x, y);
     }
+    static __device__ __forceinline__ double ident() { return KIND == 0 ? 0.0 : (KIND == 1 ? -(double)LT_INF : (double)LT_INF); }
+};
+
+// The accumulators of N reduced values: binary64 for sums, binary32 for max / min (only what a value's kind uses is kept).
+template <int N>
+struct AccumSet {
+    double sum[N][V];
+    float ext[N][V];
+    template <int ORD, int KIND>
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            if constexpr (KIND == 0) sum[ORD][i] = 0.0;
+            else ext[ORD][i] = KIND == 1 ? -LT_INF : LT_INF;
+        }
+    }
+    template <int ORD, int KIND>
+    __device__ __forceinline__ double get(int i) const {
+        if constexpr (KIND == 0) return sum[ORD][i];
+        else return (double)ext[ORD][i];
+    }
     // the values of the thread's two chunks of this iteration (either may be absent)
+    template <int ORD, int KIND>
     __device__ __forceinline__ void put(const float (&v0)[V], bool ok0, const float (&v1)[V], bool ok1) {
         if constexpr (KIND == 0) {
             if (ok0 && ok1) {
 #pragma unroll
-                for (int i = 0; i < V; ++i) a[i] += (double)__fadd_rn(v0[i], v1[i]);
+                for (int i = 0; i < V; ++i) sum[ORD][i] += (double)__fadd_rn(v0[i], v1[i]);
             } else if (ok0 || ok1) {
 #pragma unroll
-                for (int i = 0; i < V; ++i) a[i] += (double)(ok0 ? v0[i] : v1[i]);
+                for (int i = 0; i < V; ++i) sum[ORD][i] += (double)(ok0 ? v0[i] : v1[i]);
             }
         } else {
             if (ok0) {
 #pragma unroll
-                for (int i = 0; i < V; ++i) a[i] = combf(a[i], v0[i]);
+                for (int i = 0; i < V; ++i) ext[ORD][i] = AccumOps<KIND>::combf(ext[ORD][i], v0[i]);
             }
             if (ok1) {
 #pragma unroll
-                for (int i = 0; i < V; ++i) a[i] = combf(a[i], v1[i]);
+                for (int i = 0; i < V; ++i) ext[ORD][i] = AccumOps<KIND>::combf(ext[ORD][i], v1[i]);
             }
         }
     }
@@ -606,7 +635,7 @@ struct Machine {
                         if constexpr (to_bf16) v[u][i] = round_bf16(acc[u][i]);
                         else v[u][i] = acc[u][i];
                     }
-                red.put(v[0], !GUARD || ck.ok[0], v[1], !GUARD || ck.ok[1]);
+                red.template put<I::accum_ordinal(imm), I::accum_kind_of(imm)>(v[0], !GUARD || ck.ok[0], v[1], !GUARD || ck.ok[1]);
             } else if constexpr (PG::cls[imm] == LT_CLS_FULL) {
 #pragma unroll
                 for (int u = 0; u < U; ++u)
@@ -1015,16 +1044,63 @@ __global__ void __launch_bounds__(C_ROW_THREADS) lt_c_row(const __grid_constant_
 // y, y + 8, .., two at a time; the eight row lanes meet in shared memory and the CTA writes one binary64 partial per
 // column to partial[by * cols + col].  Everything: chunks strided over the grid, partial[bx] per CTA.  The partials
 // are what lt_reduce_cols / lt_reduce_all of reduce.cu read in their second stage.  Rows are whole chunks.
+// writes the partial results of the ORD-th reduced value (see lt_c_ewred), then those of the next
+template <class PG, int ORD, class R>
+__device__ __forceinline__ void ewred_finish(const LtKParams &P, const R &red, double *smem) {
+    if constexpr (ORD < Info<PG>::n_accum()) {
+        constexpr int SLOT = Info<PG>::accum_slot_at(ORD), KIND = Info<PG>::accum_kind_of(SLOT);
+        using Ops = AccumOps<KIND>;
+        double *partial = reinterpret_cast<double *>(P.ptr[SLOT]);
+        if constexpr (ORD > 0) __syncthreads();  // the previous value's partials have been read
+        if constexpr (Info<PG>::accum_axis() == 0) {
+            const uint32_t x = threadIdx.x & 31u, y = threadIdx.x >> 5;
+#pragma unroll
+            for (int i = 0; i < V; ++i) smem[y * (32 * V + 1) + x * V + i] = red.template get<ORD, KIND>(i);
+            __syncthreads();
+            const uint32_t col = blockIdx.x * 32u * V + threadIdx.x;  // 256 threads, 256 columns
+            if (col < P.cols) {
+                double v = smem[threadIdx.x];
+#pragma unroll
+                for (int k = 1; k < 8; ++k) v = Ops::comb(v, smem[k * (32 * V + 1) + threadIdx.x]);
+                partial[(uint64_t)blockIdx.y * P.cols + col] = v;
+            }
+        } else {
+            double v = Ops::comb(Ops::comb(Ops::comb(red.template get<ORD, KIND>(0), red.template get<ORD, KIND>(1)),
+                                           Ops::comb(red.template get<ORD, KIND>(2), red.template get<ORD, KIND>(3))),
+                                 Ops::comb(Ops::comb(red.template get<ORD, KIND>(4), red.template get<ORD, KIND>(5)),
+                                           Ops::comb(red.template get<ORD, KIND>(6), red.template get<ORD, KIND>(7))));
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v = Ops::comb(v, __shfl_xor_sync(0xffffffffu, v, off));
+            if ((threadIdx.x & 31u) == 0) smem[threadIdx.x >> 5] = v;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                double r = smem[0];
+                for (int w = 1; w < C_THREADS / 32; ++w) r = Ops::comb(r, smem[w]);
+                partial[blockIdx.x] = r;
+            }
+        }
+        ewred_finish<PG, ORD + 1>(P, red, smem);
+    }
+}
+
+template <class PG, int ORD, class R>
+__device__ __forceinline__ void ewred_reset(R &red) {
+    if constexpr (ORD < Info<PG>::n_accum()) {
+        red.template reset<ORD, Info<PG>::accum_kind_of(Info<PG>::accum_slot_at(ORD))>();
+        ewred_reset<PG, ORD + 1>(red);
+    }
+}
+
 template <class PG>
 __global__ void __launch_bounds__(C_THREADS) lt_c_ewred(const __grid_constant__ LtKParams P, uint32_t rows_per) {
-    constexpr int SLOT = Info<PG>::accum_slot(), AXIS = Info<PG>::accum_axis(), KIND = Info<PG>::accum_kind();
-    using R = AccumReduce<KIND>;
+    constexpr int AXIS = Info<PG>::accum_axis();
+    static_assert(Info<PG>::n_accum() >= 1 && Info<PG>::n_accum() <= C_MAX_REDUCED, "reduced values per program");
+    using R = AccumSet<Info<PG>::n_accum()>;
     __shared__ double smem[AXIS == 0 ? 8 * (32 * V + 1) : C_THREADS / 32];
     const PtrK ptr{P};
     const ScalK scal{P};
     R red;
-    red.reset();
-    double *partial = reinterpret_cast<double *>(P.ptr[SLOT]);
+    ewred_reset<PG, 0>(red);
     pdl_release();
     pdl_wait();
     if constexpr (AXIS == 0) {
@@ -1047,16 +1123,6 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_ewred(const __grid_constant__ 
                 m.issue_loads();
                 m.run();
             }
-        }
-#pragma unroll
-        for (int i = 0; i < V; ++i) smem[y * (32 * V + 1) + x * V + i] = (double)red.a[i];
-        __syncthreads();
-        const uint32_t col = blockIdx.x * 32u * V + threadIdx.x;  // 256 threads, 256 columns
-        if (col < P.cols) {
-            double v = smem[threadIdx.x];
-#pragma unroll
-            for (int k = 1; k < 8; ++k) v = R::comb(v, smem[k * (32 * V + 1) + threadIdx.x]);
-            partial[(uint64_t)blockIdx.y * P.cols + col] = v;
         }
     } else {
         const uint32_t n_chunks = (uint32_t)P.n_chunks;
@@ -1083,18 +1149,8 @@ __global__ void __launch_bounds__(C_THREADS) lt_c_ewred(const __grid_constant__ 
             m.issue_loads();
             m.run();
         }
-        double v = R::comb(R::comb(R::comb((double)red.a[0], (double)red.a[1]), R::comb((double)red.a[2], (double)red.a[3])),
-                           R::comb(R::comb((double)red.a[4], (double)red.a[5]), R::comb((double)red.a[6], (double)red.a[7])));
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) v = R::comb(v, __shfl_xor_sync(0xffffffffu, v, off));
-        if ((threadIdx.x & 31u) == 0) smem[threadIdx.x >> 5] = v;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            double r = smem[0];
-            for (int w = 1; w < C_THREADS / 32; ++w) r = R::comb(r, smem[w]);
-            partial[blockIdx.x] = r;
-        }
     }
+    ewred_finish<PG, 0>(P, red, smem);
 }
 
 // Multi-tensor: every tensor is a flat range of chunks; a super-chunk is 2048 consecutive chunks.

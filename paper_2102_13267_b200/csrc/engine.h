@@ -137,7 +137,7 @@ struct Group {
     uint8_t red_axis = 0;           // K_RED: 0 rows, 1 columns, 2 everything
     uint8_t red_kind = 0;           // K_RED: 0 sum, 1 max, 2 min
     int32_t scratch_temp = -1;      // K_RED: temporary that holds the partial results, or -1
-    bool fused_red = false;         // K_EW: one result is reduced (red_axis 1 or 2, red_kind) into partial results instead of being stored
+    bool fused_red = false;         // K_EW: up to three results are reduced over red_axis (1 or 2) into partial results instead of being stored (slot classes LT_CLS_REDUCED...)
     bool from_partials = false;     // K_RED: the first stage ran inside the elementwise kernel that computes the input
     uint16_t view_op = 0;           // K_VIEW: LT_OP_RESHAPE / NARROW / PERMUTE / UPDATE_SLICE
     uint8_t view_rank = 0;

@@ -1110,7 +1110,12 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             const int g1i = pn[v].group;
             if (g1i < 0 || (size_t)g1i >= g2i) continue;
             Group &g1 = groups[g1i];
-            if (g1.kind != K_EW || g1.fused_red || g1.rows != g2.rows || g1.cols != g2.cols) continue;
+            if (g1.kind != K_EW || g1.rows != g2.rows || g1.cols != g2.cols) continue;
+            if (g1.fused_red) {  // a group may reduce up to three values, all over the same axis
+                size_t have = 0;
+                for (const IoRef &io : g1.io) have += io.cls >= LT_CLS_REDUCED ? 1 : 0;
+                if (g1.red_axis != g2.red_axis || have >= 3) continue;
+            }
             if (g2.rows >= (1ull << 31) || g2.cols >= (1ull << 31)) continue;
             const bool whole_chunks = (g1.rowcol || g2.red_axis == 1) ? (g1.cols % LT_VM_V) == 0 : ((g1.rows * g1.cols) % LT_VM_V) == 0;
             if (!whole_chunks) continue;
@@ -1128,7 +1133,6 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             out.index = (uint32_t)g2.scratch_temp;
             g1.fused_red = true;
             g1.red_axis = g2.red_axis;
-            g1.red_kind = g2.red_kind;
             if (g2.red_axis == 1) g1.rowcol = true;  // the kernel walks rows and columns
             g2.from_partials = true;
             g2.io[0].index = (uint32_t)g2.scratch_temp;

@@ -410,3 +410,30 @@ def test_listed_reductions_of_computed_values(ctx, idiom, shape):
     assert f"compiled: {name}" in plan and "second stage only" in plan, plan
     assert st["kernels_launched"] == 2 and st["launches_compiled"] == 1 and st["launches_specialised"] == 0, st
     assert_matches(ctx.fetch(out), ref.array, "f32", f"{name} {shape}")
+
+
+@pytest.mark.parametrize("shape", [(3000, 512), (513, 72)])
+def test_several_reductions_of_values_one_group_computes(lt, shape):
+    """LayerNorm-backward style: column sums of dy * xhat and of dy, and a column maximum, from one pass over the inputs."""
+    c = lt.LazyContext(device=0)
+    c.set_option("specialise", 1)
+    g = rng.generator(76)
+    dy, xh = rng.to_bf16_bits(rng.normal_f32(g, shape)), rng.to_bf16_bits(rng.normal_f32(g, shape))
+    O = EagerOracle()
+
+    def graph(B, a, b):
+        af, bf = B.op("convert", a, dtype="f32"), B.op("convert", b, dtype="f32")
+        return [B.op("col_sum", B.op("mul", af, bf)), B.op("col_sum", B.op("mul", af, B.scalar(1.0))),
+                B.op("col_max", B.op("abs", B.op("sub", af, bf)))]
+
+    ref = graph(O, O.leaf(dy, "bf16"), O.leaf(xh, "bf16"))
+    out = graph(c, c.leaf(dy, "bf16"), c.leaf(xh, "bf16"))
+    c.barrier()
+    plan, st = c.dump_plan(), c.stats()
+    if "specialised at run time" not in plan:
+        pytest.skip("the run-time compiler library is not installed")
+    assert plan.count("second stage only") == 3 and plan.count("reduced-over-rows") == 3, plan
+    assert st["kernels_launched"] == 4 and st["launches_specialised"] == 1, st
+    for k, (t, r) in enumerate(zip(out, ref)):
+        assert_matches(c.fetch(t), r.array, "f32", f"reduction {k} {shape}")
+    c.close()
