@@ -407,6 +407,13 @@ def run_ours(args) -> None:
         extra["host_ns_per_barrier"] = {k: st[k] / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
         extra["cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "barriers": st["barriers"]}
         extra["c5_data_parallel_adam_step"] = dp_adam
+        # the same program on the other two tiers, beside the headline: the interpreter serves a program that is not in
+        # the build-time table until the run-time specialiser has built its kernel
+        oc = extra.get("other_configs", {}).get("c2", {})
+        if "interpreted_gbs" in oc:
+            roofline["same_graph_on_the_interpreter"] = {"achieved": oc["interpreted_gbs"], "frac": oc["interpreted_gbs"] / peak}
+        if "specialised_gbs" in oc:
+            roofline["same_graph_specialised_at_run_time"] = {"achieved": oc["specialised_gbs"], "frac": oc["specialised_gbs"] / peak}
     cpu = cpu_baseline() if world == 1 and not args.no_cpu else None
 
     line = {
@@ -484,6 +491,7 @@ def extra_measurements(ctx, lt, torch, timed, step, sets, nbytes) -> dict:
     del o
     out.update(adam_steps(lt, torch, ctx.device))
     out["other_configs"] = other_configs(lt, torch, ctx.device)
+    out["wider_reductions"] = wider_reductions(lt, torch, ctx.device)
     return out
 
 
@@ -599,6 +607,67 @@ def other_configs(lt, torch, device: int) -> dict:
         entry["specialised_frac_of_measured_peak"] = entry["specialised_gbs"] / peak
         if "unfused_us" in entry:
             entry["speedup_vs_unfused"] = entry["unfused_us"] / entry["fused_us"]
+        res[name] = entry
+    return res
+
+
+def wider_reductions(lt, torch, device: int) -> dict:
+    """Beyond the five configurations: rows of 16384 columns (cluster row kernel) and reductions of computed values
+    (first stage inside the computing kernel), each against the plan without that kernel.  Timed like other_configs."""
+    import math as _m
+
+    from workloads import idioms
+
+    dev = torch.device("cuda", device)
+    peak, _ = measured_peak()
+
+    def inputs(c, kinds, shape):
+        out = []
+        for k in kinds:
+            t = torch.randn(shape if k.startswith("mat") else (shape[-1],), device=dev)
+            out.append(c.from_torch(t.to(torch.bfloat16) if k.endswith("bf16") else t))
+        return out
+
+    long_shape, red_shape = (8192, 16384), (16384, 4096)
+    cases = []
+    for name in ("softmax_bf16", "layernorm_bf16"):
+        _, kinds, trace = next(e for e in idioms.ALL if e[0] == name)
+        cases.append((f"{name}_16384_columns", kinds, trace, long_shape, 2 * 2 * long_shape[0] * long_shape[1], {"debug.cluster": 1}, "cta_per_row"))
+    for name in ("sum_squares_f32", "relu_bias_grad_bf16"):
+        _, kinds, trace = next(e for e in idioms.REDUCED if e[0] == name)
+        nbytes = sum((2 if k.endswith("bf16") else 4) * red_shape[0] * red_shape[1] for k in kinds)
+        cases.append((name, kinds, trace, red_shape, nbytes, {"specialise": 0, "debug.ignore_table": 1}, "unfused"))
+    res = {}
+    for name, kinds, trace, shape, nbytes, other, other_name in cases:
+        entry = {}
+        for mode, opts in (("", {}), (other_name, other)):
+            c = lt.LazyContext(device=device)
+            for k, v in opts.items():
+                c.set_option(k, v)
+            nsets = max(2, _m.ceil(1.2e9 / nbytes))
+            sets = [inputs(c, kinds, shape) for _ in range(nsets)]
+            keep = [None] * nsets
+            for i in range(nsets + 2):
+                keep[i % nsets] = trace(c, sets[i % nsets], shape[-1])
+                c.barrier()
+            torch.cuda.synchronize()
+            iters = 20
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(int(4e-3 * 1.9e9))
+            e0.record()
+            for i in range(iters):
+                keep[i % nsets] = trace(c, sets[i % nsets], shape[-1])
+                c.barrier()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / iters
+            pre = f"{mode}_" if mode else ""
+            entry[f"{pre}us"] = 1e3 * ms
+            entry[f"{pre}gbs"] = nbytes / ms / 1e6
+            if not mode:
+                entry["frac_of_measured_peak"] = entry["gbs"] / peak
+            del keep, sets
+            c.close()
         res[name] = entry
     return res
 
