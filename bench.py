@@ -405,7 +405,28 @@ def run_ours(args) -> None:
     if not args.no_extra:
         extra = extra_measurements(ctx, lt, torch, timed, step, sets, nbytes)
         extra["host_ns_per_barrier"] = {k: st[k] / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
-        extra["cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "barriers": st["barriers"]}
+        extra["cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "barriers": st["barriers"],
+                          "traces_matched": st["traces_matched"]}
+        # the timed steps repeat one another, so their traces are only matched against the previous one (no canonical
+        # form, no hash); the same 200 steps with that switched off show what a barrier costs when the graph is built,
+        # canonicalised, hashed and looked up every time
+        plain = lt.LazyContext(device=ctx.device)
+        plain.set_option("trace_match", 0)
+        psets = [tuple(plain.from_device_ptr(ctx.device_ptr(t), t.dtype, t.shape) for t in sets[k]) for k in range(len(sets))]
+        keep = [None] * len(psets)
+        for i in range(len(psets) + 2):
+            keep[i % len(psets)] = traces.mlp_epilogue(plain, *psets[i % len(psets)], primitive_gelu=False)
+            plain.barrier()
+        plain.reset_stats()
+        for i in range(200):
+            keep[i % len(psets)] = traces.mlp_epilogue(plain, *psets[i % len(psets)], primitive_gelu=False)
+            plain.barrier()
+        torch.cuda.synchronize()
+        pst = plain.stats()
+        extra["host_ns_per_barrier_graph_built_every_step"] = {k: pst[k] / max(pst["barriers"], 1) for k in pst if k.startswith("ns_")}
+        extra["cache_graph_built_every_step"] = {"compiles": pst["compiles"], "hits": pst["cache_hits"], "barriers": pst["barriers"]}
+        del keep, psets
+        plain.close()
         extra["c5_data_parallel_adam_step"] = dp_adam
         # the same program on the other two tiers, beside the headline: the interpreter serves a program that is not in
         # the build-time table until the run-time specialiser has built its kernel
