@@ -705,7 +705,17 @@ def adam_steps(lt, torch, device: int) -> dict:
     nbytes = configs.algorithmic_bytes("c5")
     dev = torch.device("cuda", device)
     res = {}
-    for mode in ("traced", "replayed", "replayed_interpreted", "replayed_specialised"):
+    # the update of one parameter as one batched recording call (lt_op_many) instead of sixteen calls
+    class _Refs:
+        pass
+
+    batch, refs = lt.Batch(), _Refs()
+    b_in = [batch.input() for _ in range(4)]
+    scalar_names = ("beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "sqrt_bc2", "eps", "step_size")
+    for name in scalar_names:
+        setattr(refs, name, batch.input())
+    traces.adam_update(batch, *b_in, refs)
+    for mode in ("traced", "traced_batched", "replayed", "replayed_interpreted", "replayed_specialised"):
         ctx = lt.LazyContext(device=device)
         if mode == "replayed_interpreted":
             ctx.set_option("compiled", 0)
@@ -718,6 +728,13 @@ def adam_steps(lt, torch, device: int) -> dict:
         if mode == "traced":
             for step in range(1, 101):
                 traces.adam_step(ctx, P, G, M, V, step=step)
+                ctx.barrier()
+        elif mode == "traced_batched":
+            for step in range(1, 101):
+                s = traces.AdamScalars(ctx, step=step)
+                sc = [getattr(s, name) for name in scalar_names]
+                for p, g, m, v in zip(P, G, M, V):
+                    ctx.record(batch, [p, g, m, v, *sc])
                 ctx.barrier()
         else:
             s = traces.AdamScalars(ctx, step=1)
@@ -738,6 +755,8 @@ def adam_steps(lt, torch, device: int) -> dict:
         res[f"c5_adam_100_steps_{mode}_gbs"] = nbytes * 100 / sec / 1e9
         res[f"c5_adam_{mode}_cache"] = {"compiles": st["compiles"], "hits": st["cache_hits"], "replays": st["replays"],
                                          "kernels": st["kernels_launched"], "traces_matched": st["traces_matched"]}
+        if mode == "traced_batched":
+            res["c5_host_us_per_barrier_batched"] = {k: st[k] / 1e3 / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
         if mode == "traced":
             res["c5_host_us_per_barrier"] = {k: st[k] / 1e3 / max(st["barriers"], 1) for k in st if k.startswith("ns_")}
         del P, G, M, V

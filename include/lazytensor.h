@@ -291,6 +291,31 @@ lt_status lt_release(lt_ctx *ctx, lt_tensor t);
 lt_status lt_release_many(lt_ctx *ctx, const lt_tensor *handles, size_t n);
 
 /*
+ * Several recording calls in one (Section 7 of the paper: the per-operation cost of tracing from a front end whose
+ * own calls are expensive).  Entry k of `ops` is what one lt_op or lt_assign call would be; its operands are named by
+ * index: in[i] >= 0 is inputs[in[i]], in[i] < 0 is the result of entry -(in[i] + 1) of the same batch.
+ *   opcode >= 0          lt_op(opcode, operands, attrs + attr_offset, n_attrs); with `keep` non-zero the result's
+ *                        handle is written to results[k] and belongs to the caller, otherwise the result is a temporary
+ *                        of the batch, released when the batch has been recorded (results[k] = 0)
+ *   LT_BATCH_ASSIGN      lt_assign(in[0], in[1]); no result
+ * Exactly equivalent to making the calls one by one in order and then releasing the temporaries in order (the graph,
+ * its hash and what trace matching sees are the same).  On an error the entries recorded so far are undone as far as
+ * their results go (released) and the status of the failing call is returned; assignments already made stay.
+ * `results` has n_ops entries.  Arrays are the caller's and only read during the call.
+ */
+#define LT_BATCH_ASSIGN (-1)
+typedef struct {
+    int32_t opcode;
+    int32_t n_in;
+    int32_t in[3];
+    int32_t n_attrs;
+    int32_t attr_offset;
+    int32_t keep;
+} lt_batch_op;
+lt_status lt_op_many(lt_ctx *ctx, const lt_batch_op *ops, size_t n_ops, const lt_tensor *inputs, size_t n_inputs,
+                     const int64_t *attrs, lt_tensor *results);
+
+/*
  * Barrier (Section 4; mark_step / LazyTensorBarrier): materialise every live tensor that
  * has pending computation.  With `blocking` non-zero, return after the stream has drained.
  * Row reductions over more than 8192 columns: a group whose program has a kernel instantiated at build time

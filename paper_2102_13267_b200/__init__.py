@@ -51,6 +51,14 @@ class lt_allocator(ctypes.Structure):
     _fields_ = [("alloc", ALLOC_FN), ("free", FREE_FN), ("user", ctypes.c_void_p)]
 
 
+class lt_batch_op(ctypes.Structure):
+    _fields_ = [("opcode", ctypes.c_int32), ("n_in", ctypes.c_int32), ("in_", ctypes.c_int32 * 3), ("n_attrs", ctypes.c_int32),
+                ("attr_offset", ctypes.c_int32), ("keep", ctypes.c_int32)]
+
+
+LT_BATCH_ASSIGN = -1
+
+
 class lt_stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in (
         "nodes_recorded", "barriers", "compiles", "cache_hits", "kernels_launched",
@@ -82,6 +90,7 @@ _SIGNATURES = {
     "lt_view_permute": [_vp, _u64, _P(_int), _P(_u64)],
     "lt_release": [_vp, _u64],
     "lt_release_many": [_vp, _P(_u64), ctypes.c_size_t],
+    "lt_op_many": [_vp, _P(lt_batch_op), ctypes.c_size_t, _P(_u64), ctypes.c_size_t, _P(_i64), _P(_u64)],
     "lt_barrier": [_vp, _int],
     "lt_barrier_static_scratch": [_vp, _int, _int],
     "lt_debug_bounds_violations": [_vp, _P(_u64)],
@@ -210,6 +219,87 @@ class LazyTensor:
         return self.ctx.fetch(self)
 
 
+class _BatchRef:
+    """An operand inside a Batch: one of its inputs (index >= 0) or the result of one of its entries (< 0)."""
+    __slots__ = ("batch", "index")
+
+    def __init__(self, batch, index):
+        self.batch, self.index = batch, index
+
+
+class Batch:
+    """A sequence of operations written once and recorded with one call per use (lt_op_many): what a front end's
+    operator expands to, e.g. the thirteen operations and three in-place updates of one Adam parameter update.  It has
+    the recording interface of a context (`op`, `assign`), so the same function that traces on a context builds it:
+
+        b = Batch(); p, g, lr = b.input(), b.input(), b.input()
+        b.assign(p, b.op("sub", p, b.op("mul", g, lr)))
+        ...
+        ctx.record(b, [p_tensor, g_tensor, lr_scalar])        # every step, for every parameter
+    """
+
+    def __init__(self):
+        self._ops, self._attrs, self._n_inputs, self._kept = [], [], 0, []
+        self._c = None
+
+    def input(self) -> _BatchRef:
+        self._n_inputs += 1
+        return _BatchRef(self, self._n_inputs - 1)
+
+    def op(self, name: str, *inputs, **attrs) -> _BatchRef:
+        a = _attr_list(name, attrs)
+        self._ops.append((OPCODES[name], [r.index for r in inputs], len(self._attrs), len(a), 0))
+        self._attrs.extend(a)
+        self._c = None
+        return _BatchRef(self, -len(self._ops))
+
+    def assign(self, dst: _BatchRef, src: _BatchRef) -> None:
+        self._ops.append((LT_BATCH_ASSIGN, [dst.index, src.index], 0, 0, 0))
+        self._c = None
+
+    def keep(self, ref: _BatchRef) -> None:
+        """The result `ref` is handed back by LazyContext.record (in the order of the keep calls)."""
+        k = -ref.index - 1
+        op = self._ops[k]
+        self._ops[k] = op[:4] + (1,)
+        self._kept.append(k)
+        self._c = None
+
+    def _compiled(self):
+        if self._c is None:
+            ops = (lt_batch_op * max(len(self._ops), 1))()
+            for k, (code, ins, off, na, keep) in enumerate(self._ops):
+                ops[k].opcode, ops[k].n_in, ops[k].n_attrs, ops[k].attr_offset, ops[k].keep = code, len(ins), na, off, keep
+                for i, r in enumerate(ins):
+                    ops[k].in_[i] = r
+            attrs = (_i64 * max(len(self._attrs), 1))(*self._attrs)
+            self._c = (ops, attrs, (_u64 * max(len(self._ops), 1))(), (_u64 * max(self._n_inputs, 1))())
+        return self._c
+
+
+def _attr_list(name: str, attrs: dict) -> list:
+    if not attrs:
+        return []
+    if name == "convert":
+        return [DTYPES[attrs["dtype"]]]
+    if name == "reshape":
+        shp = tuple(attrs["shape"])
+        return [len(shp), *shp]
+    if name == "narrow":
+        return [int(attrs["dim"]), int(attrs["start"]), int(attrs["length"])]
+    if name == "permute":
+        return [int(p) for p in attrs["perm"]]
+    if name == "update_slice":
+        return [int(attrs["dim"]), int(attrs["start"])]
+    if name == "iota":
+        shp = tuple(attrs["shape"])
+        return [int(attrs["dim"]), len(shp), *shp]
+    shp = tuple(attrs["shape"])  # philox_bits
+    seed, off = int(attrs["seed"]), int(attrs["offset"])
+    # 64-bit patterns travel as signed int64
+    return [seed - (1 << 64) if seed >= (1 << 63) else seed, off - (1 << 64) if off >= (1 << 63) else off, len(shp), *shp]
+
+
 class LazyContext:
     """One per device: the liveness arena, IR recorder, compile cache and executor."""
 
@@ -314,26 +404,7 @@ class LazyContext:
         at = self._attrs
         na = 0
         if attrs:
-            if name == "convert":
-                a = [DTYPES[attrs["dtype"]]]
-            elif name == "reshape":
-                shp = tuple(attrs["shape"])
-                a = [len(shp), *shp]
-            elif name == "narrow":
-                a = [int(attrs["dim"]), int(attrs["start"]), int(attrs["length"])]
-            elif name == "permute":
-                a = [int(p) for p in attrs["perm"]]
-            elif name == "update_slice":
-                a = [int(attrs["dim"]), int(attrs["start"])]
-            elif name == "iota":
-                shp = tuple(attrs["shape"])
-                a = [int(attrs["dim"]), len(shp), *shp]
-            else:  # philox_bits
-                shp = tuple(attrs["shape"])
-                seed, off = int(attrs["seed"]), int(attrs["offset"])
-                # 64-bit patterns travel as signed int64
-                a = [seed - (1 << 64) if seed >= (1 << 63) else seed, off - (1 << 64) if off >= (1 << 63) else off,
-                     len(shp), *shp]
+            a = _attr_list(name, attrs)
             na = len(a)
             for i in range(na):
                 at[i] = a[i]
@@ -368,6 +439,20 @@ class LazyContext:
 
     def assign(self, dst: LazyTensor, src: LazyTensor) -> None:
         self._check(_lib.lt_assign(self._ctx, dst.handle, src.handle))
+
+    def record(self, batch: Batch, inputs) -> list:
+        """lt_op_many: records the operations of `batch` on `inputs` in one call; returns the results it keeps."""
+        ops, attrs, results, ins = batch._compiled()
+        n = 0
+        for t in inputs:
+            ins[n] = t.handle
+            n += 1
+        if n != batch._n_inputs:
+            raise ValueError(f"the batch takes {batch._n_inputs} inputs, {n} given")
+        st = _lib.lt_op_many(self._ctx, ops, len(batch._ops), ins, n, attrs, results)
+        if st:
+            self._check(st)
+        return [LazyTensor(self, results[k]) for k in batch._kept]
 
     def release(self, t: LazyTensor) -> None:
         t.ctx = None

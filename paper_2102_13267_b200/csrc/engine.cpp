@@ -1882,6 +1882,38 @@ lt_status lt_release_many(lt_ctx *c, const lt_tensor *handles, size_t n) {
     return LT_OK;
 }
 
+lt_status lt_op_many(lt_ctx *c, const lt_batch_op *ops, size_t n_ops, const lt_tensor *inputs, size_t n_inputs, const int64_t *attrs,
+                     lt_tensor *results) {
+    if (!c || (n_ops && (!ops || !results)) || (n_inputs && !inputs)) return LT_ERR_INVALID_ARG;
+    for (size_t k = 0; k < n_ops; ++k) results[k] = 0;
+    lt_status st = LT_OK;
+    size_t done = 0;
+    for (; done < n_ops && st == LT_OK; ++done) {
+        const lt_batch_op &o = ops[done];
+        const int want = o.opcode == LT_BATCH_ASSIGN ? 2 : o.n_in;
+        lt_tensor in[3] = {0, 0, 0};
+        if (want < 0 || want > 3 || o.n_attrs < 0 || (o.n_attrs > 0 && !attrs)) st = fail(c, LT_ERR_INVALID_ARG, "lt_op_many: bad operand or attribute count");
+        for (int i = 0; i < want && st == LT_OK; ++i) {
+            const int64_t r = o.in[i];
+            if (r >= 0 && (size_t)r < n_inputs) in[i] = inputs[r];
+            else if (r < 0 && (size_t)(-(r + 1)) < done && results[-(r + 1)]) in[i] = results[-(r + 1)];
+            else st = fail(c, LT_ERR_INVALID_ARG, "lt_op_many: an operand names neither an input nor an earlier result of the batch");
+        }
+        if (st != LT_OK) break;
+        if (o.opcode == LT_BATCH_ASSIGN) st = lt_assign(c, in[0], in[1]);
+        else st = lt_op(c, o.opcode, in, o.n_in, o.n_attrs ? attrs + o.attr_offset : nullptr, o.n_attrs, &results[done]);
+        if (st != LT_OK) break;
+    }
+    // the temporaries go, in order; after an error so does everything the batch made
+    for (size_t k = 0; k < n_ops; ++k) {
+        if (!results[k] || (st == LT_OK && ops[k].keep)) continue;
+        const lt_status r = lt_release(c, results[k]);
+        results[k] = 0;
+        if (st == LT_OK && r != LT_OK) st = r;
+    }
+    return st;
+}
+
 lt_status lt_barrier(lt_ctx *c, int blocking) {
     if (!c) return LT_ERR_INVALID_ARG;
     DeviceScope on_device(c->device);

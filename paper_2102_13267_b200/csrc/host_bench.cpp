@@ -151,6 +151,40 @@ std::vector<int64_t> resnet50_numels() {
     return n;
 }
 
+// the same update as one lt_op_many call per parameter
+void adam_batched(int steps) {
+    Adam A;
+    for (int64_t ne : resnet50_numels()) {
+        A.p.push_back(leaf(LT_F32, {ne}));
+        A.g.push_back(leaf(LT_F32, {ne}));
+        A.m.push_back(leaf(LT_F32, {ne}));
+        A.v.push_back(leaf(LT_F32, {ne}));
+    }
+    // inputs: 0 p, 1 g, 2 m, 3 v, 4 beta1, 5 1-beta1, 6 beta2, 7 1-beta2, 8 sqrt_bc2, 9 eps, 10 step_size; results by entry: -(k+1)
+    const lt_batch_op ops[16] = {
+        {LT_OP_MUL, 2, {2, 4, 0}, 0, 0, 0},   {LT_OP_MUL, 2, {1, 5, 0}, 0, 0, 0},   {LT_OP_ADD, 2, {-1, -2, 0}, 0, 0, 0},  // m_new = entry 2
+        {LT_OP_MUL, 2, {1, 1, 0}, 0, 0, 0},   {LT_OP_MUL, 2, {3, 6, 0}, 0, 0, 0},   {LT_OP_MUL, 2, {-4, 7, 0}, 0, 0, 0},
+        {LT_OP_ADD, 2, {-5, -6, 0}, 0, 0, 0},                                                                              // v_new = entry 6
+        {LT_OP_SQRT, 1, {-7, 0, 0}, 0, 0, 0}, {LT_OP_DIV, 2, {-8, 8, 0}, 0, 0, 0},  {LT_OP_ADD, 2, {-9, 9, 0}, 0, 0, 0},   // den = entry 9
+        {LT_OP_DIV, 2, {-3, -10, 0}, 0, 0, 0}, {LT_OP_MUL, 2, {-11, 10, 0}, 0, 0, 0}, {LT_OP_SUB, 2, {0, -12, 0}, 0, 0, 0}, // p_new = entry 12
+        {LT_BATCH_ASSIGN, 2, {2, -3, 0}, 0, 0, 0}, {LT_BATCH_ASSIGN, 2, {3, -7, 0}, 0, 0, 0}, {LT_BATCH_ASSIGN, 2, {0, -13, 0}, 0, 0, 0}};
+    lt_reset_stats(ctx);
+    const double t0 = now();
+    for (int step = 1; step <= steps; ++step) {
+        A.scalars(step);
+        for (size_t i = 0; i < A.p.size(); ++i) {
+            const lt_tensor in[11] = {A.p[i], A.g[i], A.m[i], A.v[i], A.beta1, A.omb1, A.beta2, A.omb2, A.sqrt_bc2, A.eps, A.step_size};
+            lt_tensor res[16];
+            check(lt_op_many(ctx, ops, 16, in, 11, nullptr, res), "lt_op_many");
+        }
+        A.release_scalars();
+        check(lt_barrier(ctx, 0), "lt_barrier");
+    }
+    char name[64];
+    snprintf(name, sizeof(name), "C5 Adam, %zu tensors, batched", A.p.size());
+    report(name, steps, now() - t0);
+}
+
 void adam(int steps, bool replay) {
     Adam A;
     for (int64_t ne : resnet50_numels()) {
@@ -190,6 +224,7 @@ int main() {
     elementwise_chain(20000);
     mlp_epilogue(20000);
     adam(1000, false);
+    adam_batched(1000);
     adam(1000, true);
     lt_ctx_destroy(ctx);
     return 0;

@@ -107,3 +107,34 @@ def test_matching_off_gives_the_same_bits(lt):
         assert (c.stats()["traces_matched"] > 0) == bool(on)
         c.close()
     np.testing.assert_array_equal(results[0], results[1])
+
+
+def test_adam_recorded_in_batches_matches_the_oracle(lt):
+    """One lt_op_many call per parameter and step (the update's thirteen operations and three in-place assignments)."""
+    from workloads import configs
+
+    class Names:
+        pass
+
+    batch, refs = lt.Batch(), Names()
+    b_in = [batch.input() for _ in range(4)]
+    names = ("beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "sqrt_bc2", "eps", "step_size")
+    for n in names:
+        setattr(refs, n, batch.input())
+    traces.adam_update(batch, *b_in, refs)
+    shapes = [(64, 3, 7, 7), (64,), (256, 64, 1, 1), (1000, 96), (1000,)]
+    p, g, m, v = configs.c5_inputs(350, shapes)
+    c, O = lt.LazyContext(device=0), EagerOracle()
+    gp, gg, gm, gv = ([c.leaf(a, "f32") for a in arrs] for arrs in (p, g, m, v))
+    op, og, om, ov = ([O.leaf(a, "f32") for a in arrs] for arrs in (p, g, m, v))
+    for step in range(1, 13):
+        traces.adam_step(O, op, og, om, ov, step=step)
+        s = traces.AdamScalars(c, step=step)
+        for t in zip(gp, gg, gm, gv):
+            c.record(batch, [*t, *(getattr(s, n) for n in names)])
+        c.barrier()
+    for got, ref in zip(gp + gm + gv, op + om + ov):
+        assert_matches(c.fetch(got), ref.array, "f32", "Adam recorded in batches")
+    st = c.stats()
+    assert st["compiles"] == 1 and st["cache_hits"] == 11 and st["launches_multi"] == 12 and st["traces_matched"] >= 9, st
+    c.close()

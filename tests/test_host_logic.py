@@ -450,10 +450,11 @@ def test_host_bench_driver_runs_without_python_in_the_loop():
     spec.loader.exec_module(b)
     out = subprocess.run([str(b.build_host_bench())], capture_output=True, text=True, timeout=120, check=True).stdout
     lines = out.strip().splitlines()
-    assert len(lines) == 4
+    assert len(lines) == 5
     assert "compiles 1, hits 19999" in lines[0] and "compiles 1, hits 19999" in lines[1]
     assert "compiles 1, hits 999 (998 by matched trace, 0 traces diverged)" in lines[2]
-    assert "replays 999" in lines[3]
+    assert "batched" in lines[3] and "compiles 0, hits 1000 (998 by matched trace, 0 traces diverged)" in lines[3]  # lt_op_many: the same graph, found in the cache
+    assert "replays 999" in lines[4]
 
 
 # ------------------------------------------------------------------ long rows and the other reduction shapes

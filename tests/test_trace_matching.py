@@ -341,3 +341,87 @@ def test_errors_inside_a_matched_trace_are_the_usual_errors():
         other.close()
     assert out[on] == out[off]
     assert on.stats()["traces_matched"] >= 1
+
+
+# ------------------------------------------------------------------ several recording calls in one (lt_op_many)
+class _Names:
+    pass
+
+
+def _adam_batch():
+    from workloads import traces
+
+    b = lt.Batch()
+    p, g, m, v = (b.input() for _ in range(4))
+    s = _Names()
+    for name in ("beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "sqrt_bc2", "eps", "step_size"):
+        setattr(s, name, b.input())
+    traces.adam_update(b, p, g, m, v, s)  # the same function that traces on a context builds the batch
+    return b
+
+
+def test_batched_recording_is_the_calls_one_by_one():
+    from workloads import traces
+
+    batch = _adam_batch()
+    seen = {}
+    for mode in ("calls", "batch"):
+        ctx = lt.LazyContext(device=None)
+        P, G, M, V = ([fake(ctx, (96,)) for _ in range(4)] for _ in range(4))
+        log = []
+        for step in range(1, 6):
+            s = traces.AdamScalars(ctx, step=step)
+            for p, g, m, v in zip(P, G, M, V):
+                if mode == "calls":
+                    traces.adam_update(ctx, p, g, m, v, s)
+                else:
+                    kept = ctx.record(batch, [p, g, m, v, s.beta1, s.one_minus_beta1, s.beta2, s.one_minus_beta2, s.sqrt_bc2, s.eps, s.step_size])
+                    assert kept == []
+            if step == 1:
+                log.append(ctx.dump_ir())
+            before = ctx.stats()
+            ctx.barrier()
+            log.append((delta(ctx, before), ctx.dump_plan()))
+        st = ctx.stats()
+        log.append((st["compiles"], st["cache_hits"], st["traces_matched"], st["traces_diverged"]))
+        seen[mode] = log
+        ctx.close()
+    assert seen["calls"] == seen["batch"]
+    assert seen["batch"][-1] == (1, 4, 3, 0)
+
+
+def test_batch_results_errors_and_bad_references():
+    ctx = lt.LazyContext(device=None)
+    x, y, mask = fake(ctx, (8, 16)), fake(ctx, (8, 16)), fake(ctx, (8, 16), "u8")
+    b = lt.Batch()
+    a, c_ = b.input(), b.input()
+    t = b.op("mul", b.op("add", a, c_), a)
+    u = b.op("convert", t, dtype="bf16")
+    b.keep(t)
+    b.keep(u)
+    kept = ctx.record(b, [x, y])
+    assert [k.shape for k in kept] == [(8, 16), (8, 16)] and kept[1].dtype == "bf16"
+    text = ctx.dump_ir()
+    assert text.count("lt::add(") == 1 and text.count("ROOT=") == 2  # the add is a temporary of the batch: no handle, not a root
+    ctx.barrier()
+    assert ctx.stats()["kernels_launched"] == 1
+    # an entry that fails: nothing of the batch is left behind, the error is the failing call's
+    bad = lt.Batch()
+    p, q = bad.input(), bad.input()
+    bad.keep(bad.op("exp", p))
+    bad.op("add", p, q)  # f32 + u8
+    before = ctx.stats()["nodes_recorded"]
+    with pytest.raises(lt.LazyTensorError) as err:
+        ctx.record(bad, [x, mask])
+    assert "dtype" in str(err.value)
+    assert ctx.dump_ir().count("lt::") == 0 and ctx.stats()["nodes_recorded"] == before + 1
+    with pytest.raises(ValueError):
+        ctx.record(b, [x])
+    # operands must name an input or an earlier entry
+    import ctypes
+
+    ops = (lt.lt_batch_op * 1)()
+    ops[0].opcode, ops[0].n_in, ops[0].in_[0], ops[0].keep = lt.OPCODES["exp"], 1, -1, 1
+    res, ins = (ctypes.c_uint64 * 1)(), (ctypes.c_uint64 * 1)(x.handle)
+    assert lt._lib.lt_op_many(ctx._ctx, ops, 1, ins, 1, None, res) != 0 and res[0] == 0
+    ctx.close()
