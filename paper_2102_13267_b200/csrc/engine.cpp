@@ -553,7 +553,7 @@ void trace_log_result(lt_ctx *c, uint32_t slot) {
 
 void trace_log_op(lt_ctx *c, int opcode, const uint32_t *in_slots, int n_in, const int64_t *attrs, int n_attrs, uint32_t out_slot) {
     TraceState &T = c->trace;
-    if (n_attrs > 64 || T.log.events.size() >= (1u << 24)) {
+    if (n_attrs > 64 || T.log.events.size() >= (1u << 18)) {  // (a longer trace is not worth a log of tens of megabytes)
         T.log_valid = false;
         return;
     }

@@ -425,6 +425,23 @@ struct DeviceScope {
     DeviceScope &operator=(const DeviceScope &) = delete;
 };
 
+// Chunks of eight elements per thread in the row shell (lt_c_row) for rows of `cpr` chunks: one warp per row where the
+// row fits 32 x 8 chunks, else as few threads per row as eight chunks each allow -- except, measured on rows of 2048 to
+// 4096 columns: a row that would take two warps at eight chunks per thread runs on four warps at four when its inputs
+// are 4-byte elements or the program reads column vectors (LayerNorm f32 at 4096 columns 218 against 255 us), and a
+// program with column vectors over 2-byte inputs keeps to four chunks per thread even where eight would fit one warp
+// (the vectors then stay in registers: LayerNorm bf16 at 2048 columns 103 against 120 us, at 4096 105 against 151).
+inline int row_chunks_per_thread(uint32_t cpr, bool has_vectors, bool four_byte_inputs) {
+    int u = 1;
+    while (u < 8 && cpr > 32u * (unsigned)u) u *= 2;
+    if (u == 8 && cpr <= 512u) {
+        if (cpr > 256u && (has_vectors || four_byte_inputs)) u = 4;
+        else if (has_vectors && !four_byte_inputs) u = 4;
+    }
+    while (u < 8 && cpr > 128u * (unsigned)u) u *= 2;  // a row's group is at most one CTA of 128 threads
+    return u;
+}
+
 // Long rows of up to 8 x 128 x 8 chunks run with a thread-block cluster as the row's thread group (lt_c_rowc): the
 // cluster size and the chunks per thread for rows of `cpr` chunks; false when the row is too long.  As many chunks
 // per thread as the row needs in the smallest cluster -- eight, or four when the program reads column vectors, which

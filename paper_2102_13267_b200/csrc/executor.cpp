@@ -585,8 +585,11 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     done = true;
                 } else if (ok && P.cpr <= 8u * 128u) {  // a row's group of threads is at most one CTA of 128
                     // a row lives in the registers of its thread group: up to 8 chunks per thread, one warp per row if it fits
-                    int u = 1;
-                    while (u < 8 && P.cpr > 32u * u) u *= 2;
+                    bool four_byte = false;
+                    for (size_t q = 0; q < g.io.size(); ++q)
+                        if (!g.io[q].is_store && g.io[q].cls == LT_CLS_FULL && dtype_size(g.io[q].dtype) == 4) four_byte = true;
+                    const bool integer_heavy = specialised(L) ? jit_integer_heavy(*L.jit_program) : lt_compiled_prefers_staging(L.compiled) == 0;
+                    int u = row_chunks_per_thread(P.cpr, g.n_pro > 0 && !integer_heavy, four_byte);
                     if (c->opt.compiled_row_u > 0 && !specialised(L)) u = (int)c->opt.compiled_row_u;
                     while (u < 8 && P.cpr > 128u * u) u *= 2;  // a row's group is at most one CTA of 128 threads
                     unsigned grp = 1, lg = 0;
@@ -594,7 +597,9 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     const unsigned threads = grp > 128 ? grp : 128;
                     // pipeline depth: stages of the next blocks' inputs in shared memory, within ~72 KB per CTA
                     const size_t stage = specialised(L) ? jit_row_stage_bytes(*L.jit_program, u, 128) : lt_compiled_row_stage_bytes(L.compiled, u);
-                    const bool wants_ring = specialised(L) ? !jit_integer_heavy(*L.jit_program) : lt_compiled_prefers_staging(L.compiled) != 0;
+                    // (not for programs bound by integer issue, nor for 4-byte inputs, which measured faster loaded directly:
+                    // softmax f32 at 2048 columns 169 against 248 us)
+                    const bool wants_ring = !integer_heavy && !four_byte;
                     unsigned depth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth : (wants_ring ? 2u : 0u);
                     while (depth > 0 && depth * stage > 72u * 1024u) --depth;
                     if (stage == 0 || threads != 128 || depth < 2) depth = 0;

@@ -1347,9 +1347,10 @@ lt_status build_plan(lt_ctx *c, const Canonical &cg, Plan &plan, bool isolate_lo
             jp->long_row = g.long_row;
             if (L.kind == K_ROW && !g.long_row) {
                 const uint32_t cpr = (uint32_t)((g.cols + LT_VM_V - 1) / LT_VM_V);
-                int u = 1;
-                while (u < 8 && cpr > 32u * u) u *= 2;  // (the executor's choice: one warp per row where it fits)
-                jp->row_u = u;
+                bool four_byte = false;
+                for (const IoRef &io : g.io)
+                    if (!io.is_store && io.cls == LT_CLS_FULL && dtype_size(io.dtype) == 4) four_byte = true;
+                jp->row_u = row_chunks_per_thread(cpr, g.n_pro > 0 && !jit_integer_heavy(*jp), four_byte);  // (the executor's choice)
             }
             if (L.kind == K_ROW && g.long_row) {
                 unsigned k = 0;

@@ -30,6 +30,7 @@ def main() -> None:
     ap.add_argument("configs", nargs="?", default="c1,c2,c2p,c3,c4,c5")
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate through (0 = enough for 1 GB)")
+    ap.add_argument("--long-shapes", default="8192x16384,2048x65536", help="rows x columns of the `long` case")
     ap.add_argument("--only", default="", help="of the idioms / long / reduce cases, run those whose name contains this")
     ap.add_argument("options", nargs="*")
     args = ap.parse_args()
@@ -194,7 +195,7 @@ def main() -> None:
         ctx.close()
 
     if "long" in which:
-        for rows, cols in ((8192, 16384), (2048, 65536)):
+        for rows, cols in (tuple(int(v) for v in sh.split("x")) for sh in args.long_shapes.split(",")):
             for iname in ("softmax_bf16", "layernorm_bf16", "softmax_f32", "layernorm_f32"):
                 _, kinds, trace = next(e for e in idioms.ALL if e[0] == iname)
                 es = 4 if iname.endswith("f32") else 2
