@@ -589,6 +589,36 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     for (size_t q = 0; q < g.io.size(); ++q)
                         if (!g.io[q].is_store && g.io[q].cls == LT_CLS_FULL && dtype_size(g.io[q].dtype) == 4) four_byte = true;
                     const bool integer_heavy = specialised(L) ? jit_integer_heavy(*L.jit_program) : lt_compiled_prefers_staging(L.compiled) == 0;
+                    // Rows of 4097 to 8192 columns of a program with column vectors would need eight chunks per thread here
+                    // (the vectors re-read for every row, two CTAs per SM): two CTAs of a cluster with four chunks per thread
+                    // hold such a row instead (lt_c_rowc, as for rows beyond 8192 columns).
+                    if (!specialised(L) && c->opt.cluster != 1 && g.n_pro > 0 && !integer_heavy && P.cpr > 512u) {
+                        unsigned k = 0;
+                        int cu = 0;
+                        if (cluster_shape(P.cpr, true, c->opt.cluster, 0, &k, &cu)) {
+                            const size_t cstage = lt_compiled_row_stage_bytes(L.compiled, cu);
+                            unsigned cdepth = c->opt.compiled_depth >= 0 ? (unsigned)c->opt.compiled_depth : (four_byte ? 0u : 2u);
+                            while (cdepth > 0 && cdepth * cstage > 72u * 1024u) --cdepth;
+                            if (cstage == 0) cdepth = 0;
+                            if (L.cluster_max < 0) {
+                                int n = 0;
+                                if (lt_compiled_cluster_occupancy(L.compiled, cu, 0, k, cdepth, &n) != cudaSuccess) {
+                                    cudaGetLastError();
+                                    n = 0;
+                                }
+                                L.cluster_max = n;
+                            }
+                            if (L.cluster_max >= 1) {
+                                const unsigned clusters = (unsigned)std::min<uint64_t>(P.rows, (uint64_t)L.cluster_max);
+                                if (ev0) cudaEventRecord(ev0, c->stream);
+                                e = lt_compiled_launch_cluster(L.compiled, &P, cu, 0, clusters, k, cdepth, (uint64_t)c->wait_limit_ns, c->stream);
+                                if (ev1) cudaEventRecord(ev1, c->stream);
+                                c->status_pending = true;
+                                done = true;
+                            }
+                        }
+                    }
+                    if (!done) {
                     int u = row_chunks_per_thread(P.cpr, g.n_pro > 0 && !integer_heavy, four_byte);
                     if (c->opt.compiled_row_u > 0 && !specialised(L)) u = (int)c->opt.compiled_row_u;
                     while (u < 8 && P.cpr > 128u * u) u *= 2;  // a row's group is at most one CTA of 128 threads
@@ -615,6 +645,7 @@ lt_status execute_plan(lt_ctx *c, Plan &plan, const Canonical &cg, bool *needs_s
                     e = fast_launch(c, L, &P, u, grid, threads, grp, lg, depth, depth * stage);
                     if (ev1) cudaEventRecord(ev1, c->stream);
                     done = true;
+                    }
                 }
                 if (done) c->stats.launches_compiled++;
             }

@@ -61,7 +61,9 @@ def test_listed_groups_on_long_rows_run_fused(ctx, idiom, shape):
 @pytest.mark.parametrize("vectors", [0, 1])
 @pytest.mark.parametrize("cluster", [1, 2, 4, 8])
 @pytest.mark.parametrize("idiom,shape", [("layernorm_bf16", (9, 16384)), ("layernorm_f32", (5, 10000)), ("softmax_bf16", (7, 8200)),
-                                         ("rmsnorm_bf16", (3, 32768)), ("layernorm_bf16", (3, 65536)), ("softmax_f32", (300, 12288))])
+                                         ("rmsnorm_bf16", (3, 32768)), ("layernorm_bf16", (3, 65536)), ("softmax_f32", (300, 12288)),
+                                         # 4097 to 8192 columns with column vectors: two CTAs of a cluster instead of eight chunks per thread
+                                         ("layernorm_bf16", (300, 8192)), ("layernorm_f32", (7, 6144)), ("rmsnorm_bf16", (5, 4104))])
 def test_long_rows_in_every_cluster_shape(lt, idiom, shape, cluster, vectors):
     if cluster * 128 * 8 * 8 < shape[-1] and cluster != 1:
         pytest.skip("row too long for this cluster size")
